@@ -1,0 +1,500 @@
+"""Pins for the CPU oracle: each check compares the oracle with something that is not the
+oracle -- a closed form, SciPy / NumPy routines, exact rational arithmetic, brute force on
+tiny inputs, hand-worked examples (tests/golden) and the bit-widths of the paper's
+bandwidth-phase run (Sec. 4.2)."""
+import math
+import os
+from fractions import Fraction
+
+import numpy as np
+import pytest
+import scipy.optimize
+import scipy.special
+import scipy.stats
+
+import oracle
+import synth_inputs as si
+
+ALL_BITS = [1, 2, 3, 4, 5, 6, 7, 8, 16]
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# ---------------------------------------------------------------- ACIQ F(q)
+
+@pytest.mark.parametrize("q", ALL_BITS)
+def test_F_laplace_is_lambert_w(q):
+    F = oracle.aciq_F(q, 0)
+    ref = float(np.real(scipy.special.lambertw(3.0 * 4.0 ** q)))
+    assert F == pytest.approx(ref, rel=1e-12)
+    assert F * math.exp(F) == pytest.approx(3.0 * 4.0 ** q, rel=1e-12)
+
+
+@pytest.mark.parametrize("q", [1, 2, 3, 4, 6, 8])
+def test_F_laplace_minimises_error_model(q):
+    # Laplace(0,1): clipping noise 2 exp(-a), rounding noise a^2 / (3 * 4^q)
+    model = lambda a: 2.0 * math.exp(-a) + a * a / (3.0 * 4.0 ** q)
+    r = scipy.optimize.minimize_scalar(model, bounds=(0.01, 60.0), method="bounded", options=dict(xatol=1e-10))
+    assert oracle.aciq_F(q, 0) == pytest.approx(r.x, rel=1e-5)
+
+
+@pytest.mark.parametrize("q", ALL_BITS)
+def test_F_gauss_minimises_error_model(q):
+    n = scipy.stats.norm
+    model = lambda a: 2.0 * ((1 + a * a) * n.sf(a) - a * n.pdf(a)) + a * a / (3.0 * 4.0 ** q)
+    r = scipy.optimize.minimize_scalar(model, bounds=(0.01, 12.0), method="bounded", options=dict(xatol=1e-11))
+    assert oracle.aciq_F(q, 1) == pytest.approx(r.x, rel=2e-5)
+
+
+def test_F_known_magnitudes():
+    # the Laplace clipping multipliers grow roughly linearly in q; 2-bit value near 2.83
+    assert oracle.aciq_F(2, 0) == pytest.approx(2.8307, abs=1e-4)
+    assert oracle.aciq_F(4, 0) == pytest.approx(5.0286, abs=1e-4)
+    assert oracle.aciq_F(2, 1) == pytest.approx(1.7106, abs=1e-4)
+    Fs = [oracle.aciq_F(q, 0) for q in range(1, 9)]
+    assert all(b > a for a, b in zip(Fs, Fs[1:]))
+
+
+def test_laplace_error_model_matches_data():
+    # On i.i.d. Laplace(0,1) data the measured MSE at the ACIQ clip follows the model the
+    # constants come from: 2 exp(-a) + a^2 / (3 (L-1)^2) for this grid (L-1 intervals).
+    x = si.flat_iid(1 << 22, 11, "laplace")
+    st = oracle.stats(x)
+    for q in (4, 6, 8):
+        rc, alpha, qp = oracle.aciq_alpha(st, q)
+        a = alpha / st.mad
+        model = st.mad ** 2 * (2.0 * math.exp(-a) + a * a / (3.0 * (2 ** q - 1) ** 2))
+        assert oracle.quant_mse(x, qp) == pytest.approx(model, rel=0.06)
+
+
+def test_aciq_alpha_linear_and_centred():
+    x = si.vit_activation((4, 197, 64), 5)
+    st = oracle.stats(x)
+    for q in (2, 4, 8, 16):
+        rc, alpha, qp = oracle.aciq_alpha(st, q)
+        assert rc == 0
+        assert alpha == pytest.approx(oracle.aciq_F(q) * st.mad, rel=1e-14)
+        assert qp.lo == np.float32(st.mean - alpha) and qp.hi == np.float32(st.mean + alpha)
+        st3 = oracle.stats(3.0 * x.astype(np.float64))
+        _, alpha3, _ = oracle.aciq_alpha(st3, q)
+        assert alpha3 == pytest.approx(3.0 * alpha, rel=1e-6)
+    _, a_lit, _ = oracle.aciq_alpha(st, 4, 0, 1)
+    assert a_lit == pytest.approx(oracle.aciq_F(4) * st.mean_abs, rel=1e-14)
+    _, a_g, _ = oracle.aciq_alpha(st, 4, 1, 0)
+    assert a_g == pytest.approx(oracle.aciq_F(4, 1) * math.sqrt(st.var), rel=1e-14)
+    _, a_o, _ = oracle.aciq_alpha(st, 4, 0, 0, 0.7)
+    assert a_o == pytest.approx(oracle.aciq_F(4) * 0.7, rel=1e-14)
+    assert oracle.aciq_alpha(st, 9)[0] == oracle.ERR_BITS
+
+
+# ------------------------------------------------------------------- stats
+
+def test_stats_against_numpy_and_fsum():
+    x = si.vit_activation((3, 197, 96), 7)
+    st = oracle.stats(x)
+    xd = x.astype(np.float64).reshape(-1)
+    mean = math.fsum(xd) / xd.size
+    assert st.n == xd.size and st.nonfinite == 0
+    assert st.mean == pytest.approx(mean, rel=1e-13, abs=1e-16)
+    assert st.mean_abs == pytest.approx(math.fsum(np.abs(xd)) / xd.size, rel=1e-13)
+    assert st.mad == pytest.approx(math.fsum(np.abs(xd - mean)) / xd.size, rel=1e-13)
+    assert st.var == pytest.approx(math.fsum((xd - mean) ** 2) / xd.size, rel=1e-13)
+    assert st.min == xd.min() and st.max == xd.max()
+    assert st.var == pytest.approx(np.var(xd), rel=1e-10)
+
+
+def test_stats_closed_form_and_nonfinite():
+    x = np.arange(1, 1002, dtype=np.float32)          # 1..1001: mean 501, mad 250500/1001*... closed forms
+    st = oracle.stats(x)
+    assert st.mean == 501.0 and st.min == 1.0 and st.max == 1001.0
+    assert st.mean_abs == 501.0
+    assert st.mad == pytest.approx(2 * sum(range(1, 501)) / 1001.0, rel=1e-15)
+    assert st.var == pytest.approx((1001 ** 2 - 1) / 12.0, rel=1e-15)
+    y = np.concatenate([x, np.array([np.nan, np.inf, -np.inf], dtype=np.float32)])
+    st2 = oracle.stats(y)
+    assert st2.n == 1004 and st2.nonfinite == 3
+    assert (st2.mean, st2.mad, st2.var, st2.min, st2.max) == (st.mean, st.mad, st.var, st.min, st.max)
+    st0 = oracle.stats(np.zeros(0, dtype=np.float32))
+    assert st0.n == 0 and st0.mean == 0.0 and st0.mad == 0.0
+    # cancellation: large offset, small spread
+    z = (np.float32(4096.0) + si.flat_iid(50000, 3, "normal")).astype(np.float32)
+    stz = oracle.stats(z)
+    zd = z.astype(np.float64)
+    assert stz.var == pytest.approx(np.var(zd), rel=1e-9)
+
+
+# --------------------------------------------------------------- quantizer
+
+def test_hand_examples(hand_examples):
+    assert len(hand_examples) == 5
+    for ex in hand_examples:
+        rc, qp = oracle.make_qparams(ex["lo"], ex["hi"], ex["bits"])
+        assert rc == 0
+        x = np.array(ex["x"], dtype=np.float32)
+        codes = oracle.quantize(x, qp)
+        assert codes.tolist() == ex["codes"], ex
+        packed = oracle.pack(codes, ex["bits"])
+        nb = len(ex["bytes"])
+        assert packed[:nb].tobytes() == ex["bytes"], ex
+        assert not packed[nb:].any()
+        assert packed.size % 16 == 0
+        assert oracle.unpack(packed, len(codes), ex["bits"]).tolist() == ex["codes"]
+
+
+@pytest.mark.parametrize("q", ALL_BITS)
+def test_make_qparams_definition(q):
+    lo, hi = -1.2345678901, 3.9876543212
+    rc, qp = oracle.make_qparams(lo, hi, q)
+    assert rc == 0 and qp.bits == q and qp.flags == 0
+    lo_f, hi_f = np.float32(lo), np.float32(hi)
+    rng = Fraction(float(hi_f)) - Fraction(float(lo_f))
+    L1 = 2 ** q - 1
+    # correctly rounded from the exact quotient (np.float32 of a fp64 value that is within
+    # 2^-53 relative of the exact one; ties at that level do not occur for these numbers)
+    assert qp.lo == lo_f and qp.hi == hi_f
+    assert qp.scale == np.float32(float(rng / L1))
+    assert qp.inv_scale == np.float32(float(L1 / rng))
+
+
+def test_make_qparams_degenerate_and_errors():
+    rc, qp = oracle.make_qparams(1.0, 1.0, 4)
+    assert rc == oracle.WARN_DEGENERATE and qp.flags == 1 and qp.scale == 0.0 and qp.inv_scale == 0.0
+    assert not oracle.quantize(np.array([-5, 1, 7, np.nan], dtype=np.float32), qp).any()
+    assert oracle.dequantize(np.array([0, 0], dtype=np.uint32), qp).tolist() == [1.0, 1.0]
+    assert oracle.make_qparams(2.0, 1.0, 4)[0] == oracle.WARN_DEGENERATE
+    assert oracle.make_qparams(0.0, 1.0, 0)[0] == oracle.ERR_BITS
+    assert oracle.make_qparams(0.0, 1.0, 12)[0] == oracle.ERR_BITS
+    assert oracle.make_qparams(float("nan"), 1.0, 4)[0] == oracle.ERR_ARG
+    assert oracle.make_qparams(0.0, float("inf"), 4)[0] == oracle.ERR_ARG
+
+
+@pytest.mark.parametrize("q", ALL_BITS)
+def test_quantizer_is_textbook_affine(q):
+    # naive PTQ: range = [min, max] (Sec. 3).  Compare with the affine quantizer written
+    # in fp64 NumPy; codes may differ only where the fp64 position is within 1e-4 of a tie.
+    x = si.vit_activation((2, 197, 48), 9).reshape(-1)
+    st = oracle.stats(x)
+    rc, qp = oracle.make_qparams(st.min, st.max, q)
+    codes = oracle.quantize(x, qp).astype(np.int64)
+    L1 = 2 ** q - 1
+    pos = (np.clip(x.astype(np.float64), qp.lo, qp.hi) - qp.lo) * (L1 / (float(qp.hi) - float(qp.lo)))
+    ref = np.rint(pos).astype(np.int64)
+    diff = codes != ref
+    assert np.all(np.abs(pos[diff] - np.floor(pos[diff]) - 0.5) < 1e-4 * max(1.0, L1 / 256))
+    assert diff.mean() < 1e-3 * max(1.0, L1 / 4096)
+    assert codes.min() == 0 and codes.max() == L1
+    # error bound of rounding to the nearest level
+    y = oracle.dequantize(codes.astype(np.uint32), qp).astype(np.float64)
+    assert np.max(np.abs(y - x)) <= 0.5 * float(qp.scale) * (1 + 1e-5) + 1e-6 * np.abs(x).max()
+
+
+def test_quantizer_special_values():
+    rc, qp = oracle.make_qparams(-1.0, 1.0, 4)
+    x = np.array([np.nan, np.inf, -np.inf, -1.0, 1.0, 0.0, -0.0, 1e30, -1e30], dtype=np.float32)
+    assert oracle.quantize(x, qp).tolist() == [0, 15, 0, 0, 15, 8, 8, 15, 0]  # 7.5 -> 8 (even)
+
+
+@pytest.mark.parametrize("q", ALL_BITS)
+def test_dequantize_exact_rational(q):
+    rc, qp = oracle.make_qparams(-0.7361, 2.4419, q)
+    codes = np.unique(np.concatenate([si.random_codes(300, q, 1), np.array([0, 2 ** q - 1], dtype=np.uint32)]))
+    y = oracle.dequantize(codes, qp)
+    lo, sc = Fraction(float(qp.lo)), Fraction(float(qp.scale))
+    for c, v in zip(codes.tolist(), y.tolist()):
+        exact = lo + c * sc
+        # the correctly rounded fp32 of the exact value: nearest of the two neighbours
+        f = np.float32(float(exact))
+        cands = [f, np.nextafter(f, np.float32(np.inf)), np.nextafter(f, np.float32(-np.inf))]
+        best = min(cands, key=lambda t: abs(Fraction(float(t)) - exact))
+        assert v == float(best)
+    # quantizing a reconstruction level gives its code back
+    assert np.array_equal(oracle.quantize(y, qp), codes)
+
+
+# ------------------------------------------------------------------ packing
+
+@pytest.mark.parametrize("q", ALL_BITS)
+@pytest.mark.parametrize("n", [0, 1, 7, 31, 32, 33, 127, 128, 129, 1000])
+def test_pack_is_little_endian_integer(q, n):
+    codes = si.random_codes(n, q, 100 + q)
+    packed = oracle.pack(codes, q)
+    assert packed.size == oracle.packed_bytes(n, q) == (((n * q + 7) // 8 + 15) // 16) * 16
+    big = 0
+    for i, c in enumerate(codes.tolist()):
+        big |= c << (i * q)
+    assert packed.tobytes() == big.to_bytes(packed.size, "little")     # pad bits are zero
+    # same layout through NumPy's bit packer
+    bits = ((codes[:, None] >> np.arange(q, dtype=np.uint32)[None, :]) & 1).astype(np.uint8).reshape(-1)
+    ref = np.packbits(bits, bitorder="little")
+    assert np.array_equal(packed[:ref.size], ref)
+    assert np.array_equal(oracle.unpack(packed, n, q), codes)
+
+
+def test_eight_bit_is_four_times_smaller():
+    # Sec. 3: 8-bit codes compress fp32 activations 4x
+    n = 64 * 197 * 768
+    assert oracle.packed_bytes(n, 8) * 4 == n * 4
+    assert oracle.packed_bytes(n, 2) * 16 == n * 4
+    assert oracle.packed_bytes(n, 16) == 2 * n
+    assert oracle.packed_bytes(5, 3) == 16 and oracle.packed_bytes(0, 3) == 0
+
+
+def test_quantize_pack_roundtrip_composition():
+    x = si.vit_activation((1, 50, 77), 2).reshape(-1)
+    st = oracle.stats(x)
+    for q in ALL_BITS:
+        _, _, qp = oracle.aciq_alpha(st, q)
+        p = oracle.quantize_pack(x, qp)
+        y = oracle.unpack_dequantize(p, x.size, qp)
+        assert np.array_equal(y, oracle.dequantize(oracle.quantize(x, qp), qp))
+        # idempotence: re-quantizing the reconstruction changes nothing
+        assert np.array_equal(oracle.quantize_pack(y, qp), p)
+
+
+# ---------------------------------------------------------------------- MSE
+
+def test_mse_matches_numpy_and_is_monotone_in_bits():
+    x = si.vit_activation((2, 197, 128), 4).reshape(-1)
+    st = oracle.stats(x)
+    prev = None
+    for q in range(1, 9):
+        _, _, qp = oracle.aciq_alpha(st, q)
+        y = oracle.dequantize(oracle.quantize(x, qp), qp).astype(np.float64)
+        ref = math.fsum((y - x.astype(np.float64)) ** 2) / x.size
+        m = oracle.quant_mse(x, qp)
+        assert m == pytest.approx(ref, rel=1e-12)
+        if prev is not None:
+            assert m <= prev
+        prev = m
+    xn = np.concatenate([x, np.array([np.nan, np.inf], dtype=np.float32)])
+    assert oracle.quant_mse(xn, qp) == pytest.approx(m, rel=1e-12)      # non-finite skipped
+
+
+def test_one_bit_grid_minimum_at_laplace_scale():
+    # With two levels mu +- a, Laplace(0,b) data has MSE(a) = 2b^2 - 2ab + a^2: minimum b^2 at a = b.
+    x = si.flat_iid(1 << 20, 21, "laplace")
+    st = oracle.stats(x)
+    b = st.mad
+    alphas = np.linspace(0.5 * b, 1.5 * b, 201)
+    mses = [oracle.quant_mse(x, oracle.make_qparams(st.mean - a, st.mean + a, 1)[1]) for a in alphas]
+    k = int(np.argmin(mses))
+    assert alphas[k] == pytest.approx(b, rel=0.01)
+    assert mses[k] == pytest.approx(st.var - b * b, rel=1e-3)            # E x^2 - 2ab + a^2 at a=b
+    for a, m in zip(alphas[::40], mses[::40]):
+        assert m == pytest.approx(st.var - 2 * a * b + a * a, rel=2e-3)
+
+
+def test_naive_range_is_worse_on_heavy_tails():
+    # Sec. 3: the min/max range is set by rare extreme values; clipping fixes it at low bit-widths.
+    x = si.vit_activation((8, 197, 256), 2).reshape(-1)
+    st = oracle.stats(x)
+    for q in (2, 4):
+        naive = oracle.quant_mse(x, oracle.make_qparams(st.min, st.max, q)[1])
+        aciq = oracle.quant_mse(x, oracle.aciq_alpha(st, q)[2])
+        assert naive > 3.0 * aciq
+
+
+# ---------------------------------------------------------------- histogram
+
+@pytest.mark.parametrize("nb", [1, 7, 100, 256, 2048])
+def test_histogram_counts(nb):
+    x = si.vit_activation((2, 197, 64), 6).reshape(-1)
+    x = np.concatenate([x, np.array([np.nan, np.inf], dtype=np.float32)])
+    st = oracle.stats(x)
+    peak, counts = oracle.hist_peak(x, st.min, st.max, nb)
+    fin = x[np.isfinite(x)]
+    assert counts.sum() == fin.size
+    ref, edges = np.histogram(fin.astype(np.float64), bins=nb, range=(st.min, st.max))
+    # fp32 bin positions may move elements that sit on an edge; nothing else differs
+    assert np.abs(counts.astype(np.int64) - ref).sum() <= max(2, fin.size // 2000)
+    w = (st.max - st.min) / nb
+    assert peak == pytest.approx(counts.max() / (fin.size * w), rel=1e-14)
+
+
+def test_histogram_exact_on_bin_centres_and_sorted_count():
+    nb = 16
+    centres = (np.arange(nb) + 0.5) / nb * 8.0                 # range [0, 8], exactly representable
+    reps = np.arange(1, nb + 1)
+    x = np.concatenate([np.repeat(centres, reps), [0.0, 8.0]]).astype(np.float32)
+    peak, counts = oracle.hist_peak(x, 0.0, 8.0, nb)
+    expect = reps.copy()
+    expect[0] += 1
+    expect[-1] += 1                                            # max lands in the last (closed) bin
+    assert counts.tolist() == expect.tolist()
+    assert peak == pytest.approx((nb + 1) / (x.size * 0.5), rel=1e-15)
+    assert oracle.hist_peak(x, 3.0, 3.0, nb)[0] == 0.0         # empty range
+
+
+def test_histogram_peak_of_laplace_density():
+    x = si.flat_iid(1 << 21, 8, "laplace")
+    st = oracle.stats(x)
+    peak, _ = oracle.hist_peak(x, st.min, st.max, 512)
+    assert peak == pytest.approx(0.5, rel=0.05)                # Laplace(0,1) density at 0 is 1/2
+
+
+# ----------------------------------------------------------- directed search
+
+def _numpy_candidate_mse(x, mean, alpha, q):
+    """Independent fp32 NumPy evaluation of one candidate (same single-precision steps)."""
+    lo, hi = np.float32(mean - alpha), np.float32(mean + alpha)
+    L1 = 2 ** q - 1
+    rng = float(hi) - float(lo)
+    scale, inv = np.float32(rng / L1), np.float32(L1 / rng)
+    t = np.minimum(np.maximum(x, lo), hi)
+    v = ((t - lo).astype(np.float32) * inv).astype(np.float32)
+    code = np.clip(np.rint(v), 0, L1)
+    dq = (np.float64(lo) + code.astype(np.float64) * np.float64(scale)).astype(np.float32)
+    return float(np.mean((dq.astype(np.float64) - x.astype(np.float64)) ** 2))
+
+
+@pytest.mark.parametrize("q,seed,nb", [(2, 1, 100), (4, 2, 100), (3, 3, 64), (8, 4, 100), (2, 5, 2048), (1, 6, 100)])
+def test_ds_search_equals_brute_force(q, seed, nb):
+    x = si.vit_activation((1, 16, 256), seed, outlier_frac=0.02 if seed % 2 else 0.0).reshape(-1)
+    st = oracle.stats(x)
+    rc, res, qp, curve = oracle.ds_search(x, st, q, 0, 100, nb)
+    assert rc == 0
+    fin = x.astype(np.float64)
+    counts, _ = np.histogram(fin, bins=nb, range=(st.min, st.max))
+    w = (st.max - st.min) / nb
+    peak_ref = counts.max() / (x.size * w)
+    assert res.b_e == st.mad
+    assert res.b_r == pytest.approx(1.0 / (2.0 * peak_ref), rel=0.02)   # edge elements may move one count
+    F = float(np.real(scipy.special.lambertw(3.0 * 4.0 ** q)))
+    mses = np.array([_numpy_candidate_mse(x, st.mean, F * (res.b_e + k * (res.b_r - res.b_e) / 100), q)
+                     for k in range(101)])
+    assert np.allclose(curve, mses, rtol=1e-9)
+    k_ref = int(np.argmin(mses))                       # first index of the minimum
+    assert res.k_star == k_ref or abs(mses[res.k_star] - mses[k_ref]) <= 1e-12 * mses[k_ref]
+    assert res.mse_star <= res.mse_e and res.mse_e == pytest.approx(mses[0], rel=1e-9)
+    assert res.b_star == pytest.approx(res.b_e + res.k_star * (res.b_r - res.b_e) / 100, rel=1e-15)
+    assert res.alpha_star == pytest.approx(F * res.b_star, rel=1e-12)
+    assert res.alpha_e == pytest.approx(F * res.b_e, rel=1e-12)
+    assert qp.lo == np.float32(st.mean - res.alpha_star) and qp.hi == np.float32(st.mean + res.alpha_star)
+    assert oracle.quant_mse(x, qp) == res.mse_star
+    # never worse than plain ACIQ, never better than a fine exhaustive scan of the same interval
+    lo_b, hi_b = min(res.b_e, res.b_r), max(res.b_e, res.b_r)
+    fine = min(_numpy_candidate_mse(x, st.mean, F * b, q) for b in np.linspace(lo_b, hi_b, 2001))
+    assert fine <= res.mse_star * (1 + 1e-9)
+    assert res.mse_star <= fine * 1.05 or res.k_star in (0, 100) or q == 1
+
+
+def test_ds_direction_follows_histogram_peak():
+    # flat-topped data: histogram peak lower than the Laplace fit's peak -> b_R > b_E
+    u = (si.uniform01(3, si.STREAM_VALUE, 0, 20000) * 2 - 1).astype(np.float32)
+    st = oracle.stats(u)
+    _, res, _, _ = oracle.ds_search(u, st, 2, 0, 100, 100)
+    assert res.b_r > res.b_e and res.b_e <= res.b_star <= res.b_r
+    assert 1.0 / (2 * res.b_e) > 0.5                              # max(D_E) = 1/(2 b_E) = 1 > max(D_R) ~ 0.5
+    # sharply peaked mixture: most mass in a narrow spike -> b_R < b_E
+    spike = np.concatenate([0.01 * si.flat_iid(18000, 4, "laplace"), 3.0 * si.flat_iid(2000, 5, "laplace")]).astype(np.float32)
+    st = oracle.stats(spike)
+    _, res, _, _ = oracle.ds_search(spike, st, 2, 0, 100, 2048)
+    assert res.b_r < res.b_e and res.b_r <= res.b_star <= res.b_e
+    assert res.mse_star <= res.mse_e
+
+
+def test_ds_degenerate_and_arguments():
+    c = np.full(100, 2.5, dtype=np.float32)
+    st = oracle.stats(c)
+    rc, res, qp, curve = oracle.ds_search(c, st, 2)
+    assert rc == oracle.WARN_DEGENERATE and res.k_star == 0 and res.b_star == res.b_e == 0.0
+    assert qp.flags == 1 and res.mse_star == 0.0
+    x = si.flat_iid(1000, 1, "laplace")
+    st = oracle.stats(x)
+    assert oracle.ds_search(x, st, 16)[0] == oracle.ERR_BITS
+    assert oracle.ds_search(x, st, 4, steps=0)[0] == oracle.ERR_ARG
+    # literal b_E = sum|x|/N when asked
+    _, res, _, _ = oracle.ds_search(x, st, 4, bmode=1)
+    assert res.b_e == st.mean_abs
+    # one-step search: candidates are exactly b_E and b_R
+    _, res, _, curve = oracle.ds_search(x, st, 4, steps=1)
+    assert len(curve) == 2 and res.k_star in (0, 1)
+
+
+def test_ds_never_worse_and_monotone_over_bits():
+    x = si.config_tensor("c1").reshape(-1)
+    st = oracle.stats(x)
+    prev = None
+    for q in (1, 2, 3, 4, 5, 6, 7, 8):
+        _, res, _, _ = oracle.ds_search(x, st, q)
+        assert res.mse_star <= res.mse_e
+        if prev is not None:
+            assert res.mse_star <= prev
+        prev = res.mse_star
+
+
+# -------------------------------------------------------------- select_bits
+
+def _phases():
+    rows = []
+    for line in open(os.path.join(GOLDEN, "adaptive_phases.txt")):
+        if line.strip() and not line.startswith("#"):
+            mbps, bits = line.split()
+            rows.append((float(mbps), int(bits)))
+    return rows
+
+
+def test_eq2_reproduces_paper_phases():
+    n = 64 * 197 * 768
+    for r_target in (85.0, 100.0, 160.0):
+        for q_now in (32, 16, 8, 2):                      # Eq. 2 rescales V to fp32 size first
+            v_bytes = n * q_now / 8.0
+            for mbps, bits in _phases():
+                bw = 1e12 if mbps == 0 else mbps * 1e6
+                rc, q = oracle.select_bits_eq2(v_bytes, q_now, 64, r_target, bw)
+                assert rc == 0 and q == bits, (r_target, q_now, mbps)
+
+
+def test_eq2_by_hand():
+    # c = 309.854208e6 / (0.64 * 200e6) = 2.4207 -> ceil(log2) = 2 -> 32/4 = 8
+    assert oracle.select_bits_eq2(64 * 197 * 768 * 4, 32, 64, 100, 200e6) == (0, 8)
+    assert oracle.select_bits_eq2(1000, 32, 1, 1, 8000.0) == (0, 32)       # c = 1 exactly: fits
+    assert oracle.select_bits_eq2(1000, 32, 1, 1, 7999.0) == (0, 16)
+    assert oracle.select_bits_eq2(1000, 32, 1, 1, 1.0) == (0, 1)           # clamped below
+    assert oracle.select_bits_eq2(0, 32, 1, 1, 1.0)[0] == oracle.ERR_ARG
+
+
+def test_select_bits_principle():
+    n = 64 * 197 * 768
+    budget = 0.64
+    allowed = (32, 16, 8, 6, 4, 2)
+    # the paper's phases with the table's bit-width set: same settled answers as Eq. 2
+    for mbps, bits in _phases():
+        bw = 1e12 if mbps == 0 else mbps * 1e6
+        assert oracle.select_bits(bw, budget, n, 0, allowed) == (0, bits)
+    # 6 bits is chosen in a band below 8 bits' threshold (the transient of phase 3)
+    assert oracle.select_bits(100e6, budget, n, 0, allowed) == (0, 6)
+    # exact thresholds: payload bits <= capacity
+    need = 8 * ((n * 6 + 7) // 8)
+    assert oracle.select_bits(need / budget * (1 + 1e-12), budget, n, 0, allowed)[1] == 6
+    assert oracle.select_bits(need / budget * (1 - 1e-9), budget, n, 0, allowed)[1] == 4
+    assert oracle.select_bits(need / budget * (1 + 1e-12), budget, n, 1, allowed)[1] == 4   # header bytes count
+    # monotone in bandwidth, infeasible -> smallest with a warning
+    last = 0
+    for bw in np.linspace(1e6, 600e6, 400):
+        rc, q = oracle.select_bits(bw, budget, n, 0, allowed)
+        assert q >= last
+        last = q
+        assert (rc == oracle.WARN_INFEASIBLE) == (8 * ((n * 2 + 7) // 8) > bw * budget)
+    assert oracle.select_bits(1.0, budget, n, 0, (4, 2, 8)) == (oracle.WARN_INFEASIBLE, 2)
+    assert oracle.select_bits(1e6, 1.0, 10, 0, ())[0] == oracle.ERR_ARG
+    assert oracle.select_bits(1e6, 1.0, 10, 0, (0,))[0] == oracle.ERR_ARG
+
+
+# ------------------------------------------------------------------- inputs
+
+def test_generator_is_counter_based_and_shaped():
+    a = si.flat_iid(5000, 4, "laplace")
+    b = si.laplace01(4, si.STREAM_VALUE, 1234, 100).astype(np.float32)
+    assert np.array_equal(a[1234:1334], b)
+    x = si.config_tensor("c1")
+    assert x.shape == (1, 197, 768) and x.dtype == np.float32
+    mu, s = si.channel_params(0, 768)
+    assert np.all(np.abs(x.reshape(-1, 768).mean(0) - mu) <= 6 * s * math.sqrt(2.0 / 197))
+    x3 = si.vit_activation((4, 197, 1024), 2, outlier_frac=0.01)
+    sd = x3.reshape(-1, 1024).std(0)
+    assert (sd > 8 * np.median(sd)).sum() >= 5
+    h = si.to_bf16_bits(a)
+    assert np.array_equal(oracle.widen_bf16(h), si.bf16_bits_to_f32(h))
+    assert np.max(np.abs(si.bf16_bits_to_f32(h) - a) / np.maximum(np.abs(a), 1e-30)) <= 2.0 ** -8
+    bw = si.bandwidth_trace(3, 100)
+    assert bw.min() >= 5e6 and bw.max() <= 200e6 and len(np.unique(bw)) == 100
