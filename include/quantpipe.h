@@ -1,0 +1,207 @@
+/*
+ * quantpipe.h -- C ABI of the activation-quantization path of QuantPipe (arXiv 2211.04515)
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The path (paper Sec. 3, "System Design and Implementation"):
+ *   sender    qp_stats -> [qp_dsaciq_search] -> qp_aciq_alpha / qp_aciq_qparams_device
+ *             -> qp_quantize_pack
+ *   receiver  qp_unpack_dequantize
+ *   control   qp_select_bits (bit-width from the measured link bandwidth)
+ *
+ * Conventions
+ *   - Plain C.  No exceptions cross the boundary.  Every call returns a qp_status value:
+ *     0 = QP_OK, negative = error (outputs undefined), positive = warning (outputs defined).
+ *   - "d_" arguments are DEVICE pointers, "h_" arguments are HOST pointers; the caller owns
+ *     every buffer it passes.  The library owns only the qp_ctx (a few MB of device
+ *     scratch: block partials, histogram, candidate table, counters, status word).
+ *   - Device-taking calls enqueue work on `stream` (a cudaStream_t passed as void*; NULL is
+ *     the legacy default stream) and return without synchronising.  One qp_ctx may be used
+ *     from one stream at a time.  Inputs and outputs must not overlap.
+ *   - dtype: QP_F32 (0) or QP_BF16 (1).  Tensors are contiguous; n is the element count.
+ *   - bits: 1..8 or 16 for quantize/pack and unpack/dequantize; 32 ("send raw fp32") is only
+ *     a possible result of qp_select_bits.
+ *   - Non-finite inputs: NaN quantizes to code 0, +-Inf clamps to the clip range; the
+ *     statistics and the search skip and count them.
+ */
+#ifndef QUANTPIPE_H
+#define QUANTPIPE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qp_ctx qp_ctx;
+
+enum {
+    QP_OK = 0,
+    QP_ERR_INVALID_ARG = -1,
+    QP_ERR_UNSUPPORTED_BITS = -2,
+    QP_ERR_UNSUPPORTED_DTYPE = -3,
+    QP_ERR_BUFFER_TOO_SMALL = -4,
+    QP_ERR_ALIGNMENT = -5,
+    QP_ERR_CUDA = -6,
+    QP_ERR_TIMEOUT = -7,
+    QP_WARN_INFEASIBLE = 1,   /* qp_select_bits: nothing fits, smallest width returned   */
+    QP_WARN_DEGENERATE = 2,   /* empty clip range (constant tensor): all codes are 0     */
+    QP_WARN_NONFINITE = 3     /* reported by qp_get_status: NaN/Inf were seen and skipped */
+};
+
+enum { QP_F32 = 0, QP_BF16 = 1 };
+enum { QP_DIST_LAPLACE = 0, QP_DIST_GAUSS = 1 };
+enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the formula as printed */ };
+
+#define QP_DEFAULT_STEPS 100      /* search steps t (Sec. 3, directed search) */
+#define QP_DEFAULT_HIST_BINS 100
+#define QP_MAX_STEPS 1023
+#define QP_MAX_HIST_BINS 16384
+
+/* bits of the device status word returned by qp_get_status */
+#define QP_DEV_BITS_MISMATCH 1u   /* a device-resident qp_qparams_t had other bits than the call */
+#define QP_DEV_DEGENERATE 2u
+#define QP_DEV_NONFINITE 4u
+
+/* Per-tensor statistics (Sec. 3: min/max of naive PTQ; mean and Laplace scale b of ACIQ;
+ * b_E of the directed search).  All fields but n are over the finite elements. */
+typedef struct {
+    uint64_t n;          /* elements given                                   */
+    uint64_t nonfinite;  /* NaN or +-Inf among them                          */
+    double mean;
+    double mean_abs;     /* sum|x| / N      (b_E exactly as the paper prints it) */
+    double mad;          /* sum|x - mean| / N  (Laplace scale about the mean)    */
+    double var;          /* sum (x - mean)^2 / N                              */
+    double min, max;
+} qp_stats_t;            /* 64 bytes */
+
+/* Uniform quantizer over the clip range [lo, hi] with L = 2^bits levels, both ends included. */
+typedef struct {
+    float lo, hi;
+    float scale;         /* (hi - lo) / (L - 1) */
+    float inv_scale;     /* (L - 1) / (hi - lo) */
+    int32_t bits;
+    int32_t flags;       /* bit 0: degenerate range, scale = inv_scale = 0 */
+} qp_qparams_t;          /* 24 bytes */
+
+/* Outcome of the directed search (Sec. 3, Eq. 1). */
+typedef struct {
+    double b_e;          /* scale estimated from the data                    */
+    double b_r;          /* search boundary 1 / (2 * peak of the histogram density) */
+    double b_star;       /* chosen scale                                      */
+    double alpha_e;      /* F(q) * b_e                                        */
+    double alpha_star;   /* F(q) * b_star                                     */
+    double mse_e;        /* quantization MSE at b_e                           */
+    double mse_star;     /* quantization MSE at b_star (<= mse_e)             */
+    int32_t k_star;      /* chosen step, 0 = b_e kept                         */
+    int32_t steps, hist_bins, bits;
+} qp_ds_result_t;        /* 72 bytes */
+
+/* ---- context -------------------------------------------------------------------------
+ * qp_create allocates the scratch on `device` (cudaMalloc; call it outside stream capture).
+ * qp_destroy frees it.  Errors: QP_ERR_INVALID_ARG, QP_ERR_CUDA. */
+int32_t qp_create(int device, qp_ctx** out);
+int32_t qp_destroy(qp_ctx* ctx);
+/* Waits for `stream`, then returns and clears the device status word (QP_DEV_* bits),
+ * or a negative qp_status if a CUDA error is pending. */
+int32_t qp_get_status(qp_ctx* ctx, void* stream);
+/* Text of the last error recorded on this context (never NULL). */
+const char* qp_last_error(qp_ctx* ctx);
+const char* qp_status_string(int32_t status);
+
+/* ---- sizes and parameters (host, pure) ------------------------------------------------*/
+
+/* Bytes of the packed stream: ceil(n*bits/8) rounded up to a multiple of 16.
+ * 8-bit codes take a quarter of the fp32 tensor (Sec. 3).  Returns 0 for bits outside
+ * 1..8, 16. */
+uint64_t qp_packed_bytes(uint64_t n, int bits);
+
+/* ACIQ multiplier F(q) with alpha = F(q) * b (Sec. 3).  Laplace: the minimiser of
+ * 2 b^2 exp(-alpha/b) + alpha^2 / (3 * 4^q), i.e. F = W0(3 * 4^q).  Gauss: the minimiser
+ * of the corresponding normal-tail model.  Returns 0 for unsupported bits/dist. */
+double qp_aciq_F(int bits, int dist);
+
+/* Fills a quantizer for the clip range [lo, hi]: ends rounded to fp32, scale and
+ * inv_scale derived in fp64 from the rounded ends and rounded once.
+ * Returns QP_OK, QP_WARN_DEGENERATE (hi <= lo after rounding), QP_ERR_UNSUPPORTED_BITS,
+ * QP_ERR_INVALID_ARG (NaN/Inf ends, NULL). */
+int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out);
+
+/* ---- a1: statistics (Sec. 3) ----------------------------------------------------------
+ * One call fills *d_out (device memory, 64 bytes, 8-byte aligned) from the n elements at
+ * d_x.  Two passes over x (sums/min/max, then deviations about the mean), fp64 merges in a
+ * fixed order: results are bit-reproducible run to run.  n = 0 gives all-zero statistics.
+ * d_x must be aligned to its element size.
+ * Errors: QP_ERR_INVALID_ARG (NULL), QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
+int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream);
+
+/* ---- a3: ACIQ clip (Sec. 3: alpha = F(q) * b under L(mu, b)) ---------------------------
+ * Host form: from statistics already copied to the host.  b is h_stats->mad (bmode
+ * QP_B_MAD), h_stats->mean_abs (QP_B_MEAN_ABS), sqrt(var) for QP_DIST_GAUSS, or b_override
+ * when b_override > 0.  Writes alpha (optional) and the quantizer for
+ * [mean - alpha, mean + alpha] (optional).  Returns as qp_make_qparams. */
+int32_t qp_aciq_alpha(const qp_stats_t* h_stats, int bits, int dist, int bmode, double b_override,
+                      double* h_alpha_out, qp_qparams_t* h_qp_out);
+/* Device form: same arithmetic in a one-thread kernel reading *d_stats and writing
+ * *d_qp_out, so that stats -> clip -> quantize needs no host round trip. */
+int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode,
+                               qp_qparams_t* d_qp_out, void* stream);
+
+/* ---- a2 + a4: directed search DS-ACIQ (Sec. 3 "Directed Search", Eq. 1) -----------------
+ * Histogram of x with hist_bins equal bins over [min, max]; b_R = 1 / (2 * peak density);
+ * candidates b_k = b_E + k (b_R - b_E) / steps, k = 0..steps; each is scored by the
+ * quantization MSE of x under the clip F(bits) * b_k about the mean; the smallest k with
+ * the lowest MSE wins (k = 0 keeps b_E).  d_stats must hold the statistics of the same x.
+ * Writes *d_out (optional) and the winning quantizer *d_qp_out (optional); both device
+ * memory.  bits 1..8; 1 <= steps <= QP_MAX_STEPS; 1 <= hist_bins <= QP_MAX_HIST_BINS.
+ * Errors: as qp_stats, plus QP_ERR_UNSUPPORTED_BITS. */
+int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
+                         int bits, int bmode, int steps, int hist_bins,
+                         qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, void* stream);
+/* Copies the MSE of every candidate of the last search on this context (steps+1 values)
+ * to host memory after waiting for `stream`.  Diagnostic. */
+int32_t qp_dsaciq_curve(qp_ctx* ctx, double* h_curve, int capacity, void* stream);
+/* Policy of the paper's evaluation (Sec. 3): the search is switched on at 4 bits and below. */
+int32_t qp_policy_use_ds(int bits);
+
+/* ---- a5: clamp, quantize, bit-pack (Sec. 3: uniform quantization of the clipped tensor) -
+ * code_i = round_half_even((clamp(x_i, lo, hi) - lo) * inv_scale), each fp32 operation
+ * rounded on its own.  Element i occupies stream bits [i*bits, (i+1)*bits), least
+ * significant bit first; stream bit j is bit (j mod 8) of byte (j div 8); bits = 16 is one
+ * little-endian uint16 per element.  All qp_packed_bytes(n, bits) bytes are written, pad
+ * bits zero.  `qp` is a host pointer (qp_on_device = 0, read before returning) or a
+ * device pointer (qp_on_device = 1, read by the kernel; its bits must equal `bits`,
+ * otherwise QP_DEV_BITS_MISMATCH is raised in the status word).
+ * d_packed must be 16-byte aligned; d_x aligned to its element size (16-byte alignment
+ * enables the fast path).
+ * Errors: QP_ERR_INVALID_ARG, QP_ERR_UNSUPPORTED_BITS, QP_ERR_UNSUPPORTED_DTYPE,
+ * QP_ERR_BUFFER_TOO_SMALL (packed_capacity < qp_packed_bytes), QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
+int32_t qp_quantize_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits,
+                         const qp_qparams_t* qp, int qp_on_device,
+                         void* d_packed, uint64_t packed_capacity, void* stream);
+
+/* ---- a6: unpack, dequantize (the receiver's side of Sec. 3) -----------------------------
+ * y_i = fma(code_i, scale, lo) in fp32 (one rounding), written as out_dtype (QP_F32, or
+ * QP_BF16 rounded to nearest even).  d_packed as written by qp_quantize_pack (16-byte
+ * aligned, qp_packed_bytes long); d_y aligned to its element size.
+ * Errors: as qp_quantize_pack. */
+int32_t qp_unpack_dequantize(qp_ctx* ctx, const void* d_packed, uint64_t n, int bits,
+                             const qp_qparams_t* qp, int qp_on_device,
+                             void* d_y, int out_dtype, void* stream);
+
+/* ---- a7: bit-width from bandwidth (Sec. 1, Sec. 3 "Adaptive PDA", Eq. 2) ----------------
+ * Widest allowed width whose payload fits the budget:
+ * 8 * (ceil(n_elems*q/8) + overhead_bytes) <= bandwidth_bps * budget_s; q = 32 is the raw
+ * fp32 tensor.  h_allowed: n_allowed widths in 1..32, any order; NULL selects the widths of
+ * the paper's Table 1, {32,16,8,6,4,2}.  Nothing fits: smallest allowed and
+ * QP_WARN_INFEASIBLE. */
+int32_t qp_select_bits(double bandwidth_bps, double budget_s, uint64_t n_elems, uint64_t overhead_bytes,
+                       const int32_t* h_allowed, int n_allowed, int32_t* h_bits_out);
+/* Eq. 2 as printed: q' = 32 / 2^ceil(log2((V*32/q) / ((S/R) * B))), V bytes at the current
+ * width q, B bit/s, S images per microbatch, R target images/s; clamped to [1, 32]. */
+int32_t qp_select_bits_eq2(double v_bytes, int q_t, double s_images, double r_images_per_s,
+                           double bandwidth_bps, int32_t* h_bits_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QUANTPIPE_H */

@@ -1,0 +1,282 @@
+"""ctypes binding of libquantpipe.so: argument marshalling only.
+
+Every step of the path runs in the CUDA library; this module turns torch tensors into
+pointers and sizes, passes the current CUDA stream, and raises on error codes.  There is no
+CPU fallback: if the library has not been built, loading fails with an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libquantpipe.so")
+
+QP_OK = 0
+QP_ERR_INVALID_ARG, QP_ERR_UNSUPPORTED_BITS, QP_ERR_UNSUPPORTED_DTYPE = -1, -2, -3
+QP_ERR_BUFFER_TOO_SMALL, QP_ERR_ALIGNMENT, QP_ERR_CUDA, QP_ERR_TIMEOUT = -4, -5, -6, -7
+QP_WARN_INFEASIBLE, QP_WARN_DEGENERATE, QP_WARN_NONFINITE = 1, 2, 3
+QP_F32, QP_BF16 = 0, 1
+QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
+QP_B_MAD, QP_B_MEAN_ABS = 0, 1
+QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE = 1, 2, 4
+QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
+
+EXPORTS = (
+    "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
+    "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
+    "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
+    "qp_select_bits_eq2",
+)
+
+
+class Stats(C.Structure):
+    _fields_ = [("n", C.c_uint64), ("nonfinite", C.c_uint64), ("mean", C.c_double), ("mean_abs", C.c_double),
+                ("mad", C.c_double), ("var", C.c_double), ("min", C.c_double), ("max", C.c_double)]
+
+
+class QParams(C.Structure):
+    _fields_ = [("lo", C.c_float), ("hi", C.c_float), ("scale", C.c_float), ("inv_scale", C.c_float),
+                ("bits", C.c_int32), ("flags", C.c_int32)]
+
+
+class DSResult(C.Structure):
+    _fields_ = [("b_e", C.c_double), ("b_r", C.c_double), ("b_star", C.c_double), ("alpha_e", C.c_double),
+                ("alpha_star", C.c_double), ("mse_e", C.c_double), ("mse_star", C.c_double),
+                ("k_star", C.c_int32), ("steps", C.c_int32), ("hist_bins", C.c_int32), ("bits", C.c_int32)]
+
+
+class QuantPipeError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"quantpipe status {status}: {message}")
+        self.status = status
+
+
+_lib = None
+
+
+def load() -> C.CDLL:
+    """Loads libquantpipe.so; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2211_04515_b200.build` "
+                           "(there is no CPU fallback)")
+    L = C.CDLL(LIB_PATH)
+    vp, u64, i32, dbl = C.c_void_p, C.c_uint64, C.c_int32, C.c_double
+    L.qp_create.argtypes = [C.c_int, C.POINTER(vp)]
+    L.qp_destroy.argtypes = [vp]
+    L.qp_get_status.argtypes = [vp, vp]
+    L.qp_last_error.argtypes = [vp]
+    L.qp_last_error.restype = C.c_char_p
+    L.qp_status_string.argtypes = [i32]
+    L.qp_status_string.restype = C.c_char_p
+    L.qp_packed_bytes.argtypes = [u64, C.c_int]
+    L.qp_packed_bytes.restype = u64
+    L.qp_aciq_F.argtypes = [C.c_int, C.c_int]
+    L.qp_aciq_F.restype = dbl
+    L.qp_make_qparams.argtypes = [dbl, dbl, C.c_int, C.POINTER(QParams)]
+    L.qp_stats.argtypes = [vp, vp, C.c_int, u64, vp, vp]
+    L.qp_aciq_alpha.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, dbl, C.POINTER(dbl), C.POINTER(QParams)]
+    L.qp_aciq_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.qp_dsaciq_search.argtypes = [vp, vp, C.c_int, u64, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
+    L.qp_dsaciq_curve.argtypes = [vp, C.POINTER(dbl), C.c_int, vp]
+    L.qp_policy_use_ds.argtypes = [C.c_int]
+    L.qp_quantize_pack.argtypes = [vp, vp, C.c_int, u64, C.c_int, vp, C.c_int, vp, u64, vp]
+    L.qp_unpack_dequantize.argtypes = [vp, vp, u64, C.c_int, vp, C.c_int, vp, C.c_int, vp]
+    L.qp_select_bits.argtypes = [dbl, dbl, u64, u64, C.POINTER(i32), C.c_int, C.POINTER(i32)]
+    L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
+    for name in EXPORTS:
+        fn = getattr(L, name)
+        if name not in ("qp_last_error", "qp_status_string", "qp_packed_bytes", "qp_aciq_F"):
+            fn.restype = i32
+    _lib = L
+    return L
+
+
+# ------------------------------------------------------------- host, pure
+
+def qp_packed_bytes(n: int, bits: int) -> int:
+    return int(load().qp_packed_bytes(n, bits))
+
+
+def qp_aciq_F(bits: int, dist: int = QP_DIST_LAPLACE) -> float:
+    return float(load().qp_aciq_F(bits, dist))
+
+
+def qp_status_string(status: int) -> str:
+    return load().qp_status_string(status).decode()
+
+
+def qp_make_qparams(lo: float, hi: float, bits: int):
+    qp = QParams()
+    return int(load().qp_make_qparams(lo, hi, bits, C.byref(qp))), qp
+
+
+def qp_aciq_alpha(stats: Stats, bits: int, dist: int = QP_DIST_LAPLACE, bmode: int = QP_B_MAD,
+                  b_override: float = 0.0):
+    alpha, qp = C.c_double(), QParams()
+    rc = load().qp_aciq_alpha(C.byref(stats), bits, dist, bmode, b_override, C.byref(alpha), C.byref(qp))
+    return int(rc), alpha.value, qp
+
+
+def qp_policy_use_ds(bits: int) -> bool:
+    return bool(load().qp_policy_use_ds(bits))
+
+
+def qp_select_bits(bandwidth_bps: float, budget_s: float, n_elems: int, overhead_bytes: int = 0, allowed=None):
+    out = C.c_int32()
+    if allowed is None:
+        rc = load().qp_select_bits(bandwidth_bps, budget_s, n_elems, overhead_bytes, None, 0, C.byref(out))
+    else:
+        arr = (C.c_int32 * len(allowed))(*allowed)
+        rc = load().qp_select_bits(bandwidth_bps, budget_s, n_elems, overhead_bytes, arr, len(allowed), C.byref(out))
+    return int(rc), out.value
+
+
+def qp_select_bits_eq2(v_bytes: float, q_t: int, s_images: float, r_images_per_s: float, bandwidth_bps: float):
+    out = C.c_int32()
+    rc = load().qp_select_bits_eq2(v_bytes, q_t, s_images, r_images_per_s, bandwidth_bps, C.byref(out))
+    return int(rc), out.value
+
+
+# ------------------------------------------------------------ device calls
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return QP_F32
+    if t.dtype == torch.bfloat16:
+        return QP_BF16
+    raise QuantPipeError(QP_ERR_UNSUPPORTED_DTYPE, f"unsupported dtype {t.dtype}")
+
+
+def _stream(device) -> int:
+    return torch.cuda.current_stream(device).cuda_stream
+
+
+def _as_struct(t: torch.Tensor, cls):
+    """Copies a device byte buffer holding one struct to the host (synchronises)."""
+    raw = t.detach().cpu().contiguous().numpy().tobytes()
+    return cls.from_buffer_copy(raw[:C.sizeof(cls)])
+
+
+class Context:
+    """One qp_ctx on one device.  Methods enqueue work on torch's current stream."""
+
+    def __init__(self, device: int | torch.device = 0):
+        dev = torch.device("cuda", device) if isinstance(device, int) else torch.device(device)
+        if dev.type != "cuda":
+            raise QuantPipeError(QP_ERR_INVALID_ARG, "a CUDA device is required")
+        self.device = torch.device("cuda", dev.index if dev.index is not None else torch.cuda.current_device())
+        self._lib = load()
+        handle = C.c_void_p()
+        rc = self._lib.qp_create(self.device.index, C.byref(handle))
+        if rc != QP_OK:
+            raise QuantPipeError(rc, "qp_create failed: " + qp_status_string(rc))
+        self._h = handle
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.qp_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- helpers
+    def _check(self, rc: int) -> int:
+        if rc < 0:
+            raise QuantPipeError(rc, self._lib.qp_last_error(self._h).decode())
+        return int(rc)
+
+    def _bytes(self, nbytes: int) -> torch.Tensor:
+        return torch.empty(nbytes, dtype=torch.uint8, device=self.device)
+
+    def _qp_arg(self, qp):
+        """(pointer, on_device, keepalive) for a host QParams struct or a device byte tensor."""
+        if isinstance(qp, QParams):
+            return C.cast(C.pointer(qp), C.c_void_p), 0, qp
+        if isinstance(qp, torch.Tensor) and qp.is_cuda:
+            return C.c_void_p(qp.data_ptr()), 1, qp
+        raise QuantPipeError(QP_ERR_INVALID_ARG, "qp must be a QParams struct or a device tensor")
+
+    # -- a1
+    def qp_stats(self, x: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
+        """Statistics of x into a 64-byte device buffer (returned)."""
+        assert x.is_cuda and x.is_contiguous()
+        out = self._bytes(C.sizeof(Stats)) if out is None else out
+        self._check(self._lib.qp_stats(self._h, x.data_ptr(), _dtype_code(x), x.numel(), out.data_ptr(),
+                                       _stream(self.device)))
+        return out
+
+    # -- a3
+    def qp_aciq_qparams_device(self, d_stats: torch.Tensor, bits: int, dist: int = QP_DIST_LAPLACE,
+                               bmode: int = QP_B_MAD, out: torch.Tensor | None = None) -> torch.Tensor:
+        out = self._bytes(C.sizeof(QParams)) if out is None else out
+        self._check(self._lib.qp_aciq_qparams_device(self._h, d_stats.data_ptr(), bits, dist, bmode, out.data_ptr(),
+                                                     _stream(self.device)))
+        return out
+
+    # -- a2 + a4
+    def qp_dsaciq_search(self, x: torch.Tensor, d_stats: torch.Tensor, bits: int, bmode: int = QP_B_MAD,
+                         steps: int = QP_DEFAULT_STEPS, hist_bins: int = QP_DEFAULT_HIST_BINS,
+                         out_result: torch.Tensor | None = None, out_qp: torch.Tensor | None = None):
+        """Directed search; returns (device DSResult bytes, device QParams bytes)."""
+        assert x.is_cuda and x.is_contiguous()
+        out_result = self._bytes(C.sizeof(DSResult)) if out_result is None else out_result
+        out_qp = self._bytes(C.sizeof(QParams)) if out_qp is None else out_qp
+        self._check(self._lib.qp_dsaciq_search(self._h, x.data_ptr(), _dtype_code(x), x.numel(), d_stats.data_ptr(),
+                                               bits, bmode, steps, hist_bins, out_result.data_ptr(), out_qp.data_ptr(),
+                                               _stream(self.device)))
+        return out_result, out_qp
+
+    def qp_dsaciq_curve(self, steps: int):
+        buf = (C.c_double * (steps + 1))()
+        self._check(self._lib.qp_dsaciq_curve(self._h, buf, steps + 1, _stream(self.device)))
+        return list(buf)
+
+    # -- a5
+    def qp_quantize_pack(self, x: torch.Tensor, bits: int, qp, out: torch.Tensor | None = None) -> torch.Tensor:
+        assert x.is_cuda and x.is_contiguous()
+        need = qp_packed_bytes(x.numel(), bits)
+        if out is None:
+            out = self._bytes(need)
+        ptr, on_dev, _keep = self._qp_arg(qp)
+        self._check(self._lib.qp_quantize_pack(self._h, x.data_ptr(), _dtype_code(x), x.numel(), bits, ptr, on_dev,
+                                               out.data_ptr(), out.numel() * out.element_size(),
+                                               _stream(self.device)))
+        return out
+
+    # -- a6
+    def qp_unpack_dequantize(self, packed: torch.Tensor, n: int, bits: int, qp, out: torch.Tensor | None = None,
+                             out_dtype: torch.dtype = torch.float32) -> torch.Tensor:
+        assert packed.is_cuda and packed.is_contiguous()
+        if out is None:
+            out = torch.empty(n, dtype=out_dtype, device=self.device)
+        assert out.numel() >= n and out.is_contiguous()
+        need = qp_packed_bytes(n, bits)
+        if packed.numel() * packed.element_size() < need:
+            raise QuantPipeError(QP_ERR_BUFFER_TOO_SMALL, "packed buffer shorter than qp_packed_bytes(n, bits)")
+        ptr, on_dev, _keep = self._qp_arg(qp)
+        self._check(self._lib.qp_unpack_dequantize(self._h, packed.data_ptr(), n, bits, ptr, on_dev, out.data_ptr(),
+                                                   _dtype_code(out), _stream(self.device)))
+        return out
+
+    # -- status / read-back
+    def qp_get_status(self) -> int:
+        return self._check(self._lib.qp_get_status(self._h, _stream(self.device)))
+
+    def read_stats(self, d_stats: torch.Tensor) -> Stats:
+        return _as_struct(d_stats, Stats)
+
+    def read_qparams(self, d_qp: torch.Tensor) -> QParams:
+        return _as_struct(d_qp, QParams)
+
+    def read_ds_result(self, d_res: torch.Tensor) -> DSResult:
+        return _as_struct(d_res, DSResult)

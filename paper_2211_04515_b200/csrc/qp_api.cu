@@ -1,0 +1,376 @@
+// Host side of the C ABI: context, argument checks, the O(1) host functions.
+#include <math.h>
+#include <string.h>
+
+#include <new>
+
+#include "qp_internal.cuh"
+
+// ------------------------------------------------------------------ errors
+
+int32_t qp_fail(qp_ctx* ctx, int32_t status, const char* what)
+{
+    if (ctx) snprintf(ctx->err, sizeof ctx->err, "%s: %s", qp_status_string(status), what);
+    return status;
+}
+
+int32_t qp_check_launch(qp_ctx* ctx, const char* what)
+{
+    const cudaError_t e = cudaGetLastError();
+    if (e == cudaSuccess) return QP_OK;
+    if (ctx) snprintf(ctx->err, sizeof ctx->err, "CUDA error in %s: %s", what, cudaGetErrorString(e));
+    return QP_ERR_CUDA;
+}
+
+extern "C" const char* qp_status_string(int32_t s)
+{
+    switch (s) {
+        case QP_OK: return "ok";
+        case QP_ERR_INVALID_ARG: return "invalid argument";
+        case QP_ERR_UNSUPPORTED_BITS: return "unsupported bit-width";
+        case QP_ERR_UNSUPPORTED_DTYPE: return "unsupported dtype";
+        case QP_ERR_BUFFER_TOO_SMALL: return "buffer too small";
+        case QP_ERR_ALIGNMENT: return "misaligned pointer";
+        case QP_ERR_CUDA: return "CUDA error";
+        case QP_ERR_TIMEOUT: return "device wait timed out";
+        case QP_WARN_INFEASIBLE: return "warning: no allowed bit-width fits the budget";
+        case QP_WARN_DEGENERATE: return "warning: degenerate clip range";
+        case QP_WARN_NONFINITE: return "warning: non-finite inputs were skipped";
+        default: return "unknown status";
+    }
+}
+
+extern "C" const char* qp_last_error(qp_ctx* ctx) { return ctx ? ctx->err : "no context"; }
+
+// ----------------------------------------------------------------- context
+
+static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+extern "C" int32_t qp_create(int device, qp_ctx** out)
+{
+    if (!out) return QP_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) { cudaGetLastError(); return QP_ERR_CUDA; }
+    if (device < 0 || device >= count) return QP_ERR_INVALID_ARG;
+    qp_device_guard guard(device);
+    if (!guard.ok) return QP_ERR_CUDA;
+
+    qp_ctx* c = new (std::nothrow) qp_ctx();
+    if (!c) return QP_ERR_CUDA;
+    memset(c, 0, sizeof *c);
+    c->device = device;
+    strcpy(c->err, "ok");
+    if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+        delete c;
+        return QP_ERR_CUDA;
+    }
+
+    size_t off = 0;
+    const size_t o_part = off;   off = align_up(off + sizeof(qp_stats_partial) * QP_MAX_BLOCKS, 256);
+    const size_t o_hist = off;   off = align_up(off + sizeof(unsigned long long) * QP_MAX_HIST_BINS, 256);
+    const size_t o_cand = off;   off = align_up(off + sizeof(float4) * (QP_MAX_STEPS + 1), 256);
+    const size_t o_valid = off;  off = align_up(off + sizeof(int) * (QP_MAX_STEPS + 1), 256);
+    const size_t o_sums = off;   off = align_up(off + sizeof(double) * QP_MAX_BLOCKS * QP_EVAL_K, 256);
+    const size_t o_curve = off;  off = align_up(off + sizeof(double) * (QP_MAX_STEPS + 1), 256);
+    const size_t o_setup = off;  off = align_up(off + sizeof(qp_ds_setup), 256);
+    const size_t o_ticket = off; off = align_up(off + sizeof(unsigned) * 4, 256);
+    const size_t o_status = off; off = align_up(off + sizeof(unsigned), 256);
+
+    if (cudaMalloc(&c->d_base, off) != cudaSuccess || cudaMemset(c->d_base, 0, off) != cudaSuccess) {
+        cudaGetLastError();
+        if (c->d_base) cudaFree(c->d_base);
+        delete c;
+        return QP_ERR_CUDA;
+    }
+    char* b = static_cast<char*>(c->d_base);
+    c->d_part = reinterpret_cast<qp_stats_partial*>(b + o_part);
+    c->d_hist = reinterpret_cast<unsigned long long*>(b + o_hist);
+    c->d_cand = reinterpret_cast<float4*>(b + o_cand);
+    c->d_valid = reinterpret_cast<int*>(b + o_valid);
+    c->d_sums = reinterpret_cast<double*>(b + o_sums);
+    c->d_curve = reinterpret_cast<double*>(b + o_curve);
+    c->d_setup = reinterpret_cast<qp_ds_setup*>(b + o_setup);
+    c->d_ticket = reinterpret_cast<unsigned*>(b + o_ticket);
+    c->d_status = reinterpret_cast<unsigned*>(b + o_status);
+    *out = c;
+    return QP_OK;
+}
+
+extern "C" int32_t qp_destroy(qp_ctx* ctx)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    qp_device_guard guard(ctx->device);
+    const cudaError_t e = cudaFree(ctx->d_base);
+    delete ctx;
+    return e == cudaSuccess ? QP_OK : QP_ERR_CUDA;
+}
+
+extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    qp_device_guard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned word = 0;
+    cudaError_t e = cudaMemcpyAsync(&word, ctx->d_status, sizeof word, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_status, 0, sizeof word, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_get_status: %s", cudaGetErrorString(e));
+        return QP_ERR_CUDA;
+    }
+    return (int32_t)word;
+}
+
+// ------------------------------------------------------ host, pure functions
+
+extern "C" uint64_t qp_packed_bytes(uint64_t n, int bits)
+{
+    if (!qp_bits_ok(bits)) return 0;
+    const uint64_t raw = (n * (uint64_t)bits + 7u) / 8u;
+    return (raw + 15u) / 16u * 16u;
+}
+
+// Laplace: F = W0(3 * 4^q) by Halley's iteration on w e^w = z.
+static double lambert_w0(double z)
+{
+    double w = z < 3.0 ? 0.5 : log(z) - log(log(z));
+    for (int it = 0; it < 64; ++it) {
+        const double e = exp(w);
+        const double f = w * e - z;
+        const double d = e * (w + 1.0) - (w + 2.0) * f / (2.0 * w + 2.0);
+        const double step = f / d;
+        w -= step;
+        if (fabs(step) <= 4e-16 * fabs(w)) break;
+    }
+    return w;
+}
+
+// Gauss: root of 4 [a (1 - Phi(a)) - phi(a)] + 2a / (3 * 4^q) by Newton from above
+// (the function is increasing and concave on a > 0), guarded by bisection bounds.
+static double gauss_F(int bits)
+{
+    const double c = 2.0 / (3.0 * pow(4.0, (double)bits));
+    double lo = 0.0, hi = 64.0, a = 1.0 + 0.45 * bits;
+    for (int it = 0; it < 200; ++it) {
+        const double tail = 0.5 * erfc(a * M_SQRT1_2);
+        const double pdf = exp(-0.5 * a * a) * 0.3989422804014327;
+        const double g = 4.0 * (a * tail - pdf) + c * a;
+        if (g < 0.0) lo = a; else hi = a;
+        const double dg = 4.0 * tail + c;
+        double next = a - g / dg;
+        if (!(next > lo && next < hi)) next = 0.5 * (lo + hi);
+        if (fabs(next - a) <= 1e-15 * fabs(a)) { a = next; break; }
+        a = next;
+    }
+    return a;
+}
+
+double qp_host_aciq_F(int bits, int dist)
+{
+    if (!qp_bits_ok(bits)) return 0.0;
+    if (dist == QP_DIST_LAPLACE) return lambert_w0(3.0 * pow(4.0, (double)bits));
+    if (dist == QP_DIST_GAUSS) return gauss_F(bits);
+    return 0.0;
+}
+
+extern "C" double qp_aciq_F(int bits, int dist) { return qp_host_aciq_F(bits, dist); }
+
+extern "C" int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out)
+{
+    if (!h_out) return QP_ERR_INVALID_ARG;
+    if (!qp_bits_ok(bits)) return QP_ERR_UNSUPPORTED_BITS;
+    if (!isfinite(lo) || !isfinite(hi)) return QP_ERR_INVALID_ARG;
+    return qp_fill_qparams(lo, hi, bits, h_out);
+}
+
+extern "C" int32_t qp_aciq_alpha(const qp_stats_t* h_stats, int bits, int dist, int bmode, double b_override,
+                                 double* h_alpha_out, qp_qparams_t* h_qp_out)
+{
+    if (!h_stats) return QP_ERR_INVALID_ARG;
+    if (!qp_bits_ok(bits)) return QP_ERR_UNSUPPORTED_BITS;
+    if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
+        return QP_ERR_INVALID_ARG;
+    const double b = b_override > 0.0       ? b_override
+                     : dist == QP_DIST_GAUSS ? sqrt(h_stats->var)
+                     : bmode == QP_B_MEAN_ABS ? h_stats->mean_abs
+                                              : h_stats->mad;
+    const double alpha = qp_host_aciq_F(bits, dist) * b;
+    if (h_alpha_out) *h_alpha_out = alpha;
+    if (!h_qp_out) return QP_OK;
+    const double lo = h_stats->mean - alpha, hi = h_stats->mean + alpha;
+    if (!isfinite(lo) || !isfinite(hi)) return QP_ERR_INVALID_ARG;
+    return qp_fill_qparams(lo, hi, bits, h_qp_out);
+}
+
+extern "C" int32_t qp_policy_use_ds(int bits) { return bits >= 1 && bits <= 4 ? 1 : 0; }
+
+extern "C" int32_t qp_select_bits(double bandwidth_bps, double budget_s, uint64_t n_elems, uint64_t overhead_bytes,
+                                  const int32_t* h_allowed, int n_allowed, int32_t* h_bits_out)
+{
+    static const int32_t table1[6] = {32, 16, 8, 6, 4, 2};
+    if (!h_bits_out || !(bandwidth_bps >= 0.0) || !(budget_s >= 0.0)) return QP_ERR_INVALID_ARG;
+    if (!h_allowed) { h_allowed = table1; n_allowed = 6; }
+    if (n_allowed < 1) return QP_ERR_INVALID_ARG;
+    const double capacity = bandwidth_bps * budget_s;
+    int best = 0, smallest = 33;
+    for (int i = 0; i < n_allowed; ++i) {
+        const int q = h_allowed[i];
+        if (q < 1 || q > 32) return QP_ERR_INVALID_ARG;
+        smallest = q < smallest ? q : smallest;
+        const uint64_t payload = (n_elems * (uint64_t)q + 7u) / 8u;
+        const double need = 8.0 * ((double)payload + (double)overhead_bytes);
+        if (need <= capacity && q > best) best = q;
+    }
+    if (best == 0) { *h_bits_out = smallest; return QP_WARN_INFEASIBLE; }
+    *h_bits_out = best;
+    return QP_OK;
+}
+
+extern "C" int32_t qp_select_bits_eq2(double v_bytes, int q_t, double s_images, double r_images_per_s,
+                                      double bandwidth_bps, int32_t* h_bits_out)
+{
+    if (!h_bits_out || !(v_bytes > 0.0) || q_t < 1 || q_t > 32 || !(s_images > 0.0) || !(r_images_per_s > 0.0) ||
+        !(bandwidth_bps > 0.0))
+        return QP_ERR_INVALID_ARG;
+    const double fp32_bits = v_bytes * 8.0 * 32.0 / (double)q_t;
+    const double ratio = fp32_bits / ((s_images / r_images_per_s) * bandwidth_bps);
+    double e = ceil(log2(ratio));
+    if (!(e > 0.0)) e = 0.0;
+    if (e > 5.0) e = 5.0;
+    *h_bits_out = 32 >> (int)e;
+    return QP_OK;
+}
+
+// ------------------------------------------------ device-taking entry points
+
+static int32_t check_x(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (dtype != QP_F32 && dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "dtype must be QP_F32 or QP_BF16");
+    if (n > 0 && !d_x) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null tensor");
+    const uintptr_t a = dtype == QP_F32 ? 3u : 1u;
+    if ((uintptr_t)d_x & a) return qp_fail(ctx, QP_ERR_ALIGNMENT, "tensor not aligned to its element size");
+    if (n >= (1ull << 40)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "n too large");
+    return QP_OK;
+}
+
+extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream)
+{
+    int32_t rc = check_x(ctx, d_x, dtype, n);
+    if (rc) return rc;
+    if (!d_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_out");
+    if ((uintptr_t)d_out & 7u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_out must be 8-byte aligned");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    return qp_launch_stats(ctx, d_x, dtype, n, d_out, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode,
+                                          qp_qparams_t* d_qp_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (!d_stats || !d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "dist/bmode");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    return qp_launch_aciq_device(ctx, d_stats, bits, dist, bmode, qp_host_aciq_F(bits, dist), d_qp_out,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
+                                    int bits, int bmode, int steps, int hist_bins, qp_ds_result_t* d_out,
+                                    qp_qparams_t* d_qp_out, void* stream)
+{
+    int32_t rc = check_x(ctx, d_x, dtype, n);
+    if (rc) return rc;
+    if (!d_stats) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_stats");
+    if (bits < 1 || bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
+    if (steps < 1 || steps > QP_MAX_STEPS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "steps out of range");
+    if (hist_bins < 1 || hist_bins > QP_MAX_HIST_BINS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "hist_bins out of range");
+    if (((uintptr_t)d_out & 7u) || ((uintptr_t)d_qp_out & 3u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "result pointers");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    rc = qp_launch_search(ctx, d_x, dtype, n, d_stats, bits, bmode, steps, hist_bins,
+                          qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_out, d_qp_out, static_cast<cudaStream_t>(stream));
+    if (rc == QP_OK) ctx->last_steps = steps;
+    return rc;
+}
+
+extern "C" int32_t qp_dsaciq_curve(qp_ctx* ctx, double* h_curve, int capacity, void* stream)
+{
+    if (!ctx || !h_curve) return QP_ERR_INVALID_ARG;
+    if (ctx->last_steps < 1) return qp_fail(ctx, QP_ERR_INVALID_ARG, "no search has run on this context");
+    if (capacity < ctx->last_steps + 1) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "curve buffer");
+    qp_device_guard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    cudaError_t e = cudaMemcpyAsync(h_curve, ctx->d_curve, sizeof(double) * (ctx->last_steps + 1),
+                                    cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_dsaciq_curve: %s", cudaGetErrorString(e));
+        return QP_ERR_CUDA;
+    }
+    return QP_OK;
+}
+
+static int32_t resolve_qp(qp_ctx* ctx, const qp_qparams_t* qp, int qp_on_device, int bits, const qp_qparams_t** d_qp,
+                          qp_qparams_t* h_qp)
+{
+    if (!qp) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null qparams");
+    memset(h_qp, 0, sizeof *h_qp);
+    if (qp_on_device) {
+        if ((uintptr_t)qp & 3u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "device qparams");
+        *d_qp = qp;
+    } else {
+        *d_qp = nullptr;
+        *h_qp = *qp;
+        if (h_qp->bits != bits) return qp_fail(ctx, QP_ERR_INVALID_ARG, "qparams were made for another bit-width");
+    }
+    return QP_OK;
+}
+
+extern "C" int32_t qp_quantize_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits,
+                                    const qp_qparams_t* qp, int qp_on_device, void* d_packed,
+                                    uint64_t packed_capacity, void* stream)
+{
+    int32_t rc = check_x(ctx, d_x, dtype, n);
+    if (rc) return rc;
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    const uint64_t need = qp_packed_bytes(n, bits);
+    if (packed_capacity < need) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
+    if (need > 0 && !d_packed) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_packed");
+    if ((uintptr_t)d_packed & 15u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_packed must be 16-byte aligned");
+    const qp_qparams_t* d_qp;
+    qp_qparams_t h_qp;
+    rc = resolve_qp(ctx, qp, qp_on_device, bits, &d_qp, &h_qp);
+    if (rc) return rc;
+    if (n == 0) return QP_OK;
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    return qp_launch_pack(ctx, d_x, dtype, n, bits, d_qp, h_qp, d_packed, static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t qp_unpack_dequantize(qp_ctx* ctx, const void* d_packed, uint64_t n, int bits,
+                                        const qp_qparams_t* qp, int qp_on_device, void* d_y, int out_dtype,
+                                        void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (out_dtype != QP_F32 && out_dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "out_dtype");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (n >= (1ull << 40)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "n too large");
+    if (n > 0 && (!d_packed || !d_y)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null buffer");
+    if ((uintptr_t)d_packed & 15u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_packed must be 16-byte aligned");
+    if ((uintptr_t)d_y & (out_dtype == QP_F32 ? 3u : 1u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_y");
+    const qp_qparams_t* d_qp;
+    qp_qparams_t h_qp;
+    int32_t rc = resolve_qp(ctx, qp, qp_on_device, bits, &d_qp, &h_qp);
+    if (rc) return rc;
+    if (n == 0) return QP_OK;
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    return qp_launch_unpack(ctx, d_packed, n, bits, d_qp, h_qp, d_y, out_dtype, static_cast<cudaStream_t>(stream));
+}

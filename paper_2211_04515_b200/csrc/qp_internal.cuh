@@ -1,0 +1,202 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdio.h>
+
+#include "quantpipe.h"
+
+// ------------------------------------------------------------------ context
+
+constexpr int QP_THREADS = 256;          // block size of the streaming kernels
+constexpr int QP_MAX_BLOCKS = 4096;      // upper bound on blocks that write partials
+constexpr int QP_EVAL_K = 8;             // candidates scored per thread in one pass
+
+struct qp_stats_partial {                // one per block, written by the two statistics passes
+    double s0, s1;                       // pass A: sum x, sum |x|;  pass B: sum |x-mean|, sum (x-mean)^2
+    double mn, mx;
+    unsigned long long bad;
+    unsigned long long pad;
+};
+
+struct qp_ds_setup {                     // written by the search's set-up kernel
+    double b_e, b_r, F, mean;
+    unsigned long long n_finite;
+    int degenerate;
+    int pad;
+};
+
+struct qp_ctx {
+    int device;
+    int sm_count;
+    void* d_base;                        // single allocation, carved below
+    qp_stats_partial* d_part;            // [QP_MAX_BLOCKS]
+    unsigned long long* d_hist;          // [QP_MAX_HIST_BINS]
+    float4* d_cand;                      // [QP_MAX_STEPS + 1]  (lo, hi, scale, inv_scale)
+    int* d_valid;                        // [QP_MAX_STEPS + 1]
+    double* d_sums;                      // [QP_MAX_BLOCKS * QP_EVAL_K] block partial error sums
+    double* d_curve;                     // [QP_MAX_STEPS + 1]  MSE per candidate
+    qp_ds_setup* d_setup;
+    unsigned int* d_ticket;              // [4] last-block tickets (always left at 0)
+    unsigned int* d_status;              // device status word
+    int last_steps;                      // steps of the last search (for qp_dsaciq_curve)
+    char err[256];
+};
+
+int32_t qp_fail(qp_ctx* ctx, int32_t status, const char* what);
+int32_t qp_check_launch(qp_ctx* ctx, const char* what);
+
+struct qp_device_guard {                 // makes ctx->device current for the scope
+    int prev;
+    bool ok;
+    explicit qp_device_guard(int dev) : prev(-1), ok(true)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~qp_device_guard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Shared host arithmetic (one definition each, in qp_api.cu).
+double qp_host_aciq_F(int bits, int dist);
+static inline bool qp_bits_ok(int bits) { return (bits >= 1 && bits <= 8) || bits == 16; }
+
+// ------------------------------------------------------------- device helpers
+#ifdef __CUDACC__
+
+// Quantizer set-up from a clip range, same on host and device: ends rounded to fp32, scale
+// and reciprocal from the rounded ends in fp64, rounded once.
+__host__ __device__ inline int qp_fill_qparams(double lo, double hi, int bits, qp_qparams_t* q)
+{
+    const double levels_m1 = (double)((1u << bits) - 1u);
+    const float lo_f = (float)lo, hi_f = (float)hi;
+    q->lo = lo_f;
+    q->hi = hi_f;
+    q->bits = bits;
+    q->flags = 0;
+    const bool finite = (lo_f - lo_f == 0.0f) && (hi_f - hi_f == 0.0f);
+    if (!(hi_f > lo_f) || !finite) {
+        q->scale = 0.0f;
+        q->inv_scale = 0.0f;
+        q->flags = 1;
+        return QP_WARN_DEGENERATE;
+    }
+    const double range = (double)hi_f - (double)lo_f;
+    q->scale = (float)(range / levels_m1);
+    q->inv_scale = (float)(levels_m1 / range);
+    return QP_OK;
+}
+
+constexpr float QP_MAGIC = 12582912.0f;         // 1.5 * 2^23: adding it rounds to an integer, ties to even
+constexpr unsigned QP_MAGIC_BITS = 0x4B400000u;
+
+// Position of x on the level grid: clamp (NaN -> lo), subtract, scale; each op rounded to fp32.
+__device__ __forceinline__ float qp_grid_pos(float x, float lo, float hi, float inv_scale)
+{
+    const float t = fminf(fmaxf(x, lo), hi);
+    return __fmul_rn(__fsub_rn(t, lo), inv_scale);
+}
+
+// Code of x as the low bits of (pos + 1.5*2^23): for 0 <= pos < 2^22 the float addition
+// rounds pos to the nearest integer, ties to even, and leaves it in the low mantissa bits.
+__device__ __forceinline__ unsigned qp_code(float x, float lo, float hi, float inv_scale, unsigned mask)
+{
+    return __float_as_uint(__fadd_rn(qp_grid_pos(x, lo, hi, inv_scale), QP_MAGIC)) & mask;
+}
+
+__device__ __forceinline__ float qp_bf16_to_f32(unsigned short h) { return __uint_as_float((unsigned)h << 16); }
+
+__device__ __forceinline__ unsigned short qp_f32_to_bf16(float f)   // round to nearest even
+{
+    unsigned u = __float_as_uint(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) return (unsigned short)((u >> 16) | 0x0040u);
+    return (unsigned short)((u + 0x7FFFu + ((u >> 16) & 1u)) >> 16);
+}
+
+__device__ __forceinline__ bool qp_is_finite(float x) { return fabsf(x) < __int_as_float(0x7F800000); }
+
+// A contiguous array seen as [head scalars][nvec aligned 16-byte vectors][tail scalars].
+template <typename T>
+struct qp_span {
+    uint64_t head, nvec, tail;
+    static constexpr int EPV = 16 / sizeof(T);
+    __host__ __device__ qp_span(const T* p, uint64_t n)
+    {
+        const uint64_t mis = ((uintptr_t)p & 15u) / sizeof(T);
+        head = mis ? (EPV - mis) : 0;
+        if (head > n) head = n;
+        nvec = (n - head) / EPV;
+        tail = n - head - nvec * EPV;
+    }
+};
+
+// Load one 16-byte vector of T as EPV floats.
+__device__ __forceinline__ void qp_load_vec(const float* p, float (&v)[4])
+{
+    const float4 a = __ldg(reinterpret_cast<const float4*>(p));
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+}
+__device__ __forceinline__ void qp_load_vec(const unsigned short* p, float (&v)[8])
+{
+    const uint4 a = __ldg(reinterpret_cast<const uint4*>(p));
+    v[0] = __uint_as_float(a.x << 16); v[1] = __uint_as_float(a.x & 0xFFFF0000u);
+    v[2] = __uint_as_float(a.y << 16); v[3] = __uint_as_float(a.y & 0xFFFF0000u);
+    v[4] = __uint_as_float(a.z << 16); v[5] = __uint_as_float(a.z & 0xFFFF0000u);
+    v[6] = __uint_as_float(a.w << 16); v[7] = __uint_as_float(a.w & 0xFFFF0000u);
+}
+__device__ __forceinline__ float qp_load_one(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float qp_load_one(const unsigned short* p) { return qp_bf16_to_f32(__ldg(p)); }
+
+// Deterministic block-wide sum of a double (result valid in thread 0).  `sh` holds one
+// double per warp.
+__device__ __forceinline__ double qp_block_sum(double v, double* sh)
+{
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xFFFFFFFFu, v, o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    double r = 0.0;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < nwarp; ++w) r += sh[w];
+    return r;
+}
+__device__ __forceinline__ double qp_block_min(double v, double* sh)
+{
+    for (int o = 16; o > 0; o >>= 1) v = fmin(v, __shfl_down_sync(0xFFFFFFFFu, v, o));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    double r = v;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < nwarp; ++w) r = fmin(r, sh[w]);
+    return r;
+}
+__device__ __forceinline__ double qp_block_max(double v, double* sh)
+{
+    for (int o = 16; o > 0; o >>= 1) v = fmax(v, __shfl_down_sync(0xFFFFFFFFu, v, o));
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarp = (blockDim.x + 31) >> 5;
+    __syncthreads();
+    if (lane == 0) sh[warp] = v;
+    __syncthreads();
+    double r = v;
+    if (threadIdx.x == 0)
+        for (int w = 0; w < nwarp; ++w) r = fmax(r, sh[w]);
+    return r;
+}
+
+#endif  // __CUDACC__
+
+// Kernel launchers (one per translation unit).
+int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, cudaStream_t s);
+int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats, int bits,
+                         int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
+                         qp_qparams_t* d_qp_out, cudaStream_t s);
+int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
+                              qp_qparams_t* d_qp_out, cudaStream_t s);
+int32_t qp_launch_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, const qp_qparams_t* d_qp,
+                       qp_qparams_t h_qp, void* d_packed, cudaStream_t s);
+int32_t qp_launch_unpack(qp_ctx* ctx, const void* d_packed, uint64_t n, int bits, const qp_qparams_t* d_qp,
+                         qp_qparams_t h_qp, void* d_y, int out_dtype, cudaStream_t s);

@@ -1,0 +1,352 @@
+// a2 + a3 + a4: histogram peak, ACIQ clip on the device, and the directed search DS-ACIQ
+// (paper Sec. 3 "Directed Search", Eq. 1).
+//
+//   hist      count histogram of x over [min, max] in shared memory (lane-replicated
+//             counters, no same-address contention), merged into global 64-bit counters
+//   setup     peak -> b_R, the steps+1 candidate scales b_k and their quantizers
+//   eval      every thread scores QP_EVAL_K candidates against each element it loads and
+//             keeps K error sums (fp32 over 8 elements, then fp64); blockIdx.x picks the
+//             candidate group, groups of the same chunk of x run next to each other so x
+//             is fetched from HBM once and re-read from L2; the kernel is bound by fp32
+//             ALU throughput, not by memory
+//   finalize  fixed-order merge of the block sums, MSE per candidate, first minimum wins
+#include "qp_internal.cuh"
+
+namespace {
+
+constexpr int K = QP_EVAL_K;
+
+// -------------------------------------------------------------------- histogram
+
+template <typename T, bool GUARD>
+__device__ __forceinline__ void hist_body(const T* __restrict__ x, uint64_t n, float mn, float inv_w, int nb, int rep_mask,
+                                          int rep_shift, unsigned* __restrict__ sh)
+{
+    constexpr int EPV = qp_span<T>::EPV;
+    const qp_span<T> sp(x, n);
+    const T* xv = x + sp.head;
+    const uint64_t stride = (uint64_t)gridDim.x * QP_THREADS;
+    const int lane_rep = threadIdx.x & rep_mask;
+    auto one = [&](float e) {
+        if (GUARD && !qp_is_finite(e)) return;
+        // bin = floor((x - min) * inv_w), the last bin closed; fp32, each op rounded once
+        int b = __float2int_rz(__fmul_rn(__fsub_rn(e, mn), inv_w));
+        b = min(max(b, 0), nb - 1);
+        atomicAdd(&sh[(b << rep_shift) + lane_rep], 1u);
+    };
+    for (uint64_t v = (uint64_t)blockIdx.x * QP_THREADS + threadIdx.x; v < sp.nvec; v += 2 * stride) {
+        float e0[EPV], e1[EPV];
+        const bool two = v + stride < sp.nvec;
+        qp_load_vec(xv + v * EPV, e0);
+        if (two) qp_load_vec(xv + (v + stride) * EPV, e1);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) one(e0[i]);
+        if (two) {
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) one(e1[i]);
+        }
+    }
+    if (blockIdx.x == 0) {
+        for (uint64_t i = threadIdx.x; i < sp.head; i += QP_THREADS) one(qp_load_one(x + i));
+        const uint64_t t0 = sp.head + sp.nvec * EPV;
+        for (uint64_t i = threadIdx.x; i < sp.tail; i += QP_THREADS) one(qp_load_one(x + t0 + i));
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(QP_THREADS) hist_kernel(const T* __restrict__ x, uint64_t n,
+                                                          const qp_stats_t* __restrict__ st, int nb, int rep_shift,
+                                                          unsigned long long* __restrict__ hist)
+{
+    extern __shared__ unsigned sh[];
+    const int reps = 1 << rep_shift;
+    for (int i = threadIdx.x; i < nb * reps; i += QP_THREADS) sh[i] = 0u;
+    __syncthreads();
+    const double mn = st->min, mx = st->max;
+    if (mx > mn) {
+        const float inv_w = (float)((double)nb / (mx - mn));
+        if (st->nonfinite == 0) hist_body<T, false>(x, n, (float)mn, inv_w, nb, reps - 1, rep_shift, sh);
+        else                    hist_body<T, true>(x, n, (float)mn, inv_w, nb, reps - 1, rep_shift, sh);
+    }
+    __syncthreads();
+    for (int b = threadIdx.x; b < nb; b += QP_THREADS) {
+        unsigned long long c = 0;
+        for (int r = 0; r < reps; ++r) c += sh[(b << rep_shift) + ((r + threadIdx.x) & (reps - 1))];
+        if (c) atomicAdd(&hist[b], c);
+    }
+}
+
+// ------------------------------------------------------------------------ setup
+
+__global__ void __launch_bounds__(QP_THREADS) setup_kernel(const qp_stats_t* __restrict__ st,
+                                                           const unsigned long long* __restrict__ hist, int nb, int bits,
+                                                           int bmode, int steps, double F, float4* __restrict__ cand,
+                                                           int* __restrict__ valid, qp_ds_setup* __restrict__ setup)
+{
+    __shared__ unsigned long long sh_top[QP_THREADS];
+    __shared__ qp_ds_setup s;
+    unsigned long long top = 0;
+    for (int b = threadIdx.x; b < nb; b += QP_THREADS) {
+        const unsigned long long c = hist[b];
+        top = c > top ? c : top;
+    }
+    sh_top[threadIdx.x] = top;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int i = 1; i < QP_THREADS; ++i) top = sh_top[i] > top ? sh_top[i] : top;
+        const unsigned long long nf = st->n - st->nonfinite;
+        const double mn = st->min, mx = st->max;
+        const double b_e = bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad;
+        double peak = 0.0;
+        if (mx > mn && nf > 0) {
+            const double w = (mx - mn) / (double)nb;
+            peak = (double)top / ((double)nf * w);
+        }
+        s.degenerate = !(mx > mn) || !(peak > 0.0) || !(b_e > 0.0);
+        s.b_e = b_e;
+        s.b_r = s.degenerate ? b_e : 1.0 / (2.0 * peak);
+        s.F = F;
+        s.mean = st->mean;
+        s.n_finite = nf;
+        s.pad = 0;
+        *setup = s;
+    }
+    __syncthreads();
+    for (int k = threadIdx.x; k <= steps; k += QP_THREADS) {
+        // b_k = b_E + k (b_R - b_E) / steps, evaluated in this order in fp64
+        const double b_k = s.b_e + (double)k * (s.b_r - s.b_e) / (double)steps;
+        const bool ok = (k == 0) || (!s.degenerate && b_k > 0.0);
+        qp_qparams_t q;
+        q.lo = q.hi = q.scale = q.inv_scale = 0.f;
+        if (ok) {
+            const double alpha = s.F * b_k;
+            qp_fill_qparams(s.mean - alpha, s.mean + alpha, bits, &q);
+        }
+        cand[k] = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
+        valid[k] = ok ? 1 : 0;
+    }
+}
+
+// ------------------------------------------------------------------------- eval
+
+template <bool GUARD, int NE>
+__device__ __forceinline__ void score(const float (&e)[NE], const float (&lo)[K], const float (&hi)[K],
+                                      const float (&sc)[K], const float (&iv)[K], double (&acc)[K])
+{
+    float p[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) p[k] = 0.f;
+#pragma unroll
+    for (int i = 0; i < NE; ++i) {
+        const float x = e[i];
+        const bool fin = !GUARD || qp_is_finite(x);
+#pragma unroll
+        for (int k = 0; k < K; ++k) {
+            // level index as a float: (pos + 1.5*2^23) - 1.5*2^23 rounds to nearest, ties to even
+            const float pos = qp_grid_pos(x, lo[k], hi[k], iv[k]);
+            const float r = __fsub_rn(__fadd_rn(pos, QP_MAGIC), QP_MAGIC);
+            const float d = __fsub_rn(fmaf(r, sc[k], lo[k]), x);
+            if (GUARD) { if (fin) p[k] = fmaf(d, d, p[k]); }
+            else       p[k] = fmaf(d, d, p[k]);
+        }
+    }
+#pragma unroll
+    for (int k = 0; k < K; ++k) acc[k] += (double)p[k];
+}
+
+template <typename T, bool GUARD>
+__device__ __forceinline__ void eval_body(const T* __restrict__ x, uint64_t n, unsigned chunk, unsigned chunks,
+                                          const float (&lo)[K], const float (&hi)[K], const float (&sc)[K],
+                                          const float (&iv)[K], double (&acc)[K])
+{
+    constexpr int EPV = qp_span<T>::EPV;
+    constexpr int NV = 8 / EPV;                       // 8 elements per scoring round
+    const qp_span<T> sp(x, n);
+    const T* xv = x + sp.head;
+    const uint64_t stride = (uint64_t)chunks * QP_THREADS;
+    uint64_t v = (uint64_t)chunk * QP_THREADS + threadIdx.x;
+    for (; v + (NV - 1) * stride < sp.nvec; v += NV * stride) {
+        float e[8];
+        if (NV == 2) {
+            float a[EPV], b[EPV];
+            qp_load_vec(xv + v * EPV, a);
+            qp_load_vec(xv + (v + stride) * EPV, b);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) { e[i] = a[i]; e[EPV + i] = b[i]; }
+        } else {
+            float a[EPV];
+            qp_load_vec(xv + v * EPV, a);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) e[i] = a[i];
+        }
+        score<GUARD, 8>(e, lo, hi, sc, iv, acc);
+    }
+    for (; v < sp.nvec; v += stride) {
+        float a[EPV];
+        qp_load_vec(xv + v * EPV, a);
+        score<GUARD, EPV>(a, lo, hi, sc, iv, acc);
+    }
+    if (chunk == 0) {
+        for (uint64_t i = threadIdx.x; i < sp.head; i += QP_THREADS) {
+            const float a[1] = {qp_load_one(x + i)};
+            score<GUARD, 1>(a, lo, hi, sc, iv, acc);
+        }
+        const uint64_t t0 = sp.head + sp.nvec * EPV;
+        for (uint64_t i = threadIdx.x; i < sp.tail; i += QP_THREADS) {
+            const float a[1] = {qp_load_one(x + t0 + i)};
+            score<GUARD, 1>(a, lo, hi, sc, iv, acc);
+        }
+    }
+}
+
+// grid = (groups, chunks): the candidate group is the fastest-varying block index, so the
+// groups of one chunk are scheduled together and share its lines in L2.
+template <typename T>
+__global__ void __launch_bounds__(QP_THREADS) eval_kernel(const T* __restrict__ x, uint64_t n,
+                                                          const qp_stats_t* __restrict__ st,
+                                                          const float4* __restrict__ cand, int ncand,
+                                                          double* __restrict__ sums)
+{
+    const int g = blockIdx.x;
+    const unsigned chunk = blockIdx.y, chunks = gridDim.y;
+    float lo[K], hi[K], sc[K], iv[K];
+    double acc[K];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const int c = min(g * K + k, ncand - 1);
+        const float4 q = cand[c];
+        lo[k] = q.x; hi[k] = q.y; sc[k] = q.z; iv[k] = q.w;
+        acc[k] = 0.0;
+    }
+    if (st->nonfinite == 0) eval_body<T, false>(x, n, chunk, chunks, lo, hi, sc, iv, acc);
+    else                    eval_body<T, true>(x, n, chunk, chunks, lo, hi, sc, iv, acc);
+
+    __shared__ double sh[QP_THREADS / 32];
+#pragma unroll
+    for (int k = 0; k < K; ++k) {
+        const double t = qp_block_sum(acc[k], sh);
+        if (threadIdx.x == 0) sums[((size_t)g * chunks + chunk) * K + k] = t;
+    }
+}
+
+// --------------------------------------------------------------------- finalize
+
+__global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __restrict__ sums, int chunks, int steps,
+                                                              int nb, int bits, const int* __restrict__ valid,
+                                                              const float4* __restrict__ cand,
+                                                              const qp_ds_setup* __restrict__ setup,
+                                                              double* __restrict__ curve, qp_ds_result_t* __restrict__ out,
+                                                              qp_qparams_t* __restrict__ qp_out,
+                                                              unsigned* __restrict__ status)
+{
+    const qp_ds_setup s = *setup;
+    for (int k = threadIdx.x; k <= steps; k += QP_THREADS) {
+        const int g = k / K, j = k % K;
+        double t = 0.0;
+        for (int b = 0; b < chunks; ++b) t += sums[((size_t)g * chunks + b) * K + j];
+        double mse = s.n_finite ? t / (double)s.n_finite : 0.0;
+        if (!valid[k]) mse = __longlong_as_double(0x7FF0000000000000ll);
+        curve[k] = mse;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int best = 0;
+        double best_mse = curve[0];
+        for (int k = 1; k <= steps; ++k)
+            if (curve[k] < best_mse) { best_mse = curve[k]; best = k; }
+        const double b_star = s.b_e + (double)best * (s.b_r - s.b_e) / (double)steps;
+        if (out) {
+            out->b_e = s.b_e;
+            out->b_r = s.b_r;
+            out->b_star = b_star;
+            out->alpha_e = s.F * s.b_e;
+            out->alpha_star = s.F * b_star;
+            out->mse_e = curve[0];
+            out->mse_star = best_mse;
+            out->k_star = best;
+            out->steps = steps;
+            out->hist_bins = nb;
+            out->bits = bits;
+        }
+        const float4 c = cand[best];
+        const bool degenerate_q = !(c.y > c.x);
+        if (qp_out) {
+            qp_out->lo = c.x; qp_out->hi = c.y; qp_out->scale = c.z; qp_out->inv_scale = c.w;
+            qp_out->bits = bits;
+            qp_out->flags = degenerate_q ? 1 : 0;
+        }
+        if (s.degenerate || degenerate_q) atomicOr(status, QP_DEV_DEGENERATE);
+    }
+}
+
+// one thread: ACIQ clip from device-resident statistics
+__global__ void aciq_kernel(const qp_stats_t* __restrict__ st, int bits, int dist, int bmode, double F,
+                            qp_qparams_t* __restrict__ qp_out, unsigned* __restrict__ status)
+{
+    if (threadIdx.x != 0 || blockIdx.x != 0) return;
+    const double b = dist == QP_DIST_GAUSS ? sqrt(st->var) : (bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad);
+    const double alpha = F * b;
+    qp_qparams_t q;
+    const int rc = qp_fill_qparams(st->mean - alpha, st->mean + alpha, bits, &q);
+    *qp_out = q;
+    if (rc == QP_WARN_DEGENERATE) atomicOr(status, QP_DEV_DEGENERATE);
+}
+
+template <typename T>
+int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_stats, int bits, int bmode, int steps,
+                     int nb, double F, qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, cudaStream_t s)
+{
+    // histogram: as many lane replicas of each bin as fit in 64 KB of shared memory
+    int rep_shift = 5;
+    while (rep_shift > 0 && ((size_t)nb << rep_shift) * sizeof(unsigned) > 64 * 1024) --rep_shift;
+    const size_t sh_bytes = ((size_t)nb << rep_shift) * sizeof(unsigned);
+    static bool attr_set[2] = {false, false};
+    const int ti = sizeof(T) == 4 ? 0 : 1;
+    if (!attr_set[ti]) {
+        if (cudaFuncSetAttribute(hist_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
+            return qp_check_launch(ctx, "qp_dsaciq_search (histogram attribute)");
+        attr_set[ti] = true;
+    }
+    const uint64_t per_block = (uint64_t)QP_THREADS * 2 * qp_span<T>::EPV;
+    uint64_t want = (n + per_block - 1) / per_block;
+    const uint64_t hcap = (uint64_t)ctx->sm_count * 3;
+    const int hblocks = (int)(want < 1 ? 1 : (want > hcap ? hcap : want));
+    if (cudaMemsetAsync(ctx->d_hist, 0, sizeof(unsigned long long) * nb, s) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_dsaciq_search (histogram reset)");
+    hist_kernel<T><<<hblocks, QP_THREADS, sh_bytes, s>>>(x, n, d_stats, nb, rep_shift, ctx->d_hist);
+    setup_kernel<<<1, QP_THREADS, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
+                                          ctx->d_setup);
+
+    const int ncand = steps + 1;
+    const int groups = (ncand + K - 1) / K;
+    const uint64_t per_chunk = (uint64_t)QP_THREADS * 8;
+    want = (n + per_chunk - 1) / per_chunk;
+    uint64_t ccap = (uint64_t)ctx->sm_count * 4 / (uint64_t)groups;     // about 4 resident blocks per SM in all
+    if (ccap < 1) ccap = 1;
+    if (ccap * groups > QP_MAX_BLOCKS) ccap = QP_MAX_BLOCKS / groups;
+    const int chunks = (int)(want < 1 ? 1 : (want > ccap ? ccap : want));
+    eval_kernel<T><<<dim3(groups, chunks), QP_THREADS, 0, s>>>(x, n, d_stats, ctx->d_cand, ncand, ctx->d_sums);
+    finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, chunks, steps, nb, bits, ctx->d_valid, ctx->d_cand,
+                                             ctx->d_setup, ctx->d_curve, d_out, d_qp_out, ctx->d_status);
+    return qp_check_launch(ctx, "qp_dsaciq_search");
+}
+
+}  // namespace
+
+int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats, int bits,
+                         int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out, qp_qparams_t* d_qp_out,
+                         cudaStream_t s)
+{
+    if (dtype == QP_F32)
+        return search_typed<float>(ctx, static_cast<const float*>(d_x), n, d_stats, bits, bmode, steps, hist_bins, F,
+                                   d_out, d_qp_out, s);
+    return search_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_stats, bits, bmode, steps,
+                                        hist_bins, F, d_out, d_qp_out, s);
+}
+
+int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
+                              qp_qparams_t* d_qp_out, cudaStream_t s)
+{
+    aciq_kernel<<<1, 32, 0, s>>>(d_stats, bits, dist, bmode, F, d_qp_out, ctx->d_status);
+    return qp_check_launch(ctx, "qp_aciq_qparams_device");
+}

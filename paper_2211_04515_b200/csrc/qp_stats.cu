@@ -1,0 +1,246 @@
+// a1: per-tensor statistics (paper Sec. 3: min/max, mean, Laplace scale).
+//
+// Two streaming passes, both HBM-bound (the second one is served from L2 for tensors that
+// fit there):
+//   pass A  sum x, sum |x|, min, max, non-finite count            -> mean, mean_abs, min, max
+//   pass B  sum |x - mean|, sum (x - mean)^2                      -> mad, var
+// Each thread keeps fp32 partial sums over a run of 16 (f32) or 32 (bf16) elements and
+// folds them into fp64; blocks write fp64 partials; the last block to finish (ticket
+// counter, no waiting) merges all partials in index order, so results do not depend on
+// block scheduling.
+#include "qp_internal.cuh"
+
+namespace {
+
+constexpr int UNROLL = 4;   // 16-byte loads in flight per thread
+
+struct AccA {
+    double s, sa, mn, mx;
+    unsigned long long bad;
+    __device__ void add_scalar(float v)
+    {
+        if (qp_is_finite(v)) {
+            s += (double)v;
+            sa += (double)fabsf(v);
+            mn = fmin(mn, (double)v);
+            mx = fmax(mx, (double)v);
+        } else {
+            ++bad;
+        }
+    }
+};
+
+template <typename T>
+__global__ void __launch_bounds__(QP_THREADS) stats_pass_a(const T* __restrict__ x, uint64_t n,
+                                                           qp_stats_partial* __restrict__ part,
+                                                           unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out,
+                                                           unsigned* __restrict__ status)
+{
+    constexpr int EPV = qp_span<T>::EPV;
+    const qp_span<T> sp(x, n);
+    const T* xv = x + sp.head;
+    const float inf = __int_as_float(0x7F800000);
+
+    AccA acc = {0.0, 0.0, (double)inf, (double)-inf, 0ull};
+    const uint64_t stride = (uint64_t)gridDim.x * QP_THREADS;
+    uint64_t v = (uint64_t)blockIdx.x * QP_THREADS + threadIdx.x;
+
+    for (; v + (UNROLL - 1) * stride < sp.nvec; v += UNROLL * stride) {
+        float e[UNROLL][EPV];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) qp_load_vec(xv + (v + u * stride) * EPV, e[u]);
+        float s = 0.f, sa = 0.f, mn = inf, mx = -inf;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                s += e[u][i];
+                sa += fabsf(e[u][i]);
+                mn = fminf(mn, e[u][i]);
+                mx = fmaxf(mx, e[u][i]);
+            }
+        if (sa < inf) {                       // every element finite (and no fp32 overflow)
+            acc.s += (double)s;
+            acc.sa += (double)sa;
+            acc.mn = fmin(acc.mn, (double)mn);
+            acc.mx = fmax(acc.mx, (double)mx);
+        } else {
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+                for (int i = 0; i < EPV; ++i) acc.add_scalar(e[u][i]);
+        }
+    }
+    for (; v < sp.nvec; v += stride) {
+        float e[EPV];
+        qp_load_vec(xv + v * EPV, e);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) acc.add_scalar(e[i]);
+    }
+    if (blockIdx.x == 0) {                    // unaligned head and ragged tail
+        for (uint64_t i = threadIdx.x; i < sp.head; i += QP_THREADS) acc.add_scalar(qp_load_one(x + i));
+        const uint64_t t0 = sp.head + sp.nvec * EPV;
+        for (uint64_t i = threadIdx.x; i < sp.tail; i += QP_THREADS) acc.add_scalar(qp_load_one(x + t0 + i));
+    }
+
+    __shared__ double sh[QP_THREADS / 32];
+    __shared__ bool last;
+    const double bs = qp_block_sum(acc.s, sh);
+    const double bsa = qp_block_sum(acc.sa, sh);
+    const double bmn = qp_block_min(acc.mn, sh);
+    const double bmx = qp_block_max(acc.mx, sh);
+    const double bbad = qp_block_sum((double)acc.bad, sh);   // exact: counts are far below 2^53
+    if (threadIdx.x == 0) {
+        qp_stats_partial p;
+        p.s0 = bs; p.s1 = bsa; p.mn = bmn; p.mx = bmx; p.bad = (unsigned long long)bbad; p.pad = 0;
+        part[blockIdx.x] = p;
+        __threadfence();
+        last = (atomicAdd(&ticket[0], 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+
+    double s = 0.0, sa = 0.0, mn = (double)inf, mx = (double)-inf, bad = 0.0;
+    for (unsigned b = threadIdx.x; b < gridDim.x; b += QP_THREADS) {
+        s += __ldcg(&part[b].s0);
+        sa += __ldcg(&part[b].s1);
+        mn = fmin(mn, __ldcg(&part[b].mn));
+        mx = fmax(mx, __ldcg(&part[b].mx));
+        bad += (double)__ldcg(&part[b].bad);
+    }
+    s = qp_block_sum(s, sh);
+    sa = qp_block_sum(sa, sh);
+    mn = qp_block_min(mn, sh);
+    mx = qp_block_max(mx, sh);
+    bad = qp_block_sum(bad, sh);
+    if (threadIdx.x == 0) {
+        const unsigned long long nbad = (unsigned long long)bad;
+        const unsigned long long nf = n - nbad;
+        out->n = n;
+        out->nonfinite = nbad;
+        out->mean = nf ? s / (double)nf : 0.0;
+        out->mean_abs = nf ? sa / (double)nf : 0.0;
+        out->min = nf ? mn : 0.0;
+        out->max = nf ? mx : 0.0;
+        out->mad = 0.0;
+        out->var = 0.0;
+        if (nbad) atomicOr(status, QP_DEV_NONFINITE);
+        ticket[0] = 0;
+    }
+}
+
+template <typename T, bool GUARD>
+__device__ __forceinline__ void pass_b_body(const T* __restrict__ x, uint64_t n, float m_hi, float m_lo, double& sd,
+                                            double& sv)
+{
+    constexpr int EPV = qp_span<T>::EPV;
+    const qp_span<T> sp(x, n);
+    const T* xv = x + sp.head;
+    const uint64_t stride = (uint64_t)gridDim.x * QP_THREADS;
+    uint64_t v = (uint64_t)blockIdx.x * QP_THREADS + threadIdx.x;
+
+    auto one = [&](float e, float& d1, float& d2) {
+        // x - mean with the mean held as an unevaluated fp32 pair
+        const float d = __fsub_rn(__fsub_rn(e, m_hi), m_lo);
+        if (!GUARD || qp_is_finite(e)) {
+            d1 += fabsf(d);
+            d2 = fmaf(d, d, d2);
+        }
+    };
+    for (; v + (UNROLL - 1) * stride < sp.nvec; v += UNROLL * stride) {
+        float e[UNROLL][EPV];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) qp_load_vec(xv + (v + u * stride) * EPV, e[u]);
+        float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u)
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) one(e[u][i], d1, d2);
+        sd += (double)d1;
+        sv += (double)d2;
+    }
+    for (; v < sp.nvec; v += stride) {
+        float e[EPV];
+        qp_load_vec(xv + v * EPV, e);
+        float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) one(e[i], d1, d2);
+        sd += (double)d1;
+        sv += (double)d2;
+    }
+    if (blockIdx.x == 0) {
+        float d1 = 0.f, d2 = 0.f;
+        for (uint64_t i = threadIdx.x; i < sp.head; i += QP_THREADS) one(qp_load_one(x + i), d1, d2);
+        const uint64_t t0 = sp.head + sp.nvec * EPV;
+        for (uint64_t i = threadIdx.x; i < sp.tail; i += QP_THREADS) one(qp_load_one(x + t0 + i), d1, d2);
+        sd += (double)d1;
+        sv += (double)d2;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(QP_THREADS) stats_pass_b(const T* __restrict__ x, uint64_t n,
+                                                           qp_stats_partial* __restrict__ part,
+                                                           unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out)
+{
+    const double mean = out->mean;
+    const unsigned long long nbad = out->nonfinite;
+    const float m_hi = (float)mean;
+    const float m_lo = (float)(mean - (double)m_hi);
+    double sd = 0.0, sv = 0.0;
+    if (nbad == 0) pass_b_body<T, false>(x, n, m_hi, m_lo, sd, sv);
+    else           pass_b_body<T, true>(x, n, m_hi, m_lo, sd, sv);
+
+    __shared__ double sh[QP_THREADS / 32];
+    __shared__ bool last;
+    const double bsd = qp_block_sum(sd, sh);
+    const double bsv = qp_block_sum(sv, sh);
+    if (threadIdx.x == 0) {
+        part[blockIdx.x].s0 = bsd;
+        part[blockIdx.x].s1 = bsv;
+        __threadfence();
+        last = (atomicAdd(&ticket[1], 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    double a = 0.0, b = 0.0;
+    for (unsigned k = threadIdx.x; k < gridDim.x; k += QP_THREADS) {
+        a += __ldcg(&part[k].s0);
+        b += __ldcg(&part[k].s1);
+    }
+    a = qp_block_sum(a, sh);
+    b = qp_block_sum(b, sh);
+    if (threadIdx.x == 0) {
+        const unsigned long long nf = n - nbad;
+        out->mad = nf ? a / (double)nf : 0.0;
+        out->var = nf ? b / (double)nf : 0.0;
+        ticket[1] = 0;
+    }
+}
+
+template <typename T>
+int32_t launch_typed(qp_ctx* ctx, const T* x, uint64_t n, qp_stats_t* d_out, cudaStream_t s)
+{
+    const uint64_t per_block = (uint64_t)QP_THREADS * UNROLL * qp_span<T>::EPV;
+    uint64_t want = (n + per_block - 1) / per_block;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
+    int blocks = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+    if (blocks > QP_MAX_BLOCKS) blocks = QP_MAX_BLOCKS;
+    stats_pass_a<T><<<blocks, QP_THREADS, 0, s>>>(x, n, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
+    stats_pass_b<T><<<blocks, QP_THREADS, 0, s>>>(x, n, ctx->d_part, ctx->d_ticket, d_out);
+    return qp_check_launch(ctx, "qp_stats");
+}
+
+}  // namespace
+
+int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, cudaStream_t s)
+{
+    if (n == 0) {
+        if (cudaMemsetAsync(d_out, 0, sizeof(qp_stats_t), s) != cudaSuccess) return qp_check_launch(ctx, "qp_stats");
+        return QP_OK;
+    }
+    if (dtype == QP_F32) return launch_typed<float>(ctx, static_cast<const float*>(d_x), n, d_out, s);
+    return launch_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_out, s);
+}

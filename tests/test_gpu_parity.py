@@ -1,0 +1,417 @@
+"""GPU parity: the CUDA library, called through its C ABI, against the CPU oracle on the same
+seeded inputs.
+
+Tolerances (the targets this library is built to):
+  statistics      1e-5 relative   (mean: relative to max(|mean|, mad), since the mean of a
+                                   centred tensor is near zero)
+  clipping value  1e-4 relative, or the oracle's MSE at the GPU's step within 1e-6 of the
+                  minimum (two steps of the search can tie to that level)
+  packed codes    bit-exact given the same clip range and scale
+  dequantized     1e-6 absolute
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2211_04515_b200 as qp
+import synth_inputs as si
+
+pytestmark = pytest.mark.gpu
+
+ALL_BITS = [1, 2, 3, 4, 5, 6, 7, 8, 16]
+RAGGED = [1, 7, 31, 32, 33, 127, 128, 129, 1023, 1024, 1025, 4099, 100003]
+
+
+@pytest.fixture(scope="module")
+def ctx():
+    assert torch.cuda.is_available()
+    c = qp.Context(0)
+    yield c
+    assert c.qp_get_status() >= 0
+    c.close()
+
+
+def to_qp(o):
+    return qp.QParams(o.lo, o.hi, o.scale, o.inv_scale, o.bits, o.flags)
+
+
+def dev(x_np):
+    return torch.from_numpy(np.ascontiguousarray(x_np)).cuda()
+
+
+def guarded(nbytes, fill=0xA5, guard=256):
+    """Device byte buffer with canaries on both sides; returns (whole, view)."""
+    whole = torch.full((nbytes + 2 * guard,), fill, dtype=torch.uint8, device="cuda")
+    return whole, whole[guard:guard + nbytes]
+
+
+def canaries_intact(whole, nbytes, fill=0xA5, guard=256):
+    h = whole.cpu().numpy()
+    return (h[:guard] == fill).all() and (h[guard + nbytes:] == fill).all()
+
+
+def check_stats(st, st_o):
+    assert st.n == st_o.n and st.nonfinite == st_o.nonfinite
+    assert st.min == st_o.min and st.max == st_o.max
+    assert abs(st.mean - st_o.mean) <= 1e-5 * max(abs(st_o.mean), st_o.mad)
+    for f in ("mean_abs", "mad", "var"):
+        a, b = getattr(st, f), getattr(st_o, f)
+        assert abs(a - b) <= 1e-5 * abs(b), (f, a, b)
+
+
+# ------------------------------------------------------------------ statistics
+
+@pytest.mark.parametrize("name", ["c1", "c2"])
+def test_stats_configs(ctx, name):
+    x = si.config_tensor(name).reshape(-1)
+    st = ctx.read_stats(ctx.qp_stats(dev(x)))
+    check_stats(st, oracle.stats(x))
+    # bit-reproducible: fixed merge order
+    st2 = ctx.read_stats(ctx.qp_stats(dev(x)))
+    assert bytes(st) == bytes(st2)
+
+
+@pytest.mark.parametrize("n", RAGGED + [262144 + 5])
+def test_stats_ragged_and_misaligned(ctx, n):
+    x = si.vit_activation((1, n + 3, 1), 40 + n % 7).reshape(-1) * 3.0 + 0.25
+    x = x.astype(np.float32)
+    d = dev(x)
+    for off in (0, 1, 3):
+        st = ctx.read_stats(ctx.qp_stats(d[off:off + n]))
+        check_stats(st, oracle.stats(x[off:off + n]))
+
+
+def test_stats_special(ctx):
+    st = ctx.read_stats(ctx.qp_stats(torch.empty(0, device="cuda")))
+    assert (st.n, st.nonfinite, st.mean, st.mad, st.min, st.max) == (0, 0, 0.0, 0.0, 0.0, 0.0)
+    x = si.flat_iid(50000, 9, "laplace")
+    x[[5, 777, 49999]] = [np.nan, np.inf, -np.inf]
+    st = ctx.read_stats(ctx.qp_stats(dev(x)))
+    check_stats(st, oracle.stats(x))
+    assert st.nonfinite == 3
+    assert ctx.qp_get_status() & qp.QP_DEV_NONFINITE
+    c = np.full(3000, -1.5, dtype=np.float32)
+    st = ctx.read_stats(ctx.qp_stats(dev(c)))
+    assert (st.mean, st.mad, st.var, st.min, st.max) == (-1.5, 0.0, 0.0, -1.5, -1.5)
+    big = (np.float32(4096.0) + si.flat_iid(300000, 3, "normal")).astype(np.float32)     # mean >> spread
+    check_stats(ctx.read_stats(ctx.qp_stats(dev(big))), oracle.stats(big))
+    allbad = np.full(100, np.nan, dtype=np.float32)
+    st = ctx.read_stats(ctx.qp_stats(dev(allbad)))
+    assert st.nonfinite == 100 and st.mean == 0.0 and st.mad == 0.0
+    ctx.qp_get_status()
+
+
+def test_stats_bf16(ctx):
+    x = si.vit_activation((8, 197, 96), 12).reshape(-1)
+    h = si.to_bf16_bits(x)
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    for off, n in ((0, h.size), (3, h.size - 11), (1, 77)):
+        st = ctx.read_stats(ctx.qp_stats(d[off:off + n]))
+        check_stats(st, oracle.stats(oracle.widen_bf16(h[off:off + n])))
+
+
+# ------------------------------------------------------------- quantize + pack
+
+def run_pack_unpack(ctx, x_np, d_x, qp_o, bits, out_bf16=False):
+    n = x_np.size
+    qp_h = to_qp(qp_o)
+    nbytes = qp.qp_packed_bytes(n, bits)
+    whole, view = guarded(nbytes)
+    ctx.qp_quantize_pack(d_x, bits, qp_h, out=view)
+    ref = oracle.quantize_pack(x_np, qp_o)
+    got = view.cpu().numpy()
+    assert got.size == ref.size
+    assert np.array_equal(got, ref), f"bits={bits} n={n}: first diff at byte {np.flatnonzero(got != ref)[:4]}"
+    assert canaries_intact(whole, nbytes)
+    # receiver
+    ywhole, yview = guarded(4 * n)
+    y = yview.view(torch.float32)
+    ctx.qp_unpack_dequantize(view, n, bits, qp_h, out=y)
+    y_o = oracle.unpack_dequantize(ref, n, qp_o)
+    if n:
+        assert np.max(np.abs(y.cpu().numpy().astype(np.float64) - y_o.astype(np.float64))) <= 1e-6
+    assert canaries_intact(ywhole, 4 * n)
+    # output that is only 4-byte aligned: the scalar path must give the same values
+    if n in (33, 1025, 4099):
+        zwhole, zview = guarded(4 * (n + 1))
+        z = zview[4:].view(torch.float32)
+        ctx.qp_unpack_dequantize(view, n, bits, qp_h, out=z)
+        assert torch.equal(z, y) and canaries_intact(zwhole, 4 * (n + 1))
+        assert (zview[:4].cpu().numpy() == 0xA5).all()
+    return view
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_pack_unpack_c1(ctx, bits):
+    x = si.config_tensor("c1").reshape(-1)
+    st = oracle.stats(x)
+    _, _, qp_o = oracle.aciq_alpha(st, bits)
+    run_pack_unpack(ctx, x, dev(x), qp_o, bits)
+    # naive min/max range (Sec. 3, naive PTQ) through the same kernels
+    _, qp_n = oracle.make_qparams(st.min, st.max, bits)
+    run_pack_unpack(ctx, x, dev(x), qp_n, bits)
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_pack_unpack_ragged_and_misaligned(ctx, bits):
+    base = si.vit_activation((1, 1, 110000), 17).reshape(-1)
+    d = dev(base)
+    st = oracle.stats(base)
+    _, _, qp_o = oracle.aciq_alpha(st, bits)
+    for n in RAGGED:
+        for off in (0, 1) if n > 1024 or n in (33, 1023) else (0,):
+            run_pack_unpack(ctx, base[off:off + n], d[off:off + n], qp_o, bits)
+
+
+@pytest.mark.parametrize("bits", [1, 3, 4, 8, 16])
+def test_pack_special_values_and_degenerate(ctx, bits):
+    x = si.flat_iid(5000, 23, "normal")
+    x[[0, 1, 2, 3, 4097, 4999]] = [np.nan, np.inf, -np.inf, -0.0, np.nan, 1e38]
+    _, qp_o = oracle.make_qparams(-1.75, 2.25, bits)
+    run_pack_unpack(ctx, x, dev(x), qp_o, bits)
+    rc, qp_d = oracle.make_qparams(0.5, 0.5, bits)
+    assert rc == oracle.WARN_DEGENERATE
+    packed = run_pack_unpack(ctx, x, dev(x), qp_d, bits)
+    assert not packed.cpu().numpy().any()
+    # exact ties: positions k + 0.5 must round to the even level
+    L1 = 2 ** bits - 1
+    ties = (np.arange(min(L1, 4096), dtype=np.float32) + np.float32(0.5))
+    _, qp_t = oracle.make_qparams(0.0, float(L1), bits)
+    assert qp_t.scale == 1.0 and qp_t.inv_scale == 1.0
+    run_pack_unpack(ctx, ties, dev(ties), qp_t, bits)
+
+
+@pytest.mark.parametrize("bits", [2, 5, 8, 16])
+def test_pack_bf16_input_and_output(ctx, bits):
+    x = si.vit_activation((3, 197, 64), 31).reshape(-1)
+    h = si.to_bf16_bits(x)
+    xw = oracle.widen_bf16(h)
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    _, _, qp_o = oracle.aciq_alpha(oracle.stats(xw), bits)
+    for off, n in ((0, h.size), (0, 8 * 1024 + 5), (1, 2049)):
+        packed = ctx.qp_quantize_pack(d[off:off + n], bits, to_qp(qp_o))
+        ref = oracle.quantize_pack(xw[off:off + n], qp_o)
+        assert np.array_equal(packed.cpu().numpy(), ref)
+        y = ctx.qp_unpack_dequantize(packed, n, bits, to_qp(qp_o), out_dtype=torch.bfloat16)
+        y_o = si.to_bf16_bits(oracle.unpack_dequantize(ref, n, qp_o))
+        assert np.array_equal(y.view(torch.int16).cpu().numpy().view(np.uint16), y_o)
+
+
+def test_pack_argument_errors(ctx):
+    x = torch.zeros(1000, device="cuda")
+    _, qp_h = qp.qp_make_qparams(-1.0, 1.0, 4)
+    with pytest.raises(qp.QuantPipeError) as e:
+        ctx.qp_quantize_pack(x, 4, qp_h, out=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == qp.QP_ERR_BUFFER_TOO_SMALL
+    with pytest.raises(qp.QuantPipeError) as e:
+        ctx.qp_quantize_pack(x, 9, qp_h)
+    assert e.value.status == qp.QP_ERR_UNSUPPORTED_BITS
+    with pytest.raises(qp.QuantPipeError) as e:
+        ctx.qp_quantize_pack(x, 8, qp_h)                       # quantizer made for 4 bits
+    assert e.value.status == qp.QP_ERR_INVALID_ARG
+    with pytest.raises(qp.QuantPipeError) as e:
+        ctx.qp_quantize_pack(x, 4, qp_h, out=torch.empty(1024, dtype=torch.uint8, device="cuda")[1:])
+    assert e.value.status == qp.QP_ERR_ALIGNMENT
+    with pytest.raises(qp.QuantPipeError) as e:
+        ctx.qp_quantize_pack(x.double(), 4, qp_h)
+    assert e.value.status == qp.QP_ERR_UNSUPPORTED_DTYPE
+    assert ctx.qp_quantize_pack(x[:0], 4, qp_h).numel() == 0
+    # device-resident quantizer with other bits than the call: flagged in the status word
+    d_qp = torch.from_numpy(np.frombuffer(bytes(qp_h), dtype=np.uint8).copy()).cuda()
+    ctx.qp_get_status()
+    ctx.qp_quantize_pack(x, 2, d_qp)
+    assert ctx.qp_get_status() & qp.QP_DEV_BITS_MISMATCH
+
+
+# ------------------------------------------------------------ ACIQ on device
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_aciq_device_chain(ctx, bits):
+    """stats -> clip -> quantize with no host round trip; equals the oracle's chain."""
+    x = si.config_tensor("c1").reshape(-1)
+    d = dev(x)
+    d_stats = ctx.qp_stats(d)
+    st_o = oracle.stats(x)
+    for dist, bmode in ((0, 0), (0, 1), (1, 0)):
+        d_qp = ctx.qp_aciq_qparams_device(d_stats, bits, dist, bmode)
+        got = ctx.read_qparams(d_qp)
+        _, alpha_o, qp_o = oracle.aciq_alpha(st_o, bits, dist, bmode)
+        assert got.bits == bits and got.flags == 0
+        alpha_g = 0.5 * (float(got.hi) - float(got.lo))
+        assert abs(alpha_g - alpha_o) <= 1e-4 * alpha_o
+        assert abs(got.lo - qp_o.lo) <= 1e-5 * alpha_o and abs(got.hi - qp_o.hi) <= 1e-5 * alpha_o
+    d_qp = ctx.qp_aciq_qparams_device(d_stats, bits)
+    got = ctx.read_qparams(d_qp)
+    packed = ctx.qp_quantize_pack(d, bits, d_qp)
+    o = oracle.QParams(got.lo, got.hi, got.scale, got.inv_scale, got.bits, got.flags)
+    assert np.array_equal(packed.cpu().numpy(), oracle.quantize_pack(x, o))
+    y = ctx.qp_unpack_dequantize(packed, x.size, bits, d_qp)
+    assert np.max(np.abs(y.cpu().numpy() - oracle.unpack_dequantize(packed.cpu().numpy(), x.size, o))) <= 1e-6
+
+
+# ------------------------------------------------------------ directed search
+
+def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e-6):
+    d_stats = ctx.qp_stats(d_x)
+    d_res, d_qp = ctx.qp_dsaciq_search(d_x, d_stats, bits, bmode, steps, nb)
+    res, got_qp = ctx.read_ds_result(d_res), ctx.read_qparams(d_qp)
+    curve = np.array(ctx.qp_dsaciq_curve(steps))
+    st_o = oracle.stats(x_np)
+    rc_o, res_o, qp_o, curve_o = oracle.ds_search(x_np, st_o, bits, bmode, steps, nb)
+    assert (res.steps, res.hist_bins, res.bits) == (steps, nb, bits)
+    assert abs(res.b_e - res_o.b_e) <= 1e-5 * abs(res_o.b_e) + 1e-300
+    # the histogram counts are integers computed with the same fp32 expression; b_R can
+    # differ only through the fp64 statistics it is scaled by
+    assert abs(res.b_r - res_o.b_r) <= 1e-9 * abs(res_o.b_r) + 1e-300
+    fin = np.isfinite(curve_o)
+    assert np.array_equal(np.isfinite(curve), fin)
+    assert np.all(np.abs(curve[fin] - curve_o[fin]) <= curve_rtol * curve_o[fin] + 1e-300)
+    near_tie = curve_o[res.k_star] <= res_o.mse_star * (1 + 1e-6)
+    assert res.k_star == res_o.k_star or near_tie, (res.k_star, res_o.k_star)
+    if res.k_star == res_o.k_star:
+        assert abs(res.alpha_star - res_o.alpha_star) <= 1e-4 * abs(res_o.alpha_star)
+        assert abs(got_qp.lo - qp_o.lo) <= 1e-5 * res_o.alpha_star and abs(got_qp.hi - qp_o.hi) <= 1e-5 * res_o.alpha_star
+    assert res.mse_star <= res.mse_e
+    assert abs(res.alpha_e - res_o.alpha_e) <= 1e-5 * res_o.alpha_e + 1e-300
+    assert got_qp.bits == bits
+    return res, res_o
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_search_c1(ctx, bits):
+    x = si.config_tensor("c1").reshape(-1)
+    d = dev(x)
+    check_search(ctx, x, d, bits)
+    first = ctx.qp_dsaciq_curve(100)
+    check_search(ctx, x, d, bits)
+    assert ctx.qp_dsaciq_curve(100) == first          # fixed merge order: bit-reproducible
+
+
+@pytest.mark.parametrize("nb", [1, 64, 256, 2048, 16384])
+def test_search_hist_bins_and_modes(ctx, nb):
+    x = si.vit_activation((4, 197, 256), 2, outlier_frac=0.02).reshape(-1)
+    d = dev(x)
+    check_search(ctx, x, d, 2, nb=nb)
+    check_search(ctx, x, d, 4, bmode=1, nb=nb)
+
+
+@pytest.mark.parametrize("steps", [1, 7, 8, 9, 100, 250, 1023])
+def test_search_steps(ctx, steps):
+    x = si.vit_activation((1, 64, 192), 5).reshape(-1)
+    check_search(ctx, x, dev(x), 3, steps=steps)
+
+
+@pytest.mark.parametrize("n", [1, 5, 33, 1000, 4099, 100003])
+def test_search_ragged_misaligned_nonfinite(ctx, n):
+    x = si.vit_activation((1, n + 2, 1), 60 + n % 5).reshape(-1).astype(np.float32)
+    d = dev(x)
+    for off in (0, 1):
+        if n > 1:
+            check_search(ctx, x[off:off + n], d[off:off + n], 2)
+    if n >= 1000:
+        x[[3, n // 2]] = [np.nan, np.inf]
+        check_search(ctx, x[:n], dev(x[:n]), 4)
+        ctx.qp_get_status()
+
+
+def test_search_degenerate_and_errors(ctx):
+    c = np.full(5000, 2.5, dtype=np.float32)
+    d = dev(c)
+    d_stats = ctx.qp_stats(d)
+    d_res, d_qp = ctx.qp_dsaciq_search(d, d_stats, 2)
+    res, q = ctx.read_ds_result(d_res), ctx.read_qparams(d_qp)
+    assert res.k_star == 0 and res.b_star == 0.0 and res.mse_star == 0.0 and q.flags == 1
+    assert ctx.qp_get_status() & qp.QP_DEV_DEGENERATE
+    packed = ctx.qp_quantize_pack(d, 2, d_qp)
+    assert not packed.cpu().numpy().any()
+    assert np.array_equal(ctx.qp_unpack_dequantize(packed, c.size, 2, d_qp).cpu().numpy(), c)
+    for bad in (dict(bits=16), dict(bits=0), dict(steps=0), dict(steps=1024), dict(hist_bins=0), dict(hist_bins=16385)):
+        kw = dict(bits=2, steps=100, hist_bins=100)
+        kw.update(bad)
+        with pytest.raises(qp.QuantPipeError):
+            ctx.qp_dsaciq_search(d, d_stats, kw["bits"], 0, kw["steps"], kw["hist_bins"])
+
+
+def test_search_bf16(ctx):
+    x = si.vit_activation((4, 197, 128), 8).reshape(-1)
+    h = si.to_bf16_bits(x)
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    check_search(ctx, oracle.widen_bf16(h), d, 2)
+    check_search(ctx, oracle.widen_bf16(h[1:-2]), d[1:-2], 4)
+
+
+# ----------------------------------------------------- full-size configurations
+
+@pytest.mark.parametrize("name", ["c2", "c3", "c4"])
+def test_full_size_configs(ctx, name):
+    """The benchmark configurations at full size: statistics, search at the bit-widths where
+    the paper switches it on (<= 4), and pack/unpack at every listed width, all element by
+    element against the oracle."""
+    cfg = si.CONFIGS[name]
+    x = si.config_tensor(name).reshape(-1)
+    d = dev(x)
+    st_o = oracle.stats(x)
+    check_stats(ctx.read_stats(ctx.qp_stats(d)), st_o)
+    ds_bits = [b for b in cfg["bits"] if b <= 4] if name != "c4" else [2]
+    for bits in ds_bits:
+        res, res_o = check_search(ctx, x, d, bits)
+    for bits in cfg["bits"]:
+        _, _, qp_o = oracle.aciq_alpha(st_o, bits)
+        qp_h = to_qp(qp_o)
+        packed = ctx.qp_quantize_pack(d, bits, qp_h)
+        ref = oracle.quantize_pack(x, qp_o)
+        assert np.array_equal(packed.cpu().numpy(), ref), (name, bits)
+        y = ctx.qp_unpack_dequantize(packed, x.size, bits, qp_h).cpu().numpy()
+        y_o = oracle.unpack_dequantize(ref, x.size, qp_o)
+        assert np.max(np.abs(y.astype(np.float64) - y_o.astype(np.float64))) <= 1e-6
+        del packed, y
+
+
+@pytest.mark.parametrize("log2n,dist", [(18, "laplace"), (21, "normal"), (24, "laplace"), (26, "normal")])
+def test_roofline_sweep_sizes(ctx, log2n, dist):
+    n = 1 << log2n
+    x = si.flat_iid(n, si.C5_SEED, dist)
+    d = dev(x)
+    st_o = oracle.stats(x)
+    check_stats(ctx.read_stats(ctx.qp_stats(d)), st_o)
+    for bits in si.C5_BITS:
+        _, _, qp_o = oracle.aciq_alpha(st_o, bits, 1 if dist == "normal" else 0)
+        packed = ctx.qp_quantize_pack(d, bits, to_qp(qp_o))
+        ref = oracle.quantize_pack(x, qp_o)
+        assert np.array_equal(packed.cpu().numpy(), ref), (log2n, bits)
+        y = ctx.qp_unpack_dequantize(packed, n, bits, to_qp(qp_o)).cpu().numpy()
+        assert np.max(np.abs(y.astype(np.float64) - oracle.unpack_dequantize(ref, n, qp_o).astype(np.float64))) <= 1e-6
+    # bf16 input of the same element count
+    h = si.to_bf16_bits(x)
+    db = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    xw = oracle.widen_bf16(h)
+    _, _, qp_o = oracle.aciq_alpha(oracle.stats(xw), 4)
+    assert np.array_equal(ctx.qp_quantize_pack(db, 4, to_qp(qp_o)).cpu().numpy(), oracle.quantize_pack(xw, qp_o))
+
+
+def test_largest_sweep_size_sampled(ctx):
+    """1 GiB fp32 (2^28 elements): packed words and reconstructions checked on sampled
+    positions the oracle computes one by one, plus whole-buffer invariants."""
+    n = 1 << 28
+    x = si.flat_iid(n, si.C5_SEED, "laplace")
+    d = dev(x)
+    st = ctx.read_stats(ctx.qp_stats(d))
+    assert abs(st.mean) < 1e-3 and abs(st.mad - 1.0) < 1e-3 and st.n == n
+    starts = [0, 1024 * 12345, n // 2 - 512, n - 4096]
+    for bits in (1, 3, 4, 8, 16):
+        rc, alpha, qp_h = qp.qp_aciq_alpha(st, bits)
+        qp_o = oracle.QParams(qp_h.lo, qp_h.hi, qp_h.scale, qp_h.inv_scale, qp_h.bits, qp_h.flags)
+        packed = ctx.qp_quantize_pack(d, bits, qp_h)
+        assert packed.numel() == n * bits // 8
+        y = ctx.qp_unpack_dequantize(packed, n, bits, qp_h)
+        for s0 in starts:
+            win = x[s0:s0 + 4096]
+            ref = oracle.quantize_pack(win, qp_o)[:4096 * bits // 8]
+            got = packed[s0 * bits // 8:(s0 + 4096) * bits // 8].cpu().numpy()
+            assert np.array_equal(got, ref), (bits, s0)
+            y_o = oracle.unpack_dequantize(ref, 4096, qp_o)
+            assert np.max(np.abs(y[s0:s0 + 4096].cpu().numpy().astype(np.float64) - y_o)) <= 1e-6
+        # every reconstruction lies on the level grid inside the clip range
+        assert float(y.min()) >= qp_h.lo - 1e-6 and float(y.max()) <= qp_h.hi + 1e-5
+        del packed, y
