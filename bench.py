@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the activation-quantization path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one pass of the whole path over one batch of the ViT-Huge-shaped workload
+(fp32 [128,197,1280], 129 MB): bit-width from the step's link bandwidth (qp_select_bits on a
+seeded 100-step trace), statistics, clip (directed search at <= 4 bits, plain ACIQ above),
+quantize+pack, and the receiver's unpack+dequantize.  `value` is GB/s of fp32 input pushed
+through the whole step with inputs resident in HBM; `e2e` is the same through the
+host-buffer entry points with the host<->device copies inside the timed region.
+
+`--impl reference` times the CPU oracle (as it stands, single thread) on a bounded sample of
+the same workload and prints the same line shape.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synth_inputs as si  # noqa: E402
+
+WORKLOAD = "c4"
+METRIC = "quantize+pack and unpack+dequant throughput, fp32 in, whole path per step"
+UNIT = "GB/s"
+OPS_PER_CANDIDATE = 9          # fp32 instructions per element and candidate in the search kernel
+SAMPLE_IMAGES = 8              # CPU baseline leg: the first 8 images of the batch (2.0 M elements)
+ORACLE_US_PER_ELEM = 0.31      # rough cost of one oracle step per element (search on ~half the steps)
+
+
+def peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return float(d["hbm_gbs"]), float(d.get("sm_max_mhz", 1965.0)), "measured"
+    return 6650.0, 1965.0, "fallback"
+
+
+def step_bits(n_elems: int, select):
+    """Bit-width of every step of the bandwidth trace (host, O(1) per step)."""
+    trace = si.bandwidth_trace(si.CONFIGS[WORKLOAD]["seed"], si.C4_TRACE_STEPS)
+    out = []
+    for bw in trace:
+        rc, q = select(float(bw), si.C4_BUDGET_S, n_elems, 24, si.C4_ALLOWED_BITS)
+        out.append(q)
+    return out
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML (read-only) while running."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksThrottleReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksThrottleReasonSwPowerCap", 0x4): "sw_power_cap",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                r = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=1.0)
+        med = statistics.median(self.samples) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------- CPU oracle legs
+
+def oracle_step(oracle, x, bits, use_ds):
+    """One pass of the path in the oracle on host array x; returns nothing (timed by caller)."""
+    st = oracle.stats(x)
+    if use_ds:
+        _, _, qp, _ = oracle.ds_search(x, st, bits)
+    else:
+        _, _, qp = oracle.aciq_alpha(st, bits)
+    packed = oracle.quantize_pack(x, qp)
+    oracle.unpack_dequantize(packed, x.size, qp)
+
+
+def sample_images_for(steps: int, budget_s: float = 90.0) -> int:
+    """Images per step such that `steps` oracle steps take about budget_s seconds."""
+    per_image = 197 * 1280 * ORACLE_US_PER_ELEM * 1e-6
+    return int(max(1, min(16, budget_s / (steps * per_image))))
+
+
+def run_oracle_steps(first_step: int, count: int, bits_of_step, images: int = SAMPLE_IMAGES):
+    import oracle
+    x = si.vit_activation((images, 197, 1280), si.CONFIGS[WORKLOAD]["seed"]).reshape(-1)
+    oracle.lib()
+    t0 = time.perf_counter()
+    for t in range(first_step, first_step + count):
+        q = bits_of_step[t % len(bits_of_step)]
+        oracle_step(oracle, x, q, 1 <= q <= 4)
+    dt = time.perf_counter() - t0
+    return dt, x.size
+
+
+def reference_main(args):
+    """The CPU oracle as the reference arm: same metric, bounded sample per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    shape = si.CONFIGS[WORKLOAD]["shape"]
+    n_full = int(np.prod(shape))
+    bits_of_step = step_bits(n_full, oracle.select_bits)
+    images = sample_images_for(args.steps + args.warmup)
+    run_oracle_steps(0, args.warmup, bits_of_step, images)
+    dt, n_sample = run_oracle_steps(args.warmup, args.steps, bits_of_step, images)
+    gbs = args.steps * 4.0 * n_sample / dt / 1e9
+    sample = f"first {images} images of the batch ({n_sample} elements) per step, steps of the same trace"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": f"{WORKLOAD}: fp32 {list(shape)} ViT-Huge activations, adaptive bits from a 100-step "
+                               f"bandwidth trace; timed on a sample: {sample}"},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ------------------------------------------------------------------------- CUDA arm
+
+def ours_main(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2211_04515_b200 as qp
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback); use --impl reference for the oracle")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    hbm_peak, sm_max_mhz, peak_kind = peaks()
+
+    cfg = si.CONFIGS[WORKLOAD]
+    shape = cfg["shape"]
+    n = int(np.prod(shape))
+    bits_of_step = step_bits(n, qp.qp_select_bits)
+    ctx = qp.Context(local)
+
+    # inputs: ROT rotating copies so that a step never finds its input in L2 from the step before
+    ROT = 3
+    x_host = torch.empty(n, dtype=torch.float32, pin_memory=True)
+    si.config_tensor(WORKLOAD, out=x_host.numpy())
+    xs = [x_host.cuda(non_blocking=True) for _ in range(ROT)]
+    max_packed = qp.qp_packed_bytes(n, 16)
+    packed = torch.empty(max_packed, dtype=torch.uint8, device="cuda")
+    y = torch.empty(n, dtype=torch.float32, device="cuda")
+    d_stats = torch.empty(64, dtype=torch.uint8, device="cuda")
+    d_qp = torch.empty(24, dtype=torch.uint8, device="cuda")
+    d_res = torch.empty(72, dtype=torch.uint8, device="cuda")
+    torch.cuda.synchronize()
+
+    stage_names = ("stats", "clip", "quantize_pack", "unpack_dequantize")
+
+    def step(t, events=None):
+        q = bits_of_step[t % len(bits_of_step)]
+        x = xs[t % ROT]
+        marks = []
+        if events is not None:
+            marks = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+            marks[0].record()
+        ctx.qp_stats(x, out=d_stats)
+        if events is not None:
+            marks[1].record()
+        if qp.qp_policy_use_ds(q):
+            ctx.qp_dsaciq_search(x, d_stats, q, out_result=d_res, out_qp=d_qp)
+        else:
+            ctx.qp_aciq_qparams_device(d_stats, q, out=d_qp)
+        if events is not None:
+            marks[2].record()
+        ctx.qp_quantize_pack(x, q, d_qp, out=packed)
+        if events is not None:
+            marks[3].record()
+        ctx.qp_unpack_dequantize(packed, n, q, d_qp, out=y)
+        if events is not None:
+            marks[4].record()
+            events.append((q, marks))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for t in range(args.warmup):
+        step(t)
+    barrier()
+    assert ctx.qp_get_status() & ~qp.QP_DEV_NONFINITE == 0
+
+    # ---- timed region: exactly K steps, device-timed
+    events = []
+    launches0 = ctx.qp_launch_count()
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for t in range(args.warmup, args.warmup + args.steps):
+        step(t, events)
+    e1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.qp_launch_count() - launches0
+    if world > 1:
+        tt = torch.tensor([ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        ms = float(tt.item())
+    value = world * args.steps * 4.0 * n / (ms * 1e-3) / 1e9
+
+    # ---- per-stage device times from the events recorded inside the timed region
+    per = {}
+    for q, m in events:
+        for i, name in enumerate(stage_names):
+            per.setdefault((name, q), []).append(m[i].elapsed_time(m[i + 1]))
+    stage_ms = {name: sum(sum(v) for (nm, q), v in per.items() if nm == name) for name in stage_names}
+    kernels = {}
+    for (name, q), v in sorted(per.items()):
+        avg = sum(v) / len(v)
+        if name == "stats":
+            bytes_alg = 4.0 * n
+        elif name == "quantize_pack" or name == "unpack_dequantize":
+            bytes_alg = (4.0 + q / 8.0) * n
+        else:
+            bytes_alg = None
+        key = f"{name}@{q}b"
+        if bytes_alg is not None:
+            gbs = bytes_alg / (avg * 1e-3) / 1e9
+            kernels[key] = {"ms": round(avg, 4), "bound": "hbm", "achieved": round(gbs, 1), "peak": hbm_peak,
+                            "unit": "GB/s", "frac": round(gbs / hbm_peak, 4), "calls": len(v)}
+        elif qp.qp_policy_use_ds(q):
+            ops = float(n) * 101 * OPS_PER_CANDIDATE
+            alu_peak = 148 * 128 * sm_max_mhz * 1e6 / 1e12
+            tops = ops / (avg * 1e-3) / 1e12
+            kernels[key] = {"ms": round(avg, 4), "bound": "alu", "achieved": round(tops, 3), "peak": round(alu_peak, 2),
+                            "unit": "Tinstr/s", "frac": round(tops / alu_peak, 4), "calls": len(v)}
+        else:
+            kernels[key] = {"ms": round(avg, 4), "calls": len(v)}
+    # the dominant kernel of the step (largest share of device time)
+    dom = max(stage_ms, key=stage_ms.get)
+    dom_keys = [k for k in kernels if k.startswith(dom + "@") and "achieved" in kernels[k]]
+    tot_ms = sum(kernels[k]["ms"] * kernels[k]["calls"] for k in dom_keys)
+    ach = sum(kernels[k]["achieved"] * kernels[k]["ms"] * kernels[k]["calls"] for k in dom_keys) / tot_ms
+    first = kernels[dom_keys[0]]
+    roofline = {"kernel": dom, "bound": first["bound"], "achieved": round(ach, 3), "peak": first["peak"],
+                "unit": first["unit"], "frac": round(ach / first["peak"], 4), "peak_kind": peak_kind,
+                "traffic": None, "share_of_step_time": round(stage_ms[dom] / sum(stage_ms.values()), 3)}
+
+    # ---- end to end through the host-buffer entry points (pinned host memory, copies timed)
+    e2e_steps = max(3, min(args.steps, 30))
+    h_packed = torch.empty(max_packed, dtype=torch.uint8, pin_memory=True)
+    h_y = torch.empty(n, dtype=torch.float32, pin_memory=True)
+    h_qp = qp.QParams()
+    d_x_work = xs[0]
+
+    def e2e_step(t):
+        q = bits_of_step[t % len(bits_of_step)]
+        ctx.qp_sender_host(x_host, q, qp.qp_policy_use_ds(q), d_x_work, packed, h_packed, h_qp)
+        torch.cuda.current_stream().synchronize()          # the receiver needs the quantizer on the host
+        ctx.qp_receiver_host(h_packed, n, q, h_qp, packed, y, h_y)
+        return 4 * n + qp.qp_packed_bytes(n, q), qp.qp_packed_bytes(n, q) + 24 + 4 * n
+
+    for t in range(2):
+        e2e_step(t)
+    barrier()
+    t0 = time.perf_counter()
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    h2d = d2h = 0
+    for t in range(args.warmup, args.warmup + e2e_steps):
+        a, b = e2e_step(t)
+        h2d += a
+        d2h += b
+    s1.record()
+    barrier()
+    e2e_ms = max(s0.elapsed_time(s1), (time.perf_counter() - t0) * 1e3)
+    if world > 1:
+        tt = torch.tensor([e2e_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        e2e_ms = float(tt.item())
+    e2e = {"value": world * e2e_steps * 4.0 * n / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+           "h2d_bytes_per_step": h2d // e2e_steps, "d2h_bytes_per_step": d2h // e2e_steps, "steps": e2e_steps}
+
+    # ---- CPU oracle beside it (rank 0, N=1 only): bounded sample, same trace
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_steps = 16
+        dt, n_sample = run_oracle_steps(args.warmup, cpu_steps, bits_of_step)
+        cpu = {"value": cpu_steps * 4.0 * n_sample / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"{cpu_steps} steps of the same trace on the first {SAMPLE_IMAGES} images of the batch "
+                         f"({n_sample} elements), {dt:.1f} s"}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": f"{WORKLOAD}: fp32 {list(shape)} ViT-Huge activations (129 MB), adaptive bits "
+                                   f"{list(si.C4_ALLOWED_BITS)} from a seeded 100-step bandwidth trace, search at <=4 bits",
+                       "replicas": world, "l2": f"inputs larger than L2 (129 MB > 126 MB), {ROT} rotating input buffers",
+                       "bits_mix": {str(b): bits_of_step.count(b) for b in sorted(set(bits_of_step))}},
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
+            "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+    ctx.close()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return reference_main(args)
+    return ours_main(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -107,6 +107,8 @@ int32_t qp_get_status(qp_ctx* ctx, void* stream);
 /* Text of the last error recorded on this context (never NULL). */
 const char* qp_last_error(qp_ctx* ctx);
 const char* qp_status_string(int32_t status);
+/* Number of kernels this context has launched since qp_create (host-side count). */
+uint64_t qp_launch_count(qp_ctx* ctx);
 
 /* ---- sizes and parameters (host, pure) ------------------------------------------------*/
 
@@ -200,6 +202,24 @@ int32_t qp_select_bits(double bandwidth_bps, double budget_s, uint64_t n_elems, 
  * width q, B bit/s, S images per microbatch, R target images/s; clamped to [1, 32]. */
 int32_t qp_select_bits_eq2(double v_bytes, int q_t, double s_images, double r_images_per_s,
                            double bandwidth_bps, int32_t* h_bits_out);
+
+/* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
+ * output and the link, and between the link and the next stage's input) -------------------
+ * qp_sender_host: copies the n elements at h_x to d_x_work, runs statistics, the clip
+ * (directed search when use_ds != 0, plain ACIQ otherwise; Laplace model), quantize+pack
+ * into d_packed_work, and copies the packed stream to h_packed and the quantizer to
+ * *h_qp_out.  qp_receiver_host: copies h_packed to d_packed_work, unpacks+dequantizes into
+ * d_y_work and copies the tensor to h_y.  Everything is enqueued on `stream`; host outputs
+ * are valid after the caller has synchronised the stream.  Host buffers should be
+ * page-locked for the copies to be asynchronous.  The caller owns all six buffers:
+ * d_x_work >= n elements of dtype, d_packed_work and h_packed >= qp_packed_bytes(n, bits)
+ * (d_packed_work 16-byte aligned), d_y_work and h_y >= n elements of out_dtype.
+ * Errors: as the calls they are made of. */
+int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+                       int steps, int hist_bins, void* d_x_work, void* d_packed_work, void* h_packed,
+                       uint64_t packed_capacity, qp_qparams_t* h_qp_out, void* stream);
+int32_t qp_receiver_host(qp_ctx* ctx, const void* h_packed, uint64_t n, int bits, const qp_qparams_t* h_qp,
+                         void* d_packed_work, void* d_y_work, void* h_y, int out_dtype, void* stream);
 
 #ifdef __cplusplus
 }

@@ -28,7 +28,7 @@ EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
-    "qp_select_bits_eq2",
+    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host",
 )
 
 
@@ -89,9 +89,14 @@ def load() -> C.CDLL:
     L.qp_unpack_dequantize.argtypes = [vp, vp, u64, C.c_int, vp, C.c_int, vp, C.c_int, vp]
     L.qp_select_bits.argtypes = [dbl, dbl, u64, u64, C.POINTER(i32), C.c_int, C.POINTER(i32)]
     L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
+    L.qp_launch_count.argtypes = [vp]
+    L.qp_launch_count.restype = u64
+    L.qp_sender_host.argtypes = [vp, vp, C.c_int, u64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, u64,
+                                 C.POINTER(QParams), vp]
+    L.qp_receiver_host.argtypes = [vp, vp, u64, C.c_int, C.POINTER(QParams), vp, vp, vp, C.c_int, vp]
     for name in EXPORTS:
         fn = getattr(L, name)
-        if name not in ("qp_last_error", "qp_status_string", "qp_packed_bytes", "qp_aciq_F"):
+        if name not in ("qp_last_error", "qp_status_string", "qp_packed_bytes", "qp_aciq_F", "qp_launch_count"):
             fn.restype = i32
     _lib = L
     return L
@@ -267,6 +272,28 @@ class Context:
         self._check(self._lib.qp_unpack_dequantize(self._h, packed.data_ptr(), n, bits, ptr, on_dev, out.data_ptr(),
                                                    _dtype_code(out), _stream(self.device)))
         return out
+
+    # -- host-buffer sender / receiver
+    def qp_sender_host(self, h_x: torch.Tensor, bits: int, use_ds: bool, d_x_work: torch.Tensor,
+                       d_packed_work: torch.Tensor, h_packed: torch.Tensor, h_qp_out: QParams,
+                       bmode: int = QP_B_MAD, steps: int = QP_DEFAULT_STEPS, hist_bins: int = QP_DEFAULT_HIST_BINS):
+        """Host tensor in, packed host bytes + quantizer out (valid after a stream synchronise)."""
+        assert not h_x.is_cuda and h_x.is_contiguous() and not h_packed.is_cuda
+        self._check(self._lib.qp_sender_host(self._h, h_x.data_ptr(), _dtype_code(h_x), h_x.numel(), bits,
+                                             1 if use_ds else 0, bmode, steps, hist_bins, d_x_work.data_ptr(),
+                                             d_packed_work.data_ptr(), h_packed.data_ptr(),
+                                             h_packed.numel() * h_packed.element_size(), C.byref(h_qp_out),
+                                             _stream(self.device)))
+
+    def qp_receiver_host(self, h_packed: torch.Tensor, n: int, bits: int, h_qp: QParams, d_packed_work: torch.Tensor,
+                         d_y_work: torch.Tensor, h_y: torch.Tensor):
+        assert not h_packed.is_cuda and not h_y.is_cuda and h_y.is_contiguous() and h_y.numel() >= n
+        self._check(self._lib.qp_receiver_host(self._h, h_packed.data_ptr(), n, bits, C.byref(h_qp),
+                                               d_packed_work.data_ptr(), d_y_work.data_ptr(), h_y.data_ptr(),
+                                               _dtype_code(h_y), _stream(self.device)))
+
+    def qp_launch_count(self) -> int:
+        return int(self._lib.qp_launch_count(self._h))
 
     # -- status / read-back
     def qp_get_status(self) -> int:

@@ -76,6 +76,8 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     const size_t o_setup = off;  off = align_up(off + sizeof(qp_ds_setup), 256);
     const size_t o_ticket = off; off = align_up(off + sizeof(unsigned) * 4, 256);
     const size_t o_status = off; off = align_up(off + sizeof(unsigned), 256);
+    const size_t o_tstats = off; off = align_up(off + sizeof(qp_stats_t), 256);
+    const size_t o_tqp = off;    off = align_up(off + sizeof(qp_qparams_t), 256);
 
     if (cudaMalloc(&c->d_base, off) != cudaSuccess || cudaMemset(c->d_base, 0, off) != cudaSuccess) {
         cudaGetLastError();
@@ -93,6 +95,8 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     c->d_setup = reinterpret_cast<qp_ds_setup*>(b + o_setup);
     c->d_ticket = reinterpret_cast<unsigned*>(b + o_ticket);
     c->d_status = reinterpret_cast<unsigned*>(b + o_status);
+    c->d_tmp_stats = reinterpret_cast<qp_stats_t*>(b + o_tstats);
+    c->d_tmp_qp = reinterpret_cast<qp_qparams_t*>(b + o_tqp);
     *out = c;
     return QP_OK;
 }
@@ -121,6 +125,8 @@ extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
     }
     return (int32_t)word;
 }
+
+extern "C" uint64_t qp_launch_count(qp_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
 // ------------------------------------------------------ host, pure functions
 
@@ -373,4 +379,67 @@ extern "C" int32_t qp_unpack_dequantize(qp_ctx* ctx, const void* d_packed, uint6
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
     return qp_launch_unpack(ctx, d_packed, n, bits, d_qp, h_qp, d_y, out_dtype, static_cast<cudaStream_t>(stream));
+}
+
+// ------------------------------------------- host-buffer sender and receiver
+
+extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+                                  int steps, int hist_bins, void* d_x_work, void* d_packed_work, void* h_packed,
+                                  uint64_t packed_capacity, qp_qparams_t* h_qp_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (dtype != QP_F32 && dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "dtype");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (use_ds && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if (!h_qp_out || (n > 0 && (!h_x || !d_x_work || !d_packed_work || !h_packed)))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "null buffer");
+    const uint64_t need = qp_packed_bytes(n, bits);
+    if (packed_capacity < need) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esz = dtype == QP_F32 ? 4 : 2;
+    {
+        qp_device_guard guard(ctx->device);
+        if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+        if (n && cudaMemcpyAsync(d_x_work, h_x, n * esz, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return qp_check_launch(ctx, "qp_sender_host (copy in)");
+    }
+    int32_t rc = qp_stats(ctx, d_x_work, dtype, n, ctx->d_tmp_stats, stream);
+    if (rc < 0) return rc;
+    if (use_ds) rc = qp_dsaciq_search(ctx, d_x_work, dtype, n, ctx->d_tmp_stats, bits, bmode, steps, hist_bins, nullptr,
+                                      ctx->d_tmp_qp, stream);
+    else        rc = qp_aciq_qparams_device(ctx, ctx->d_tmp_stats, bits, QP_DIST_LAPLACE, bmode, ctx->d_tmp_qp, stream);
+    if (rc < 0) return rc;
+    rc = qp_quantize_pack(ctx, d_x_work, dtype, n, bits, ctx->d_tmp_qp, 1, d_packed_work, need, stream);
+    if (rc < 0) return rc;
+    qp_device_guard guard(ctx->device);
+    cudaError_t e = cudaSuccess;
+    if (need) e = cudaMemcpyAsync(h_packed, d_packed_work, need, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(h_qp_out, ctx->d_tmp_qp, sizeof(qp_qparams_t), cudaMemcpyDeviceToHost, s);
+    if (e != cudaSuccess) return qp_check_launch(ctx, "qp_sender_host (copy out)");
+    return QP_OK;
+}
+
+extern "C" int32_t qp_receiver_host(qp_ctx* ctx, const void* h_packed, uint64_t n, int bits, const qp_qparams_t* h_qp,
+                                    void* d_packed_work, void* d_y_work, void* h_y, int out_dtype, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (out_dtype != QP_F32 && out_dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "out_dtype");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (!h_qp || (n > 0 && (!h_packed || !d_packed_work || !d_y_work || !h_y)))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "null buffer");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint64_t need = qp_packed_bytes(n, bits);
+    {
+        qp_device_guard guard(ctx->device);
+        if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+        if (need && cudaMemcpyAsync(d_packed_work, h_packed, need, cudaMemcpyHostToDevice, s) != cudaSuccess)
+            return qp_check_launch(ctx, "qp_receiver_host (copy in)");
+    }
+    const int32_t rc = qp_unpack_dequantize(ctx, d_packed_work, n, bits, h_qp, 0, d_y_work, out_dtype, stream);
+    if (rc < 0) return rc;
+    qp_device_guard guard(ctx->device);
+    const size_t esz = out_dtype == QP_F32 ? 4 : 2;
+    if (n && cudaMemcpyAsync(h_y, d_y_work, n * esz, cudaMemcpyDeviceToHost, s) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_receiver_host (copy out)");
+    return QP_OK;
 }

@@ -40,6 +40,9 @@ struct qp_ctx {
     qp_ds_setup* d_setup;
     unsigned int* d_ticket;              // [4] last-block tickets (always left at 0)
     unsigned int* d_status;              // device status word
+    qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
+    qp_qparams_t* d_tmp_qp;
+    unsigned long long launches;         // kernels launched through this context (host count)
     int last_steps;                      // steps of the last search (for qp_dsaciq_curve)
     char err[256];
 };

@@ -185,6 +185,7 @@ int32_t pack_typed(qp_ctx* ctx, const T* x, uint64_t n, int bits, const qp_qpara
         uint64_t want = (nvec_out + QP_THREADS - 1) / QP_THREADS;
         const uint64_t cap = (uint64_t)ctx->sm_count * 64;
         const int blocks = (int)(want > cap ? cap : want);
+        ctx->launches += 1;
         if (aligned)
             pack16_kernel<T, true><<<blocks, QP_THREADS, 0, s>>>(x, n, d_qp, h_qp, static_cast<uint4*>(d_packed), nvec_out, ctx->d_status);
         else
@@ -197,6 +198,7 @@ int32_t pack_typed(qp_ctx* ctx, const T* x, uint64_t n, int bits, const qp_qpara
         uint64_t want = (ntiles + WARPS - 1) / WARPS;
         const uint64_t cap = (uint64_t)ctx->sm_count * 64;
         const int blocks = (int)(want > cap ? cap : want);
+        ctx->launches += 1;
 #define QP_PACK_CASE(B) case B: pack_kernel<B, T><<<blocks, QP_THREADS, 0, s>>>(x, ntiles, d_qp, h_qp, out, ctx->d_status); break;
         switch (bits) {
             QP_PACK_CASE(1) QP_PACK_CASE(2) QP_PACK_CASE(3) QP_PACK_CASE(4)
@@ -210,6 +212,7 @@ int32_t pack_typed(qp_ctx* ctx, const T* x, uint64_t n, int bits, const qp_qpara
         const uint64_t nwords = total_words - done_words;
         const uint64_t threads = (nwords + bits - 1) / bits;
         const uint64_t blocks = (threads + QP_THREADS - 1) / QP_THREADS;
+        ctx->launches += 1;
         pack_tail_kernel<T><<<(unsigned)blocks, QP_THREADS, 0, s>>>(x, ntiles * TILE, n, bits, d_qp, h_qp,
                                                                      out + done_words, nwords, ctx->d_status);
     }

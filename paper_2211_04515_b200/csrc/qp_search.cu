@@ -328,6 +328,7 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     eval_kernel<T><<<dim3(groups, chunks), QP_THREADS, 0, s>>>(x, n, d_stats, ctx->d_cand, ncand, ctx->d_sums);
     finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, chunks, steps, nb, bits, ctx->d_valid, ctx->d_cand,
                                              ctx->d_setup, ctx->d_curve, d_out, d_qp_out, ctx->d_status);
+    ctx->launches += 4;
     return qp_check_launch(ctx, "qp_dsaciq_search");
 }
 
@@ -348,5 +349,6 @@ int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, 
                               qp_qparams_t* d_qp_out, cudaStream_t s)
 {
     aciq_kernel<<<1, 32, 0, s>>>(d_stats, bits, dist, bmode, F, d_qp_out, ctx->d_status);
+    ctx->launches += 1;
     return qp_check_launch(ctx, "qp_aciq_qparams_device");
 }

@@ -230,6 +230,7 @@ int32_t launch_typed(qp_ctx* ctx, const T* x, uint64_t n, qp_stats_t* d_out, cud
     if (blocks > QP_MAX_BLOCKS) blocks = QP_MAX_BLOCKS;
     stats_pass_a<T><<<blocks, QP_THREADS, 0, s>>>(x, n, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
     stats_pass_b<T><<<blocks, QP_THREADS, 0, s>>>(x, n, ctx->d_part, ctx->d_ticket, d_out);
+    ctx->launches += 2;
     return qp_check_launch(ctx, "qp_stats");
 }
 

@@ -177,6 +177,7 @@ int32_t unpack_typed(qp_ctx* ctx, const void* d_packed, uint64_t n, int bits, co
         uint64_t want = (nvec + QP_THREADS - 1) / QP_THREADS;
         const uint64_t cap = (uint64_t)ctx->sm_count * 64;
         const int blocks = (int)(want > cap ? cap : want);
+        ctx->launches += 1;
         if (aligned)
             unpack16_kernel<TO, true><<<blocks, QP_THREADS, 0, s>>>(static_cast<const uint4*>(d_packed), n, d_qp, h_qp, y, ctx->d_status);
         else
@@ -189,6 +190,7 @@ int32_t unpack_typed(qp_ctx* ctx, const void* d_packed, uint64_t n, int bits, co
         uint64_t want = (ntiles + WARPS - 1) / WARPS;
         const uint64_t cap = (uint64_t)ctx->sm_count * 64;
         const int blocks = (int)(want > cap ? cap : want);
+        ctx->launches += 1;
 #define QP_UNPACK_CASE(B) case B: unpack_kernel<B, TO><<<blocks, QP_THREADS, 0, s>>>(in, ntiles, d_qp, h_qp, y, ctx->d_status); break;
         switch (bits) {
             QP_UNPACK_CASE(1) QP_UNPACK_CASE(2) QP_UNPACK_CASE(3) QP_UNPACK_CASE(4)
@@ -200,6 +202,7 @@ int32_t unpack_typed(qp_ctx* ctx, const void* d_packed, uint64_t n, int bits, co
     if (n > first) {
         const uint64_t threads = (n - first + 31) / 32;
         const uint64_t blocks = (threads + QP_THREADS - 1) / QP_THREADS;
+        ctx->launches += 1;
         unpack_tail_kernel<TO><<<(unsigned)blocks, QP_THREADS, 0, s>>>(in + ntiles * 32 * (uint64_t)bits, first, n, bits,
                                                                        d_qp, h_qp, y, ctx->d_status);
     }
