@@ -43,6 +43,7 @@ enum {
     QP_ERR_ALIGNMENT = -5,
     QP_ERR_CUDA = -6,
     QP_ERR_TIMEOUT = -7,
+    QP_ERR_TOO_LARGE = -8,    /* size beyond a stated maximum of the entry point          */
     QP_WARN_INFEASIBLE = 1,   /* qp_select_bits: nothing fits, smallest width returned   */
     QP_WARN_DEGENERATE = 2,   /* empty clip range (constant tensor): all codes are 0     */
     QP_WARN_NONFINITE = 3     /* reported by qp_get_status: NaN/Inf were seen and skipped */
@@ -135,6 +136,26 @@ int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out);
  * d_x must be aligned to its element size.
  * Errors: QP_ERR_INVALID_ARG (NULL), QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
 int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream);
+
+/* Statistics for callers that cannot allocate device memory (no counterpart in the paper;
+ * same results as qp_stats).  Some code may not call cudaMalloc or any allocating routine:
+ * it runs while the framework's memory pool is frozen, or all device memory was handed out
+ * before this library came in.  This entry point takes no qp_ctx and allocates nothing: its
+ * scratch (block partials, tickets, status word; 49,408 bytes) is a fixed array inside the
+ * library image, resident on every GPU that loads the library until the process exits.
+ * It works on the calling thread's current device and enqueues on `stream`.
+ *   - The first call on each device looks up the array's device address (a set-up step that
+ *     talks to the driver): make that first call before starting any stream capture.
+ *   - n may not exceed QP_STATS_STATIC_MAX_N; larger tensors return QP_ERR_TOO_LARGE and
+ *     nothing is enqueued (use qp_stats, whose context has room for them).
+ *   - All calls on a device share the one array, which keeps the previous call's contents
+ *     (the counters that must start at zero are cleared on `stream` first).  Two calls
+ *     that overlap on the GPU (different streams, no ordering between them) race on it and
+ *     give wrong statistics: order them.
+ * Errors: QP_ERR_INVALID_ARG (NULL), QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT,
+ * QP_ERR_TOO_LARGE, QP_ERR_CUDA. */
+#define QP_STATS_STATIC_MAX_N (1ull << 31)
+int32_t qp_stats_static(const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream);
 
 /* ---- a3: ACIQ clip (Sec. 3: alpha = F(q) * b under L(mu, b)) ---------------------------
  * Host form: from statistics already copied to the host.  b is h_stats->mad (bmode

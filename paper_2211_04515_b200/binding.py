@@ -17,6 +17,8 @@ LIB_PATH = os.path.join(_PKG, "libquantpipe.so")
 QP_OK = 0
 QP_ERR_INVALID_ARG, QP_ERR_UNSUPPORTED_BITS, QP_ERR_UNSUPPORTED_DTYPE = -1, -2, -3
 QP_ERR_BUFFER_TOO_SMALL, QP_ERR_ALIGNMENT, QP_ERR_CUDA, QP_ERR_TIMEOUT = -4, -5, -6, -7
+QP_ERR_TOO_LARGE = -8
+QP_STATS_STATIC_MAX_N = 1 << 31
 QP_WARN_INFEASIBLE, QP_WARN_DEGENERATE, QP_WARN_NONFINITE = 1, 2, 3
 QP_F32, QP_BF16 = 0, 1
 QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
@@ -28,7 +30,7 @@ EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
-    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host",
+    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static",
 )
 
 
@@ -89,6 +91,7 @@ def load() -> C.CDLL:
     L.qp_unpack_dequantize.argtypes = [vp, vp, u64, C.c_int, vp, C.c_int, vp, C.c_int, vp]
     L.qp_select_bits.argtypes = [dbl, dbl, u64, u64, C.POINTER(i32), C.c_int, C.POINTER(i32)]
     L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
+    L.qp_stats_static.argtypes = [vp, C.c_int, u64, vp, vp]
     L.qp_launch_count.argtypes = [vp]
     L.qp_launch_count.restype = u64
     L.qp_sender_host.argtypes = [vp, vp, C.c_int, u64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, u64,
@@ -149,6 +152,16 @@ def qp_select_bits_eq2(v_bytes: float, q_t: int, s_images: float, r_images_per_s
 
 
 # ------------------------------------------------------------ device calls
+
+def qp_stats_static(x: "torch.Tensor", out: "torch.Tensor", n: int | None = None) -> int:
+    """Statistics of x into the 64-byte device buffer `out`, for callers that may not
+    allocate: no context, no allocation here or in the library (the caller brings `out`).
+    Runs on x's device, which must be the current one, on torch's current stream.
+    Returns the status code; negative codes are errors (QP_ERR_TOO_LARGE above
+    QP_STATS_STATIC_MAX_N elements)."""
+    count = x.numel() if n is None else n
+    return int(load().qp_stats_static(x.data_ptr(), _dtype_code(x), count, out.data_ptr(), _stream(x.device)))
+
 
 def _dtype_code(t: torch.Tensor) -> int:
     if t.dtype == torch.float32:

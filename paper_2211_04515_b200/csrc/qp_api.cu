@@ -33,6 +33,7 @@ extern "C" const char* qp_status_string(int32_t s)
         case QP_ERR_ALIGNMENT: return "misaligned pointer";
         case QP_ERR_CUDA: return "CUDA error";
         case QP_ERR_TIMEOUT: return "device wait timed out";
+        case QP_ERR_TOO_LARGE: return "size exceeds the maximum this entry point supports";
         case QP_WARN_INFEASIBLE: return "warning: no allowed bit-width fits the budget";
         case QP_WARN_DEGENERATE: return "warning: degenerate clip range";
         case QP_WARN_NONFINITE: return "warning: non-finite inputs were skipped";

@@ -245,3 +245,82 @@ int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_
     if (dtype == QP_F32) return launch_typed<float>(ctx, static_cast<const float*>(d_x), n, d_out, s);
     return launch_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_out, s);
 }
+
+// ---------------------------------------------------------------------------------------
+// Statistics without a context and without any allocation.
+//
+// Some callers must not allocate device memory at all: code that runs while a memory pool
+// is frozen, inside a region where the allocator may not be re-entered, or in a process
+// whose whole device budget was handed out before this library was loaded.  For them the
+// scratch that qp_stats keeps in its qp_ctx (block partials, two tickets, a status word)
+// lives in the fixed array below, which every GPU that loads the library holds until the
+// process exits.  Its size bounds the grid (QP_STATIC_BLOCKS partials), not the tensor.
+#include <mutex>
+
+namespace {
+
+constexpr int QP_STATIC_BLOCKS = 1024;
+constexpr size_t QP_STATIC_PART_BYTES = sizeof(qp_stats_partial) * QP_STATIC_BLOCKS;      // 48 KiB
+constexpr size_t QP_STATIC_BYTES = QP_STATIC_PART_BYTES + 256;                            // + tickets, status
+
+// In host code this name is only a handle for cudaGetSymbolAddress, never a device address.
+static __device__ __align__(256) unsigned char qp_static_scratch[QP_STATIC_BYTES];
+
+constexpr int QP_STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mu;
+unsigned char* g_static_ptr[QP_STATIC_MAX_DEVICES] = {};
+int g_static_sms[QP_STATIC_MAX_DEVICES] = {};
+
+template <typename T>
+int32_t static_typed(const T* x, uint64_t n, qp_stats_t* d_out, unsigned char* scratch, int sms, cudaStream_t s)
+{
+    qp_stats_partial* part = reinterpret_cast<qp_stats_partial*>(scratch);
+    unsigned* ticket = reinterpret_cast<unsigned*>(scratch + QP_STATIC_PART_BYTES);        // [0], [1]
+    unsigned* status = ticket + 4;
+    // the array keeps whatever the last call left: tickets and status must start at zero
+    if (cudaMemsetAsync(ticket, 0, 256, s) != cudaSuccess) { cudaGetLastError(); return QP_ERR_CUDA; }
+    const uint64_t per_block = (uint64_t)QP_THREADS * UNROLL * qp_span<T>::EPV;
+    uint64_t want = (n + per_block - 1) / per_block;
+    const uint64_t cap = (uint64_t)sms * 6;
+    int blocks = (int)(want < 1 ? 1 : (want > cap ? cap : want));
+    if (blocks > QP_STATIC_BLOCKS) blocks = QP_STATIC_BLOCKS;
+    stats_pass_a<T><<<blocks, QP_THREADS, 0, s>>>(x, n, part, ticket, d_out, status);
+    stats_pass_b<T><<<blocks, QP_THREADS, 0, s>>>(x, n, part, ticket, d_out);
+    return cudaGetLastError() == cudaSuccess ? QP_OK : QP_ERR_CUDA;
+}
+
+}  // namespace
+
+extern "C" int32_t qp_stats_static(const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream)
+{
+    if (dtype != QP_F32 && dtype != QP_BF16) return QP_ERR_UNSUPPORTED_DTYPE;
+    if (!d_out || (n > 0 && !d_x)) return QP_ERR_INVALID_ARG;
+    if (((uintptr_t)d_x & (dtype == QP_F32 ? 3u : 1u)) || ((uintptr_t)d_out & 7u)) return QP_ERR_ALIGNMENT;
+    if (n > QP_STATS_STATIC_MAX_N) return QP_ERR_TOO_LARGE;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) { cudaGetLastError(); return QP_ERR_CUDA; }
+    if (dev < 0 || dev >= QP_STATIC_MAX_DEVICES) return QP_ERR_INVALID_ARG;
+    unsigned char* scratch = nullptr;
+    int sms = 0;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mu);
+        if (!g_static_ptr[dev]) {
+            // once per device, with that device current: resolve the array's device address
+            void* p = nullptr;
+            if (cudaGetSymbolAddress(&p, qp_static_scratch) != cudaSuccess || !p) { cudaGetLastError(); return QP_ERR_CUDA; }
+            int count = 0;
+            if (cudaDeviceGetAttribute(&count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || count < 1) {
+                cudaGetLastError();
+                return QP_ERR_CUDA;
+            }
+            g_static_sms[dev] = count;
+            g_static_ptr[dev] = static_cast<unsigned char*>(p);
+        }
+        scratch = g_static_ptr[dev];
+        sms = g_static_sms[dev];
+    }
+    if (n == 0) return cudaMemsetAsync(d_out, 0, sizeof(qp_stats_t), s) == cudaSuccess ? QP_OK : QP_ERR_CUDA;
+    if (dtype == QP_F32) return static_typed<float>(static_cast<const float*>(d_x), n, d_out, scratch, sms, s);
+    return static_typed<unsigned short>(static_cast<const unsigned short*>(d_x), n, d_out, scratch, sms, s);
+}
