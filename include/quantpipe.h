@@ -180,6 +180,15 @@ int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits,
 int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                          int bits, int bmode, int steps, int hist_bins,
                          qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, void* stream);
+/* How qp_dsaciq_search scores the candidates.  Both ways give the same MSE per candidate
+ * (to ~1e-8 relative) and the same winner.
+ *   QP_SEARCH_CANDIDATES  every element is quantized under every candidate (any bits/steps)
+ *   QP_SEARCH_INTERVALS   one pass gathers moments per interval between the candidates'
+ *                         decision thresholds; used where (steps+1)*(2^bits-1) <= 2049 and
+ *                         n < ~1.2e9, otherwise the call falls back to the first way
+ *   QP_SEARCH_AUTO        intervals for n >= 2^20 where they apply (default) */
+enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2 };
+int32_t qp_set_search_path(qp_ctx* ctx, int path);
 /* Copies the MSE of every candidate of the last search on this context (steps+1 values)
  * to host memory after waiting for `stream`.  Diagnostic. */
 int32_t qp_dsaciq_curve(qp_ctx* ctx, double* h_curve, int capacity, void* stream);

@@ -25,12 +25,13 @@ QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
 QP_B_MAD, QP_B_MEAN_ABS = 0, 1
 QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE = 1, 2, 4
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
+QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
 
 EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
-    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static",
+    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path",
 )
 
 
@@ -92,6 +93,7 @@ def load() -> C.CDLL:
     L.qp_select_bits.argtypes = [dbl, dbl, u64, u64, C.POINTER(i32), C.c_int, C.POINTER(i32)]
     L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
     L.qp_stats_static.argtypes = [vp, C.c_int, u64, vp, vp]
+    L.qp_set_search_path.argtypes = [vp, C.c_int]
     L.qp_launch_count.argtypes = [vp]
     L.qp_launch_count.restype = u64
     L.qp_sender_host.argtypes = [vp, vp, C.c_int, u64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, u64,
@@ -253,6 +255,9 @@ class Context:
                                                bits, bmode, steps, hist_bins, out_result.data_ptr(), out_qp.data_ptr(),
                                                _stream(self.device)))
         return out_result, out_qp
+
+    def qp_set_search_path(self, path: int):
+        self._check(self._lib.qp_set_search_path(self._h, path))
 
     def qp_dsaciq_curve(self, steps: int):
         buf = (C.c_double * (steps + 1))()

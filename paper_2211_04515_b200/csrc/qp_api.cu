@@ -77,6 +77,14 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     const size_t o_setup = off;  off = align_up(off + sizeof(qp_ds_setup), 256);
     const size_t o_ticket = off; off = align_up(off + sizeof(unsigned) * 4, 256);
     const size_t o_status = off; off = align_up(off + sizeof(unsigned), 256);
+    c->iv_blocks = c->sm_count * QP_IV_BLOCKS_PER_SM;
+    const size_t o_ivbnd = off;  off = align_up(off + sizeof(float) * QP_IV_MAXB, 256);
+    const size_t o_ivbb = off;   off = align_up(off + sizeof(float) * (QP_IV_MAXB + 1), 256);
+    const size_t o_ivedge = off; off = align_up(off + sizeof(float) * (QP_IV_CELLS + 1), 256);
+    const size_t o_ivfirst = off; off = align_up(off + sizeof(unsigned) * (QP_IV_CELLS + 2), 256);
+    const size_t o_ivpart = off; off = align_up(off + sizeof(ulonglong2) * (size_t)c->iv_blocks * (QP_IV_MAXB + 1), 256);
+    const size_t o_ivouter = off; off = align_up(off + sizeof(double) * 8 * c->iv_blocks, 256);
+    const size_t o_ivtot = off;  off = align_up(off + sizeof(qp_iv_total) * (QP_IV_MAXB + 1), 256);
     const size_t o_tstats = off; off = align_up(off + sizeof(qp_stats_t), 256);
     const size_t o_tqp = off;    off = align_up(off + sizeof(qp_qparams_t), 256);
 
@@ -96,6 +104,13 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     c->d_setup = reinterpret_cast<qp_ds_setup*>(b + o_setup);
     c->d_ticket = reinterpret_cast<unsigned*>(b + o_ticket);
     c->d_status = reinterpret_cast<unsigned*>(b + o_status);
+    c->d_iv_bnd = reinterpret_cast<float*>(b + o_ivbnd);
+    c->d_iv_bb = reinterpret_cast<float*>(b + o_ivbb);
+    c->d_iv_edges = reinterpret_cast<float*>(b + o_ivedge);
+    c->d_iv_first = reinterpret_cast<unsigned*>(b + o_ivfirst);
+    c->d_iv_part = reinterpret_cast<ulonglong2*>(b + o_ivpart);
+    c->d_iv_outer = reinterpret_cast<double*>(b + o_ivouter);
+    c->d_iv_tot = reinterpret_cast<qp_iv_total*>(b + o_ivtot);
     c->d_tmp_stats = reinterpret_cast<qp_stats_t*>(b + o_tstats);
     c->d_tmp_qp = reinterpret_cast<qp_qparams_t*>(b + o_tqp);
     *out = c;
@@ -128,6 +143,14 @@ extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
 }
 
 extern "C" uint64_t qp_launch_count(qp_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int32_t qp_set_search_path(qp_ctx* ctx, int path)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
+    ctx->search_path = path;
+    return QP_OK;
+}
 
 // ------------------------------------------------------ host, pure functions
 

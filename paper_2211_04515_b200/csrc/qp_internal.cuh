@@ -25,7 +25,19 @@ struct qp_ds_setup {                     // written by the search's set-up kerne
     unsigned long long n_finite;
     int degenerate;
     int pad;
+    // interval-moment path: the grid that covers every candidate's clip range
+    float g_lo, g_hi;                    // min lo_k, max hi_k over the valid candidates
+    float inv_gw;                        // QP_IV_CELLS / (g_hi - g_lo), 0 for an empty range
+    float inv_u;                         // 1 / u, u = fixed-point unit of offsets inside an interval (a power of two)
+    double u;
 };
+
+constexpr int QP_IV_CELLS = 2048;        // uniform cells over [g_lo, g_hi]
+constexpr int QP_IV_MAXB = 4096;         // most interval boundaries (candidate thresholds + cell edges)
+constexpr int QP_IV_THREADS = 512;
+constexpr int QP_IV_BLOCKS_PER_SM = 2;
+
+struct qp_iv_total { unsigned long long n, s1, s2; };   // per interval: count, sum d, sum d^2 (fixed point)
 
 struct qp_ctx {
     int device;
@@ -40,6 +52,15 @@ struct qp_ctx {
     qp_ds_setup* d_setup;
     unsigned int* d_ticket;              // [4] last-block tickets (always left at 0)
     unsigned int* d_status;              // device status word
+    float* d_iv_bnd;                     // [QP_IV_MAXB] unsorted boundaries
+    float* d_iv_bb;                      // [QP_IV_MAXB + 1] g_lo followed by the sorted boundaries
+    float* d_iv_edges;                   // [QP_IV_CELLS + 1] left edge of every cell
+    unsigned* d_iv_first;                // [QP_IV_CELLS + 2] first interval of every cell; last entry = boundary count
+    ulonglong2* d_iv_part;               // [blocks][QP_IV_MAXB + 1] per-block (count<<40 | sum d, sum d^2)
+    double* d_iv_outer;                  // [blocks][8] sums over the elements outside [g_lo, g_hi]
+    qp_iv_total* d_iv_tot;               // [QP_IV_MAXB + 1]
+    int iv_blocks;                       // blocks of the interval-moment kernel (fixed per context)
+    int search_path;                     // 0 auto, 1 candidate scoring, 2 interval moments
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
     qp_qparams_t* d_tmp_qp;
     unsigned long long launches;         // kernels launched through this context (host count)
@@ -197,6 +218,8 @@ int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_
 int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats, int bits,
                          int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                          qp_qparams_t* d_qp_out, cudaStream_t s);
+int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
+                                  int bits, int steps, cudaStream_t s);
 int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
                               qp_qparams_t* d_qp_out, cudaStream_t s);
 int32_t qp_launch_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, const qp_qparams_t* d_qp,

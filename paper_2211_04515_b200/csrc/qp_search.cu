@@ -232,6 +232,7 @@ __global__ void __launch_bounds__(QP_THREADS) eval_kernel(const T* __restrict__ 
 // --------------------------------------------------------------------- finalize
 
 __global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __restrict__ sums, int chunks, int steps,
+                                                              int from_sums,
                                                               int nb, int bits, const int* __restrict__ valid,
                                                               const float4* __restrict__ cand,
                                                               const qp_ds_setup* __restrict__ setup,
@@ -240,7 +241,7 @@ __global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __re
                                                               unsigned* __restrict__ status)
 {
     const qp_ds_setup s = *setup;
-    for (int k = threadIdx.x; k <= steps; k += QP_THREADS) {
+    for (int k = threadIdx.x; from_sums && k <= steps; k += QP_THREADS) {
         const int g = k / K, j = k % K;
         double t = 0.0;
         for (int b = 0; b < chunks; ++b) t += sums[((size_t)g * chunks + b) * K + j];
@@ -300,13 +301,8 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     int rep_shift = 5;
     while (rep_shift > 0 && ((size_t)nb << rep_shift) * sizeof(unsigned) > 64 * 1024) --rep_shift;
     const size_t sh_bytes = ((size_t)nb << rep_shift) * sizeof(unsigned);
-    static bool attr_set[2] = {false, false};
-    const int ti = sizeof(T) == 4 ? 0 : 1;
-    if (!attr_set[ti]) {
-        if (cudaFuncSetAttribute(hist_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
-            return qp_check_launch(ctx, "qp_dsaciq_search (histogram attribute)");
-        attr_set[ti] = true;
-    }
+    if (cudaFuncSetAttribute(hist_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, 64 * 1024) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_dsaciq_search (histogram attribute)");
     const uint64_t per_block = (uint64_t)QP_THREADS * 2 * qp_span<T>::EPV;
     uint64_t want = (n + per_block - 1) / per_block;
     const uint64_t hcap = (uint64_t)ctx->sm_count * 3;
@@ -318,6 +314,19 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
                                           ctx->d_setup);
 
     const int ncand = steps + 1;
+    // interval-moment scoring where its tables fit and its fixed-point sums cannot overflow
+    const bool iv_fits = ncand * ((1 << bits) - 1) + QP_IV_CELLS - 1 <= QP_IV_MAXB &&
+                         n / (uint64_t)ctx->iv_blocks + 65536 < (1ull << 22);
+    const bool use_iv = iv_fits && (ctx->search_path == QP_SEARCH_INTERVALS ||
+                                    (ctx->search_path == QP_SEARCH_AUTO && n >= (1ull << 20)));
+    if (use_iv) {
+        const int32_t rc = qp_launch_interval_search(ctx, x, sizeof(T) == 4 ? QP_F32 : QP_BF16, n, d_stats, bits, steps, s);
+        if (rc != QP_OK) return rc;
+        finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, 0, steps, 0, nb, bits, ctx->d_valid, ctx->d_cand,
+                                                 ctx->d_setup, ctx->d_curve, d_out, d_qp_out, ctx->d_status);
+        ctx->launches += 3;
+        return qp_check_launch(ctx, "qp_dsaciq_search");
+    }
     const int groups = (ncand + K - 1) / K;
     const uint64_t per_chunk = (uint64_t)QP_THREADS * 8;
     want = (n + per_chunk - 1) / per_chunk;
@@ -326,7 +335,7 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     if (ccap * groups > QP_MAX_BLOCKS) ccap = QP_MAX_BLOCKS / groups;
     const int chunks = (int)(want < 1 ? 1 : (want > ccap ? ccap : want));
     eval_kernel<T><<<dim3(groups, chunks), QP_THREADS, 0, s>>>(x, n, d_stats, ctx->d_cand, ncand, ctx->d_sums);
-    finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, chunks, steps, nb, bits, ctx->d_valid, ctx->d_cand,
+    finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, chunks, steps, 1, nb, bits, ctx->d_valid, ctx->d_cand,
                                              ctx->d_setup, ctx->d_curve, d_out, d_qp_out, ctx->d_status);
     ctx->launches += 4;
     return qp_check_launch(ctx, "qp_dsaciq_search");

@@ -9,6 +9,7 @@
 // counter, no waiting) merges all partials in index order, so results do not depend on
 // block scheduling.
 #include "qp_internal.cuh"
+#include "qp_stream.cuh"
 
 namespace {
 
@@ -220,6 +221,212 @@ __global__ void __launch_bounds__(QP_THREADS) stats_pass_b(const T* __restrict__
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Streamed versions for 16-byte aligned tensors: tiles of 16 KB arrive in shared memory
+// through the bulk-copy ring (qp_stream.cuh), 4 stages per block, so about 190 KB per SM are
+// in flight whatever the consumers are doing.  Same arithmetic and merge as above.  Pass B
+// walks the tiles in the opposite direction to pass A, so it starts on the part of the
+// tensor that pass A left in L2.
+
+constexpr int ST_TILE = 16384;
+constexpr int ST_STAGES = 4;
+constexpr int ST_BLOCKS_PER_SM = 3;
+
+template <typename T>
+__device__ __forceinline__ void lds_vec(const unsigned char* p, float (&v)[qp_span<T>::EPV])
+{
+    if constexpr (sizeof(T) == 4) {
+        const float4 a = *reinterpret_cast<const float4*>(p);
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+    } else {
+        const uint4 a = *reinterpret_cast<const uint4*>(p);
+        v[0] = __uint_as_float(a.x << 16); v[1] = __uint_as_float(a.x & 0xFFFF0000u);
+        v[2] = __uint_as_float(a.y << 16); v[3] = __uint_as_float(a.y & 0xFFFF0000u);
+        v[4] = __uint_as_float(a.z << 16); v[5] = __uint_as_float(a.z & 0xFFFF0000u);
+        v[6] = __uint_as_float(a.w << 16); v[7] = __uint_as_float(a.w & 0xFFFF0000u);
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(QP_THREADS) stats_stream_a(const T* __restrict__ x, uint64_t n, uint64_t ntiles,
+                                                             qp_stats_partial* __restrict__ part,
+                                                             unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out,
+                                                             unsigned* __restrict__ status)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    constexpr int EPV = qp_span<T>::EPV;
+    constexpr int VPT = ST_TILE / 16 / QP_THREADS;           // 16-byte vectors per thread and tile (4)
+    const float inf = __int_as_float(0x7F800000);
+    AccA acc = {0.0, 0.0, (double)inf, (double)-inf, 0ull};
+    float tmn = inf, tmx = -inf;                             // exact in fp32: kept out of the fp64 path
+
+    qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
+        reinterpret_cast<const unsigned char*>(x), ntiles, false, ring, status,
+        [&](const unsigned char* tile, uint64_t) {
+            float e[VPT][EPV];
+#pragma unroll
+            for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * QP_THREADS + threadIdx.x) * 16, e[u]);
+            float s = 0.f, sa = 0.f, mn = inf, mx = -inf;
+#pragma unroll
+            for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                for (int i = 0; i < EPV; ++i) {
+                    s += e[u][i];
+                    sa += fabsf(e[u][i]);
+                    mn = fminf(mn, e[u][i]);
+                    mx = fmaxf(mx, e[u][i]);
+                }
+            if (sa < inf) {
+                acc.s += (double)s;
+                acc.sa += (double)sa;
+                tmn = fminf(tmn, mn);
+                tmx = fmaxf(tmx, mx);
+            } else {
+#pragma unroll
+                for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) acc.add_scalar(e[u][i]);
+            }
+        });
+    acc.mn = fmin(acc.mn, (double)tmn);
+    acc.mx = fmax(acc.mx, (double)tmx);
+    if (blockIdx.x == 0) {                                   // elements after the last whole tile
+        const uint64_t t0 = ntiles * (ST_TILE / sizeof(T));
+        for (uint64_t i = t0 + threadIdx.x; i < n; i += QP_THREADS) acc.add_scalar(qp_load_one(x + i));
+    }
+
+    __shared__ double sh[QP_THREADS / 32];
+    __shared__ bool last;
+    const double bs = qp_block_sum(acc.s, sh);
+    const double bsa = qp_block_sum(acc.sa, sh);
+    const double bmn = qp_block_min(acc.mn, sh);
+    const double bmx = qp_block_max(acc.mx, sh);
+    const double bbad = qp_block_sum((double)acc.bad, sh);
+    if (threadIdx.x == 0) {
+        qp_stats_partial p;
+        p.s0 = bs; p.s1 = bsa; p.mn = bmn; p.mx = bmx; p.bad = (unsigned long long)bbad; p.pad = 0;
+        part[blockIdx.x] = p;
+        __threadfence();
+        last = (atomicAdd(&ticket[0], 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    double s = 0.0, sa = 0.0, mn = (double)inf, mx = (double)-inf, bad = 0.0;
+    for (unsigned b = threadIdx.x; b < gridDim.x; b += QP_THREADS) {
+        s += __ldcg(&part[b].s0);
+        sa += __ldcg(&part[b].s1);
+        mn = fmin(mn, __ldcg(&part[b].mn));
+        mx = fmax(mx, __ldcg(&part[b].mx));
+        bad += (double)__ldcg(&part[b].bad);
+    }
+    s = qp_block_sum(s, sh);
+    sa = qp_block_sum(sa, sh);
+    mn = qp_block_min(mn, sh);
+    mx = qp_block_max(mx, sh);
+    bad = qp_block_sum(bad, sh);
+    if (threadIdx.x == 0) {
+        const unsigned long long nbad = (unsigned long long)bad;
+        const unsigned long long nf = n - nbad;
+        out->n = n;
+        out->nonfinite = nbad;
+        out->mean = nf ? s / (double)nf : 0.0;
+        out->mean_abs = nf ? sa / (double)nf : 0.0;
+        out->min = nf ? mn : 0.0;
+        out->max = nf ? mx : 0.0;
+        out->mad = 0.0;
+        out->var = 0.0;
+        if (nbad) atomicOr(status, QP_DEV_NONFINITE);
+        ticket[0] = 0;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict__ x, uint64_t n, uint64_t ntiles,
+                                                             qp_stats_partial* __restrict__ part,
+                                                             unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out,
+                                                             unsigned* __restrict__ status)
+{
+    extern __shared__ __align__(128) unsigned char ring[];
+    constexpr int EPV = qp_span<T>::EPV;
+    constexpr int VPT = ST_TILE / 16 / QP_THREADS;
+    const double mean = out->mean;
+    const bool guard = out->nonfinite != 0;
+    const float m_hi = (float)mean;
+    const float m_lo = (float)(mean - (double)m_hi);
+    double sd = 0.0, sv = 0.0;
+    auto one = [&](float e, float& d1, float& d2) {
+        const float d = __fsub_rn(__fsub_rn(e, m_hi), m_lo);
+        if (!guard || qp_is_finite(e)) {
+            d1 += fabsf(d);
+            d2 = fmaf(d, d, d2);
+        }
+    };
+    qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
+        reinterpret_cast<const unsigned char*>(x), ntiles, true, ring, status,
+        [&](const unsigned char* tile, uint64_t) {
+            float e[VPT][EPV];
+#pragma unroll
+            for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * QP_THREADS + threadIdx.x) * 16, e[u]);
+            float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+            for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                for (int i = 0; i < EPV; ++i) one(e[u][i], d1, d2);
+            sd += (double)d1;
+            sv += (double)d2;
+        });
+    if (blockIdx.x == 0) {
+        float d1 = 0.f, d2 = 0.f;
+        const uint64_t t0 = ntiles * (ST_TILE / sizeof(T));
+        for (uint64_t i = t0 + threadIdx.x; i < n; i += QP_THREADS) one(qp_load_one(x + i), d1, d2);
+        sd += (double)d1;
+        sv += (double)d2;
+    }
+    __shared__ double sh[QP_THREADS / 32];
+    __shared__ bool last;
+    const double bsd = qp_block_sum(sd, sh);
+    const double bsv = qp_block_sum(sv, sh);
+    if (threadIdx.x == 0) {
+        part[blockIdx.x].s0 = bsd;
+        part[blockIdx.x].s1 = bsv;
+        __threadfence();
+        last = (atomicAdd(&ticket[1], 1u) == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    double a = 0.0, b = 0.0;
+    for (unsigned k = threadIdx.x; k < gridDim.x; k += QP_THREADS) {
+        a += __ldcg(&part[k].s0);
+        b += __ldcg(&part[k].s1);
+    }
+    a = qp_block_sum(a, sh);
+    b = qp_block_sum(b, sh);
+    if (threadIdx.x == 0) {
+        const unsigned long long nf = n - out->nonfinite;
+        out->mad = nf ? a / (double)nf : 0.0;
+        out->var = nf ? b / (double)nf : 0.0;
+        ticket[1] = 0;
+    }
+}
+
+template <typename T>
+int32_t launch_streamed(qp_ctx* ctx, const T* x, uint64_t n, uint64_t ntiles, qp_stats_t* d_out, cudaStream_t s)
+{
+    constexpr size_t smem = qp_stream::ring_bytes<ST_TILE, ST_STAGES>();
+    // per device, cheap: done on every call so that every device the process uses is covered
+    if (cudaFuncSetAttribute(stats_stream_a<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
+        cudaFuncSetAttribute(stats_stream_b<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_stats (shared memory attribute)");
+    const uint64_t cap = (uint64_t)ctx->sm_count * ST_BLOCKS_PER_SM;
+    const int blocks = (int)(ntiles > cap ? cap : ntiles);
+    stats_stream_a<T><<<blocks, QP_THREADS, smem, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
+    stats_stream_b<T><<<blocks, QP_THREADS, smem, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
+    ctx->launches += 2;
+    return qp_check_launch(ctx, "qp_stats");
+}
+
 template <typename T>
 int32_t launch_typed(qp_ctx* ctx, const T* x, uint64_t n, qp_stats_t* d_out, cudaStream_t s)
 {
@@ -241,6 +448,11 @@ int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_
     if (n == 0) {
         if (cudaMemsetAsync(d_out, 0, sizeof(qp_stats_t), s) != cudaSuccess) return qp_check_launch(ctx, "qp_stats");
         return QP_OK;
+    }
+    const uint64_t ntiles = ((uintptr_t)d_x & 15u) ? 0 : n * (dtype == QP_F32 ? 4 : 2) / ST_TILE;
+    if (ntiles >= 8) {                        // aligned and large enough for the streamed kernels to pay
+        if (dtype == QP_F32) return launch_streamed<float>(ctx, static_cast<const float*>(d_x), n, ntiles, d_out, s);
+        return launch_streamed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, ntiles, d_out, s);
     }
     if (dtype == QP_F32) return launch_typed<float>(ctx, static_cast<const float*>(d_x), n, d_out, s);
     return launch_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_out, s);

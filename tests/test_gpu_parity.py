@@ -252,9 +252,17 @@ def test_aciq_device_chain(ctx, bits):
 
 # ------------------------------------------------------------ directed search
 
-def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e-6):
+BOTH_PATHS = [qp.QP_SEARCH_CANDIDATES, qp.QP_SEARCH_INTERVALS]
+
+
+def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e-6, tie_rtol=1e-6,
+                 path=qp.QP_SEARCH_AUTO):
     d_stats = ctx.qp_stats(d_x)
-    d_res, d_qp = ctx.qp_dsaciq_search(d_x, d_stats, bits, bmode, steps, nb)
+    ctx.qp_set_search_path(path)
+    try:
+        d_res, d_qp = ctx.qp_dsaciq_search(d_x, d_stats, bits, bmode, steps, nb)
+    finally:
+        ctx.qp_set_search_path(qp.QP_SEARCH_AUTO)
     res, got_qp = ctx.read_ds_result(d_res), ctx.read_qparams(d_qp)
     curve = np.array(ctx.qp_dsaciq_curve(steps))
     st_o = oracle.stats(x_np)
@@ -267,7 +275,7 @@ def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e
     fin = np.isfinite(curve_o)
     assert np.array_equal(np.isfinite(curve), fin)
     assert np.all(np.abs(curve[fin] - curve_o[fin]) <= curve_rtol * curve_o[fin] + 1e-300)
-    near_tie = curve_o[res.k_star] <= res_o.mse_star * (1 + 1e-6)
+    near_tie = curve_o[res.k_star] <= res_o.mse_star * (1 + tie_rtol)
     assert res.k_star == res_o.k_star or near_tie, (res.k_star, res_o.k_star)
     if res.k_star == res_o.k_star:
         assert abs(res.alpha_star - res_o.alpha_star) <= 1e-4 * abs(res_o.alpha_star)
@@ -278,51 +286,78 @@ def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e
     return res, res_o
 
 
+@pytest.mark.parametrize("path", BOTH_PATHS)
 @pytest.mark.parametrize("bits", [1, 2, 3, 4, 5, 6, 7, 8])
-def test_search_c1(ctx, bits):
+def test_search_c1(ctx, bits, path):
     x = si.config_tensor("c1").reshape(-1)
     d = dev(x)
-    check_search(ctx, x, d, bits)
+    check_search(ctx, x, d, bits, path=path)
     first = ctx.qp_dsaciq_curve(100)
-    check_search(ctx, x, d, bits)
-    assert ctx.qp_dsaciq_curve(100) == first          # fixed merge order: bit-reproducible
+    check_search(ctx, x, d, bits, path=path)
+    assert ctx.qp_dsaciq_curve(100) == first          # fixed merge order / integer sums: bit-reproducible
 
 
+@pytest.mark.parametrize("path", BOTH_PATHS)
 @pytest.mark.parametrize("nb", [1, 64, 256, 2048, 16384])
-def test_search_hist_bins_and_modes(ctx, nb):
+def test_search_hist_bins_and_modes(ctx, nb, path):
     x = si.vit_activation((4, 197, 256), 2, outlier_frac=0.02).reshape(-1)
     d = dev(x)
-    check_search(ctx, x, d, 2, nb=nb)
-    check_search(ctx, x, d, 4, bmode=1, nb=nb)
+    check_search(ctx, x, d, 2, nb=nb, path=path)
+    check_search(ctx, x, d, 4, bmode=1, nb=nb, path=path)
 
 
+@pytest.mark.parametrize("path", BOTH_PATHS)
 @pytest.mark.parametrize("steps", [1, 7, 8, 9, 100, 250, 1023])
-def test_search_steps(ctx, steps):
+def test_search_steps(ctx, steps, path):
     x = si.vit_activation((1, 64, 192), 5).reshape(-1)
-    check_search(ctx, x, dev(x), 3, steps=steps)
+    check_search(ctx, x, dev(x), 3, steps=steps, path=path)    # 1023 steps: the interval tables do not fit, falls back
+    check_search(ctx, x, dev(x), 1, steps=steps, path=path)
 
 
+@pytest.mark.parametrize("path", BOTH_PATHS)
 @pytest.mark.parametrize("n", [1, 5, 33, 1000, 4099, 100003])
-def test_search_ragged_misaligned_nonfinite(ctx, n):
+def test_search_ragged_misaligned_nonfinite(ctx, n, path):
     x = si.vit_activation((1, n + 2, 1), 60 + n % 5).reshape(-1).astype(np.float32)
     d = dev(x)
     for off in (0, 1):
         if n > 1:
-            check_search(ctx, x[off:off + n], d[off:off + n], 2)
+            check_search(ctx, x[off:off + n], d[off:off + n], 2, path=path)
     if n >= 1000:
         x[[3, n // 2]] = [np.nan, np.inf]
-        check_search(ctx, x[:n], dev(x[:n]), 4)
+        check_search(ctx, x[:n], dev(x[:n]), 4, path=path)
         ctx.qp_get_status()
+
+
+@pytest.mark.parametrize("path", BOTH_PATHS)
+def test_search_large_offset_and_outliers(ctx, path):
+    """Mean far from zero (few floats per grid cell) and heavy outliers on both sides."""
+    # At |mean| = 4096 one fp32 ulp of a clip end is 4.9e-4, i.e. ~1e-4 of the clip width: the
+    # statistics of the two sides agree to ~1e-9 relative, which is enough to round an end of
+    # some candidate to the neighbouring float and move that candidate's MSE by ~1e-4.  The
+    # comparison is therefore made at 1e-3 here; everywhere else it is 2e-6.
+    big = (np.float32(4096.0) + si.flat_iid(200000, 3, "normal")).astype(np.float32)
+    check_search(ctx, big, dev(big), 2, path=path, curve_rtol=1e-3, tie_rtol=1e-3)
+    check_search(ctx, big, dev(big), 4, nb=2048, path=path, curve_rtol=1e-3, tie_rtol=1e-3)
+    x = si.vit_activation((2, 197, 512), 2, outlier_frac=0.03).reshape(-1)
+    x[::1000] *= -50.0
+    for bits in (1, 2, 3, 4):
+        check_search(ctx, x, dev(x), bits, path=path)
 
 
 def test_search_degenerate_and_errors(ctx):
     c = np.full(5000, 2.5, dtype=np.float32)
     d = dev(c)
     d_stats = ctx.qp_stats(d)
-    d_res, d_qp = ctx.qp_dsaciq_search(d, d_stats, 2)
-    res, q = ctx.read_ds_result(d_res), ctx.read_qparams(d_qp)
-    assert res.k_star == 0 and res.b_star == 0.0 and res.mse_star == 0.0 and q.flags == 1
-    assert ctx.qp_get_status() & qp.QP_DEV_DEGENERATE
+    for path in BOTH_PATHS:
+        ctx.qp_set_search_path(path)
+        d_res, d_qp = ctx.qp_dsaciq_search(d, d_stats, 2)
+        res, q = ctx.read_ds_result(d_res), ctx.read_qparams(d_qp)
+        assert res.k_star == 0 and res.b_star == 0.0 and res.mse_star == 0.0 and q.flags == 1
+        assert ctx.qp_get_status() & qp.QP_DEV_DEGENERATE
+        two = np.array([1.0, 1.0, 1.0, 3.0], dtype=np.float32)          # two distinct values
+        check_search(ctx, two, dev(two), 2, path=path)
+        ctx.qp_get_status()
+    ctx.qp_set_search_path(qp.QP_SEARCH_AUTO)
     packed = ctx.qp_quantize_pack(d, 2, d_qp)
     assert not packed.cpu().numpy().any()
     assert np.array_equal(ctx.qp_unpack_dequantize(packed, c.size, 2, d_qp).cpu().numpy(), c)
@@ -333,12 +368,13 @@ def test_search_degenerate_and_errors(ctx):
             ctx.qp_dsaciq_search(d, d_stats, kw["bits"], 0, kw["steps"], kw["hist_bins"])
 
 
-def test_search_bf16(ctx):
+@pytest.mark.parametrize("path", BOTH_PATHS)
+def test_search_bf16(ctx, path):
     x = si.vit_activation((4, 197, 128), 8).reshape(-1)
     h = si.to_bf16_bits(x)
     d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
-    check_search(ctx, oracle.widen_bf16(h), d, 2)
-    check_search(ctx, oracle.widen_bf16(h[1:-2]), d[1:-2], 4)
+    check_search(ctx, oracle.widen_bf16(h), d, 2, path=path)
+    check_search(ctx, oracle.widen_bf16(h[1:-2]), d[1:-2], 4, path=path)
 
 
 # ----------------------------------------------------- full-size configurations
@@ -355,7 +391,9 @@ def test_full_size_configs(ctx, name):
     check_stats(ctx.read_stats(ctx.qp_stats(d)), st_o)
     ds_bits = [b for b in cfg["bits"] if b <= 4] if name != "c4" else [2]
     for bits in ds_bits:
-        res, res_o = check_search(ctx, x, d, bits)
+        res, res_o = check_search(ctx, x, d, bits)                  # automatic choice: interval moments at this size
+    if name == "c2":
+        check_search(ctx, x, d, 2, path=qp.QP_SEARCH_CANDIDATES)    # and the candidate-scoring kernel at full size
     for bits in cfg["bits"]:
         _, _, qp_o = oracle.aciq_alpha(st_o, bits)
         qp_h = to_qp(qp_o)
