@@ -82,8 +82,8 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     const size_t o_ivbb = off;   off = align_up(off + sizeof(float) * (QP_IV_MAXB + 1), 256);
     const size_t o_ivedge = off; off = align_up(off + sizeof(float) * (QP_IV_CELLS + 1), 256);
     const size_t o_ivfirst = off; off = align_up(off + sizeof(unsigned) * (QP_IV_CELLS + 2), 256);
-    const size_t o_ivpart = off; off = align_up(off + sizeof(ulonglong2) * (size_t)c->iv_blocks * (QP_IV_MAXB + 1), 256);
-    const size_t o_ivouter = off; off = align_up(off + sizeof(double) * 8 * c->iv_blocks, 256);
+    const size_t o_ivpart = off; off = align_up(off + sizeof(unsigned long long) * (size_t)c->iv_blocks * (QP_IV_MAXB + 1), 256);
+    const size_t o_ivouter = off; off = align_up(off + sizeof(double) * 8 * (c->iv_blocks + 1), 256);
     const size_t o_ivtot = off;  off = align_up(off + sizeof(qp_iv_total) * (QP_IV_MAXB + 1), 256);
     const size_t o_tstats = off; off = align_up(off + sizeof(qp_stats_t), 256);
     const size_t o_tqp = off;    off = align_up(off + sizeof(qp_qparams_t), 256);
@@ -108,7 +108,7 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     c->d_iv_bb = reinterpret_cast<float*>(b + o_ivbb);
     c->d_iv_edges = reinterpret_cast<float*>(b + o_ivedge);
     c->d_iv_first = reinterpret_cast<unsigned*>(b + o_ivfirst);
-    c->d_iv_part = reinterpret_cast<ulonglong2*>(b + o_ivpart);
+    c->d_iv_part = reinterpret_cast<unsigned long long*>(b + o_ivpart);
     c->d_iv_outer = reinterpret_cast<double*>(b + o_ivouter);
     c->d_iv_tot = reinterpret_cast<qp_iv_total*>(b + o_ivtot);
     c->d_tmp_stats = reinterpret_cast<qp_stats_t*>(b + o_tstats);

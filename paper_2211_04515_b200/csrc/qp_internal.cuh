@@ -35,9 +35,9 @@ struct qp_ds_setup {                     // written by the search's set-up kerne
 constexpr int QP_IV_CELLS = 2048;        // uniform cells over [g_lo, g_hi]
 constexpr int QP_IV_MAXB = 4096;         // most interval boundaries (candidate thresholds + cell edges)
 constexpr int QP_IV_THREADS = 512;
-constexpr int QP_IV_BLOCKS_PER_SM = 2;
+constexpr int QP_IV_BLOCKS_PER_SM = 3;
 
-struct qp_iv_total { unsigned long long n, s1, s2; };   // per interval: count, sum d, sum d^2 (fixed point)
+struct qp_iv_total { unsigned long long n, s1; };       // per interval: count, sum of offsets (fixed point)
 
 struct qp_ctx {
     int device;
@@ -55,9 +55,9 @@ struct qp_ctx {
     float* d_iv_bnd;                     // [QP_IV_MAXB] unsorted boundaries
     float* d_iv_bb;                      // [QP_IV_MAXB + 1] g_lo followed by the sorted boundaries
     float* d_iv_edges;                   // [QP_IV_CELLS + 1] left edge of every cell
-    unsigned* d_iv_first;                // [QP_IV_CELLS + 2] first interval of every cell; last entry = boundary count
-    ulonglong2* d_iv_part;               // [blocks][QP_IV_MAXB + 1] per-block (count<<40 | sum d, sum d^2)
-    double* d_iv_outer;                  // [blocks][8] sums over the elements outside [g_lo, g_hi]
+    unsigned* d_iv_first;                // [0]: number of finite boundaries m
+    unsigned long long* d_iv_part;       // [blocks][QP_IV_MAXB + 1] per-block count << 40 | sum of offsets
+    double* d_iv_outer;                  // [blocks + 1][8] per-block sums that need no interval, then their totals
     qp_iv_total* d_iv_tot;               // [QP_IV_MAXB + 1]
     int iv_blocks;                       // blocks of the interval-moment kernel (fixed per context)
     int search_path;                     // 0 auto, 1 candidate scoring, 2 interval moments

@@ -250,11 +250,14 @@ __global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __re
         curve[k] = mse;
     }
     __syncthreads();
+    __shared__ double s_curve[QP_MAX_STEPS + 1];
+    for (int k = threadIdx.x; k <= steps; k += QP_THREADS) s_curve[k] = curve[k];
+    __syncthreads();
     if (threadIdx.x == 0) {
         int best = 0;
-        double best_mse = curve[0];
+        double best_mse = s_curve[0];
         for (int k = 1; k <= steps; ++k)
-            if (curve[k] < best_mse) { best_mse = curve[k]; best = k; }
+            if (s_curve[k] < best_mse) { best_mse = s_curve[k]; best = k; }
         const double b_star = s.b_e + (double)best * (s.b_r - s.b_e) / (double)steps;
         if (out) {
             out->b_e = s.b_e;
@@ -262,7 +265,7 @@ __global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __re
             out->b_star = b_star;
             out->alpha_e = s.F * s.b_e;
             out->alpha_star = s.F * b_star;
-            out->mse_e = curve[0];
+            out->mse_e = s_curve[0];
             out->mse_star = best_mse;
             out->k_star = best;
             out->steps = steps;

@@ -61,41 +61,53 @@ __device__ __forceinline__ float first_true(float lo_x, float hi_x, P pred)
 
 // ------------------------------------------------------------------ grid + boundaries
 
-// one block: the grid that covers all valid candidates, and the fixed-point unit
-__global__ void iv_grid_kernel(const float4* __restrict__ cand, const int* __restrict__ valid, int ncand,
-                               qp_ds_setup* __restrict__ setup)
-{
-    if (threadIdx.x != 0) return;
-    float lo = cand[0].x, hi = cand[0].y;
-    for (int k = 1; k < ncand; ++k)
-        if (valid[k]) { lo = fminf(lo, cand[k].x); hi = fmaxf(hi, cand[k].y); }
-    const double width = (double)hi - (double)lo;
-    float inv_gw = 0.f;
-    double u = 1.0;
-    if (width > 0.0) {
-        inv_gw = (float)((double)G / width);
-        int e;
-        frexp(width / (double)G, &e);               // cell width in (2^(e-1), 2^e]
-        u = ldexp(1.0, e - 17);                     // offsets inside a cell stay below 2^17 units
-    }
-    setup->g_lo = lo;
-    setup->g_hi = hi;
-    setup->inv_gw = inv_gw;
-    setup->u = u;
-    setup->inv_u = (float)(1.0 / u);
-}
-
-// thread t < nthr: threshold (k, j) of candidate k = t / (L-1), code j = 1 + t % (L-1);
-// thread nthr + c - 1: left edge of grid cell c = 1..G-1.  Entries that do not exist are +inf.
+// Every block first derives the grid that covers all valid candidates (block 0 stores it),
+// then: thread t < nthr finds threshold (k, j) of candidate k = t / (L-1), code
+// j = 1 + t % (L-1); thread nthr + c - 1 finds the left edge of grid cell c = 1..G-1.
+// Entries that do not exist are +inf.
 __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict__ cand, const int* __restrict__ valid,
-                                                        int ncand, int bits, const qp_ds_setup* __restrict__ setup,
+                                                        int ncand, int bits, qp_ds_setup* __restrict__ setup,
                                                         float* __restrict__ bnd, float* __restrict__ edges)
 {
+    __shared__ float s_lo[8], s_hi[8];
+    __shared__ float sg_lo, sg_hi, sg_inv;
+    const float inf = __int_as_float(0x7F800000);
+    float lo = inf, hi = -inf;
+    for (int k = threadIdx.x; k < ncand; k += 256)
+        if (k == 0 || valid[k]) { lo = fminf(lo, cand[k].x); hi = fmaxf(hi, cand[k].y); }
+    for (int o = 16; o > 0; o >>= 1) {
+        lo = fminf(lo, __shfl_down_sync(0xFFFFFFFFu, lo, o));
+        hi = fmaxf(hi, __shfl_down_sync(0xFFFFFFFFu, hi, o));
+    }
+    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); }
+        const double width = (double)hi - (double)lo;
+        float inv_gw = 0.f;
+        double u = 1.0;
+        if (width > 0.0) {
+            inv_gw = (float)((double)G / width);
+            int e;
+            frexp(width / (double)G, &e);               // cell width in [2^(e-1), 2^e)
+            u = ldexp(1.0, e - 17);                     // offsets inside a cell stay below 2^17 units
+        }
+        sg_lo = lo; sg_hi = hi; sg_inv = inv_gw;
+        if (blockIdx.x == 0) {
+            setup->g_lo = lo;
+            setup->g_hi = hi;
+            setup->inv_gw = inv_gw;
+            setup->u = u;
+            setup->inv_u = (float)(1.0 / u);
+            edges[0] = lo;
+            edges[G] = inf;
+        }
+    }
+    __syncthreads();
+    const float g_lo = sg_lo, g_hi = sg_hi, inv_gw = sg_inv;
     const int t = blockIdx.x * blockDim.x + threadIdx.x;
     const int L1 = (1 << bits) - 1;
     const int nthr = ncand * L1;
-    const float inf = __int_as_float(0x7F800000);
-    const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw;
     if (t < nthr) {
         const int k = t / L1, j = 1 + t % L1;
         float out = inf;
@@ -118,59 +130,40 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
     } else if (t < MAXB) {
         bnd[t] = inf;
     }
-    if (t == 0) { edges[0] = g_lo; edges[G] = inf; }
 }
 
-// one block of 1024 threads: bitonic sort of the MAXB boundaries, then the per-cell lookup
-__global__ void __launch_bounds__(1024) iv_sort_kernel(const float* __restrict__ bnd, const float* __restrict__ edges,
-                                                       const qp_ds_setup* __restrict__ setup, float* __restrict__ bb,
-                                                       unsigned* __restrict__ first)
+// Rank sort of the MAXB boundaries: every block holds the whole array in shared memory and
+// places 256 of its entries (rank = entries that are smaller, or equal with a lower index).
+// bb[0] = g_lo, bb[1 + r] = entry of rank r; +inf entries end up behind the finite ones.
+__global__ void __launch_bounds__(256) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
+                                                      float* __restrict__ bb)
 {
     __shared__ float s[MAXB];
-    for (int i = threadIdx.x; i < MAXB; i += 1024) s[i] = bnd[i];
+    for (int i = threadIdx.x; i < MAXB; i += 256) s[i] = bnd[i];
     __syncthreads();
-    for (int size = 2; size <= MAXB; size <<= 1)
-        for (int stride = size >> 1; stride > 0; stride >>= 1) {
-            for (int t = threadIdx.x; t < MAXB / 2; t += 1024) {
-                const int i = ((t / stride) * stride * 2) + (t % stride);
-                const int j = i + stride;
-                const bool up = ((i & size) == 0);
-                const float a = s[i], b = s[j];
-                if ((a > b) == up) { s[i] = b; s[j] = a; }
-            }
-            __syncthreads();
-        }
-    const float inf = __int_as_float(0x7F800000);
-    // bb[0] = g_lo, bb[i + 1] = i-th smallest boundary (+inf beyond the finite ones)
-    for (int i = threadIdx.x; i < MAXB; i += 1024) bb[i + 1] = s[i];
-    if (threadIdx.x == 0) bb[0] = setup->g_lo;
-    // m = number of finite boundaries.  first[c] = number of boundaries <= left edge of cell c
-    // (the edge itself included), so the intervals that meet cell c are first[c] .. first[c+1]-1;
-    // a cell whose edge does not exist (+inf) gets m + 1, which ends its left neighbour at m.
-    for (int c = threadIdx.x; c <= G + 1; c += 1024) {
-        const float e = (c <= G) ? edges[c] : inf;
-        int lo = 0, hi = MAXB;                       // count of s[i] <= e (for e = inf: the finite ones)
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            const bool le = (e == inf) ? (s[mid] < inf) : (s[mid] <= e);
-            if (le) lo = mid + 1; else hi = mid;
-        }
-        if (c <= G) first[c] = (e == inf) ? (unsigned)lo + 1u : (unsigned)lo;
-        else first[G + 1] = (unsigned)lo;
+    const int me = blockIdx.x * 256 + threadIdx.x;
+    const float v = s[me];
+    int rank = 0;
+#pragma unroll 8
+    for (int j = 0; j < MAXB; ++j) {
+        const float w = s[j];
+        rank += (w < v || (w == v && j < me)) ? 1 : 0;
     }
+    bb[1 + rank] = v;
+    if (me == 0) bb[0] = setup->g_lo;
 }
 
 // ------------------------------------------------------------------------ moments
 
 struct IvShared {
     float* bb;                      // [MAXB + 1]
-    unsigned short* first;          // [G + 1]
+    unsigned* cell;                 // [G] first interval of the cell | last interval << 16
     unsigned long long* A;          // [MAXB + 1] count << 40 | sum of offsets
-    unsigned long long* B;          // [MAXB + 1] sum of squared offsets
 };
 
 struct IvOuter {
     double s1_lo, s2_lo, s1_hi, s2_hi;
+    unsigned long long s2_in;       // sum of squared offsets of the in-grid elements (fixed point)
     unsigned n_lo, n_hi;
 };
 
@@ -186,15 +179,15 @@ __device__ __forceinline__ void iv_one(float x, const IvShared& sh, float g_lo, 
         const double d = (double)__fsub_rn(x, g_hi);
         ++o.n_hi; o.s1_hi += d; o.s2_hi += d * d;
     } else {
-        const int c = cell_of(x, g_lo, inv_gw);
-        unsigned lo = sh.first[c], hi = sh.first[c + 1] - 1u;
+        const unsigned ci = sh.cell[cell_of(x, g_lo, inv_gw)];
+        unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
         while (lo < hi) {                                   // largest i in [lo, hi] with bb[i] <= x
             const unsigned mid = (lo + hi + 1u) >> 1;
             if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
         }
         const unsigned d1 = __float2uint_rn(__fmul_rn(__fsub_rn(x, sh.bb[lo]), inv_u));
         atomicAdd(&sh.A[lo], (1ull << 40) + (unsigned long long)d1);
-        atomicAdd(&sh.B[lo], (unsigned long long)d1 * (unsigned long long)d1);
+        o.s2_in += (unsigned long long)d1 * (unsigned long long)d1;
     }
 }
 
@@ -203,24 +196,47 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
                                                                    const qp_stats_t* __restrict__ st,
                                                                    const qp_ds_setup* __restrict__ setup,
                                                                    const float* __restrict__ g_bb,
-                                                                   const unsigned* __restrict__ g_first,
-                                                                   ulonglong2* __restrict__ part,
+                                                                   const float* __restrict__ g_edges,
+                                                                   unsigned* __restrict__ g_m,
+                                                                   unsigned long long* __restrict__ part,
                                                                    double* __restrict__ outer)
 {
     extern __shared__ __align__(16) unsigned char raw[];
+    __shared__ unsigned s_m;
     IvShared sh;
     sh.A = reinterpret_cast<unsigned long long*>(raw);
-    sh.B = sh.A + (MAXB + 1);
-    sh.bb = reinterpret_cast<float*>(sh.B + (MAXB + 1));
-    sh.first = reinterpret_cast<unsigned short*>(sh.bb + (MAXB + 1));
-    const unsigned m = g_first[G + 1];                       // finite boundaries; intervals 0..m
-    for (unsigned i = threadIdx.x; i <= (unsigned)MAXB; i += QP_IV_THREADS) { sh.A[i] = 0ull; sh.B[i] = 0ull; }
-    for (unsigned i = threadIdx.x; i <= (unsigned)MAXB; i += QP_IV_THREADS) sh.bb[i] = g_bb[i];
-    for (unsigned c = threadIdx.x; c <= (unsigned)G; c += QP_IV_THREADS) sh.first[c] = (unsigned short)g_first[c];
+    sh.bb = reinterpret_cast<float*>(sh.A + (MAXB + 1));
+    sh.cell = reinterpret_cast<unsigned*>(sh.bb + (MAXB + 1));
+    const float inf = __int_as_float(0x7F800000);
+    for (unsigned i = threadIdx.x; i <= (unsigned)MAXB; i += QP_IV_THREADS) { sh.A[i] = 0ull; sh.bb[i] = g_bb[i]; }
     __syncthreads();
+    // s(j) = bb[1 + j] are the sorted boundaries.  count_le(e) = number of s(j) <= e.
+    auto count_le = [&](float e, bool finite_only) {
+        int lo = 0, hi = MAXB;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            const float v = sh.bb[1 + mid];
+            if (finite_only ? (v < inf) : (v <= e)) lo = mid + 1; else hi = mid;
+        }
+        return (unsigned)lo;
+    };
+    if (threadIdx.x == 0) s_m = count_le(inf, true);         // m finite boundaries, intervals 0..m
+    __syncthreads();
+    const unsigned m = s_m;
+    // cell c meets intervals first(c) .. first(c+1)-1, first(c) = boundaries <= left edge of c
+    // (the edge itself is one of them); a cell whose edge does not exist counts as m + 1
+    for (unsigned c = threadIdx.x; c < (unsigned)G; c += QP_IV_THREADS) {
+        const float e0 = g_edges[c], e1 = g_edges[c + 1];
+        const unsigned f0 = (e0 == inf) ? m + 1u : count_le(e0, false);
+        const unsigned f1 = (e1 == inf) ? m + 1u : count_le(e1, false);
+        sh.cell[c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
+    }
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) *g_m = m;
+
     const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw, inv_u = setup->inv_u;
     const bool guard = st->nonfinite != 0;
-    IvOuter o = {0.0, 0.0, 0.0, 0.0, 0u, 0u};
+    IvOuter o = {0.0, 0.0, 0.0, 0.0, 0ull, 0u, 0u};
 
     constexpr int EPV = qp_span<T>::EPV;
     const qp_span<T> sp(x, n);
@@ -254,44 +270,55 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     };
     if (guard) body(std::true_type{}); else body(std::false_type{});
     __syncthreads();
-    ulonglong2* mine = part + (size_t)blockIdx.x * (MAXB + 1);
-    for (unsigned i = threadIdx.x; i <= m; i += QP_IV_THREADS) mine[i] = make_ulonglong2(sh.A[i], sh.B[i]);
+    unsigned long long* mine = part + (size_t)blockIdx.x * (MAXB + 1);
+    for (unsigned i = threadIdx.x; i <= m; i += QP_IV_THREADS) mine[i] = sh.A[i];
 
     __shared__ double red[QP_IV_THREADS / 32];
     const double r0 = qp_block_sum(o.s1_lo, red), r1 = qp_block_sum(o.s2_lo, red);
     const double r2 = qp_block_sum(o.s1_hi, red), r3 = qp_block_sum(o.s2_hi, red);
     const double r4 = qp_block_sum((double)o.n_lo, red), r5 = qp_block_sum((double)o.n_hi, red);
+    const double r6 = qp_block_sum((double)o.s2_in, red);   // a thread's sum stays far below 2^53: exact
     if (threadIdx.x == 0) {
         double* dst = outer + (size_t)blockIdx.x * 8;
-        dst[0] = r0; dst[1] = r1; dst[2] = r2; dst[3] = r3; dst[4] = r4; dst[5] = r5;
+        dst[0] = r0; dst[1] = r1; dst[2] = r2; dst[3] = r3; dst[4] = r4; dst[5] = r5; dst[6] = r6;
     }
 }
 
-// totals over the blocks' partials, in block order
-__global__ void __launch_bounds__(256) iv_reduce_kernel(const ulonglong2* __restrict__ part, int blocks,
-                                                        const unsigned* __restrict__ g_first,
-                                                        qp_iv_total* __restrict__ tot)
+// totals over the blocks' partials.  grid (ceil((MAXB+1)/256), SLICES): slice s adds blocks
+// s, s + SLICES, ... and merges with integer atomics (order-independent); block (0,0) also
+// adds up the outer sums in block order.
+constexpr int IV_SLICES = 8;
+__global__ void __launch_bounds__(256) iv_reduce_kernel(const unsigned long long* __restrict__ part, int blocks,
+                                                        const unsigned* __restrict__ g_m,
+                                                        qp_iv_total* __restrict__ tot, const double* __restrict__ outer,
+                                                        double* __restrict__ outer_tot)
 {
-    const unsigned m = g_first[G + 1];
+    const unsigned m = *g_m;
     const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i > m) return;
-    unsigned long long n = 0, s1 = 0, s2 = 0;
-    for (int b = 0; b < blocks; ++b) {
-        const ulonglong2 p = part[(size_t)b * (MAXB + 1) + i];
-        n += p.x >> 40;
-        s1 += p.x & S1_MASK;
-        s2 += p.y;
+    if (i <= m) {
+        unsigned long long n = 0, s1 = 0;
+        for (int b = blockIdx.y; b < blocks; b += IV_SLICES) {
+            const unsigned long long p = part[(size_t)b * (MAXB + 1) + i];
+            n += p >> 40;
+            s1 += p & S1_MASK;
+        }
+        if (n) {
+            atomicAdd(&tot[i].n, n);
+            atomicAdd(&tot[i].s1, s1);
+        }
     }
-    qp_iv_total t;
-    t.n = n; t.s1 = s1; t.s2 = s2;
-    tot[i] = t;
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 7) {
+        double t = 0.0;
+        for (int b = 0; b < blocks; ++b) t += outer[(size_t)b * 8 + threadIdx.x];
+        outer_tot[threadIdx.x] = t;
+    }
 }
 
 // block k: squared error of candidate k from the interval moments, fixed summation order
 __global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total* __restrict__ tot,
                                                               const float* __restrict__ bb,
-                                                              const unsigned* __restrict__ g_first,
-                                                              const double* __restrict__ outer, int blocks,
+                                                              const unsigned* __restrict__ g_m,
+                                                              const double* __restrict__ outer_tot,
                                                               const float4* __restrict__ cand,
                                                               const int* __restrict__ valid, int bits,
                                                               const qp_ds_setup* __restrict__ setup,
@@ -305,7 +332,7 @@ __global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total*
     }
     const float4 q = cand[k];
     const unsigned mask = (1u << bits) - 1u;
-    const unsigned m = g_first[G + 1];
+    const unsigned m = *g_m;
     const double u = setup->u;
     auto level = [&](float r) {      // reconstruction level that candidate k assigns to r
         const unsigned c = qp_code(r, q.x, q.y, q.w, mask);
@@ -313,21 +340,19 @@ __global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total*
     };
     double acc = 0.0;
     for (unsigned i = threadIdx.x; i <= m; i += QP_THREADS) {
-        const qp_iv_total t = tot[i];
-        if (t.n == 0) continue;
+        const unsigned long long n_i = tot[i].n;
+        if (n_i == 0) continue;
         const float r = bb[i];
         const double a = level(r) - (double)r;
-        acc += (double)t.n * a * a - 2.0 * a * ((double)t.s1 * u) + (double)t.s2 * (u * u);
+        acc += (double)n_i * a * a - 2.0 * a * ((double)tot[i].s1 * u);
     }
     double total = qp_block_sum(acc, red);
     if (threadIdx.x == 0) {
-        double s1_lo = 0, s2_lo = 0, s1_hi = 0, s2_hi = 0, n_lo = 0, n_hi = 0;
-        for (int b = 0; b < blocks; ++b) {
-            const double* o = outer + (size_t)b * 8;
-            s1_lo += o[0]; s2_lo += o[1]; s1_hi += o[2]; s2_hi += o[3]; n_lo += o[4]; n_hi += o[5];
-        }
+        const double s1_lo = outer_tot[0], s2_lo = outer_tot[1], s1_hi = outer_tot[2], s2_hi = outer_tot[3];
+        const double n_lo = outer_tot[4], n_hi = outer_tot[5], s2_in = outer_tot[6];
         const double a_lo = level(setup->g_lo) - (double)setup->g_lo;      // >= 0: below every clip range
         const double a_hi = level(setup->g_hi) - (double)setup->g_hi;      // <= 0: above every clip range
+        total += s2_in * (u * u);                  // sum of squared offsets: the same for every candidate
         total += n_lo * a_lo * a_lo + 2.0 * a_lo * s1_lo + s2_lo;
         total += n_hi * a_hi * a_hi - 2.0 * a_hi * s1_hi + s2_hi;
         const unsigned long long nf = setup->n_finite;
@@ -343,20 +368,24 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     const int L1 = (1 << bits) - 1;
     const int nbnd = ncand * L1 + G - 1;
     if (nbnd > MAXB) return qp_fail(ctx, QP_ERR_INVALID_ARG, "too many boundaries for the interval path");
-    constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 8 + 4) + (size_t)(G + 1) * 2 + 16;
+    constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)G * 4 + 16;
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
-    iv_grid_kernel<<<1, 32, 0, s>>>(ctx->d_cand, ctx->d_valid, ncand, ctx->d_setup);
+    if (cudaMemsetAsync(ctx->d_iv_tot, 0, sizeof(qp_iv_total) * (MAXB + 1), s) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(ctx->d_cand, ctx->d_valid, ncand, bits, ctx->d_setup, ctx->d_iv_bnd,
                                                 ctx->d_iv_edges);
-    iv_sort_kernel<<<1, 1024, 0, s>>>(ctx->d_iv_bnd, ctx->d_iv_edges, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first);
+    iv_rank_kernel<<<MAXB / 256, 256, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb);
     const int blocks = ctx->iv_blocks;
-    iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
-                                                             ctx->d_iv_part, ctx->d_iv_outer);
-    iv_reduce_kernel<<<(MAXB + 1 + 255) / 256, 256, 0, s>>>(ctx->d_iv_part, blocks, ctx->d_iv_first, ctx->d_iv_tot);
-    iv_curve_kernel<<<ncand, QP_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, ctx->d_iv_first, ctx->d_iv_outer, blocks,
-                                                 ctx->d_cand, ctx->d_valid, bits, ctx->d_setup, ctx->d_curve);
-    ctx->launches += 6;
+    iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_edges,
+                                                             ctx->d_iv_first, ctx->d_iv_part, ctx->d_iv_outer);
+    iv_reduce_kernel<<<dim3((MAXB + 1 + 255) / 256, IV_SLICES), 256, 0, s>>>(ctx->d_iv_part, blocks, ctx->d_iv_first,
+                                                                            ctx->d_iv_tot, ctx->d_iv_outer,
+                                                                            ctx->d_iv_outer + (size_t)blocks * 8);
+    iv_curve_kernel<<<ncand, QP_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, ctx->d_iv_first,
+                                                 ctx->d_iv_outer + (size_t)blocks * 8, ctx->d_cand, ctx->d_valid, bits,
+                                                 ctx->d_setup, ctx->d_curve);
+    ctx->launches += 5;
     return qp_check_launch(ctx, "qp_dsaciq_search (interval path)");
 }
 
