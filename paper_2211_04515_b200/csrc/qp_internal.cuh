@@ -29,6 +29,8 @@ struct qp_ds_setup {                     // written by the search's set-up kerne
     float g_lo, g_hi;                    // min lo_k, max hi_k over the valid candidates
     float inv_gw;                        // QP_IV_CELLS / (g_hi - g_lo), 0 for an empty range
     float inv_u;                         // 1 / u, u = fixed-point unit of offsets inside an interval (a power of two)
+    float gw;                            // cell width (g_hi - g_lo) / QP_IV_CELLS
+    float pad2;
     double u;
 };
 

@@ -47,6 +47,15 @@ __device__ __forceinline__ int cell_of(float x, float g_lo, float inv_gw)
     return min(__float2int_rz(__fmul_rn(__fsub_rn(x, g_lo), inv_gw)), G - 1);
 }
 
+// Reference point of every interval inside cell c: half a cell below the cell's nominal
+// left edge, so that offsets x - ref are positive (between ~0.5 and ~1.5 cells) whatever the
+// rounding of the edge.  Any fixed function of c would do; it only has to be the same where
+// the moments are gathered and where they are used.
+__device__ __forceinline__ float cell_ref(int c, float g_lo, float gw)
+{
+    return fmaf((float)c - 0.5f, gw, g_lo);
+}
+
 // smallest float in (lo_x, hi_x] for which pred holds, given !pred(lo_x) and pred(hi_x), pred monotone
 template <typename P>
 __device__ __forceinline__ float first_true(float lo_x, float hi_x, P pred)
@@ -90,7 +99,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
             inv_gw = (float)((double)G / width);
             int e;
             frexp(width / (double)G, &e);               // cell width in [2^(e-1), 2^e)
-            u = ldexp(1.0, e - 17);                     // offsets inside a cell stay below 2^17 units
+            u = ldexp(1.0, e - 16);                     // offsets (up to ~1.5 cells) stay below 2^17.6 units
         }
         sg_lo = lo; sg_hi = hi; sg_inv = inv_gw;
         if (blockIdx.x == 0) {
@@ -99,6 +108,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
             setup->inv_gw = inv_gw;
             setup->u = u;
             setup->inv_u = (float)(1.0 / u);
+            setup->gw = (float)(width / (double)G);
             edges[0] = lo;
             edges[G] = inf;
         }
@@ -132,25 +142,32 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
     }
 }
 
-// Rank sort of the MAXB boundaries: every block holds the whole array in shared memory and
-// places 256 of its entries (rank = entries that are smaller, or equal with a lower index).
+// Rank sort of the MAXB boundaries.  Block b places entries [64b, 64b+64): thread t compares
+// entry 64b + (t & 63) with the 256 entries of slice t >> 6, the 16 slice counts are merged in
+// shared memory (rank = entries that are smaller, or equal with a lower index).
 // bb[0] = g_lo, bb[1 + r] = entry of rank r; +inf entries end up behind the finite ones.
-__global__ void __launch_bounds__(256) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
-                                                      float* __restrict__ bb)
+__global__ void __launch_bounds__(1024) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
+                                                       float* __restrict__ bb)
 {
     __shared__ float s[MAXB];
-    for (int i = threadIdx.x; i < MAXB; i += 256) s[i] = bnd[i];
+    __shared__ int rank[64];
+    for (int i = threadIdx.x; i < MAXB; i += 1024) s[i] = bnd[i];
+    if (threadIdx.x < 64) rank[threadIdx.x] = 0;
     __syncthreads();
-    const int me = blockIdx.x * 256 + threadIdx.x;
+    const int local = threadIdx.x & 63, slice = threadIdx.x >> 6;
+    const int me = blockIdx.x * 64 + local;
     const float v = s[me];
-    int rank = 0;
+    int cnt = 0;
+    const int j0 = slice * (MAXB / 16);
 #pragma unroll 8
-    for (int j = 0; j < MAXB; ++j) {
+    for (int j = j0; j < j0 + MAXB / 16; ++j) {
         const float w = s[j];
-        rank += (w < v || (w == v && j < me)) ? 1 : 0;
+        cnt += (w < v || (w == v && j < me)) ? 1 : 0;
     }
-    bb[1 + rank] = v;
-    if (me == 0) bb[0] = setup->g_lo;
+    atomicAdd(&rank[local], cnt);
+    __syncthreads();
+    if (threadIdx.x < 64) bb[1 + rank[threadIdx.x]] = s[blockIdx.x * 64 + threadIdx.x];
+    if (blockIdx.x == 0 && threadIdx.x == 0) bb[0] = setup->g_lo;
 }
 
 // ------------------------------------------------------------------------ moments
@@ -168,8 +185,8 @@ struct IvOuter {
 };
 
 template <bool GUARD>
-__device__ __forceinline__ void iv_one(float x, const IvShared& sh, float g_lo, float g_hi, float inv_gw, float inv_u,
-                                       IvOuter& o)
+__device__ __forceinline__ void iv_one(float x, const IvShared& sh, float g_lo, float g_hi, float inv_gw, float gw,
+                                       float inv_u, IvOuter& o)
 {
     if (GUARD && !qp_is_finite(x)) return;
     if (x < g_lo) {
@@ -179,13 +196,14 @@ __device__ __forceinline__ void iv_one(float x, const IvShared& sh, float g_lo, 
         const double d = (double)__fsub_rn(x, g_hi);
         ++o.n_hi; o.s1_hi += d; o.s2_hi += d * d;
     } else {
-        const unsigned ci = sh.cell[cell_of(x, g_lo, inv_gw)];
+        const int c = cell_of(x, g_lo, inv_gw);
+        const unsigned ci = sh.cell[c];
         unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
         while (lo < hi) {                                   // largest i in [lo, hi] with bb[i] <= x
             const unsigned mid = (lo + hi + 1u) >> 1;
             if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
         }
-        const unsigned d1 = __float2uint_rn(__fmul_rn(__fsub_rn(x, sh.bb[lo]), inv_u));
+        const unsigned d1 = __float2uint_rn(__fmul_rn(__fsub_rn(x, cell_ref(c, g_lo, gw)), inv_u));
         atomicAdd(&sh.A[lo], (1ull << 40) + (unsigned long long)d1);
         o.s2_in += (unsigned long long)d1 * (unsigned long long)d1;
     }
@@ -234,7 +252,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     __syncthreads();
     if (blockIdx.x == 0 && threadIdx.x == 0) *g_m = m;
 
-    const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw, inv_u = setup->inv_u;
+    const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw, inv_u = setup->inv_u, gw = setup->gw;
     const bool guard = st->nonfinite != 0;
     IvOuter o = {0.0, 0.0, 0.0, 0.0, 0ull, 0u, 0u};
 
@@ -250,22 +268,22 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
             qp_load_vec(xv + v * EPV, a);
             qp_load_vec(xv + (v + stride) * EPV, b);
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, g_lo, g_hi, inv_gw, inv_u, o);
+            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv_one<GD>(b[i], sh, g_lo, g_hi, inv_gw, inv_u, o);
+            for (int i = 0; i < EPV; ++i) iv_one<GD>(b[i], sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
         }
         for (; v < sp.nvec; v += stride) {
             float a[EPV];
             qp_load_vec(xv + v * EPV, a);
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, g_lo, g_hi, inv_gw, inv_u, o);
+            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
         }
         if (blockIdx.x == 0) {
             for (uint64_t i = threadIdx.x; i < sp.head; i += QP_IV_THREADS)
-                iv_one<GD>(qp_load_one(x + i), sh, g_lo, g_hi, inv_gw, inv_u, o);
+                iv_one<GD>(qp_load_one(x + i), sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
             const uint64_t t0 = sp.head + sp.nvec * EPV;
             for (uint64_t i = threadIdx.x; i < sp.tail; i += QP_IV_THREADS)
-                iv_one<GD>(qp_load_one(x + t0 + i), sh, g_lo, g_hi, inv_gw, inv_u, o);
+                iv_one<GD>(qp_load_one(x + t0 + i), sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
         }
     };
     if (guard) body(std::true_type{}); else body(std::false_type{});
@@ -287,7 +305,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
 // totals over the blocks' partials.  grid (ceil((MAXB+1)/256), SLICES): slice s adds blocks
 // s, s + SLICES, ... and merges with integer atomics (order-independent); block (0,0) also
 // adds up the outer sums in block order.
-constexpr int IV_SLICES = 8;
+constexpr int IV_SLICES = 32;
 __global__ void __launch_bounds__(256) iv_reduce_kernel(const unsigned long long* __restrict__ part, int blocks,
                                                         const unsigned* __restrict__ g_m,
                                                         qp_iv_total* __restrict__ tot, const double* __restrict__ outer,
@@ -307,10 +325,13 @@ __global__ void __launch_bounds__(256) iv_reduce_kernel(const unsigned long long
             atomicAdd(&tot[i].s1, s1);
         }
     }
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 7) {
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 7 * 32) {
+        // warp w adds up quantity w: lane l takes blocks l, l+32, ... then a fixed shuffle tree
+        const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
         double t = 0.0;
-        for (int b = 0; b < blocks; ++b) t += outer[(size_t)b * 8 + threadIdx.x];
-        outer_tot[threadIdx.x] = t;
+        for (int b = l; b < blocks; b += 32) t += outer[(size_t)b * 8 + w];
+        for (int o = 16; o > 0; o >>= 1) t += __shfl_down_sync(0xFFFFFFFFu, t, o);
+        if (l == 0) outer_tot[w] = t;
     }
 }
 
@@ -334,6 +355,7 @@ __global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total*
     const unsigned mask = (1u << bits) - 1u;
     const unsigned m = *g_m;
     const double u = setup->u;
+    const float g_lo = setup->g_lo, inv_gw = setup->inv_gw, gw = setup->gw;
     auto level = [&](float r) {      // reconstruction level that candidate k assigns to r
         const unsigned c = qp_code(r, q.x, q.y, q.w, mask);
         return (double)fmaf(__fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.0f), q.z, q.x);
@@ -342,8 +364,9 @@ __global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total*
     for (unsigned i = threadIdx.x; i <= m; i += QP_THREADS) {
         const unsigned long long n_i = tot[i].n;
         if (n_i == 0) continue;
-        const float r = bb[i];
-        const double a = level(r) - (double)r;
+        const float left = bb[i];                                   // an element of the interval: fixes its codes
+        const float r = cell_ref(cell_of(left, g_lo, inv_gw), g_lo, gw);
+        const double a = level(left) - (double)r;
         acc += (double)n_i * a * a - 2.0 * a * ((double)tot[i].s1 * u);
     }
     double total = qp_block_sum(acc, red);
@@ -375,7 +398,7 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
         return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(ctx->d_cand, ctx->d_valid, ncand, bits, ctx->d_setup, ctx->d_iv_bnd,
                                                 ctx->d_iv_edges);
-    iv_rank_kernel<<<MAXB / 256, 256, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb);
+    iv_rank_kernel<<<MAXB / 64, 1024, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb);
     const int blocks = ctx->iv_blocks;
     iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_edges,
                                                              ctx->d_iv_first, ctx->d_iv_part, ctx->d_iv_outer);
