@@ -197,7 +197,7 @@ def ours_main(args):
     max_packed = qp.qp_packed_bytes(n, 16)
     packed = torch.empty(max_packed, dtype=torch.uint8, device="cuda")
     y = torch.empty(n, dtype=torch.float32, device="cuda")
-    d_stats = torch.empty(64, dtype=torch.uint8, device="cuda")
+    d_stats = torch.empty(80, dtype=torch.uint8, device="cuda")
     d_qp = torch.empty(24, dtype=torch.uint8, device="cuda")
     d_res = torch.empty(72, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
@@ -211,10 +211,11 @@ def ours_main(args):
         if events is not None:
             marks = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
             marks[0].record()
-        ctx.qp_stats(x, out=d_stats)
+        use_ds = qp.qp_policy_use_ds(q)
+        ctx.qp_stats(x, out=d_stats, hist_bins=qp.QP_DEFAULT_HIST_BINS if use_ds else 0)
         if events is not None:
             marks[1].record()
-        if qp.qp_policy_use_ds(q):
+        if use_ds:
             ctx.qp_dsaciq_search(x, d_stats, q, out_result=d_res, out_qp=d_qp)
         else:
             ctx.qp_aciq_qparams_device(d_stats, q, out=d_qp)
@@ -235,6 +236,11 @@ def ours_main(args):
 
     for t in range(args.warmup):
         step(t)
+    seen = set()
+    for t, q in enumerate(bits_of_step):                 # one untimed step per bit-width: every kernel variant is loaded
+        if q not in seen:
+            seen.add(q)
+            step(t)
     barrier()
     assert ctx.qp_get_status() & ~qp.QP_DEV_NONFINITE == 0
 

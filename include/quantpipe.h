@@ -73,7 +73,10 @@ typedef struct {
     double mad;          /* sum|x - mean| / N  (Laplace scale about the mean)    */
     double var;          /* sum (x - mean)^2 / N                              */
     double min, max;
-} qp_stats_t;            /* 64 bytes */
+    uint64_t hist_peak;  /* largest bin count of the hist_bins-bin histogram over [min, max] */
+    int32_t hist_bins;   /* bins of that histogram; 0 = qp_stats did not compute one          */
+    int32_t reserved;
+} qp_stats_t;            /* 80 bytes */
 
 /* Uniform quantizer over the clip range [lo, hi] with L = 2^bits levels, both ends included. */
 typedef struct {
@@ -129,13 +132,20 @@ double qp_aciq_F(int bits, int dist);
  * QP_ERR_INVALID_ARG (NaN/Inf ends, NULL). */
 int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out);
 
-/* ---- a1: statistics (Sec. 3) ----------------------------------------------------------
- * One call fills *d_out (device memory, 64 bytes, 8-byte aligned) from the n elements at
+/* ---- a1 (+ a2): statistics (Sec. 3) ----------------------------------------------------
+ * One call fills *d_out (device memory, 80 bytes, 8-byte aligned) from the n elements at
  * d_x.  Two passes over x (sums/min/max, then deviations about the mean), fp64 merges in a
  * fixed order: results are bit-reproducible run to run.  n = 0 gives all-zero statistics.
+ * hist_bins > 0 asks the second pass to carry the directed search's histogram along
+ * (hist_bins equal bins over [min, max]; only its peak count is kept, in hist_peak): a later
+ * qp_dsaciq_search with the same hist_bins then skips its own histogram pass.  The fusion is
+ * done for 16-byte aligned tensors of at least 128 KB and hist_bins <= 4096; otherwise, and
+ * for hist_bins = 0, d_out->hist_bins is 0 and the search counts for itself.
  * d_x must be aligned to its element size.
- * Errors: QP_ERR_INVALID_ARG (NULL), QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
-int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream);
+ * Errors: QP_ERR_INVALID_ARG (NULL, hist_bins outside 0..QP_MAX_HIST_BINS),
+ * QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
+int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
+                 void* stream);
 
 /* Statistics for callers that cannot allocate device memory (no counterpart in the paper;
  * same results as qp_stats).  Some code may not call cudaMalloc or any allocating routine:

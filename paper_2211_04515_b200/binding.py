@@ -37,7 +37,8 @@ EXPORTS = (
 
 class Stats(C.Structure):
     _fields_ = [("n", C.c_uint64), ("nonfinite", C.c_uint64), ("mean", C.c_double), ("mean_abs", C.c_double),
-                ("mad", C.c_double), ("var", C.c_double), ("min", C.c_double), ("max", C.c_double)]
+                ("mad", C.c_double), ("var", C.c_double), ("min", C.c_double), ("max", C.c_double),
+                ("hist_peak", C.c_uint64), ("hist_bins", C.c_int32), ("reserved", C.c_int32)]
 
 
 class QParams(C.Structure):
@@ -82,7 +83,7 @@ def load() -> C.CDLL:
     L.qp_aciq_F.argtypes = [C.c_int, C.c_int]
     L.qp_aciq_F.restype = dbl
     L.qp_make_qparams.argtypes = [dbl, dbl, C.c_int, C.POINTER(QParams)]
-    L.qp_stats.argtypes = [vp, vp, C.c_int, u64, vp, vp]
+    L.qp_stats.argtypes = [vp, vp, C.c_int, u64, C.c_int, vp, vp]
     L.qp_aciq_alpha.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, dbl, C.POINTER(dbl), C.POINTER(QParams)]
     L.qp_aciq_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
     L.qp_dsaciq_search.argtypes = [vp, vp, C.c_int, u64, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
@@ -156,7 +157,7 @@ def qp_select_bits_eq2(v_bytes: float, q_t: int, s_images: float, r_images_per_s
 # ------------------------------------------------------------ device calls
 
 def qp_stats_static(x: "torch.Tensor", out: "torch.Tensor", n: int | None = None) -> int:
-    """Statistics of x into the 64-byte device buffer `out`, for callers that may not
+    """Statistics of x into the device buffer `out` (sizeof(Stats) bytes), for callers that may not
     allocate: no context, no allocation here or in the library (the caller brings `out`).
     Runs on x's device, which must be the current one, on torch's current stream.
     Returns the status code; negative codes are errors (QP_ERR_TOO_LARGE above
@@ -227,11 +228,12 @@ class Context:
         raise QuantPipeError(QP_ERR_INVALID_ARG, "qp must be a QParams struct or a device tensor")
 
     # -- a1
-    def qp_stats(self, x: torch.Tensor, out: torch.Tensor | None = None) -> torch.Tensor:
-        """Statistics of x into a 64-byte device buffer (returned)."""
+    def qp_stats(self, x: torch.Tensor, out: torch.Tensor | None = None, hist_bins: int = 0) -> torch.Tensor:
+        """Statistics of x into an 80-byte device buffer (returned); hist_bins > 0 also asks
+        for the peak of the search's histogram."""
         assert x.is_cuda and x.is_contiguous()
         out = self._bytes(C.sizeof(Stats)) if out is None else out
-        self._check(self._lib.qp_stats(self._h, x.data_ptr(), _dtype_code(x), x.numel(), out.data_ptr(),
+        self._check(self._lib.qp_stats(self._h, x.data_ptr(), _dtype_code(x), x.numel(), hist_bins, out.data_ptr(),
                                        _stream(self.device)))
         return out
 

@@ -285,15 +285,17 @@ static int32_t check_x(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n)
     return QP_OK;
 }
 
-extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, void* stream)
+extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
+                            void* stream)
 {
     int32_t rc = check_x(ctx, d_x, dtype, n);
     if (rc) return rc;
+    if (hist_bins < 0 || hist_bins > QP_MAX_HIST_BINS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "hist_bins out of range");
     if (!d_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_out");
     if ((uintptr_t)d_out & 7u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_out must be 8-byte aligned");
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
-    return qp_launch_stats(ctx, d_x, dtype, n, d_out, static_cast<cudaStream_t>(stream));
+    return qp_launch_stats(ctx, d_x, dtype, n, hist_bins, d_out, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode,
@@ -427,7 +429,7 @@ extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint6
         if (n && cudaMemcpyAsync(d_x_work, h_x, n * esz, cudaMemcpyHostToDevice, s) != cudaSuccess)
             return qp_check_launch(ctx, "qp_sender_host (copy in)");
     }
-    int32_t rc = qp_stats(ctx, d_x_work, dtype, n, ctx->d_tmp_stats, stream);
+    int32_t rc = qp_stats(ctx, d_x_work, dtype, n, use_ds ? hist_bins : 0, ctx->d_tmp_stats, stream);
     if (rc < 0) return rc;
     if (use_ds) rc = qp_dsaciq_search(ctx, d_x_work, dtype, n, ctx->d_tmp_stats, bits, bmode, steps, hist_bins, nullptr,
                                       ctx->d_tmp_qp, stream);

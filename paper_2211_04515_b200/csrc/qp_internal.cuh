@@ -216,7 +216,8 @@ __device__ __forceinline__ double qp_block_max(double v, double* sh)
 #endif  // __CUDACC__
 
 // Kernel launchers (one per translation unit).
-int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, cudaStream_t s);
+int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
+                        cudaStream_t s);
 int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats, int bits,
                          int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                          qp_qparams_t* d_qp_out, cudaStream_t s);

@@ -59,6 +59,7 @@ __global__ void __launch_bounds__(QP_THREADS) hist_kernel(const T* __restrict__ 
                                                           unsigned long long* __restrict__ hist)
 {
     extern __shared__ unsigned sh[];
+    if (st->hist_bins == nb) return;                 // the statistics already carry this histogram's peak
     const int reps = 1 << rep_shift;
     for (int i = threadIdx.x; i < nb * reps; i += QP_THREADS) sh[i] = 0u;
     __syncthreads();
@@ -86,7 +87,8 @@ __global__ void __launch_bounds__(QP_THREADS) setup_kernel(const qp_stats_t* __r
     __shared__ unsigned long long sh_top[QP_THREADS];
     __shared__ qp_ds_setup s;
     unsigned long long top = 0;
-    for (int b = threadIdx.x; b < nb; b += QP_THREADS) {
+    const bool from_stats = st->hist_bins == nb;
+    for (int b = threadIdx.x; !from_stats && b < nb; b += QP_THREADS) {
         const unsigned long long c = hist[b];
         top = c > top ? c : top;
     }
@@ -94,6 +96,7 @@ __global__ void __launch_bounds__(QP_THREADS) setup_kernel(const qp_stats_t* __r
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int i = 1; i < QP_THREADS; ++i) top = sh_top[i] > top ? sh_top[i] : top;
+        if (from_stats) top = st->hist_peak;
         const unsigned long long nf = st->n - st->nonfinite;
         const double mn = st->min, mx = st->max;
         const double b_e = bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad;

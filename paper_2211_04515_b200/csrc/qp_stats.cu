@@ -126,6 +126,9 @@ __global__ void __launch_bounds__(QP_THREADS) stats_pass_a(const T* __restrict__
         out->max = nf ? mx : 0.0;
         out->mad = 0.0;
         out->var = 0.0;
+        out->hist_peak = 0;
+        out->hist_bins = 0;
+        out->reserved = 0;
         if (nbad) atomicOr(status, QP_DEV_NONFINITE);
         ticket[0] = 0;
     }
@@ -230,7 +233,8 @@ __global__ void __launch_bounds__(QP_THREADS) stats_pass_b(const T* __restrict__
 
 constexpr int ST_TILE = 16384;
 constexpr int ST_STAGES = 4;
-constexpr int ST_BLOCKS_PER_SM = 3;
+constexpr int ST_BLOCKS_PER_SM = 2;
+constexpr int ST_FUSED_HIST_MAX = 4096;     // largest histogram that pass B carries along
 
 template <typename T>
 __device__ __forceinline__ void lds_vec(const unsigned char* p, float (&v)[qp_span<T>::EPV])
@@ -336,30 +340,53 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_a(const T* __restrict
         out->max = nf ? mx : 0.0;
         out->mad = 0.0;
         out->var = 0.0;
+        out->hist_peak = 0;
+        out->hist_bins = 0;
+        out->reserved = 0;
         if (nbad) atomicOr(status, QP_DEV_NONFINITE);
         ticket[0] = 0;
     }
 }
 
-template <typename T>
+// Pass B, optionally with the histogram of the directed search fused in (HIST): nb equal bins
+// over [min, max], bin = floor((x - min) * inv_w) in fp32 with the last bin closed, counted in
+// shared memory with one replica of every bin per lane group (no same-address contention),
+// merged into 64-bit global counters; the last block extracts the peak count.
+template <typename T, bool HIST>
 __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict__ x, uint64_t n, uint64_t ntiles,
                                                              qp_stats_partial* __restrict__ part,
                                                              unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out,
-                                                             unsigned* __restrict__ status)
+                                                             unsigned* __restrict__ status, int nb, int rep_shift,
+                                                             unsigned long long* __restrict__ hist)
 {
     extern __shared__ __align__(128) unsigned char ring[];
     constexpr int EPV = qp_span<T>::EPV;
     constexpr int VPT = ST_TILE / 16 / QP_THREADS;
+    unsigned* sh_hist = reinterpret_cast<unsigned*>(ring + qp_stream::ring_bytes<ST_TILE, ST_STAGES>());
     const double mean = out->mean;
     const bool guard = out->nonfinite != 0;
     const float m_hi = (float)mean;
     const float m_lo = (float)(mean - (double)m_hi);
+    const double dmn = out->min, dmx = out->max;
+    const bool hist_on = HIST && dmx > dmn;
+    const float mn = (float)dmn;
+    const float inv_w = hist_on ? (float)((double)nb / (dmx - dmn)) : 0.f;
+    const int lane_rep = threadIdx.x & ((1 << rep_shift) - 1);
+    if (HIST) {
+        for (int i = threadIdx.x; i < (nb << rep_shift); i += QP_THREADS) sh_hist[i] = 0u;
+        __syncthreads();
+    }
     double sd = 0.0, sv = 0.0;
     auto one = [&](float e, float& d1, float& d2) {
         const float d = __fsub_rn(__fsub_rn(e, m_hi), m_lo);
         if (!guard || qp_is_finite(e)) {
             d1 += fabsf(d);
             d2 = fmaf(d, d, d2);
+            if (HIST && hist_on) {
+                int b = __float2int_rz(__fmul_rn(__fsub_rn(e, mn), inv_w));
+                b = min(max(b, 0), nb - 1);
+                atomicAdd(&sh_hist[(b << rep_shift) + lane_rep], 1u);
+            }
         }
     };
     qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
@@ -383,6 +410,16 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
         sd += (double)d1;
         sv += (double)d2;
     }
+    if (HIST) {
+        __syncthreads();
+        const int reps = 1 << rep_shift;
+        for (int b = threadIdx.x; b < nb; b += QP_THREADS) {
+            unsigned long long c = 0;
+            for (int r = 0; r < reps; ++r) c += sh_hist[(b << rep_shift) + ((r + threadIdx.x) & (reps - 1))];
+            if (c) atomicAdd(&hist[b], c);
+        }
+        __threadfence();                          // counts are out before this block takes its ticket
+    }
     __shared__ double sh[QP_THREADS / 32];
     __shared__ bool last;
     const double bsd = qp_block_sum(sd, sh);
@@ -403,26 +440,49 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
     }
     a = qp_block_sum(a, sh);
     b = qp_block_sum(b, sh);
+    double top = 0.0;
+    if (HIST) {
+        for (int k = threadIdx.x; k < nb; k += QP_THREADS) top = fmax(top, (double)__ldcg(&hist[k]));   // counts < 2^53
+        top = qp_block_max(top, sh);
+    }
     if (threadIdx.x == 0) {
         const unsigned long long nf = n - out->nonfinite;
         out->mad = nf ? a / (double)nf : 0.0;
         out->var = nf ? b / (double)nf : 0.0;
+        if (HIST) {
+            out->hist_peak = (unsigned long long)top;
+            out->hist_bins = nb;
+        }
         ticket[1] = 0;
     }
 }
 
 template <typename T>
-int32_t launch_streamed(qp_ctx* ctx, const T* x, uint64_t n, uint64_t ntiles, qp_stats_t* d_out, cudaStream_t s)
+int32_t launch_streamed(qp_ctx* ctx, const T* x, uint64_t n, uint64_t ntiles, int hist_bins, qp_stats_t* d_out,
+                        cudaStream_t s)
 {
-    constexpr size_t smem = qp_stream::ring_bytes<ST_TILE, ST_STAGES>();
+    constexpr size_t ring = qp_stream::ring_bytes<ST_TILE, ST_STAGES>();
+    // fused histogram: as many lane replicas of each bin as fit in 16 KB of shared memory
+    const bool fuse = hist_bins >= 1 && hist_bins <= ST_FUSED_HIST_MAX;
+    int rep_shift = 5;
+    while (fuse && rep_shift > 0 && ((size_t)hist_bins << rep_shift) * sizeof(unsigned) > 16 * 1024) --rep_shift;
+    const size_t smem_b = ring + (fuse ? ((size_t)hist_bins << rep_shift) * sizeof(unsigned) : 0);
     // per device, cheap: done on every call so that every device the process uses is covered
-    if (cudaFuncSetAttribute(stats_stream_a<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess ||
-        cudaFuncSetAttribute(stats_stream_b<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(stats_stream_a<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring) != cudaSuccess ||
+        cudaFuncSetAttribute(stats_stream_b<T, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ring) != cudaSuccess ||
+        cudaFuncSetAttribute(stats_stream_b<T, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)(ring + 16 * 1024)) != cudaSuccess)
         return qp_check_launch(ctx, "qp_stats (shared memory attribute)");
+    if (fuse && cudaMemsetAsync(ctx->d_hist, 0, sizeof(unsigned long long) * hist_bins, s) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_stats (histogram reset)");
     const uint64_t cap = (uint64_t)ctx->sm_count * ST_BLOCKS_PER_SM;
     const int blocks = (int)(ntiles > cap ? cap : ntiles);
-    stats_stream_a<T><<<blocks, QP_THREADS, smem, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
-    stats_stream_b<T><<<blocks, QP_THREADS, smem, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
+    stats_stream_a<T><<<blocks, QP_THREADS, ring, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
+    if (fuse)
+        stats_stream_b<T, true><<<blocks, QP_THREADS, smem_b, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out,
+                                                                   ctx->d_status, hist_bins, rep_shift, ctx->d_hist);
+    else
+        stats_stream_b<T, false><<<blocks, QP_THREADS, ring, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out,
+                                                                  ctx->d_status, 0, 0, ctx->d_hist);
     ctx->launches += 2;
     return qp_check_launch(ctx, "qp_stats");
 }
@@ -443,7 +503,8 @@ int32_t launch_typed(qp_ctx* ctx, const T* x, uint64_t n, qp_stats_t* d_out, cud
 
 }  // namespace
 
-int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_stats_t* d_out, cudaStream_t s)
+int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
+                        cudaStream_t s)
 {
     if (n == 0) {
         if (cudaMemsetAsync(d_out, 0, sizeof(qp_stats_t), s) != cudaSuccess) return qp_check_launch(ctx, "qp_stats");
@@ -451,8 +512,9 @@ int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, qp_
     }
     const uint64_t ntiles = ((uintptr_t)d_x & 15u) ? 0 : n * (dtype == QP_F32 ? 4 : 2) / ST_TILE;
     if (ntiles >= 8) {                        // aligned and large enough for the streamed kernels to pay
-        if (dtype == QP_F32) return launch_streamed<float>(ctx, static_cast<const float*>(d_x), n, ntiles, d_out, s);
-        return launch_streamed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, ntiles, d_out, s);
+        if (dtype == QP_F32)
+            return launch_streamed<float>(ctx, static_cast<const float*>(d_x), n, ntiles, hist_bins, d_out, s);
+        return launch_streamed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, ntiles, hist_bins, d_out, s);
     }
     if (dtype == QP_F32) return launch_typed<float>(ctx, static_cast<const float*>(d_x), n, d_out, s);
     return launch_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_out, s);

@@ -82,7 +82,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity)
 
 // Shared-memory footprint of a ring (bytes, incl. barriers), for the dynamic allocation.
 template <int TILE_BYTES, int STAGES>
-constexpr size_t ring_bytes() { return (size_t)TILE_BYTES * STAGES + 8 * STAGES + 16; }
+__host__ __device__ constexpr size_t ring_bytes() { return (size_t)TILE_BYTES * STAGES + 8 * STAGES + 16; }
 
 // Streams tiles [0, ntiles) of TILE_BYTES each, starting at `base` (16-byte aligned), to
 // consume(tile_pointer_in_shared_memory, tile_index), called by every thread of the block.

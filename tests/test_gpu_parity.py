@@ -66,10 +66,23 @@ def check_stats(st, st_o):
 def test_stats_configs(ctx, name):
     x = si.config_tensor(name).reshape(-1)
     st = ctx.read_stats(ctx.qp_stats(dev(x)))
-    check_stats(st, oracle.stats(x))
+    st_o = oracle.stats(x)
+    check_stats(st, st_o)
+    assert st.hist_bins == 0
     # bit-reproducible: fixed merge order
     st2 = ctx.read_stats(ctx.qp_stats(dev(x)))
     assert bytes(st) == bytes(st2)
+    # histogram carried along by the second pass: integer-identical peak count
+    for nb in (100, 7, 2048, 4096):
+        sth = ctx.read_stats(ctx.qp_stats(dev(x), hist_bins=nb))
+        _, counts = oracle.hist_peak(x, st_o.min, st_o.max, nb)
+        assert sth.hist_bins == nb and sth.hist_peak == int(counts.max())
+        assert (sth.mean, sth.mad, sth.var) == (st.mean, st.mad, st.var)
+    assert ctx.read_stats(ctx.qp_stats(dev(x), hist_bins=8192)).hist_bins == 0      # too many bins to fuse
+    xs = dev(x)[1:]                                                                  # not 16-byte aligned: not fused
+    assert ctx.read_stats(ctx.qp_stats(xs, hist_bins=100)).hist_bins == 0
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_stats(dev(x), hist_bins=-1)
 
 
 @pytest.mark.parametrize("n", RAGGED + [262144 + 5])
@@ -91,6 +104,13 @@ def test_stats_special(ctx):
     check_stats(st, oracle.stats(x))
     assert st.nonfinite == 3
     assert ctx.qp_get_status() & qp.QP_DEV_NONFINITE
+    xl = si.flat_iid(300000, 9, "laplace")
+    xl[[5, 777, 299999]] = [np.nan, np.inf, -np.inf]
+    stl = ctx.read_stats(ctx.qp_stats(dev(xl), hist_bins=64))
+    sto = oracle.stats(xl)
+    check_stats(stl, sto)
+    assert stl.hist_peak == int(oracle.hist_peak(xl, sto.min, sto.max, 64)[1].max())
+    ctx.qp_get_status()
     c = np.full(3000, -1.5, dtype=np.float32)
     st = ctx.read_stats(ctx.qp_stats(dev(c)))
     assert (st.mean, st.mad, st.var, st.min, st.max) == (-1.5, 0.0, 0.0, -1.5, -1.5)
@@ -257,7 +277,9 @@ BOTH_PATHS = [qp.QP_SEARCH_CANDIDATES, qp.QP_SEARCH_INTERVALS]
 
 def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e-6, tie_rtol=1e-6,
                  path=qp.QP_SEARCH_AUTO):
-    d_stats = ctx.qp_stats(d_x)
+    # statistics with the histogram carried along, except when the candidate-scoring path is
+    # forced (then the search counts its own histogram): both ways are exercised
+    d_stats = ctx.qp_stats(d_x, hist_bins=0 if path == qp.QP_SEARCH_CANDIDATES else nb)
     ctx.qp_set_search_path(path)
     try:
         d_res, d_qp = ctx.qp_dsaciq_search(d_x, d_stats, bits, bmode, steps, nb)

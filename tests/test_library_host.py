@@ -32,7 +32,7 @@ def test_exports_every_declared_symbol(lib):
 
 def test_struct_layouts():
     import ctypes as C
-    assert C.sizeof(qp.Stats) == 64 and C.sizeof(qp.QParams) == 24 and C.sizeof(qp.DSResult) == 72
+    assert C.sizeof(qp.Stats) == 80 and C.sizeof(qp.QParams) == 24 and C.sizeof(qp.DSResult) == 72
     assert C.sizeof(oracle.Stats) == 64 and C.sizeof(oracle.QParams) == 24 and C.sizeof(oracle.DSResult) == 72
 
 
@@ -85,7 +85,7 @@ def test_make_qparams_bit_identical_to_oracle(lib, bits):
 def test_aciq_alpha_matches_oracle(lib):
     x = si.config_tensor("c1")
     st_o = oracle.stats(x)
-    st = qp.Stats(st_o.n, st_o.nonfinite, st_o.mean, st_o.mean_abs, st_o.mad, st_o.var, st_o.min, st_o.max)
+    st = qp.Stats(st_o.n, st_o.nonfinite, st_o.mean, st_o.mean_abs, st_o.mad, st_o.var, st_o.min, st_o.max, 0, 0, 0)
     for bits in ALL_BITS:
         for dist, bmode, ov in ((0, 0, 0.0), (0, 1, 0.0), (1, 0, 0.0), (0, 0, 0.83)):
             rc, alpha, q = qp.qp_aciq_alpha(st, bits, dist, bmode, ov)

@@ -10,6 +10,8 @@ the ordinary, context-based qp_stats within the statistics tolerance of the pari
 already run every other test; it needs nothing from them and passes alone in a fresh
 process as well.
 """
+import ctypes
+
 import numpy as np
 import pytest
 import torch
@@ -18,6 +20,8 @@ import paper_2211_04515_b200 as qp
 import synth_inputs as si
 
 pytestmark = pytest.mark.gpu
+
+STATS_BYTES = ctypes.sizeof(qp.Stats)
 
 
 def _close(a, b):
@@ -36,7 +40,7 @@ def test_static_stats_matches_context_stats_twice():
     x2_h = si.vit_activation((3, 197, 1024), 42, outlier_frac=0.01).reshape(-1)
     x2_h[[7, 1000]] = [np.nan, np.inf]                      # exercises the non-finite path and the status word
     x2 = torch.from_numpy(x2_h).cuda()[1:]                  # and a 4-byte-aligned, ragged view
-    out = torch.empty(64, dtype=torch.uint8, device="cuda")  # the caller's buffer; nothing else is needed
+    out = torch.empty(STATS_BYTES, dtype=torch.uint8, device="cuda")  # the caller's buffer; nothing else is needed
     for x in (x1, x2):                                       # two calls in a row on the shared scratch
         want = ctx.read_stats(ctx.qp_stats(x))
         out.fill_(0xEE)
@@ -56,7 +60,7 @@ def test_static_stats_matches_context_stats_twice():
 
 def test_static_stats_rejects_bad_arguments():
     x = torch.zeros(1024, device="cuda")
-    out = torch.empty(64, dtype=torch.uint8, device="cuda")
+    out = torch.empty(STATS_BYTES, dtype=torch.uint8, device="cuda")
     # beyond the stated maximum: refused before anything is enqueued or read
     assert qp.qp_stats_static(x, out, n=qp.QP_STATS_STATIC_MAX_N + 1) == qp.QP_ERR_TOO_LARGE
     assert "maximum" in qp.qp_status_string(qp.QP_ERR_TOO_LARGE)
