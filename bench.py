@@ -377,7 +377,8 @@ def ours_main(args):
 def sweep_main(args):
     """Each stage timed alone, cold: the buffers of consecutive launches rotate through more than
     4x the L2 capacity, so no launch finds its input (or output lines) in L2.  One JSON line per
-    (workload, dtype, stage, bits): median and best time of 20 launches after 5 warm-ups."""
+    (workload, dtype, stage, bits): median and best per-launch time over 5 groups of 20
+    back-to-back launches after 5 warm-ups."""
     import torch
 
     import paper_2211_04515_b200 as qp
@@ -392,18 +393,23 @@ def sweep_main(args):
         count = max(2, int(4 * L2_BYTES // max(nbytes, 1)) + 1)
         return [make() for _ in range(min(count, 64))]
 
-    def timed(fn, nbuf, reps=20, warm=5):
+    def timed(fn, nbuf, reps=20, warm=5, groups=5):
+        """Median and best per-launch time over `groups` groups of `reps` back-to-back launches
+        (events around each group, no host synchronisation inside a group, so the device never
+        waits for the host)."""
         for i in range(warm):
             fn(i % nbuf)
         torch.cuda.synchronize()
-        ts = []
-        for i in range(reps):
+        ts, k = [], warm
+        for _ in range(groups):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
-            fn((warm + i) % nbuf)
+            for _ in range(reps):
+                fn(k % nbuf)
+                k += 1
             b.record()
             b.synchronize()
-            ts.append(a.elapsed_time(b))
+            ts.append(a.elapsed_time(b) / reps)
         ts.sort()
         return ts[len(ts) // 2], ts[0]
 
