@@ -213,6 +213,82 @@ __device__ __forceinline__ double qp_block_max(double v, double* sh)
     return r;
 }
 
+// ---- pieces of the directed search shared by its two scoring paths
+
+// b_E, b_R and friends from the statistics and the histogram's peak count `top`
+__device__ inline void qp_ds_make_setup(const qp_stats_t* __restrict__ st, unsigned long long top, int nb, int bmode,
+                                        double F, qp_ds_setup& s)
+{
+    const unsigned long long nf = st->n - st->nonfinite;
+    const double mn = st->min, mx = st->max;
+    const double b_e = bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad;
+    double peak = 0.0;
+    if (mx > mn && nf > 0) {
+        const double w = (mx - mn) / (double)nb;
+        peak = (double)top / ((double)nf * w);
+    }
+    s.degenerate = !(mx > mn) || !(peak > 0.0) || !(b_e > 0.0);
+    s.b_e = b_e;
+    s.b_r = s.degenerate ? b_e : 1.0 / (2.0 * peak);
+    s.F = F;
+    s.mean = st->mean;
+    s.n_finite = nf;
+    s.pad = 0;
+}
+
+// candidate k: b_k = b_E + k (b_R - b_E) / steps, evaluated in this order in fp64; its quantizer
+__device__ inline void qp_ds_candidate(const qp_ds_setup& s, int k, int steps, int bits, float4& c, int& ok)
+{
+    const double b_k = s.b_e + (double)k * (s.b_r - s.b_e) / (double)steps;
+    ok = ((k == 0) || (!s.degenerate && b_k > 0.0)) ? 1 : 0;
+    qp_qparams_t q;
+    q.lo = q.hi = q.scale = q.inv_scale = 0.f;
+    if (ok) {
+        const double alpha = s.F * b_k;
+        qp_fill_qparams(s.mean - alpha, s.mean + alpha, bits, &q);
+    }
+    c = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
+}
+
+// Block-wide: first minimum of the MSE curve wins (k = 0 keeps b_E); writes the result and
+// the winning quantizer.  s_curve: shared scratch of steps + 1 doubles.
+__device__ inline void qp_ds_pick(const double* __restrict__ curve, int steps, int nb, int bits,
+                                  const float4* __restrict__ cand, const qp_ds_setup* __restrict__ setup,
+                                  qp_ds_result_t* __restrict__ out, qp_qparams_t* __restrict__ qp_out,
+                                  unsigned* __restrict__ status, double* s_curve)
+{
+    for (int k = threadIdx.x; k <= steps; k += blockDim.x) s_curve[k] = __ldcg(&curve[k]);
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    const qp_ds_setup s = *setup;
+    int best = 0;
+    double best_mse = s_curve[0];
+    for (int k = 1; k <= steps; ++k)
+        if (s_curve[k] < best_mse) { best_mse = s_curve[k]; best = k; }
+    const double b_star = s.b_e + (double)best * (s.b_r - s.b_e) / (double)steps;
+    if (out) {
+        out->b_e = s.b_e;
+        out->b_r = s.b_r;
+        out->b_star = b_star;
+        out->alpha_e = s.F * s.b_e;
+        out->alpha_star = s.F * b_star;
+        out->mse_e = s_curve[0];
+        out->mse_star = best_mse;
+        out->k_star = best;
+        out->steps = steps;
+        out->hist_bins = nb;
+        out->bits = bits;
+    }
+    const float4 c = __ldcg(&cand[best]);
+    const bool degenerate_q = !(c.y > c.x);
+    if (qp_out) {
+        qp_out->lo = c.x; qp_out->hi = c.y; qp_out->scale = c.z; qp_out->inv_scale = c.w;
+        qp_out->bits = bits;
+        qp_out->flags = degenerate_q ? 1 : 0;
+    }
+    if (s.degenerate || degenerate_q) atomicOr(status, QP_DEV_DEGENERATE);
+}
+
 #endif  // __CUDACC__
 
 // Kernel launchers (one per translation unit).
@@ -222,7 +298,8 @@ int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
                          int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                          qp_qparams_t* d_qp_out, cudaStream_t s);
 int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
-                                  int bits, int steps, cudaStream_t s);
+                                  int bits, int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
+                                  qp_qparams_t* d_qp_out, cudaStream_t s);
 int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
                               qp_qparams_t* d_qp_out, cudaStream_t s);
 int32_t qp_launch_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, const qp_qparams_t* d_qp,

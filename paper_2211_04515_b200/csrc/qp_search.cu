@@ -97,36 +97,16 @@ __global__ void __launch_bounds__(QP_THREADS) setup_kernel(const qp_stats_t* __r
     if (threadIdx.x == 0) {
         for (int i = 1; i < QP_THREADS; ++i) top = sh_top[i] > top ? sh_top[i] : top;
         if (from_stats) top = st->hist_peak;
-        const unsigned long long nf = st->n - st->nonfinite;
-        const double mn = st->min, mx = st->max;
-        const double b_e = bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad;
-        double peak = 0.0;
-        if (mx > mn && nf > 0) {
-            const double w = (mx - mn) / (double)nb;
-            peak = (double)top / ((double)nf * w);
-        }
-        s.degenerate = !(mx > mn) || !(peak > 0.0) || !(b_e > 0.0);
-        s.b_e = b_e;
-        s.b_r = s.degenerate ? b_e : 1.0 / (2.0 * peak);
-        s.F = F;
-        s.mean = st->mean;
-        s.n_finite = nf;
-        s.pad = 0;
+        qp_ds_make_setup(st, top, nb, bmode, F, s);
         *setup = s;
     }
     __syncthreads();
     for (int k = threadIdx.x; k <= steps; k += QP_THREADS) {
-        // b_k = b_E + k (b_R - b_E) / steps, evaluated in this order in fp64
-        const double b_k = s.b_e + (double)k * (s.b_r - s.b_e) / (double)steps;
-        const bool ok = (k == 0) || (!s.degenerate && b_k > 0.0);
-        qp_qparams_t q;
-        q.lo = q.hi = q.scale = q.inv_scale = 0.f;
-        if (ok) {
-            const double alpha = s.F * b_k;
-            qp_fill_qparams(s.mean - alpha, s.mean + alpha, bits, &q);
-        }
-        cand[k] = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
-        valid[k] = ok ? 1 : 0;
+        float4 c;
+        int ok;
+        qp_ds_candidate(s, k, steps, bits, c, ok);
+        cand[k] = c;
+        valid[k] = ok;
     }
 }
 
@@ -253,37 +233,9 @@ __global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __re
         curve[k] = mse;
     }
     __syncthreads();
+    __threadfence_block();
     __shared__ double s_curve[QP_MAX_STEPS + 1];
-    for (int k = threadIdx.x; k <= steps; k += QP_THREADS) s_curve[k] = curve[k];
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int best = 0;
-        double best_mse = s_curve[0];
-        for (int k = 1; k <= steps; ++k)
-            if (s_curve[k] < best_mse) { best_mse = s_curve[k]; best = k; }
-        const double b_star = s.b_e + (double)best * (s.b_r - s.b_e) / (double)steps;
-        if (out) {
-            out->b_e = s.b_e;
-            out->b_r = s.b_r;
-            out->b_star = b_star;
-            out->alpha_e = s.F * s.b_e;
-            out->alpha_star = s.F * b_star;
-            out->mse_e = s_curve[0];
-            out->mse_star = best_mse;
-            out->k_star = best;
-            out->steps = steps;
-            out->hist_bins = nb;
-            out->bits = bits;
-        }
-        const float4 c = cand[best];
-        const bool degenerate_q = !(c.y > c.x);
-        if (qp_out) {
-            qp_out->lo = c.x; qp_out->hi = c.y; qp_out->scale = c.z; qp_out->inv_scale = c.w;
-            qp_out->bits = bits;
-            qp_out->flags = degenerate_q ? 1 : 0;
-        }
-        if (s.degenerate || degenerate_q) atomicOr(status, QP_DEV_DEGENERATE);
-    }
+    qp_ds_pick(curve, steps, nb, bits, cand, setup, out, qp_out, status, s_curve);
 }
 
 // one thread: ACIQ clip from device-resident statistics
@@ -313,11 +265,11 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     uint64_t want = (n + per_block - 1) / per_block;
     const uint64_t hcap = (uint64_t)ctx->sm_count * 3;
     const int hblocks = (int)(want < 1 ? 1 : (want > hcap ? hcap : want));
+    // returns at once when the statistics already carry this histogram's peak
     if (cudaMemsetAsync(ctx->d_hist, 0, sizeof(unsigned long long) * nb, s) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (histogram reset)");
     hist_kernel<T><<<hblocks, QP_THREADS, sh_bytes, s>>>(x, n, d_stats, nb, rep_shift, ctx->d_hist);
-    setup_kernel<<<1, QP_THREADS, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
-                                          ctx->d_setup);
+    ctx->launches += 1;
 
     const int ncand = steps + 1;
     // interval-moment scoring where its tables fit and its fixed-point sums cannot overflow
@@ -325,14 +277,11 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
                          n / (uint64_t)ctx->iv_blocks + 65536 < (1ull << 22);
     const bool use_iv = iv_fits && (ctx->search_path == QP_SEARCH_INTERVALS ||
                                     (ctx->search_path == QP_SEARCH_AUTO && n >= (1ull << 20)));
-    if (use_iv) {
-        const int32_t rc = qp_launch_interval_search(ctx, x, sizeof(T) == 4 ? QP_F32 : QP_BF16, n, d_stats, bits, steps, s);
-        if (rc != QP_OK) return rc;
-        finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, 0, steps, 0, nb, bits, ctx->d_valid, ctx->d_cand,
-                                                 ctx->d_setup, ctx->d_curve, d_out, d_qp_out, ctx->d_status);
-        ctx->launches += 3;
-        return qp_check_launch(ctx, "qp_dsaciq_search");
-    }
+    if (use_iv)
+        return qp_launch_interval_search(ctx, x, sizeof(T) == 4 ? QP_F32 : QP_BF16, n, d_stats, bits, bmode, steps, nb, F,
+                                         d_out, d_qp_out, s);
+    setup_kernel<<<1, QP_THREADS, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
+                                          ctx->d_setup);
     const int groups = (ncand + K - 1) / K;
     const uint64_t per_chunk = (uint64_t)QP_THREADS * 8;
     want = (n + per_chunk - 1) / per_chunk;
@@ -343,7 +292,7 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     eval_kernel<T><<<dim3(groups, chunks), QP_THREADS, 0, s>>>(x, n, d_stats, ctx->d_cand, ncand, ctx->d_sums);
     finalize_kernel<<<1, QP_THREADS, 0, s>>>(ctx->d_sums, chunks, steps, 1, nb, bits, ctx->d_valid, ctx->d_cand,
                                              ctx->d_setup, ctx->d_curve, d_out, d_qp_out, ctx->d_status);
-    ctx->launches += 4;
+    ctx->launches += 3;
     return qp_check_launch(ctx, "qp_dsaciq_search");
 }
 

@@ -70,25 +70,61 @@ __device__ __forceinline__ float first_true(float lo_x, float hi_x, P pred)
 
 // ------------------------------------------------------------------ grid + boundaries
 
-// Every block first derives the grid that covers all valid candidates (block 0 stores it),
-// then: thread t < nthr finds threshold (k, j) of candidate k = t / (L-1), code
-// j = 1 + t % (L-1); thread nthr + c - 1 finds the left edge of grid cell c = 1..G-1.
-// Entries that do not exist are +inf.
-__global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict__ cand, const int* __restrict__ valid,
-                                                        int ncand, int bits, qp_ds_setup* __restrict__ setup,
+// Set-up and boundaries in one launch.  Every block repeats the cheap part (peak of the
+// histogram -> b_R, the candidates and their quantizers, the grid that covers all valid
+// candidates; block 0 stores them for the later kernels), then: thread t < nthr finds
+// threshold (k, j) of candidate k = t / (L-1), code j = 1 + t % (L-1); thread nthr + c - 1
+// finds the left edge of grid cell c = 1..G-1.  Entries that do not exist are +inf.
+constexpr int IV_MAX_CAND = 1024;
+__global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __restrict__ st,
+                                                        const unsigned long long* __restrict__ hist, int nb, int bits,
+                                                        int bmode, int steps, double F, float4* __restrict__ cand,
+                                                        int* __restrict__ valid, qp_ds_setup* __restrict__ setup,
                                                         float* __restrict__ bnd, float* __restrict__ edges)
 {
+    __shared__ unsigned long long s_top[8];
     __shared__ float s_lo[8], s_hi[8];
     __shared__ float sg_lo, sg_hi, sg_inv;
+    __shared__ qp_ds_setup s;
+    __shared__ float4 s_cand[IV_MAX_CAND];
+    __shared__ unsigned char s_valid[IV_MAX_CAND];
     const float inf = __int_as_float(0x7F800000);
+    const int ncand = steps + 1;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    unsigned long long top = 0;
+    const bool from_stats = st->hist_bins == nb;
+    for (int b = threadIdx.x; !from_stats && b < nb; b += 256) {
+        const unsigned long long c = hist[b];
+        top = c > top ? c : top;
+    }
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_down_sync(0xFFFFFFFFu, top, o);
+        top = other > top ? other : top;
+    }
+    if (lane == 0) s_top[warp] = top;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < 8; ++w) top = s_top[w] > top ? s_top[w] : top;
+        if (from_stats) top = st->hist_peak;
+        qp_ds_make_setup(st, top, nb, bmode, F, s);
+    }
+    __syncthreads();
     float lo = inf, hi = -inf;
-    for (int k = threadIdx.x; k < ncand; k += 256)
-        if (k == 0 || valid[k]) { lo = fminf(lo, cand[k].x); hi = fmaxf(hi, cand[k].y); }
+    for (int k = threadIdx.x; k < ncand; k += 256) {
+        float4 c;
+        int ok;
+        qp_ds_candidate(s, k, steps, bits, c, ok);
+        s_cand[k] = c;
+        s_valid[k] = (unsigned char)ok;
+        if (blockIdx.x == 0) { cand[k] = c; valid[k] = ok; }
+        if (ok) { lo = fminf(lo, c.x); hi = fmaxf(hi, c.y); }
+    }
     for (int o = 16; o > 0; o >>= 1) {
         lo = fminf(lo, __shfl_down_sync(0xFFFFFFFFu, lo, o));
         hi = fmaxf(hi, __shfl_down_sync(0xFFFFFFFFu, hi, o));
     }
-    if ((threadIdx.x & 31) == 0) { s_lo[threadIdx.x >> 5] = lo; s_hi[threadIdx.x >> 5] = hi; }
+    if (lane == 0) { s_lo[warp] = lo; s_hi[warp] = hi; }
     __syncthreads();
     if (threadIdx.x == 0) {
         for (int w = 1; w < 8; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); }
@@ -103,12 +139,14 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
         }
         sg_lo = lo; sg_hi = hi; sg_inv = inv_gw;
         if (blockIdx.x == 0) {
-            setup->g_lo = lo;
-            setup->g_hi = hi;
-            setup->inv_gw = inv_gw;
-            setup->u = u;
-            setup->inv_u = (float)(1.0 / u);
-            setup->gw = (float)(width / (double)G);
+            s.g_lo = lo;
+            s.g_hi = hi;
+            s.inv_gw = inv_gw;
+            s.u = u;
+            s.inv_u = (float)(1.0 / u);
+            s.gw = (float)(width / (double)G);
+            s.pad2 = 0.f;
+            *setup = s;
             edges[0] = lo;
             edges[G] = inf;
         }
@@ -121,8 +159,8 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
     if (t < nthr) {
         const int k = t / L1, j = 1 + t % L1;
         float out = inf;
-        if (valid[k] && g_hi > g_lo) {
-            const float4 q = cand[k];
+        if (s_valid[k] && g_hi > g_lo) {
+            const float4 q = s_cand[k];
             const unsigned mask = (unsigned)L1;
             auto pred = [&](float x) { return (int)qp_code(x, q.x, q.y, q.w, mask) >= j; };
             if (!pred(g_lo) && pred(g_hi)) out = first_true(g_lo, g_hi, pred);
@@ -142,20 +180,21 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const float4* __restrict
     }
 }
 
-// Rank sort of the MAXB boundaries.  Block b places entries [64b, 64b+64): thread t compares
-// entry 64b + (t & 63) with the 256 entries of slice t >> 6, the 16 slice counts are merged in
+// Rank sort of the MAXB boundaries.  Block b places entries [32b, 32b+32): thread t compares
+// entry 32b + (t & 31) with the 256 entries of slice t >> 5, the 16 slice counts are merged in
 // shared memory (rank = entries that are smaller, or equal with a lower index).
 // bb[0] = g_lo, bb[1 + r] = entry of rank r; +inf entries end up behind the finite ones.
-__global__ void __launch_bounds__(1024) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
-                                                       float* __restrict__ bb)
+constexpr int IV_RANK_PER_BLOCK = 32;
+__global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
+                                                      float* __restrict__ bb)
 {
     __shared__ float s[MAXB];
-    __shared__ int rank[64];
-    for (int i = threadIdx.x; i < MAXB; i += 1024) s[i] = bnd[i];
-    if (threadIdx.x < 64) rank[threadIdx.x] = 0;
+    __shared__ int rank[IV_RANK_PER_BLOCK];
+    for (int i = threadIdx.x; i < MAXB; i += 512) s[i] = bnd[i];
+    if (threadIdx.x < IV_RANK_PER_BLOCK) rank[threadIdx.x] = 0;
     __syncthreads();
-    const int local = threadIdx.x & 63, slice = threadIdx.x >> 6;
-    const int me = blockIdx.x * 64 + local;
+    const int local = threadIdx.x & 31, slice = threadIdx.x >> 5;
+    const int me = blockIdx.x * IV_RANK_PER_BLOCK + local;
     const float v = s[me];
     int cnt = 0;
     const int j0 = slice * (MAXB / 16);
@@ -166,7 +205,7 @@ __global__ void __launch_bounds__(1024) iv_rank_kernel(const float* __restrict__
     }
     atomicAdd(&rank[local], cnt);
     __syncthreads();
-    if (threadIdx.x < 64) bb[1 + rank[threadIdx.x]] = s[blockIdx.x * 64 + threadIdx.x];
+    if (threadIdx.x < IV_RANK_PER_BLOCK) bb[1 + rank[threadIdx.x]] = s[blockIdx.x * IV_RANK_PER_BLOCK + threadIdx.x];
     if (blockIdx.x == 0 && threadIdx.x == 0) bb[0] = setup->g_lo;
 }
 
@@ -335,22 +374,28 @@ __global__ void __launch_bounds__(256) iv_reduce_kernel(const unsigned long long
     }
 }
 
-// block k: squared error of candidate k from the interval moments, fixed summation order
-__global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total* __restrict__ tot,
-                                                              const float* __restrict__ bb,
-                                                              const unsigned* __restrict__ g_m,
-                                                              const double* __restrict__ outer_tot,
-                                                              const float4* __restrict__ cand,
-                                                              const int* __restrict__ valid, int bits,
-                                                              const qp_ds_setup* __restrict__ setup,
-                                                              double* __restrict__ curve)
+// block k: squared error of candidate k from the interval moments, fixed summation order;
+// the last block to finish (ticket, no waiting) picks the winner
+constexpr int IV_CURVE_THREADS = 512;
+__global__ void __launch_bounds__(IV_CURVE_THREADS) iv_curve_kernel(const qp_iv_total* __restrict__ tot,
+                                                                    const float* __restrict__ bb,
+                                                                    const unsigned* __restrict__ g_m,
+                                                                    const double* __restrict__ outer_tot,
+                                                                    const float4* __restrict__ cand,
+                                                                    const int* __restrict__ valid, int bits, int steps,
+                                                                    int nb, const qp_ds_setup* __restrict__ setup,
+                                                                    double* __restrict__ curve,
+                                                                    unsigned* __restrict__ ticket,
+                                                                    qp_ds_result_t* __restrict__ out,
+                                                                    qp_qparams_t* __restrict__ qp_out,
+                                                                    unsigned* __restrict__ status)
 {
     const int k = blockIdx.x;
-    __shared__ double red[QP_THREADS / 32];
-    if (!valid[k]) {
-        if (threadIdx.x == 0) curve[k] = __longlong_as_double(0x7FF0000000000000ll);
-        return;
-    }
+    __shared__ double red[IV_CURVE_THREADS / 32];
+    __shared__ bool last;
+    __shared__ double s_curve[IV_MAX_CAND];
+    double total = 0.0;
+    const bool ok = valid[k] != 0;
     const float4 q = cand[k];
     const unsigned mask = (1u << bits) - 1u;
     const unsigned m = *g_m;
@@ -360,54 +405,69 @@ __global__ void __launch_bounds__(QP_THREADS) iv_curve_kernel(const qp_iv_total*
         const unsigned c = qp_code(r, q.x, q.y, q.w, mask);
         return (double)fmaf(__fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.0f), q.z, q.x);
     };
-    double acc = 0.0;
-    for (unsigned i = threadIdx.x; i <= m; i += QP_THREADS) {
-        const unsigned long long n_i = tot[i].n;
-        if (n_i == 0) continue;
-        const float left = bb[i];                                   // an element of the interval: fixes its codes
-        const float r = cell_ref(cell_of(left, g_lo, inv_gw), g_lo, gw);
-        const double a = level(left) - (double)r;
-        acc += (double)n_i * a * a - 2.0 * a * ((double)tot[i].s1 * u);
+    if (ok) {
+        double acc = 0.0;
+        for (unsigned i = threadIdx.x; i <= m; i += IV_CURVE_THREADS) {
+            const unsigned long long n_i = tot[i].n;
+            if (n_i == 0) continue;
+            const float left = bb[i];                                   // an element of the interval: fixes its codes
+            const float r = cell_ref(cell_of(left, g_lo, inv_gw), g_lo, gw);
+            const double a = level(left) - (double)r;
+            acc += (double)n_i * a * a - 2.0 * a * ((double)tot[i].s1 * u);
+        }
+        total = qp_block_sum(acc, red);
     }
-    double total = qp_block_sum(acc, red);
     if (threadIdx.x == 0) {
-        const double s1_lo = outer_tot[0], s2_lo = outer_tot[1], s1_hi = outer_tot[2], s2_hi = outer_tot[3];
-        const double n_lo = outer_tot[4], n_hi = outer_tot[5], s2_in = outer_tot[6];
-        const double a_lo = level(setup->g_lo) - (double)setup->g_lo;      // >= 0: below every clip range
-        const double a_hi = level(setup->g_hi) - (double)setup->g_hi;      // <= 0: above every clip range
-        total += s2_in * (u * u);                  // sum of squared offsets: the same for every candidate
-        total += n_lo * a_lo * a_lo + 2.0 * a_lo * s1_lo + s2_lo;
-        total += n_hi * a_hi * a_hi - 2.0 * a_hi * s1_hi + s2_hi;
-        const unsigned long long nf = setup->n_finite;
-        curve[k] = nf ? total / (double)nf : 0.0;
+        double mse = __longlong_as_double(0x7FF0000000000000ll);
+        if (ok) {
+            const double s1_lo = outer_tot[0], s2_lo = outer_tot[1], s1_hi = outer_tot[2], s2_hi = outer_tot[3];
+            const double n_lo = outer_tot[4], n_hi = outer_tot[5], s2_in = outer_tot[6];
+            const double a_lo = level(setup->g_lo) - (double)setup->g_lo;      // >= 0: below every clip range
+            const double a_hi = level(setup->g_hi) - (double)setup->g_hi;      // <= 0: above every clip range
+            total += s2_in * (u * u);                  // sum of squared offsets: the same for every candidate
+            total += n_lo * a_lo * a_lo + 2.0 * a_lo * s1_lo + s2_lo;
+            total += n_hi * a_hi * a_hi - 2.0 * a_hi * s1_hi + s2_hi;
+            const unsigned long long nf = setup->n_finite;
+            mse = nf ? total / (double)nf : 0.0;
+        }
+        curve[k] = mse;
+        __threadfence();
+        last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
     }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *ticket = 0;
+    qp_ds_pick(curve, steps, nb, bits, cand, setup, out, qp_out, status, s_curve);
 }
 
 template <typename T>
-int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_stats, int bits, int steps,
-                       cudaStream_t s)
+int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_stats, int bits, int bmode, int steps,
+                       int nb, double F, qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, cudaStream_t s)
 {
     const int ncand = steps + 1;
     const int L1 = (1 << bits) - 1;
     const int nbnd = ncand * L1 + G - 1;
-    if (nbnd > MAXB) return qp_fail(ctx, QP_ERR_INVALID_ARG, "too many boundaries for the interval path");
+    if (nbnd > MAXB || ncand > IV_MAX_CAND)
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "too many boundaries for the interval path");
     constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)G * 4 + 16;
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
     if (cudaMemsetAsync(ctx->d_iv_tot, 0, sizeof(qp_iv_total) * (MAXB + 1), s) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
-    iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(ctx->d_cand, ctx->d_valid, ncand, bits, ctx->d_setup, ctx->d_iv_bnd,
-                                                ctx->d_iv_edges);
-    iv_rank_kernel<<<MAXB / 64, 1024, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb);
+    iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
+                                                ctx->d_setup, ctx->d_iv_bnd, ctx->d_iv_edges);
+    iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb);
     const int blocks = ctx->iv_blocks;
     iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_edges,
                                                              ctx->d_iv_first, ctx->d_iv_part, ctx->d_iv_outer);
     iv_reduce_kernel<<<dim3((MAXB + 1 + 255) / 256, IV_SLICES), 256, 0, s>>>(ctx->d_iv_part, blocks, ctx->d_iv_first,
                                                                             ctx->d_iv_tot, ctx->d_iv_outer,
                                                                             ctx->d_iv_outer + (size_t)blocks * 8);
-    iv_curve_kernel<<<ncand, QP_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, ctx->d_iv_first,
-                                                 ctx->d_iv_outer + (size_t)blocks * 8, ctx->d_cand, ctx->d_valid, bits,
-                                                 ctx->d_setup, ctx->d_curve);
+    iv_curve_kernel<<<ncand, IV_CURVE_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, ctx->d_iv_first,
+                                                       ctx->d_iv_outer + (size_t)blocks * 8, ctx->d_cand, ctx->d_valid,
+                                                       bits, steps, nb, ctx->d_setup, ctx->d_curve, ctx->d_ticket + 2,
+                                                       d_out, d_qp_out, ctx->d_status);
     ctx->launches += 5;
     return qp_check_launch(ctx, "qp_dsaciq_search (interval path)");
 }
@@ -415,8 +475,12 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
 }  // namespace
 
 int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
-                                  int bits, int steps, cudaStream_t s)
+                                  int bits, int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
+                                  qp_qparams_t* d_qp_out, cudaStream_t s)
 {
-    if (dtype == QP_F32) return interval_typed<float>(ctx, static_cast<const float*>(d_x), n, d_stats, bits, steps, s);
-    return interval_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_stats, bits, steps, s);
+    if (dtype == QP_F32)
+        return interval_typed<float>(ctx, static_cast<const float*>(d_x), n, d_stats, bits, bmode, steps, hist_bins, F,
+                                     d_out, d_qp_out, s);
+    return interval_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, d_stats, bits, bmode, steps,
+                                          hist_bins, F, d_out, d_qp_out, s);
 }
