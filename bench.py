@@ -34,6 +34,10 @@ import synth_inputs as si  # noqa: E402
 WORKLOAD = "c4"
 METRIC = "quantize+pack and unpack+dequant throughput, fp32 in, whole path per step"
 UNIT = "GB/s"
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's main kernel on this
+# workload, from the ncu captures summarised in profiles/kernels_c4_ncu_full.md (None once a
+# kernel has changed since its capture)
+NCU_TRAFFIC_BYTES = {"clip": 133.1e6, "stats": 2 * 133.6e6, "quantize_pack": 144.9e6, "unpack_dequantize": 103.3e6}
 SAMPLE_IMAGES = 8              # CPU baseline leg: the first 8 images of the batch (2.0 M elements)
 ORACLE_US_PER_ELEM = 0.31      # rough cost of one oracle step per element (search on ~half the steps)
 
@@ -310,7 +314,7 @@ def ours_main(args):
     first = kernels[dom_keys[0]]
     roofline = {"kernel": dom, "bound": first["bound"], "achieved": round(ach, 3), "peak": first["peak"],
                 "unit": first["unit"], "frac": round(ach / first["peak"], 4), "peak_kind": peak_kind,
-                "traffic": None, "share_of_step_time": round(stage_ms[dom] / sum(stage_ms.values()), 3)}
+                "traffic": NCU_TRAFFIC_BYTES.get(dom), "share_of_step_time": round(stage_ms[dom] / sum(stage_ms.values()), 3)}
 
     # ---- end to end through the host-buffer entry points (pinned host memory, copies timed)
     e2e_steps = max(3, min(args.steps, 30))

@@ -62,6 +62,7 @@ enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the form
 #define QP_DEV_BITS_MISMATCH 1u   /* a device-resident qp_qparams_t had other bits than the call */
 #define QP_DEV_DEGENERATE 2u
 #define QP_DEV_NONFINITE 4u
+#define QP_DEV_STREAM_TIMEOUT 8u  /* a bounded wait for a tile copy ran out; results of that call are invalid */
 
 /* Per-tensor statistics (Sec. 3: min/max of naive PTQ; mean and Laplace scale b of ACIQ;
  * b_E of the directed search).  All fields but n are over the finite elements. */

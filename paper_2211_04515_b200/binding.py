@@ -23,7 +23,7 @@ QP_WARN_INFEASIBLE, QP_WARN_DEGENERATE, QP_WARN_NONFINITE = 1, 2, 3
 QP_F32, QP_BF16 = 0, 1
 QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
 QP_B_MAD, QP_B_MEAN_ABS = 0, 1
-QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE = 1, 2, 4
+QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT = 1, 2, 4, 8
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
 

@@ -16,7 +16,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
-constexpr unsigned QP_DEV_STREAM_TIMEOUT = 8u;               // status-word bit
+#include "quantpipe.h"                                        // QP_DEV_STREAM_TIMEOUT
+
 constexpr long long QP_STREAM_TIMEOUT_CYCLES = 4000000000ll;  // about two seconds
 
 namespace qp_stream {
