@@ -16,7 +16,8 @@
 //
 // The thresholds come from bisection over float bit patterns with the quantizer's own code
 // function, so the partition is exact.  Offsets x - r_i are smaller than one grid cell and
-// are accumulated in fixed point with unit u (a power of two below cell/2^16), as
+// (taken from a reference point per cell) are accumulated in fixed point with unit u (a
+// power of two below cell/2^15) by two 32-bit shared-memory atomics per element, as
 // integers: sums are exact and order-independent (bit-reproducible); the only approximation
 // is the rounding of each offset to u, which moves a candidate's MSE by less than 1e-6
 // relative in the worst case (all roundings aligned) and by ~1e-11 in practice.
@@ -185,11 +186,17 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
 // shared memory (rank = entries that are smaller, or equal with a lower index).
 // bb[0] = g_lo, bb[1 + r] = entry of rank r; +inf entries end up behind the finite ones.
 constexpr int IV_RANK_PER_BLOCK = 32;
+// The last block to finish (ticket, no waiting) then builds the cell table once for all
+// blocks of the moments kernel: table[0] = m, the number of finite boundaries (intervals
+// 0..m); table[1 + c] = first interval that meets cell c | last one << 16.
 __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
-                                                      float* __restrict__ bb)
+                                                      float* __restrict__ bb, const float* __restrict__ edges,
+                                                      unsigned* __restrict__ table, unsigned* __restrict__ ticket)
 {
     __shared__ float s[MAXB];
     __shared__ int rank[IV_RANK_PER_BLOCK];
+    __shared__ bool last;
+    __shared__ unsigned s_m;
     for (int i = threadIdx.x; i < MAXB; i += 512) s[i] = bnd[i];
     if (threadIdx.x < IV_RANK_PER_BLOCK) rank[threadIdx.x] = 0;
     __syncthreads();
@@ -207,6 +214,37 @@ __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ 
     __syncthreads();
     if (threadIdx.x < IV_RANK_PER_BLOCK) bb[1 + rank[threadIdx.x]] = s[blockIdx.x * IV_RANK_PER_BLOCK + threadIdx.x];
     if (blockIdx.x == 0 && threadIdx.x == 0) bb[0] = setup->g_lo;
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    if (threadIdx.x == 0) *ticket = 0;
+    const float inf = __int_as_float(0x7F800000);
+    for (int i = threadIdx.x; i < MAXB; i += 512) s[i] = __ldcg(&bb[1 + i]);        // now sorted
+    __syncthreads();
+    auto count_le = [&](float e, bool finite_only) {      // number of sorted boundaries <= e (or finite)
+        int lo = 0, hi = MAXB;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            const float v = s[mid];
+            if (finite_only ? (v < inf) : (v <= e)) lo = mid + 1; else hi = mid;
+        }
+        return (unsigned)lo;
+    };
+    if (threadIdx.x == 0) s_m = count_le(inf, true);
+    __syncthreads();
+    const unsigned m = s_m;
+    // cell c meets intervals first(c) .. first(c+1)-1, first(c) = boundaries <= left edge of c
+    // (the edge itself is one of them); a cell whose edge does not exist counts as m + 1
+    for (unsigned c = threadIdx.x; c < (unsigned)G; c += 512) {
+        const float e0 = edges[c], e1 = edges[c + 1];
+        const unsigned f0 = (e0 == inf) ? m + 1u : count_le(e0, false);
+        const unsigned f1 = (e1 == inf) ? m + 1u : count_le(e1, false);
+        table[1 + c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
+    }
+    if (threadIdx.x == 0) table[0] = m;
 }
 
 // ------------------------------------------------------------------------ moments
@@ -214,7 +252,8 @@ __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ 
 struct IvShared {
     float* bb;                      // [MAXB + 1]
     unsigned* cell;                 // [G] first interval of the cell | last interval << 16
-    unsigned long long* A;          // [MAXB + 1] count << 40 | sum of offsets
+    unsigned* cnt;                  // [MAXB + 1] count (bits 0-23) | carries out of s1 (bits 24-31)
+    unsigned* s1;                   // [MAXB + 1] low 32 bits of the sum of offsets
 };
 
 struct IvOuter {
@@ -243,7 +282,11 @@ __device__ __forceinline__ void iv_one(float x, const IvShared& sh, float g_lo, 
             if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
         }
         const unsigned d1 = __float2uint_rn(__fmul_rn(__fsub_rn(x, cell_ref(c, g_lo, gw)), inv_u));
-        atomicAdd(&sh.A[lo], (1ull << 40) + (unsigned long long)d1);
+        // two 32-bit atomics (fewer bank conflicts than one 64-bit one); a wrap of the low word
+        // of the sum is carried into the top byte of the count word, so nothing is lost
+        atomicAdd(&sh.cnt[lo], 1u);
+        const unsigned old = atomicAdd(&sh.s1[lo], d1);
+        if (old + d1 < old) atomicAdd(&sh.cnt[lo], 1u << 24);
         o.s2_in += (unsigned long long)d1 * (unsigned long long)d1;
     }
 }
@@ -253,43 +296,25 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
                                                                    const qp_stats_t* __restrict__ st,
                                                                    const qp_ds_setup* __restrict__ setup,
                                                                    const float* __restrict__ g_bb,
-                                                                   const float* __restrict__ g_edges,
-                                                                   unsigned* __restrict__ g_m,
+                                                                   const unsigned* __restrict__ g_table,
                                                                    unsigned long long* __restrict__ part,
                                                                    double* __restrict__ outer)
 {
     extern __shared__ __align__(16) unsigned char raw[];
-    __shared__ unsigned s_m;
     IvShared sh;
-    sh.A = reinterpret_cast<unsigned long long*>(raw);
-    sh.bb = reinterpret_cast<float*>(sh.A + (MAXB + 1));
+    sh.cnt = reinterpret_cast<unsigned*>(raw);
+    sh.s1 = sh.cnt + (MAXB + 1);
+    sh.bb = reinterpret_cast<float*>(sh.s1 + (MAXB + 1));
     sh.cell = reinterpret_cast<unsigned*>(sh.bb + (MAXB + 1));
     const float inf = __int_as_float(0x7F800000);
-    for (unsigned i = threadIdx.x; i <= (unsigned)MAXB; i += QP_IV_THREADS) { sh.A[i] = 0ull; sh.bb[i] = g_bb[i]; }
-    __syncthreads();
-    // s(j) = bb[1 + j] are the sorted boundaries.  count_le(e) = number of s(j) <= e.
-    auto count_le = [&](float e, bool finite_only) {
-        int lo = 0, hi = MAXB;
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            const float v = sh.bb[1 + mid];
-            if (finite_only ? (v < inf) : (v <= e)) lo = mid + 1; else hi = mid;
-        }
-        return (unsigned)lo;
-    };
-    if (threadIdx.x == 0) s_m = count_le(inf, true);         // m finite boundaries, intervals 0..m
-    __syncthreads();
-    const unsigned m = s_m;
-    // cell c meets intervals first(c) .. first(c+1)-1, first(c) = boundaries <= left edge of c
-    // (the edge itself is one of them); a cell whose edge does not exist counts as m + 1
-    for (unsigned c = threadIdx.x; c < (unsigned)G; c += QP_IV_THREADS) {
-        const float e0 = g_edges[c], e1 = g_edges[c + 1];
-        const unsigned f0 = (e0 == inf) ? m + 1u : count_le(e0, false);
-        const unsigned f1 = (e1 == inf) ? m + 1u : count_le(e1, false);
-        sh.cell[c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
+    for (unsigned i = threadIdx.x; i <= (unsigned)MAXB; i += QP_IV_THREADS) {
+        sh.cnt[i] = 0u;
+        sh.s1[i] = 0u;
+        sh.bb[i] = g_bb[i];
     }
+    for (unsigned c = threadIdx.x; c < (unsigned)G; c += QP_IV_THREADS) sh.cell[c] = g_table[1 + c];
     __syncthreads();
-    if (blockIdx.x == 0 && threadIdx.x == 0) *g_m = m;
+    const unsigned m = g_table[0];                           // finite boundaries; intervals 0..m
 
     const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw, inv_u = setup->inv_u, gw = setup->gw;
     const bool guard = st->nonfinite != 0;
@@ -328,7 +353,10 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     if (guard) body(std::true_type{}); else body(std::false_type{});
     __syncthreads();
     unsigned long long* mine = part + (size_t)blockIdx.x * (MAXB + 1);
-    for (unsigned i = threadIdx.x; i <= m; i += QP_IV_THREADS) mine[i] = sh.A[i];
+    for (unsigned i = threadIdx.x; i <= m; i += QP_IV_THREADS) {      // count << 40 | 40-bit sum of offsets
+        const unsigned c = sh.cnt[i];
+        mine[i] = ((unsigned long long)(c & 0xFFFFFFu) << 40) | ((unsigned long long)(c >> 24) << 32) | sh.s1[i];
+    }
 
     __shared__ double red[QP_IV_THREADS / 32];
     const double r0 = qp_block_sum(o.s1_lo, red), r1 = qp_block_sum(o.s2_lo, red);
@@ -457,10 +485,11 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
         return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
                                                 ctx->d_setup, ctx->d_iv_bnd, ctx->d_iv_edges);
-    iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb);
+    iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_edges,
+                                                            ctx->d_iv_first, ctx->d_ticket + 3);
     const int blocks = ctx->iv_blocks;
-    iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_edges,
-                                                             ctx->d_iv_first, ctx->d_iv_part, ctx->d_iv_outer);
+    iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
+                                                             ctx->d_iv_part, ctx->d_iv_outer);
     iv_reduce_kernel<<<dim3((MAXB + 1 + 255) / 256, IV_SLICES), 256, 0, s>>>(ctx->d_iv_part, blocks, ctx->d_iv_first,
                                                                             ctx->d_iv_tot, ctx->d_iv_outer,
                                                                             ctx->d_iv_outer + (size_t)blocks * 8);
