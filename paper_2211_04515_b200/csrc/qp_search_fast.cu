@@ -185,66 +185,44 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
 // entry 32b + (t & 31) with the 256 entries of slice t >> 5, the 16 slice counts are merged in
 // shared memory (rank = entries that are smaller, or equal with a lower index).
 // bb[0] = g_lo, bb[1 + r] = entry of rank r; +inf entries end up behind the finite ones.
+// For the entry that is the left edge of grid cell c it also stores
+// first[c] = number of boundaries <= that edge (the edge included), or ~0 if the cell does
+// not exist: cell c then meets the intervals first[c] .. first[c+1] - 1.
 constexpr int IV_RANK_PER_BLOCK = 32;
-// The last block to finish (ticket, no waiting) then builds the cell table once for all
-// blocks of the moments kernel: table[0] = m, the number of finite boundaries (intervals
-// 0..m); table[1 + c] = first interval that meets cell c | last one << 16.
 __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ bnd, const qp_ds_setup* __restrict__ setup,
-                                                      float* __restrict__ bb, const float* __restrict__ edges,
-                                                      unsigned* __restrict__ table, unsigned* __restrict__ ticket)
+                                                      int nthr, float* __restrict__ bb, unsigned* __restrict__ first)
 {
     __shared__ float s[MAXB];
-    __shared__ int rank[IV_RANK_PER_BLOCK];
-    __shared__ bool last;
-    __shared__ unsigned s_m;
+    __shared__ int rank[IV_RANK_PER_BLOCK], le[IV_RANK_PER_BLOCK];
     for (int i = threadIdx.x; i < MAXB; i += 512) s[i] = bnd[i];
-    if (threadIdx.x < IV_RANK_PER_BLOCK) rank[threadIdx.x] = 0;
+    if (threadIdx.x < IV_RANK_PER_BLOCK) { rank[threadIdx.x] = 0; le[threadIdx.x] = 0; }
     __syncthreads();
     const int local = threadIdx.x & 31, slice = threadIdx.x >> 5;
     const int me = blockIdx.x * IV_RANK_PER_BLOCK + local;
     const float v = s[me];
-    int cnt = 0;
+    int cnt = 0, cnt_le = 0;
     const int j0 = slice * (MAXB / 16);
 #pragma unroll 8
     for (int j = j0; j < j0 + MAXB / 16; ++j) {
         const float w = s[j];
         cnt += (w < v || (w == v && j < me)) ? 1 : 0;
+        cnt_le += (w <= v) ? 1 : 0;
     }
     atomicAdd(&rank[local], cnt);
+    atomicAdd(&le[local], cnt_le);
     __syncthreads();
-    if (threadIdx.x < IV_RANK_PER_BLOCK) bb[1 + rank[threadIdx.x]] = s[blockIdx.x * IV_RANK_PER_BLOCK + threadIdx.x];
-    if (blockIdx.x == 0 && threadIdx.x == 0) bb[0] = setup->g_lo;
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) last = (atomicAdd(ticket, 1u) == gridDim.x - 1);
-    __syncthreads();
-    if (!last) return;
-    __threadfence();
-    if (threadIdx.x == 0) *ticket = 0;
-    const float inf = __int_as_float(0x7F800000);
-    for (int i = threadIdx.x; i < MAXB; i += 512) s[i] = __ldcg(&bb[1 + i]);        // now sorted
-    __syncthreads();
-    auto count_le = [&](float e, bool finite_only) {      // number of sorted boundaries <= e (or finite)
-        int lo = 0, hi = MAXB;
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            const float v = s[mid];
-            if (finite_only ? (v < inf) : (v <= e)) lo = mid + 1; else hi = mid;
-        }
-        return (unsigned)lo;
-    };
-    if (threadIdx.x == 0) s_m = count_le(inf, true);
-    __syncthreads();
-    const unsigned m = s_m;
-    // cell c meets intervals first(c) .. first(c+1)-1, first(c) = boundaries <= left edge of c
-    // (the edge itself is one of them); a cell whose edge does not exist counts as m + 1
-    for (unsigned c = threadIdx.x; c < (unsigned)G; c += 512) {
-        const float e0 = edges[c], e1 = edges[c + 1];
-        const unsigned f0 = (e0 == inf) ? m + 1u : count_le(e0, false);
-        const unsigned f1 = (e1 == inf) ? m + 1u : count_le(e1, false);
-        table[1 + c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
+    if (threadIdx.x < IV_RANK_PER_BLOCK) {
+        const int t = blockIdx.x * IV_RANK_PER_BLOCK + threadIdx.x;
+        const float mine = s[t];
+        bb[1 + rank[threadIdx.x]] = mine;
+        if (t >= nthr && t < nthr + G - 1)
+            first[t - nthr + 1] = (mine < __int_as_float(0x7F800000)) ? (unsigned)le[threadIdx.x] : 0xFFFFFFFFu;
     }
-    if (threadIdx.x == 0) table[0] = m;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        bb[0] = setup->g_lo;
+        first[0] = 0u;                   // every boundary lies above g_lo
+        first[G] = 0xFFFFFFFFu;
+    }
 }
 
 // ------------------------------------------------------------------------ moments
@@ -296,7 +274,8 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
                                                                    const qp_stats_t* __restrict__ st,
                                                                    const qp_ds_setup* __restrict__ setup,
                                                                    const float* __restrict__ g_bb,
-                                                                   const unsigned* __restrict__ g_table,
+                                                                   const unsigned* __restrict__ g_first,
+                                                                   unsigned* __restrict__ g_m,
                                                                    unsigned long long* __restrict__ part,
                                                                    double* __restrict__ outer)
 {
@@ -312,9 +291,27 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
         sh.s1[i] = 0u;
         sh.bb[i] = g_bb[i];
     }
-    for (unsigned c = threadIdx.x; c < (unsigned)G; c += QP_IV_THREADS) sh.cell[c] = g_table[1 + c];
     __syncthreads();
-    const unsigned m = g_table[0];                           // finite boundaries; intervals 0..m
+    __shared__ unsigned s_m;
+    if (threadIdx.x == 0) {                                  // m = finite boundaries (sorted: a binary search)
+        int lo = 0, hi = MAXB;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (sh.bb[1 + mid] < inf) lo = mid + 1; else hi = mid;
+        }
+        s_m = (unsigned)lo;
+        if (blockIdx.x == 0) *g_m = (unsigned)lo;
+    }
+    __syncthreads();
+    const unsigned m = s_m;                                  // intervals 0..m
+    // cell c meets intervals first[c] .. first[c+1]-1; a cell that does not exist counts as m + 1
+    for (unsigned c = threadIdx.x; c < (unsigned)G; c += QP_IV_THREADS) {
+        unsigned f0 = g_first[c], f1 = g_first[c + 1];
+        f0 = (f0 == 0xFFFFFFFFu) ? m + 1u : f0;
+        f1 = (f1 == 0xFFFFFFFFu) ? m + 1u : f1;
+        sh.cell[c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
+    }
+    __syncthreads();
 
     const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw, inv_u = setup->inv_u, gw = setup->gw;
     const bool guard = st->nonfinite != 0;
@@ -485,15 +482,16 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
         return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
                                                 ctx->d_setup, ctx->d_iv_bnd, ctx->d_iv_edges);
-    iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_edges,
-                                                            ctx->d_iv_first, ctx->d_ticket + 3);
+    unsigned* g_m = ctx->d_iv_first + G + 1;                 // behind first[0..G]
+    iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ncand * L1, ctx->d_iv_bb,
+                                                            ctx->d_iv_first);
     const int blocks = ctx->iv_blocks;
     iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
-                                                             ctx->d_iv_part, ctx->d_iv_outer);
-    iv_reduce_kernel<<<dim3((MAXB + 1 + 255) / 256, IV_SLICES), 256, 0, s>>>(ctx->d_iv_part, blocks, ctx->d_iv_first,
+                                                             g_m, ctx->d_iv_part, ctx->d_iv_outer);
+    iv_reduce_kernel<<<dim3((MAXB + 1 + 255) / 256, IV_SLICES), 256, 0, s>>>(ctx->d_iv_part, blocks, g_m,
                                                                             ctx->d_iv_tot, ctx->d_iv_outer,
                                                                             ctx->d_iv_outer + (size_t)blocks * 8);
-    iv_curve_kernel<<<ncand, IV_CURVE_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, ctx->d_iv_first,
+    iv_curve_kernel<<<ncand, IV_CURVE_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, g_m,
                                                        ctx->d_iv_outer + (size_t)blocks * 8, ctx->d_cand, ctx->d_valid,
                                                        bits, steps, nb, ctx->d_setup, ctx->d_curve, ctx->d_ticket + 2,
                                                        d_out, d_qp_out, ctx->d_status);
