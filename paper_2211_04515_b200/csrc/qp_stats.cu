@@ -8,6 +8,8 @@
 // folds them into fp64; blocks write fp64 partials; the last block to finish (ticket
 // counter, no waiting) merges all partials in index order, so results do not depend on
 // block scheduling.
+#include <type_traits>
+
 #include "qp_internal.cuh"
 #include "qp_stream.cuh"
 
@@ -371,45 +373,50 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
     const bool hist_on = HIST && dmx > dmn;
     const float mn = (float)dmn;
     const float inv_w = hist_on ? (float)((double)nb / (dmx - dmn)) : 0.f;
-    const int lane_rep = threadIdx.x & ((1 << rep_shift) - 1);
+    // every lane counts in its own replica of the bins: my_hist[bin << rep_shift]
+    unsigned* my_hist = sh_hist + (threadIdx.x & ((1 << rep_shift) - 1));
+    const int top_bin = nb - 1;
     if (HIST) {
         for (int i = threadIdx.x; i < (nb << rep_shift); i += QP_THREADS) sh_hist[i] = 0u;
         __syncthreads();
     }
     double sd = 0.0, sv = 0.0;
-    auto one = [&](float e, float& d1, float& d2) {
-        const float d = __fsub_rn(__fsub_rn(e, m_hi), m_lo);
-        if (!guard || qp_is_finite(e)) {
-            d1 += fabsf(d);
-            d2 = fmaf(d, d, d2);
-            if (HIST && hist_on) {
-                int b = __float2int_rz(__fmul_rn(__fsub_rn(e, mn), inv_w));
-                b = min(max(b, 0), nb - 1);
-                atomicAdd(&sh_hist[(b << rep_shift) + lane_rep], 1u);
+    auto run = [&](auto guard_tag) {
+        constexpr bool GD = decltype(guard_tag)::value;
+        auto one = [&](float e, float& d1, float& d2) {
+            const float d = __fsub_rn(__fsub_rn(e, m_hi), m_lo);
+            if (!GD || qp_is_finite(e)) {
+                d1 += fabsf(d);
+                d2 = fmaf(d, d, d2);
+                if (HIST) {      // x >= min, so the position is never negative; an empty range gives bin 0
+                    const int b = min(__float2int_rz(__fmul_rn(__fsub_rn(e, mn), inv_w)), top_bin);
+                    atomicAdd(&my_hist[b << rep_shift], 1u);
+                }
             }
-        }
-    };
-    qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
-        reinterpret_cast<const unsigned char*>(x), ntiles, true, ring, status,
-        [&](const unsigned char* tile, uint64_t) {
-            float e[VPT][EPV];
+        };
+        qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
+            reinterpret_cast<const unsigned char*>(x), ntiles, true, ring, status,
+            [&](const unsigned char* tile, uint64_t) {
+                float e[VPT][EPV];
 #pragma unroll
-            for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * QP_THREADS + threadIdx.x) * 16, e[u]);
+                for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * QP_THREADS + threadIdx.x) * 16, e[u]);
+                float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+                for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) one(e[u][i], d1, d2);
+                sd += (double)d1;
+                sv += (double)d2;
+            });
+        if (blockIdx.x == 0) {
             float d1 = 0.f, d2 = 0.f;
-#pragma unroll
-            for (int u = 0; u < VPT; ++u)
-#pragma unroll
-                for (int i = 0; i < EPV; ++i) one(e[u][i], d1, d2);
+            const uint64_t t0 = ntiles * (ST_TILE / sizeof(T));
+            for (uint64_t i = t0 + threadIdx.x; i < n; i += QP_THREADS) one(qp_load_one(x + i), d1, d2);
             sd += (double)d1;
             sv += (double)d2;
-        });
-    if (blockIdx.x == 0) {
-        float d1 = 0.f, d2 = 0.f;
-        const uint64_t t0 = ntiles * (ST_TILE / sizeof(T));
-        for (uint64_t i = t0 + threadIdx.x; i < n; i += QP_THREADS) one(qp_load_one(x + i), d1, d2);
-        sd += (double)d1;
-        sv += (double)d2;
-    }
+        }
+    };
+    if (guard) run(std::true_type{}); else run(std::false_type{});
     if (HIST) {
         __syncthreads();
         const int reps = 1 << rep_shift;
@@ -450,7 +457,7 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
         out->mad = nf ? a / (double)nf : 0.0;
         out->var = nf ? b / (double)nf : 0.0;
         if (HIST) {
-            out->hist_peak = (unsigned long long)top;
+            out->hist_peak = hist_on ? (unsigned long long)top : 0ull;     // empty range: no histogram
             out->hist_bins = nb;
         }
         ticket[1] = 0;
