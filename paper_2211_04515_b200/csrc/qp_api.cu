@@ -81,7 +81,7 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     const size_t o_ivbnd = off;  off = align_up(off + sizeof(float) * QP_IV_MAXB, 256);
     const size_t o_ivbb = off;   off = align_up(off + sizeof(float) * (QP_IV_MAXB + 1), 256);
     const size_t o_ivedge = off; off = align_up(off + sizeof(float) * (QP_IV_CELLS + 1), 256);
-    const size_t o_ivfirst = off; off = align_up(off + sizeof(unsigned) * (QP_IV_CELLS + 2), 256);
+    const size_t o_ivfirst = off; off = align_up(off + sizeof(unsigned) * (QP_IV_CELLS + 8), 256);
     const size_t o_ivpart = off; off = align_up(off + sizeof(unsigned long long) * (size_t)c->iv_blocks * (QP_IV_MAXB + 1), 256);
     const size_t o_ivouter = off; off = align_up(off + sizeof(double) * 8 * (c->iv_blocks + 1), 256);
     const size_t o_ivtot = off;  off = align_up(off + sizeof(qp_iv_total) * (QP_IV_MAXB + 1), 256);

@@ -57,7 +57,7 @@ struct qp_ctx {
     float* d_iv_bnd;                     // [QP_IV_MAXB] unsorted boundaries
     float* d_iv_bb;                      // [QP_IV_MAXB + 1] g_lo followed by the sorted boundaries
     float* d_iv_edges;                   // [QP_IV_CELLS + 1] left edge of every cell
-    unsigned* d_iv_first;                // [c], c = 0..G: boundaries <= left edge of cell c; [G + 1]: finite boundaries m
+    unsigned* d_iv_first;                // [c], c = 0..G+1: boundaries <= left edge of cell c; [G + 2]: finite boundaries m
     unsigned long long* d_iv_part;       // [blocks][QP_IV_MAXB + 1] per-block count << 40 | sum of offsets
     double* d_iv_outer;                  // [blocks + 1][8] per-block sums that need no interval, then their totals
     qp_iv_total* d_iv_tot;               // [QP_IV_MAXB + 1]

@@ -42,19 +42,27 @@ __device__ __forceinline__ float float_of(unsigned k)
     return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
 }
 
-// grid cell of x (x >= g_lo): fp32, each operation rounded on its own
+// Grid cell of x in [g_lo, g_hi]: its position in cell units, rounded to the nearest integer
+// (0..G, so G + 1 cells).  The rounding is done by adding 2^23 (no conversion instruction):
+// `pm` keeps the cell number in its low mantissa bits.  Each operation is rounded on its own,
+// so the function is monotone in x.
+constexpr float IV_MAGIC = 8388608.0f;
+__device__ __forceinline__ float cell_pm(float x, float g_lo, float inv_gw)
+{
+    return __fadd_rn(__fmul_rn(__fsub_rn(x, g_lo), inv_gw), IV_MAGIC);
+}
 __device__ __forceinline__ int cell_of(float x, float g_lo, float inv_gw)
 {
-    return min(__float2int_rz(__fmul_rn(__fsub_rn(x, g_lo), inv_gw)), G - 1);
+    return (int)(__float_as_uint(cell_pm(x, g_lo, inv_gw)) & 0x7FFFFFu);
 }
 
-// Reference point of every interval inside cell c: half a cell below the cell's nominal
-// left edge, so that offsets x - ref are positive (between ~0.5 and ~1.5 cells) whatever the
-// rounding of the edge.  Any fixed function of c would do; it only has to be the same where
-// the moments are gathered and where they are used.
-__device__ __forceinline__ float cell_ref(int c, float g_lo, float gw)
+// Reference point of every interval inside the cell whose `pm` is given: one cell below the
+// cell's centre, so that offsets x - ref are positive (between ~0.5 and ~1.5 cells).  Any
+// fixed function of the cell would do; it only has to be the same where the moments are
+// gathered and where they are used.
+__device__ __forceinline__ float cell_ref(float pm, float g_lo, float gw)
 {
-    return fmaf((float)c - 0.5f, gw, g_lo);
+    return fmaf(__fsub_rn(pm, IV_MAGIC + 1.0f), gw, g_lo);      // (cell - 1) * gw + g_lo
 }
 
 // smallest float in (lo_x, hi_x] for which pred holds, given !pred(lo_x) and pred(hi_x), pred monotone
@@ -75,13 +83,13 @@ __device__ __forceinline__ float first_true(float lo_x, float hi_x, P pred)
 // histogram -> b_R, the candidates and their quantizers, the grid that covers all valid
 // candidates; block 0 stores them for the later kernels), then: thread t < nthr finds
 // threshold (k, j) of candidate k = t / (L-1), code j = 1 + t % (L-1); thread nthr + c - 1
-// finds the left edge of grid cell c = 1..G-1.  Entries that do not exist are +inf.
+// finds the left edge of grid cell c = 1..G.  Entries that do not exist are +inf.
 constexpr int IV_MAX_CAND = 1024;
 __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __restrict__ st,
                                                         const unsigned long long* __restrict__ hist, int nb, int bits,
                                                         int bmode, int steps, double F, float4* __restrict__ cand,
                                                         int* __restrict__ valid, qp_ds_setup* __restrict__ setup,
-                                                        float* __restrict__ bnd, float* __restrict__ edges)
+                                                        float* __restrict__ bnd)
 {
     __shared__ unsigned long long s_top[8];
     __shared__ float s_lo[8], s_hi[8];
@@ -148,8 +156,6 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
             s.gw = (float)(width / (double)G);
             s.pad2 = 0.f;
             *setup = s;
-            edges[0] = lo;
-            edges[G] = inf;
         }
     }
     __syncthreads();
@@ -167,7 +173,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
             if (!pred(g_lo) && pred(g_hi)) out = first_true(g_lo, g_hi, pred);
         }
         bnd[t] = out;
-    } else if (t < nthr + G - 1) {
+    } else if (t < nthr + G) {
         const int c = t - nthr + 1;
         float out = inf;
         if (g_hi > g_lo) {
@@ -175,7 +181,6 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
             if (!pred(g_lo) && pred(g_hi)) out = first_true(g_lo, g_hi, pred);
         }
         bnd[t] = out;
-        edges[c] = out;
     } else if (t < MAXB) {
         bnd[t] = inf;
     }
@@ -215,13 +220,13 @@ __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ 
         const int t = blockIdx.x * IV_RANK_PER_BLOCK + threadIdx.x;
         const float mine = s[t];
         bb[1 + rank[threadIdx.x]] = mine;
-        if (t >= nthr && t < nthr + G - 1)
+        if (t >= nthr && t < nthr + G)
             first[t - nthr + 1] = (mine < __int_as_float(0x7F800000)) ? (unsigned)le[threadIdx.x] : 0xFFFFFFFFu;
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         bb[0] = setup->g_lo;
         first[0] = 0u;                   // every boundary lies above g_lo
-        first[G] = 0xFFFFFFFFu;
+        first[G + 1] = 0xFFFFFFFFu;
     }
 }
 
@@ -229,43 +234,58 @@ __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ 
 
 struct IvShared {
     float* bb;                      // [MAXB + 1]
-    unsigned* cell;                 // [G] first interval of the cell | last interval << 16
+    unsigned* cell;                 // [G + 1] first interval of the cell | last interval << 16
     unsigned* cnt;                  // [MAXB + 1] count (bits 0-23) | carries out of s1 (bits 24-31)
     unsigned* s1;                   // [MAXB + 1] low 32 bits of the sum of offsets
 };
 
-struct IvOuter {
-    double s1_lo, s2_lo, s1_hi, s2_hi;
-    unsigned long long s2_in;       // sum of squared offsets of the in-grid elements (fixed point)
+struct IvOuter {                    // per thread, fp64: elements outside [g_lo, g_hi], and sum d^2 inside
+    double s1_lo, s2_lo, s1_hi, s2_hi, s2_in;
     unsigned n_lo, n_hi;
 };
+struct IvBatch {                    // the same over one batch of <= 8 elements, fp32
+    float s1_lo, s2_lo, s1_hi, s2_hi, s2_in;
+    unsigned n_lo, n_hi;
+};
+__device__ __forceinline__ void iv_flush(IvOuter& o, const IvBatch& b)
+{
+    o.s1_lo += (double)b.s1_lo; o.s2_lo += (double)b.s2_lo;
+    o.s1_hi += (double)b.s1_hi; o.s2_hi += (double)b.s2_hi;
+    o.s2_in += (double)b.s2_in;
+    o.n_lo += b.n_lo; o.n_hi += b.n_hi;
+}
+
+struct IvConst { float g_lo, g_hi, inv_gw, gw, inv_u; };
 
 template <bool GUARD>
-__device__ __forceinline__ void iv_one(float x, const IvShared& sh, float g_lo, float g_hi, float inv_gw, float gw,
-                                       float inv_u, IvOuter& o)
+__device__ __forceinline__ void iv_one(float x, const IvShared& sh, const IvConst& k, IvBatch& b)
 {
     if (GUARD && !qp_is_finite(x)) return;
-    if (x < g_lo) {
-        const double d = (double)__fsub_rn(g_lo, x);
-        ++o.n_lo; o.s1_lo += d; o.s2_lo += d * d;
-    } else if (x > g_hi) {
-        const double d = (double)__fsub_rn(x, g_hi);
-        ++o.n_hi; o.s1_hi += d; o.s2_hi += d * d;
+    if (x < k.g_lo) {
+        const float d = __fsub_rn(k.g_lo, x);
+        ++b.n_lo; b.s1_lo += d; b.s2_lo = fmaf(d, d, b.s2_lo);
+    } else if (x > k.g_hi) {
+        const float d = __fsub_rn(x, k.g_hi);
+        ++b.n_hi; b.s1_hi += d; b.s2_hi = fmaf(d, d, b.s2_hi);
     } else {
-        const int c = cell_of(x, g_lo, inv_gw);
-        const unsigned ci = sh.cell[c];
+        const float pm = cell_pm(x, k.g_lo, k.inv_gw);
+        const unsigned ci = sh.cell[__float_as_uint(pm) & 0x7FFFFFu];
         unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
         while (lo < hi) {                                   // largest i in [lo, hi] with bb[i] <= x
             const unsigned mid = (lo + hi + 1u) >> 1;
             if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
         }
-        const unsigned d1 = __float2uint_rn(__fmul_rn(__fsub_rn(x, cell_ref(c, g_lo, gw)), inv_u));
+        // offset in units of u, rounded to an integer by the same 2^23 trick (u is a power of two,
+        // so the product is exact and the only rounding is the one to the integer)
+        const float dm = fmaf(__fsub_rn(x, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
+        const unsigned d1 = __float_as_uint(dm) & 0x7FFFFFu;
+        const float d1f = __fsub_rn(dm, IV_MAGIC);
+        b.s2_in = fmaf(d1f, d1f, b.s2_in);
         // two 32-bit atomics (fewer bank conflicts than one 64-bit one); a wrap of the low word
         // of the sum is carried into the top byte of the count word, so nothing is lost
         atomicAdd(&sh.cnt[lo], 1u);
         const unsigned old = atomicAdd(&sh.s1[lo], d1);
         if (old + d1 < old) atomicAdd(&sh.cnt[lo], 1u << 24);
-        o.s2_in += (unsigned long long)d1 * (unsigned long long)d1;
     }
 }
 
@@ -305,7 +325,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     __syncthreads();
     const unsigned m = s_m;                                  // intervals 0..m
     // cell c meets intervals first[c] .. first[c+1]-1; a cell that does not exist counts as m + 1
-    for (unsigned c = threadIdx.x; c < (unsigned)G; c += QP_IV_THREADS) {
+    for (unsigned c = threadIdx.x; c <= (unsigned)G; c += QP_IV_THREADS) {
         unsigned f0 = g_first[c], f1 = g_first[c + 1];
         f0 = (f0 == 0xFFFFFFFFu) ? m + 1u : f0;
         f1 = (f1 == 0xFFFFFFFFu) ? m + 1u : f1;
@@ -313,9 +333,9 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     }
     __syncthreads();
 
-    const float g_lo = setup->g_lo, g_hi = setup->g_hi, inv_gw = setup->inv_gw, inv_u = setup->inv_u, gw = setup->gw;
+    const IvConst k = {setup->g_lo, setup->g_hi, setup->inv_gw, setup->gw, setup->inv_u};
     const bool guard = st->nonfinite != 0;
-    IvOuter o = {0.0, 0.0, 0.0, 0.0, 0ull, 0u, 0u};
+    IvOuter o = {0.0, 0.0, 0.0, 0.0, 0.0, 0u, 0u};
 
     constexpr int EPV = qp_span<T>::EPV;
     const qp_span<T> sp(x, n);
@@ -328,23 +348,28 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
             float a[EPV], b[EPV];
             qp_load_vec(xv + v * EPV, a);
             qp_load_vec(xv + (v + stride) * EPV, b);
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f, 0.f, 0u, 0u};
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
+            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, k, bt);
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv_one<GD>(b[i], sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
+            for (int i = 0; i < EPV; ++i) iv_one<GD>(b[i], sh, k, bt);
+            iv_flush(o, bt);
         }
         for (; v < sp.nvec; v += stride) {
             float a[EPV];
             qp_load_vec(xv + v * EPV, a);
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f, 0.f, 0u, 0u};
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
+            for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, k, bt);
+            iv_flush(o, bt);
         }
         if (blockIdx.x == 0) {
-            for (uint64_t i = threadIdx.x; i < sp.head; i += QP_IV_THREADS)
-                iv_one<GD>(qp_load_one(x + i), sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
             const uint64_t t0 = sp.head + sp.nvec * EPV;
-            for (uint64_t i = threadIdx.x; i < sp.tail; i += QP_IV_THREADS)
-                iv_one<GD>(qp_load_one(x + t0 + i), sh, g_lo, g_hi, inv_gw, gw, inv_u, o);
+            for (uint64_t i = threadIdx.x; i < sp.head + sp.tail; i += QP_IV_THREADS) {
+                IvBatch bt = {0.f, 0.f, 0.f, 0.f, 0.f, 0u, 0u};
+                iv_one<GD>(qp_load_one(x + (i < sp.head ? i : t0 + (i - sp.head))), sh, k, bt);
+                iv_flush(o, bt);
+            }
         }
     };
     if (guard) body(std::true_type{}); else body(std::false_type{});
@@ -359,7 +384,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     const double r0 = qp_block_sum(o.s1_lo, red), r1 = qp_block_sum(o.s2_lo, red);
     const double r2 = qp_block_sum(o.s1_hi, red), r3 = qp_block_sum(o.s2_hi, red);
     const double r4 = qp_block_sum((double)o.n_lo, red), r5 = qp_block_sum((double)o.n_hi, red);
-    const double r6 = qp_block_sum((double)o.s2_in, red);   // a thread's sum stays far below 2^53: exact
+    const double r6 = qp_block_sum(o.s2_in, red);
     if (threadIdx.x == 0) {
         double* dst = outer + (size_t)blockIdx.x * 8;
         dst[0] = r0; dst[1] = r1; dst[2] = r2; dst[3] = r3; dst[4] = r4; dst[5] = r5; dst[6] = r6;
@@ -436,7 +461,7 @@ __global__ void __launch_bounds__(IV_CURVE_THREADS) iv_curve_kernel(const qp_iv_
             const unsigned long long n_i = tot[i].n;
             if (n_i == 0) continue;
             const float left = bb[i];                                   // an element of the interval: fixes its codes
-            const float r = cell_ref(cell_of(left, g_lo, inv_gw), g_lo, gw);
+            const float r = cell_ref(cell_pm(left, g_lo, inv_gw), g_lo, gw);
             const double a = level(left) - (double)r;
             acc += (double)n_i * a * a - 2.0 * a * ((double)tot[i].s1 * u);
         }
@@ -472,17 +497,17 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
 {
     const int ncand = steps + 1;
     const int L1 = (1 << bits) - 1;
-    const int nbnd = ncand * L1 + G - 1;
+    const int nbnd = ncand * L1 + G;
     if (nbnd > MAXB || ncand > IV_MAX_CAND)
         return qp_fail(ctx, QP_ERR_INVALID_ARG, "too many boundaries for the interval path");
-    constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)G * 4 + 16;
+    constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)(G + 1) * 4 + 16;
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
     if (cudaMemsetAsync(ctx->d_iv_tot, 0, sizeof(qp_iv_total) * (MAXB + 1), s) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
-                                                ctx->d_setup, ctx->d_iv_bnd, ctx->d_iv_edges);
-    unsigned* g_m = ctx->d_iv_first + G + 1;                 // behind first[0..G]
+                                                ctx->d_setup, ctx->d_iv_bnd);
+    unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]
     iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ncand * L1, ctx->d_iv_bb,
                                                             ctx->d_iv_first);
     const int blocks = ctx->iv_blocks;
