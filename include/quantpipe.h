@@ -244,6 +244,43 @@ int32_t qp_select_bits(double bandwidth_bps, double budget_s, uint64_t n_elems, 
 int32_t qp_select_bits_eq2(double v_bytes, int q_t, double s_images, double r_images_per_s,
                            double bandwidth_bps, int32_t* h_bits_out);
 
+/* ---- adaptive controller (Sec. 3 "Adaptive PDA", Sec. 4.2) -------------------------------
+ * Host-only state machine of the paper's runtime loop: the monitor reports every
+ * microbatch's transfer (bytes put on the link, seconds it took); the averages are taken
+ * over a window of microbatches (50 in the paper); at the end of a window the link
+ * bandwidth is 8 * sum(bytes) / sum(seconds), and if it differs from the bandwidth of the
+ * last decision by more than rel_change (relative; 0 = decide at every window) the
+ * bit-width is chosen anew for the budget S / R seconds per microbatch:
+ *   QP_CTRL_FIT  widest allowed width whose payload fits (qp_select_bits)
+ *   QP_CTRL_EQ2  Eq. 2 as printed (qp_select_bits_eq2), from the current width and payload
+ * The struct is plain data owned by the caller (copy it to snapshot the controller). */
+enum { QP_CTRL_FIT = 0, QP_CTRL_EQ2 = 1 };
+#define QP_CTRL_MAX_ALLOWED 8
+typedef struct {
+    int32_t window, count;            /* microbatches per decision; seen so far in this window   */
+    int32_t bits, mode;               /* width in force (32 = raw fp32); QP_CTRL_FIT / QP_CTRL_EQ2 */
+    double s_images, r_images_per_s;  /* microbatch size S and target rate R                      */
+    uint64_t n_elems, overhead_bytes; /* tensor elements per microbatch; header bytes per transfer */
+    double rel_change;
+    double sum_bytes, sum_seconds;    /* of the current window                                    */
+    double ref_bandwidth_bps;         /* window bandwidth at the last decision; 0 before the first */
+    int32_t n_allowed;
+    int32_t allowed[QP_CTRL_MAX_ALLOWED];
+} qp_controller_t;
+/* h_allowed NULL selects the widths of the paper's Table 1, {32,16,8,6,4,2}.
+ * Errors: QP_ERR_INVALID_ARG (NULL, window < 1, S or R not positive, widths outside 1..32,
+ * more than QP_CTRL_MAX_ALLOWED widths, unknown mode, rel_change < 0). */
+int32_t qp_controller_init(qp_controller_t* h_c, int window, double s_images, double r_images_per_s,
+                           uint64_t n_elems, uint64_t overhead_bytes, const int32_t* h_allowed, int n_allowed,
+                           int mode, double rel_change, int initial_bits);
+/* One microbatch's transfer.  *h_bits_out = width to use from now on; *h_decided_out = 1 when
+ * this call closed a window and chose the width anew.  Returns QP_OK, QP_WARN_INFEASIBLE (the
+ * smallest width does not fit either; it is chosen) or QP_ERR_INVALID_ARG. */
+int32_t qp_controller_observe(qp_controller_t* h_c, double bytes_sent, double seconds, int32_t* h_bits_out,
+                              int32_t* h_decided_out);
+/* Payload of one microbatch at `bits` (32 = raw fp32): ceil(n_elems*bits/8) + overhead_bytes. */
+uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
+
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------
  * qp_sender_host: copies the n elements at h_x to d_x_work, runs statistics, the clip

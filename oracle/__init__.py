@@ -49,6 +49,14 @@ class DSResult(C.Structure):
                 ("k_star", C.c_int32), ("steps", C.c_int32), ("hist_bins", C.c_int32), ("bits", C.c_int32)]
 
 
+class Controller(C.Structure):
+    _fields_ = [("window", C.c_int32), ("count", C.c_int32), ("bits", C.c_int32), ("mode", C.c_int32),
+                ("s_images", C.c_double), ("r_images_per_s", C.c_double), ("n_elems", C.c_uint64),
+                ("overhead_bytes", C.c_uint64), ("rel_change", C.c_double), ("sum_bytes", C.c_double),
+                ("sum_seconds", C.c_double), ("ref_bw", C.c_double), ("n_allowed", C.c_int32),
+                ("allowed", C.c_int32 * 8)]
+
+
 OK, ERR_ARG, ERR_BITS, WARN_INFEASIBLE, WARN_DEGENERATE = 0, -1, -2, 1, 2
 
 _lib = None
@@ -92,6 +100,11 @@ def lib():
         L.orc_select_bits.restype = C.c_int
         L.orc_select_bits_eq2.argtypes = [C.c_double, C.c_int, C.c_double, C.c_double, C.c_double, C.POINTER(C.c_int32)]
         L.orc_select_bits_eq2.restype = C.c_int
+        L.orc_controller_init.argtypes = [C.POINTER(Controller), C.c_int, C.c_double, C.c_double, C.c_uint64,
+                                          C.c_uint64, C.POINTER(C.c_int32), C.c_int, C.c_int, C.c_double, C.c_int]
+        L.orc_controller_init.restype = None
+        L.orc_controller_observe.argtypes = [C.POINTER(Controller), C.c_double, C.c_double, C.POINTER(C.c_int32)]
+        L.orc_controller_observe.restype = C.c_int
         _lib = L
     return _lib
 
@@ -209,3 +222,18 @@ def select_bits_eq2(v_bytes: float, q_t: int, s_images: float, r_images_per_s: f
     out = C.c_int32()
     rc = lib().orc_select_bits_eq2(v_bytes, q_t, s_images, r_images_per_s, bandwidth_bps, C.byref(out))
     return rc, out.value
+
+
+def controller_init(window, s_images, r_images_per_s, n_elems, overhead_bytes=0, allowed=(32, 16, 8, 6, 4, 2), mode=0,
+                    rel_change=0.0, initial_bits=32) -> Controller:
+    c = Controller()
+    arr = (C.c_int32 * len(allowed))(*allowed)
+    lib().orc_controller_init(C.byref(c), window, s_images, r_images_per_s, n_elems, overhead_bytes, arr, len(allowed),
+                              mode, rel_change, initial_bits)
+    return c
+
+
+def controller_observe(c: Controller, bytes_sent: float, seconds: float):
+    out = C.c_int32()
+    decided = lib().orc_controller_observe(C.byref(c), bytes_sent, seconds, C.byref(out))
+    return out.value, bool(decided)

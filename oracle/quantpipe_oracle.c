@@ -423,3 +423,65 @@ int orc_select_bits_eq2(double v_bytes, int q_t, double s_images, double r_image
     *bits_out = (int32_t)q;
     return ORC_OK;
 }
+
+/* --------------------------------------------------------- adaptive controller */
+
+/* The runtime loop of Sec. 3 "Adaptive PDA" / Sec. 4.2, one microbatch at a time: transfers
+ * are averaged over a window of microbatches; when a window closes, the link bandwidth is
+ * total bits over total seconds, and if it moved by more than rel_change relative to the
+ * bandwidth of the last decision, the width is chosen again for the budget S / R per
+ * microbatch (mode 0: widest allowed width that fits; mode 1: Eq. 2 as printed). */
+typedef struct {
+    int32_t window, count, bits, mode;
+    double s_images, r_images_per_s;
+    uint64_t n_elems, overhead_bytes;
+    double rel_change, sum_bytes, sum_seconds, ref_bw;
+    int32_t n_allowed;
+    int32_t allowed[8];
+} orc_controller_t;
+
+void orc_controller_init(orc_controller_t* c, int window, double s_images, double r_images_per_s, uint64_t n_elems,
+                         uint64_t overhead_bytes, const int32_t* allowed, int n_allowed, int mode, double rel_change,
+                         int initial_bits)
+{
+    memset(c, 0, sizeof *c);
+    c->window = window;
+    c->bits = initial_bits;
+    c->mode = mode;
+    c->s_images = s_images;
+    c->r_images_per_s = r_images_per_s;
+    c->n_elems = n_elems;
+    c->overhead_bytes = overhead_bytes;
+    c->rel_change = rel_change;
+    c->n_allowed = n_allowed;
+    for (int i = 0; i < n_allowed; ++i) c->allowed[i] = allowed[i];
+}
+
+/* returns 1 if this microbatch closed a window and a new decision was taken */
+int orc_controller_observe(orc_controller_t* c, double bytes_sent, double seconds, int32_t* bits_out)
+{
+    c->sum_bytes += bytes_sent;
+    c->sum_seconds += seconds;
+    c->count += 1;
+    *bits_out = c->bits;
+    if (c->count < c->window) return 0;
+    double bw = c->sum_seconds > 0.0 ? 8.0 * c->sum_bytes / c->sum_seconds : 0.0;
+    c->count = 0;
+    c->sum_bytes = 0.0;
+    c->sum_seconds = 0.0;
+    if (!(bw > 0.0)) return 0;
+    if (c->ref_bw > 0.0 && fabs(bw - c->ref_bw) <= c->rel_change * c->ref_bw) return 0;
+    int32_t q = c->bits;
+    if (c->mode == 1) {
+        double v = (double)((c->n_elems * (uint64_t)c->bits + 7u) / 8u + c->overhead_bytes);
+        if (orc_select_bits_eq2(v, c->bits, c->s_images, c->r_images_per_s, bw, &q) < 0) return 0;
+    } else {
+        if (orc_select_bits(bw, c->s_images / c->r_images_per_s, c->n_elems, c->overhead_bytes, c->allowed,
+                            c->n_allowed, &q) < 0)
+            return 0;
+    }
+    c->ref_bw = bw;
+    c->bits = q;
+    *bits_out = q;
+    return 1;
+}

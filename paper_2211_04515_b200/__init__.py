@@ -3,4 +3,4 @@ statistics, ACIQ clip, directed search, quantize + bit-pack, unpack + dequantize
 selection.  The work is done by libquantpipe.so (hand-written sm_100a CUDA behind a C ABI,
 declared in include/quantpipe.h); this package only marshals arguments."""
 from .binding import *  # noqa: F401,F403
-from .binding import Context, DSResult, QParams, QuantPipeError, Stats, load  # noqa: F401
+from .binding import Context, Controller, DSResult, QParams, QuantPipeError, Stats, load  # noqa: F401

@@ -31,7 +31,8 @@ EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
-    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path",
+    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
+    "qp_controller_payload_bytes",
 )
 
 
@@ -50,6 +51,17 @@ class DSResult(C.Structure):
     _fields_ = [("b_e", C.c_double), ("b_r", C.c_double), ("b_star", C.c_double), ("alpha_e", C.c_double),
                 ("alpha_star", C.c_double), ("mse_e", C.c_double), ("mse_star", C.c_double),
                 ("k_star", C.c_int32), ("steps", C.c_int32), ("hist_bins", C.c_int32), ("bits", C.c_int32)]
+
+
+class Controller(C.Structure):
+    _fields_ = [("window", C.c_int32), ("count", C.c_int32), ("bits", C.c_int32), ("mode", C.c_int32),
+                ("s_images", C.c_double), ("r_images_per_s", C.c_double), ("n_elems", C.c_uint64),
+                ("overhead_bytes", C.c_uint64), ("rel_change", C.c_double), ("sum_bytes", C.c_double),
+                ("sum_seconds", C.c_double), ("ref_bandwidth_bps", C.c_double), ("n_allowed", C.c_int32),
+                ("allowed", C.c_int32 * 8)]
+
+
+QP_CTRL_FIT, QP_CTRL_EQ2 = 0, 1
 
 
 class QuantPipeError(RuntimeError):
@@ -95,6 +107,11 @@ def load() -> C.CDLL:
     L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
     L.qp_stats_static.argtypes = [vp, C.c_int, u64, vp, vp]
     L.qp_set_search_path.argtypes = [vp, C.c_int]
+    L.qp_controller_init.argtypes = [C.POINTER(Controller), C.c_int, dbl, dbl, u64, u64, C.POINTER(i32), C.c_int,
+                                     C.c_int, dbl, C.c_int]
+    L.qp_controller_observe.argtypes = [C.POINTER(Controller), dbl, dbl, C.POINTER(i32), C.POINTER(i32)]
+    L.qp_controller_payload_bytes.argtypes = [C.POINTER(Controller), C.c_int]
+    L.qp_controller_payload_bytes.restype = u64
     L.qp_launch_count.argtypes = [vp]
     L.qp_launch_count.restype = u64
     L.qp_sender_host.argtypes = [vp, vp, C.c_int, u64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, u64,
@@ -102,7 +119,8 @@ def load() -> C.CDLL:
     L.qp_receiver_host.argtypes = [vp, vp, u64, C.c_int, C.POINTER(QParams), vp, vp, vp, C.c_int, vp]
     for name in EXPORTS:
         fn = getattr(L, name)
-        if name not in ("qp_last_error", "qp_status_string", "qp_packed_bytes", "qp_aciq_F", "qp_launch_count"):
+        if name not in ("qp_last_error", "qp_status_string", "qp_packed_bytes", "qp_aciq_F", "qp_launch_count",
+                        "qp_controller_payload_bytes"):
             fn.restype = i32
     _lib = L
     return L
@@ -152,6 +170,29 @@ def qp_select_bits_eq2(v_bytes: float, q_t: int, s_images: float, r_images_per_s
     out = C.c_int32()
     rc = load().qp_select_bits_eq2(v_bytes, q_t, s_images, r_images_per_s, bandwidth_bps, C.byref(out))
     return int(rc), out.value
+
+
+def qp_controller_init(window: int, s_images: float, r_images_per_s: float, n_elems: int, overhead_bytes: int = 0,
+                       allowed=None, mode: int = QP_CTRL_FIT, rel_change: float = 0.0, initial_bits: int = 32):
+    c = Controller()
+    if allowed is None:
+        rc = load().qp_controller_init(C.byref(c), window, s_images, r_images_per_s, n_elems, overhead_bytes, None, 0,
+                                       mode, rel_change, initial_bits)
+    else:
+        arr = (C.c_int32 * len(allowed))(*allowed)
+        rc = load().qp_controller_init(C.byref(c), window, s_images, r_images_per_s, n_elems, overhead_bytes, arr,
+                                       len(allowed), mode, rel_change, initial_bits)
+    return int(rc), c
+
+
+def qp_controller_observe(c: Controller, bytes_sent: float, seconds: float):
+    bits, decided = C.c_int32(), C.c_int32()
+    rc = load().qp_controller_observe(C.byref(c), bytes_sent, seconds, C.byref(bits), C.byref(decided))
+    return int(rc), bits.value, bool(decided.value)
+
+
+def qp_controller_payload_bytes(c: Controller, bits: int) -> int:
+    return int(load().qp_controller_payload_bytes(C.byref(c), bits))
 
 
 # ------------------------------------------------------------ device calls

@@ -272,6 +272,75 @@ extern "C" int32_t qp_select_bits_eq2(double v_bytes, int q_t, double s_images, 
     return QP_OK;
 }
 
+// ------------------------------------------------------- adaptive controller
+
+extern "C" uint64_t qp_controller_payload_bytes(const qp_controller_t* c, int bits)
+{
+    if (!c || bits < 1 || bits > 32) return 0;
+    return (c->n_elems * (uint64_t)bits + 7u) / 8u + c->overhead_bytes;
+}
+
+extern "C" int32_t qp_controller_init(qp_controller_t* c, int window, double s_images, double r_images_per_s,
+                                      uint64_t n_elems, uint64_t overhead_bytes, const int32_t* h_allowed,
+                                      int n_allowed, int mode, double rel_change, int initial_bits)
+{
+    static const int32_t table1[6] = {32, 16, 8, 6, 4, 2};
+    if (!c || window < 1 || !(s_images > 0.0) || !(r_images_per_s > 0.0) || !(rel_change >= 0.0)) return QP_ERR_INVALID_ARG;
+    if (mode != QP_CTRL_FIT && mode != QP_CTRL_EQ2) return QP_ERR_INVALID_ARG;
+    if (initial_bits < 1 || initial_bits > 32) return QP_ERR_INVALID_ARG;
+    if (!h_allowed) { h_allowed = table1; n_allowed = 6; }
+    if (n_allowed < 1 || n_allowed > QP_CTRL_MAX_ALLOWED) return QP_ERR_INVALID_ARG;
+    memset(c, 0, sizeof *c);
+    for (int i = 0; i < n_allowed; ++i) {
+        if (h_allowed[i] < 1 || h_allowed[i] > 32) return QP_ERR_INVALID_ARG;
+        c->allowed[i] = h_allowed[i];
+    }
+    c->n_allowed = n_allowed;
+    c->window = window;
+    c->bits = initial_bits;
+    c->mode = mode;
+    c->s_images = s_images;
+    c->r_images_per_s = r_images_per_s;
+    c->n_elems = n_elems;
+    c->overhead_bytes = overhead_bytes;
+    c->rel_change = rel_change;
+    return QP_OK;
+}
+
+extern "C" int32_t qp_controller_observe(qp_controller_t* c, double bytes_sent, double seconds, int32_t* h_bits_out,
+                                         int32_t* h_decided_out)
+{
+    if (!c || !h_bits_out || !(bytes_sent >= 0.0) || !(seconds >= 0.0) || c->window < 1) return QP_ERR_INVALID_ARG;
+    if (h_decided_out) *h_decided_out = 0;
+    c->sum_bytes += bytes_sent;
+    c->sum_seconds += seconds;
+    c->count += 1;
+    *h_bits_out = c->bits;
+    if (c->count < c->window) return QP_OK;
+    // window closed: average bandwidth of the window
+    const double bw = c->sum_seconds > 0.0 ? 8.0 * c->sum_bytes / c->sum_seconds : 0.0;
+    c->count = 0;
+    c->sum_bytes = 0.0;
+    c->sum_seconds = 0.0;
+    if (!(bw > 0.0)) return QP_OK;                               // nothing was measured
+    if (c->ref_bandwidth_bps > 0.0 && fabs(bw - c->ref_bandwidth_bps) <= c->rel_change * c->ref_bandwidth_bps)
+        return QP_OK;                                            // no significant change
+    int32_t rc, q = c->bits;
+    if (c->mode == QP_CTRL_EQ2) {
+        rc = qp_select_bits_eq2((double)qp_controller_payload_bytes(c, c->bits), c->bits, c->s_images,
+                                c->r_images_per_s, bw, &q);
+    } else {
+        rc = qp_select_bits(bw, c->s_images / c->r_images_per_s, c->n_elems, c->overhead_bytes, c->allowed,
+                            c->n_allowed, &q);
+    }
+    if (rc < 0) return rc;
+    c->ref_bandwidth_bps = bw;
+    c->bits = q;
+    *h_bits_out = q;
+    if (h_decided_out) *h_decided_out = 1;
+    return rc;
+}
+
 // ------------------------------------------------ device-taking entry points
 
 static int32_t check_x(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n)
