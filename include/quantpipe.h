@@ -293,6 +293,15 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  * d_x_work >= n elements of dtype, d_packed_work and h_packed >= qp_packed_bytes(n, bits)
  * (d_packed_work 16-byte aligned), d_y_work and h_y >= n elements of out_dtype.
  * Errors: as the calls they are made of. */
+/* qp_sender_device: the sender's whole chain on DEVICE buffers in one call, nothing read back
+ * to the host: statistics (carrying the histogram along when use_ds != 0), the clip
+ * (directed search when use_ds != 0, plain ACIQ otherwise; Laplace model), quantize+pack.
+ * Writes the packed stream to d_packed, the quantizer to *d_qp_out (what the receiver needs)
+ * and, if d_stats_out is not NULL, the statistics.  Equivalent to qp_stats +
+ * qp_dsaciq_search / qp_aciq_qparams_device + qp_quantize_pack with the same arguments. */
+int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+                         int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
+                         qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream);
 int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
                        int steps, int hist_bins, void* d_x_work, void* d_packed_work, void* h_packed,
                        uint64_t packed_capacity, qp_qparams_t* h_qp_out, void* stream);

@@ -32,7 +32,7 @@ EXPORTS = (
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
-    "qp_controller_payload_bytes",
+    "qp_controller_payload_bytes", "qp_sender_device",
 )
 
 
@@ -116,6 +116,7 @@ def load() -> C.CDLL:
     L.qp_launch_count.restype = u64
     L.qp_sender_host.argtypes = [vp, vp, C.c_int, u64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp, u64,
                                  C.POINTER(QParams), vp]
+    L.qp_sender_device.argtypes = [vp, vp, C.c_int, u64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, vp, u64, vp, vp, vp]
     L.qp_receiver_host.argtypes = [vp, vp, u64, C.c_int, C.POINTER(QParams), vp, vp, vp, C.c_int, vp]
     for name in EXPORTS:
         fn = getattr(L, name)
@@ -333,6 +334,21 @@ class Context:
         self._check(self._lib.qp_unpack_dequantize(self._h, packed.data_ptr(), n, bits, ptr, on_dev, out.data_ptr(),
                                                    _dtype_code(out), _stream(self.device)))
         return out
+
+    # -- whole sender on device buffers
+    def qp_sender_device(self, x: torch.Tensor, bits: int, use_ds: bool, out_packed: torch.Tensor | None = None,
+                         out_qp: torch.Tensor | None = None, out_stats: torch.Tensor | None = None,
+                         bmode: int = QP_B_MAD, steps: int = QP_DEFAULT_STEPS, hist_bins: int = QP_DEFAULT_HIST_BINS):
+        """stats -> clip -> quantize+pack in one call; returns (packed, device QParams bytes)."""
+        assert x.is_cuda and x.is_contiguous()
+        out_packed = self._bytes(qp_packed_bytes(x.numel(), bits)) if out_packed is None else out_packed
+        out_qp = self._bytes(C.sizeof(QParams)) if out_qp is None else out_qp
+        self._check(self._lib.qp_sender_device(self._h, x.data_ptr(), _dtype_code(x), x.numel(), bits,
+                                               1 if use_ds else 0, bmode, steps, hist_bins, out_packed.data_ptr(),
+                                               out_packed.numel() * out_packed.element_size(), out_qp.data_ptr(),
+                                               out_stats.data_ptr() if out_stats is not None else None,
+                                               _stream(self.device)))
+        return out_packed, out_qp
 
     # -- host-buffer sender / receiver
     def qp_sender_host(self, h_x: torch.Tensor, bits: int, use_ds: bool, d_x_work: torch.Tensor,

@@ -476,6 +476,27 @@ extern "C" int32_t qp_unpack_dequantize(qp_ctx* ctx, const void* d_packed, uint6
     return qp_launch_unpack(ctx, d_packed, n, bits, d_qp, h_qp, d_y, out_dtype, static_cast<cudaStream_t>(stream));
 }
 
+// ------------------------------------------- whole sender on device buffers
+
+extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+                                    int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
+                                    qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (!d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_qp_out");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (use_ds && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if (packed_capacity < qp_packed_bytes(n, bits))
+        return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
+    qp_stats_t* st = d_stats_out ? d_stats_out : ctx->d_tmp_stats;
+    int32_t rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
+    if (rc < 0) return rc;
+    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
+    else        rc = qp_aciq_qparams_device(ctx, st, bits, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
+    if (rc < 0) return rc;
+    return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
+}
+
 // ------------------------------------------- host-buffer sender and receiver
 
 extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,

@@ -399,6 +399,47 @@ def test_search_bf16(ctx, path):
     check_search(ctx, oracle.widen_bf16(h[1:-2]), d[1:-2], 4, path=path)
 
 
+# ----------------------------------------------------------- whole-sender calls
+
+@pytest.mark.parametrize("bits,use_ds", [(2, True), (4, True), (8, False), (16, False), (3, False)])
+def test_sender_device_equals_separate_calls(ctx, bits, use_ds):
+    x = si.vit_activation((6, 197, 256), 77).reshape(-1)
+    d = dev(x)
+    d_stats = ctx.qp_stats(d, hist_bins=100 if use_ds else 0)
+    if use_ds:
+        _, d_qp = ctx.qp_dsaciq_search(d, d_stats, bits)
+    else:
+        d_qp = ctx.qp_aciq_qparams_device(d_stats, bits)
+    want = ctx.qp_quantize_pack(d, bits, d_qp)
+    got, got_qp = ctx.qp_sender_device(d, bits, use_ds)
+    assert torch.equal(got, want) and torch.equal(got_qp, d_qp)
+    q = ctx.read_qparams(got_qp)
+    o = oracle.QParams(q.lo, q.hi, q.scale, q.inv_scale, q.bits, q.flags)
+    assert np.array_equal(got.cpu().numpy(), oracle.quantize_pack(x, o))
+
+
+def test_sender_and_receiver_host_buffers(ctx):
+    x = si.vit_activation((2, 197, 384), 78).reshape(-1)
+    n = x.size
+    hx = torch.from_numpy(x).pin_memory()
+    for bits, use_ds in ((2, True), (8, False)):
+        nbytes = qp.qp_packed_bytes(n, bits)
+        d_x, d_p = torch.empty(n, device="cuda"), torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+        h_p = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+        h_qp = qp.QParams()
+        ctx.qp_sender_host(hx, bits, use_ds, d_x, d_p, h_p, h_qp)
+        torch.cuda.synchronize()
+        want, want_qp = ctx.qp_sender_device(dev(x), bits, use_ds)
+        assert np.array_equal(h_p.numpy(), want.cpu().numpy())
+        assert bytes(h_qp) == bytes(ctx.read_qparams(want_qp))
+        d_y, h_y = torch.empty(n, device="cuda"), torch.empty(n).pin_memory()
+        ctx.qp_receiver_host(h_p, n, bits, h_qp, d_p, d_y, h_y)
+        torch.cuda.synchronize()
+        o = oracle.QParams(h_qp.lo, h_qp.hi, h_qp.scale, h_qp.inv_scale, h_qp.bits, h_qp.flags)
+        y_o = oracle.unpack_dequantize(h_p.numpy(), n, o)
+        assert np.max(np.abs(h_y.numpy().astype(np.float64) - y_o.astype(np.float64))) <= 1e-6
+
+
 # ----------------------------------------------------- full-size configurations
 
 @pytest.mark.parametrize("name", ["c2", "c3", "c4"])
