@@ -457,13 +457,26 @@ __global__ void __launch_bounds__(IV_CURVE_THREADS) iv_curve_kernel(const qp_iv_
     };
     if (ok) {
         double acc = 0.0;
-        for (unsigned i = threadIdx.x; i <= m; i += IV_CURVE_THREADS) {
-            const unsigned long long n_i = tot[i].n;
-            if (n_i == 0) continue;
-            const float left = bb[i];                                   // an element of the interval: fixes its codes
-            const float r = cell_ref(cell_pm(left, g_lo, inv_gw), g_lo, gw);
-            const double a = level(left) - (double)r;
-            acc += (double)n_i * a * a - 2.0 * a * ((double)tot[i].s1 * u);
+        // all loads first (independent), then the arithmetic; same summation order as a plain loop
+        constexpr int PER = (MAXB + 1 + IV_CURVE_THREADS - 1) / IV_CURVE_THREADS;
+        ulonglong2 t[PER];
+        float left[PER];
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const unsigned i = threadIdx.x + j * IV_CURVE_THREADS;
+            t[j] = make_ulonglong2(0ull, 0ull);
+            left[j] = 0.f;
+            if (i <= m) {
+                t[j] = *reinterpret_cast<const ulonglong2*>(&tot[i]);
+                left[j] = bb[i];                                        // an element of the interval: fixes its codes
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            if (t[j].x == 0) continue;
+            const float r = cell_ref(cell_pm(left[j], g_lo, inv_gw), g_lo, gw);
+            const double a = level(left[j]) - (double)r;
+            acc += (double)t[j].x * a * a - 2.0 * a * ((double)t[j].y * u);
         }
         total = qp_block_sum(acc, red);
     }
