@@ -200,6 +200,18 @@ int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
  *   QP_SEARCH_AUTO        intervals for n >= 2^20 where they apply (default) */
 enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2 };
 int32_t qp_set_search_path(qp_ctx* ctx, int path);
+/* Graph replay of the multi-kernel calls (an execution option; the paper has no counterpart,
+ * results are unchanged).  With on = 1, qp_stats, qp_dsaciq_search and qp_sender_device
+ * record their kernels into a CUDA graph the first time they see an argument set (all
+ * pointers, sizes and options; not the stream) and launch the stored graph on later calls
+ * with the same arguments, which removes most of the gaps between the small kernels.  Up to
+ * 32 graphs are kept per context, the least recently used one is dropped.  A call on the
+ * legacy default stream (NULL), or on a stream the caller is capturing, is enqueued directly.
+ * The buffers of a recorded call must stay valid while it may be replayed; on = 0 drops all
+ * stored graphs.  Default off.  qp_graph_replays counts the calls served by a stored graph.
+ * Errors: QP_ERR_INVALID_ARG. */
+int32_t qp_set_graph_replay(qp_ctx* ctx, int on);
+uint64_t qp_graph_replays(qp_ctx* ctx);
 /* Copies the MSE of every candidate of the last search on this context (steps+1 values)
  * to host memory after waiting for `stream`.  Diagnostic. */
 int32_t qp_dsaciq_curve(qp_ctx* ctx, double* h_curve, int capacity, void* stream);

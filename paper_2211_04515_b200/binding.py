@@ -32,7 +32,7 @@ EXPORTS = (
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
-    "qp_controller_payload_bytes", "qp_sender_device",
+    "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays",
 )
 
 
@@ -107,6 +107,9 @@ def load() -> C.CDLL:
     L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
     L.qp_stats_static.argtypes = [vp, C.c_int, u64, vp, vp]
     L.qp_set_search_path.argtypes = [vp, C.c_int]
+    L.qp_set_graph_replay.argtypes = [vp, C.c_int]
+    L.qp_graph_replays.argtypes = [vp]
+    L.qp_graph_replays.restype = u64
     L.qp_controller_init.argtypes = [C.POINTER(Controller), C.c_int, dbl, dbl, u64, u64, C.POINTER(i32), C.c_int,
                                      C.c_int, dbl, C.c_int]
     L.qp_controller_observe.argtypes = [C.POINTER(Controller), dbl, dbl, C.POINTER(i32), C.POINTER(i32)]
@@ -121,7 +124,7 @@ def load() -> C.CDLL:
     for name in EXPORTS:
         fn = getattr(L, name)
         if name not in ("qp_last_error", "qp_status_string", "qp_packed_bytes", "qp_aciq_F", "qp_launch_count",
-                        "qp_controller_payload_bytes"):
+                        "qp_controller_payload_bytes", "qp_graph_replays"):
             fn.restype = i32
     _lib = L
     return L
@@ -302,6 +305,12 @@ class Context:
 
     def qp_set_search_path(self, path: int):
         self._check(self._lib.qp_set_search_path(self._h, path))
+
+    def qp_set_graph_replay(self, on: bool):
+        self._check(self._lib.qp_set_graph_replay(self._h, 1 if on else 0))
+
+    def qp_graph_replays(self) -> int:
+        return int(self._lib.qp_graph_replays(self._h))
 
     def qp_dsaciq_curve(self, steps: int):
         buf = (C.c_double * (steps + 1))()

@@ -117,10 +117,13 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     return QP_OK;
 }
 
+static void qp_drop_graphs(qp_ctx* ctx);
+
 extern "C" int32_t qp_destroy(qp_ctx* ctx)
 {
     if (!ctx) return QP_ERR_INVALID_ARG;
     qp_device_guard guard(ctx->device);
+    qp_drop_graphs(ctx);
     const cudaError_t e = cudaFree(ctx->d_base);
     delete ctx;
     return e == cudaSuccess ? QP_OK : QP_ERR_CUDA;
@@ -354,6 +357,95 @@ static int32_t check_x(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n)
     return QP_OK;
 }
 
+// ------------------------------------------- optional graph replay of the multi-kernel calls
+//
+// A call such as qp_dsaciq_search enqueues up to nine small kernels; at the sizes of the
+// paper's micro-batches the gaps between them are a visible share of its time.  With replay
+// switched on, the first call with a given argument set records its kernels into a CUDA graph
+// (stream capture on the caller's stream), and every later call with the same arguments
+// launches the stored graph instead.  Calls on the legacy default stream, or on a stream the
+// caller is itself capturing, are enqueued directly as before.
+template <typename F>
+static int32_t qp_graphed(qp_ctx* ctx, cudaStream_t stream, const unsigned long long (&key)[8], F&& enqueue)
+{
+    if (!ctx->graphs_on || stream == nullptr || stream == cudaStreamLegacy || stream == cudaStreamPerThread)
+        return enqueue();
+    cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+        cudaGetLastError();
+        return enqueue();
+    }
+    ++ctx->graph_clock;
+    for (int i = 0; i < ctx->n_graphs; ++i) {
+        qp_graph_entry& e = ctx->graphs[i];
+        if (memcmp(e.key, key, sizeof key) != 0) continue;
+        if (cudaGraphLaunch(e.exec, stream) != cudaSuccess) return qp_check_launch(ctx, "graph replay");
+        e.used = ctx->graph_clock;
+        ctx->launches += e.launches;
+        ++ctx->graph_hits;
+        return e.rc;
+    }
+    if (cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+        cudaGetLastError();
+        return enqueue();
+    }
+    const unsigned long long before = ctx->launches;
+    const int32_t rc = enqueue();
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(stream, &graph);
+    const unsigned recorded = (unsigned)(ctx->launches - before);
+    ctx->launches = before;                                  // nothing has run yet
+    if (rc < 0) {                                            // the call refused its arguments: nothing is enqueued
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        return rc;
+    }
+    cudaGraphExec_t exec = nullptr;
+    if (ce != cudaSuccess || !graph || cudaGraphInstantiate(&exec, graph, 0) != cudaSuccess) {
+        if (graph) cudaGraphDestroy(graph);
+        cudaGetLastError();
+        return enqueue();                                    // recording failed: run the call the plain way
+    }
+    cudaGraphDestroy(graph);
+    int slot = ctx->n_graphs;
+    if (slot == QP_GRAPH_SLOTS) {                            // full: drop the entry unused for longest
+        slot = 0;
+        for (int i = 1; i < QP_GRAPH_SLOTS; ++i)
+            if (ctx->graphs[i].used < ctx->graphs[slot].used) slot = i;
+        cudaGraphExecDestroy(ctx->graphs[slot].exec);
+    } else {
+        ++ctx->n_graphs;
+    }
+    qp_graph_entry& e = ctx->graphs[slot];
+    memcpy(e.key, key, sizeof key);
+    e.exec = exec;
+    e.launches = recorded;
+    e.rc = rc;
+    e.used = ctx->graph_clock;
+    if (cudaGraphLaunch(exec, stream) != cudaSuccess) return qp_check_launch(ctx, "graph launch");
+    ctx->launches += recorded;
+    return rc;
+}
+
+static void qp_drop_graphs(qp_ctx* ctx)
+{
+    for (int i = 0; i < ctx->n_graphs; ++i) cudaGraphExecDestroy(ctx->graphs[i].exec);
+    ctx->n_graphs = 0;
+}
+
+extern "C" int32_t qp_set_graph_replay(qp_ctx* ctx, int on)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (on != 0 && on != 1) return qp_fail(ctx, QP_ERR_INVALID_ARG, "on must be 0 or 1");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    if (!on) qp_drop_graphs(ctx);
+    ctx->graphs_on = on;
+    return QP_OK;
+}
+
+extern "C" uint64_t qp_graph_replays(qp_ctx* ctx) { return ctx ? ctx->graph_hits : 0; }
+
 extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
                             void* stream)
 {
@@ -364,7 +456,10 @@ extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n,
     if ((uintptr_t)d_out & 7u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_out must be 8-byte aligned");
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
-    return qp_launch_stats(ctx, d_x, dtype, n, hist_bins, d_out, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const unsigned long long key[8] = {1, (unsigned long long)(uintptr_t)d_x, (unsigned long long)dtype, n,
+                                       (unsigned long long)hist_bins, (unsigned long long)(uintptr_t)d_out, 0, 0};
+    return qp_graphed(ctx, s, key, [&] { return qp_launch_stats(ctx, d_x, dtype, n, hist_bins, d_out, s); });
 }
 
 extern "C" int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode,
@@ -395,8 +490,16 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
     if (((uintptr_t)d_out & 7u) || ((uintptr_t)d_qp_out & 3u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "result pointers");
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
-    rc = qp_launch_search(ctx, d_x, dtype, n, d_stats, bits, bmode, steps, hist_bins,
-                          qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_out, d_qp_out, static_cast<cudaStream_t>(stream));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const unsigned long long key[8] = {2, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_stats,
+                                       (unsigned long long)dtype | (unsigned long long)bits << 8 |
+                                           (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
+                                           (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
+                                       (unsigned long long)(uintptr_t)d_out, (unsigned long long)(uintptr_t)d_qp_out, 0};
+    rc = qp_graphed(ctx, s, key, [&] {
+        return qp_launch_search(ctx, d_x, dtype, n, d_stats, bits, bmode, steps, hist_bins,
+                                qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_out, d_qp_out, s);
+    });
     if (rc == QP_OK) ctx->last_steps = steps;
     return rc;
 }
@@ -489,12 +592,22 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
     if (packed_capacity < qp_packed_bytes(n, bits))
         return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
     qp_stats_t* st = d_stats_out ? d_stats_out : ctx->d_tmp_stats;
-    int32_t rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
-    if (rc < 0) return rc;
-    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
-    else        rc = qp_aciq_qparams_device(ctx, st, bits, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
-    if (rc < 0) return rc;
-    return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
+    // The inner calls see a capturing stream while this one records, and enqueue directly into it.
+    const unsigned long long key[8] = {3, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_packed,
+                                       (unsigned long long)dtype | (unsigned long long)bits << 8 |
+                                           (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
+                                           (unsigned long long)(use_ds != 0) << 28 |
+                                           (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
+                                       packed_capacity, (unsigned long long)(uintptr_t)d_qp_out,
+                                       (unsigned long long)(uintptr_t)st};
+    return qp_graphed(ctx, static_cast<cudaStream_t>(stream), key, [&]() -> int32_t {
+        int32_t rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
+        if (rc < 0) return rc;
+        if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
+        else        rc = qp_aciq_qparams_device(ctx, st, bits, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
+        if (rc < 0) return rc;
+        return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
+    });
 }
 
 // ------------------------------------------- host-buffer sender and receiver

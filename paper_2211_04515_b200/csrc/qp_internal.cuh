@@ -41,6 +41,16 @@ constexpr int QP_IV_BLOCKS_PER_SM = 3;
 
 struct qp_iv_total { unsigned long long n, s1; };       // per interval: count, sum of offsets (fixed point)
 
+// One instantiated graph of a multi-kernel call, keyed by every argument that the kernels bake in.
+struct qp_graph_entry {
+    unsigned long long key[8];
+    cudaGraphExec_t exec;
+    unsigned launches;                   // kernels inside the graph
+    int32_t rc;                          // status the recorded call returned (QP_OK or a warning)
+    unsigned long long used;
+};
+#define QP_GRAPH_SLOTS 32
+
 struct qp_ctx {
     int device;
     int sm_count;
@@ -66,6 +76,11 @@ struct qp_ctx {
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
     qp_qparams_t* d_tmp_qp;
     unsigned long long launches;         // kernels launched through this context (host count)
+    int graphs_on;                       // replay repeated multi-kernel calls as CUDA graphs (qp_set_graph_replay)
+    int n_graphs;
+    unsigned long long graph_clock;      // use counter for least-recently-used eviction
+    unsigned long long graph_hits;       // calls served by replaying a stored graph
+    qp_graph_entry graphs[QP_GRAPH_SLOTS];
     int last_steps;                      // steps of the last search (for qp_dsaciq_curve)
     char err[256];
 };

@@ -9,6 +9,7 @@ Tolerances (the targets this library is built to):
   packed codes    bit-exact given the same clip range and scale
   dequantized     1e-6 absolute
 """
+import ctypes
 import numpy as np
 import pytest
 import torch
@@ -516,3 +517,65 @@ def test_largest_sweep_size_sampled(ctx):
         # every reconstruction lies on the level grid inside the clip range
         assert float(y.min()) >= qp_h.lo - 1e-6 and float(y.max()) <= qp_h.hi + 1e-5
         del packed, y
+
+
+# ------------------------------------------------------------------ graph replay (execution option)
+
+@pytest.mark.parametrize("n_images,path", [(6, qp.QP_SEARCH_CANDIDATES), (40, qp.QP_SEARCH_AUTO)])
+def test_graph_replay_gives_the_same_bytes(n_images, path):
+    """With replay on, a repeated call launches the graph recorded by the first one.  The
+    results must be the bytes of the plain launches, also after the input buffer's CONTENTS
+    changed between replays, and the launch counter must advance as if launched one by one."""
+    plain, replay = qp.Context(0), qp.Context(0)
+    for c in (plain, replay):
+        c.qp_set_search_path(path)
+    replay.qp_set_graph_replay(True)
+    inputs = [si.vit_activation((n_images, 197, 256), 90 + i, outlier_frac=0.002 * i).reshape(-1) for i in range(3)]
+    n = inputs[0].size
+    d_x = torch.empty(n, device="cuda")
+    st, res, dq = (torch.empty(k, dtype=torch.uint8, device="cuda")
+                   for k in (ctypes.sizeof(qp.Stats), ctypes.sizeof(qp.DSResult), ctypes.sizeof(qp.QParams)))
+    packed = torch.empty(qp.qp_packed_bytes(n, 2), dtype=torch.uint8, device="cuda")
+    side = torch.cuda.Stream()
+    per_call = None
+    for i, x in enumerate(inputs + inputs[:1]):
+        d_x.copy_(torch.from_numpy(x))
+        want_st = plain.qp_stats(d_x, hist_bins=100)
+        want_res, want_qp = plain.qp_dsaciq_search(d_x, want_st, 2)
+        want_packed, want_qp2 = plain.qp_sender_device(d_x, 2, True)
+        torch.cuda.synchronize()
+        before = replay.qp_launch_count()
+        with torch.cuda.stream(side):
+            replay.qp_stats(d_x, out=st, hist_bins=100)
+            replay.qp_dsaciq_search(d_x, st, 2, out_result=res, out_qp=dq)
+            replay.qp_sender_device(d_x, 2, True, out_packed=packed, out_qp=dq)
+        side.synchronize()
+        launched = replay.qp_launch_count() - before
+        per_call = launched if per_call is None else per_call
+        assert launched == per_call and launched >= 5
+        assert replay.qp_graph_replays() == 3 * i
+        assert torch.equal(st, want_st) and torch.equal(res, want_res)
+        assert torch.equal(dq, want_qp2) and torch.equal(want_qp, want_qp2) and torch.equal(packed, want_packed)
+        o = oracle.QParams(*[getattr(replay.read_qparams(dq), f) for f in ("lo", "hi", "scale", "inv_scale", "bits", "flags")])
+        assert np.array_equal(packed.cpu().numpy(), oracle.quantize_pack(x, o))
+    # the legacy default stream cannot be captured: the call is enqueued directly and still right
+    hits = replay.qp_graph_replays()
+    replay.qp_stats(d_x, out=st, hist_bins=100)
+    torch.cuda.synchronize()
+    assert replay.qp_graph_replays() == hits and torch.equal(st, want_st)
+    # a refused call records nothing and leaves the stream usable
+    with torch.cuda.stream(side):
+        with pytest.raises(qp.QuantPipeError):
+            replay.qp_dsaciq_search(d_x, st, 9, out_result=res, out_qp=dq)
+        replay.qp_stats(d_x, out=st, hist_bins=100)
+    side.synchronize()
+    assert torch.equal(st, want_st)
+    # switching replay off drops the graphs; calls go back to plain launches
+    replay.qp_set_graph_replay(False)
+    hits = replay.qp_graph_replays()
+    with torch.cuda.stream(side):
+        replay.qp_stats(d_x, out=st, hist_bins=100)
+    side.synchronize()
+    assert replay.qp_graph_replays() == hits and torch.equal(st, want_st)
+    assert replay.qp_get_status() == 0 and plain.qp_get_status() == 0
+    plain.close(); replay.close()
