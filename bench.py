@@ -426,7 +426,8 @@ def sweep_main(args):
     assert torch.cuda.is_available(), "the sweep needs a CUDA device"
     torch.cuda.set_device(0)
     hbm_peak, _, peak_kind = peaks()
-    ctx = qp.Context(0)
+    ctx, gctx = qp.Context(0), qp.Context(0)
+    side = torch.cuda.Stream()
     L2_BYTES = 126e6
 
     def rotating(make, nbytes):
@@ -479,6 +480,28 @@ def sweep_main(args):
         for q in search_bits:
             med, best = timed(lambda i: ctx.qp_dsaciq_search(xs[i], d_stats[i], q, out_result=d_res, out_qp=d_qp), nb)
             emit(name, dtype, "dsaciq_search", q, n, med, best, esz * n)
+        # the sender in one call (statistics -> clip -> quantize+pack): the kernel chain and, for small
+        # tensors, the single cooperative launch; each launched directly and as a recorded graph (one
+        # graph per input buffer, on a stream of its own)
+        for q, use_ds in ((2, True), (8, False)):
+            pk = [torch.empty(qp.qp_packed_bytes(n, q), dtype=torch.uint8, device="cuda") for _ in range(nb)]
+            call = lambda c: (lambda i: c.qp_sender_device(xs[i], q, use_ds, out_packed=pk[i], out_qp=d_qp,
+                                                           out_stats=d_stats[i]))
+            paths = [("chain", qp.QP_SENDER_CHAIN)] + ([("fused", qp.QP_SENDER_FUSED)] if n <= (1 << 20) else [])
+            for label, path in paths:
+                stage = f"sender_device[{label}{', search' if use_ds else ''}]"
+                ctx.qp_set_sender_path(path)
+                med, best = timed(call(ctx), nb)
+                emit(name, dtype, stage, q, n, med, best, None)
+                ctx.qp_set_sender_path(qp.QP_SENDER_AUTO)
+                torch.cuda.synchronize()
+                gctx.qp_set_sender_path(path)
+                with torch.cuda.stream(side):
+                    gctx.qp_set_graph_replay(True)
+                    med, best = timed(call(gctx), nb, warm=nb + 5)
+                    gctx.qp_set_graph_replay(False)           # drops this workload's graphs
+                emit(name, dtype, stage + "+graph", q, n, med, best, None)
+            del pk
         ys = None
         for q in bits_list:
             rc, alpha, qp_h = qp.qp_aciq_alpha(st, q)
@@ -510,6 +533,7 @@ def sweep_main(args):
             if dist == "laplace" and log2n in (22, 26):
                 run_workload(f"c5-{dist}-2^{log2n}", x.to(torch.bfloat16), (2, 4, 8, 16), "bf16")
     ctx.close()
+    gctx.close()
     return 0
 
 

@@ -205,7 +205,7 @@ int32_t qp_set_search_path(qp_ctx* ctx, int path);
  * record their kernels into a CUDA graph the first time they see an argument set (all
  * pointers, sizes and options; not the stream) and launch the stored graph on later calls
  * with the same arguments, which removes most of the gaps between the small kernels.  Up to
- * 32 graphs are kept per context, the least recently used one is dropped.  A call on the
+ * 64 graphs are kept per context, the least recently used one is dropped.  A call on the
  * legacy default stream (NULL), or on a stream the caller is capturing, is enqueued directly.
  * The buffers of a recorded call must stay valid while it may be replayed; on = 0 drops all
  * stored graphs.  Default off.  qp_graph_replays counts the calls served by a stored graph.
@@ -310,7 +310,23 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  * (directed search when use_ds != 0, plain ACIQ otherwise; Laplace model), quantize+pack.
  * Writes the packed stream to d_packed, the quantizer to *d_qp_out (what the receiver needs)
  * and, if d_stats_out is not NULL, the statistics.  Equivalent to qp_stats +
- * qp_dsaciq_search / qp_aciq_qparams_device + qp_quantize_pack with the same arguments. */
+ * qp_dsaciq_search / qp_aciq_qparams_device + qp_quantize_pack with the same arguments.
+ *
+ * How the chain runs (qp_set_sender_path; the paper has no counterpart):
+ *   QP_SENDER_CHAIN  the kernels of the separate calls, one after the other; the outputs are
+ *                    bit for bit those of the separate calls
+ *   QP_SENDER_FUSED  one cooperative launch for 0 < n <= 2^20 (and steps <= 127, hist_bins <=
+ *                    4096 when searching): every SM keeps its slice of x in shared memory, the
+ *                    tensor-wide steps are separated by grid barriers.  Same arithmetic per
+ *                    element, but the sums are merged in another order: statistics agree with
+ *                    the chain to ~1e-15 relative, the error curve to ~1e-6, so the clip range
+ *                    can differ in its last fp32 bit or, where two steps of the search tie, by
+ *                    one step.  Other arguments fall back to the chain.
+ *   QP_SENDER_AUTO   fused where it applies (default)
+ * A grid barrier that does not complete within about a quarter of a second sets
+ * QP_DEV_STREAM_TIMEOUT in the status word and the launch ends without output. */
+enum { QP_SENDER_AUTO = 0, QP_SENDER_CHAIN = 1, QP_SENDER_FUSED = 2 };
+int32_t qp_set_sender_path(qp_ctx* ctx, int path);
 int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
                          int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
                          qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream);

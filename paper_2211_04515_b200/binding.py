@@ -26,13 +26,14 @@ QP_B_MAD, QP_B_MEAN_ABS = 0, 1
 QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT = 1, 2, 4, 8
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
+QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
 
 EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
-    "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays",
+    "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
 )
 
 
@@ -108,6 +109,7 @@ def load() -> C.CDLL:
     L.qp_stats_static.argtypes = [vp, C.c_int, u64, vp, vp]
     L.qp_set_search_path.argtypes = [vp, C.c_int]
     L.qp_set_graph_replay.argtypes = [vp, C.c_int]
+    L.qp_set_sender_path.argtypes = [vp, C.c_int]
     L.qp_graph_replays.argtypes = [vp]
     L.qp_graph_replays.restype = u64
     L.qp_controller_init.argtypes = [C.POINTER(Controller), C.c_int, dbl, dbl, u64, u64, C.POINTER(i32), C.c_int,
@@ -305,6 +307,9 @@ class Context:
 
     def qp_set_search_path(self, path: int):
         self._check(self._lib.qp_set_search_path(self._h, path))
+
+    def qp_set_sender_path(self, path: int):
+        self._check(self._lib.qp_set_sender_path(self._h, path))
 
     def qp_set_graph_replay(self, on: bool):
         self._check(self._lib.qp_set_graph_replay(self._h, 1 if on else 0))

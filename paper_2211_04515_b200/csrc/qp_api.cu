@@ -87,6 +87,7 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     const size_t o_ivtot = off;  off = align_up(off + sizeof(qp_iv_total) * (QP_IV_MAXB + 1), 256);
     const size_t o_tstats = off; off = align_up(off + sizeof(qp_stats_t), 256);
     const size_t o_tqp = off;    off = align_up(off + sizeof(qp_qparams_t), 256);
+    const size_t o_fused = off;  off = align_up(off + 256 + sizeof(unsigned long long) * 4096, 256);
 
     if (cudaMalloc(&c->d_base, off) != cudaSuccess || cudaMemset(c->d_base, 0, off) != cudaSuccess) {
         cudaGetLastError();
@@ -113,6 +114,7 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     c->d_iv_tot = reinterpret_cast<qp_iv_total*>(b + o_ivtot);
     c->d_tmp_stats = reinterpret_cast<qp_stats_t*>(b + o_tstats);
     c->d_tmp_qp = reinterpret_cast<qp_qparams_t*>(b + o_tqp);
+    c->d_fused = b + o_fused;
     *out = c;
     return QP_OK;
 }
@@ -142,6 +144,15 @@ extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
         snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_get_status: %s", cudaGetErrorString(e));
         return QP_ERR_CUDA;
     }
+    if (word & QP_DEV_STREAM_TIMEOUT) {
+        // a cooperative sender that gave up left its arrival counter and histogram mid-way
+        e = cudaMemsetAsync(ctx->d_fused, 0, 256 + sizeof(unsigned long long) * 4096, s);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+        if (e != cudaSuccess) {
+            snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_get_status: %s", cudaGetErrorString(e));
+            return QP_ERR_CUDA;
+        }
+    }
     return (int32_t)word;
 }
 
@@ -152,6 +163,14 @@ extern "C" int32_t qp_set_search_path(qp_ctx* ctx, int path)
     if (!ctx) return QP_ERR_INVALID_ARG;
     if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
     ctx->search_path = path;
+    return QP_OK;
+}
+
+extern "C" int32_t qp_set_sender_path(qp_ctx* ctx, int path)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (path < QP_SENDER_AUTO || path > QP_SENDER_FUSED) return qp_fail(ctx, QP_ERR_INVALID_ARG, "sender path");
+    ctx->sender_path = path;
     return QP_OK;
 }
 
@@ -581,6 +600,38 @@ extern "C" int32_t qp_unpack_dequantize(qp_ctx* ctx, const void* d_packed, uint6
 
 // ------------------------------------------- whole sender on device buffers
 
+// statistics -> clip -> quantize+pack on device buffers: one cooperative launch where that
+// applies (small tensors), the kernel chain of the separate calls otherwise
+static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+                                int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
+                                qp_qparams_t* d_qp_out, qp_stats_t* st, void* stream)
+{
+    int32_t rc;
+    if (ctx->sender_path != QP_SENDER_CHAIN && qp_sender_fused_applies(n, use_ds, steps, hist_bins)) {
+        // the checks of the separate calls
+        rc = check_x(ctx, d_x, dtype, n);
+        if (rc) return rc;
+        if (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
+        if (use_ds && (steps < 1 || hist_bins < 1)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "steps / hist_bins out of range");
+        if (!d_packed) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_packed");
+        if ((uintptr_t)d_packed & 15u) return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_packed must be 16-byte aligned");
+        if (((uintptr_t)st & 7u) || ((uintptr_t)d_qp_out & 3u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "result pointers");
+        qp_device_guard guard(ctx->device);
+        if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+        rc = qp_launch_sender_fused(ctx, d_x, dtype, n, bits, use_ds, bmode, steps, hist_bins,
+                                    qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_packed, d_qp_out, st,
+                                    static_cast<cudaStream_t>(stream));
+        if (rc == QP_OK && use_ds) ctx->last_steps = steps;
+        if (rc != QP_WARN_INFEASIBLE) return rc;               // else: this device cannot hold the grid
+    }
+    rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
+    if (rc < 0) return rc;
+    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
+    else        rc = qp_aciq_qparams_device(ctx, st, bits, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
+    if (rc < 0) return rc;
+    return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
+}
+
 extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
                                     int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
                                     qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream)
@@ -597,16 +648,13 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
                                        (unsigned long long)dtype | (unsigned long long)bits << 8 |
                                            (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
                                            (unsigned long long)(use_ds != 0) << 28 |
+                                           (unsigned long long)ctx->sender_path << 29 |
                                            (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
                                        packed_capacity, (unsigned long long)(uintptr_t)d_qp_out,
                                        (unsigned long long)(uintptr_t)st};
     return qp_graphed(ctx, static_cast<cudaStream_t>(stream), key, [&]() -> int32_t {
-        int32_t rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
-        if (rc < 0) return rc;
-        if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
-        else        rc = qp_aciq_qparams_device(ctx, st, bits, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
-        if (rc < 0) return rc;
-        return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
+        return sender_on_device(ctx, d_x, dtype, n, bits, use_ds, bmode, steps, hist_bins, d_packed, packed_capacity,
+                                d_qp_out, st, stream);
     });
 }
 
@@ -632,13 +680,8 @@ extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint6
         if (n && cudaMemcpyAsync(d_x_work, h_x, n * esz, cudaMemcpyHostToDevice, s) != cudaSuccess)
             return qp_check_launch(ctx, "qp_sender_host (copy in)");
     }
-    int32_t rc = qp_stats(ctx, d_x_work, dtype, n, use_ds ? hist_bins : 0, ctx->d_tmp_stats, stream);
-    if (rc < 0) return rc;
-    if (use_ds) rc = qp_dsaciq_search(ctx, d_x_work, dtype, n, ctx->d_tmp_stats, bits, bmode, steps, hist_bins, nullptr,
-                                      ctx->d_tmp_qp, stream);
-    else        rc = qp_aciq_qparams_device(ctx, ctx->d_tmp_stats, bits, QP_DIST_LAPLACE, bmode, ctx->d_tmp_qp, stream);
-    if (rc < 0) return rc;
-    rc = qp_quantize_pack(ctx, d_x_work, dtype, n, bits, ctx->d_tmp_qp, 1, d_packed_work, need, stream);
+    int32_t rc = sender_on_device(ctx, d_x_work, dtype, n, bits, use_ds, bmode, steps, hist_bins, d_packed_work, need,
+                                  ctx->d_tmp_qp, ctx->d_tmp_stats, stream);
     if (rc < 0) return rc;
     qp_device_guard guard(ctx->device);
     cudaError_t e = cudaSuccess;

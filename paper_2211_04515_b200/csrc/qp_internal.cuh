@@ -49,7 +49,7 @@ struct qp_graph_entry {
     int32_t rc;                          // status the recorded call returned (QP_OK or a warning)
     unsigned long long used;
 };
-#define QP_GRAPH_SLOTS 32
+#define QP_GRAPH_SLOTS 64
 
 struct qp_ctx {
     int device;
@@ -73,6 +73,9 @@ struct qp_ctx {
     qp_iv_total* d_iv_tot;               // [QP_IV_MAXB + 1]
     int iv_blocks;                       // blocks of the interval-moment kernel (fixed per context)
     int search_path;                     // 0 auto, 1 candidate scoring, 2 interval moments
+    int sender_path;                     // 0 auto, 1 kernel chain, 2 single cooperative launch where it applies
+    int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
+    void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
     qp_qparams_t* d_tmp_qp;
     unsigned long long launches;         // kernels launched through this context (host count)
@@ -265,6 +268,34 @@ __device__ inline void qp_ds_candidate(const qp_ds_setup& s, int k, int steps, i
     c = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
 }
 
+// One thread: the search's result record and the winning quantizer for the chosen step `best`.
+__device__ inline void qp_ds_write_result(int best, const double* s_curve, const qp_ds_setup& s, int steps, int nb, int bits,
+                                          float4 c, qp_ds_result_t* __restrict__ out, qp_qparams_t* __restrict__ qp_out,
+                                          unsigned* __restrict__ status)
+{
+    const double b_star = s.b_e + (double)best * (s.b_r - s.b_e) / (double)steps;
+    if (out) {
+        out->b_e = s.b_e;
+        out->b_r = s.b_r;
+        out->b_star = b_star;
+        out->alpha_e = s.F * s.b_e;
+        out->alpha_star = s.F * b_star;
+        out->mse_e = s_curve[0];
+        out->mse_star = s_curve[best];
+        out->k_star = best;
+        out->steps = steps;
+        out->hist_bins = nb;
+        out->bits = bits;
+    }
+    const bool degenerate_q = !(c.y > c.x);
+    if (qp_out) {
+        qp_out->lo = c.x; qp_out->hi = c.y; qp_out->scale = c.z; qp_out->inv_scale = c.w;
+        qp_out->bits = bits;
+        qp_out->flags = degenerate_q ? 1 : 0;
+    }
+    if (s.degenerate || degenerate_q) atomicOr(status, QP_DEV_DEGENERATE);
+}
+
 // Block-wide: first minimum of the MSE curve wins (k = 0 keeps b_E); writes the result and
 // the winning quantizer.  s_curve: shared scratch of steps + 1 doubles.
 __device__ inline void qp_ds_pick(const double* __restrict__ curve, int steps, int nb, int bits,
@@ -280,28 +311,7 @@ __device__ inline void qp_ds_pick(const double* __restrict__ curve, int steps, i
     double best_mse = s_curve[0];
     for (int k = 1; k <= steps; ++k)
         if (s_curve[k] < best_mse) { best_mse = s_curve[k]; best = k; }
-    const double b_star = s.b_e + (double)best * (s.b_r - s.b_e) / (double)steps;
-    if (out) {
-        out->b_e = s.b_e;
-        out->b_r = s.b_r;
-        out->b_star = b_star;
-        out->alpha_e = s.F * s.b_e;
-        out->alpha_star = s.F * b_star;
-        out->mse_e = s_curve[0];
-        out->mse_star = best_mse;
-        out->k_star = best;
-        out->steps = steps;
-        out->hist_bins = nb;
-        out->bits = bits;
-    }
-    const float4 c = __ldcg(&cand[best]);
-    const bool degenerate_q = !(c.y > c.x);
-    if (qp_out) {
-        qp_out->lo = c.x; qp_out->hi = c.y; qp_out->scale = c.z; qp_out->inv_scale = c.w;
-        qp_out->bits = bits;
-        qp_out->flags = degenerate_q ? 1 : 0;
-    }
-    if (s.degenerate || degenerate_q) atomicOr(status, QP_DEV_DEGENERATE);
+    qp_ds_write_result(best, s_curve, s, steps, nb, bits, __ldcg(&cand[best]), out, qp_out, status);
 }
 
 #endif  // __CUDACC__
@@ -315,6 +325,10 @@ int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
 int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                                   int bits, int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                                   qp_qparams_t* d_qp_out, cudaStream_t s);
+bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins);
+int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+                               int steps, int hist_bins, double F, void* d_packed, qp_qparams_t* d_qp_out,
+                               qp_stats_t* d_stats_out, cudaStream_t s);
 int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
                               qp_qparams_t* d_qp_out, cudaStream_t s);
 int32_t qp_launch_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, const qp_qparams_t* d_qp,

@@ -412,11 +412,129 @@ def test_sender_device_equals_separate_calls(ctx, bits, use_ds):
     else:
         d_qp = ctx.qp_aciq_qparams_device(d_stats, bits)
     want = ctx.qp_quantize_pack(d, bits, d_qp)
-    got, got_qp = ctx.qp_sender_device(d, bits, use_ds)
+    ctx.qp_set_sender_path(qp.QP_SENDER_CHAIN)               # the chain is bit for bit the separate calls
+    try:
+        got, got_qp = ctx.qp_sender_device(d, bits, use_ds)
+    finally:
+        ctx.qp_set_sender_path(qp.QP_SENDER_AUTO)
     assert torch.equal(got, want) and torch.equal(got_qp, d_qp)
     q = ctx.read_qparams(got_qp)
     o = oracle.QParams(q.lo, q.hi, q.scale, q.inv_scale, q.bits, q.flags)
     assert np.array_equal(got.cpu().numpy(), oracle.quantize_pack(x, o))
+
+
+def check_fused_sender(x_np, d_x, bits, use_ds, bmode=0, steps=100, nb=100, curve_rtol=2e-6, tie_rtol=1e-6):
+    """The single-launch sender against the oracle: statistics, clip (a step of the search that the
+    oracle's curve ranks within the tie tolerance of its minimum), and the packed stream bit for
+    bit under the quantizer the kernel chose."""
+    c = qp.Context(0)
+    try:
+        c.qp_set_sender_path(qp.QP_SENDER_FUSED)
+        n = x_np.size
+        nbytes = qp.qp_packed_bytes(n, bits)
+        whole, packed = guarded(nbytes)
+        d_stats = torch.empty(ctypes.sizeof(qp.Stats), dtype=torch.uint8, device="cuda")
+        before = c.qp_launch_count()
+        _, d_qp = c.qp_sender_device(d_x, bits, use_ds, out_packed=packed, out_stats=d_stats, bmode=bmode, steps=steps,
+                                     hist_bins=nb)
+        torch.cuda.synchronize()
+        assert c.qp_launch_count() - before == 1                      # one kernel did all of it
+        assert canaries_intact(whole, nbytes)
+        st, st_o = c.read_stats(d_stats), oracle.stats(x_np)
+        check_stats(st, st_o)
+        got = c.read_qparams(d_qp)
+        assert got.bits == bits
+        if use_ds:
+            assert st.hist_bins == nb
+            rc_o, res_o, qp_o, curve_o = oracle.ds_search(x_np, st_o, bits, bmode, steps, nb)
+            curve = np.array(c.qp_dsaciq_curve(steps))
+            fin = np.isfinite(curve_o)
+            assert np.array_equal(np.isfinite(curve), fin)
+            # fp32 error of one element's d = dq - x is ~2^-23 |x|, so d^2 is off by 2 |d| 2^-23 |x|; over n
+            # elements these average out as 1/sqrt(n), which only matters for a handful of elements
+            xmax = float(np.max(np.abs(x_np[np.isfinite(x_np)]), initial=0.0))
+            small_n = 12 * 2.0 ** -23 * xmax * np.sqrt(curve_o[fin]) / np.sqrt(n)
+            assert np.all(np.abs(curve[fin] - curve_o[fin]) <= curve_rtol * curve_o[fin] + small_n + 1e-300)
+            F = oracle.aciq_F(bits, 0)
+            ends = []
+            for k in np.flatnonzero(fin & (curve_o <= res_o.mse_star * (1 + tie_rtol))):
+                alpha = F * (res_o.b_e + k * (res_o.b_r - res_o.b_e) / steps)
+                q = oracle.make_qparams(st_o.mean - alpha, st_o.mean + alpha, bits)[1]
+                ends.append((q.lo, q.hi, alpha))
+            assert any(abs(got.lo - lo) <= 1e-5 * a + 1e-30 and abs(got.hi - hi) <= 1e-5 * a + 1e-30 for lo, hi, a in ends)
+        else:
+            rc_o, alpha_o, qp_o = oracle.aciq_alpha(st_o, bits, 0, bmode, 0.0)
+            assert abs(got.lo - qp_o.lo) <= 1e-5 * alpha_o + 1e-30 and abs(got.hi - qp_o.hi) <= 1e-5 * alpha_o + 1e-30
+        rc2, again = oracle.make_qparams(got.lo, got.hi, bits)        # scale and reciprocal follow from the ends
+        assert (again.scale, again.inv_scale, again.flags) == (got.scale, got.inv_scale, got.flags)
+        o = oracle.QParams(got.lo, got.hi, got.scale, got.inv_scale, got.bits, got.flags)
+        assert np.array_equal(packed.cpu().numpy(), oracle.quantize_pack(x_np, o))
+        return c.qp_get_status(), got
+    finally:
+        c.close()
+
+
+@pytest.mark.parametrize("bits,use_ds", [(1, True), (2, True), (3, True), (4, True), (8, True), (3, False), (5, False),
+                                         (6, False), (8, False), (16, False)])
+def test_fused_sender_c1(bits, use_ds):
+    x = si.config_tensor("c1").reshape(-1)
+    status, _ = check_fused_sender(x, dev(x), bits, use_ds)
+    assert status == 0
+
+
+@pytest.mark.parametrize("n", RAGGED + [151297, (1 << 20) - 5, 1 << 20])
+def test_fused_sender_ragged_and_misaligned(n):
+    x = si.vit_activation((1, n + 2, 1), 30 + n % 7).reshape(-1).astype(np.float32)
+    d = dev(x)
+    for off, bits, use_ds in ((0, 2, True), (1, 3, False), (1, 4, True), (0, 16, False), (0, 1, False)):
+        if n == 1 and use_ds:
+            continue                                                  # one element: nothing to search
+        status, _ = check_fused_sender(x[off:off + n], d[off:off + n], bits, use_ds)
+        assert status & ~qp.QP_DEV_DEGENERATE == 0
+
+
+def test_fused_sender_special_values_modes_and_bf16():
+    x = si.vit_activation((3, 197, 200), 31, outlier_frac=0.02).reshape(-1)
+    x[[0, 77, x.size - 1]] = [np.nan, np.inf, -np.inf]
+    for bits, use_ds in ((2, True), (8, False)):
+        status, _ = check_fused_sender(x, dev(x), bits, use_ds)
+        assert status == qp.QP_DEV_NONFINITE
+    x = si.vit_activation((2, 197, 160), 32).reshape(-1)
+    check_fused_sender(x, dev(x), 4, True, bmode=1, steps=127, nb=4096)
+    check_fused_sender(x, dev(x), 2, True, steps=1, nb=1)
+    check_fused_sender(x, dev(x), 6, False, bmode=1)
+    const = np.full(3000, -1.25, dtype=np.float32)                    # no spread: code 0 everywhere
+    for use_ds in (True, False):
+        status, got = check_fused_sender(const, dev(const), 2, use_ds)
+        assert status == qp.QP_DEV_DEGENERATE and got.flags == 1
+    h = si.to_bf16_bits(x)
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    check_fused_sender(oracle.widen_bf16(h), d, 2, True)
+    check_fused_sender(oracle.widen_bf16(h[1:-2]), d[1:-2], 8, False)
+
+
+def test_fused_sender_falls_back_outside_its_range():
+    """Beyond 2^20 elements, 127 steps or 4096 bins the call runs the kernel chain, whatever the path."""
+    c = qp.Context(0)
+    c.qp_set_sender_path(qp.QP_SENDER_FUSED)
+    x = si.vit_activation((1, (1 << 20) + 1, 1), 33).reshape(-1)
+    d = dev(x)
+    for kw in (dict(), ):
+        before = c.qp_launch_count()
+        packed, d_qp = c.qp_sender_device(d, 8, False)
+        assert c.qp_launch_count() - before > 1
+    small = d[:5000]
+    for kw in (dict(steps=128), dict(hist_bins=4097)):
+        before = c.qp_launch_count()
+        c.qp_sender_device(small, 2, True, **kw)
+        assert c.qp_launch_count() - before > 1
+    before = c.qp_launch_count()
+    c.qp_sender_device(small, 2, True)
+    assert c.qp_launch_count() - before == 1
+    with pytest.raises(qp.QuantPipeError):
+        c.qp_set_sender_path(3)
+    assert c.qp_get_status() == 0
+    c.close()
 
 
 def test_sender_and_receiver_host_buffers(ctx):
