@@ -90,6 +90,9 @@ def lib():
         L.orc_unpack.restype = None
         L.orc_aciq_alpha.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_double, dp, C.POINTER(QParams)]
         L.orc_aciq_alpha.restype = C.c_int
+        L.orc_clip_range.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, dp, dp,
+                                     C.POINTER(QParams)]
+        L.orc_clip_range.restype = C.c_int
         L.orc_hist_peak.argtypes = [fp, C.c_uint64, C.c_double, C.c_double, C.c_int, u64p]
         L.orc_hist_peak.restype = C.c_double
         L.orc_ds_search.argtypes = [fp, C.c_uint64, C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int,
@@ -145,6 +148,18 @@ def aciq_alpha(st: Stats, bits: int, dist: int = 0, bmode: int = 0, b_override: 
     qp = QParams()
     rc = lib().orc_aciq_alpha(C.byref(st), bits, dist, bmode, b_override, C.byref(alpha), C.byref(qp))
     return rc, alpha.value, qp
+
+
+CLIP_ACIQ, CLIP_MINMAX = 0, 2
+
+
+def clip_range(st: Stats, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0):
+    """(rc, lo, hi, quantizer) of the clip range by method: ACIQ, or naive PTQ's [min, max]."""
+    lo, hi = C.c_double(), C.c_double()
+    qp = QParams()
+    rc = lib().orc_clip_range(C.byref(st), bits, method, 1 if intersect else 0, dist, bmode, C.byref(lo), C.byref(hi),
+                              C.byref(qp))
+    return rc, lo.value, hi.value, qp
 
 
 def quantize(x, qp: QParams) -> np.ndarray:

@@ -294,6 +294,40 @@ int orc_aciq_alpha(const orc_stats_t* st, int bits, int dist, int bmode, double 
     return ORC_OK;
 }
 
+/* Clip range by method (Sec. 3, "Naive PTQ and ACIQ").
+ *   method 0  ACIQ: [mean - alpha, mean + alpha] with alpha = F(q) b, as orc_aciq_alpha
+ *   method 2  naive PTQ: the tensor's own [min, max]
+ * intersect != 0 (method 0 only): the ACIQ range cut back to the data's range,
+ *   [max(mean - alpha, min), min(mean + alpha, max)].  No element lies outside [min, max], so
+ *   the clipping error is unchanged while the step gets smaller whenever alpha reaches past
+ *   the data.  This is a variant of this library; the paper clips at mean -/+ alpha only. */
+int orc_clip_range(const orc_stats_t* st, int bits, int method, int intersect, int dist, int bmode,
+                   double* lo_out, double* hi_out, orc_qparams_t* qp)
+{
+    if (!bits_ok(bits)) return ORC_ERR_BITS;
+    if (method != 0 && method != 2) return ORC_ERR_ARG;
+    if (method == 2 && intersect) return ORC_ERR_ARG;
+    double lo, hi;
+    if (method == 2) {
+        lo = st->min;
+        hi = st->max;
+    } else {
+        double alpha;
+        int rc = orc_aciq_alpha(st, bits, dist, bmode, 0.0, &alpha, NULL);
+        if (rc < 0) return rc;
+        lo = st->mean - alpha;
+        hi = st->mean + alpha;
+        if (intersect) {
+            if (st->min > lo) lo = st->min;
+            if (st->max < hi) hi = st->max;
+        }
+    }
+    if (lo_out) *lo_out = lo;
+    if (hi_out) *hi_out = hi;
+    if (qp) return orc_make_qparams(lo, hi, bits, qp);
+    return ORC_OK;
+}
+
 /* ------------------------------------------------------- histogram of D_R */
 
 /* Density histogram D_R of the data, nb equal bins over [min, max] (Sec. 3, directed

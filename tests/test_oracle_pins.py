@@ -480,6 +480,61 @@ def test_select_bits_principle():
     assert oracle.select_bits(1e6, 1.0, 10, 0, (0,))[0] == oracle.ERR_ARG
 
 
+# ------------------------------------------------------------- clip range by method
+
+def test_naive_ptq_range_is_min_max_hand_example():
+    """Sec. 3: naive PTQ divides the tensor's own range into equal intervals.  By hand: the values
+    0, 0.9, 2.2, 3 at 2 bits have range [0, 3], four levels 0, 1, 2, 3 -> codes 0, 1, 2, 3 and
+    reconstructions 0, 1, 2, 3."""
+    x = np.array([0.0, 0.9, 2.2, 3.0], dtype=np.float32)
+    rc, lo, hi, q = oracle.clip_range(oracle.stats(x), 2, oracle.CLIP_MINMAX)
+    assert rc == 0 and (lo, hi) == (0.0, 3.0) and q.scale == 1.0
+    codes = oracle.quantize(x, q)
+    assert codes.tolist() == [0, 1, 2, 3]
+    assert oracle.dequantize(codes, q).tolist() == [0.0, 1.0, 2.0, 3.0]
+    # the extremes always take the end codes and are reconstructed exactly
+    y = si.flat_iid(10000, 9, "laplace")
+    for bits in (1, 3, 8, 16):
+        rc, lo, hi, q = oracle.clip_range(oracle.stats(y), bits, oracle.CLIP_MINMAX)
+        c = oracle.quantize(y, q)
+        assert c[np.argmin(y)] == 0 and c[np.argmax(y)] == (1 << bits) - 1
+        d = oracle.dequantize(c, q)
+        assert d[np.argmin(y)] == y.min() and abs(d[np.argmax(y)] - y.max()) <= 2e-7 * abs(y.max())
+        # nothing is clipped; the position on the grid is an fp32 number of up to 2^bits, so half a
+        # step is met up to its rounding
+        assert np.max(np.abs(d - y)) <= (0.5 + 2.0 ** -22 * (1 << bits)) * q.scale
+
+
+def test_clip_range_aciq_equals_aciq_alpha_and_intersection_properties():
+    y = si.flat_iid(50000, 10, "laplace") * np.float32(0.7) + np.float32(0.3)
+    st = oracle.stats(y)
+    for bits in (2, 4, 8, 16):
+        rc, alpha, q_a = oracle.aciq_alpha(st, bits)
+        rc, lo, hi, q = oracle.clip_range(st, bits, oracle.CLIP_ACIQ)
+        assert (lo, hi) == (st.mean - alpha, st.mean + alpha) and bytes(q) == bytes(q_a)
+        rc, lo_i, hi_i, q_i = oracle.clip_range(st, bits, oracle.CLIP_ACIQ, intersect=True)
+        assert lo_i == max(lo, st.min) and hi_i == min(hi, st.max)       # never wider, never inside the data
+        if lo > st.min and hi < st.max:
+            assert bytes(q_i) == bytes(q)                                # alpha inside the data: nothing changes
+    # at 16 bits alpha = F(16) b reaches far past this sample's extremes: the cut range is naive PTQ's
+    rc, lo_i, hi_i, q_i = oracle.clip_range(st, 16, oracle.CLIP_ACIQ, intersect=True)
+    rc, lo_n, hi_n, q_n = oracle.clip_range(st, 16, oracle.CLIP_MINMAX)
+    assert (lo_i, hi_i) == (lo_n, hi_n) == (st.min, st.max) and bytes(q_i) == bytes(q_n)
+    # and it lowers the error there (same clipping error - none - and a smaller step)
+    rc, lo, hi, q = oracle.clip_range(st, 16, oracle.CLIP_ACIQ)
+    assert oracle.quant_mse(y, q_i) < 0.5 * oracle.quant_mse(y, q)
+    # a one-sided cut: shift the data so that only the lower end of the ACIQ range passes the minimum
+    z = np.abs(y).astype(np.float32)
+    sz = oracle.stats(z)
+    rc, lo, hi, q = oracle.clip_range(sz, 3, oracle.CLIP_ACIQ)
+    rc, lo_i, hi_i, q_i = oracle.clip_range(sz, 3, oracle.CLIP_ACIQ, intersect=True)
+    assert lo < sz.min and hi < sz.max and lo_i == sz.min and hi_i == hi
+    assert oracle.quant_mse(z, q_i) < oracle.quant_mse(z, q)
+    assert oracle.clip_range(st, 9)[0] == oracle.ERR_BITS
+    assert oracle.clip_range(st, 4, 1)[0] == oracle.ERR_ARG               # the search is not a closed form
+    assert oracle.clip_range(st, 4, oracle.CLIP_MINMAX, intersect=True)[0] == oracle.ERR_ARG
+
+
 # ------------------------------------------------------------------- inputs
 
 def test_generator_is_counter_based_and_shaped():
