@@ -179,6 +179,25 @@ int32_t qp_aciq_alpha(const qp_stats_t* h_stats, int bits, int dist, int bmode, 
  * *d_qp_out, so that stats -> clip -> quantize needs no host round trip. */
 int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode,
                                qp_qparams_t* d_qp_out, void* stream);
+/* Clip range by method (Sec. 3, "Naive PTQ and ACIQ"):
+ *   QP_CLIP_ACIQ    [mean - alpha, mean + alpha], alpha = F(q) b (as qp_aciq_alpha)
+ *   QP_CLIP_DSACIQ  ACIQ refined by the directed search (qp_dsaciq_search / qp_sender_*; not a
+ *                   closed form of the statistics, so not accepted by the two calls below)
+ *   QP_CLIP_MINMAX  naive PTQ: the tensor's own [min, max]
+ * QP_CLIP_ACIQ | QP_CLIP_INTERSECT cuts the ACIQ range back to the data's range,
+ * [max(mean - alpha, min), min(mean + alpha, max)]: no element lies outside [min, max], so
+ * the clipping error is unchanged and the step shrinks whenever alpha reaches past the data
+ * (a variant of this library; the paper clips at mean -/+ alpha only).
+ * qp_clip_range: host form, writes the ends (optional) and the quantizer (optional).
+ * qp_clip_qparams_device: one-thread kernel from device-resident statistics.
+ * Errors: QP_ERR_INVALID_ARG (NULL, unknown method, dist, bmode), QP_ERR_UNSUPPORTED_BITS;
+ * QP_WARN_DEGENERATE as qp_make_qparams (host form; status word on the device). */
+enum { QP_CLIP_ACIQ = 0, QP_CLIP_DSACIQ = 1, QP_CLIP_MINMAX = 2 };
+#define QP_CLIP_INTERSECT 0x10
+int32_t qp_clip_range(const qp_stats_t* h_stats, int bits, int method, int dist, int bmode, double* h_lo_out,
+                      double* h_hi_out, qp_qparams_t* h_qp_out);
+int32_t qp_clip_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int method, int dist, int bmode,
+                               qp_qparams_t* d_qp_out, void* stream);
 
 /* ---- a2 + a4: directed search DS-ACIQ (Sec. 3 "Directed Search", Eq. 1) -----------------
  * Histogram of x with hist_bins equal bins over [min, max]; b_R = 1 / (2 * peak density);
@@ -296,7 +315,7 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------
  * qp_sender_host: copies the n elements at h_x to d_x_work, runs statistics, the clip
- * (directed search when use_ds != 0, plain ACIQ otherwise; Laplace model), quantize+pack
+ * by `method` (as qp_sender_device), quantize+pack
  * into d_packed_work, and copies the packed stream to h_packed and the quantizer to
  * *h_qp_out.  qp_receiver_host: copies h_packed to d_packed_work, unpacks+dequantizes into
  * d_y_work and copies the tensor to h_y.  Everything is enqueued on `stream`; host outputs
@@ -306,8 +325,9 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  * (d_packed_work 16-byte aligned), d_y_work and h_y >= n elements of out_dtype.
  * Errors: as the calls they are made of. */
 /* qp_sender_device: the sender's whole chain on DEVICE buffers in one call, nothing read back
- * to the host: statistics (carrying the histogram along when use_ds != 0), the clip
- * (directed search when use_ds != 0, plain ACIQ otherwise; Laplace model), quantize+pack.
+ * to the host: statistics (carrying the histogram along for the search), the clip by
+ * `method` (QP_CLIP_ACIQ = 0, optionally | QP_CLIP_INTERSECT; QP_CLIP_DSACIQ = 1, bits <= 8;
+ * QP_CLIP_MINMAX = 2; Laplace model), quantize+pack.
  * Writes the packed stream to d_packed, the quantizer to *d_qp_out (what the receiver needs)
  * and, if d_stats_out is not NULL, the statistics.  Equivalent to qp_stats +
  * qp_dsaciq_search / qp_aciq_qparams_device + qp_quantize_pack with the same arguments.
@@ -327,10 +347,10 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  * QP_DEV_STREAM_TIMEOUT in the status word and the launch ends without output. */
 enum { QP_SENDER_AUTO = 0, QP_SENDER_CHAIN = 1, QP_SENDER_FUSED = 2 };
 int32_t qp_set_sender_path(qp_ctx* ctx, int path);
-int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,
                          int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
                          qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream);
-int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int method, int bmode,
                        int steps, int hist_bins, void* d_x_work, void* d_packed_work, void* h_packed,
                        uint64_t packed_capacity, qp_qparams_t* h_qp_out, void* stream);
 int32_t qp_receiver_host(qp_ctx* ctx, const void* h_packed, uint64_t n, int bits, const qp_qparams_t* h_qp,

@@ -27,6 +27,7 @@ QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
+QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT = 0, 1, 2, 0x10
 
 EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
@@ -34,6 +35,7 @@ EXPORTS = (
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
+    "qp_clip_range", "qp_clip_qparams_device",
 )
 
 
@@ -99,6 +101,9 @@ def load() -> C.CDLL:
     L.qp_stats.argtypes = [vp, vp, C.c_int, u64, C.c_int, vp, vp]
     L.qp_aciq_alpha.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, dbl, C.POINTER(dbl), C.POINTER(QParams)]
     L.qp_aciq_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.qp_clip_range.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(dbl), C.POINTER(dbl),
+                                C.POINTER(QParams)]
+    L.qp_clip_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.qp_dsaciq_search.argtypes = [vp, vp, C.c_int, u64, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
     L.qp_dsaciq_curve.argtypes = [vp, C.POINTER(dbl), C.c_int, vp]
     L.qp_policy_use_ds.argtypes = [C.c_int]
@@ -156,6 +161,15 @@ def qp_aciq_alpha(stats: Stats, bits: int, dist: int = QP_DIST_LAPLACE, bmode: i
     alpha, qp = C.c_double(), QParams()
     rc = load().qp_aciq_alpha(C.byref(stats), bits, dist, bmode, b_override, C.byref(alpha), C.byref(qp))
     return int(rc), alpha.value, qp
+
+
+def qp_clip_range(stats: Stats, bits: int, method: int = QP_CLIP_ACIQ, dist: int = QP_DIST_LAPLACE,
+                  bmode: int = QP_B_MAD):
+    """(status, lo, hi, quantizer) of the closed-form clip range: ACIQ (optionally | QP_CLIP_INTERSECT)
+    or QP_CLIP_MINMAX."""
+    lo, hi, qp = C.c_double(), C.c_double(), QParams()
+    rc = load().qp_clip_range(C.byref(stats), bits, method, dist, bmode, C.byref(lo), C.byref(hi), C.byref(qp))
+    return int(rc), lo.value, hi.value, qp
 
 
 def qp_policy_use_ds(bits: int) -> bool:
@@ -285,6 +299,14 @@ class Context:
         return out
 
     # -- a3
+    def qp_clip_qparams_device(self, d_stats: torch.Tensor, bits: int, method: int = QP_CLIP_ACIQ,
+                               dist: int = QP_DIST_LAPLACE, bmode: int = QP_B_MAD,
+                               out: torch.Tensor | None = None) -> torch.Tensor:
+        out = self._bytes(C.sizeof(QParams)) if out is None else out
+        self._check(self._lib.qp_clip_qparams_device(self._h, d_stats.data_ptr(), bits, method, dist, bmode,
+                                                     out.data_ptr(), _stream(self.device)))
+        return out
+
     def qp_aciq_qparams_device(self, d_stats: torch.Tensor, bits: int, dist: int = QP_DIST_LAPLACE,
                                bmode: int = QP_B_MAD, out: torch.Tensor | None = None) -> torch.Tensor:
         out = self._bytes(C.sizeof(QParams)) if out is None else out
@@ -353,12 +375,13 @@ class Context:
     def qp_sender_device(self, x: torch.Tensor, bits: int, use_ds: bool, out_packed: torch.Tensor | None = None,
                          out_qp: torch.Tensor | None = None, out_stats: torch.Tensor | None = None,
                          bmode: int = QP_B_MAD, steps: int = QP_DEFAULT_STEPS, hist_bins: int = QP_DEFAULT_HIST_BINS):
-        """stats -> clip -> quantize+pack in one call; returns (packed, device QParams bytes)."""
+        """stats -> clip -> quantize+pack in one call; returns (packed, device QParams bytes).
+        use_ds: False/True (ACIQ / directed search) or a QP_CLIP_* method."""
         assert x.is_cuda and x.is_contiguous()
         out_packed = self._bytes(qp_packed_bytes(x.numel(), bits)) if out_packed is None else out_packed
         out_qp = self._bytes(C.sizeof(QParams)) if out_qp is None else out_qp
         self._check(self._lib.qp_sender_device(self._h, x.data_ptr(), _dtype_code(x), x.numel(), bits,
-                                               1 if use_ds else 0, bmode, steps, hist_bins, out_packed.data_ptr(),
+                                               int(use_ds), bmode, steps, hist_bins, out_packed.data_ptr(),
                                                out_packed.numel() * out_packed.element_size(), out_qp.data_ptr(),
                                                out_stats.data_ptr() if out_stats is not None else None,
                                                _stream(self.device)))
@@ -371,7 +394,7 @@ class Context:
         """Host tensor in, packed host bytes + quantizer out (valid after a stream synchronise)."""
         assert not h_x.is_cuda and h_x.is_contiguous() and not h_packed.is_cuda
         self._check(self._lib.qp_sender_host(self._h, h_x.data_ptr(), _dtype_code(h_x), h_x.numel(), bits,
-                                             1 if use_ds else 0, bmode, steps, hist_bins, d_x_work.data_ptr(),
+                                             int(use_ds), bmode, steps, hist_bins, d_x_work.data_ptr(),
                                              d_packed_work.data_ptr(), h_packed.data_ptr(),
                                              h_packed.numel() * h_packed.element_size(), C.byref(h_qp_out),
                                              _stream(self.device)))

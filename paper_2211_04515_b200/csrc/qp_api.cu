@@ -255,6 +255,28 @@ extern "C" int32_t qp_aciq_alpha(const qp_stats_t* h_stats, int bits, int dist, 
     return qp_fill_qparams(lo, hi, bits, h_qp_out);
 }
 
+static bool clip_method_closed_form(int method)
+{
+    return method == QP_CLIP_ACIQ || method == (QP_CLIP_ACIQ | QP_CLIP_INTERSECT) || method == QP_CLIP_MINMAX;
+}
+
+extern "C" int32_t qp_clip_range(const qp_stats_t* h_stats, int bits, int method, int dist, int bmode, double* h_lo_out,
+                                 double* h_hi_out, qp_qparams_t* h_qp_out)
+{
+    if (!h_stats) return QP_ERR_INVALID_ARG;
+    if (!qp_bits_ok(bits)) return QP_ERR_UNSUPPORTED_BITS;
+    if (!clip_method_closed_form(method)) return QP_ERR_INVALID_ARG;
+    if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
+        return QP_ERR_INVALID_ARG;
+    double lo, hi;
+    qp_clip_ends(*h_stats, method, dist, bmode, qp_host_aciq_F(bits, dist), lo, hi);
+    if (h_lo_out) *h_lo_out = lo;
+    if (h_hi_out) *h_hi_out = hi;
+    if (!h_qp_out) return QP_OK;
+    if (!isfinite(lo) || !isfinite(hi)) return QP_ERR_INVALID_ARG;
+    return qp_fill_qparams(lo, hi, bits, h_qp_out);
+}
+
 extern "C" int32_t qp_policy_use_ds(int bits) { return bits >= 1 && bits <= 4 ? 1 : 0; }
 
 extern "C" int32_t qp_select_bits(double bandwidth_bps, double budget_s, uint64_t n_elems, uint64_t overhead_bytes,
@@ -491,7 +513,22 @@ extern "C" int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats
         return qp_fail(ctx, QP_ERR_INVALID_ARG, "dist/bmode");
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
-    return qp_launch_aciq_device(ctx, d_stats, bits, dist, bmode, qp_host_aciq_F(bits, dist), d_qp_out,
+    return qp_launch_aciq_device(ctx, d_stats, bits, QP_CLIP_ACIQ, dist, bmode, qp_host_aciq_F(bits, dist), d_qp_out,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+extern "C" int32_t qp_clip_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int method, int dist,
+                                          int bmode, qp_qparams_t* d_qp_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (!d_stats || !d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (!clip_method_closed_form(method)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT) or MINMAX");
+    if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "dist/bmode");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    return qp_launch_aciq_device(ctx, d_stats, bits, method, dist, bmode, qp_host_aciq_F(bits, dist), d_qp_out,
                                  static_cast<cudaStream_t>(stream));
 }
 
@@ -602,11 +639,12 @@ extern "C" int32_t qp_unpack_dequantize(qp_ctx* ctx, const void* d_packed, uint6
 
 // statistics -> clip -> quantize+pack on device buffers: one cooperative launch where that
 // applies (small tensors), the kernel chain of the separate calls otherwise
-static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,
                                 int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
                                 qp_qparams_t* d_qp_out, qp_stats_t* st, void* stream)
 {
     int32_t rc;
+    const int use_ds = method == QP_CLIP_DSACIQ;
     if (ctx->sender_path != QP_SENDER_CHAIN && qp_sender_fused_applies(n, use_ds, steps, hist_bins)) {
         // the checks of the separate calls
         rc = check_x(ctx, d_x, dtype, n);
@@ -618,7 +656,7 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
         if (((uintptr_t)st & 7u) || ((uintptr_t)d_qp_out & 3u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "result pointers");
         qp_device_guard guard(ctx->device);
         if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
-        rc = qp_launch_sender_fused(ctx, d_x, dtype, n, bits, use_ds, bmode, steps, hist_bins,
+        rc = qp_launch_sender_fused(ctx, d_x, dtype, n, bits, method, bmode, steps, hist_bins,
                                     qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_packed, d_qp_out, st,
                                     static_cast<cudaStream_t>(stream));
         if (rc == QP_OK && use_ds) ctx->last_steps = steps;
@@ -627,19 +665,20 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
     rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
     if (rc < 0) return rc;
     if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
-    else        rc = qp_aciq_qparams_device(ctx, st, bits, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
+    else        rc = qp_clip_qparams_device(ctx, st, bits, method, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
     if (rc < 0) return rc;
     return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
 }
 
-extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,
                                     int steps, int hist_bins, void* d_packed, uint64_t packed_capacity,
                                     qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream)
 {
     if (!ctx) return QP_ERR_INVALID_ARG;
     if (!d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_qp_out");
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    if (use_ds && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if (method != QP_CLIP_DSACIQ && !clip_method_closed_form(method)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "clip method");
+    if (method == QP_CLIP_DSACIQ && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
     if (packed_capacity < qp_packed_bytes(n, bits))
         return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
     qp_stats_t* st = d_stats_out ? d_stats_out : ctx->d_tmp_stats;
@@ -647,27 +686,28 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
     const unsigned long long key[8] = {3, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_packed,
                                        (unsigned long long)dtype | (unsigned long long)bits << 8 |
                                            (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
-                                           (unsigned long long)(use_ds != 0) << 28 |
+                                           (unsigned long long)(method == QP_CLIP_DSACIQ) << 28 | (unsigned long long)method << 56 |
                                            (unsigned long long)ctx->sender_path << 29 |
                                            (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
                                        packed_capacity, (unsigned long long)(uintptr_t)d_qp_out,
                                        (unsigned long long)(uintptr_t)st};
     return qp_graphed(ctx, static_cast<cudaStream_t>(stream), key, [&]() -> int32_t {
-        return sender_on_device(ctx, d_x, dtype, n, bits, use_ds, bmode, steps, hist_bins, d_packed, packed_capacity,
+        return sender_on_device(ctx, d_x, dtype, n, bits, method, bmode, steps, hist_bins, d_packed, packed_capacity,
                                 d_qp_out, st, stream);
     });
 }
 
 // ------------------------------------------- host-buffer sender and receiver
 
-extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint64_t n, int bits, int method, int bmode,
                                   int steps, int hist_bins, void* d_x_work, void* d_packed_work, void* h_packed,
                                   uint64_t packed_capacity, qp_qparams_t* h_qp_out, void* stream)
 {
     if (!ctx) return QP_ERR_INVALID_ARG;
     if (dtype != QP_F32 && dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "dtype");
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    if (use_ds && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if (method != QP_CLIP_DSACIQ && !clip_method_closed_form(method)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "clip method");
+    if (method == QP_CLIP_DSACIQ && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
     if (!h_qp_out || (n > 0 && (!h_x || !d_x_work || !d_packed_work || !h_packed)))
         return qp_fail(ctx, QP_ERR_INVALID_ARG, "null buffer");
     const uint64_t need = qp_packed_bytes(n, bits);
@@ -680,7 +720,7 @@ extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint6
         if (n && cudaMemcpyAsync(d_x_work, h_x, n * esz, cudaMemcpyHostToDevice, s) != cudaSuccess)
             return qp_check_launch(ctx, "qp_sender_host (copy in)");
     }
-    int32_t rc = sender_on_device(ctx, d_x_work, dtype, n, bits, use_ds, bmode, steps, hist_bins, d_packed_work, need,
+    int32_t rc = sender_on_device(ctx, d_x_work, dtype, n, bits, method, bmode, steps, hist_bins, d_packed_work, need,
                                   ctx->d_tmp_qp, ctx->d_tmp_stats, stream);
     if (rc < 0) return rc;
     qp_device_guard guard(ctx->device);

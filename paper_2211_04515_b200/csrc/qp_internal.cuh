@@ -231,6 +231,26 @@ __device__ __forceinline__ double qp_block_max(double v, double* sh)
     return r;
 }
 
+// Closed-form clip range from the statistics: ACIQ (optionally cut back to [min, max]) or the
+// tensor's own range; same on host and device.
+__host__ __device__ inline void qp_clip_ends(const qp_stats_t& st, int method, int dist, int bmode, double F, double& lo,
+                                             double& hi)
+{
+    if ((method & 0xF) == QP_CLIP_MINMAX) {
+        lo = st.min;
+        hi = st.max;
+        return;
+    }
+    const double b = dist == QP_DIST_GAUSS ? sqrt(st.var) : (bmode == QP_B_MEAN_ABS ? st.mean_abs : st.mad);
+    const double alpha = F * b;
+    lo = st.mean - alpha;
+    hi = st.mean + alpha;
+    if (method & QP_CLIP_INTERSECT) {
+        if (st.min > lo) lo = st.min;
+        if (st.max < hi) hi = st.max;
+    }
+}
+
 // ---- pieces of the directed search shared by its two scoring paths
 
 // b_E, b_R and friends from the statistics and the histogram's peak count `top`
@@ -326,10 +346,10 @@ int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint6
                                   int bits, int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                                   qp_qparams_t* d_qp_out, cudaStream_t s);
 bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins);
-int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,
                                int steps, int hist_bins, double F, void* d_packed, qp_qparams_t* d_qp_out,
                                qp_stats_t* d_stats_out, cudaStream_t s);
-int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
+int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int method, int dist, int bmode, double F,
                               qp_qparams_t* d_qp_out, cudaStream_t s);
 int32_t qp_launch_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, const qp_qparams_t* d_qp,
                        qp_qparams_t h_qp, void* d_packed, cudaStream_t s);

@@ -238,15 +238,16 @@ __global__ void __launch_bounds__(QP_THREADS) finalize_kernel(const double* __re
     qp_ds_pick(curve, steps, nb, bits, cand, setup, out, qp_out, status, s_curve);
 }
 
-// one thread: ACIQ clip from device-resident statistics
-__global__ void aciq_kernel(const qp_stats_t* __restrict__ st, int bits, int dist, int bmode, double F,
+// one thread: closed-form clip (ACIQ, ACIQ cut back to the data range, or min/max) from
+// device-resident statistics
+__global__ void aciq_kernel(const qp_stats_t* __restrict__ st, int bits, int method, int dist, int bmode, double F,
                             qp_qparams_t* __restrict__ qp_out, unsigned* __restrict__ status)
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
-    const double b = dist == QP_DIST_GAUSS ? sqrt(st->var) : (bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad);
-    const double alpha = F * b;
+    double lo, hi;
+    qp_clip_ends(*st, method, dist, bmode, F, lo, hi);
     qp_qparams_t q;
-    const int rc = qp_fill_qparams(st->mean - alpha, st->mean + alpha, bits, &q);
+    const int rc = qp_fill_qparams(lo, hi, bits, &q);
     *qp_out = q;
     if (rc == QP_WARN_DEGENERATE) atomicOr(status, QP_DEV_DEGENERATE);
 }
@@ -309,10 +310,10 @@ int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
                                         hist_bins, F, d_out, d_qp_out, s);
 }
 
-int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int dist, int bmode, double F,
+int32_t qp_launch_aciq_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int method, int dist, int bmode, double F,
                               qp_qparams_t* d_qp_out, cudaStream_t s)
 {
-    aciq_kernel<<<1, 32, 0, s>>>(d_stats, bits, dist, bmode, F, d_qp_out, ctx->d_status);
+    aciq_kernel<<<1, 32, 0, s>>>(d_stats, bits, method, dist, bmode, F, d_qp_out, ctx->d_status);
     ctx->launches += 1;
     return qp_check_launch(ctx, "qp_aciq_qparams_device");
 }

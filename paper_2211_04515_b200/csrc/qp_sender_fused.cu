@@ -38,7 +38,7 @@ constexpr int K = QP_EVAL_K;
 struct FsArgs {
     const void* x;
     uint64_t n;
-    int bits, use_ds, bmode, steps, nb;
+    int bits, use_ds, method, bmode, steps, nb;         // use_ds: method is the directed search
     double F;
     uint32_t* out;
     uint64_t total_words;
@@ -272,9 +272,9 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
                 s_setup.g_lo = s_setup.g_hi = s_setup.inv_gw = s_setup.inv_u = s_setup.gw = s_setup.pad2 = 0.f;
                 s_setup.u = 0.0;
             } else {
-                const double b = a.bmode == QP_B_MEAN_ABS ? s_st.mean_abs : s_st.mad;
-                const double alpha = a.F * b;
-                const int rc = qp_fill_qparams(mean - alpha, mean + alpha, a.bits, &s_qp);
+                double lo, hi;
+                qp_clip_ends(s_st, a.method, QP_DIST_LAPLACE, a.bmode, a.F, lo, hi);
+                const int rc = qp_fill_qparams(lo, hi, a.bits, &s_qp);
                 if (blockIdx.x == 0) {
                     *a.qp_out = s_qp;
                     if (rc == QP_WARN_DEGENERATE) atomicOr(a.status, QP_DEV_DEGENERATE);
@@ -465,10 +465,11 @@ bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins)
 
 // Returns QP_OK when the launch was enqueued, a negative status on an error, and
 // QP_WARN_INFEASIBLE when this device cannot hold the grid (the caller then runs the chain).
-int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int use_ds, int bmode,
+int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,
                                int steps, int hist_bins, double F, void* d_packed, qp_qparams_t* d_qp_out,
                                qp_stats_t* d_stats_out, cudaStream_t s)
 {
+    const int use_ds = method == QP_CLIP_DSACIQ;
     const uint64_t total_words = qp_packed_bytes(n, bits) / 4;
     const uint64_t groups = (total_words + bits - 1) / bits;             // 32-element groups, pad words included
     const unsigned G = (unsigned)ctx->sm_count;
@@ -497,7 +498,7 @@ int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t
     // The arrival counter and the histogram start at zero: the context allocates them zeroed and
     // every completed launch leaves them so (a timed-out one does not: qp_get_status clears them).
     FsArgs a;
-    a.x = d_x; a.n = n; a.bits = bits; a.use_ds = use_ds; a.bmode = bmode; a.steps = steps; a.nb = hist_bins; a.F = F;
+    a.x = d_x; a.n = n; a.bits = bits; a.use_ds = use_ds; a.method = method; a.bmode = bmode; a.steps = steps; a.nb = hist_bins; a.F = F;
     a.out = static_cast<uint32_t*>(d_packed);
     a.total_words = total_words;
     a.groups_per_block = gpb;

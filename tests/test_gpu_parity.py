@@ -537,6 +537,50 @@ def test_fused_sender_falls_back_outside_its_range():
     c.close()
 
 
+# clip methods of the sender: ACIQ, ACIQ cut back to the data range, naive PTQ's min/max
+CLIP_CASES = [(qp.QP_CLIP_ACIQ, oracle.CLIP_ACIQ, False), (qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT, oracle.CLIP_ACIQ, True),
+              (qp.QP_CLIP_MINMAX, oracle.CLIP_MINMAX, False)]
+
+
+@pytest.mark.parametrize("method,o_method,cut", CLIP_CASES)
+@pytest.mark.parametrize("path", [qp.QP_SENDER_CHAIN, qp.QP_SENDER_FUSED])
+def test_sender_clip_methods(ctx, method, o_method, cut, path):
+    x = si.vit_activation((3, 197, 192), 81, outlier_frac=0.01).reshape(-1)
+    d = dev(x)
+    st_o = oracle.stats(x)
+    ctx.qp_set_sender_path(path)
+    try:
+        for bits in (2, 4, 8, 16):
+            d_stats = torch.empty(ctypes.sizeof(qp.Stats), dtype=torch.uint8, device="cuda")
+            packed, d_qp = ctx.qp_sender_device(d, bits, method, out_stats=d_stats)
+            got = ctx.read_qparams(d_qp)
+            rc_o, lo_o, hi_o, q_o = oracle.clip_range(st_o, bits, o_method, cut)
+            width = hi_o - lo_o
+            assert abs(got.lo - q_o.lo) <= 1e-5 * width and abs(got.hi - q_o.hi) <= 1e-5 * width
+            if method == qp.QP_CLIP_MINMAX:                     # min and max are exact, so is the quantizer
+                assert bytes(got) == bytes(to_qp(q_o))
+            o = oracle.QParams(got.lo, got.hi, got.scale, got.inv_scale, got.bits, got.flags)
+            assert np.array_equal(packed.cpu().numpy(), oracle.quantize_pack(x, o))
+            # the device form of the closed-form clip gives the same quantizer from the same statistics
+            assert torch.equal(ctx.qp_clip_qparams_device(d_stats, bits, method), d_qp)
+    finally:
+        ctx.qp_set_sender_path(qp.QP_SENDER_AUTO)
+    assert ctx.qp_get_status() == 0
+
+
+def test_clip_method_errors(ctx):
+    x = dev(si.flat_iid(4096, 5, "laplace"))
+    d_stats = ctx.qp_stats(x)
+    for bad in (qp.QP_CLIP_DSACIQ, 3, qp.QP_CLIP_MINMAX | qp.QP_CLIP_INTERSECT):
+        with pytest.raises(qp.QuantPipeError):
+            ctx.qp_clip_qparams_device(d_stats, 4, bad)
+    for bad in (3, qp.QP_CLIP_DSACIQ | qp.QP_CLIP_INTERSECT, qp.QP_CLIP_MINMAX | qp.QP_CLIP_INTERSECT):
+        with pytest.raises(qp.QuantPipeError):
+            ctx.qp_sender_device(x, 4, bad)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_sender_device(x, 16, qp.QP_CLIP_DSACIQ)
+
+
 def test_sender_and_receiver_host_buffers(ctx):
     x = si.vit_activation((2, 197, 384), 78).reshape(-1)
     n = x.size

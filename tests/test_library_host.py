@@ -97,6 +97,26 @@ def test_aciq_alpha_matches_oracle(lib):
     assert qp.qp_aciq_alpha(st, 4, 3)[0] == qp.QP_ERR_INVALID_ARG
 
 
+def test_clip_range_matches_oracle(lib):
+    x = si.vit_activation((2, 197, 96), 21, outlier_frac=0.02)
+    st_o = oracle.stats(x)
+    st = qp.Stats(st_o.n, st_o.nonfinite, st_o.mean, st_o.mean_abs, st_o.mad, st_o.var, st_o.min, st_o.max, 0, 0, 0)
+    for bits in ALL_BITS:
+        for method, o_method, cut in ((qp.QP_CLIP_ACIQ, oracle.CLIP_ACIQ, False), (qp.QP_CLIP_MINMAX, oracle.CLIP_MINMAX, False),
+                                      (qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT, oracle.CLIP_ACIQ, True)):
+            for dist, bmode in ((0, 0), (0, 1), (1, 0)):
+                rc, lo, hi, q = qp.qp_clip_range(st, bits, method, dist, bmode)
+                rc_o, lo_o, hi_o, q_o = oracle.clip_range(st_o, bits, o_method, cut, dist, bmode)
+                assert rc == rc_o == 0
+                assert lo == pytest.approx(lo_o, rel=1e-12, abs=1e-300) and hi == pytest.approx(hi_o, rel=1e-12, abs=1e-300)
+                assert _same_qp(q, q_o)
+    assert qp.qp_clip_range(st, 4, qp.QP_CLIP_DSACIQ)[0] == qp.QP_ERR_INVALID_ARG      # needs the tensor, not a closed form
+    assert qp.qp_clip_range(st, 4, qp.QP_CLIP_MINMAX | qp.QP_CLIP_INTERSECT)[0] == qp.QP_ERR_INVALID_ARG
+    assert qp.qp_clip_range(st, 9)[0] == qp.QP_ERR_UNSUPPORTED_BITS
+    const = qp.Stats(10, 0, 2.0, 2.0, 0.0, 0.0, 2.0, 2.0, 0, 0, 0)
+    assert qp.qp_clip_range(const, 4, qp.QP_CLIP_MINMAX)[0] == qp.QP_WARN_DEGENERATE
+
+
 def test_select_bits_matches_oracle(lib):
     n = 128 * 197 * 1280
     trace = si.bandwidth_trace(3, si.C4_TRACE_STEPS)
