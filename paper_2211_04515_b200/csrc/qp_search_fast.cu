@@ -390,30 +390,51 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     }
 }
 
-// totals over the blocks' partials.  grid (ceil((MAXB+1)/256), SLICES): slice s adds blocks
-// s, s + SLICES, ... and merges with integer atomics (order-independent); block (0,0) also
-// adds up the outer sums in block order.
-constexpr int IV_SLICES = 32;
-__global__ void __launch_bounds__(256) iv_reduce_kernel(const unsigned long long* __restrict__ part, int blocks,
-                                                        const unsigned* __restrict__ g_m,
-                                                        qp_iv_total* __restrict__ tot, const double* __restrict__ outer,
-                                                        double* __restrict__ outer_tot)
+// Totals over the blocks' partials.  A block takes 32 consecutive intervals: lane = interval
+// (one 256-byte row segment per warp load), warp w adds the partials of blocks w, w + 16, ...
+// (eight loads in flight), the 16 warp sums are merged through shared memory and written
+// once.  Integer sums, so the order does not matter.  Block 0 also adds up the outer sums
+// in block order.
+constexpr int IV_RED_THREADS = 512;
+constexpr int IV_RED_WARPS = IV_RED_THREADS / 32;
+__global__ void __launch_bounds__(IV_RED_THREADS) iv_reduce_kernel(const unsigned long long* __restrict__ part, int blocks,
+                                                                   const unsigned* __restrict__ g_m,
+                                                                   qp_iv_total* __restrict__ tot,
+                                                                   const double* __restrict__ outer,
+                                                                   double* __restrict__ outer_tot)
 {
+    __shared__ unsigned long long s_n[IV_RED_WARPS][32], s_s[IV_RED_WARPS][32];
     const unsigned m = *g_m;
-    const unsigned i = blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const unsigned i = blockIdx.x * 32 + lane;
+    unsigned long long n = 0, s1 = 0;
     if (i <= m) {
-        unsigned long long n = 0, s1 = 0;
-        for (int b = blockIdx.y; b < blocks; b += IV_SLICES) {
-            const unsigned long long p = part[(size_t)b * (MAXB + 1) + i];
-            n += p >> 40;
-            s1 += p & S1_MASK;
-        }
-        if (n) {
-            atomicAdd(&tot[i].n, n);
-            atomicAdd(&tot[i].s1, s1);
+        for (int b0 = warp; b0 < blocks; b0 += IV_RED_WARPS * 8) {
+            unsigned long long p[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int b = b0 + u * IV_RED_WARPS;
+                p[u] = b < blocks ? part[(size_t)b * (MAXB + 1) + i] : 0ull;
+            }
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                n += p[u] >> 40;
+                s1 += p[u] & S1_MASK;
+            }
         }
     }
-    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x < 7 * 32) {
+    s_n[warp][lane] = n;
+    s_s[warp][lane] = s1;
+    __syncthreads();
+    if (warp == 0 && i <= m) {
+        for (int w = 1; w < IV_RED_WARPS; ++w) {
+            n += s_n[w][lane];
+            s1 += s_s[w][lane];
+        }
+        tot[i].n = n;
+        tot[i].s1 = s1;
+    }
+    if (blockIdx.x == 0 && threadIdx.x < 7 * 32) {
         // warp w adds up quantity w: lane l takes blocks l, l+32, ... then a fixed shuffle tree
         const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
         double t = 0.0;
@@ -515,8 +536,6 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)(G + 1) * 4 + 16;
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
-    if (cudaMemsetAsync(ctx->d_iv_tot, 0, sizeof(qp_iv_total) * (MAXB + 1), s) != cudaSuccess)
-        return qp_check_launch(ctx, "qp_dsaciq_search (interval totals reset)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
                                                 ctx->d_setup, ctx->d_iv_bnd);
     unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]
@@ -525,9 +544,9 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     const int blocks = ctx->iv_blocks;
     iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
                                                              g_m, ctx->d_iv_part, ctx->d_iv_outer);
-    iv_reduce_kernel<<<dim3((MAXB + 1 + 255) / 256, IV_SLICES), 256, 0, s>>>(ctx->d_iv_part, blocks, g_m,
-                                                                            ctx->d_iv_tot, ctx->d_iv_outer,
-                                                                            ctx->d_iv_outer + (size_t)blocks * 8);
+    iv_reduce_kernel<<<(MAXB + 1 + 31) / 32, IV_RED_THREADS, 0, s>>>(ctx->d_iv_part, blocks, g_m, ctx->d_iv_tot,
+                                                                    ctx->d_iv_outer,
+                                                                    ctx->d_iv_outer + (size_t)blocks * 8);
     iv_curve_kernel<<<ncand, IV_CURVE_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, g_m,
                                                        ctx->d_iv_outer + (size_t)blocks * 8, ctx->d_cand, ctx->d_valid,
                                                        bits, steps, nb, ctx->d_setup, ctx->d_curve, ctx->d_ticket + 2,
