@@ -335,14 +335,16 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  * How the chain runs (qp_set_sender_path; the paper has no counterpart):
  *   QP_SENDER_CHAIN  the kernels of the separate calls, one after the other; the outputs are
  *                    bit for bit those of the separate calls
- *   QP_SENDER_FUSED  one cooperative launch for 0 < n <= 2^20 (and steps <= 127, hist_bins <=
- *                    4096 when searching): every SM keeps its slice of x in shared memory, the
- *                    tensor-wide steps are separated by grid barriers.  Same arithmetic per
- *                    element, but the sums are merged in another order: statistics agree with
- *                    the chain to ~1e-15 relative, the error curve to ~1e-6, so the clip range
- *                    can differ in its last fp32 bit or, where two steps of the search tie, by
- *                    one step.  Other arguments fall back to the chain.
- *   QP_SENDER_AUTO   fused where it applies (default)
+ *   QP_SENDER_FUSED  one cooperative launch: every SM keeps its slice of x in shared memory, the
+ *                    tensor-wide steps are separated by grid barriers.  Applies to 0 < n <= 2^20
+ *                    with the search (and steps <= 127, hist_bins <= 4096) and to n <= 6.5e6
+ *                    with a closed-form clip (less where the GPU's shared memory holds less);
+ *                    other arguments fall back to the chain.  Same arithmetic per element, but
+ *                    the sums are merged in another order: statistics agree with the chain to
+ *                    ~1e-15 relative, the error curve to ~1e-6, so the clip range can differ in
+ *                    its last fp32 bit or, where two steps of the search tie, by one step.
+ *   QP_SENDER_AUTO   fused where it is the faster of the two on a B200: n <= 2^20 with the
+ *                    search, n <= 2^21 otherwise (default)
  * A grid barrier that does not complete within about a quarter of a second sets
  * QP_DEV_STREAM_TIMEOUT in the status word and the launch ends without output. */
 enum { QP_SENDER_AUTO = 0, QP_SENDER_CHAIN = 1, QP_SENDER_FUSED = 2 };

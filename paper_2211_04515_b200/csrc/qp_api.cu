@@ -645,7 +645,8 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
 {
     int32_t rc;
     const int use_ds = method == QP_CLIP_DSACIQ;
-    if (ctx->sender_path != QP_SENDER_CHAIN && qp_sender_fused_applies(n, use_ds, steps, hist_bins)) {
+    if (ctx->sender_path != QP_SENDER_CHAIN &&
+        qp_sender_fused_applies(n, use_ds, steps, hist_bins, ctx->sender_path == QP_SENDER_FUSED)) {
         // the checks of the separate calls
         rc = check_x(ctx, d_x, dtype, n);
         if (rc) return rc;

@@ -75,6 +75,7 @@ struct qp_ctx {
     int search_path;                     // 0 auto, 1 candidate scoring, 2 interval moments
     int sender_path;                     // 0 auto, 1 kernel chain, 2 single cooperative launch where it applies
     int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
+    size_t fused_dyn_max;                // largest slice (bytes of dynamic shared memory) per block
     void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
     qp_qparams_t* d_tmp_qp;
@@ -345,7 +346,7 @@ int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
 int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                                   int bits, int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                                   qp_qparams_t* d_qp_out, cudaStream_t s);
-bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins);
+bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins, bool forced);
 int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,
                                int steps, int hist_bins, double F, void* d_packed, qp_qparams_t* d_qp_out,
                                qp_stats_t* d_stats_out, cudaStream_t s);

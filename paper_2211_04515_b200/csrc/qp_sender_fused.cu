@@ -30,7 +30,9 @@ constexpr int FS_THREADS = 512;
 constexpr int FS_WARPS = FS_THREADS / 32;
 constexpr int FS_MAX_STEPS = 127;                 // candidates fit the per-block tables
 constexpr int FS_MAX_BINS = 4096;
-constexpr uint64_t FS_MAX_N = 1ull << 20;         // above this the per-candidate scoring stops paying
+constexpr uint64_t FS_MAX_N_SEARCH = 1ull << 20;  // above this the per-candidate scoring stops paying
+constexpr uint64_t FS_AUTO_N = 1ull << 21;
+constexpr uint64_t FS_MAX_N = 6500000;            // slices of 148 SMs x ~190 KB of shared memory (checked per device)
 constexpr int FS_PART = 8;                        // doubles per block partial
 constexpr unsigned FS_SPIN_LIMIT = 1u << 22;      // x 64 ns sleeps: a quarter of a second at least
 constexpr int K = QP_EVAL_K;
@@ -151,28 +153,60 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
     {
         const T* x = static_cast<const T*>(a.x);
         double v5[5] = {0.0, 0.0, inf, -inf, 0.0};            // sum, sum |x|, min, max, non-finite
-        for (int i0 = tid; i0 < cnt; i0 += 8 * FS_THREADS) {   // eight loads in flight per thread
-            float e[8];
+        auto one = [&](float v) {                             // element by element: skips and counts NaN/Inf
+            if (qp_is_finite(v)) {
+                v5[0] += (double)v;
+                v5[1] += (double)fabsf(v);
+                v5[2] = fmin(v5[2], (double)v);
+                v5[3] = fmax(v5[3], (double)v);
+            } else {
+                v5[4] += 1.0;
+            }
+        };
+        constexpr int EPV = qp_span<T>::EPV;
+        const T* xb = x + e0;
+        const float finf = __int_as_float(0x7F800000);
+        // 16-byte loads where the slice is aligned (its start is a multiple of 32 elements from x),
+        // four in flight per thread; fp32 partial sums over one vector, folded into fp64
+        const int nvec = (((uintptr_t)xb & 15u) == 0) ? cnt / EPV : 0;
+        for (int v0 = tid; v0 < nvec; v0 += 4 * FS_THREADS) {
+            float e[4][EPV];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + u * FS_THREADS;
-                e[u] = i < cnt ? qp_load_one(x + e0 + i) : 0.f;
+            for (int u = 0; u < 4; ++u) {
+                const int v = v0 + u * FS_THREADS;
+                if (v < nvec) qp_load_vec(xb + (size_t)v * EPV, e[u]);
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
-                const int i = i0 + u * FS_THREADS;
-                if (i >= cnt) break;
-                const float v = e[u];
-                xs[i + (i >> 5)] = v;
-                if (qp_is_finite(v)) {
-                    v5[0] += (double)v;
-                    v5[1] += (double)fabsf(v);
-                    v5[2] = fmin(v5[2], (double)v);
-                    v5[3] = fmax(v5[3], (double)v);
+            for (int u = 0; u < 4; ++u) {
+                const int v = v0 + u * FS_THREADS;
+                if (v >= nvec) break;
+                const int i0 = v * EPV;                       // EPV consecutive elements stay inside one 32-element row
+                float* dst = xs + i0 + (i0 >> 5);
+                float ps = 0.f, psa = 0.f, pmn = finf, pmx = -finf;
+#pragma unroll
+                for (int i = 0; i < EPV; ++i) {
+                    const float val = e[u][i];
+                    dst[i] = val;
+                    ps += val;
+                    psa += fabsf(val);
+                    pmn = fminf(pmn, val);
+                    pmx = fmaxf(pmx, val);
+                }
+                if (psa < finf) {                             // every element finite (and no fp32 overflow)
+                    v5[0] += (double)ps;
+                    v5[1] += (double)psa;
+                    v5[2] = fmin(v5[2], (double)pmn);
+                    v5[3] = fmax(v5[3], (double)pmx);
                 } else {
-                    v5[4] += 1.0;
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) one(e[u][i]);
                 }
             }
+        }
+        for (int i = nvec * EPV + tid; i < cnt; i += FS_THREADS) {   // unaligned slice, ragged end
+            const float v = qp_load_one(xb + i);
+            xs[i + (i >> 5)] = v;
+            one(v);
         }
         fs_reduce<0, 0, 1, 2, 0>(v5, s_red);
         if (tid == 0) {
@@ -214,18 +248,26 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
         const float h_mn = (float)mn_all;
         const float inv_w = want_hist ? (float)((double)a.nb / (mx_all - mn_all)) : 0.f;
         double v2[2] = {0.0, 0.0};
-        for (int i = tid; i < cnt; i += FS_THREADS) {
-            const float v = xs[i + (i >> 5)];
-            if (!qp_is_finite(v)) continue;
-            const float d = __fsub_rn(__fsub_rn(v, m_hi), m_lo);
-            v2[0] += (double)fabsf(d);
-            v2[1] += (double)d * (double)d;
-            if (want_hist) {
-                // bin = floor((x - min) * inv_w), the last bin closed; fp32, each op rounded once
-                int b = __float2int_rz(__fmul_rn(__fsub_rn(v, h_mn), inv_w));
-                b = min(max(b, 0), a.nb - 1);
-                atomicAdd(&s_hist[b], 1u);
+        for (int i0 = tid; i0 < cnt; i0 += 8 * FS_THREADS) {  // fp32 sums over 8 elements, then fp64
+            float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+            for (int u = 0; u < 8; ++u) {
+                const int i = i0 + u * FS_THREADS;
+                if (i >= cnt) break;
+                const float v = xs[i + (i >> 5)];
+                if (!qp_is_finite(v)) continue;
+                const float d = __fsub_rn(__fsub_rn(v, m_hi), m_lo);
+                d1 += fabsf(d);
+                d2 = fmaf(d, d, d2);
+                if (want_hist) {
+                    // bin = floor((x - min) * inv_w), the last bin closed; fp32, each op rounded once
+                    int b = __float2int_rz(__fmul_rn(__fsub_rn(v, h_mn), inv_w));
+                    b = min(max(b, 0), a.nb - 1);
+                    atomicAdd(&s_hist[b], 1u);
+                }
             }
+            v2[0] += (double)d1;
+            v2[1] += (double)d2;
         }
         fs_reduce<0, 0>(v2, s_red);                            // (its barriers also order the shared atomics)
         if (tid == 0) {
@@ -456,9 +498,13 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
 
 }  // namespace
 
-bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins)
+bool qp_sender_fused_applies(uint64_t n, int use_ds, int steps, int hist_bins, bool forced)
 {
-    if (n == 0 || n > FS_MAX_N) return false;
+    // measured against the kernel chain: the single launch wins up to ~2^21 elements with a
+    // closed-form clip and up to 2^20 with the search; when forced it runs up to what the
+    // shared memory of all SMs holds
+    const uint64_t max_n = use_ds ? FS_MAX_N_SEARCH : (forced ? FS_MAX_N : FS_AUTO_N);
+    if (n == 0 || n > max_n) return false;
     if (use_ds && (steps > FS_MAX_STEPS || hist_bins > FS_MAX_BINS)) return false;
     return true;
 }
@@ -477,23 +523,32 @@ int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t
     const size_t dyn = (size_t)gpb * 33 * sizeof(float);
     void* kernel = dtype == QP_F32 ? (void*)sender_fused_kernel<float> : (void*)sender_fused_kernel<unsigned short>;
 
-    if (!ctx->fused_checked) {                   // once: can one block per SM be resident at the largest slice?
+    if (!ctx->fused_checked) {                   // once: how large a slice can one block per SM hold?
         ctx->fused_checked = 1;
         ctx->fused_ok = 0;
-        const size_t dyn_max = (size_t)((((FS_MAX_N + 31) / 32 + 3) + G - 1) / G + 1) * 33 * sizeof(float);
-        int coop = 0, per_sm = 0;
+        ctx->fused_dyn_max = 0;
+        int coop = 0, optin = 0;
         bool ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
+                  cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) == cudaSuccess &&
                   (size_t)G * (FS_MAX_STEPS + 1) <= (size_t)QP_MAX_BLOCKS * QP_EVAL_K && G <= QP_MAX_BLOCKS;
+        size_t dyn_max = 0;
         for (int t = 0; ok && t < 2; ++t) {
             void* kf = t ? (void*)sender_fused_kernel<unsigned short> : (void*)sender_fused_kernel<float>;
-            ok = cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn_max) == cudaSuccess &&
-                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kf, FS_THREADS, dyn_max) == cudaSuccess &&
+            cudaFuncAttributes fa;
+            int per_sm = 0;
+            ok = cudaFuncGetAttributes(&fa, kf) == cudaSuccess && (size_t)optin > fa.sharedSizeBytes + 2048;
+            if (!ok) break;
+            const size_t room = (size_t)optin - fa.sharedSizeBytes - 1024;     // 1 KB the system keeps per block
+            dyn_max = t ? (room < dyn_max ? room : dyn_max) : room;
+            ok = cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)room) == cudaSuccess &&
+                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kf, FS_THREADS, room) == cudaSuccess &&
                  per_sm >= 1;
         }
         if (!ok) cudaGetLastError();
         ctx->fused_ok = ok ? 1 : 0;
+        ctx->fused_dyn_max = ok ? dyn_max : 0;
     }
-    if (!ctx->fused_ok) return QP_WARN_INFEASIBLE;
+    if (!ctx->fused_ok || dyn > ctx->fused_dyn_max) return QP_WARN_INFEASIBLE;   // the caller runs the chain
 
     // The arrival counter and the histogram start at zero: the context allocates them zeroed and
     // every completed launch leaves them so (a timed-out one does not: qp_get_status clears them).

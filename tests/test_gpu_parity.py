@@ -513,27 +513,34 @@ def test_fused_sender_special_values_modes_and_bf16():
     check_fused_sender(oracle.widen_bf16(h[1:-2]), d[1:-2], 8, False)
 
 
-def test_fused_sender_falls_back_outside_its_range():
-    """Beyond 2^20 elements, 127 steps or 4096 bins the call runs the kernel chain, whatever the path."""
+def test_fused_sender_range_and_fallback():
+    """Forced, the single launch takes a closed-form clip up to what shared memory holds (millions of
+    elements) and the search up to 2^20; beyond that, or beyond 127 steps or 4096 bins, the call runs the
+    kernel chain.  AUTO switches to the chain earlier (2^21), where the chain is the faster one."""
     c = qp.Context(0)
-    c.qp_set_sender_path(qp.QP_SENDER_FUSED)
-    x = si.vit_activation((1, (1 << 20) + 1, 1), 33).reshape(-1)
+    x = si.vit_activation((1, 3000000, 1), 33).reshape(-1)
     d = dev(x)
-    for kw in (dict(), ):
+    c.qp_set_sender_path(qp.QP_SENDER_FUSED)
+    status, _ = check_fused_sender(x, d, 8, False)                     # 3 M elements, one launch
+    assert status == 0
+    big = torch.zeros(7000000, device="cuda")
+    for t, use_ds, want_one in ((big, False, False), (d[:(1 << 20) + 1], True, False), (d[:1 << 20], True, True),
+                                (d[:5000], True, True)):
         before = c.qp_launch_count()
-        packed, d_qp = c.qp_sender_device(d, 8, False)
-        assert c.qp_launch_count() - before > 1
-    small = d[:5000]
+        c.qp_sender_device(t, 2, use_ds)
+        assert (c.qp_launch_count() - before == 1) == want_one
     for kw in (dict(steps=128), dict(hist_bins=4097)):
         before = c.qp_launch_count()
-        c.qp_sender_device(small, 2, True, **kw)
+        c.qp_sender_device(d[:5000], 2, True, **kw)
         assert c.qp_launch_count() - before > 1
-    before = c.qp_launch_count()
-    c.qp_sender_device(small, 2, True)
-    assert c.qp_launch_count() - before == 1
+    c.qp_set_sender_path(qp.QP_SENDER_AUTO)
+    for n, want_one in ((1 << 21, True), ((1 << 21) + 1, False)):
+        before = c.qp_launch_count()
+        c.qp_sender_device(d[:n], 8, False)
+        assert (c.qp_launch_count() - before == 1) == want_one
     with pytest.raises(qp.QuantPipeError):
         c.qp_set_sender_path(3)
-    assert c.qp_get_status() == 0
+    assert c.qp_get_status() & ~qp.QP_DEV_DEGENERATE == 0              # (the all-zero tensor has no spread)
     c.close()
 
 
