@@ -93,6 +93,15 @@ def lib():
         L.orc_clip_range.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, dp, dp,
                                      C.POINTER(QParams)]
         L.orc_clip_range.restype = C.c_int
+        L.orc_stats_channels.argtypes = [fp, C.c_uint64, C.c_uint64, C.POINTER(Stats)]
+        L.orc_stats_channels.restype = C.c_int
+        L.orc_clip_channels.argtypes = [C.POINTER(Stats), C.c_uint64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                        C.POINTER(QParams)]
+        L.orc_clip_channels.restype = C.c_int
+        L.orc_quantize_channels.argtypes = [fp, C.c_uint64, C.c_uint64, C.POINTER(QParams), u32p]
+        L.orc_quantize_channels.restype = None
+        L.orc_dequantize_channels.argtypes = [u32p, C.c_uint64, C.c_uint64, C.POINTER(QParams), fp]
+        L.orc_dequantize_channels.restype = None
         L.orc_hist_peak.argtypes = [fp, C.c_uint64, C.c_double, C.c_double, C.c_int, u64p]
         L.orc_hist_peak.restype = C.c_double
         L.orc_ds_search.argtypes = [fp, C.c_uint64, C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int,
@@ -198,6 +207,39 @@ def unpack(packed, n: int, bits: int) -> np.ndarray:
     codes = np.empty(n, dtype=np.uint32)
     lib().orc_unpack(_ptr(p, C.c_uint8), n, bits, _ptr(codes, C.c_uint32))
     return codes
+
+
+def stats_channels(x, channels: int):
+    """Per-channel statistics of a [rows, channels] tensor: a ctypes array of `channels` Stats."""
+    a = _f32(x)
+    rows = a.size // channels
+    assert rows * channels == a.size
+    out = (Stats * channels)()
+    rc = lib().orc_stats_channels(_ptr(a, C.c_float), rows, channels, out)
+    assert rc == 0
+    return out
+
+
+def clip_channels(st, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0):
+    """(rc, ctypes array of per-channel QParams) from per-channel statistics."""
+    channels = len(st)
+    qp = (QParams * channels)()
+    rc = lib().orc_clip_channels(st, channels, bits, method, 1 if intersect else 0, dist, bmode, qp)
+    return rc, qp
+
+
+def quantize_channels(x, channels: int, qp) -> np.ndarray:
+    a = _f32(x)
+    codes = np.empty(a.size, dtype=np.uint32)
+    lib().orc_quantize_channels(_ptr(a, C.c_float), a.size // channels, channels, qp, _ptr(codes, C.c_uint32))
+    return codes
+
+
+def dequantize_channels(codes, channels: int, qp) -> np.ndarray:
+    c = np.ascontiguousarray(codes, dtype=np.uint32)
+    y = np.empty(c.size, dtype=np.float32)
+    lib().orc_dequantize_channels(_ptr(c, C.c_uint32), c.size // channels, channels, qp, _ptr(y, C.c_float))
+    return y
 
 
 def quantize_pack(x, qp: QParams) -> np.ndarray:

@@ -239,6 +239,53 @@ double orc_quant_mse(const float* x, uint64_t n, const orc_qparams_t* qp)
     return nf ? ksum_get(&s) / (double)nf : 0.0;
 }
 
+/* ------------------------------------------------- per-channel quantization */
+
+/* Channel-wise variant of the per-tensor method (Sec. 3 applies one clip range to the whole
+ * tensor; channel-wise ranges are the alternative the paper's cited PTQ work uses for
+ * activations with outlier channels).  The tensor is [rows, channels], row-major, so element
+ * i belongs to channel i mod channels; every channel gets the statistics, the clip range and
+ * the quantizer that the per-tensor functions give for its column alone, and all channels
+ * share the bit-width and the packed layout. */
+
+/* Statistics of each column: out[c] = orc_stats of x[c], x[c + channels], ... */
+int orc_stats_channels(const float* x, uint64_t rows, uint64_t channels, orc_stats_t* out)
+{
+    if (channels < 1) return ORC_ERR_ARG;
+    float* col = (float*)malloc((size_t)(rows ? rows : 1) * sizeof(float));
+    if (!col) return ORC_ERR_ARG;
+    for (uint64_t c = 0; c < channels; ++c) {
+        for (uint64_t r = 0; r < rows; ++r) col[r] = x[r * channels + c];
+        orc_stats(col, rows, &out[c]);
+    }
+    free(col);
+    return ORC_OK;
+}
+
+/* Quantizer of each channel from its statistics (orc_clip_range per channel).  Returns
+ * ORC_WARN_DEGENERATE if any channel has an empty range (that channel's codes are all 0). */
+int orc_clip_channels(const orc_stats_t* st, uint64_t channels, int bits, int method, int intersect, int dist,
+                      int bmode, orc_qparams_t* qp)
+{
+    int worst = ORC_OK;
+    for (uint64_t c = 0; c < channels; ++c) {
+        int rc = orc_clip_range(&st[c], bits, method, intersect, dist, bmode, NULL, NULL, &qp[c]);
+        if (rc < 0) return rc;
+        if (rc == ORC_WARN_DEGENERATE) worst = rc;
+    }
+    return worst;
+}
+
+void orc_quantize_channels(const float* x, uint64_t rows, uint64_t channels, const orc_qparams_t* qp, uint32_t* codes)
+{
+    for (uint64_t i = 0; i < rows * channels; ++i) codes[i] = quantize_one(x[i], &qp[i % channels]);
+}
+
+void orc_dequantize_channels(const uint32_t* codes, uint64_t rows, uint64_t channels, const orc_qparams_t* qp, float* y)
+{
+    for (uint64_t i = 0; i < rows * channels; ++i) y[i] = dequantize_one(codes[i], &qp[i % channels]);
+}
+
 /* ----------------------------------------------------------------- packing */
 
 /* Packed length: ceil(n * bits / 8) bytes rounded up to a multiple of 16. */

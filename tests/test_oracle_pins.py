@@ -535,6 +535,89 @@ def test_clip_range_aciq_equals_aciq_alpha_and_intersection_properties():
     assert oracle.clip_range(st, 4, oracle.CLIP_MINMAX, intersect=True)[0] == oracle.ERR_ARG
 
 
+# ------------------------------------------------------- per-channel quantization
+
+def test_channels_hand_example_two_scales():
+    """Two channels whose scales differ by ten: channel 0 holds 0, 1, 2, 3 and channel 1 holds 0, 10, 20,
+    30.  With the min/max range at 2 bits each channel has its own four levels, so every value is a level
+    and is reconstructed exactly; one range for the whole tensor, [0, 30] with levels 0, 10, 20, 30, sends
+    channel 0's 1, 2, 3 to 0 (by hand)."""
+    x = np.array([[0, 0], [1, 10], [2, 20], [3, 30]], dtype=np.float32)
+    st = oracle.stats_channels(x, 2)
+    assert [(s.min, s.max, s.n) for s in st] == [(0.0, 3.0, 4), (0.0, 30.0, 4)]
+    rc, qp = oracle.clip_channels(st, 2, oracle.CLIP_MINMAX)
+    assert rc == 0 and (qp[0].scale, qp[1].scale) == (1.0, 10.0)
+    codes = oracle.quantize_channels(x, 2, qp)
+    assert codes.reshape(4, 2).tolist() == [[0, 0], [1, 1], [2, 2], [3, 3]]
+    assert np.array_equal(oracle.dequantize_channels(codes, 2, qp).reshape(4, 2), x)
+    whole = oracle.clip_range(oracle.stats(x), 2, oracle.CLIP_MINMAX)[3]
+    assert oracle.dequantize(oracle.quantize(x, whole), whole).reshape(4, 2)[:, 0].tolist() == [0.0, 0.0, 0.0, 0.0]
+
+
+def test_channels_statistics_against_numpy_columns():
+    x = si.vit_activation((3, 50, 24), 11, outlier_frac=0.1).reshape(-1, 24)
+    x[5, 3] = np.nan
+    x[7, 3] = np.inf
+    st = oracle.stats_channels(x, 24)
+    x64 = x.astype(np.float64)
+    for c in range(24):
+        col = x64[:, c]
+        col = col[np.isfinite(col)]
+        assert st[c].n == 150 and st[c].nonfinite == (2 if c == 3 else 0)
+        assert st[c].mean == pytest.approx(col.mean(), rel=1e-12, abs=1e-15)
+        assert st[c].mean_abs == pytest.approx(np.abs(col).mean(), rel=1e-12)
+        assert st[c].mad == pytest.approx(np.abs(col - col.mean()).mean(), rel=1e-12)
+        assert st[c].var == pytest.approx(col.var(), rel=1e-12)
+        assert (st[c].min, st[c].max) == (col.min(), col.max())
+
+
+def test_channels_one_channel_is_the_per_tensor_path_and_symmetries():
+    y = si.flat_iid(6000, 12, "laplace")
+    # a single channel: exactly the per-tensor functions
+    st1 = oracle.stats_channels(y, 1)
+    assert bytes(st1[0]) == bytes(oracle.stats(y))
+    for bits in (2, 4, 8):
+        rc, qp1 = oracle.clip_channels(st1, bits)
+        q = oracle.aciq_alpha(oracle.stats(y), bits)[2]
+        assert bytes(qp1[0]) == bytes(q)
+        assert np.array_equal(oracle.quantize_channels(y, 1, qp1), oracle.quantize(y, q))
+        assert np.array_equal(oracle.dequantize_channels(oracle.quantize(y, q), 1, qp1), oracle.dequantize(oracle.quantize(y, q), q))
+    # element i belongs to channel i mod C (not i div rows): transposing the roles must change the answer
+    x = si.vit_activation((1, 40, 6), 13, outlier_frac=0.2).reshape(40, 6)
+    st = oracle.stats_channels(x, 6)
+    assert all(st[c].mean == pytest.approx(float(x[:, c].astype(np.float64).mean()), rel=1e-12) for c in range(6))
+    rc, qp = oracle.clip_channels(st, 4)
+    codes = oracle.quantize_channels(x, 6, qp).reshape(40, 6)
+    # channels do not interact: scaling one channel by a power of two scales its range and leaves all codes alone
+    x2 = x.copy()
+    x2[:, 2] *= np.float32(8.0)
+    st2 = oracle.stats_channels(x2, 6)
+    rc, qp2 = oracle.clip_channels(st2, 4)
+    assert (qp2[2].lo, qp2[2].hi, qp2[2].scale) == (8 * qp[2].lo, 8 * qp[2].hi, 8 * qp[2].scale)
+    assert all(bytes(qp2[c]) == bytes(qp[c]) for c in range(6) if c != 2)
+    assert np.array_equal(oracle.quantize_channels(x2, 6, qp2).reshape(40, 6), codes)
+    # permuting the channels permutes statistics, quantizers and codes
+    perm = np.array([3, 0, 5, 1, 4, 2])
+    xp = np.ascontiguousarray(x[:, perm])
+    stp = oracle.stats_channels(xp, 6)
+    rc, qpp = oracle.clip_channels(stp, 4)
+    assert all(bytes(qpp[j]) == bytes(qp[perm[j]]) for j in range(6))
+    assert np.array_equal(oracle.quantize_channels(xp, 6, qpp).reshape(40, 6), codes[:, perm])
+    # with outlier channels, channel-wise ranges lower the error of the whole tensor
+    z = si.vit_activation((2, 197, 64), 14, outlier_frac=0.05).reshape(-1, 64)
+    stz = oracle.stats_channels(z, 64)
+    rc, qz = oracle.clip_channels(stz, 4)
+    err_c = np.mean((oracle.dequantize_channels(oracle.quantize_channels(z, 64, qz), 64, qz).astype(np.float64) - z.reshape(-1)) ** 2)
+    q_t = oracle.aciq_alpha(oracle.stats(z), 4)[2]
+    assert err_c < 0.5 * oracle.quant_mse(z, q_t)
+    # a constant channel is degenerate: code 0, reconstructed exactly, and the call says so
+    z[:, 7] = np.float32(1.5)
+    rc, qz = oracle.clip_channels(oracle.stats_channels(z, 64), 4)
+    assert rc == oracle.WARN_DEGENERATE and qz[7].flags == 1
+    back = oracle.dequantize_channels(oracle.quantize_channels(z, 64, qz), 64, qz).reshape(-1, 64)
+    assert np.all(back[:, 7] == np.float32(1.5))
+
+
 # ------------------------------------------------------------------- inputs
 
 def test_generator_is_counter_based_and_shaped():
