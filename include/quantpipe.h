@@ -312,6 +312,32 @@ int32_t qp_controller_observe(qp_controller_t* h_c, double bytes_sent, double se
 /* Payload of one microbatch at `bits` (32 = raw fp32): ceil(n_elems*bits/8) + overhead_bytes. */
 uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
 
+/* ---- channel-wise variant (the paper, Sec. 3, clips per tensor; this is the per-channel form
+ * that its cited PTQ work uses for activations with outlier channels) ----------------------
+ * The tensor is [rows, channels], row-major: element i belongs to channel i mod channels.
+ * Every channel gets the statistics, clip range and quantizer that the per-tensor calls give
+ * for its column alone; bit-width and packed layout (qp_packed_bytes(rows * channels, bits))
+ * are shared, so the receiver needs the `channels` quantizers (24 bytes each) with the stream.
+ *   qp_stats_channels                fills d_out[0..channels) (hist fields 0).  Keeps its block
+ *                                    partials in the context, allocated on the first call and
+ *                                    when a larger tensor comes (cudaMalloc: not during capture).
+ *   qp_clip_qparams_channels_device  d_qp_out[c] from d_stats[c]; method, dist, bmode as
+ *                                    qp_clip_qparams_device.
+ *   qp_quantize_pack_channels        code of element i with d_qp[i mod channels].
+ *   qp_unpack_dequantize_channels    the inverse, fp32 or bf16 out.
+ * d_stats, d_qp: device arrays of `channels` entries.  1 <= channels <= QP_MAX_CHANNELS.
+ * Errors: as the per-tensor calls, plus QP_ERR_INVALID_ARG for channels out of range. */
+#define QP_MAX_CHANNELS 4096
+int32_t qp_stats_channels(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels,
+                          qp_stats_t* d_out, void* stream);
+int32_t qp_clip_qparams_channels_device(qp_ctx* ctx, const qp_stats_t* d_stats, uint32_t channels, int bits,
+                                        int method, int dist, int bmode, qp_qparams_t* d_qp_out, void* stream);
+int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels,
+                                  int bits, const qp_qparams_t* d_qp, void* d_packed, uint64_t packed_capacity,
+                                  void* stream);
+int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_packed, uint64_t rows, uint32_t channels, int bits,
+                                      const qp_qparams_t* d_qp, void* d_y, int out_dtype, void* stream);
+
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------
  * qp_sender_host: copies the n elements at h_x to d_x_work, runs statistics, the clip

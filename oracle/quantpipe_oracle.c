@@ -241,6 +241,9 @@ double orc_quant_mse(const float* x, uint64_t n, const orc_qparams_t* qp)
 
 /* ------------------------------------------------- per-channel quantization */
 
+int orc_clip_range(const orc_stats_t* st, int bits, int method, int intersect, int dist, int bmode,
+                   double* lo_out, double* hi_out, orc_qparams_t* qp);   /* defined with the ACIQ clip below */
+
 /* Channel-wise variant of the per-tensor method (Sec. 3 applies one clip range to the whole
  * tensor; channel-wise ranges are the alternative the paper's cited PTQ work uses for
  * activations with outlier channels).  The tensor is [rows, channels], row-major, so element

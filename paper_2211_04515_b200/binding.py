@@ -35,7 +35,8 @@ EXPORTS = (
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
-    "qp_clip_range", "qp_clip_qparams_device",
+    "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_clip_qparams_channels_device",
+    "qp_quantize_pack_channels", "qp_unpack_dequantize_channels",
 )
 
 
@@ -104,6 +105,10 @@ def load() -> C.CDLL:
     L.qp_clip_range.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(dbl), C.POINTER(dbl),
                                 C.POINTER(QParams)]
     L.qp_clip_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.qp_stats_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, vp, vp]
+    L.qp_clip_qparams_channels_device.argtypes = [vp, vp, C.c_uint32, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.qp_quantize_pack_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, vp, vp, u64, vp]
+    L.qp_unpack_dequantize_channels.argtypes = [vp, vp, u64, C.c_uint32, C.c_int, vp, vp, C.c_int, vp]
     L.qp_dsaciq_search.argtypes = [vp, vp, C.c_int, u64, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
     L.qp_dsaciq_curve.argtypes = [vp, C.POINTER(dbl), C.c_int, vp]
     L.qp_policy_use_ds.argtypes = [C.c_int]
@@ -386,6 +391,39 @@ class Context:
                                                out_stats.data_ptr() if out_stats is not None else None,
                                                _stream(self.device)))
         return out_packed, out_qp
+
+    # -- channel-wise variant: x is [rows, channels], the last dimension contiguous
+    def qp_stats_channels(self, x: torch.Tensor, channels: int, out: torch.Tensor | None = None) -> torch.Tensor:
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        out = self._bytes(C.sizeof(Stats) * channels) if out is None else out
+        self._check(self._lib.qp_stats_channels(self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels, channels,
+                                                out.data_ptr(), _stream(self.device)))
+        return out
+
+    def qp_clip_qparams_channels_device(self, d_stats: torch.Tensor, channels: int, bits: int, method: int = QP_CLIP_ACIQ,
+                                        dist: int = QP_DIST_LAPLACE, bmode: int = QP_B_MAD,
+                                        out: torch.Tensor | None = None) -> torch.Tensor:
+        out = self._bytes(C.sizeof(QParams) * channels) if out is None else out
+        self._check(self._lib.qp_clip_qparams_channels_device(self._h, d_stats.data_ptr(), channels, bits, method, dist,
+                                                              bmode, out.data_ptr(), _stream(self.device)))
+        return out
+
+    def qp_quantize_pack_channels(self, x: torch.Tensor, channels: int, bits: int, d_qp: torch.Tensor,
+                                  out: torch.Tensor | None = None) -> torch.Tensor:
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        out = self._bytes(qp_packed_bytes(x.numel(), bits)) if out is None else out
+        self._check(self._lib.qp_quantize_pack_channels(self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels,
+                                                        channels, bits, d_qp.data_ptr(), out.data_ptr(),
+                                                        out.numel() * out.element_size(), _stream(self.device)))
+        return out
+
+    def qp_unpack_dequantize_channels(self, packed: torch.Tensor, rows: int, channels: int, bits: int, d_qp: torch.Tensor,
+                                      out: torch.Tensor | None = None, out_dtype=torch.float32) -> torch.Tensor:
+        out = torch.empty(rows * channels, dtype=out_dtype, device=packed.device) if out is None else out
+        self._check(self._lib.qp_unpack_dequantize_channels(self._h, packed.data_ptr(), rows, channels, bits,
+                                                            d_qp.data_ptr(), out.data_ptr(), _dtype_code(out),
+                                                            _stream(self.device)))
+        return out
 
     # -- host-buffer sender / receiver
     def qp_sender_host(self, h_x: torch.Tensor, bits: int, use_ds: bool, d_x_work: torch.Tensor,

@@ -126,6 +126,7 @@ extern "C" int32_t qp_destroy(qp_ctx* ctx)
     if (!ctx) return QP_ERR_INVALID_ARG;
     qp_device_guard guard(ctx->device);
     qp_drop_graphs(ctx);
+    if (ctx->d_ch_part) cudaFree(ctx->d_ch_part);
     const cudaError_t e = cudaFree(ctx->d_base);
     delete ctx;
     return e == cudaSuccess ? QP_OK : QP_ERR_CUDA;

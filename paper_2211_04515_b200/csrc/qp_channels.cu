@@ -1,0 +1,635 @@
+// Channel-wise variant of the path (a variant of this library: the paper, Sec. 3, uses one clip
+// range per tensor; channel-wise ranges are what its cited PTQ work uses for activations with
+// outlier channels).  The tensor is [rows, channels], row-major: element i belongs to channel
+// i mod channels.  Every channel gets the statistics, clip range and quantizer that the
+// per-tensor functions give for its column alone; bit-width and packed layout are shared.
+//
+//   ch_stats_a / ch_stats_b   column reductions, HBM-bound: a thread owns V consecutive channels
+//                             (one 16-byte load per row when the layout allows), a block walks
+//                             rows blockIdx.x, blockIdx.x + gridDim.x, ... with 8 rows in flight,
+//                             fp32 sums over those 8 rows folded into fp64; block partials
+//                             [block][channel] are merged per channel in block order by
+//                             ch_merge_a / ch_merge_b (bit-reproducible)
+//   ch_clip_kernel            one thread per channel: closed-form clip -> quantizer
+//   ch_pack_kernel            tile of 8192 elements: coalesced loads, quantize with the channel's
+//                             parameters (table in shared memory), 16-bit codes into padded shared
+//                             memory; then each thread packs 32 consecutive codes = `bits` words
+//   ch_unpack_kernel          mirror image: words -> codes in shared memory -> coalesced stores
+#include "qp_internal.cuh"
+
+namespace {
+
+constexpr int CH_THREADS = 256;
+constexpr int CH_TILE = CH_THREADS * 32;          // elements per tile
+constexpr int CH_CODE_WORDS = CH_THREADS * 17;    // 16 words of codes per 32 elements + 1 pad word
+constexpr int CH_ROWS_IN_FLIGHT = 8;
+
+struct ChPart {                                   // one per (row block, channel)
+    double s0, s1;                                // pass A: sum x, sum |x|;  pass B: sum |x-mean|, sum (x-mean)^2
+    float mn, mx;
+    unsigned bad, pad;
+};
+
+template <typename T, int V>
+__device__ __forceinline__ void ch_load(const T* p, float (&e)[V])
+{
+    if constexpr (V == 1) {
+        e[0] = qp_load_one(p);
+    } else {
+        qp_load_vec(p, e);
+    }
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(CH_THREADS) ch_stats_a(const T* __restrict__ x, uint64_t rows, uint32_t C,
+                                                         ChPart* __restrict__ part)
+{
+    const uint32_t col0 = (blockIdx.y * CH_THREADS + threadIdx.x) * V;
+    if (col0 >= C) return;
+    const float inf = __int_as_float(0x7F800000);
+    double s[V], sa[V];
+    float mn[V], mx[V];
+    unsigned bad[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) { s[i] = 0.0; sa[i] = 0.0; mn[i] = inf; mx[i] = -inf; bad[i] = 0u; }
+    const uint64_t step = gridDim.x;
+    for (uint64_t r0 = blockIdx.x; r0 < rows; r0 += CH_ROWS_IN_FLIGHT * step) {
+        float e[CH_ROWS_IN_FLIGHT][V];
+#pragma unroll
+        for (int u = 0; u < CH_ROWS_IN_FLIGHT; ++u) {
+            const uint64_t r = r0 + u * step;
+            if (r < rows) ch_load<T, V>(x + r * C + col0, e[u]);
+        }
+        float ps[V], psa[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) { ps[i] = 0.f; psa[i] = 0.f; }
+#pragma unroll
+        for (int u = 0; u < CH_ROWS_IN_FLIGHT; ++u) {
+            if (r0 + u * step >= rows) break;
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const float v = e[u][i];
+                if (qp_is_finite(v)) {
+                    ps[i] += v;
+                    psa[i] += fabsf(v);
+                    mn[i] = fminf(mn[i], v);
+                    mx[i] = fmaxf(mx[i], v);
+                } else {
+                    ++bad[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < V; ++i) { s[i] += (double)ps[i]; sa[i] += (double)psa[i]; }
+    }
+    ChPart* dst = part + (size_t)blockIdx.x * C + col0;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        ChPart p;
+        p.s0 = s[i]; p.s1 = sa[i]; p.mn = mn[i]; p.mx = mx[i]; p.bad = bad[i]; p.pad = 0u;
+        dst[i] = p;
+    }
+}
+
+__global__ void __launch_bounds__(CH_THREADS) ch_merge_a(const ChPart* __restrict__ part, int blocks, uint64_t rows,
+                                                         uint32_t C, qp_stats_t* __restrict__ out,
+                                                         unsigned* __restrict__ status)
+{
+    const uint32_t c = blockIdx.x * CH_THREADS + threadIdx.x;
+    if (c >= C) return;
+    const float inf = __int_as_float(0x7F800000);
+    double s = 0.0, sa = 0.0;
+    float mn = inf, mx = -inf;
+    unsigned long long bad = 0;
+    for (int b0 = 0; b0 < blocks; b0 += 8) {              // block order; eight loads in flight
+        ChPart p[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (b0 + u < blocks) p[u] = part[(size_t)(b0 + u) * C + c];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (b0 + u >= blocks) break;
+            s += p[u].s0;
+            sa += p[u].s1;
+            mn = fminf(mn, p[u].mn);
+            mx = fmaxf(mx, p[u].mx);
+            bad += p[u].bad;
+        }
+    }
+    const unsigned long long nf = rows - bad;
+    qp_stats_t st;
+    st.n = rows;
+    st.nonfinite = bad;
+    st.mean = nf ? s / (double)nf : 0.0;
+    st.mean_abs = nf ? sa / (double)nf : 0.0;
+    st.mad = 0.0;
+    st.var = 0.0;
+    st.min = nf ? (double)mn : 0.0;
+    st.max = nf ? (double)mx : 0.0;
+    st.hist_peak = 0;
+    st.hist_bins = 0;
+    st.reserved = 0;
+    out[c] = st;
+    if (bad) atomicOr(status, QP_DEV_NONFINITE);
+}
+
+template <typename T, int V>
+__global__ void __launch_bounds__(CH_THREADS) ch_stats_b(const T* __restrict__ x, uint64_t rows, uint32_t C,
+                                                         const qp_stats_t* __restrict__ st, ChPart* __restrict__ part)
+{
+    const uint32_t col0 = (blockIdx.y * CH_THREADS + threadIdx.x) * V;
+    if (col0 >= C) return;
+    float m_hi[V], m_lo[V];                               // each channel's mean as an unevaluated fp32 pair
+    double sd[V], sv[V];
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        const double mean = st[col0 + i].mean;
+        m_hi[i] = (float)mean;
+        m_lo[i] = (float)(mean - (double)m_hi[i]);
+        sd[i] = 0.0;
+        sv[i] = 0.0;
+    }
+    const uint64_t step = gridDim.x;
+    for (uint64_t r0 = blockIdx.x; r0 < rows; r0 += CH_ROWS_IN_FLIGHT * step) {
+        float e[CH_ROWS_IN_FLIGHT][V];
+#pragma unroll
+        for (int u = 0; u < CH_ROWS_IN_FLIGHT; ++u) {
+            const uint64_t r = r0 + u * step;
+            if (r < rows) ch_load<T, V>(x + r * C + col0, e[u]);
+        }
+        float d1[V], d2[V];
+#pragma unroll
+        for (int i = 0; i < V; ++i) { d1[i] = 0.f; d2[i] = 0.f; }
+#pragma unroll
+        for (int u = 0; u < CH_ROWS_IN_FLIGHT; ++u) {
+            if (r0 + u * step >= rows) break;
+#pragma unroll
+            for (int i = 0; i < V; ++i) {
+                const float v = e[u][i];
+                if (!qp_is_finite(v)) continue;
+                const float d = __fsub_rn(__fsub_rn(v, m_hi[i]), m_lo[i]);
+                d1[i] += fabsf(d);
+                d2[i] = fmaf(d, d, d2[i]);
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < V; ++i) { sd[i] += (double)d1[i]; sv[i] += (double)d2[i]; }
+    }
+    ChPart* dst = part + (size_t)blockIdx.x * C + col0;
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        dst[i].s0 = sd[i];
+        dst[i].s1 = sv[i];
+    }
+}
+
+__global__ void __launch_bounds__(CH_THREADS) ch_merge_b(const ChPart* __restrict__ part, int blocks, uint32_t C,
+                                                         qp_stats_t* __restrict__ out)
+{
+    const uint32_t c = blockIdx.x * CH_THREADS + threadIdx.x;
+    if (c >= C) return;
+    double sd = 0.0, sv = 0.0;
+    for (int b0 = 0; b0 < blocks; b0 += 8) {
+        double a[8], b[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            if (b0 + u < blocks) {
+                a[u] = part[(size_t)(b0 + u) * C + c].s0;
+                b[u] = part[(size_t)(b0 + u) * C + c].s1;
+            }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            if (b0 + u >= blocks) break;
+            sd += a[u];
+            sv += b[u];
+        }
+    }
+    const unsigned long long nf = out[c].n - out[c].nonfinite;
+    out[c].mad = nf ? sd / (double)nf : 0.0;
+    out[c].var = nf ? sv / (double)nf : 0.0;
+}
+
+__global__ void __launch_bounds__(128) ch_clip_kernel(const qp_stats_t* __restrict__ st, uint32_t C, int bits, int method,
+                                                      int dist, int bmode, double F, qp_qparams_t* __restrict__ qp_out,
+                                                      unsigned* __restrict__ status)
+{
+    const uint32_t c = blockIdx.x * 128 + threadIdx.x;
+    if (c >= C) return;
+    double lo, hi;
+    qp_clip_ends(st[c], method, dist, bmode, F, lo, hi);
+    qp_qparams_t q;
+    const int rc = qp_fill_qparams(lo, hi, bits, &q);
+    qp_out[c] = q;
+    if (rc == QP_WARN_DEGENERATE) atomicOr(status, QP_DEV_DEGENERATE);
+}
+
+// ---- quantize + pack
+
+// shared-memory word that holds the 16-bit codes of local elements le, le + 1 (le even)
+__device__ __forceinline__ int ch_code_word(int le) { return (le >> 1) + (le >> 5); }
+
+__device__ __forceinline__ void ch_load_table(const qp_qparams_t* __restrict__ d_qp, uint32_t C, int bits, float4* tab,
+                                              unsigned* status)
+{
+    bool mismatch = false;
+    for (uint32_t c = threadIdx.x; c < C; c += CH_THREADS) {
+        const qp_qparams_t q = d_qp[c];
+        tab[c] = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
+        mismatch |= q.bits != bits;
+    }
+    if (mismatch && blockIdx.x == 0) atomicOr(status, QP_DEV_BITS_MISMATCH);
+}
+
+template <typename T, bool VEC>
+__global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict__ x, uint64_t n, uint32_t C, int bits,
+                                                             const qp_qparams_t* __restrict__ d_qp,
+                                                             uint32_t* __restrict__ out, uint64_t total_words,
+                                                             uint64_t ntiles, unsigned* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char raw[];
+    float4* tab = reinterpret_cast<float4*>(raw);                                  // [C] lo, hi, scale, inv_scale
+    uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)); // [CH_CODE_WORDS]
+    ch_load_table(d_qp, C, bits, tab, status);
+    __syncthreads();
+    constexpr int EPV = qp_span<T>::EPV;
+    const unsigned mask = (1u << bits) - 1u;
+    const int tid = threadIdx.x;
+    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint64_t base = tile * CH_TILE;
+        if (VEC) {
+            // thread takes vectors tid, tid + 256, ...: its channel advances by (256 * EPV) mod C each time
+            uint32_t c = (uint32_t)((base + (uint64_t)tid * EPV) % C);
+            const uint32_t cstep = (uint32_t)(((uint64_t)CH_THREADS * EPV) % C);
+            constexpr int NV = CH_TILE / (CH_THREADS * EPV);
+#pragma unroll
+            for (int k0 = 0; k0 < NV; k0 += 4) {
+                float e[4][EPV];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const uint64_t el = base + (uint64_t)((k0 + u) * CH_THREADS + tid) * EPV;
+                    if (el + EPV <= n) {
+                        qp_load_vec(x + el, e[u]);
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < EPV; ++i) e[u][i] = el + i < n ? qp_load_one(x + el + i) : 0.f;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int le = ((k0 + u) * CH_THREADS + tid) * EPV;
+                    const uint64_t el = base + le;
+                    unsigned cd[EPV];
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) {
+                        const float4 q = tab[c + i];             // EPV divides C: the vector stays in one row
+                        cd[i] = el + i < n ? qp_code(e[u][i], q.x, q.y, q.w, mask) : 0u;
+                    }
+#pragma unroll
+                    for (int i = 0; i < EPV; i += 2) codes[ch_code_word(le + i)] = cd[i] | (cd[i + 1] << 16);
+                    c += cstep;
+                    if (c >= C) c -= C;
+                }
+            }
+        } else {
+            unsigned short* ch = reinterpret_cast<unsigned short*>(codes);
+            for (int k = 0; k < 32; ++k) {
+                const int le = k * CH_THREADS + tid;
+                const uint64_t el = base + le;
+                unsigned cd = 0u;
+                if (el < n) {
+                    const float4 q = tab[el % C];
+                    cd = qp_code(qp_load_one(x + el), q.x, q.y, q.w, mask);
+                }
+                ch[le + ((le >> 5) << 1)] = (unsigned short)cd;
+            }
+        }
+        __syncthreads();
+        {
+            const uint64_t w0 = (tile * CH_THREADS + tid) * (uint64_t)bits;   // this thread's group of 32 elements
+            if (w0 < total_words) {
+                uint32_t w[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j) w[j] = codes[17 * tid + j];
+                unsigned long long acc = 0ull;
+                int fill = 0;
+                uint32_t* dst = out + w0;
+                const uint32_t* end = out + total_words;
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    const unsigned cd = (w[i >> 1] >> ((i & 1) * 16)) & 0xFFFFu;
+                    acc |= (unsigned long long)cd << fill;
+                    fill += bits;
+                    if (fill >= 32) {
+                        if (dst < end) *dst = (uint32_t)acc;
+                        ++dst;
+                        acc >>= 32;
+                        fill -= 32;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ---- unpack + dequantize
+
+__device__ __forceinline__ float ch_code_to_float(unsigned c) { return __fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.0f); }
+
+__device__ __forceinline__ void ch_store4(float* y, uint64_t el, const float (&v)[4])
+{
+    *reinterpret_cast<float4*>(y + el) = make_float4(v[0], v[1], v[2], v[3]);
+}
+__device__ __forceinline__ void ch_store4(unsigned short* y, uint64_t el, const float (&v)[4])
+{
+    uint2 o;
+    o.x = (unsigned)qp_f32_to_bf16(v[0]) | ((unsigned)qp_f32_to_bf16(v[1]) << 16);
+    o.y = (unsigned)qp_f32_to_bf16(v[2]) | ((unsigned)qp_f32_to_bf16(v[3]) << 16);
+    *reinterpret_cast<uint2*>(y + el) = o;
+}
+__device__ __forceinline__ void ch_store1(float* y, uint64_t el, float v) { y[el] = v; }
+__device__ __forceinline__ void ch_store1(unsigned short* y, uint64_t el, float v) { y[el] = qp_f32_to_bf16(v); }
+
+template <typename TO, bool VEC>
+__global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* __restrict__ in, uint64_t n, uint32_t C,
+                                                               int bits, const qp_qparams_t* __restrict__ d_qp,
+                                                               TO* __restrict__ y, uint64_t total_words, uint64_t ntiles,
+                                                               unsigned* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char raw[];
+    float4* tab = reinterpret_cast<float4*>(raw);
+    uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4));
+    ch_load_table(d_qp, C, bits, tab, status);
+    __syncthreads();
+    const unsigned mask = (1u << bits) - 1u;
+    const int tid = threadIdx.x;
+    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
+        const uint64_t base = tile * CH_TILE;
+        {
+            // this thread's group of 32 elements: `bits` words -> 32 codes -> 16 shared-memory words
+            const uint64_t w0 = (tile * CH_THREADS + tid) * (uint64_t)bits;
+            uint32_t w[16];
+#pragma unroll
+            for (int m = 0; m < 16; ++m) w[m] = (m < bits && w0 + m < total_words) ? __ldg(in + w0 + m) : 0u;
+            unsigned long long acc = 0ull;                     // bits not yet consumed, oldest lowest
+            int have = 0, i = 0;
+            unsigned prev = 0u;
+#pragma unroll
+            for (int m = 0; m < 16; ++m) {
+                if (m < bits) {
+                    acc |= (unsigned long long)w[m] << have;
+                    have += 32;
+                    while (have >= bits) {
+                        const unsigned cd = (unsigned)acc & mask;
+                        acc >>= bits;
+                        have -= bits;
+                        if (i & 1) codes[17 * tid + (i >> 1)] = prev | (cd << 16);
+                        else       prev = cd;
+                        ++i;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+        if (VEC) {
+            uint32_t c = (uint32_t)((base + (uint64_t)tid * 4) % C);
+            const uint32_t cstep = (uint32_t)(((uint64_t)CH_THREADS * 4) % C);
+#pragma unroll
+            for (int k = 0; k < CH_TILE / (CH_THREADS * 4); ++k) {
+                const int le = (k * CH_THREADS + tid) * 4;
+                const uint64_t el = base + le;
+                const uint32_t a = codes[ch_code_word(le)], b = codes[ch_code_word(le + 2)];
+                const unsigned cd[4] = {a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16};
+                float v[4];
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float4 q = tab[c + i];
+                    v[i] = fmaf(ch_code_to_float(cd[i]), q.z, q.x);
+                }
+                if (el + 4 <= n) {
+                    ch_store4(y, el, v);
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        if (el + i < n) ch_store1(y, el + i, v[i]);
+                }
+                c += cstep;
+                if (c >= C) c -= C;
+            }
+        } else {
+            const unsigned short* ch = reinterpret_cast<const unsigned short*>(codes);
+            for (int k = 0; k < 32; ++k) {
+                const int le = k * CH_THREADS + tid;
+                const uint64_t el = base + le;
+                if (el < n) {
+                    const float4 q = tab[el % C];
+                    ch_store1(y, el, fmaf(ch_code_to_float(ch[le + ((le >> 5) << 1)]), q.z, q.x));
+                }
+            }
+        }
+        __syncthreads();
+    }
+}
+
+// ---- host side
+
+int32_t ch_check(qp_ctx* ctx, uint64_t rows, uint32_t channels)
+{
+    if (channels < 1 || channels > QP_MAX_CHANNELS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "channels must be 1..QP_MAX_CHANNELS");
+    if (rows >= (1ull << 40) / channels) return qp_fail(ctx, QP_ERR_INVALID_ARG, "tensor too large");
+    return QP_OK;
+}
+
+// block partials of the column reductions: grown on demand, kept by the context
+int32_t ch_scratch(qp_ctx* ctx, size_t bytes)
+{
+    if (ctx->ch_part_bytes >= bytes) return QP_OK;
+    if (ctx->d_ch_part) cudaFree(ctx->d_ch_part);
+    ctx->d_ch_part = nullptr;
+    ctx->ch_part_bytes = 0;
+    if (cudaMalloc(&ctx->d_ch_part, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        return qp_fail(ctx, QP_ERR_CUDA, "cannot allocate the channel partials");
+    }
+    ctx->ch_part_bytes = bytes;
+    return QP_OK;
+}
+
+template <typename T>
+int32_t stats_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C, qp_stats_t* d_out, cudaStream_t s)
+{
+    constexpr int EPV = qp_span<T>::EPV;
+    const bool vec = (C % EPV == 0) && (((uintptr_t)x & 15u) == 0);
+    const int V = vec ? EPV : 1;
+    const unsigned col_blocks = (C / V + CH_THREADS - 1) / CH_THREADS;
+    // enough row blocks to fill the GPU a few times over, no more than there are rows
+    // about two blocks per SM in all: 8 x 16-byte loads in flight per thread keep HBM busy, and
+    // the partials (32 bytes per row block and channel) stay a few percent of the tensor
+    uint64_t want = (uint64_t)ctx->sm_count * 2 / col_blocks;
+    if (want < (uint64_t)ctx->sm_count) want = ctx->sm_count;
+    const int row_blocks = (int)(rows < want ? rows : want);
+    int32_t rc = ch_scratch(ctx, sizeof(ChPart) * (size_t)row_blocks * C);
+    if (rc) return rc;
+    ChPart* part = static_cast<ChPart*>(ctx->d_ch_part);
+    const dim3 grid(row_blocks, col_blocks);
+    const unsigned merge_blocks = (C + CH_THREADS - 1) / CH_THREADS;
+    if (vec) ch_stats_a<T, EPV><<<grid, CH_THREADS, 0, s>>>(x, rows, C, part);
+    else     ch_stats_a<T, 1><<<grid, CH_THREADS, 0, s>>>(x, rows, C, part);
+    ch_merge_a<<<merge_blocks, CH_THREADS, 0, s>>>(part, row_blocks, rows, C, d_out, ctx->d_status);
+    if (vec) ch_stats_b<T, EPV><<<grid, CH_THREADS, 0, s>>>(x, rows, C, d_out, part);
+    else     ch_stats_b<T, 1><<<grid, CH_THREADS, 0, s>>>(x, rows, C, d_out, part);
+    ch_merge_b<<<merge_blocks, CH_THREADS, 0, s>>>(part, row_blocks, C, d_out);
+    ctx->launches += 4;
+    return qp_check_launch(ctx, "qp_stats_channels");
+}
+
+size_t ch_pack_smem(uint32_t C) { return (size_t)C * sizeof(float4) + (size_t)CH_CODE_WORDS * sizeof(uint32_t); }
+
+template <typename K>
+bool ch_allow_smem(K kernel, size_t bytes)
+{
+    return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes) == cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" int32_t qp_stats_channels(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels,
+                                     qp_stats_t* d_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (dtype != QP_F32 && dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "dtype must be QP_F32 or QP_BF16");
+    int32_t rc = ch_check(ctx, rows, channels);
+    if (rc) return rc;
+    if (!d_out || (rows > 0 && !d_x)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
+    if (((uintptr_t)d_x & (dtype == QP_F32 ? 3u : 1u)) || ((uintptr_t)d_out & 7u))
+        return qp_fail(ctx, QP_ERR_ALIGNMENT, "tensor or d_out not aligned");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (rows == 0) {
+        if (cudaMemsetAsync(d_out, 0, sizeof(qp_stats_t) * channels, s) != cudaSuccess)
+            return qp_check_launch(ctx, "qp_stats_channels");
+        return QP_OK;
+    }
+    if (dtype == QP_F32) return stats_channels_typed<float>(ctx, static_cast<const float*>(d_x), rows, channels, d_out, s);
+    return stats_channels_typed<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), rows, channels, d_out, s);
+}
+
+extern "C" int32_t qp_clip_qparams_channels_device(qp_ctx* ctx, const qp_stats_t* d_stats, uint32_t channels, int bits,
+                                                   int method, int dist, int bmode, qp_qparams_t* d_qp_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    int32_t rc = ch_check(ctx, 0, channels);
+    if (rc) return rc;
+    if (!d_stats || !d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (method != QP_CLIP_ACIQ && method != (QP_CLIP_ACIQ | QP_CLIP_INTERSECT) && method != QP_CLIP_MINMAX)
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT) or MINMAX");
+    if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "dist/bmode");
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    ch_clip_kernel<<<(channels + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(
+        d_stats, channels, bits, method, dist, bmode, qp_host_aciq_F(bits, dist), d_qp_out, ctx->d_status);
+    ctx->launches += 1;
+    return qp_check_launch(ctx, "qp_clip_qparams_channels_device");
+}
+
+extern "C" int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels,
+                                             int bits, const qp_qparams_t* d_qp, void* d_packed,
+                                             uint64_t packed_capacity, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (dtype != QP_F32 && dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "dtype must be QP_F32 or QP_BF16");
+    int32_t rc = ch_check(ctx, rows, channels);
+    if (rc) return rc;
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    const uint64_t n = rows * channels;
+    const uint64_t need = qp_packed_bytes(n, bits);
+    if (packed_capacity < need) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
+    if (!d_qp || (n > 0 && (!d_x || !d_packed))) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
+    if (((uintptr_t)d_x & (dtype == QP_F32 ? 3u : 1u)) || ((uintptr_t)d_packed & 15u) || ((uintptr_t)d_qp & 3u))
+        return qp_fail(ctx, QP_ERR_ALIGNMENT, "tensor, d_packed (16 bytes) or d_qp not aligned");
+    if (n == 0) return QP_OK;
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint64_t total_words = need / 4;
+    const uint64_t groups = (total_words + bits - 1) / bits;
+    const uint64_t ntiles = (groups + CH_THREADS - 1) / CH_THREADS;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 4;
+    const unsigned blocks = (unsigned)(ntiles < cap ? ntiles : cap);
+    const size_t smem = ch_pack_smem(channels);
+    uint32_t* out = static_cast<uint32_t*>(d_packed);
+    bool ok;
+    if (dtype == QP_F32) {
+        const float* x = static_cast<const float*>(d_x);
+        if (channels % 4 == 0 && ((uintptr_t)x & 15u) == 0) {
+            ok = ch_allow_smem(ch_pack_kernel<float, true>, smem);
+            if (ok) ch_pack_kernel<float, true><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
+        } else {
+            ok = ch_allow_smem(ch_pack_kernel<float, false>, smem);
+            if (ok) ch_pack_kernel<float, false><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
+        }
+    } else {
+        const unsigned short* x = static_cast<const unsigned short*>(d_x);
+        if (channels % 8 == 0 && ((uintptr_t)x & 15u) == 0) {
+            ok = ch_allow_smem(ch_pack_kernel<unsigned short, true>, smem);
+            if (ok) ch_pack_kernel<unsigned short, true><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
+        } else {
+            ok = ch_allow_smem(ch_pack_kernel<unsigned short, false>, smem);
+            if (ok) ch_pack_kernel<unsigned short, false><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
+        }
+    }
+    if (!ok) return qp_check_launch(ctx, "qp_quantize_pack_channels (shared memory)");
+    ctx->launches += 1;
+    return qp_check_launch(ctx, "qp_quantize_pack_channels");
+}
+
+extern "C" int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_packed, uint64_t rows, uint32_t channels,
+                                                 int bits, const qp_qparams_t* d_qp, void* d_y, int out_dtype,
+                                                 void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (out_dtype != QP_F32 && out_dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "out_dtype");
+    int32_t rc = ch_check(ctx, rows, channels);
+    if (rc) return rc;
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    const uint64_t n = rows * channels;
+    if (!d_qp || (n > 0 && (!d_packed || !d_y))) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
+    if (((uintptr_t)d_packed & 15u) || ((uintptr_t)d_qp & 3u) || ((uintptr_t)d_y & (out_dtype == QP_F32 ? 3u : 1u)))
+        return qp_fail(ctx, QP_ERR_ALIGNMENT, "d_packed (16 bytes), d_qp or d_y not aligned");
+    if (n == 0) return QP_OK;
+    qp_device_guard guard(ctx->device);
+    if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const uint64_t total_words = qp_packed_bytes(n, bits) / 4;
+    const uint64_t ntiles = (n + CH_TILE - 1) / CH_TILE;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 4;
+    const unsigned blocks = (unsigned)(ntiles < cap ? ntiles : cap);
+    const size_t smem = ch_pack_smem(channels);
+    const uint32_t* in = static_cast<const uint32_t*>(d_packed);
+    bool ok;
+    if (out_dtype == QP_F32) {
+        float* y = static_cast<float*>(d_y);
+        if (channels % 4 == 0 && ((uintptr_t)y & 15u) == 0) {
+            ok = ch_allow_smem(ch_unpack_kernel<float, true>, smem);
+            if (ok) ch_unpack_kernel<float, true><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
+        } else {
+            ok = ch_allow_smem(ch_unpack_kernel<float, false>, smem);
+            if (ok) ch_unpack_kernel<float, false><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
+        }
+    } else {
+        unsigned short* y = static_cast<unsigned short*>(d_y);
+        if (channels % 4 == 0 && ((uintptr_t)y & 7u) == 0) {
+            ok = ch_allow_smem(ch_unpack_kernel<unsigned short, true>, smem);
+            if (ok) ch_unpack_kernel<unsigned short, true><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
+        } else {
+            ok = ch_allow_smem(ch_unpack_kernel<unsigned short, false>, smem);
+            if (ok) ch_unpack_kernel<unsigned short, false><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
+        }
+    }
+    if (!ok) return qp_check_launch(ctx, "qp_unpack_dequantize_channels (shared memory)");
+    ctx->launches += 1;
+    return qp_check_launch(ctx, "qp_unpack_dequantize_channels");
+}

@@ -77,6 +77,8 @@ struct qp_ctx {
     int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
     size_t fused_dyn_max;                // largest slice (bytes of dynamic shared memory) per block
     void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
+    void* d_ch_part;                     // channel-wise statistics: block partials, allocated on first use
+    size_t ch_part_bytes;
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
     qp_qparams_t* d_tmp_qp;
     unsigned long long launches;         // kernels launched through this context (host count)

@@ -748,3 +748,129 @@ def test_graph_replay_gives_the_same_bytes(n_images, path):
     assert replay.qp_graph_replays() == hits and torch.equal(st, want_st)
     assert replay.qp_get_status() == 0 and plain.qp_get_status() == 0
     plain.close(); replay.close()
+
+
+# ------------------------------------------------------------------ channel-wise variant
+
+def _read_array(t, ctype, count):
+    raw = t.cpu().numpy().tobytes()
+    return (ctype * count).from_buffer_copy(raw)
+
+
+def check_channels(ctx, x_np, d_x, channels, bits, method=qp.QP_CLIP_ACIQ, out_bf16=False):
+    """Statistics, quantizers, packed stream and reconstruction of the channel-wise calls against the
+    oracle.  The statistics are compared at 1e-5; the packed stream bit for bit under the quantizers the
+    kernels produced, and those quantizers against the oracle's per channel."""
+    rows = x_np.size // channels
+    d_stats = ctx.qp_stats_channels(d_x, channels)
+    st = _read_array(d_stats, qp.Stats, channels)
+    st_o = oracle.stats_channels(x_np, channels)
+    for c in range(channels):
+        check_stats(st[c], st_o[c])
+    o_method, cut = (oracle.CLIP_MINMAX, False) if method == qp.QP_CLIP_MINMAX else (oracle.CLIP_ACIQ, bool(method & qp.QP_CLIP_INTERSECT))
+    d_qp = ctx.qp_clip_qparams_channels_device(d_stats, channels, bits, method)
+    got = _read_array(d_qp, qp.QParams, channels)
+    rc_o, qp_o = oracle.clip_channels(st_o, bits, o_method, cut)
+    for c in range(channels):
+        width = max(qp_o[c].hi - qp_o[c].lo, 1e-30)
+        assert abs(got[c].lo - qp_o[c].lo) <= 1e-5 * width and abs(got[c].hi - qp_o[c].hi) <= 1e-5 * width, c
+        assert got[c].bits == bits and got[c].flags == qp_o[c].flags
+        rc2, again = oracle.make_qparams(got[c].lo, got[c].hi, bits)
+        assert (again.scale, again.inv_scale) == (got[c].scale, got[c].inv_scale)
+    mine = (oracle.QParams * channels)(*[oracle.QParams(g.lo, g.hi, g.scale, g.inv_scale, g.bits, g.flags) for g in got])
+    nbytes = qp.qp_packed_bytes(x_np.size, bits)
+    whole, packed = guarded(nbytes)
+    ctx.qp_quantize_pack_channels(d_x, channels, bits, d_qp, out=packed)
+    codes_o = oracle.quantize_channels(x_np, channels, mine)
+    assert np.array_equal(packed.cpu().numpy(), oracle.pack(codes_o, bits))
+    assert canaries_intact(whole, nbytes)
+    esz = 2 if out_bf16 else 4
+    whole_y, y_bytes = guarded(x_np.size * esz)
+    y = y_bytes.view(torch.bfloat16 if out_bf16 else torch.float32)
+    ctx.qp_unpack_dequantize_channels(packed, rows, channels, bits, d_qp, out=y)
+    y_o = oracle.dequantize_channels(codes_o, channels, mine)
+    if out_bf16:
+        want = si.bf16_bits_to_f32(si.to_bf16_bits(y_o))
+        assert np.array_equal(y.float().cpu().numpy(), want)
+    else:
+        assert np.max(np.abs(y.cpu().numpy().astype(np.float64) - y_o.astype(np.float64)), initial=0.0) <= 1e-6
+    assert canaries_intact(whole_y, x_np.size * esz)
+    return got
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_channels_vit_shapes(ctx, bits):
+    x = si.vit_activation((2, 197, 768), 101, outlier_frac=0.01).reshape(-1)
+    check_channels(ctx, x, dev(x), 768, bits)
+    assert ctx.qp_get_status() == 0
+
+
+@pytest.mark.parametrize("channels,rows", [(1, 5000), (3, 777), (4, 1), (20, 411), (64, 2049), (1000, 37), (1280, 300),
+                                            (4096, 9)])
+def test_channels_shapes_ragged_and_methods(ctx, channels, rows):
+    x = si.vit_activation((1, rows, channels), 102 + channels % 5, outlier_frac=0.05).reshape(-1)
+    d = dev(x)
+    for bits, method in ((2, qp.QP_CLIP_ACIQ), (5, qp.QP_CLIP_MINMAX), (8, qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT),
+                         (16, qp.QP_CLIP_ACIQ)):
+        check_channels(ctx, x, d, channels, bits, method)
+    ctx.qp_get_status()                                         # single-row tensors have no spread: degenerate
+
+
+def test_channels_misaligned_nonfinite_bf16(ctx):
+    x = si.vit_activation((1, 301, 96), 107, outlier_frac=0.03).reshape(-1).astype(np.float32)
+    big = dev(np.concatenate([np.zeros(1, np.float32), x]))
+    check_channels(ctx, x, big[1:], 96, 4)                      # 4-byte aligned only: scalar paths
+    x[[5, 96 * 7 + 5, 96 * 100 + 17]] = [np.nan, np.inf, -np.inf]
+    check_channels(ctx, x, dev(x), 96, 3)
+    assert ctx.qp_get_status() & qp.QP_DEV_NONFINITE
+    h = si.to_bf16_bits(si.vit_activation((1, 150, 256), 108).reshape(-1))
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    check_channels(ctx, oracle.widen_bf16(h), d, 256, 4)
+    check_channels(ctx, oracle.widen_bf16(h), d, 256, 8, out_bf16=True)
+    check_channels(ctx, oracle.widen_bf16(h[:150 * 100]), d[:150 * 100], 100, 6, out_bf16=True)   # 100 % 8 != 0
+    const = np.tile(np.array([1.5, -2.0, 0.0, 7.25], dtype=np.float32), 500)                      # every channel constant
+    got = check_channels(ctx, const, dev(const), 4, 4)
+    assert all(g.flags == 1 for g in got) and ctx.qp_get_status() & qp.QP_DEV_DEGENERATE
+
+
+def test_channels_errors_and_empty(ctx):
+    x = dev(si.flat_iid(4096, 6, "laplace"))
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_stats_channels(torch.zeros(2 * 8192, device="cuda"), 8192)      # beyond QP_MAX_CHANNELS
+    d_stats = ctx.qp_stats_channels(x, 64)
+    for bad in (qp.QP_CLIP_DSACIQ, 3):
+        with pytest.raises(qp.QuantPipeError):
+            ctx.qp_clip_qparams_channels_device(d_stats, 64, 4, bad)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_clip_qparams_channels_device(d_stats, 64, 9)
+    d_qp = ctx.qp_clip_qparams_channels_device(d_stats, 64, 4)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_quantize_pack_channels(x, 64, 4, d_qp, out=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    ctx.qp_quantize_pack_channels(x, 64, 8, d_qp)               # quantizers made for 4 bits: flagged on the device
+    assert ctx.qp_get_status() & qp.QP_DEV_BITS_MISMATCH
+    empty = torch.empty(0, device="cuda")
+    st = _read_array(ctx.qp_stats_channels(empty, 16), qp.Stats, 16)
+    assert all(s.n == 0 and s.mean == 0.0 for s in st)
+
+
+def test_channels_full_size_c2_sampled(ctx):
+    """ViT-Base micro-batch of 64 images, 768 channels: statistics of sampled channels and the packed
+    words of sampled rows against the oracle."""
+    x = si.config_tensor("c2").reshape(-1, 768)
+    d = dev(x.reshape(-1))
+    d_stats = ctx.qp_stats_channels(d, 768)
+    st = _read_array(d_stats, qp.Stats, 768)
+    for c in (0, 1, 255, 500, 767):
+        check_stats(st[c], oracle.stats(np.ascontiguousarray(x[:, c])))
+    d_qp = ctx.qp_clip_qparams_channels_device(d_stats, 768, 4)
+    got = _read_array(d_qp, qp.QParams, 768)
+    mine = (oracle.QParams * 768)(*[oracle.QParams(g.lo, g.hi, g.scale, g.inv_scale, g.bits, g.flags) for g in got])
+    packed = ctx.qp_quantize_pack_channels(d, 768, 4, d_qp).cpu().numpy()
+    y = ctx.qp_unpack_dequantize_channels(torch.from_numpy(packed).cuda(), x.shape[0], 768, 4, d_qp).cpu().numpy().reshape(-1, 768)
+    for r0 in (0, 4097, x.shape[0] - 3):
+        rows = x[r0:r0 + 3]
+        codes = oracle.quantize_channels(rows, 768, mine)
+        nb = 3 * 768 * 4 // 8
+        assert np.array_equal(packed[r0 * 768 // 2: r0 * 768 // 2 + nb], oracle.pack(codes, 4)[:nb])
+        assert np.max(np.abs(y[r0:r0 + 3].reshape(-1) - oracle.dequantize_channels(codes, 768, mine))) <= 1e-6
+    assert ctx.qp_get_status() == 0
