@@ -464,7 +464,7 @@ def sweep_main(args):
                         "frac_of_8000": round(g / 8000.0, 3), "peak_kind": peak_kind})
         print(json.dumps(row), flush=True)
 
-    def run_workload(name, x_host, bits_list, dtype="f32", search_bits=()):
+    def run_workload(name, x_host, bits_list, dtype="f32", search_bits=(), channels=0):
         n = x_host.numel()
         esz = 4 if dtype == "f32" else 2
         xs = rotating(lambda: x_host.cuda(), n * esz)
@@ -502,6 +502,27 @@ def sweep_main(args):
                     gctx.qp_set_graph_replay(False)           # drops this workload's graphs
                 emit(name, dtype, stage + "+graph", q, n, med, best, None)
             del pk
+        # channel-wise variant ([rows, channels], one quantizer per channel), ViT-shaped workloads only
+        if channels:
+            d_cst = torch.empty(80 * channels, dtype=torch.uint8, device="cuda")
+            med, best = timed(lambda i: ctx.qp_stats_channels(xs[i], channels, out=d_cst), nb)
+            emit(name, dtype, f"stats_channels[{channels}]", 0, n, med, best, esz * n)
+            for q in (4, 8):
+                d_cqp = ctx.qp_clip_qparams_channels_device(d_cst, channels, q)
+                pk = rotating(lambda: torch.empty(qp.qp_packed_bytes(n, q), dtype=torch.uint8, device="cuda"),
+                              n * esz + qp.qp_packed_bytes(n, q))
+                npk = len(pk)
+                med, best = timed(lambda i: ctx.qp_quantize_pack_channels(xs[i % nb], channels, q, d_cqp, out=pk[i % npk]),
+                                  max(nb, npk))
+                emit(name, dtype, f"quantize_pack_channels[{channels}]", q, n, med, best, (esz + q / 8.0) * n)
+                if dtype == "f32":
+                    ysc = rotating(lambda: torch.empty(n, dtype=torch.float32, device="cuda"), 4 * n)
+                    nyc = len(ysc)
+                    med, best = timed(lambda i: ctx.qp_unpack_dequantize_channels(pk[i % npk], n // channels, channels, q,
+                                                                                  d_cqp, out=ysc[i % nyc]), max(nyc, npk))
+                    emit(name, dtype, f"unpack_dequantize_channels[{channels}]", q, n, med, best, (4 + q / 8.0) * n)
+                    del ysc
+                del pk
         ys = None
         for q in bits_list:
             rc, alpha, qp_h = qp.qp_aciq_alpha(st, q)
@@ -523,7 +544,7 @@ def sweep_main(args):
     for name in ("c1", "c2", "c3", "c4"):
         cfg = si.CONFIGS[name]
         x = torch.from_numpy(si.config_tensor(name).reshape(-1))
-        run_workload(name, x, cfg["bits"], "f32", [b for b in cfg["bits"] if b <= 4][:2])
+        run_workload(name, x, cfg["bits"], "f32", [b for b in cfg["bits"] if b <= 4][:2], channels=cfg["shape"][-1])
     for log2n in range(18, args.sweep_max_log2 + 1, 2):
         for dist in ("laplace", "normal"):
             if dist == "normal" and log2n not in (22, 26):

@@ -6,23 +6,22 @@
 //
 //   ch_stats_a / ch_stats_b   column reductions, HBM-bound: a thread owns V consecutive channels
 //                             (one 16-byte load per row when the layout allows), a block walks
-//                             rows blockIdx.x, blockIdx.x + gridDim.x, ... with 8 rows in flight,
-//                             fp32 sums over those 8 rows folded into fp64; block partials
+//                             rows blockIdx.x, blockIdx.x + gridDim.x, ... with 8 rows in flight (4 for
+//                             bf16), fp32 sums over those rows folded into fp64; block partials
 //                             [block][channel] are merged per channel in block order by
 //                             ch_merge_a / ch_merge_b (bit-reproducible)
 //   ch_clip_kernel            one thread per channel: closed-form clip -> quantizer
-//   ch_pack_kernel            tile of 8192 elements: coalesced loads, quantize with the channel's
-//                             parameters (table in shared memory), 16-bit codes into padded shared
-//                             memory; then each thread packs 32 consecutive codes = `bits` words
-//   ch_unpack_kernel          mirror image: words -> codes in shared memory -> coalesced stores
+//   ch_pack_kernel            warp tile of 1024 elements: coalesced loads, quantize with the channel's
+//                             parameters (table in shared memory), 16-bit codes into the warp's
+//                             padded staging rows; then each lane packs 32 consecutive codes
+//   ch_unpack_kernel          mirror image: words -> codes in the staging rows -> coalesced stores
 #include "qp_internal.cuh"
 
 namespace {
 
 constexpr int CH_THREADS = 256;
-constexpr int CH_TILE = CH_THREADS * 32;          // elements per tile
-constexpr int CH_CODE_WORDS = CH_THREADS * 17;    // 16 words of codes per 32 elements + 1 pad word
-constexpr int CH_ROWS_IN_FLIGHT = 8;
+template <int V> struct ChRows { static constexpr int N = V >= 8 ? 4 : 8; };   // rows in flight per thread
+constexpr int CH_STATS_MAX_THREADS = 512;      // column-reduction blocks: one thread per group of V channels
 
 struct ChPart {                                   // one per (row block, channel)
     double s0, s1;                                // pass A: sum x, sum |x|;  pass B: sum |x-mean|, sum (x-mean)^2
@@ -41,10 +40,10 @@ __device__ __forceinline__ void ch_load(const T* p, float (&e)[V])
 }
 
 template <typename T, int V>
-__global__ void __launch_bounds__(CH_THREADS) ch_stats_a(const T* __restrict__ x, uint64_t rows, uint32_t C,
+__global__ void __launch_bounds__(CH_STATS_MAX_THREADS) ch_stats_a(const T* __restrict__ x, uint64_t rows, uint32_t C,
                                                          ChPart* __restrict__ part)
 {
-    const uint32_t col0 = (blockIdx.y * CH_THREADS + threadIdx.x) * V;
+    const uint32_t col0 = (blockIdx.y * blockDim.x + threadIdx.x) * V;
     if (col0 >= C) return;
     const float inf = __int_as_float(0x7F800000);
     double s[V], sa[V];
@@ -52,6 +51,7 @@ __global__ void __launch_bounds__(CH_THREADS) ch_stats_a(const T* __restrict__ x
     unsigned bad[V];
 #pragma unroll
     for (int i = 0; i < V; ++i) { s[i] = 0.0; sa[i] = 0.0; mn[i] = inf; mx[i] = -inf; bad[i] = 0u; }
+    constexpr int CH_ROWS_IN_FLIGHT = ChRows<V>::N;
     const uint64_t step = gridDim.x;
     for (uint64_t r0 = blockIdx.x; r0 < rows; r0 += CH_ROWS_IN_FLIGHT * step) {
         float e[CH_ROWS_IN_FLIGHT][V];
@@ -91,30 +91,51 @@ __global__ void __launch_bounds__(CH_THREADS) ch_stats_a(const T* __restrict__ x
     }
 }
 
+// Merge of the row blocks' partials: a block takes 32 channels (lane = channel, so a warp reads
+// 1 KB rows of partials), warp w adds row blocks w, w + 8, ... in order with four loads in
+// flight, and the eight warp sums are combined in warp order: the same bits on every run.
+constexpr int CH_MERGE_WARPS = CH_THREADS / 32;
 __global__ void __launch_bounds__(CH_THREADS) ch_merge_a(const ChPart* __restrict__ part, int blocks, uint64_t rows,
                                                          uint32_t C, qp_stats_t* __restrict__ out,
                                                          unsigned* __restrict__ status)
 {
-    const uint32_t c = blockIdx.x * CH_THREADS + threadIdx.x;
-    if (c >= C) return;
+    __shared__ double s_s[CH_MERGE_WARPS][32], s_sa[CH_MERGE_WARPS][32];
+    __shared__ float s_mn[CH_MERGE_WARPS][32], s_mx[CH_MERGE_WARPS][32];
+    __shared__ unsigned long long s_bad[CH_MERGE_WARPS][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t c = blockIdx.x * 32 + lane;
     const float inf = __int_as_float(0x7F800000);
     double s = 0.0, sa = 0.0;
     float mn = inf, mx = -inf;
     unsigned long long bad = 0;
-    for (int b0 = 0; b0 < blocks; b0 += 8) {              // block order; eight loads in flight
-        ChPart p[8];
+    if (c < C) {
+        for (int b0 = warp; b0 < blocks; b0 += 4 * CH_MERGE_WARPS) {
+            ChPart p[4];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (b0 + u < blocks) p[u] = part[(size_t)(b0 + u) * C + c];
+            for (int u = 0; u < 4; ++u) {
+                const int b = b0 + u * CH_MERGE_WARPS;
+                if (b < blocks) p[u] = part[(size_t)b * C + c];
+            }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            if (b0 + u >= blocks) break;
-            s += p[u].s0;
-            sa += p[u].s1;
-            mn = fminf(mn, p[u].mn);
-            mx = fmaxf(mx, p[u].mx);
-            bad += p[u].bad;
+            for (int u = 0; u < 4; ++u) {
+                if (b0 + u * CH_MERGE_WARPS >= blocks) break;
+                s += p[u].s0;
+                sa += p[u].s1;
+                mn = fminf(mn, p[u].mn);
+                mx = fmaxf(mx, p[u].mx);
+                bad += p[u].bad;
+            }
         }
+    }
+    s_s[warp][lane] = s; s_sa[warp][lane] = sa; s_mn[warp][lane] = mn; s_mx[warp][lane] = mx; s_bad[warp][lane] = bad;
+    __syncthreads();
+    if (warp != 0 || c >= C) return;
+    for (int w = 1; w < CH_MERGE_WARPS; ++w) {
+        s += s_s[w][lane];
+        sa += s_sa[w][lane];
+        mn = fminf(mn, s_mn[w][lane]);
+        mx = fmaxf(mx, s_mx[w][lane]);
+        bad += s_bad[w][lane];
     }
     const unsigned long long nf = rows - bad;
     qp_stats_t st;
@@ -134,10 +155,10 @@ __global__ void __launch_bounds__(CH_THREADS) ch_merge_a(const ChPart* __restric
 }
 
 template <typename T, int V>
-__global__ void __launch_bounds__(CH_THREADS) ch_stats_b(const T* __restrict__ x, uint64_t rows, uint32_t C,
+__global__ void __launch_bounds__(CH_STATS_MAX_THREADS) ch_stats_b(const T* __restrict__ x, uint64_t rows, uint32_t C,
                                                          const qp_stats_t* __restrict__ st, ChPart* __restrict__ part)
 {
-    const uint32_t col0 = (blockIdx.y * CH_THREADS + threadIdx.x) * V;
+    const uint32_t col0 = (blockIdx.y * blockDim.x + threadIdx.x) * V;
     if (col0 >= C) return;
     float m_hi[V], m_lo[V];                               // each channel's mean as an unevaluated fp32 pair
     double sd[V], sv[V];
@@ -149,6 +170,7 @@ __global__ void __launch_bounds__(CH_THREADS) ch_stats_b(const T* __restrict__ x
         sd[i] = 0.0;
         sv[i] = 0.0;
     }
+    constexpr int CH_ROWS_IN_FLIGHT = ChRows<V>::N;
     const uint64_t step = gridDim.x;
     for (uint64_t r0 = blockIdx.x; r0 < rows; r0 += CH_ROWS_IN_FLIGHT * step) {
         float e[CH_ROWS_IN_FLIGHT][V];
@@ -186,23 +208,36 @@ __global__ void __launch_bounds__(CH_THREADS) ch_stats_b(const T* __restrict__ x
 __global__ void __launch_bounds__(CH_THREADS) ch_merge_b(const ChPart* __restrict__ part, int blocks, uint32_t C,
                                                          qp_stats_t* __restrict__ out)
 {
-    const uint32_t c = blockIdx.x * CH_THREADS + threadIdx.x;
-    if (c >= C) return;
+    __shared__ double s_d[CH_MERGE_WARPS][32], s_v[CH_MERGE_WARPS][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t c = blockIdx.x * 32 + lane;
     double sd = 0.0, sv = 0.0;
-    for (int b0 = 0; b0 < blocks; b0 += 8) {
-        double a[8], b[8];
+    if (c < C) {
+        for (int b0 = warp; b0 < blocks; b0 += 4 * CH_MERGE_WARPS) {
+            double a[4], b[4];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
-            if (b0 + u < blocks) {
-                a[u] = part[(size_t)(b0 + u) * C + c].s0;
-                b[u] = part[(size_t)(b0 + u) * C + c].s1;
+            for (int u = 0; u < 4; ++u) {
+                const int bb = b0 + u * CH_MERGE_WARPS;
+                if (bb < blocks) {
+                    a[u] = part[(size_t)bb * C + c].s0;
+                    b[u] = part[(size_t)bb * C + c].s1;
+                }
             }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            if (b0 + u >= blocks) break;
-            sd += a[u];
-            sv += b[u];
+            for (int u = 0; u < 4; ++u) {
+                if (b0 + u * CH_MERGE_WARPS >= blocks) break;
+                sd += a[u];
+                sv += b[u];
+            }
         }
+    }
+    s_d[warp][lane] = sd;
+    s_v[warp][lane] = sv;
+    __syncthreads();
+    if (warp != 0 || c >= C) return;
+    for (int w = 1; w < CH_MERGE_WARPS; ++w) {
+        sd += s_d[w][lane];
+        sv += s_v[w][lane];
     }
     const unsigned long long nf = out[c].n - out[c].nonfinite;
     out[c].mad = nf ? sd / (double)nf : 0.0;
@@ -224,20 +259,46 @@ __global__ void __launch_bounds__(128) ch_clip_kernel(const qp_stats_t* __restri
 }
 
 // ---- quantize + pack
+//
+// A warp owns a tile of 1024 consecutive elements (= 32 * bits output words) and never waits for
+// another warp: coalesced 16-byte loads (lane l takes vectors l, l + 32, ..., all issued first),
+// every element quantized with its channel's parameters from the table in shared memory, 16-bit
+// codes into the warp's own 32 x 17-word staging rows (row = 32 consecutive elements, one pad
+// word: conflict-free both ways), then lane l packs row l into `bits` words.
 
-// shared-memory word that holds the 16-bit codes of local elements le, le + 1 (le even)
+constexpr int CH_WARPS = CH_THREADS / 32;
+constexpr int CH_WTILE = 1024;                    // elements per warp tile
+constexpr int CH_STAGE_WORDS = 32 * 17;           // per warp
+
+// staging word that holds the codes of tile elements le, le + 1 (le even)
 __device__ __forceinline__ int ch_code_word(int le) { return (le >> 1) + (le >> 5); }
 
-__device__ __forceinline__ void ch_load_table(const qp_qparams_t* __restrict__ d_qp, uint32_t C, int bits, float4* tab,
-                                              unsigned* status)
+// Per-channel parameters in shared memory as four arrays [C] (lo, hi, scale, inv_scale): a lane
+// reads the parameters of its 4 consecutive channels as one 16-byte vector per array, and the
+// lanes of a warp read consecutive vectors (no bank conflicts).
+struct ChTable {
+    const float *lo, *hi, *scale, *inv;
+};
+__device__ __forceinline__ ChTable ch_load_table(const qp_qparams_t* __restrict__ d_qp, uint32_t C, int bits, float* tab,
+                                                 unsigned* status)
 {
     bool mismatch = false;
     for (uint32_t c = threadIdx.x; c < C; c += CH_THREADS) {
         const qp_qparams_t q = d_qp[c];
-        tab[c] = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
+        tab[c] = q.lo;
+        tab[C + c] = q.hi;
+        tab[2 * C + c] = q.scale;
+        tab[3 * C + c] = q.inv_scale;
         mismatch |= q.bits != bits;
     }
     if (mismatch && blockIdx.x == 0) atomicOr(status, QP_DEV_BITS_MISMATCH);
+    ChTable t = {tab, tab + C, tab + 2 * C, tab + 3 * C};
+    return t;
+}
+__device__ __forceinline__ void ch_lds4(const float* p, float (&v)[4])
+{
+    const float4 a = *reinterpret_cast<const float4*>(p);
+    v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
 }
 
 template <typename T, bool VEC>
@@ -247,69 +308,70 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
                                                              uint64_t ntiles, unsigned* __restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char raw[];
-    float4* tab = reinterpret_cast<float4*>(raw);                                  // [C] lo, hi, scale, inv_scale
-    uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)); // [CH_CODE_WORDS]
-    ch_load_table(d_qp, C, bits, tab, status);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)) + warp * CH_STAGE_WORDS;
+    const ChTable tab = ch_load_table(d_qp, C, bits, reinterpret_cast<float*>(raw), status);
     __syncthreads();
     constexpr int EPV = qp_span<T>::EPV;
+    constexpr int NV = CH_WTILE / (32 * EPV);                  // vectors per lane and tile: 8 (f32) or 4 (bf16)
     const unsigned mask = (1u << bits) - 1u;
-    const int tid = threadIdx.x;
-    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const uint64_t base = tile * CH_TILE;
+    const uint32_t cstep = (uint32_t)((32u * EPV) % C);        // channel advance from one of a lane's vectors to the next
+    const uint64_t wstride = (uint64_t)gridDim.x * CH_WARPS;
+    for (uint64_t tile = (uint64_t)blockIdx.x * CH_WARPS + warp; tile < ntiles; tile += wstride) {
+        const uint64_t base = tile * CH_WTILE;
         if (VEC) {
-            // thread takes vectors tid, tid + 256, ...: its channel advances by (256 * EPV) mod C each time
-            uint32_t c = (uint32_t)((base + (uint64_t)tid * EPV) % C);
-            const uint32_t cstep = (uint32_t)(((uint64_t)CH_THREADS * EPV) % C);
-            constexpr int NV = CH_TILE / (CH_THREADS * EPV);
+            float e[NV][EPV];
 #pragma unroll
-            for (int k0 = 0; k0 < NV; k0 += 4) {
-                float e[4][EPV];
+            for (int j = 0; j < NV; ++j) {
+                const uint64_t el = base + (uint64_t)(j * 32 + lane) * EPV;
+                if (el + EPV <= n) {
+                    qp_load_vec(x + el, e[j]);
+                } else {
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const uint64_t el = base + (uint64_t)((k0 + u) * CH_THREADS + tid) * EPV;
-                    if (el + EPV <= n) {
-                        qp_load_vec(x + el, e[u]);
-                    } else {
+                    for (int i = 0; i < EPV; ++i) e[j][i] = el + i < n ? qp_load_one(x + el + i) : 0.f;
+                }
+            }
+            uint32_t c = (uint32_t)((base + (uint64_t)lane * EPV) % C);
 #pragma unroll
-                        for (int i = 0; i < EPV; ++i) e[u][i] = el + i < n ? qp_load_one(x + el + i) : 0.f;
-                    }
+            for (int j = 0; j < NV; ++j) {
+                const int le = (j * 32 + lane) * EPV;
+                const uint64_t el = base + le;
+                unsigned cd[EPV];
+#pragma unroll
+                for (int h = 0; h < EPV; h += 4) {               // EPV divides C: the vector stays in one row
+                    float lo[4], hi[4], inv[4];
+                    ch_lds4(tab.lo + c + h, lo);
+                    ch_lds4(tab.hi + c + h, hi);
+                    ch_lds4(tab.inv + c + h, inv);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i)
+                        cd[h + i] = el + h + i < n ? qp_code(e[j][h + i], lo[i], hi[i], inv[i], mask) : 0u;
                 }
 #pragma unroll
-                for (int u = 0; u < 4; ++u) {
-                    const int le = ((k0 + u) * CH_THREADS + tid) * EPV;
-                    const uint64_t el = base + le;
-                    unsigned cd[EPV];
-#pragma unroll
-                    for (int i = 0; i < EPV; ++i) {
-                        const float4 q = tab[c + i];             // EPV divides C: the vector stays in one row
-                        cd[i] = el + i < n ? qp_code(e[u][i], q.x, q.y, q.w, mask) : 0u;
-                    }
-#pragma unroll
-                    for (int i = 0; i < EPV; i += 2) codes[ch_code_word(le + i)] = cd[i] | (cd[i + 1] << 16);
-                    c += cstep;
-                    if (c >= C) c -= C;
-                }
+                for (int i = 0; i < EPV; i += 2) codes[ch_code_word(le + i)] = cd[i] | (cd[i + 1] << 16);
+                c += cstep;
+                if (c >= C) c -= C;
             }
         } else {
             unsigned short* ch = reinterpret_cast<unsigned short*>(codes);
             for (int k = 0; k < 32; ++k) {
-                const int le = k * CH_THREADS + tid;
+                const int le = k * 32 + lane;
                 const uint64_t el = base + le;
                 unsigned cd = 0u;
                 if (el < n) {
-                    const float4 q = tab[el % C];
-                    cd = qp_code(qp_load_one(x + el), q.x, q.y, q.w, mask);
+                    const uint32_t c = (uint32_t)(el % C);
+                    cd = qp_code(qp_load_one(x + el), tab.lo[c], tab.hi[c], tab.inv[c], mask);
                 }
                 ch[le + ((le >> 5) << 1)] = (unsigned short)cd;
             }
         }
-        __syncthreads();
+        __syncwarp();
         {
-            const uint64_t w0 = (tile * CH_THREADS + tid) * (uint64_t)bits;   // this thread's group of 32 elements
+            const uint64_t w0 = (tile * 32 + lane) * (uint64_t)bits;          // this lane's group of 32 elements
             if (w0 < total_words) {
                 uint32_t w[16];
 #pragma unroll
-                for (int j = 0; j < 16; ++j) w[j] = codes[17 * tid + j];
+                for (int j = 0; j < 16; ++j) w[j] = codes[17 * lane + j];
                 unsigned long long acc = 0ull;
                 int fill = 0;
                 uint32_t* dst = out + w0;
@@ -328,11 +390,11 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
                 }
             }
         }
-        __syncthreads();
+        __syncwarp();
     }
 }
 
-// ---- unpack + dequantize
+// ---- unpack + dequantize (mirror image)
 
 __device__ __forceinline__ float ch_code_to_float(unsigned c) { return __fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.0f); }
 
@@ -357,17 +419,18 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
                                                                unsigned* __restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char raw[];
-    float4* tab = reinterpret_cast<float4*>(raw);
-    uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4));
-    ch_load_table(d_qp, C, bits, tab, status);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)) + warp * CH_STAGE_WORDS;
+    const ChTable tab = ch_load_table(d_qp, C, bits, reinterpret_cast<float*>(raw), status);
     __syncthreads();
     const unsigned mask = (1u << bits) - 1u;
-    const int tid = threadIdx.x;
-    for (uint64_t tile = blockIdx.x; tile < ntiles; tile += gridDim.x) {
-        const uint64_t base = tile * CH_TILE;
+    const uint32_t cstep = (uint32_t)(128u % C);               // a lane's vectors of 4 are 128 elements apart
+    const uint64_t wstride = (uint64_t)gridDim.x * CH_WARPS;
+    for (uint64_t tile = (uint64_t)blockIdx.x * CH_WARPS + warp; tile < ntiles; tile += wstride) {
+        const uint64_t base = tile * CH_WTILE;
         {
-            // this thread's group of 32 elements: `bits` words -> 32 codes -> 16 shared-memory words
-            const uint64_t w0 = (tile * CH_THREADS + tid) * (uint64_t)bits;
+            // this lane's group of 32 elements: `bits` words -> 32 codes -> its staging row
+            const uint64_t w0 = (tile * 32 + lane) * (uint64_t)bits;
             uint32_t w[16];
 #pragma unroll
             for (int m = 0; m < 16; ++m) w[m] = (m < bits && w0 + m < total_words) ? __ldg(in + w0 + m) : 0u;
@@ -383,29 +446,27 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
                         const unsigned cd = (unsigned)acc & mask;
                         acc >>= bits;
                         have -= bits;
-                        if (i & 1) codes[17 * tid + (i >> 1)] = prev | (cd << 16);
+                        if (i & 1) codes[17 * lane + (i >> 1)] = prev | (cd << 16);
                         else       prev = cd;
                         ++i;
                     }
                 }
             }
         }
-        __syncthreads();
+        __syncwarp();
         if (VEC) {
-            uint32_t c = (uint32_t)((base + (uint64_t)tid * 4) % C);
-            const uint32_t cstep = (uint32_t)(((uint64_t)CH_THREADS * 4) % C);
+            uint32_t c = (uint32_t)((base + (uint64_t)lane * 4) % C);
 #pragma unroll
-            for (int k = 0; k < CH_TILE / (CH_THREADS * 4); ++k) {
-                const int le = (k * CH_THREADS + tid) * 4;
+            for (int j = 0; j < CH_WTILE / 128; ++j) {
+                const int le = (j * 32 + lane) * 4;
                 const uint64_t el = base + le;
                 const uint32_t a = codes[ch_code_word(le)], b = codes[ch_code_word(le + 2)];
                 const unsigned cd[4] = {a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16};
-                float v[4];
+                float v[4], lo[4], sc[4];
+                ch_lds4(tab.lo + c, lo);
+                ch_lds4(tab.scale + c, sc);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const float4 q = tab[c + i];
-                    v[i] = fmaf(ch_code_to_float(cd[i]), q.z, q.x);
-                }
+                for (int i = 0; i < 4; ++i) v[i] = fmaf(ch_code_to_float(cd[i]), sc[i], lo[i]);
                 if (el + 4 <= n) {
                     ch_store4(y, el, v);
                 } else {
@@ -419,15 +480,15 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
         } else {
             const unsigned short* ch = reinterpret_cast<const unsigned short*>(codes);
             for (int k = 0; k < 32; ++k) {
-                const int le = k * CH_THREADS + tid;
+                const int le = k * 32 + lane;
                 const uint64_t el = base + le;
                 if (el < n) {
-                    const float4 q = tab[el % C];
-                    ch_store1(y, el, fmaf(ch_code_to_float(ch[le + ((le >> 5) << 1)]), q.z, q.x));
+                    const uint32_t c = (uint32_t)(el % C);
+                    ch_store1(y, el, fmaf(ch_code_to_float(ch[le + ((le >> 5) << 1)]), tab.scale[c], tab.lo[c]));
                 }
             }
         }
-        __syncthreads();
+        __syncwarp();
     }
 }
 
@@ -461,29 +522,33 @@ int32_t stats_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C,
     constexpr int EPV = qp_span<T>::EPV;
     const bool vec = (C % EPV == 0) && (((uintptr_t)x & 15u) == 0);
     const int V = vec ? EPV : 1;
-    const unsigned col_blocks = (C / V + CH_THREADS - 1) / CH_THREADS;
-    // enough row blocks to fill the GPU a few times over, no more than there are rows
-    // about two blocks per SM in all: 8 x 16-byte loads in flight per thread keep HBM busy, and
-    // the partials (32 bytes per row block and channel) stay a few percent of the tensor
-    uint64_t want = (uint64_t)ctx->sm_count * 2 / col_blocks;
-    if (want < (uint64_t)ctx->sm_count) want = ctx->sm_count;
+    // one thread per group of V channels; a block spans all of them where 512 threads suffice
+    const unsigned groups = C / V;
+    unsigned threads = (groups + 31) / 32 * 32;
+    if (threads > CH_STATS_MAX_THREADS) threads = CH_STATS_MAX_THREADS;
+    const unsigned col_blocks = (groups + threads - 1) / threads;
+    // about 640 threads per SM in all: 8 x 16-byte loads in flight per thread keep HBM busy, and the
+    // partials (32 bytes per row block and channel) stay a few percent of the tensor
+    uint64_t want = (uint64_t)ctx->sm_count * 640 / ((uint64_t)threads * col_blocks);
+    if (want < 1) want = 1;
+    if (want > 1024) want = 1024;
     const int row_blocks = (int)(rows < want ? rows : want);
     int32_t rc = ch_scratch(ctx, sizeof(ChPart) * (size_t)row_blocks * C);
     if (rc) return rc;
     ChPart* part = static_cast<ChPart*>(ctx->d_ch_part);
     const dim3 grid(row_blocks, col_blocks);
-    const unsigned merge_blocks = (C + CH_THREADS - 1) / CH_THREADS;
-    if (vec) ch_stats_a<T, EPV><<<grid, CH_THREADS, 0, s>>>(x, rows, C, part);
-    else     ch_stats_a<T, 1><<<grid, CH_THREADS, 0, s>>>(x, rows, C, part);
+    const unsigned merge_blocks = (C + 31) / 32;
+    if (vec) ch_stats_a<T, EPV><<<grid, threads, 0, s>>>(x, rows, C, part);
+    else     ch_stats_a<T, 1><<<grid, threads, 0, s>>>(x, rows, C, part);
     ch_merge_a<<<merge_blocks, CH_THREADS, 0, s>>>(part, row_blocks, rows, C, d_out, ctx->d_status);
-    if (vec) ch_stats_b<T, EPV><<<grid, CH_THREADS, 0, s>>>(x, rows, C, d_out, part);
-    else     ch_stats_b<T, 1><<<grid, CH_THREADS, 0, s>>>(x, rows, C, d_out, part);
+    if (vec) ch_stats_b<T, EPV><<<grid, threads, 0, s>>>(x, rows, C, d_out, part);
+    else     ch_stats_b<T, 1><<<grid, threads, 0, s>>>(x, rows, C, d_out, part);
     ch_merge_b<<<merge_blocks, CH_THREADS, 0, s>>>(part, row_blocks, C, d_out);
     ctx->launches += 4;
     return qp_check_launch(ctx, "qp_stats_channels");
 }
 
-size_t ch_pack_smem(uint32_t C) { return (size_t)C * sizeof(float4) + (size_t)CH_CODE_WORDS * sizeof(uint32_t); }
+size_t ch_pack_smem(uint32_t C) { return (size_t)C * sizeof(float4) + (size_t)CH_WARPS * CH_STAGE_WORDS * sizeof(uint32_t); }
 
 template <typename K>
 bool ch_allow_smem(K kernel, size_t bytes)
@@ -556,9 +621,10 @@ extern "C" int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int d
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint64_t total_words = need / 4;
     const uint64_t groups = (total_words + bits - 1) / bits;
-    const uint64_t ntiles = (groups + CH_THREADS - 1) / CH_THREADS;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 4;
-    const unsigned blocks = (unsigned)(ntiles < cap ? ntiles : cap);
+    const uint64_t ntiles = (groups + 31) / 32;                               // warp tiles, pad words included
+    const uint64_t want = (ntiles + CH_WARPS - 1) / CH_WARPS;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
+    const unsigned blocks = (unsigned)(want < cap ? want : cap);
     const size_t smem = ch_pack_smem(channels);
     uint32_t* out = static_cast<uint32_t*>(d_packed);
     bool ok;
@@ -604,9 +670,10 @@ extern "C" int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_pack
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const uint64_t total_words = qp_packed_bytes(n, bits) / 4;
-    const uint64_t ntiles = (n + CH_TILE - 1) / CH_TILE;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 4;
-    const unsigned blocks = (unsigned)(ntiles < cap ? ntiles : cap);
+    const uint64_t ntiles = (n + CH_WTILE - 1) / CH_WTILE;
+    const uint64_t want = (ntiles + CH_WARPS - 1) / CH_WARPS;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
+    const unsigned blocks = (unsigned)(want < cap ? want : cap);
     const size_t smem = ch_pack_smem(channels);
     const uint32_t* in = static_cast<const uint32_t*>(d_packed);
     bool ok;
