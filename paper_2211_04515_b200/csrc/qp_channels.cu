@@ -301,14 +301,16 @@ __device__ __forceinline__ void ch_lds4(const float* p, float (&v)[4])
     v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
 }
 
-template <typename T, bool VEC>
-__global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict__ x, uint64_t n, uint32_t C, int bits,
+// BITS > 0: the bit-width as a compile-time constant (shifts become immediates); 0: `bits_rt`.
+template <typename T, bool VEC, int BITS>
+__global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict__ x, uint64_t n, uint32_t C, int bits_rt,
                                                              const qp_qparams_t* __restrict__ d_qp,
                                                              uint32_t* __restrict__ out, uint64_t total_words,
                                                              uint64_t ntiles, unsigned* __restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int bits = BITS ? BITS : bits_rt;
     uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)) + warp * CH_STAGE_WORDS;
     const ChTable tab = ch_load_table(d_qp, C, bits, reinterpret_cast<float*>(raw), status);
     __syncthreads();
@@ -320,11 +322,12 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
     for (uint64_t tile = (uint64_t)blockIdx.x * CH_WARPS + warp; tile < ntiles; tile += wstride) {
         const uint64_t base = tile * CH_WTILE;
         if (VEC) {
+            const bool full = base + CH_WTILE <= n;              // no element of the tile lies beyond the tensor
             float e[NV][EPV];
 #pragma unroll
             for (int j = 0; j < NV; ++j) {
                 const uint64_t el = base + (uint64_t)(j * 32 + lane) * EPV;
-                if (el + EPV <= n) {
+                if (full || el + EPV <= n) {
                     qp_load_vec(x + el, e[j]);
                 } else {
 #pragma unroll
@@ -344,8 +347,11 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
                     ch_lds4(tab.hi + c + h, hi);
                     ch_lds4(tab.inv + c + h, inv);
 #pragma unroll
-                    for (int i = 0; i < 4; ++i)
-                        cd[h + i] = el + h + i < n ? qp_code(e[j][h + i], lo[i], hi[i], inv[i], mask) : 0u;
+                    for (int i = 0; i < 4; ++i) cd[h + i] = qp_code(e[j][h + i], lo[i], hi[i], inv[i], mask);
+                }
+                if (!full) {
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) cd[i] = el + i < n ? cd[i] : 0u;
                 }
 #pragma unroll
                 for (int i = 0; i < EPV; i += 2) codes[ch_code_word(le + i)] = cd[i] | (cd[i + 1] << 16);
@@ -412,14 +418,15 @@ __device__ __forceinline__ void ch_store4(unsigned short* y, uint64_t el, const 
 __device__ __forceinline__ void ch_store1(float* y, uint64_t el, float v) { y[el] = v; }
 __device__ __forceinline__ void ch_store1(unsigned short* y, uint64_t el, float v) { y[el] = qp_f32_to_bf16(v); }
 
-template <typename TO, bool VEC>
+template <typename TO, bool VEC, int BITS>
 __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* __restrict__ in, uint64_t n, uint32_t C,
-                                                               int bits, const qp_qparams_t* __restrict__ d_qp,
+                                                               int bits_rt, const qp_qparams_t* __restrict__ d_qp,
                                                                TO* __restrict__ y, uint64_t total_words, uint64_t ntiles,
                                                                unsigned* __restrict__ status)
 {
     extern __shared__ __align__(16) unsigned char raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int bits = BITS ? BITS : bits_rt;
     uint32_t* codes = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)) + warp * CH_STAGE_WORDS;
     const ChTable tab = ch_load_table(d_qp, C, bits, reinterpret_cast<float*>(raw), status);
     __syncthreads();
@@ -434,21 +441,36 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
             uint32_t w[16];
 #pragma unroll
             for (int m = 0; m < 16; ++m) w[m] = (m < bits && w0 + m < total_words) ? __ldg(in + w0 + m) : 0u;
-            unsigned long long acc = 0ull;                     // bits not yet consumed, oldest lowest
-            int have = 0, i = 0;
-            unsigned prev = 0u;
+            if (BITS) {
 #pragma unroll
-            for (int m = 0; m < 16; ++m) {
-                if (m < bits) {
-                    acc |= (unsigned long long)w[m] << have;
-                    have += 32;
-                    while (have >= bits) {
-                        const unsigned cd = (unsigned)acc & mask;
-                        acc >>= bits;
-                        have -= bits;
-                        if (i & 1) codes[17 * lane + (i >> 1)] = prev | (cd << 16);
-                        else       prev = cd;
-                        ++i;
+                for (int i = 0; i < 32; i += 2) {              // positions known at compile time
+                    unsigned two[2];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const int bit = (i + h) * (BITS ? BITS : 1), word = bit >> 5, sh = bit & 31;
+                        unsigned cd = w[word] >> sh;
+                        if (sh + (BITS ? BITS : 1) > 32) cd |= w[(word + 1) & 15] << (32 - sh);
+                        two[h] = cd & mask;
+                    }
+                    codes[17 * lane + (i >> 1)] = two[0] | (two[1] << 16);
+                }
+            } else {
+                unsigned long long acc = 0ull;                 // bits not yet consumed, oldest lowest
+                int have = 0, i = 0;
+                unsigned prev = 0u;
+#pragma unroll
+                for (int m = 0; m < 16; ++m) {
+                    if (m < bits) {
+                        acc |= (unsigned long long)w[m] << have;
+                        have += 32;
+                        while (have >= bits) {
+                            const unsigned cd = (unsigned)acc & mask;
+                            acc >>= bits;
+                            have -= bits;
+                            if (i & 1) codes[17 * lane + (i >> 1)] = prev | (cd << 16);
+                            else       prev = cd;
+                            ++i;
+                        }
                     }
                 }
             }
@@ -627,26 +649,36 @@ extern "C" int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int d
     const unsigned blocks = (unsigned)(want < cap ? want : cap);
     const size_t smem = ch_pack_smem(channels);
     uint32_t* out = static_cast<uint32_t*>(d_packed);
-    bool ok;
+    bool ok = false;
+#define QP_CH_PACK(T, VEC, B)                                                                                          \
+    do {                                                                                                               \
+        ok = ch_allow_smem(ch_pack_kernel<T, VEC, B>, smem);                                                           \
+        if (ok) ch_pack_kernel<T, VEC, B><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out,           \
+                                                                          total_words, ntiles, ctx->d_status);        \
+    } while (0)
+#define QP_CH_PACK_BITS(T)                                                                                             \
+    switch (bits) {                                                                                                    \
+        case 1: QP_CH_PACK(T, true, 1); break;                                                                         \
+        case 2: QP_CH_PACK(T, true, 2); break;                                                                         \
+        case 3: QP_CH_PACK(T, true, 3); break;                                                                         \
+        case 4: QP_CH_PACK(T, true, 4); break;                                                                         \
+        case 5: QP_CH_PACK(T, true, 5); break;                                                                         \
+        case 6: QP_CH_PACK(T, true, 6); break;                                                                         \
+        case 7: QP_CH_PACK(T, true, 7); break;                                                                         \
+        case 8: QP_CH_PACK(T, true, 8); break;                                                                         \
+        default: QP_CH_PACK(T, true, 16); break;                                                                       \
+    }
     if (dtype == QP_F32) {
         const float* x = static_cast<const float*>(d_x);
-        if (channels % 4 == 0 && ((uintptr_t)x & 15u) == 0) {
-            ok = ch_allow_smem(ch_pack_kernel<float, true>, smem);
-            if (ok) ch_pack_kernel<float, true><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
-        } else {
-            ok = ch_allow_smem(ch_pack_kernel<float, false>, smem);
-            if (ok) ch_pack_kernel<float, false><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
-        }
+        if (channels % 4 == 0 && ((uintptr_t)x & 15u) == 0) { QP_CH_PACK_BITS(float) }
+        else QP_CH_PACK(float, false, 0);
     } else {
         const unsigned short* x = static_cast<const unsigned short*>(d_x);
-        if (channels % 8 == 0 && ((uintptr_t)x & 15u) == 0) {
-            ok = ch_allow_smem(ch_pack_kernel<unsigned short, true>, smem);
-            if (ok) ch_pack_kernel<unsigned short, true><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
-        } else {
-            ok = ch_allow_smem(ch_pack_kernel<unsigned short, false>, smem);
-            if (ok) ch_pack_kernel<unsigned short, false><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out, total_words, ntiles, ctx->d_status);
-        }
+        if (channels % 8 == 0 && ((uintptr_t)x & 15u) == 0) { QP_CH_PACK_BITS(unsigned short) }
+        else QP_CH_PACK(unsigned short, false, 0);
     }
+#undef QP_CH_PACK_BITS
+#undef QP_CH_PACK
     if (!ok) return qp_check_launch(ctx, "qp_quantize_pack_channels (shared memory)");
     ctx->launches += 1;
     return qp_check_launch(ctx, "qp_quantize_pack_channels");
@@ -676,26 +708,36 @@ extern "C" int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_pack
     const unsigned blocks = (unsigned)(want < cap ? want : cap);
     const size_t smem = ch_pack_smem(channels);
     const uint32_t* in = static_cast<const uint32_t*>(d_packed);
-    bool ok;
+    bool ok = false;
+#define QP_CH_UNPACK(T, VEC, B)                                                                                        \
+    do {                                                                                                               \
+        ok = ch_allow_smem(ch_unpack_kernel<T, VEC, B>, smem);                                                         \
+        if (ok) ch_unpack_kernel<T, VEC, B><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y,          \
+                                                                            total_words, ntiles, ctx->d_status);      \
+    } while (0)
+#define QP_CH_UNPACK_BITS(T)                                                                                           \
+    switch (bits) {                                                                                                    \
+        case 1: QP_CH_UNPACK(T, true, 1); break;                                                                       \
+        case 2: QP_CH_UNPACK(T, true, 2); break;                                                                       \
+        case 3: QP_CH_UNPACK(T, true, 3); break;                                                                       \
+        case 4: QP_CH_UNPACK(T, true, 4); break;                                                                       \
+        case 5: QP_CH_UNPACK(T, true, 5); break;                                                                       \
+        case 6: QP_CH_UNPACK(T, true, 6); break;                                                                       \
+        case 7: QP_CH_UNPACK(T, true, 7); break;                                                                       \
+        case 8: QP_CH_UNPACK(T, true, 8); break;                                                                       \
+        default: QP_CH_UNPACK(T, true, 16); break;                                                                     \
+    }
     if (out_dtype == QP_F32) {
         float* y = static_cast<float*>(d_y);
-        if (channels % 4 == 0 && ((uintptr_t)y & 15u) == 0) {
-            ok = ch_allow_smem(ch_unpack_kernel<float, true>, smem);
-            if (ok) ch_unpack_kernel<float, true><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
-        } else {
-            ok = ch_allow_smem(ch_unpack_kernel<float, false>, smem);
-            if (ok) ch_unpack_kernel<float, false><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
-        }
+        if (channels % 4 == 0 && ((uintptr_t)y & 15u) == 0) { QP_CH_UNPACK_BITS(float) }
+        else QP_CH_UNPACK(float, false, 0);
     } else {
         unsigned short* y = static_cast<unsigned short*>(d_y);
-        if (channels % 4 == 0 && ((uintptr_t)y & 7u) == 0) {
-            ok = ch_allow_smem(ch_unpack_kernel<unsigned short, true>, smem);
-            if (ok) ch_unpack_kernel<unsigned short, true><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
-        } else {
-            ok = ch_allow_smem(ch_unpack_kernel<unsigned short, false>, smem);
-            if (ok) ch_unpack_kernel<unsigned short, false><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y, total_words, ntiles, ctx->d_status);
-        }
+        if (channels % 4 == 0 && ((uintptr_t)y & 7u) == 0) { QP_CH_UNPACK_BITS(unsigned short) }
+        else QP_CH_UNPACK(unsigned short, false, 0);
     }
+#undef QP_CH_UNPACK_BITS
+#undef QP_CH_UNPACK
     if (!ok) return qp_check_launch(ctx, "qp_unpack_dequantize_channels (shared memory)");
     ctx->launches += 1;
     return qp_check_launch(ctx, "qp_unpack_dequantize_channels");
