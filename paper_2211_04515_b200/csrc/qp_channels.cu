@@ -92,10 +92,11 @@ __global__ void __launch_bounds__(CH_STATS_MAX_THREADS) ch_stats_a(const T* __re
 }
 
 // Merge of the row blocks' partials: a block takes 32 channels (lane = channel, so a warp reads
-// 1 KB rows of partials), warp w adds row blocks w, w + 8, ... in order with four loads in
-// flight, and the eight warp sums are combined in warp order: the same bits on every run.
-constexpr int CH_MERGE_WARPS = CH_THREADS / 32;
-__global__ void __launch_bounds__(CH_THREADS) ch_merge_a(const ChPart* __restrict__ part, int blocks, uint64_t rows,
+// 1 KB rows of partials), warp w adds row blocks w, w + 32, ... in order with four loads in
+// flight, and the 32 warp sums are combined in warp order: the same bits on every run.
+constexpr int CH_MERGE_THREADS = 1024;
+constexpr int CH_MERGE_WARPS = CH_MERGE_THREADS / 32;
+__global__ void __launch_bounds__(CH_MERGE_THREADS) ch_merge_a(const ChPart* __restrict__ part, int blocks, uint64_t rows,
                                                          uint32_t C, qp_stats_t* __restrict__ out,
                                                          unsigned* __restrict__ status)
 {
@@ -205,7 +206,7 @@ __global__ void __launch_bounds__(CH_STATS_MAX_THREADS) ch_stats_b(const T* __re
     }
 }
 
-__global__ void __launch_bounds__(CH_THREADS) ch_merge_b(const ChPart* __restrict__ part, int blocks, uint32_t C,
+__global__ void __launch_bounds__(CH_MERGE_THREADS) ch_merge_b(const ChPart* __restrict__ part, int blocks, uint32_t C,
                                                          qp_stats_t* __restrict__ out)
 {
     __shared__ double s_d[CH_MERGE_WARPS][32], s_v[CH_MERGE_WARPS][32];
@@ -562,10 +563,10 @@ int32_t stats_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C,
     const unsigned merge_blocks = (C + 31) / 32;
     if (vec) ch_stats_a<T, EPV><<<grid, threads, 0, s>>>(x, rows, C, part);
     else     ch_stats_a<T, 1><<<grid, threads, 0, s>>>(x, rows, C, part);
-    ch_merge_a<<<merge_blocks, CH_THREADS, 0, s>>>(part, row_blocks, rows, C, d_out, ctx->d_status);
+    ch_merge_a<<<merge_blocks, CH_MERGE_THREADS, 0, s>>>(part, row_blocks, rows, C, d_out, ctx->d_status);
     if (vec) ch_stats_b<T, EPV><<<grid, threads, 0, s>>>(x, rows, C, d_out, part);
     else     ch_stats_b<T, 1><<<grid, threads, 0, s>>>(x, rows, C, d_out, part);
-    ch_merge_b<<<merge_blocks, CH_THREADS, 0, s>>>(part, row_blocks, C, d_out);
+    ch_merge_b<<<merge_blocks, CH_MERGE_THREADS, 0, s>>>(part, row_blocks, C, d_out);
     ctx->launches += 4;
     return qp_check_launch(ctx, "qp_stats_channels");
 }
