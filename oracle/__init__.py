@@ -102,6 +102,8 @@ def lib():
         L.orc_quantize_channels.restype = None
         L.orc_dequantize_channels.argtypes = [u32p, C.c_uint64, C.c_uint64, C.POINTER(QParams), fp]
         L.orc_dequantize_channels.restype = None
+        L.orc_midrise_range.argtypes = [C.c_double, C.c_double, C.c_int, dp, dp]
+        L.orc_midrise_range.restype = None
         L.orc_hist_peak.argtypes = [fp, C.c_uint64, C.c_double, C.c_double, C.c_int, u64p]
         L.orc_hist_peak.restype = C.c_double
         L.orc_ds_search.argtypes = [fp, C.c_uint64, C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int,
@@ -162,13 +164,23 @@ def aciq_alpha(st: Stats, bits: int, dist: int = 0, bmode: int = 0, b_override: 
 CLIP_ACIQ, CLIP_MINMAX = 0, 2
 
 
-def clip_range(st: Stats, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0):
+B_MIDRISE = 0x10          # ds_search: bmode | B_MIDRISE scores every candidate on the mid-rise grid
+
+
+def clip_range(st: Stats, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0,
+               midrise: bool = False):
     """(rc, lo, hi, quantizer) of the clip range by method: ACIQ, or naive PTQ's [min, max]."""
     lo, hi = C.c_double(), C.c_double()
     qp = QParams()
-    rc = lib().orc_clip_range(C.byref(st), bits, method, 1 if intersect else 0, dist, bmode, C.byref(lo), C.byref(hi),
-                              C.byref(qp))
+    rc = lib().orc_clip_range(C.byref(st), bits, method, (1 if intersect else 0) | (2 if midrise else 0), dist, bmode,
+                              C.byref(lo), C.byref(hi), C.byref(qp))
     return rc, lo.value, hi.value, qp
+
+
+def midrise_range(lo: float, hi: float, bits: int):
+    a, b = C.c_double(), C.c_double()
+    lib().orc_midrise_range(lo, hi, bits, C.byref(a), C.byref(b))
+    return a.value, b.value
 
 
 def quantize(x, qp: QParams) -> np.ndarray:
@@ -220,11 +232,12 @@ def stats_channels(x, channels: int):
     return out
 
 
-def clip_channels(st, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0):
+def clip_channels(st, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0,
+                  midrise: bool = False):
     """(rc, ctypes array of per-channel QParams) from per-channel statistics."""
     channels = len(st)
     qp = (QParams * channels)()
-    rc = lib().orc_clip_channels(st, channels, bits, method, 1 if intersect else 0, dist, bmode, qp)
+    rc = lib().orc_clip_channels(st, channels, bits, method, (1 if intersect else 0) | (2 if midrise else 0), dist, bmode, qp)
     return rc, qp
 
 

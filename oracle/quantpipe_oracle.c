@@ -241,7 +241,7 @@ double orc_quant_mse(const float* x, uint64_t n, const orc_qparams_t* qp)
 
 /* ------------------------------------------------- per-channel quantization */
 
-int orc_clip_range(const orc_stats_t* st, int bits, int method, int intersect, int dist, int bmode,
+int orc_clip_range(const orc_stats_t* st, int bits, int method, int flags, int dist, int bmode,
                    double* lo_out, double* hi_out, orc_qparams_t* qp);   /* defined with the ACIQ clip below */
 
 /* Channel-wise variant of the per-tensor method (Sec. 3 applies one clip range to the whole
@@ -267,12 +267,12 @@ int orc_stats_channels(const float* x, uint64_t rows, uint64_t channels, orc_sta
 
 /* Quantizer of each channel from its statistics (orc_clip_range per channel).  Returns
  * ORC_WARN_DEGENERATE if any channel has an empty range (that channel's codes are all 0). */
-int orc_clip_channels(const orc_stats_t* st, uint64_t channels, int bits, int method, int intersect, int dist,
+int orc_clip_channels(const orc_stats_t* st, uint64_t channels, int bits, int method, int flags, int dist,
                       int bmode, orc_qparams_t* qp)
 {
     int worst = ORC_OK;
     for (uint64_t c = 0; c < channels; ++c) {
-        int rc = orc_clip_range(&st[c], bits, method, intersect, dist, bmode, NULL, NULL, &qp[c]);
+        int rc = orc_clip_range(&st[c], bits, method, flags, dist, bmode, NULL, NULL, &qp[c]);
         if (rc < 0) return rc;
         if (rc == ORC_WARN_DEGENERATE) worst = rc;
     }
@@ -344,19 +344,33 @@ int orc_aciq_alpha(const orc_stats_t* st, int bits, int dist, int bmode, double 
     return ORC_OK;
 }
 
+/* Mid-rise grid on a clip range (the other reading of Sec. 3's "divides the data range into
+ * equal intervals": 2^q equal bins over [lo, hi], every element reconstructed at the centre of
+ * its bin - the grid that the ACIQ noise term alpha^2 / (3 * 4^q) models).  With bin width
+ * w = (hi - lo) / 2^q the centres are lo + w/2, lo + 3w/2, ..., hi - w/2: exactly the 2^q levels
+ * of the uniform quantizer on [lo + w/2, hi - w/2], whose rounding boundaries are the bin
+ * edges.  So the grid is a change of the clip range and nothing else. */
+void orc_midrise_range(double lo, double hi, int bits, double* lo_out, double* hi_out)
+{
+    double half = (hi - lo) / ldexp(1.0, bits + 1);
+    *lo_out = lo + half;
+    *hi_out = hi - half;
+}
+
 /* Clip range by method (Sec. 3, "Naive PTQ and ACIQ").
  *   method 0  ACIQ: [mean - alpha, mean + alpha] with alpha = F(q) b, as orc_aciq_alpha
  *   method 2  naive PTQ: the tensor's own [min, max]
- * intersect != 0 (method 0 only): the ACIQ range cut back to the data's range,
+ * flags bit 0 (method 0 only): the ACIQ range cut back to the data's range,
  *   [max(mean - alpha, min), min(mean + alpha, max)].  No element lies outside [min, max], so
  *   the clipping error is unchanged while the step gets smaller whenever alpha reaches past
- *   the data.  This is a variant of this library; the paper clips at mean -/+ alpha only. */
-int orc_clip_range(const orc_stats_t* st, int bits, int method, int intersect, int dist, int bmode,
+ *   the data.  This is a variant of this library; the paper clips at mean -/+ alpha only.
+ * flags bit 1: mid-rise grid on the resulting range (orc_midrise_range), applied last. */
+int orc_clip_range(const orc_stats_t* st, int bits, int method, int flags, int dist, int bmode,
                    double* lo_out, double* hi_out, orc_qparams_t* qp)
 {
     if (!bits_ok(bits)) return ORC_ERR_BITS;
     if (method != 0 && method != 2) return ORC_ERR_ARG;
-    if (method == 2 && intersect) return ORC_ERR_ARG;
+    if (flags < 0 || flags > 3 || (method == 2 && (flags & 1))) return ORC_ERR_ARG;
     double lo, hi;
     if (method == 2) {
         lo = st->min;
@@ -367,11 +381,12 @@ int orc_clip_range(const orc_stats_t* st, int bits, int method, int intersect, i
         if (rc < 0) return rc;
         lo = st->mean - alpha;
         hi = st->mean + alpha;
-        if (intersect) {
+        if (flags & 1) {
             if (st->min > lo) lo = st->min;
             if (st->max < hi) hi = st->max;
         }
     }
+    if (flags & 2) orc_midrise_range(lo, hi, bits, &lo, &hi);
     if (lo_out) *lo_out = lo;
     if (hi_out) *hi_out = hi;
     if (qp) return orc_make_qparams(lo, hi, bits, qp);
@@ -419,6 +434,7 @@ double orc_hist_peak(const float* x, uint64_t n, double mn, double mx, int nb, u
  *   b_R      = 1 / (2 max(D_R)), D_R the histogram density of the data
  *   b_k      = b_E + k (b_R - b_E) / t,  k = 0..t   (towards b_R, whichever side it lies)
  *   mse_k    = quantization MSE of the tensor with clip alpha_k = F(q) b_k about the mean
+ *              (bmode | 0x10: on the mid-rise grid, orc_midrise_range)
  *   k*       = smallest k attaining the minimum; k = 0 is b_E itself, so b_E is kept
  *              unless some step is strictly better.
  * mse_curve (t+1 doubles) optional. */
@@ -427,6 +443,8 @@ int orc_ds_search(const float* x, uint64_t n, const orc_stats_t* st, int bits, i
                   double* mse_curve)
 {
     if (!(bits >= 1 && bits <= 8)) return ORC_ERR_BITS;
+    int midrise = (bmode & 0x10) != 0;                     /* every candidate on the mid-rise grid */
+    bmode &= ~0x10;
     if (steps < 1 || hist_bins < 1 || (bmode != 0 && bmode != 1)) return ORC_ERR_ARG;
     double F = orc_aciq_F_laplace(bits);
     double b_e = bmode == 1 ? st->mean_abs : st->mad;
@@ -449,7 +467,9 @@ int orc_ds_search(const float* x, uint64_t n, const orc_stats_t* st, int bits, i
             mse = INFINITY;                                  /* not a candidate */
         } else {
             double alpha = F * b_k;
-            orc_make_qparams(st->mean - alpha, st->mean + alpha, bits, &qp);
+            double lo = st->mean - alpha, hi = st->mean + alpha;
+            if (midrise) orc_midrise_range(lo, hi, bits, &lo, &hi);
+            orc_make_qparams(lo, hi, bits, &qp);
             mse = orc_quant_mse(x, n, &qp);
         }
         if (mse_curve) mse_curve[k] = mse;
