@@ -52,6 +52,7 @@ enum {
 enum { QP_F32 = 0, QP_BF16 = 1 };
 enum { QP_DIST_LAPLACE = 0, QP_DIST_GAUSS = 1 };
 enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the formula as printed */ };
+#define QP_B_MIDRISE 0x10  /* qp_dsaciq_search: bmode | QP_B_MIDRISE scores every candidate on the mid-rise grid */
 
 #define QP_DEFAULT_STEPS 100      /* search steps t (Sec. 3, directed search) */
 #define QP_DEFAULT_HIST_BINS 100
@@ -188,12 +189,21 @@ int32_t qp_aciq_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits,
  * [max(mean - alpha, min), min(mean + alpha, max)]: no element lies outside [min, max], so
  * the clipping error is unchanged and the step shrinks whenever alpha reaches past the data
  * (a variant of this library; the paper clips at mean -/+ alpha only).
+ * ... | QP_CLIP_MIDRISE (any method) puts the mid-rise grid on the range: 2^bits equal bins,
+ * every element reconstructed at the centre of its bin (the other reading of Sec. 3's "equal
+ * intervals", and the grid the ACIQ noise term alpha^2 / (3 * 4^q) models).  The bin centres
+ * are the levels of the ordinary quantizer on the range pulled in by half a bin on each side,
+ * [lo + w/2, hi - w/2] with w = (hi - lo) / 2^bits, and its rounding boundaries are the bin
+ * edges: the flag changes the clip range and nothing else (qp_midrise_range does just that),
+ * so packing and the receiver are the same.
  * qp_clip_range: host form, writes the ends (optional) and the quantizer (optional).
  * qp_clip_qparams_device: one-thread kernel from device-resident statistics.
  * Errors: QP_ERR_INVALID_ARG (NULL, unknown method, dist, bmode), QP_ERR_UNSUPPORTED_BITS;
  * QP_WARN_DEGENERATE as qp_make_qparams (host form; status word on the device). */
 enum { QP_CLIP_ACIQ = 0, QP_CLIP_DSACIQ = 1, QP_CLIP_MINMAX = 2 };
 #define QP_CLIP_INTERSECT 0x10
+#define QP_CLIP_MIDRISE 0x20
+int32_t qp_midrise_range(double lo, double hi, int bits, double* h_lo_out, double* h_hi_out);
 int32_t qp_clip_range(const qp_stats_t* h_stats, int bits, int method, int dist, int bmode, double* h_lo_out,
                       double* h_hi_out, qp_qparams_t* h_qp_out);
 int32_t qp_clip_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits, int method, int dist, int bmode,
@@ -205,7 +215,8 @@ int32_t qp_clip_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits,
  * quantization MSE of x under the clip F(bits) * b_k about the mean; the smallest k with
  * the lowest MSE wins (k = 0 keeps b_E).  d_stats must hold the statistics of the same x.
  * Writes *d_out (optional) and the winning quantizer *d_qp_out (optional); both device
- * memory.  bits 1..8; 1 <= steps <= QP_MAX_STEPS; 1 <= hist_bins <= QP_MAX_HIST_BINS.
+ * memory.  bits 1..8; 1 <= steps <= QP_MAX_STEPS; 1 <= hist_bins <= QP_MAX_HIST_BINS;
+ * bmode QP_B_MAD or QP_B_MEAN_ABS, optionally | QP_B_MIDRISE.
  * Errors: as qp_stats, plus QP_ERR_UNSUPPORTED_BITS. */
 int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                          int bits, int bmode, int steps, int hist_bins,
@@ -353,7 +364,7 @@ int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_packed, uint64_
 /* qp_sender_device: the sender's whole chain on DEVICE buffers in one call, nothing read back
  * to the host: statistics (carrying the histogram along for the search), the clip by
  * `method` (QP_CLIP_ACIQ = 0, optionally | QP_CLIP_INTERSECT; QP_CLIP_DSACIQ = 1, bits <= 8;
- * QP_CLIP_MINMAX = 2; Laplace model), quantize+pack.
+ * QP_CLIP_MINMAX = 2; each optionally | QP_CLIP_MIDRISE; Laplace model), quantize+pack.
  * Writes the packed stream to d_packed, the quantizer to *d_qp_out (what the receiver needs)
  * and, if d_stats_out is not NULL, the statistics.  Equivalent to qp_stats +
  * qp_dsaciq_search / qp_aciq_qparams_device + qp_quantize_pack with the same arguments.

@@ -27,7 +27,8 @@ QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
-QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT = 0, 1, 2, 0x10
+QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT, QP_CLIP_MIDRISE = 0, 1, 2, 0x10, 0x20
+QP_B_MIDRISE = 0x10
 
 EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
@@ -36,7 +37,7 @@ EXPORTS = (
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
     "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_clip_qparams_channels_device",
-    "qp_quantize_pack_channels", "qp_unpack_dequantize_channels",
+    "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range",
 )
 
 
@@ -105,6 +106,7 @@ def load() -> C.CDLL:
     L.qp_clip_range.argtypes = [C.POINTER(Stats), C.c_int, C.c_int, C.c_int, C.c_int, C.POINTER(dbl), C.POINTER(dbl),
                                 C.POINTER(QParams)]
     L.qp_clip_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.qp_midrise_range.argtypes = [dbl, dbl, C.c_int, C.POINTER(dbl), C.POINTER(dbl)]
     L.qp_stats_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, vp, vp]
     L.qp_clip_qparams_channels_device.argtypes = [vp, vp, C.c_uint32, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.qp_quantize_pack_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, vp, vp, u64, vp]
@@ -175,6 +177,12 @@ def qp_clip_range(stats: Stats, bits: int, method: int = QP_CLIP_ACIQ, dist: int
     lo, hi, qp = C.c_double(), C.c_double(), QParams()
     rc = load().qp_clip_range(C.byref(stats), bits, method, dist, bmode, C.byref(lo), C.byref(hi), C.byref(qp))
     return int(rc), lo.value, hi.value, qp
+
+
+def qp_midrise_range(lo: float, hi: float, bits: int):
+    a, b = C.c_double(), C.c_double()
+    rc = load().qp_midrise_range(lo, hi, bits, C.byref(a), C.byref(b))
+    return int(rc), a.value, b.value
 
 
 def qp_policy_use_ds(bits: int) -> bool:

@@ -256,9 +256,23 @@ extern "C" int32_t qp_aciq_alpha(const qp_stats_t* h_stats, int bits, int dist, 
     return qp_fill_qparams(lo, hi, bits, h_qp_out);
 }
 
-static bool clip_method_closed_form(int method)
+bool qp_clip_method_closed_form(int method)
 {
-    return method == QP_CLIP_ACIQ || method == (QP_CLIP_ACIQ | QP_CLIP_INTERSECT) || method == QP_CLIP_MINMAX;
+    const int base = method & 0xF, flags = method & ~0xF;
+    if (flags & ~(QP_CLIP_INTERSECT | QP_CLIP_MIDRISE)) return false;
+    if (base == QP_CLIP_ACIQ) return true;
+    return base == QP_CLIP_MINMAX && !(flags & QP_CLIP_INTERSECT);
+}
+static bool clip_method_closed_form(int method) { return qp_clip_method_closed_form(method); }
+
+extern "C" int32_t qp_midrise_range(double lo, double hi, int bits, double* h_lo_out, double* h_hi_out)
+{
+    if (!qp_bits_ok(bits)) return QP_ERR_UNSUPPORTED_BITS;
+    if (!h_lo_out || !h_hi_out || !isfinite(lo) || !isfinite(hi)) return QP_ERR_INVALID_ARG;
+    qp_midrise_ends(bits, lo, hi);
+    *h_lo_out = lo;
+    *h_hi_out = hi;
+    return QP_OK;
 }
 
 extern "C" int32_t qp_clip_range(const qp_stats_t* h_stats, int bits, int method, int dist, int bmode, double* h_lo_out,
@@ -270,7 +284,7 @@ extern "C" int32_t qp_clip_range(const qp_stats_t* h_stats, int bits, int method
     if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
         return QP_ERR_INVALID_ARG;
     double lo, hi;
-    qp_clip_ends(*h_stats, method, dist, bmode, qp_host_aciq_F(bits, dist), lo, hi);
+    qp_clip_ends(*h_stats, method, dist, bmode, bits, qp_host_aciq_F(bits, dist), lo, hi);
     if (h_lo_out) *h_lo_out = lo;
     if (h_hi_out) *h_hi_out = hi;
     if (!h_qp_out) return QP_OK;
@@ -541,7 +555,8 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
     if (rc) return rc;
     if (!d_stats) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_stats");
     if (bits < 1 || bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
-    if (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
+    if ((bmode & ~QP_B_MIDRISE) != QP_B_MAD && (bmode & ~QP_B_MIDRISE) != QP_B_MEAN_ABS)
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
     if (steps < 1 || steps > QP_MAX_STEPS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "steps out of range");
     if (hist_bins < 1 || hist_bins > QP_MAX_HIST_BINS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "hist_bins out of range");
     if (((uintptr_t)d_out & 7u) || ((uintptr_t)d_qp_out & 3u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "result pointers");
@@ -645,7 +660,8 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
                                 qp_qparams_t* d_qp_out, qp_stats_t* st, void* stream)
 {
     int32_t rc;
-    const int use_ds = method == QP_CLIP_DSACIQ;
+    const int use_ds = (method & 0xF) == QP_CLIP_DSACIQ;
+    const int search_mode = bmode | ((method & QP_CLIP_MIDRISE) ? QP_B_MIDRISE : 0);
     if (ctx->sender_path != QP_SENDER_CHAIN &&
         qp_sender_fused_applies(n, use_ds, steps, hist_bins, ctx->sender_path == QP_SENDER_FUSED)) {
         // the checks of the separate calls
@@ -666,7 +682,7 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
     }
     rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
     if (rc < 0) return rc;
-    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, bmode, steps, hist_bins, nullptr, d_qp_out, stream);
+    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, search_mode, steps, hist_bins, nullptr, d_qp_out, stream);
     else        rc = qp_clip_qparams_device(ctx, st, bits, method, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
     if (rc < 0) return rc;
     return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);
@@ -679,8 +695,9 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
     if (!ctx) return QP_ERR_INVALID_ARG;
     if (!d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_qp_out");
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    if (method != QP_CLIP_DSACIQ && !clip_method_closed_form(method)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "clip method");
-    if (method == QP_CLIP_DSACIQ && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if ((method & ~QP_CLIP_MIDRISE) != QP_CLIP_DSACIQ && !clip_method_closed_form(method))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "clip method");
+    if ((method & 0xF) == QP_CLIP_DSACIQ && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
     if (packed_capacity < qp_packed_bytes(n, bits))
         return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
     qp_stats_t* st = d_stats_out ? d_stats_out : ctx->d_tmp_stats;
@@ -688,7 +705,7 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
     const unsigned long long key[8] = {3, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_packed,
                                        (unsigned long long)dtype | (unsigned long long)bits << 8 |
                                            (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
-                                           (unsigned long long)(method == QP_CLIP_DSACIQ) << 28 | (unsigned long long)method << 56 |
+                                           (unsigned long long)((method & 0xF) == QP_CLIP_DSACIQ) << 28 | (unsigned long long)method << 56 |
                                            (unsigned long long)ctx->sender_path << 29 |
                                            (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
                                        packed_capacity, (unsigned long long)(uintptr_t)d_qp_out,
@@ -708,8 +725,9 @@ extern "C" int32_t qp_sender_host(qp_ctx* ctx, const void* h_x, int dtype, uint6
     if (!ctx) return QP_ERR_INVALID_ARG;
     if (dtype != QP_F32 && dtype != QP_BF16) return qp_fail(ctx, QP_ERR_UNSUPPORTED_DTYPE, "dtype");
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    if (method != QP_CLIP_DSACIQ && !clip_method_closed_form(method)) return qp_fail(ctx, QP_ERR_INVALID_ARG, "clip method");
-    if (method == QP_CLIP_DSACIQ && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
+    if ((method & ~QP_CLIP_MIDRISE) != QP_CLIP_DSACIQ && !clip_method_closed_form(method))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "clip method");
+    if ((method & 0xF) == QP_CLIP_DSACIQ && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
     if (!h_qp_out || (n > 0 && (!h_x || !d_x_work || !d_packed_work || !h_packed)))
         return qp_fail(ctx, QP_ERR_INVALID_ARG, "null buffer");
     const uint64_t need = qp_packed_bytes(n, bits);

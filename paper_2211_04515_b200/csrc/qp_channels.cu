@@ -252,7 +252,7 @@ __global__ void __launch_bounds__(128) ch_clip_kernel(const qp_stats_t* __restri
     const uint32_t c = blockIdx.x * 128 + threadIdx.x;
     if (c >= C) return;
     double lo, hi;
-    qp_clip_ends(st[c], method, dist, bmode, F, lo, hi);
+    qp_clip_ends(st[c], method, dist, bmode, bits, F, lo, hi);
     qp_qparams_t q;
     const int rc = qp_fill_qparams(lo, hi, bits, &q);
     qp_out[c] = q;
@@ -611,8 +611,8 @@ extern "C" int32_t qp_clip_qparams_channels_device(qp_ctx* ctx, const qp_stats_t
     if (rc) return rc;
     if (!d_stats || !d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    if (method != QP_CLIP_ACIQ && method != (QP_CLIP_ACIQ | QP_CLIP_INTERSECT) && method != QP_CLIP_MINMAX)
-        return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT) or MINMAX");
+    if (!qp_clip_method_closed_form(method))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT) or MINMAX, optionally | MIDRISE");
     if ((dist != QP_DIST_LAPLACE && dist != QP_DIST_GAUSS) || (bmode != QP_B_MAD && bmode != QP_B_MEAN_ABS))
         return qp_fail(ctx, QP_ERR_INVALID_ARG, "dist/bmode");
     qp_device_guard guard(ctx->device);

@@ -108,6 +108,7 @@ struct qp_device_guard {                 // makes ctx->device current for the sc
 // Shared host arithmetic (one definition each, in qp_api.cu).
 double qp_host_aciq_F(int bits, int dist);
 static inline bool qp_bits_ok(int bits) { return (bits >= 1 && bits <= 8) || bits == 16; }
+bool qp_clip_method_closed_form(int method);     // ACIQ (| INTERSECT) or MINMAX, optionally | MIDRISE
 
 // ------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
@@ -234,24 +235,36 @@ __device__ __forceinline__ double qp_block_max(double v, double* sh)
     return r;
 }
 
+// Mid-rise grid on a clip range: 2^bits equal bins over [lo, hi], reconstruction at the bin
+// centres.  The centres are the 2^bits levels of the uniform quantizer on the range pulled in
+// by half a bin on each side, and its rounding boundaries are the bin edges, so the grid is a
+// change of the clip range and nothing else.
+__host__ __device__ inline void qp_midrise_ends(int bits, double& lo, double& hi)
+{
+    const double half = (hi - lo) / (double)(2ull << bits);
+    lo += half;
+    hi -= half;
+}
+
 // Closed-form clip range from the statistics: ACIQ (optionally cut back to [min, max]) or the
-// tensor's own range; same on host and device.
-__host__ __device__ inline void qp_clip_ends(const qp_stats_t& st, int method, int dist, int bmode, double F, double& lo,
-                                             double& hi)
+// tensor's own range, optionally on the mid-rise grid; same on host and device.
+__host__ __device__ inline void qp_clip_ends(const qp_stats_t& st, int method, int dist, int bmode, int bits, double F,
+                                             double& lo, double& hi)
 {
     if ((method & 0xF) == QP_CLIP_MINMAX) {
         lo = st.min;
         hi = st.max;
-        return;
+    } else {
+        const double b = dist == QP_DIST_GAUSS ? sqrt(st.var) : (bmode == QP_B_MEAN_ABS ? st.mean_abs : st.mad);
+        const double alpha = F * b;
+        lo = st.mean - alpha;
+        hi = st.mean + alpha;
+        if (method & QP_CLIP_INTERSECT) {
+            if (st.min > lo) lo = st.min;
+            if (st.max < hi) hi = st.max;
+        }
     }
-    const double b = dist == QP_DIST_GAUSS ? sqrt(st.var) : (bmode == QP_B_MEAN_ABS ? st.mean_abs : st.mad);
-    const double alpha = F * b;
-    lo = st.mean - alpha;
-    hi = st.mean + alpha;
-    if (method & QP_CLIP_INTERSECT) {
-        if (st.min > lo) lo = st.min;
-        if (st.max < hi) hi = st.max;
-    }
+    if (method & QP_CLIP_MIDRISE) qp_midrise_ends(bits, lo, hi);
 }
 
 // ---- pieces of the directed search shared by its two scoring paths
@@ -262,7 +275,7 @@ __device__ inline void qp_ds_make_setup(const qp_stats_t* __restrict__ st, unsig
 {
     const unsigned long long nf = st->n - st->nonfinite;
     const double mn = st->min, mx = st->max;
-    const double b_e = bmode == QP_B_MEAN_ABS ? st->mean_abs : st->mad;
+    const double b_e = (bmode & 0xF) == QP_B_MEAN_ABS ? st->mean_abs : st->mad;
     double peak = 0.0;
     if (mx > mn && nf > 0) {
         const double w = (mx - mn) / (double)nb;
@@ -278,7 +291,8 @@ __device__ inline void qp_ds_make_setup(const qp_stats_t* __restrict__ st, unsig
 }
 
 // candidate k: b_k = b_E + k (b_R - b_E) / steps, evaluated in this order in fp64; its quantizer
-__device__ inline void qp_ds_candidate(const qp_ds_setup& s, int k, int steps, int bits, float4& c, int& ok)
+// (midrise != 0: on the mid-rise grid)
+__device__ inline void qp_ds_candidate(const qp_ds_setup& s, int k, int steps, int bits, int midrise, float4& c, int& ok)
 {
     const double b_k = s.b_e + (double)k * (s.b_r - s.b_e) / (double)steps;
     ok = ((k == 0) || (!s.degenerate && b_k > 0.0)) ? 1 : 0;
@@ -286,7 +300,9 @@ __device__ inline void qp_ds_candidate(const qp_ds_setup& s, int k, int steps, i
     q.lo = q.hi = q.scale = q.inv_scale = 0.f;
     if (ok) {
         const double alpha = s.F * b_k;
-        qp_fill_qparams(s.mean - alpha, s.mean + alpha, bits, &q);
+        double lo = s.mean - alpha, hi = s.mean + alpha;
+        if (midrise) qp_midrise_ends(bits, lo, hi);
+        qp_fill_qparams(lo, hi, bits, &q);
     }
     c = make_float4(q.lo, q.hi, q.scale, q.inv_scale);
 }

@@ -104,7 +104,7 @@ __global__ void __launch_bounds__(QP_THREADS) setup_kernel(const qp_stats_t* __r
     for (int k = threadIdx.x; k <= steps; k += QP_THREADS) {
         float4 c;
         int ok;
-        qp_ds_candidate(s, k, steps, bits, c, ok);
+        qp_ds_candidate(s, k, steps, bits, bmode & QP_B_MIDRISE, c, ok);
         cand[k] = c;
         valid[k] = ok;
     }
@@ -245,7 +245,7 @@ __global__ void aciq_kernel(const qp_stats_t* __restrict__ st, int bits, int met
 {
     if (threadIdx.x != 0 || blockIdx.x != 0) return;
     double lo, hi;
-    qp_clip_ends(*st, method, dist, bmode, F, lo, hi);
+    qp_clip_ends(*st, method, dist, bmode, bits, F, lo, hi);
     qp_qparams_t q;
     const int rc = qp_fill_qparams(lo, hi, bits, &q);
     *qp_out = q;

@@ -123,7 +123,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
     for (int k = threadIdx.x; k < ncand; k += 256) {
         float4 c;
         int ok;
-        qp_ds_candidate(s, k, steps, bits, c, ok);
+        qp_ds_candidate(s, k, steps, bits, bmode & QP_B_MIDRISE, c, ok);
         s_cand[k] = c;
         s_valid[k] = (unsigned char)ok;
         if (blockIdx.x == 0) { cand[k] = c; valid[k] = ok; }

@@ -315,7 +315,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
                 s_setup.u = 0.0;
             } else {
                 double lo, hi;
-                qp_clip_ends(s_st, a.method, QP_DIST_LAPLACE, a.bmode, a.F, lo, hi);
+                qp_clip_ends(s_st, a.method, QP_DIST_LAPLACE, a.bmode, a.bits, a.F, lo, hi);
                 const int rc = qp_fill_qparams(lo, hi, a.bits, &s_qp);
                 if (blockIdx.x == 0) {
                     *a.qp_out = s_qp;
@@ -331,7 +331,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
         for (int k = tid; k < ncand; k += FS_THREADS) {
             float4 c;
             int ok;
-            qp_ds_candidate(s_setup, k, a.steps, a.bits, c, ok);
+            qp_ds_candidate(s_setup, k, a.steps, a.bits, a.method & QP_CLIP_MIDRISE, c, ok);
             s_cand[k] = c;
             s_valid[k] = ok;
         }
@@ -515,7 +515,7 @@ int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t
                                int steps, int hist_bins, double F, void* d_packed, qp_qparams_t* d_qp_out,
                                qp_stats_t* d_stats_out, cudaStream_t s)
 {
-    const int use_ds = method == QP_CLIP_DSACIQ;
+    const int use_ds = (method & 0xF) == QP_CLIP_DSACIQ;
     const uint64_t total_words = qp_packed_bytes(n, bits) / 4;
     const uint64_t groups = (total_words + bits - 1) / bits;             // 32-element groups, pad words included
     const unsigned G = (unsigned)ctx->sm_count;

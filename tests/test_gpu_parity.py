@@ -392,6 +392,20 @@ def test_search_degenerate_and_errors(ctx):
 
 
 @pytest.mark.parametrize("path", BOTH_PATHS)
+@pytest.mark.parametrize("bits", [1, 2, 4, 6])
+def test_search_midrise_grid(ctx, bits, path):
+    """Every candidate on the mid-rise grid (bmode | QP_B_MIDRISE): same b_E, b_R and steps, other ranges."""
+    x = si.config_tensor("c1").reshape(-1)
+    res, res_o = check_search(ctx, x, dev(x), bits, bmode=qp.QP_B_MIDRISE, path=path)
+    plain, _ = check_search(ctx, x, dev(x), bits, path=path)
+    assert (res.b_e, res.b_r) == (plain.b_e, plain.b_r) and res.mse_e != plain.mse_e
+    y = si.vit_activation((5, 197, 200), 55, outlier_frac=0.02).reshape(-1)
+    check_search(ctx, y, dev(y), bits, bmode=qp.QP_B_MEAN_ABS | qp.QP_B_MIDRISE, path=path)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_dsaciq_search(dev(y), ctx.qp_stats(dev(y)), bits, 0x20)
+
+
+@pytest.mark.parametrize("path", BOTH_PATHS)
 def test_search_bf16(ctx, path):
     x = si.vit_activation((4, 197, 128), 8).reshape(-1)
     h = si.to_bf16_bits(x)
@@ -546,7 +560,9 @@ def test_fused_sender_range_and_fallback():
 
 # clip methods of the sender: ACIQ, ACIQ cut back to the data range, naive PTQ's min/max
 CLIP_CASES = [(qp.QP_CLIP_ACIQ, oracle.CLIP_ACIQ, False), (qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT, oracle.CLIP_ACIQ, True),
-              (qp.QP_CLIP_MINMAX, oracle.CLIP_MINMAX, False)]
+              (qp.QP_CLIP_MINMAX, oracle.CLIP_MINMAX, False), (qp.QP_CLIP_ACIQ | qp.QP_CLIP_MIDRISE, oracle.CLIP_ACIQ, False),
+              (qp.QP_CLIP_MINMAX | qp.QP_CLIP_MIDRISE, oracle.CLIP_MINMAX, False),
+              (qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT | qp.QP_CLIP_MIDRISE, oracle.CLIP_ACIQ, True)]
 
 
 @pytest.mark.parametrize("method,o_method,cut", CLIP_CASES)
@@ -561,15 +577,44 @@ def test_sender_clip_methods(ctx, method, o_method, cut, path):
             d_stats = torch.empty(ctypes.sizeof(qp.Stats), dtype=torch.uint8, device="cuda")
             packed, d_qp = ctx.qp_sender_device(d, bits, method, out_stats=d_stats)
             got = ctx.read_qparams(d_qp)
-            rc_o, lo_o, hi_o, q_o = oracle.clip_range(st_o, bits, o_method, cut)
+            rc_o, lo_o, hi_o, q_o = oracle.clip_range(st_o, bits, o_method, cut, midrise=bool(method & qp.QP_CLIP_MIDRISE))
             width = hi_o - lo_o
             assert abs(got.lo - q_o.lo) <= 1e-5 * width and abs(got.hi - q_o.hi) <= 1e-5 * width
-            if method == qp.QP_CLIP_MINMAX:                     # min and max are exact, so is the quantizer
+            if method & 0xF == qp.QP_CLIP_MINMAX:               # min and max are exact, so is the quantizer
                 assert bytes(got) == bytes(to_qp(q_o))
             o = oracle.QParams(got.lo, got.hi, got.scale, got.inv_scale, got.bits, got.flags)
             assert np.array_equal(packed.cpu().numpy(), oracle.quantize_pack(x, o))
             # the device form of the closed-form clip gives the same quantizer from the same statistics
             assert torch.equal(ctx.qp_clip_qparams_device(d_stats, bits, method), d_qp)
+    finally:
+        ctx.qp_set_sender_path(qp.QP_SENDER_AUTO)
+    assert ctx.qp_get_status() == 0
+
+
+@pytest.mark.parametrize("path", [qp.QP_SENDER_CHAIN, qp.QP_SENDER_FUSED])
+def test_sender_search_on_midrise_grid(ctx, path):
+    x = si.vit_activation((3, 197, 192), 82, outlier_frac=0.01).reshape(-1)
+    d = dev(x)
+    st_o = oracle.stats(x)
+    ctx.qp_set_sender_path(path)
+    try:
+        for bits in (2, 4):
+            packed, d_qp = ctx.qp_sender_device(d, bits, qp.QP_CLIP_DSACIQ | qp.QP_CLIP_MIDRISE)
+            got = ctx.read_qparams(d_qp)
+            rc_o, res_o, qp_o, curve_o = oracle.ds_search(x, st_o, bits, oracle.B_MIDRISE)
+            curve = np.array(ctx.qp_dsaciq_curve(100))
+            assert np.all(np.abs(curve - curve_o) <= 2e-6 * curve_o)
+            F = oracle.aciq_F(bits, 0)
+            ok = False
+            for k in np.flatnonzero(curve_o <= res_o.mse_star * (1 + 1e-6)):
+                alpha = F * (res_o.b_e + k * (res_o.b_r - res_o.b_e) / 100)
+                lo, hi = oracle.midrise_range(st_o.mean - alpha, st_o.mean + alpha, bits)
+                ok = ok or (abs(got.lo - lo) <= 1e-5 * alpha and abs(got.hi - hi) <= 1e-5 * alpha)
+            assert ok
+            o = oracle.QParams(got.lo, got.hi, got.scale, got.inv_scale, got.bits, got.flags)
+            assert np.array_equal(packed.cpu().numpy(), oracle.quantize_pack(x, o))
+            plain = ctx.read_qparams(ctx.qp_sender_device(d, bits, qp.QP_CLIP_DSACIQ)[1])
+            assert (plain.lo, plain.hi) != (got.lo, got.hi)
     finally:
         ctx.qp_set_sender_path(qp.QP_SENDER_AUTO)
     assert ctx.qp_get_status() == 0
@@ -767,10 +812,10 @@ def check_channels(ctx, x_np, d_x, channels, bits, method=qp.QP_CLIP_ACIQ, out_b
     st_o = oracle.stats_channels(x_np, channels)
     for c in range(channels):
         check_stats(st[c], st_o[c])
-    o_method, cut = (oracle.CLIP_MINMAX, False) if method == qp.QP_CLIP_MINMAX else (oracle.CLIP_ACIQ, bool(method & qp.QP_CLIP_INTERSECT))
+    o_method, cut = (oracle.CLIP_MINMAX, False) if method & 0xF == qp.QP_CLIP_MINMAX else (oracle.CLIP_ACIQ, bool(method & qp.QP_CLIP_INTERSECT))
     d_qp = ctx.qp_clip_qparams_channels_device(d_stats, channels, bits, method)
     got = _read_array(d_qp, qp.QParams, channels)
-    rc_o, qp_o = oracle.clip_channels(st_o, bits, o_method, cut)
+    rc_o, qp_o = oracle.clip_channels(st_o, bits, o_method, cut, midrise=bool(method & qp.QP_CLIP_MIDRISE))
     for c in range(channels):
         width = max(qp_o[c].hi - qp_o[c].lo, 1e-30)
         assert abs(got[c].lo - qp_o[c].lo) <= 1e-5 * width and abs(got[c].hi - qp_o[c].hi) <= 1e-5 * width, c
@@ -811,7 +856,8 @@ def test_channels_shapes_ragged_and_methods(ctx, channels, rows):
     x = si.vit_activation((1, rows, channels), 102 + channels % 5, outlier_frac=0.05).reshape(-1)
     d = dev(x)
     for bits, method in ((2, qp.QP_CLIP_ACIQ), (5, qp.QP_CLIP_MINMAX), (8, qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT),
-                         (16, qp.QP_CLIP_ACIQ)):
+                         (16, qp.QP_CLIP_ACIQ), (4, qp.QP_CLIP_ACIQ | qp.QP_CLIP_MIDRISE),
+                         (3, qp.QP_CLIP_MINMAX | qp.QP_CLIP_MIDRISE)):
         check_channels(ctx, x, d, channels, bits, method)
     ctx.qp_get_status()                                         # single-row tensors have no spread: degenerate
 

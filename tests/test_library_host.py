@@ -110,7 +110,18 @@ def test_clip_range_matches_oracle(lib):
                 assert rc == rc_o == 0
                 assert lo == pytest.approx(lo_o, rel=1e-12, abs=1e-300) and hi == pytest.approx(hi_o, rel=1e-12, abs=1e-300)
                 assert _same_qp(q, q_o)
+    # mid-rise grid: the same ranges pulled in by half a bin
+    for bits in (1, 4, 8, 16):
+        for method, o_method, cut in ((qp.QP_CLIP_ACIQ, oracle.CLIP_ACIQ, False), (qp.QP_CLIP_MINMAX, oracle.CLIP_MINMAX, False),
+                                      (qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT, oracle.CLIP_ACIQ, True)):
+            rc, lo, hi, q = qp.qp_clip_range(st, bits, method | qp.QP_CLIP_MIDRISE)
+            rc_o, lo_o, hi_o, q_o = oracle.clip_range(st_o, bits, o_method, cut, midrise=True)
+            assert rc == rc_o == 0 and lo == pytest.approx(lo_o, rel=1e-12) and hi == pytest.approx(hi_o, rel=1e-12)
+            assert _same_qp(q, q_o)
+    assert qp.qp_midrise_range(0.0, 4.0, 2) == (0, 0.5, 3.5) and oracle.midrise_range(0.0, 4.0, 2) == (0.5, 3.5)
+    assert qp.qp_midrise_range(0.0, 4.0, 9)[0] == qp.QP_ERR_UNSUPPORTED_BITS
     assert qp.qp_clip_range(st, 4, qp.QP_CLIP_DSACIQ)[0] == qp.QP_ERR_INVALID_ARG      # needs the tensor, not a closed form
+    assert qp.qp_clip_range(st, 4, qp.QP_CLIP_ACIQ | 0x40)[0] == qp.QP_ERR_INVALID_ARG
     assert qp.qp_clip_range(st, 4, qp.QP_CLIP_MINMAX | qp.QP_CLIP_INTERSECT)[0] == qp.QP_ERR_INVALID_ARG
     assert qp.qp_clip_range(st, 9)[0] == qp.QP_ERR_UNSUPPORTED_BITS
     const = qp.Stats(10, 0, 2.0, 2.0, 0.0, 0.0, 2.0, 2.0, 0, 0, 0)
