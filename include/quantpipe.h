@@ -336,6 +336,11 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  *                                    qp_clip_qparams_device.
  *   qp_quantize_pack_channels        code of element i with d_qp[i mod channels].
  *   qp_unpack_dequantize_channels    the inverse, fp32 or bf16 out.
+ *   qp_sender_channels_device        the three sender calls in one: statistics -> clip by `method`
+ *                                    (Laplace model) -> quantize+pack; writes the packed stream,
+ *                                    d_qp_out[0..channels) and, if d_stats_out is not NULL, the
+ *                                    statistics (otherwise they stay in a buffer of the context,
+ *                                    allocated on first use).
  * d_stats, d_qp: device arrays of `channels` entries.  1 <= channels <= QP_MAX_CHANNELS.
  * Errors: as the per-tensor calls, plus QP_ERR_INVALID_ARG for channels out of range. */
 #define QP_MAX_CHANNELS 4096
@@ -348,6 +353,9 @@ int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int dtype, uint6
                                   void* stream);
 int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_packed, uint64_t rows, uint32_t channels, int bits,
                                       const qp_qparams_t* d_qp, void* d_y, int out_dtype, void* stream);
+int32_t qp_sender_channels_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels, int bits,
+                                  int method, int bmode, void* d_packed, uint64_t packed_capacity,
+                                  qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream);
 
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------

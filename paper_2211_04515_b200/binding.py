@@ -37,7 +37,7 @@ EXPORTS = (
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
     "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_clip_qparams_channels_device",
-    "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range",
+    "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range", "qp_sender_channels_device",
 )
 
 
@@ -111,6 +111,7 @@ def load() -> C.CDLL:
     L.qp_clip_qparams_channels_device.argtypes = [vp, vp, C.c_uint32, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.qp_quantize_pack_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, vp, vp, u64, vp]
     L.qp_unpack_dequantize_channels.argtypes = [vp, vp, u64, C.c_uint32, C.c_int, vp, vp, C.c_int, vp]
+    L.qp_sender_channels_device.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, C.c_int, C.c_int, vp, u64, vp, vp, vp]
     L.qp_dsaciq_search.argtypes = [vp, vp, C.c_int, u64, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
     L.qp_dsaciq_curve.argtypes = [vp, C.POINTER(dbl), C.c_int, vp]
     L.qp_policy_use_ds.argtypes = [C.c_int]
@@ -432,6 +433,19 @@ class Context:
                                                             d_qp.data_ptr(), out.data_ptr(), _dtype_code(out),
                                                             _stream(self.device)))
         return out
+
+    def qp_sender_channels_device(self, x: torch.Tensor, channels: int, bits: int, method: int = QP_CLIP_ACIQ,
+                                  bmode: int = QP_B_MAD, out_packed: torch.Tensor | None = None,
+                                  out_qp: torch.Tensor | None = None, out_stats: torch.Tensor | None = None):
+        """Channel-wise statistics -> clip -> quantize+pack in one call; returns (packed, device QParams[channels])."""
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        out_packed = self._bytes(qp_packed_bytes(x.numel(), bits)) if out_packed is None else out_packed
+        out_qp = self._bytes(C.sizeof(QParams) * channels) if out_qp is None else out_qp
+        self._check(self._lib.qp_sender_channels_device(
+            self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels, channels, bits, method, bmode,
+            out_packed.data_ptr(), out_packed.numel() * out_packed.element_size(), out_qp.data_ptr(),
+            out_stats.data_ptr() if out_stats is not None else None, _stream(self.device)))
+        return out_packed, out_qp
 
     # -- host-buffer sender / receiver
     def qp_sender_host(self, h_x: torch.Tensor, bits: int, use_ds: bool, d_x_work: torch.Tensor,

@@ -127,6 +127,7 @@ extern "C" int32_t qp_destroy(qp_ctx* ctx)
     qp_device_guard guard(ctx->device);
     qp_drop_graphs(ctx);
     if (ctx->d_ch_part) cudaFree(ctx->d_ch_part);
+    if (ctx->d_ch_stats) cudaFree(ctx->d_ch_stats);
     const cudaError_t e = cudaFree(ctx->d_base);
     delete ctx;
     return e == cudaSuccess ? QP_OK : QP_ERR_CUDA;

@@ -743,3 +743,42 @@ extern "C" int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_pack
     ctx->launches += 1;
     return qp_check_launch(ctx, "qp_unpack_dequantize_channels");
 }
+
+// The channel-wise sender in one call: statistics -> per-channel clip -> quantize+pack, nothing read
+// back to the host.  The statistics go to d_stats_out, or to a buffer the context keeps when that is NULL.
+extern "C" int32_t qp_sender_channels_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels,
+                                             int bits, int method, int bmode, void* d_packed, uint64_t packed_capacity,
+                                             qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    int32_t rc = ch_check(ctx, rows, channels);
+    if (rc) return rc;
+    if (!d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_qp_out");
+    if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
+    if (!qp_clip_method_closed_form(method))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT) or MINMAX, optionally | MIDRISE");
+    if (packed_capacity < qp_packed_bytes(rows * channels, bits))
+        return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(rows * channels, bits)");
+    qp_stats_t* st = d_stats_out;
+    if (!st) {
+        const size_t need = sizeof(qp_stats_t) * (size_t)channels;
+        if (ctx->ch_stats_bytes < need) {
+            qp_device_guard guard(ctx->device);
+            if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
+            if (ctx->d_ch_stats) cudaFree(ctx->d_ch_stats);
+            ctx->d_ch_stats = nullptr;
+            ctx->ch_stats_bytes = 0;
+            if (cudaMalloc(&ctx->d_ch_stats, need) != cudaSuccess) {
+                cudaGetLastError();
+                return qp_fail(ctx, QP_ERR_CUDA, "cannot allocate the channel statistics");
+            }
+            ctx->ch_stats_bytes = need;
+        }
+        st = static_cast<qp_stats_t*>(ctx->d_ch_stats);
+    }
+    rc = qp_stats_channels(ctx, d_x, dtype, rows, channels, st, stream);
+    if (rc < 0) return rc;
+    rc = qp_clip_qparams_channels_device(ctx, st, channels, bits, method, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
+    if (rc < 0) return rc;
+    return qp_quantize_pack_channels(ctx, d_x, dtype, rows, channels, bits, d_qp_out, d_packed, packed_capacity, stream);
+}

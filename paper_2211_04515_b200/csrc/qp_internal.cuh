@@ -79,6 +79,8 @@ struct qp_ctx {
     void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
     void* d_ch_part;                     // channel-wise statistics: block partials, allocated on first use
     size_t ch_part_bytes;
+    void* d_ch_stats;                    // channel-wise sender: statistics when the caller wants none back
+    size_t ch_stats_bytes;
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
     qp_qparams_t* d_tmp_qp;
     unsigned long long launches;         // kernels launched through this context (host count)

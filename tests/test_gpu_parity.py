@@ -920,3 +920,20 @@ def test_channels_full_size_c2_sampled(ctx):
         assert np.array_equal(packed[r0 * 768 // 2: r0 * 768 // 2 + nb], oracle.pack(codes, 4)[:nb])
         assert np.max(np.abs(y[r0:r0 + 3].reshape(-1) - oracle.dequantize_channels(codes, 768, mine))) <= 1e-6
     assert ctx.qp_get_status() == 0
+
+
+def test_channels_sender_in_one_call(ctx):
+    x = si.vit_activation((2, 197, 384), 109, outlier_frac=0.02).reshape(-1)
+    d = dev(x)
+    for bits, method in ((4, qp.QP_CLIP_ACIQ), (8, qp.QP_CLIP_MINMAX | qp.QP_CLIP_MIDRISE)):
+        d_stats = ctx.qp_stats_channels(d, 384)
+        d_qp = ctx.qp_clip_qparams_channels_device(d_stats, 384, bits, method)
+        want = ctx.qp_quantize_pack_channels(d, 384, bits, d_qp)
+        got, got_qp = ctx.qp_sender_channels_device(d, 384, bits, method)            # statistics kept by the context
+        assert torch.equal(got, want) and torch.equal(got_qp, d_qp)
+        st_out = torch.empty(384 * ctypes.sizeof(qp.Stats), dtype=torch.uint8, device="cuda")
+        got2, _ = ctx.qp_sender_channels_device(d, 384, bits, method, out_stats=st_out)
+        assert torch.equal(got2, want) and torch.equal(st_out, d_stats)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_sender_channels_device(d, 384, 4, qp.QP_CLIP_DSACIQ)
+    assert ctx.qp_get_status() == 0
