@@ -186,9 +186,14 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
     }
 }
 
-// Rank sort of the MAXB boundaries.  Block b places entries [32b, 32b+32): thread t compares
-// entry 32b + (t & 31) with the 256 entries of slice t >> 5, the 16 slice counts are merged in
-// shared memory (rank = entries that are smaller, or equal with a lower index).
+// Rank sort of the MAXB boundaries (rank = entries that are smaller, or equal with a lower
+// index).  The array is [nthr thresholds in any order][cell edges, then +inf fillers]; the
+// second part is already non-decreasing (the edge of a cell is never below the edge of the
+// cell before it, missing cells are +inf at the end), so only the thresholds need comparing:
+//   threshold:  rank = thresholds before it + tail entries strictly below it (binary search)
+//   tail entry: rank = thresholds <= it + its own position in the tail
+// Block b places entries [32b, 32b+32): thread t compares entry 32b + (t & 31) with the
+// thresholds of slice t >> 5, the 16 slice counts are merged in shared memory.
 // bb[0] = g_lo, bb[1 + r] = entry of rank r; +inf entries end up behind the finite ones.
 // For the entry that is the left edge of grid cell c it also stores
 // first[c] = number of boundaries <= that edge (the edge included), or ~0 if the cell does
@@ -206,12 +211,32 @@ __global__ void __launch_bounds__(512) iv_rank_kernel(const float* __restrict__ 
     const int me = blockIdx.x * IV_RANK_PER_BLOCK + local;
     const float v = s[me];
     int cnt = 0, cnt_le = 0;
-    const int j0 = slice * (MAXB / 16);
-#pragma unroll 8
-    for (int j = j0; j < j0 + MAXB / 16; ++j) {
+    const int per = (nthr + 15) / 16;                         // thresholds per slice
+    const int j1 = min(nthr, (slice + 1) * per);
+    for (int j = slice * per; j < j1; ++j) {
         const float w = s[j];
         cnt += (w < v || (w == v && j < me)) ? 1 : 0;
         cnt_le += (w <= v) ? 1 : 0;
+    }
+    if (slice == 0) {                                         // the sorted tail: binary searches
+        const float* tail = s + nthr;
+        const int len = MAXB - nthr;
+        int lo = 0, hi = len;                                 // entries strictly below v
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (tail[mid] < v) lo = mid + 1; else hi = mid;
+        }
+        const int below = lo;
+        hi = len;                                             // entries <= v (continue from `below`)
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (tail[mid] <= v) lo = mid + 1; else hi = mid;
+        }
+        cnt_le += lo;
+        // a threshold counts the tail entries below it; a tail entry counts its own position (equal
+        // tail entries before it have lower indices; the loop above has counted the thresholds <= it,
+        // which all have lower indices too)
+        cnt += me < nthr ? below : (me - nthr);
     }
     atomicAdd(&rank[local], cnt);
     atomicAdd(&le[local], cnt_le);
