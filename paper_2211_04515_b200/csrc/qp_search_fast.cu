@@ -416,11 +416,11 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
 }
 
 // Totals over the blocks' partials.  A block takes 32 consecutive intervals: lane = interval
-// (one 256-byte row segment per warp load), warp w adds the partials of blocks w, w + 16, ...
-// (eight loads in flight), the 16 warp sums are merged through shared memory and written
+// (one 256-byte row segment per warp load), warp w adds the partials of blocks w, w + 32, ...
+// (all of its loads in flight at once), the 32 warp sums are merged through shared memory and written
 // once.  Integer sums, so the order does not matter.  Block 0 also adds up the outer sums
 // in block order.
-constexpr int IV_RED_THREADS = 512;
+constexpr int IV_RED_THREADS = 1024;
 constexpr int IV_RED_WARPS = IV_RED_THREADS / 32;
 __global__ void __launch_bounds__(IV_RED_THREADS) iv_reduce_kernel(const unsigned long long* __restrict__ part, int blocks,
                                                                    const unsigned* __restrict__ g_m,
@@ -434,15 +434,15 @@ __global__ void __launch_bounds__(IV_RED_THREADS) iv_reduce_kernel(const unsigne
     const unsigned i = blockIdx.x * 32 + lane;
     unsigned long long n = 0, s1 = 0;
     if (i <= m) {
-        for (int b0 = warp; b0 < blocks; b0 += IV_RED_WARPS * 8) {
-            unsigned long long p[8];
+        for (int b0 = warp; b0 < blocks; b0 += IV_RED_WARPS * 16) {
+            unsigned long long p[16];
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 const int b = b0 + u * IV_RED_WARPS;
                 p[u] = b < blocks ? part[(size_t)b * (MAXB + 1) + i] : 0ull;
             }
 #pragma unroll
-            for (int u = 0; u < 8; ++u) {
+            for (int u = 0; u < 16; ++u) {
                 n += p[u] >> 40;
                 s1 += p[u] & S1_MASK;
             }
