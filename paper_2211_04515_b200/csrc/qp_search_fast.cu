@@ -266,18 +266,19 @@ struct IvShared {
 
 // Elements outside [g_lo, g_hi] are clipped by every candidate.  They go through the interval
 // of the end they were clamped to (which contributes (level - end)^2 for them), and the rest of
-// their error, -2 (level - end) e + e^2 with e = distance beyond the end, needs only sum e and
-// sum e^2 per side, kept per thread.
+// their error, -2 (level - end) e + e^2 with e = signed distance beyond the end (negative below
+// g_lo, positive above g_hi, zero inside), needs only the sums of e on each side and of e^2.
+// Kept per thread as sum e, sum |e| (the two sides are their half sum and half difference) and
+// sum e^2: one subtraction and three accumulations per element.
 struct IvOuter {                    // per thread, fp64
-    double s1_lo, s2_lo, s1_hi, s2_hi, s2_in;
+    double s1, s1a, s2, s2_in;
 };
 struct IvBatch {                    // the same over one batch of <= 8 elements, fp32
-    float s1_lo, s2_lo, s1_hi, s2_hi, s2_in;
+    float s1, s1a, s2, s2_in;
 };
 __device__ __forceinline__ void iv_flush(IvOuter& o, const IvBatch& b)
 {
-    o.s1_lo += (double)b.s1_lo; o.s2_lo += (double)b.s2_lo;
-    o.s1_hi += (double)b.s1_hi; o.s2_hi += (double)b.s2_hi;
+    o.s1 += (double)b.s1; o.s1a += (double)b.s1a; o.s2 += (double)b.s2;
     o.s2_in += (double)b.s2_in;
 }
 
@@ -288,10 +289,10 @@ __device__ __forceinline__ void iv_one(float x, const IvShared& sh, const IvCons
 {
     if (GUARD && !qp_is_finite(x)) return;
     {
-        const float e_lo = fmaxf(__fsub_rn(k.g_lo, x), 0.f), e_hi = fmaxf(__fsub_rn(x, k.g_hi), 0.f);
-        b.s1_lo += e_lo; b.s2_lo = fmaf(e_lo, e_lo, b.s2_lo);
-        b.s1_hi += e_hi; b.s2_hi = fmaf(e_hi, e_hi, b.s2_hi);
-        x = fminf(fmaxf(x, k.g_lo), k.g_hi);
+        const float xc = fminf(fmaxf(x, k.g_lo), k.g_hi);
+        const float e = __fsub_rn(x, xc);
+        b.s1 += e; b.s1a += fabsf(e); b.s2 = fmaf(e, e, b.s2);
+        x = xc;
         const float pm = cell_pm(x, k.g_lo, k.inv_gw);
         const unsigned ci = sh.cell[__float_as_uint(pm) & 0x7FFFFFu];
         unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
@@ -359,7 +360,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
 
     const IvConst k = {setup->g_lo, setup->g_hi, setup->inv_gw, setup->gw, setup->inv_u};
     const bool guard = st->nonfinite != 0;
-    IvOuter o = {0.0, 0.0, 0.0, 0.0, 0.0};
+    IvOuter o = {0.0, 0.0, 0.0, 0.0};
 
     constexpr int EPV = qp_span<T>::EPV;
     const qp_span<T> sp(x, n);
@@ -372,7 +373,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
             float a[EPV], b[EPV];
             qp_load_vec(xv + v * EPV, a);
             qp_load_vec(xv + (v + stride) * EPV, b);
-            IvBatch bt = {0.f, 0.f, 0.f, 0.f, 0.f};
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, k, bt);
 #pragma unroll
@@ -382,7 +383,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
         for (; v < sp.nvec; v += stride) {
             float a[EPV];
             qp_load_vec(xv + v * EPV, a);
-            IvBatch bt = {0.f, 0.f, 0.f, 0.f, 0.f};
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int i = 0; i < EPV; ++i) iv_one<GD>(a[i], sh, k, bt);
             iv_flush(o, bt);
@@ -390,7 +391,7 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
         if (blockIdx.x == 0) {
             const uint64_t t0 = sp.head + sp.nvec * EPV;
             for (uint64_t i = threadIdx.x; i < sp.head + sp.tail; i += QP_IV_THREADS) {
-                IvBatch bt = {0.f, 0.f, 0.f, 0.f, 0.f};
+                IvBatch bt = {0.f, 0.f, 0.f, 0.f};
                 iv_one<GD>(qp_load_one(x + (i < sp.head ? i : t0 + (i - sp.head))), sh, k, bt);
                 iv_flush(o, bt);
             }
@@ -405,8 +406,8 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     }
 
     __shared__ double red[QP_IV_THREADS / 32];
-    const double r0 = qp_block_sum(o.s1_lo, red), r1 = qp_block_sum(o.s2_lo, red);
-    const double r2 = qp_block_sum(o.s1_hi, red), r3 = qp_block_sum(o.s2_hi, red);
+    const double r0 = qp_block_sum(o.s1, red), r1 = qp_block_sum(o.s1a, red);
+    const double r2 = qp_block_sum(o.s2, red), r3 = 0.0;
     const double r4 = 0.0, r5 = 0.0;
     const double r6 = qp_block_sum(o.s2_in, red);
     if (threadIdx.x == 0) {
@@ -528,13 +529,13 @@ __global__ void __launch_bounds__(IV_CURVE_THREADS) iv_curve_kernel(const qp_iv_
     if (threadIdx.x == 0) {
         double mse = __longlong_as_double(0x7FF0000000000000ll);
         if (ok) {
-            const double s1_lo = outer_tot[0], s2_lo = outer_tot[1], s1_hi = outer_tot[2], s2_hi = outer_tot[3];
+            const double s1 = outer_tot[0], s1a = outer_tot[1], s2 = outer_tot[2];
+            const double s1_lo = 0.5 * (s1a - s1), s1_hi = 0.5 * (s1a + s1);   // sums of the distances beyond each end
             const double s2_in = outer_tot[6];
             const double a_lo = level(setup->g_lo) - (double)setup->g_lo;      // >= 0: below every clip range
             const double a_hi = level(setup->g_hi) - (double)setup->g_hi;      // <= 0: above every clip range
             total += s2_in * (u * u);                  // sum of squared offsets: the same for every candidate
-            total += 2.0 * a_lo * s1_lo + s2_lo;         // what lies beyond the ends (see IvOuter)
-            total += -2.0 * a_hi * s1_hi + s2_hi;
+            total += 2.0 * a_lo * s1_lo - 2.0 * a_hi * s1_hi + s2;   // what lies beyond the ends (see IvOuter)
             const unsigned long long nf = setup->n_finite;
             mse = nf ? total / (double)nf : 0.0;
         }
