@@ -39,14 +39,14 @@ __device__ __forceinline__ float dequant(unsigned c, const DQ& q) { return fmaf(
 
 __device__ __forceinline__ void store_out(float* y, uint64_t i4, const float (&v)[4])
 {
-    reinterpret_cast<float4*>(y)[i4] = make_float4(v[0], v[1], v[2], v[3]);
+    __stcs(reinterpret_cast<float4*>(y) + i4, make_float4(v[0], v[1], v[2], v[3]));
 }
 __device__ __forceinline__ void store_out(unsigned short* y, uint64_t i4, const float (&v)[4])
 {
     uint2 o;
     o.x = (unsigned)qp_f32_to_bf16(v[0]) | ((unsigned)qp_f32_to_bf16(v[1]) << 16);
     o.y = (unsigned)qp_f32_to_bf16(v[2]) | ((unsigned)qp_f32_to_bf16(v[3]) << 16);
-    reinterpret_cast<uint2*>(y)[i4] = o;
+    __stcs(reinterpret_cast<uint2*>(y) + i4, o);
 }
 __device__ __forceinline__ void store_one(float* y, uint64_t i, float v) { y[i] = v; }
 __device__ __forceinline__ void store_one(unsigned short* y, uint64_t i, float v) { y[i] = qp_f32_to_bf16(v); }
