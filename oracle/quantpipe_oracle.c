@@ -437,6 +437,11 @@ double orc_hist_peak(const float* x, uint64_t n, double mn, double mx, int nb, u
  *              (bmode | 0x10: on the mid-rise grid, orc_midrise_range)
  *   k*       = smallest k attaining the minimum; k = 0 is b_E itself, so b_E is kept
  *              unless some step is strictly better.
+ * bmode | 0x20: the same search under the Gaussian model that ACIQ also offers (a variant of
+ *   this library; the paper searches under the Laplace model only).  The scale is the
+ *   standard deviation: sigma_E = sqrt(var); the peak of N(mu, sigma) is 1 / (sigma sqrt(2 pi)),
+ *   so sigma_R = 1 / (sqrt(2 pi) max(D_R)); sigma_k between them as above, alpha_k = F_G(q) sigma_k.
+ *   The result's b_e, b_r, b_star then hold sigma_E, sigma_R, sigma*.
  * mse_curve (t+1 doubles) optional. */
 int orc_ds_search(const float* x, uint64_t n, const orc_stats_t* st, int bits, int bmode,
                   int steps, int hist_bins, orc_ds_result_t* res, orc_qparams_t* qp_out,
@@ -444,13 +449,15 @@ int orc_ds_search(const float* x, uint64_t n, const orc_stats_t* st, int bits, i
 {
     if (!(bits >= 1 && bits <= 8)) return ORC_ERR_BITS;
     int midrise = (bmode & 0x10) != 0;                     /* every candidate on the mid-rise grid */
-    bmode &= ~0x10;
-    if (steps < 1 || hist_bins < 1 || (bmode != 0 && bmode != 1)) return ORC_ERR_ARG;
-    double F = orc_aciq_F_laplace(bits);
-    double b_e = bmode == 1 ? st->mean_abs : st->mad;
+    int gauss = (bmode & 0x20) != 0;                       /* Gaussian model: scale = standard deviation */
+    bmode &= ~0x30;
+    if (steps < 1 || hist_bins < 1 || (bmode != 0 && bmode != 1) || (gauss && bmode != 0)) return ORC_ERR_ARG;
+    double F = gauss ? orc_aciq_F_gauss(bits) : orc_aciq_F_laplace(bits);
+    double b_e = gauss ? sqrt(st->var) : (bmode == 1 ? st->mean_abs : st->mad);
     double peak = orc_hist_peak(x, n, st->min, st->max, hist_bins, NULL);
     int degenerate = !(st->max > st->min) || !(peak > 0.0) || !(b_e > 0.0);
-    double b_r = degenerate ? b_e : 1.0 / (2.0 * peak);
+    double peak_factor = gauss ? sqrt(2.0 * 3.14159265358979323846) : 2.0;   /* density peak = 1 / (factor * scale) */
+    double b_r = degenerate ? b_e : 1.0 / (peak_factor * peak);
     memset(res, 0, sizeof *res);
     res->b_e = b_e;
     res->b_r = b_r;

@@ -392,6 +392,68 @@ def test_ds_direction_follows_histogram_peak():
     assert res.mse_star <= res.mse_e
 
 
+def _gauss_F_numeric(q):
+    """Minimiser of the normal clipping-plus-rounding model, by SciPy (independent of the oracle's bisection)."""
+    from scipy.optimize import minimize_scalar
+    from scipy.stats import norm
+    model = lambda a: 2.0 * ((1.0 + a * a) * norm.sf(a) - a * norm.pdf(a)) + a * a / (3.0 * 4.0 ** q)
+    return minimize_scalar(model, bounds=(0.1, 12.0), method="bounded", options={"xatol": 1e-12}).x
+
+
+@pytest.mark.parametrize("q,seed,nb", [(2, 1, 100), (4, 2, 100), (3, 3, 256)])
+def test_ds_search_gaussian_model(q, seed, nb):
+    """bmode | 0x20: the directed search with the normal density's scale and peak, against an
+    independent evaluation of its 101 candidates."""
+    x = si.vit_activation((1, 16, 256), seed, outlier_frac=0.02 if seed % 2 else 0.0).reshape(-1)
+    st = oracle.stats(x)
+    rc, res, qp, curve = oracle.ds_search(x, st, q, 0x20, 100, nb)
+    assert rc == 0
+    counts, _ = np.histogram(x.astype(np.float64), bins=nb, range=(st.min, st.max))
+    peak_ref = counts.max() / (x.size * (st.max - st.min) / nb)
+    assert res.b_e == math.sqrt(st.var)                                          # sigma_E
+    assert res.b_r == pytest.approx(1.0 / (math.sqrt(2.0 * math.pi) * peak_ref), rel=0.02)   # sigma_R
+    F = _gauss_F_numeric(q)
+    mses = np.array([_numpy_candidate_mse(x, st.mean, F * (res.b_e + k * (res.b_r - res.b_e) / 100), q)
+                     for k in range(101)])
+    assert np.allclose(curve, mses, rtol=1e-5)              # F from two solvers: alpha agrees to ~1e-8
+    k_ref = int(np.argmin(mses))
+    assert res.k_star == k_ref or abs(mses[res.k_star] - mses[k_ref]) <= 1e-6 * mses[k_ref]
+    assert res.mse_star <= res.mse_e
+    assert res.alpha_e == pytest.approx(F * math.sqrt(st.var), rel=1e-6)       # a numeric minimiser finds F to ~1e-8
+    assert res.alpha_star == pytest.approx(F * res.b_star, rel=1e-6)
+    # step 0 is plain Gaussian ACIQ
+    _, alpha0, qp0 = oracle.aciq_alpha(st, q, dist=1)
+    assert alpha0 == res.alpha_e and curve[0] == oracle.quant_mse(x, qp0)
+    assert oracle.quant_mse(x, qp) == res.mse_star
+
+
+def test_ds_search_gaussian_peak_relation_and_direction():
+    # normal data: the histogram peak estimates 1 / (sigma sqrt(2 pi)), so sigma_R ~ sigma_E
+    g = (0.7 * si.flat_iid(1 << 20, 11, "normal")).astype(np.float32)
+    st = oracle.stats(g)
+    _, res, _, _ = oracle.ds_search(g, st, 4, 0x20, 100, 256)
+    assert res.b_e == pytest.approx(0.7, rel=0.01) and res.b_r == pytest.approx(res.b_e, rel=0.05)
+    # the Laplace-model search on the same data sees a peak below a Laplace fit's: b_R > b_E
+    _, res_l, _, _ = oracle.ds_search(g, st, 4, 0, 100, 256)
+    assert res_l.b_r > res_l.b_e
+    # uniform data is flatter than a normal of the same variance: sigma_R = 2a / sqrt(2 pi) > a / sqrt(3)
+    u = (si.uniform01(3, si.STREAM_VALUE, 0, 200000) * 2 - 1).astype(np.float32)
+    st = oracle.stats(u)
+    _, res, _, _ = oracle.ds_search(u, st, 2, 0x20, 100, 100)
+    assert res.b_e == pytest.approx(1 / math.sqrt(3), rel=0.01)
+    # the fullest of 100 bins of 2000 expected counts lies ~2.5 Poisson deviations above the mean (+6 %)
+    assert 0.93 * 2 / math.sqrt(2 * math.pi) < res.b_r <= 2 / math.sqrt(2 * math.pi) and res.b_r > res.b_e
+    # Laplace data is more peaked than a normal of the same variance: sigma_R < sigma_E
+    lap = si.flat_iid(1 << 18, 12, "laplace")
+    st = oracle.stats(lap)
+    _, res, _, _ = oracle.ds_search(lap, st, 2, 0x20, 100, 256)
+    assert res.b_r < res.b_e and res.b_r <= res.b_star <= res.b_e
+    # the literal-formula scale has no Gaussian counterpart; flags combine with the mid-rise grid
+    assert oracle.ds_search(lap, st, 2, 0x21)[0] == oracle.ERR_ARG
+    rc, res_m, qp_m, _ = oracle.ds_search(lap, st, 2, 0x30, 100, 256)
+    assert rc == 0 and res_m.b_e == res.b_e and res_m.b_r == res.b_r
+
+
 def test_ds_degenerate_and_arguments():
     c = np.full(100, 2.5, dtype=np.float32)
     st = oracle.stats(c)
