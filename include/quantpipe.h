@@ -53,6 +53,7 @@ enum { QP_F32 = 0, QP_BF16 = 1 };
 enum { QP_DIST_LAPLACE = 0, QP_DIST_GAUSS = 1 };
 enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the formula as printed */ };
 #define QP_B_MIDRISE 0x10  /* qp_dsaciq_search: bmode | QP_B_MIDRISE scores every candidate on the mid-rise grid */
+#define QP_B_GAUSS 0x20    /* qp_dsaciq_search: QP_B_MAD | QP_B_GAUSS searches under the normal model (see there) */
 
 #define QP_DEFAULT_STEPS 100      /* search steps t (Sec. 3, directed search) */
 #define QP_DEFAULT_HIST_BINS 100
@@ -217,6 +218,11 @@ int32_t qp_clip_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits,
  * Writes *d_out (optional) and the winning quantizer *d_qp_out (optional); both device
  * memory.  bits 1..8; 1 <= steps <= QP_MAX_STEPS; 1 <= hist_bins <= QP_MAX_HIST_BINS;
  * bmode QP_B_MAD or QP_B_MEAN_ABS, optionally | QP_B_MIDRISE.
+ * QP_B_MAD | QP_B_GAUSS (optionally | QP_B_MIDRISE) runs the same search under the normal
+ * model that ACIQ also offers (the paper searches under the Laplace model only): the scale is
+ * the standard deviation, sigma_E = sqrt(var); a normal density peaks at 1 / (sigma sqrt(2 pi)),
+ * so sigma_R = 1 / (sqrt(2 pi) * peak density); the clip is F_gauss(bits) * sigma_k.  The
+ * result's b_e, b_r, b_star then hold sigma_E, sigma_R, sigma*.
  * Errors: as qp_stats, plus QP_ERR_UNSUPPORTED_BITS. */
 int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                          int bits, int bmode, int steps, int hist_bins,

@@ -29,6 +29,7 @@ QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
 QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT, QP_CLIP_MIDRISE = 0, 1, 2, 0x10, 0x20
 QP_B_MIDRISE = 0x10
+QP_B_GAUSS = 0x20
 
 EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",

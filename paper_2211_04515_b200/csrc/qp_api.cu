@@ -516,6 +516,8 @@ extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n,
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const unsigned long long key[8] = {1, (unsigned long long)(uintptr_t)d_x, (unsigned long long)dtype, n,
                                        (unsigned long long)hist_bins, (unsigned long long)(uintptr_t)d_out, 0, 0};
+    ctx->last_x = d_x;                    // the second pass walks backwards (the plain kernels for small tensors do not,
+    ctx->last_x_end = 0;                  // but those tensors sit in L2 whole)
     return qp_graphed(ctx, s, key, [&] { return qp_launch_stats(ctx, d_x, dtype, n, hist_bins, d_out, s); });
 }
 
@@ -556,8 +558,11 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
     if (rc) return rc;
     if (!d_stats) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_stats");
     if (bits < 1 || bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
-    if ((bmode & ~QP_B_MIDRISE) != QP_B_MAD && (bmode & ~QP_B_MIDRISE) != QP_B_MEAN_ABS)
-        return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
+    {
+        const int base = bmode & ~(QP_B_MIDRISE | QP_B_GAUSS);
+        if ((base != QP_B_MAD && base != QP_B_MEAN_ABS) || ((bmode & QP_B_GAUSS) && base != QP_B_MAD))
+            return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
+    }
     if (steps < 1 || steps > QP_MAX_STEPS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "steps out of range");
     if (hist_bins < 1 || hist_bins > QP_MAX_HIST_BINS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "hist_bins out of range");
     if (((uintptr_t)d_out & 7u) || ((uintptr_t)d_qp_out & 3u)) return qp_fail(ctx, QP_ERR_ALIGNMENT, "result pointers");
@@ -571,9 +576,12 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
                                        (unsigned long long)(uintptr_t)d_out, (unsigned long long)(uintptr_t)d_qp_out, 0};
     rc = qp_graphed(ctx, s, key, [&] {
         return qp_launch_search(ctx, d_x, dtype, n, d_stats, bits, bmode, steps, hist_bins,
-                                qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_out, d_qp_out, s);
+                                qp_host_aciq_F(bits, (bmode & QP_B_GAUSS) ? QP_DIST_GAUSS : QP_DIST_LAPLACE), d_out,
+                                d_qp_out, s);
     });
     if (rc == QP_OK) ctx->last_steps = steps;
+    ctx->last_x = d_x;                    // both scoring paths walk x forwards
+    ctx->last_x_end = 1;
     return rc;
 }
 

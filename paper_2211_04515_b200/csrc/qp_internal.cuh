@@ -90,6 +90,8 @@ struct qp_ctx {
     unsigned long long graph_hits;       // calls served by replaying a stored graph
     qp_graph_entry graphs[QP_GRAPH_SLOTS];
     int last_steps;                      // steps of the last search (for qp_dsaciq_curve)
+    const void* last_x;                  // tensor of the last full pass on this context and where that pass
+    int last_x_end;                      // stopped (1 = at the end of the tensor): the next pass starts there (L2)
     char err[256];
 };
 
@@ -277,7 +279,8 @@ __device__ inline void qp_ds_make_setup(const qp_stats_t* __restrict__ st, unsig
 {
     const unsigned long long nf = st->n - st->nonfinite;
     const double mn = st->min, mx = st->max;
-    const double b_e = (bmode & 0xF) == QP_B_MEAN_ABS ? st->mean_abs : st->mad;
+    const bool gauss = (bmode & QP_B_GAUSS) != 0;       // normal model: scale = standard deviation
+    const double b_e = gauss ? sqrt(st->var) : ((bmode & 0xF) == QP_B_MEAN_ABS ? st->mean_abs : st->mad);
     double peak = 0.0;
     if (mx > mn && nf > 0) {
         const double w = (mx - mn) / (double)nb;
@@ -285,7 +288,8 @@ __device__ inline void qp_ds_make_setup(const qp_stats_t* __restrict__ st, unsig
     }
     s.degenerate = !(mx > mn) || !(peak > 0.0) || !(b_e > 0.0);
     s.b_e = b_e;
-    s.b_r = s.degenerate ? b_e : 1.0 / (2.0 * peak);
+    // the model's density peaks at 1 / (factor * scale): factor 2 (Laplace) or sqrt(2 pi) (normal)
+    s.b_r = s.degenerate ? b_e : 1.0 / ((gauss ? 2.5066282746310002 : 2.0) * peak);
     s.F = F;
     s.mean = st->mean;
     s.n_finite = nf;

@@ -53,7 +53,8 @@ __device__ __forceinline__ unsigned quad_of(const float* e, const QP4& q)
 template <int BITS, typename T>
 __global__ void __launch_bounds__(QP_THREADS) pack_kernel(const T* __restrict__ x, uint64_t ntiles,
                                                           const qp_qparams_t* __restrict__ d_qp, qp_qparams_t h_qp,
-                                                          uint32_t* __restrict__ out, unsigned* __restrict__ status)
+                                                          uint32_t* __restrict__ out, unsigned* __restrict__ status,
+                                                          int reverse)
 {
     constexpr int EPV = qp_span<T>::EPV;          // 4 (f32) or 8 (bf16) elements per 16-byte vector
     constexpr int NLOAD = TILE / (32 * EPV);      // 8 or 4 vector loads per lane
@@ -63,7 +64,10 @@ __global__ void __launch_bounds__(QP_THREADS) pack_kernel(const T* __restrict__ 
     uint32_t* sw = stage[warp];
     const uint64_t wstride = (uint64_t)gridDim.x * WARPS;
 
-    for (uint64_t tile = (uint64_t)blockIdx.x * WARPS + warp; tile < ntiles; tile += wstride) {
+    // `reverse`: the grid walks the tensor from its end (the tiles are the same), for a call that
+    // follows a pass which ended there and left that part of x in L2
+    for (uint64_t it = (uint64_t)blockIdx.x * WARPS + warp; it < ntiles; it += wstride) {
+        const uint64_t tile = reverse ? ntiles - 1 - it : it;
         const T* xt = x + tile * TILE;
         float e[NLOAD][EPV];
 #pragma unroll
@@ -194,12 +198,16 @@ int32_t pack_typed(qp_ctx* ctx, const T* x, uint64_t n, int bits, const qp_qpara
     }
     const uint64_t ntiles = aligned ? n / TILE : 0;
     uint32_t* out = static_cast<uint32_t*>(d_packed);
+    // a hint, not a dependency: start where the last pass over this tensor stopped
+    const int reverse = (ctx->last_x == static_cast<const void*>(x) && ctx->last_x_end) ? 1 : 0;
+    ctx->last_x = x;
+    ctx->last_x_end = reverse ? 0 : 1;
     if (ntiles) {
         uint64_t want = (ntiles + WARPS - 1) / WARPS;
         const uint64_t cap = (uint64_t)ctx->sm_count * 64;
         const int blocks = (int)(want > cap ? cap : want);
         ctx->launches += 1;
-#define QP_PACK_CASE(B) case B: pack_kernel<B, T><<<blocks, QP_THREADS, 0, s>>>(x, ntiles, d_qp, h_qp, out, ctx->d_status); break;
+#define QP_PACK_CASE(B) case B: pack_kernel<B, T><<<blocks, QP_THREADS, 0, s>>>(x, ntiles, d_qp, h_qp, out, ctx->d_status, reverse); break;
         switch (bits) {
             QP_PACK_CASE(1) QP_PACK_CASE(2) QP_PACK_CASE(3) QP_PACK_CASE(4)
             QP_PACK_CASE(5) QP_PACK_CASE(6) QP_PACK_CASE(7) QP_PACK_CASE(8)

@@ -402,7 +402,23 @@ def test_search_midrise_grid(ctx, bits, path):
     y = si.vit_activation((5, 197, 200), 55, outlier_frac=0.02).reshape(-1)
     check_search(ctx, y, dev(y), bits, bmode=qp.QP_B_MEAN_ABS | qp.QP_B_MIDRISE, path=path)
     with pytest.raises(qp.QuantPipeError):
-        ctx.qp_dsaciq_search(dev(y), ctx.qp_stats(dev(y)), bits, 0x20)
+        ctx.qp_dsaciq_search(dev(y), ctx.qp_stats(dev(y)), bits, 0x40)
+
+
+@pytest.mark.parametrize("path", BOTH_PATHS)
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
+def test_search_gaussian_model(ctx, bits, path):
+    """QP_B_GAUSS: scale = standard deviation, sigma_R from the normal density's peak, F of the normal model."""
+    x = si.config_tensor("c1").reshape(-1)
+    res, res_o = check_search(ctx, x, dev(x), bits, bmode=qp.QP_B_GAUSS, path=path)
+    plain, _ = check_search(ctx, x, dev(x), bits, path=path)
+    st_o = oracle.stats(x)
+    assert abs(res.b_e - np.sqrt(st_o.var)) <= 1e-5 * res.b_e
+    assert abs(res.b_r / plain.b_r - 2.0 / np.sqrt(2.0 * np.pi)) <= 1e-9      # the same peak count, another model
+    g = (0.3 + 0.7 * si.flat_iid(200003, 17, "normal")).astype(np.float32)     # normal data, ragged size
+    check_search(ctx, g, dev(g), bits, bmode=qp.QP_B_GAUSS | qp.QP_B_MIDRISE, nb=256, path=path)
+    with pytest.raises(qp.QuantPipeError):                                     # the printed formula has no normal form
+        ctx.qp_dsaciq_search(dev(g), ctx.qp_stats(dev(g)), bits, qp.QP_B_MEAN_ABS | qp.QP_B_GAUSS)
 
 
 @pytest.mark.parametrize("path", BOTH_PATHS)
