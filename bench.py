@@ -218,6 +218,7 @@ def ours_main(args):
     d_res = torch.empty(72, dtype=torch.uint8, device="cuda")
     torch.cuda.synchronize()
 
+    assert all(qp.qp_stats_carries_histogram(x, qp.QP_DEFAULT_HIST_BINS) for x in xs)
     stage_names = ("stats", "clip", "quantize_pack", "unpack_dequantize")
     STAGE_EVERY = 3 if args.steps >= 60 else 1          # coprime with the 100-step trace: every bit-width is sampled
 
@@ -233,8 +234,8 @@ def ours_main(args):
         ctx.qp_stats(x, out=d_stats, hist_bins=qp.QP_DEFAULT_HIST_BINS if use_ds else 0)
         if events is not None:
             marks[1].record()
-        if use_ds:
-            ctx.qp_dsaciq_search(x, d_stats, q, out_result=d_res, out_qp=d_qp)
+        if use_ds:      # the statistics just written carry the histogram (checked once below): the search need not look
+            ctx.qp_dsaciq_search(x, d_stats, q, bmode=qp.QP_B_MAD | qp.QP_B_HIST_IN_STATS, out_result=d_res, out_qp=d_qp)
         else:
             ctx.qp_aciq_qparams_device(d_stats, q, out=d_qp)
         if events is not None:

@@ -54,6 +54,7 @@ enum { QP_DIST_LAPLACE = 0, QP_DIST_GAUSS = 1 };
 enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the formula as printed */ };
 #define QP_B_MIDRISE 0x10  /* qp_dsaciq_search: bmode | QP_B_MIDRISE scores every candidate on the mid-rise grid */
 #define QP_B_GAUSS 0x20    /* qp_dsaciq_search: QP_B_MAD | QP_B_GAUSS searches under the normal model (see there) */
+#define QP_B_HIST_IN_STATS 0x40  /* qp_dsaciq_search: the caller vouches that d_stats carries this histogram (see there) */
 
 #define QP_DEFAULT_STEPS 100      /* search steps t (Sec. 3, directed search) */
 #define QP_DEFAULT_HIST_BINS 100
@@ -65,6 +66,7 @@ enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the form
 #define QP_DEV_DEGENERATE 2u
 #define QP_DEV_NONFINITE 4u
 #define QP_DEV_STREAM_TIMEOUT 8u  /* a bounded wait for a tile copy ran out; results of that call are invalid */
+#define QP_DEV_HIST_MISSING 16u   /* a search was promised a histogram in the statistics (QP_B_HIST_IN_STATS) that is not there */
 
 /* Per-tensor statistics (Sec. 3: min/max of naive PTQ; mean and Laplace scale b of ACIQ;
  * b_E of the directed search).  All fields but n are over the finite elements. */
@@ -149,6 +151,10 @@ int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out);
  * QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
 int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
                  void* stream);
+/* 1 if qp_stats with these arguments carries the histogram along (so that d_out->hist_bins
+ * will equal hist_bins), else 0.  Host, pure: it depends only on the pointer's alignment, the
+ * size and hist_bins. */
+int qp_stats_carries_histogram(const void* d_x, int dtype, uint64_t n, int hist_bins);
 
 /* Statistics for callers that cannot allocate device memory (no counterpart in the paper;
  * same results as qp_stats).  Some code may not call cudaMalloc or any allocating routine:
@@ -223,6 +229,11 @@ int32_t qp_clip_qparams_device(qp_ctx* ctx, const qp_stats_t* d_stats, int bits,
  * the standard deviation, sigma_E = sqrt(var); a normal density peaks at 1 / (sigma sqrt(2 pi)),
  * so sigma_R = 1 / (sqrt(2 pi) * peak density); the clip is F_gauss(bits) * sigma_k.  The
  * result's b_e, b_r, b_star then hold sigma_E, sigma_R, sigma*.
+ * The call first checks on the device whether d_stats already carries the peak of this
+ * histogram (qp_stats with the same hist_bins) and counts for itself if not; that check is a
+ * memset and a kernel launch.  bmode | QP_B_HIST_IN_STATS skips them: the caller vouches that
+ * d_stats came from qp_stats(x, hist_bins) with qp_stats_carries_histogram() = 1.  If it did
+ * not, QP_DEV_HIST_MISSING is raised in the status word and the search keeps b_E (k* = 0).
  * Errors: as qp_stats, plus QP_ERR_UNSUPPORTED_BITS. */
 int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                          int bits, int bmode, int steps, int hist_bins,

@@ -23,19 +23,20 @@ QP_WARN_INFEASIBLE, QP_WARN_DEGENERATE, QP_WARN_NONFINITE = 1, 2, 3
 QP_F32, QP_BF16 = 0, 1
 QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
 QP_B_MAD, QP_B_MEAN_ABS = 0, 1
-QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT = 1, 2, 4, 8
+QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT, QP_DEV_HIST_MISSING = 1, 2, 4, 8, 16
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS = 0, 1, 2
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
 QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT, QP_CLIP_MIDRISE = 0, 1, 2, 0x10, 0x20
 QP_B_MIDRISE = 0x10
 QP_B_GAUSS = 0x20
+QP_B_HIST_IN_STATS = 0x40
 
 EXPORTS = (
     "qp_create", "qp_destroy", "qp_get_status", "qp_last_error", "qp_status_string", "qp_packed_bytes",
     "qp_aciq_F", "qp_make_qparams", "qp_stats", "qp_aciq_alpha", "qp_aciq_qparams_device", "qp_dsaciq_search",
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
-    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_controller_init", "qp_controller_observe",
+    "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_stats_carries_histogram", "qp_controller_init", "qp_controller_observe",
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
     "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_clip_qparams_channels_device",
     "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range", "qp_sender_channels_device",
@@ -122,6 +123,8 @@ def load() -> C.CDLL:
     L.qp_select_bits_eq2.argtypes = [dbl, C.c_int, dbl, dbl, dbl, C.POINTER(i32)]
     L.qp_stats_static.argtypes = [vp, C.c_int, u64, vp, vp]
     L.qp_set_search_path.argtypes = [vp, C.c_int]
+    L.qp_stats_carries_histogram.argtypes = [vp, C.c_int, u64, C.c_int]
+    L.qp_stats_carries_histogram.restype = C.c_int
     L.qp_set_graph_replay.argtypes = [vp, C.c_int]
     L.qp_set_sender_path.argtypes = [vp, C.c_int]
     L.qp_graph_replays.argtypes = [vp]
@@ -185,6 +188,10 @@ def qp_midrise_range(lo: float, hi: float, bits: int):
     a, b = C.c_double(), C.c_double()
     rc = load().qp_midrise_range(lo, hi, bits, C.byref(a), C.byref(b))
     return int(rc), a.value, b.value
+
+
+def qp_stats_carries_histogram(x: torch.Tensor, hist_bins: int) -> bool:
+    return bool(load().qp_stats_carries_histogram(x.data_ptr(), _dtype_code(x), x.numel(), hist_bins))
 
 
 def qp_policy_use_ds(bits: int) -> bool:

@@ -559,7 +559,7 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
     if (!d_stats) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_stats");
     if (bits < 1 || bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
     {
-        const int base = bmode & ~(QP_B_MIDRISE | QP_B_GAUSS);
+        const int base = bmode & ~(QP_B_MIDRISE | QP_B_GAUSS | QP_B_HIST_IN_STATS);
         if ((base != QP_B_MAD && base != QP_B_MEAN_ABS) || ((bmode & QP_B_GAUSS) && base != QP_B_MAD))
             return qp_fail(ctx, QP_ERR_INVALID_ARG, "bmode");
     }
@@ -691,7 +691,9 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
     }
     rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
     if (rc < 0) return rc;
-    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, search_mode, steps, hist_bins, nullptr, d_qp_out, stream);
+    // the statistics above carry the histogram whenever they can: then the search need not look
+    const int in_stats = (use_ds && qp_stats_carries_histogram(d_x, dtype, n, hist_bins)) ? QP_B_HIST_IN_STATS : 0;
+    if (use_ds) rc = qp_dsaciq_search(ctx, d_x, dtype, n, st, bits, search_mode | in_stats, steps, hist_bins, nullptr, d_qp_out, stream);
     else        rc = qp_clip_qparams_device(ctx, st, bits, method, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
     if (rc < 0) return rc;
     return qp_quantize_pack(ctx, d_x, dtype, n, bits, d_qp_out, 1, d_packed, packed_capacity, stream);

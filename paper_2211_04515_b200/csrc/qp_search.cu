@@ -82,13 +82,16 @@ __global__ void __launch_bounds__(QP_THREADS) hist_kernel(const T* __restrict__ 
 __global__ void __launch_bounds__(QP_THREADS) setup_kernel(const qp_stats_t* __restrict__ st,
                                                            const unsigned long long* __restrict__ hist, int nb, int bits,
                                                            int bmode, int steps, double F, float4* __restrict__ cand,
-                                                           int* __restrict__ valid, qp_ds_setup* __restrict__ setup)
+                                                           int* __restrict__ valid, qp_ds_setup* __restrict__ setup,
+                                                           unsigned* __restrict__ status)
 {
     __shared__ unsigned long long sh_top[QP_THREADS];
     __shared__ qp_ds_setup s;
     unsigned long long top = 0;
     const bool from_stats = st->hist_bins == nb;
-    for (int b = threadIdx.x; !from_stats && b < nb; b += QP_THREADS) {
+    const bool promised = (bmode & QP_B_HIST_IN_STATS) != 0;      // then nobody has counted into hist
+    if (promised && !from_stats && threadIdx.x == 0) atomicOr(status, QP_DEV_HIST_MISSING);
+    for (int b = threadIdx.x; !from_stats && !promised && b < nb; b += QP_THREADS) {
         const unsigned long long c = hist[b];
         top = c > top ? c : top;
     }
@@ -266,11 +269,13 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     uint64_t want = (n + per_block - 1) / per_block;
     const uint64_t hcap = (uint64_t)ctx->sm_count * 3;
     const int hblocks = (int)(want < 1 ? 1 : (want > hcap ? hcap : want));
-    // returns at once when the statistics already carry this histogram's peak
-    if (cudaMemsetAsync(ctx->d_hist, 0, sizeof(unsigned long long) * nb, s) != cudaSuccess)
-        return qp_check_launch(ctx, "qp_dsaciq_search (histogram reset)");
-    hist_kernel<T><<<hblocks, QP_THREADS, sh_bytes, s>>>(x, n, d_stats, nb, rep_shift, ctx->d_hist);
-    ctx->launches += 1;
+    if (!(bmode & QP_B_HIST_IN_STATS)) {
+        // returns at once when the statistics already carry this histogram's peak
+        if (cudaMemsetAsync(ctx->d_hist, 0, sizeof(unsigned long long) * nb, s) != cudaSuccess)
+            return qp_check_launch(ctx, "qp_dsaciq_search (histogram reset)");
+        hist_kernel<T><<<hblocks, QP_THREADS, sh_bytes, s>>>(x, n, d_stats, nb, rep_shift, ctx->d_hist);
+        ctx->launches += 1;
+    }
 
     const int ncand = steps + 1;
     // interval-moment scoring where its tables fit and its fixed-point sums cannot overflow
@@ -282,7 +287,7 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
         return qp_launch_interval_search(ctx, x, sizeof(T) == 4 ? QP_F32 : QP_BF16, n, d_stats, bits, bmode, steps, nb, F,
                                          d_out, d_qp_out, s);
     setup_kernel<<<1, QP_THREADS, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
-                                          ctx->d_setup);
+                                          ctx->d_setup, ctx->d_status);
     const int groups = (ncand + K - 1) / K;
     const uint64_t per_chunk = (uint64_t)QP_THREADS * 8;
     want = (n + per_chunk - 1) / per_chunk;

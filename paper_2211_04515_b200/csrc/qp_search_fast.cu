@@ -89,7 +89,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
                                                         const unsigned long long* __restrict__ hist, int nb, int bits,
                                                         int bmode, int steps, double F, float4* __restrict__ cand,
                                                         int* __restrict__ valid, qp_ds_setup* __restrict__ setup,
-                                                        float* __restrict__ bnd)
+                                                        float* __restrict__ bnd, unsigned* __restrict__ status)
 {
     __shared__ unsigned long long s_top[8];
     __shared__ float s_lo[8], s_hi[8];
@@ -103,7 +103,9 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
 
     unsigned long long top = 0;
     const bool from_stats = st->hist_bins == nb;
-    for (int b = threadIdx.x; !from_stats && b < nb; b += 256) {
+    const bool promised = (bmode & QP_B_HIST_IN_STATS) != 0;      // then nobody has counted into hist
+    if (promised && !from_stats && blockIdx.x == 0 && threadIdx.x == 0) atomicOr(status, QP_DEV_HIST_MISSING);
+    for (int b = threadIdx.x; !from_stats && !promised && b < nb; b += 256) {
         const unsigned long long c = hist[b];
         top = c > top ? c : top;
     }
@@ -563,7 +565,7 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
-                                                ctx->d_setup, ctx->d_iv_bnd);
+                                                ctx->d_setup, ctx->d_iv_bnd, ctx->d_status);
     unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]
     iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ncand * L1, ctx->d_iv_bb,
                                                             ctx->d_iv_first);

@@ -510,6 +510,14 @@ int32_t launch_typed(qp_ctx* ctx, const T* x, uint64_t n, qp_stats_t* d_out, cud
 
 }  // namespace
 
+extern "C" int qp_stats_carries_histogram(const void* d_x, int dtype, uint64_t n, int hist_bins)
+{
+    if (dtype != QP_F32 && dtype != QP_BF16) return 0;
+    // the streamed kernels (aligned, at least 8 tiles) with a histogram small enough to ride along
+    const uint64_t ntiles = ((uintptr_t)d_x & 15u) ? 0 : n * (dtype == QP_F32 ? 4 : 2) / ST_TILE;
+    return (ntiles >= 8 && hist_bins >= 1 && hist_bins <= ST_FUSED_HIST_MAX) ? 1 : 0;
+}
+
 int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_bins, qp_stats_t* d_out,
                         cudaStream_t s)
 {

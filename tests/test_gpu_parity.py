@@ -402,7 +402,7 @@ def test_search_midrise_grid(ctx, bits, path):
     y = si.vit_activation((5, 197, 200), 55, outlier_frac=0.02).reshape(-1)
     check_search(ctx, y, dev(y), bits, bmode=qp.QP_B_MEAN_ABS | qp.QP_B_MIDRISE, path=path)
     with pytest.raises(qp.QuantPipeError):
-        ctx.qp_dsaciq_search(dev(y), ctx.qp_stats(dev(y)), bits, 0x40)
+        ctx.qp_dsaciq_search(dev(y), ctx.qp_stats(dev(y)), bits, 0x80)
 
 
 @pytest.mark.parametrize("path", BOTH_PATHS)
@@ -419,6 +419,35 @@ def test_search_gaussian_model(ctx, bits, path):
     check_search(ctx, g, dev(g), bits, bmode=qp.QP_B_GAUSS | qp.QP_B_MIDRISE, nb=256, path=path)
     with pytest.raises(qp.QuantPipeError):                                     # the printed formula has no normal form
         ctx.qp_dsaciq_search(dev(g), ctx.qp_stats(dev(g)), bits, qp.QP_B_MEAN_ABS | qp.QP_B_GAUSS)
+
+
+@pytest.mark.parametrize("path", BOTH_PATHS)
+def test_search_histogram_promise(ctx, path):
+    """QP_B_HIST_IN_STATS: no histogram pass of its own, same result; a broken promise is reported."""
+    x = si.vit_activation((8, 197, 256), 21).reshape(-1)              # 1.6 MB: the statistics carry the histogram
+    d = dev(x)
+    assert qp.qp_stats_carries_histogram(d, 100) and not qp.qp_stats_carries_histogram(d[1:], 100)
+    assert not qp.qp_stats_carries_histogram(d, 8192) and not qp.qp_stats_carries_histogram(d[:1000], 100)
+    ctx.qp_set_search_path(path)
+    try:
+        d_stats = ctx.qp_stats(d, hist_bins=100)
+        n0 = ctx.qp_launch_count()
+        d_res, d_qp = ctx.qp_dsaciq_search(d, d_stats, 2, qp.QP_B_MAD, 100, 100)
+        n1 = ctx.qp_launch_count()
+        d_res2, d_qp2 = ctx.qp_dsaciq_search(d, d_stats, 2, qp.QP_B_MAD | qp.QP_B_HIST_IN_STATS, 100, 100)
+        n2 = ctx.qp_launch_count()
+        assert bytes(ctx.read_ds_result(d_res)) == bytes(ctx.read_ds_result(d_res2))
+        assert bytes(ctx.read_qparams(d_qp)) == bytes(ctx.read_qparams(d_qp2))
+        assert (n1 - n0) - (n2 - n1) == 1                              # one launch fewer
+        assert ctx.qp_get_status() == 0
+        # statistics without the histogram, yet the promise: reported, and b_E is kept
+        d_plain = ctx.qp_stats(d, hist_bins=0)
+        d_res3, _ = ctx.qp_dsaciq_search(d, d_plain, 2, qp.QP_B_MAD | qp.QP_B_HIST_IN_STATS, 100, 100)
+        res3 = ctx.read_ds_result(d_res3)
+        assert ctx.qp_get_status() & qp.QP_DEV_HIST_MISSING
+        assert res3.k_star == 0 and res3.b_star == res3.b_e
+    finally:
+        ctx.qp_set_search_path(qp.QP_SEARCH_AUTO)
 
 
 @pytest.mark.parametrize("path", BOTH_PATHS)
