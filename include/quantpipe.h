@@ -242,10 +242,14 @@ int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
  * (to ~1e-8 relative) and the same winner.
  *   QP_SEARCH_CANDIDATES  every element is quantized under every candidate (any bits/steps)
  *   QP_SEARCH_INTERVALS   one pass gathers moments per interval between the candidates'
- *                         decision thresholds; used where (steps+1)*(2^bits-1) <= 2048 and
- *                         n < ~1.2e9, otherwise the call falls back to the first way
- *   QP_SEARCH_AUTO        intervals for n >= 2^20 where they apply (default) */
-enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2 };
+ *                         decision thresholds; used where (steps+1)*(2^bits-1) <= 3584 and
+ *                         n < ~0.9e9, otherwise the call falls back to the first way
+ *   QP_SEARCH_AUTO        intervals for n >= 2^20 where they apply (default)
+ * The pass over x that gathers the moments has two forms with identical results: the plain one
+ * (every element looks its interval up), and one that adds elements of grid cells without a
+ * threshold straight into per-cell, per-lane sums and looks up only the others; the second is
+ * used up to ~150 M elements, QP_SEARCH_INTERVALS_PLAIN forces the first. */
+enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2, QP_SEARCH_INTERVALS_PLAIN = 3 };
 int32_t qp_set_search_path(qp_ctx* ctx, int path);
 /* Graph replay of the multi-kernel calls (an execution option; the paper has no counterpart,
  * results are unchanged).  With on = 1, qp_stats, qp_dsaciq_search and qp_sender_device

@@ -163,8 +163,9 @@ extern "C" uint64_t qp_launch_count(qp_ctx* ctx) { return ctx ? ctx->launches : 
 extern "C" int32_t qp_set_search_path(qp_ctx* ctx, int path)
 {
     if (!ctx) return QP_ERR_INVALID_ARG;
-    if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
-    ctx->search_path = path;
+    if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS_PLAIN) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
+    ctx->moments_form = path == QP_SEARCH_INTERVALS_PLAIN ? 1 : 0;
+    ctx->search_path = path == QP_SEARCH_INTERVALS_PLAIN ? QP_SEARCH_INTERVALS : path;
     return QP_OK;
 }
 
@@ -571,7 +572,7 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const unsigned long long key[8] = {2, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_stats,
                                        (unsigned long long)dtype | (unsigned long long)bits << 8 |
-                                           (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
+                                           (unsigned long long)bmode << 16 | (unsigned long long)(ctx->search_path | ctx->moments_form << 2) << 24 |
                                            (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
                                        (unsigned long long)(uintptr_t)d_out, (unsigned long long)(uintptr_t)d_qp_out, 0};
     rc = qp_graphed(ctx, s, key, [&] {
@@ -715,7 +716,7 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
     // The inner calls see a capturing stream while this one records, and enqueue directly into it.
     const unsigned long long key[8] = {3, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_packed,
                                        (unsigned long long)dtype | (unsigned long long)bits << 8 |
-                                           (unsigned long long)bmode << 16 | (unsigned long long)ctx->search_path << 24 |
+                                           (unsigned long long)bmode << 16 | (unsigned long long)(ctx->search_path | ctx->moments_form << 2) << 24 |
                                            (unsigned long long)((method & 0xF) == QP_CLIP_DSACIQ) << 28 | (unsigned long long)method << 56 |
                                            (unsigned long long)ctx->sender_path << 29 |
                                            (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,

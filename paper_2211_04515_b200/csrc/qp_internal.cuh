@@ -34,7 +34,7 @@ struct qp_ds_setup {                     // written by the search's set-up kerne
     double u;
 };
 
-constexpr int QP_IV_CELLS = 2048;        // uniform cells over [g_lo, g_hi]
+constexpr int QP_IV_CELLS = 512;         // uniform cells over [g_lo, g_hi]
 constexpr int QP_IV_MAXB = 4096;         // most interval boundaries (candidate thresholds + cell edges)
 constexpr int QP_IV_THREADS = 512;
 constexpr int QP_IV_BLOCKS_PER_SM = 3;
@@ -73,6 +73,7 @@ struct qp_ctx {
     qp_iv_total* d_iv_tot;               // [QP_IV_MAXB + 1]
     int iv_blocks;                       // blocks of the interval-moment kernel (fixed per context)
     int search_path;                     // 0 auto, 1 candidate scoring, 2 interval moments
+    int moments_form;                    // interval moments: 0 auto (second form where it applies), 1 always the first form
     int sender_path;                     // 0 auto, 1 kernel chain, 2 single cooperative launch where it applies
     int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
     size_t fused_dyn_max;                // largest slice (bytes of dynamic shared memory) per block

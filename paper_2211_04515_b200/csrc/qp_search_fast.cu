@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
             inv_gw = (float)((double)G / width);
             int e;
             frexp(width / (double)G, &e);               // cell width in [2^(e-1), 2^e)
-            u = ldexp(1.0, e - 16);                     // offsets (up to ~1.5 cells) stay below 2^17.6 units
+            u = ldexp(1.0, e - 18);                     // offsets (up to ~1.5 cells) stay below 1.5 * 2^18 units
         }
         sg_lo = lo; sg_hi = hi; sg_inv = inv_gw;
         if (blockIdx.x == 0) {
@@ -418,6 +418,235 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
     }
 }
 
+// ---------------------------------------------------------------- moments, second form
+//
+// Same result as iv_moments_kernel (the same per-block rows of count << 40 | sum of offsets,
+// the same outer sums), gathered with less work per element.  Most grid cells hold no
+// threshold: such a cell is one interval, and its two sums need neither the table look-up nor
+// the search.  They are kept in a table indexed by cell and LANE (32 replicas of every cell, so
+// a warp's 32 atomics always hit 32 different banks and elements of one value never queue up
+// behind one counter).  Cells that do hold thresholds ("split" cells) carry a mark in the top
+// bit of their replica counters; the counter's old value, which the atomic returns anyway,
+// tells the thread that its element needs the exact treatment.  Those elements are not
+// handled on the spot (a warp would run the whole search for a few active lanes): each warp
+// collects them in a small buffer of its own and works them off 32 at a time with all lanes
+// busy, through the same cell table, search and interval sums as the first form.
+// One block of 1024 threads per SM (the replica table takes 131 KB).
+constexpr int IV2_THREADS = 1024;
+constexpr int IV2_WARPS = IV2_THREADS / 32;
+constexpr int IV2_STAGE = 64;                        // buffered elements per warp (worked off from 32 on)
+constexpr unsigned IV2_SPLIT = 0x80000000u;
+// replica sums are 32 bit: elements per block * largest offset (1.5 * 2^18 units) / 32 replicas < 2^32
+constexpr uint64_t IV2_MAX_PER_BLOCK = 340000;
+
+struct Iv2Shared {
+    unsigned* rcnt;                 // [(G + 1) * 32] per cell and lane: count (| IV2_SPLIT in split cells)
+    unsigned* rs1;                  // [(G + 1) * 32] per cell and lane: sum of offsets
+    float* stage;                   // [IV2_WARPS][IV2_STAGE]
+};
+
+// exact treatment of one clamped, finite element of a split cell: as iv_one without the sums
+// that the fast path has already taken
+__device__ __forceinline__ void iv2_exact(float x, const IvShared& sh, const IvConst& k)
+{
+    const float pm = cell_pm(x, k.g_lo, k.inv_gw);
+    const unsigned ci = sh.cell[__float_as_uint(pm) & 0x7FFFFFu];
+    unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
+    while (lo < hi) {                                   // largest i in [lo, hi] with bb[i] <= x
+        const unsigned mid = (lo + hi + 1u) >> 1;
+        if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
+    }
+    const float dm = fmaf(__fsub_rn(x, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
+    const unsigned d1 = __float_as_uint(dm) & 0x7FFFFFu;
+    atomicAdd(&sh.cnt[lo], 1u);
+    const unsigned old = atomicAdd(&sh.s1[lo], d1);
+    if (old + d1 < old) atomicAdd(&sh.cnt[lo], 1u << 24);
+}
+
+// One element: clamp, outer sums, cell, offset, the two replica atomics.  If its cell turns out to
+// be split it goes into the warp's buffer; from 32 buffered elements on, the warp works 32 of
+// them off with every lane busy.  Called by all 32 lanes together (lanes without an element pass
+// a non-finite value to the guarded form).
+template <bool GUARD>
+__device__ __forceinline__ void iv2_one(float x, const IvShared& sh, const Iv2Shared& s2, const IvConst& k, IvBatch& b,
+                                        float* my_stage, unsigned& staged, unsigned lane)
+{
+    const unsigned full = 0xFFFFFFFFu;
+    bool split = false;
+    float xc = x;
+    if (!GUARD || qp_is_finite(x)) {
+        xc = fminf(fmaxf(x, k.g_lo), k.g_hi);
+        const float e = __fsub_rn(x, xc);
+        b.s1 += e; b.s1a += fabsf(e); b.s2 = fmaf(e, e, b.s2);
+        const float pm = cell_pm(xc, k.g_lo, k.inv_gw);
+        const float dm = fmaf(__fsub_rn(xc, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
+        const float d1f = __fsub_rn(dm, IV_MAGIC);
+        b.s2_in = fmaf(d1f, d1f, b.s2_in);
+        const unsigned idx = ((__float_as_uint(pm) & 0x7FFFFFu) << 5) + lane;
+        const unsigned old = atomicAdd(&s2.rcnt[idx], 1u);
+        atomicAdd(&s2.rs1[idx], __float_as_uint(dm) & 0x7FFFFFu);     // ignored later if the cell is split
+        split = (old & IV2_SPLIT) != 0u;
+    }
+    const unsigned m = __ballot_sync(full, split);
+    if (m) {                                             // warp-uniform
+        if (split) my_stage[staged + __popc(m & ((1u << lane) - 1u))] = xc;
+        staged += __popc(m);
+        if (staged >= 32u) {
+            __syncwarp();
+            staged -= 32u;
+            iv2_exact(my_stage[staged + lane], sh, k);
+            __syncwarp();
+        }
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __restrict__ x, uint64_t n,
+                                                                     const qp_stats_t* __restrict__ st,
+                                                                     const qp_ds_setup* __restrict__ setup,
+                                                                     const float* __restrict__ g_bb,
+                                                                     const unsigned* __restrict__ g_first,
+                                                                     unsigned* __restrict__ g_m,
+                                                                     unsigned long long* __restrict__ part,
+                                                                     double* __restrict__ outer)
+{
+    extern __shared__ __align__(16) unsigned char raw[];
+    IvShared sh;
+    Iv2Shared s2;
+    s2.rcnt = reinterpret_cast<unsigned*>(raw);
+    s2.rs1 = s2.rcnt + (G + 1) * 32;
+    sh.cnt = s2.rs1 + (G + 1) * 32;
+    sh.s1 = sh.cnt + (MAXB + 1);
+    sh.bb = reinterpret_cast<float*>(sh.s1 + (MAXB + 1));
+    sh.cell = reinterpret_cast<unsigned*>(sh.bb + (MAXB + 1));
+    s2.stage = reinterpret_cast<float*>(sh.cell + (G + 1));
+    const float inf = __int_as_float(0x7F800000);
+    for (unsigned i = threadIdx.x; i <= (unsigned)MAXB; i += IV2_THREADS) {
+        sh.cnt[i] = 0u;
+        sh.s1[i] = 0u;
+        sh.bb[i] = g_bb[i];
+    }
+    __syncthreads();
+    __shared__ unsigned s_m;
+    if (threadIdx.x == 0) {                                  // m = finite boundaries (sorted: a binary search)
+        int lo = 0, hi = MAXB;
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            if (sh.bb[1 + mid] < inf) lo = mid + 1; else hi = mid;
+        }
+        s_m = (unsigned)lo;
+        if (blockIdx.x == 0) *g_m = (unsigned)lo;
+    }
+    __syncthreads();
+    const unsigned m = s_m;                                  // intervals 0..m
+    // cell c meets intervals first[c] .. first[c+1]-1 (a cell that does not exist counts as m + 1);
+    // more than one interval = the cell holds a threshold
+    for (unsigned c = threadIdx.x; c <= (unsigned)G; c += IV2_THREADS) {
+        unsigned f0 = g_first[c], f1 = g_first[c + 1];
+        f0 = (f0 == 0xFFFFFFFFu) ? m + 1u : f0;
+        f1 = (f1 == 0xFFFFFFFFu) ? m + 1u : f1;
+        sh.cell[c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
+    }
+    __syncthreads();
+    for (unsigned i = threadIdx.x; i < (unsigned)(G + 1) * 32u; i += IV2_THREADS) {
+        const unsigned ci = sh.cell[i >> 5];
+        s2.rcnt[i] = ((ci >> 16) != (ci & 0xFFFFu)) ? IV2_SPLIT : 0u;
+        s2.rs1[i] = 0u;
+    }
+    __syncthreads();
+
+    const IvConst k = {setup->g_lo, setup->g_hi, setup->inv_gw, setup->gw, setup->inv_u};
+    const bool guard = st->nonfinite != 0;
+    IvOuter o = {0.0, 0.0, 0.0, 0.0};
+    const unsigned lane = threadIdx.x & 31u;
+    float* my_stage = s2.stage + (threadIdx.x >> 5) * IV2_STAGE;
+    unsigned staged = 0;                                     // warp-uniform
+
+    constexpr int EPV = qp_span<T>::EPV;
+    const qp_span<T> sp(x, n);
+    const T* xv = x + sp.head;
+    const uint64_t stride = (uint64_t)gridDim.x * IV2_THREADS;
+    // every lane of a warp runs the same number of iterations (ballots inside): the loops below
+    // are bounded by warp-uniform conditions and lanes without an element pass a non-finite one
+    auto body = [&](auto guard_tag) {
+        constexpr bool GD = decltype(guard_tag)::value;
+        const float skip = __int_as_float(0x7FC00000);       // NaN: ignored by the guarded form
+        uint64_t v = (uint64_t)blockIdx.x * IV2_THREADS + threadIdx.x;
+        // two vectors per lane while the warp's last lane still has both (v - lane + 31 is its first vector)
+        for (; v - lane + 31u + stride < sp.nvec; v += 2 * stride) {
+            float a[EPV], b[EPV];
+            qp_load_vec(xv + v * EPV, a);
+            qp_load_vec(xv + (v + stride) * EPV, b);
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) iv2_one<GD>(a[i], sh, s2, k, bt, my_stage, staged, lane);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) iv2_one<GD>(b[i], sh, s2, k, bt, my_stage, staged, lane);
+            iv_flush(o, bt);
+        }
+        // the rest: warps may be partly filled, so every lane of a warp that still has work goes on
+        const uint64_t warp_v0 = v - lane;                   // vector of lane 0 (v advanced alike in all lanes)
+        for (uint64_t w0 = warp_v0; w0 < sp.nvec; w0 += stride) {
+            const uint64_t mine = w0 + lane;
+            const bool have = mine < sp.nvec;
+            float a[EPV];
+            if (have) qp_load_vec(xv + mine * EPV, a);
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) iv2_one<true>(have ? a[i] : skip, sh, s2, k, bt, my_stage, staged, lane);
+            iv_flush(o, bt);
+        }
+        if (blockIdx.x == 0) {
+            const uint64_t t0 = sp.head + sp.nvec * EPV;
+            const uint64_t extra = sp.head + sp.tail;
+            for (uint64_t i0 = (threadIdx.x & ~31u); i0 < extra; i0 += IV2_THREADS) {
+                const uint64_t i = i0 + lane;
+                const bool have = i < extra;
+                IvBatch bt = {0.f, 0.f, 0.f, 0.f};
+                const float x1 = have ? qp_load_one(x + (i < sp.head ? i : t0 + (i - sp.head))) : skip;
+                iv2_one<true>(x1, sh, s2, k, bt, my_stage, staged, lane);
+                iv_flush(o, bt);
+            }
+        }
+    };
+    if (guard) body(std::true_type{}); else body(std::false_type{});
+    __syncwarp();
+    if (lane < staged) iv2_exact(my_stage[lane], sh, k);     // what is left in the warp's buffer (< 32)
+    __syncthreads();
+
+    // this block's row: a whole cell is its one interval (replicas added up); a split cell's
+    // intervals come from the exact sums
+    unsigned long long* mine = part + (size_t)blockIdx.x * (MAXB + 1);
+    for (unsigned c = threadIdx.x; c <= (unsigned)G; c += IV2_THREADS) {
+        const unsigned ci = sh.cell[c];
+        const unsigned i0 = ci & 0xFFFFu, i1 = ci >> 16;
+        if (i0 > m) continue;                                // the cell does not exist
+        if (i0 == i1) {
+            unsigned long long cn = 0, cs = 0;
+            for (unsigned r = 0; r < 32u; ++r) {
+                const unsigned rr = (r + lane) & 31u;        // lanes start at different replicas: no bank conflicts
+                cn += s2.rcnt[(c << 5) + rr];
+                cs += s2.rs1[(c << 5) + rr];
+            }
+            mine[i0] = (cn << 40) | cs;
+        } else {
+            for (unsigned i = i0; i <= i1 && i <= m; ++i) {
+                const unsigned cw = sh.cnt[i];
+                mine[i] = ((unsigned long long)(cw & 0xFFFFFFu) << 40) | ((unsigned long long)(cw >> 24) << 32) | sh.s1[i];
+            }
+        }
+    }
+
+    __shared__ double red[IV2_THREADS / 32];
+    const double r0 = qp_block_sum(o.s1, red), r1 = qp_block_sum(o.s1a, red);
+    const double r2 = qp_block_sum(o.s2, red);
+    const double r6 = qp_block_sum(o.s2_in, red);
+    if (threadIdx.x == 0) {
+        double* dst = outer + (size_t)blockIdx.x * 8;
+        dst[0] = r0; dst[1] = r1; dst[2] = r2; dst[3] = 0.0; dst[4] = 0.0; dst[5] = 0.0; dst[6] = r6;
+    }
+}
+
 // Totals over the blocks' partials.  A block takes 32 consecutive intervals: lane = interval
 // (one 256-byte row segment per warp load), warp w adds the partials of blocks w, w + 32, ...
 // (all of its loads in flight at once), the 32 warp sums are merged through shared memory and written
@@ -569,9 +798,23 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]
     iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ncand * L1, ctx->d_iv_bb,
                                                             ctx->d_iv_first);
-    const int blocks = ctx->iv_blocks;
-    iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
-                                                             g_m, ctx->d_iv_part, ctx->d_iv_outer);
+    // second form where its 32-bit replica sums cannot wrap: one block per SM, more for longer tensors
+    constexpr size_t smem2 = (size_t)(G + 1) * 32 * 8 + (size_t)(MAXB + 1) * 12 + (size_t)(G + 1) * 4 +
+                             (size_t)IV2_WARPS * IV2_STAGE * 4 + 16;
+    uint64_t blocks2 = (uint64_t)ctx->sm_count;
+    while (n / blocks2 > IV2_MAX_PER_BLOCK && blocks2 + (uint64_t)ctx->sm_count <= (uint64_t)ctx->iv_blocks)
+        blocks2 += (uint64_t)ctx->sm_count;
+    const bool second = ctx->moments_form != 1 && n / blocks2 <= IV2_MAX_PER_BLOCK;
+    const int blocks = second ? (int)blocks2 : ctx->iv_blocks;
+    if (second) {
+        if (cudaFuncSetAttribute(iv_moments2_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2) != cudaSuccess)
+            return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
+        iv_moments2_kernel<T><<<blocks, IV2_THREADS, smem2, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
+                                                                g_m, ctx->d_iv_part, ctx->d_iv_outer);
+    } else {
+        iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
+                                                                 g_m, ctx->d_iv_part, ctx->d_iv_outer);
+    }
     iv_reduce_kernel<<<(MAXB + 1 + 31) / 32, IV_RED_THREADS, 0, s>>>(ctx->d_iv_part, blocks, g_m, ctx->d_iv_tot,
                                                                     ctx->d_iv_outer,
                                                                     ctx->d_iv_outer + (size_t)blocks * 8);

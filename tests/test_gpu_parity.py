@@ -273,7 +273,7 @@ def test_aciq_device_chain(ctx, bits):
 
 # ------------------------------------------------------------ directed search
 
-BOTH_PATHS = [qp.QP_SEARCH_CANDIDATES, qp.QP_SEARCH_INTERVALS]
+BOTH_PATHS = [qp.QP_SEARCH_CANDIDATES, qp.QP_SEARCH_INTERVALS, qp.QP_SEARCH_INTERVALS_PLAIN]
 
 
 def check_search(ctx, x_np, d_x, bits, bmode=0, steps=100, nb=100, curve_rtol=2e-6, tie_rtol=1e-6,
