@@ -242,8 +242,8 @@ int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
  * (to ~1e-8 relative) and the same winner.
  *   QP_SEARCH_CANDIDATES  every element is quantized under every candidate (any bits/steps)
  *   QP_SEARCH_INTERVALS   one pass gathers moments per interval between the candidates'
- *                         decision thresholds; used where (steps+1)*(2^bits-1) <= 3584 and
- *                         n < ~0.9e9, otherwise the call falls back to the first way
+ *                         decision thresholds; used where (steps+1)*(2^bits-1) <= 2048 and
+ *                         n < ~1.8e9, otherwise the call falls back to the first way
  *   QP_SEARCH_AUTO        intervals for n >= 2^20 where they apply (default)
  * The pass over x that gathers the moments has two forms with identical results: the plain one
  * (every element looks its interval up), and one that adds elements of grid cells without a

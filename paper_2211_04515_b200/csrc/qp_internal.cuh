@@ -34,7 +34,7 @@ struct qp_ds_setup {                     // written by the search's set-up kerne
     double u;
 };
 
-constexpr int QP_IV_CELLS = 512;         // uniform cells over [g_lo, g_hi]
+constexpr int QP_IV_CELLS = 2048;        // uniform cells over [g_lo, g_hi]
 constexpr int QP_IV_MAXB = 4096;         // most interval boundaries (candidate thresholds + cell edges)
 constexpr int QP_IV_THREADS = 512;
 constexpr int QP_IV_BLOCKS_PER_SM = 3;

@@ -280,7 +280,7 @@ int32_t search_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_st
     const int ncand = steps + 1;
     // interval-moment scoring where its tables fit and its fixed-point sums cannot overflow
     const bool iv_fits = ncand * ((1 << bits) - 1) + QP_IV_CELLS <= QP_IV_MAXB &&
-                         n / (uint64_t)ctx->iv_blocks + 65536 < (1ull << 21);    // 40-bit sums of offsets < 1.5 * 2^18
+                         n / (uint64_t)ctx->iv_blocks + 65536 < (1ull << 22);
     const bool use_iv = iv_fits && (ctx->search_path == QP_SEARCH_INTERVALS ||
                                     (ctx->search_path == QP_SEARCH_AUTO && n >= (1ull << 20)));
     if (use_iv)

@@ -146,7 +146,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
             inv_gw = (float)((double)G / width);
             int e;
             frexp(width / (double)G, &e);               // cell width in [2^(e-1), 2^e)
-            u = ldexp(1.0, e - 18);                     // offsets (up to ~1.5 cells) stay below 1.5 * 2^18 units
+            u = ldexp(1.0, e - 16);                     // offsets (up to ~1.5 cells) stay below 2^17.6 units
         }
         sg_lo = lo; sg_hi = hi; sg_inv = inv_gw;
         if (blockIdx.x == 0) {
@@ -423,25 +423,28 @@ __global__ void __launch_bounds__(QP_IV_THREADS) iv_moments_kernel(const T* __re
 // Same result as iv_moments_kernel (the same per-block rows of count << 40 | sum of offsets,
 // the same outer sums), gathered with less work per element.  Most grid cells hold no
 // threshold: such a cell is one interval, and its two sums need neither the table look-up nor
-// the search.  They are kept in a table indexed by cell and LANE (32 replicas of every cell, so
-// a warp's 32 atomics always hit 32 different banks and elements of one value never queue up
-// behind one counter).  Cells that do hold thresholds ("split" cells) carry a mark in the top
-// bit of their replica counters; the counter's old value, which the atomic returns anyway,
-// tells the thread that its element needs the exact treatment.  Those elements are not
+// the search.  They are kept in a table indexed by cell and replica (8 replicas of every cell,
+// chosen by lane, so that elements of one value do not queue up behind one counter and a warp's
+// atomics spread over the banks).  Cells that do hold thresholds ("split" cells) carry a mark
+// in the top bit of their replica counters; the counter's old value, which the atomic returns
+// anyway, tells the thread that its element needs the exact treatment.  Those elements are not
 // handled on the spot (a warp would run the whole search for a few active lanes): each warp
 // collects them in a small buffer of its own and works them off 32 at a time with all lanes
 // busy, through the same cell table, search and interval sums as the first form.
-// One block of 1024 threads per SM (the replica table takes 131 KB).
+// One block of 1024 threads per SM (the replica table takes 131 KB).  512 cells x 32 replicas
+// (conflict-free, but more split cells) and 1024 x 16 were tried too: within 3 % of each other.
 constexpr int IV2_THREADS = 1024;
 constexpr int IV2_WARPS = IV2_THREADS / 32;
 constexpr int IV2_STAGE = 64;                        // buffered elements per warp (worked off from 32 on)
 constexpr unsigned IV2_SPLIT = 0x80000000u;
-// replica sums are 32 bit: elements per block * largest offset (1.5 * 2^18 units) / 32 replicas < 2^32
+constexpr int IV2_RS = 3;                            // log2 of the replicas per cell
+constexpr unsigned IV2_R = 1u << IV2_RS;
+// replica sums are 32 bit: elements per block * largest offset (1.5 * 2^16 units) / 8 replicas < 2^32
 constexpr uint64_t IV2_MAX_PER_BLOCK = 340000;
 
 struct Iv2Shared {
-    unsigned* rcnt;                 // [(G + 1) * 32] per cell and lane: count (| IV2_SPLIT in split cells)
-    unsigned* rs1;                  // [(G + 1) * 32] per cell and lane: sum of offsets
+    unsigned* rcnt;                 // [(G + 1) * IV2_R] per cell and replica: count (| IV2_SPLIT in split cells)
+    unsigned* rs1;                  // [(G + 1) * IV2_R] per cell and replica: sum of offsets
     float* stage;                   // [IV2_WARPS][IV2_STAGE]
 };
 
@@ -482,7 +485,7 @@ __device__ __forceinline__ void iv2_one(float x, const IvShared& sh, const Iv2Sh
         const float dm = fmaf(__fsub_rn(xc, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
         const float d1f = __fsub_rn(dm, IV_MAGIC);
         b.s2_in = fmaf(d1f, d1f, b.s2_in);
-        const unsigned idx = ((__float_as_uint(pm) & 0x7FFFFFu) << 5) + lane;
+        const unsigned idx = ((__float_as_uint(pm) & 0x7FFFFFu) << IV2_RS) + (lane & (IV2_R - 1u));
         const unsigned old = atomicAdd(&s2.rcnt[idx], 1u);
         atomicAdd(&s2.rs1[idx], __float_as_uint(dm) & 0x7FFFFFu);     // ignored later if the cell is split
         split = (old & IV2_SPLIT) != 0u;
@@ -514,8 +517,8 @@ __global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __
     IvShared sh;
     Iv2Shared s2;
     s2.rcnt = reinterpret_cast<unsigned*>(raw);
-    s2.rs1 = s2.rcnt + (G + 1) * 32;
-    sh.cnt = s2.rs1 + (G + 1) * 32;
+    s2.rs1 = s2.rcnt + (G + 1) * IV2_R;
+    sh.cnt = s2.rs1 + (G + 1) * IV2_R;
     sh.s1 = sh.cnt + (MAXB + 1);
     sh.bb = reinterpret_cast<float*>(sh.s1 + (MAXB + 1));
     sh.cell = reinterpret_cast<unsigned*>(sh.bb + (MAXB + 1));
@@ -548,8 +551,8 @@ __global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __
         sh.cell[c] = (f0 & 0xFFFFu) | ((f1 - 1u) << 16);
     }
     __syncthreads();
-    for (unsigned i = threadIdx.x; i < (unsigned)(G + 1) * 32u; i += IV2_THREADS) {
-        const unsigned ci = sh.cell[i >> 5];
+    for (unsigned i = threadIdx.x; i < (unsigned)(G + 1) * IV2_R; i += IV2_THREADS) {
+        const unsigned ci = sh.cell[i >> IV2_RS];
         s2.rcnt[i] = ((ci >> 16) != (ci & 0xFFFFu)) ? IV2_SPLIT : 0u;
         s2.rs1[i] = 0u;
     }
@@ -623,10 +626,10 @@ __global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __
         if (i0 > m) continue;                                // the cell does not exist
         if (i0 == i1) {
             unsigned long long cn = 0, cs = 0;
-            for (unsigned r = 0; r < 32u; ++r) {
-                const unsigned rr = (r + lane) & 31u;        // lanes start at different replicas: no bank conflicts
-                cn += s2.rcnt[(c << 5) + rr];
-                cs += s2.rs1[(c << 5) + rr];
+            for (unsigned r = 0; r < IV2_R; ++r) {
+                const unsigned rr = (r + lane) & (IV2_R - 1u);   // lanes start at different replicas
+                cn += s2.rcnt[(c << IV2_RS) + rr];
+                cs += s2.rs1[(c << IV2_RS) + rr];
             }
             mine[i0] = (cn << 40) | cs;
         } else {
@@ -799,7 +802,7 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ncand * L1, ctx->d_iv_bb,
                                                             ctx->d_iv_first);
     // second form where its 32-bit replica sums cannot wrap: one block per SM, more for longer tensors
-    constexpr size_t smem2 = (size_t)(G + 1) * 32 * 8 + (size_t)(MAXB + 1) * 12 + (size_t)(G + 1) * 4 +
+    constexpr size_t smem2 = (size_t)(G + 1) * IV2_R * 8 + (size_t)(MAXB + 1) * 12 + (size_t)(G + 1) * 4 +
                              (size_t)IV2_WARPS * IV2_STAGE * 4 + 16;
     uint64_t blocks2 = (uint64_t)ctx->sm_count;
     while (n / blocks2 > IV2_MAX_PER_BLOCK && blocks2 + (uint64_t)ctx->sm_count <= (uint64_t)ctx->iv_blocks)
