@@ -37,7 +37,7 @@ UNIT = "GB/s"
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's main kernel on this
 # workload, from the ncu captures summarised in profiles/kernels_c4_ncu_full.md (None once a
 # kernel has changed since its capture)
-NCU_TRAFFIC_BYTES = {"clip": 131.0e6, "stats": 2 * 133.4e6, "quantize_pack": 145.2e6, "unpack_dequantize": 104.0e6}
+NCU_TRAFFIC_BYTES = {"clip": 133.2e6, "stats": 2 * 133.4e6, "quantize_pack": 141.5e6, "unpack_dequantize": 99.3e6}
 SAMPLE_IMAGES = 8              # CPU baseline leg: the first 8 images of the batch (2.0 M elements)
 ORACLE_US_PER_ELEM = 0.31      # rough cost of one oracle step per element (search on ~half the steps)
 
