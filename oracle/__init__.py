@@ -98,6 +98,9 @@ def lib():
         L.orc_clip_channels.argtypes = [C.POINTER(Stats), C.c_uint64, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
                                         C.POINTER(QParams)]
         L.orc_clip_channels.restype = C.c_int
+        L.orc_ds_search_channels.argtypes = [fp, C.c_uint64, C.c_uint64, C.POINTER(Stats), C.c_int, C.c_int, C.c_int,
+                                             C.c_int, C.POINTER(DSResult), C.POINTER(QParams), C.POINTER(C.c_double)]
+        L.orc_ds_search_channels.restype = C.c_int
         L.orc_quantize_channels.argtypes = [fp, C.c_uint64, C.c_uint64, C.POINTER(QParams), u32p]
         L.orc_quantize_channels.restype = None
         L.orc_dequantize_channels.argtypes = [u32p, C.c_uint64, C.c_uint64, C.POINTER(QParams), fp]
@@ -278,6 +281,19 @@ def ds_search(x, st: Stats, bits: int, bmode: int = 0, steps: int = 100, hist_bi
     rc = lib().orc_ds_search(_ptr(a, C.c_float), a.size, C.byref(st), bits, bmode, steps, hist_bins,
                              C.byref(res), C.byref(qp), _ptr(curve, C.c_double))
     return rc, res, qp, curve
+
+
+def ds_search_channels(x, channels: int, st, bits: int, bmode: int = 0, steps: int = 100, hist_bins: int = 100):
+    """Directed search per channel of a [rows, channels] tensor: (rc, DSResult[channels], QParams[channels], curves)."""
+    a = _f32(x)
+    rows = a.size // channels
+    assert rows * channels == a.size
+    res = (DSResult * channels)()
+    qp = (QParams * channels)()
+    curves = np.empty((channels, steps + 1), dtype=np.float64)
+    rc = lib().orc_ds_search_channels(_ptr(a, C.c_float), rows, channels, st, bits, bmode, steps, hist_bins, res, qp,
+                                      _ptr(curves, C.c_double))
+    return rc, res, qp, curves
 
 
 def select_bits(bandwidth_bps: float, budget_s: float, n_elems: int, overhead_bytes: int = 0,

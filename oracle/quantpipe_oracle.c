@@ -492,6 +492,29 @@ int orc_ds_search(const float* x, uint64_t n, const orc_stats_t* st, int bits, i
     return degenerate ? ORC_WARN_DEGENERATE : ORC_OK;
 }
 
+/* The directed search run for every channel of a [rows, channels] tensor on its column alone
+ * (channel-wise variant, see orc_stats_channels): res[c], qp[c] and, if curves is not NULL,
+ * curves[c * (steps + 1) + k] are what orc_ds_search gives for column c with statistics st[c].
+ * Returns ORC_WARN_DEGENERATE if any channel's search was degenerate. */
+int orc_ds_search_channels(const float* x, uint64_t rows, uint64_t channels, const orc_stats_t* st, int bits,
+                           int bmode, int steps, int hist_bins, orc_ds_result_t* res, orc_qparams_t* qp,
+                           double* curves)
+{
+    if (channels < 1) return ORC_ERR_ARG;
+    float* col = (float*)malloc((size_t)(rows ? rows : 1) * sizeof(float));
+    if (!col) return ORC_ERR_ARG;
+    int worst = ORC_OK;
+    for (uint64_t c = 0; c < channels; ++c) {
+        for (uint64_t r = 0; r < rows; ++r) col[r] = x[r * channels + c];
+        int rc = orc_ds_search(col, rows, &st[c], bits, bmode, steps, hist_bins, &res[c], &qp[c],
+                               curves ? curves + c * (uint64_t)(steps + 1) : NULL);
+        if (rc < 0) { free(col); return rc; }
+        if (rc == ORC_WARN_DEGENERATE) worst = rc;
+    }
+    free(col);
+    return worst;
+}
+
 /* -------------------------------------------------------- bit-width choice */
 
 /* Widest allowed code whose payload fits the link budget (the selection principle of

@@ -750,6 +750,49 @@ def test_channels_one_channel_is_the_per_tensor_path_and_symmetries():
     assert np.all(back[:, 7] == np.float32(1.5))
 
 
+def test_channels_directed_search():
+    """The search per channel: every column gets what the per-tensor search gives for it alone."""
+    C_, rows = 5, 3000
+    x = si.vit_activation((1, rows, C_), 15, outlier_frac=0.2).reshape(rows, C_)
+    st = oracle.stats_channels(x, C_)
+    rc, res, qp, curves = oracle.ds_search_channels(x, C_, st, 2, 0, 100, 64)
+    assert rc == 0 and curves.shape == (C_, 101)
+    F = float(np.real(scipy.special.lambertw(3.0 * 4.0 ** 2)))
+    for c in range(C_):
+        col = np.ascontiguousarray(x[:, c])
+        # independent evaluation of the column's candidates (NumPy histogram and quantizer)
+        counts, _ = np.histogram(col.astype(np.float64), bins=64, range=(st[c].min, st[c].max))
+        peak = counts.max() / (rows * (st[c].max - st[c].min) / 64)
+        assert res[c].b_e == st[c].mad and res[c].b_r == pytest.approx(1.0 / (2.0 * peak), rel=0.03)
+        mses = np.array([_numpy_candidate_mse(col, st[c].mean, F * (res[c].b_e + k * (res[c].b_r - res[c].b_e) / 100), 2)
+                         for k in range(101)])
+        assert np.allclose(curves[c], mses, rtol=1e-9)
+        k_ref = int(np.argmin(mses))
+        assert res[c].k_star == k_ref or abs(mses[res[c].k_star] - mses[k_ref]) <= 1e-12 * mses[k_ref]
+        assert qp[c].lo == np.float32(st[c].mean - res[c].alpha_star) and qp[c].hi == np.float32(st[c].mean + res[c].alpha_star)
+        assert res[c].mse_star <= res[c].mse_e
+    # the searched quantizers lower the whole tensor's error below the channel-wise ACIQ ranges
+    back = oracle.dequantize_channels(oracle.quantize_channels(x, C_, qp), C_, qp).astype(np.float64)
+    err_ds = np.mean((back - x.reshape(-1)) ** 2)
+    _, qa = oracle.clip_channels(st, 2)
+    back_a = oracle.dequantize_channels(oracle.quantize_channels(x, C_, qa), C_, qa).astype(np.float64)
+    assert err_ds <= np.mean((back_a - x.reshape(-1)) ** 2)
+    assert err_ds == pytest.approx(np.mean([res[c].mse_star for c in range(C_)]), rel=1e-12)
+    # one channel: the per-tensor search, byte for byte
+    y = np.ascontiguousarray(x[:, 3])
+    st1 = oracle.stats_channels(y, 1)
+    _, res1, qp1, curve1 = oracle.ds_search_channels(y, 1, st1, 3, 0x10, 50, 100)
+    _, res_t, qp_t, curve_t = oracle.ds_search(y, oracle.stats(y), 3, 0x10, 50, 100)
+    assert bytes(res1[0]) == bytes(res_t) and bytes(qp1[0]) == bytes(qp_t) and np.array_equal(curve1[0], curve_t)
+    # channels do not interact; a constant channel is reported and keeps b_E = 0
+    x2 = x.copy()
+    x2[:, 1] = np.float32(-2.0)
+    rc2, res2, qp2, _ = oracle.ds_search_channels(x2, C_, oracle.stats_channels(x2, C_), 2, 0, 100, 64)
+    assert rc2 == oracle.WARN_DEGENERATE and qp2[1].flags == 1 and res2[1].k_star == 0
+    assert all(bytes(res2[c]) == bytes(res[c]) and bytes(qp2[c]) == bytes(qp[c]) for c in range(C_) if c != 1)
+    assert oracle.ds_search_channels(x, C_, st, 16)[0] == oracle.ERR_BITS
+
+
 # ------------------------------------------------------------------- inputs
 
 def test_generator_is_counter_based_and_shaped():
