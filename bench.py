@@ -514,6 +514,12 @@ def sweep_main(args):
             d_cst = torch.empty(80 * channels, dtype=torch.uint8, device="cuda")
             med, best = timed(lambda i: ctx.qp_stats_channels(xs[i], channels, out=d_cst), nb)
             emit(name, dtype, f"stats_channels[{channels}]", 0, n, med, best, esz * n)
+            d_cres = torch.empty(72 * channels, dtype=torch.uint8, device="cuda")
+            d_csqp = torch.empty(24 * channels, dtype=torch.uint8, device="cuda")
+            for q in (2, 4):                  # every candidate scored on every element: fp32-ALU-bound
+                med, best = timed(lambda i: ctx.qp_dsaciq_search_channels(xs[i], channels, d_cst, q, out_result=d_cres,
+                                                                          out_qp=d_csqp), nb)
+                emit(name, dtype, f"dsaciq_search_channels[{channels}]", q, n, med, best, esz * n)
             for q in (4, 8):
                 d_cqp = ctx.qp_clip_qparams_channels_device(d_cst, channels, q)
                 pk = rotating(lambda: torch.empty(qp.qp_packed_bytes(n, q), dtype=torch.uint8, device="cuda"),

@@ -378,6 +378,26 @@ int32_t qp_sender_channels_device(qp_ctx* ctx, const void* d_x, int dtype, uint6
                                   int method, int bmode, void* d_packed, uint64_t packed_capacity,
                                   qp_qparams_t* d_qp_out, qp_stats_t* d_stats_out, void* stream);
 
+/* Channel-wise directed search (the search of Sec. 3 / Eq. 1 applied to each column of the
+ * [rows, channels] tensor; the paper searches per tensor): channel c gets the histogram,
+ * b_R, candidates, MSE curve and winner that qp_dsaciq_search gives for its column alone with
+ * d_stats[c] (from qp_stats_channels).  Writes d_qp_out[0..channels) and, if not NULL,
+ * d_out[0..channels).  Every candidate is scored on every element (the per-tensor candidate
+ * path's arithmetic), so the cost is (steps + 1) * 9 fp32 instructions per element.
+ * bits 1..8; 1 <= steps <= QP_CH_MAX_STEPS; 1 <= hist_bins <= QP_CH_MAX_HIST_BINS; bmode as for
+ * qp_dsaciq_search (QP_B_HIST_IN_STATS has no meaning here and is rejected).  Scratch
+ * (histograms, candidates, block partials: about (4 hist_bins + 28 (steps + 1) + 8 (steps + 1)
+ * * row blocks) bytes per channel) is allocated by the context on first use and kept.
+ * qp_dsaciq_curve_channels copies the MSE curve of one channel of the last such search to
+ * host memory (steps + 1 doubles) and synchronizes the stream.
+ * Errors: as qp_dsaciq_search, plus QP_ERR_INVALID_ARG for channels out of range. */
+#define QP_CH_MAX_STEPS 127
+#define QP_CH_MAX_HIST_BINS 256
+int32_t qp_dsaciq_search_channels(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t channels,
+                                  const qp_stats_t* d_stats, int bits, int bmode, int steps, int hist_bins,
+                                  qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, void* stream);
+int32_t qp_dsaciq_curve_channels(qp_ctx* ctx, uint32_t channel, double* h_curve, int capacity, void* stream);
+
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------
  * qp_sender_host: copies the n elements at h_x to d_x_work, runs statistics, the clip

@@ -38,7 +38,7 @@ EXPORTS = (
     "qp_dsaciq_curve", "qp_policy_use_ds", "qp_quantize_pack", "qp_unpack_dequantize", "qp_select_bits",
     "qp_select_bits_eq2", "qp_launch_count", "qp_sender_host", "qp_receiver_host", "qp_stats_static", "qp_set_search_path", "qp_stats_carries_histogram", "qp_controller_init", "qp_controller_observe",
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
-    "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_clip_qparams_channels_device",
+    "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_dsaciq_search_channels", "qp_dsaciq_curve_channels", "qp_clip_qparams_channels_device",
     "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range", "qp_sender_channels_device",
 )
 
@@ -110,6 +110,9 @@ def load() -> C.CDLL:
     L.qp_clip_qparams_device.argtypes = [vp, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.qp_midrise_range.argtypes = [dbl, dbl, C.c_int, C.POINTER(dbl), C.POINTER(dbl)]
     L.qp_stats_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, vp, vp]
+    L.qp_dsaciq_search_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp,
+                                            vp]
+    L.qp_dsaciq_curve_channels.argtypes = [vp, C.c_uint32, C.POINTER(dbl), C.c_int, vp]
     L.qp_clip_qparams_channels_device.argtypes = [vp, vp, C.c_uint32, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
     L.qp_quantize_pack_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, vp, vp, u64, vp]
     L.qp_unpack_dequantize_channels.argtypes = [vp, vp, u64, C.c_uint32, C.c_int, vp, vp, C.c_int, vp]
@@ -416,6 +419,24 @@ class Context:
         self._check(self._lib.qp_stats_channels(self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels, channels,
                                                 out.data_ptr(), _stream(self.device)))
         return out
+
+    def qp_dsaciq_search_channels(self, x: torch.Tensor, channels: int, d_stats: torch.Tensor, bits: int,
+                                  bmode: int = QP_B_MAD, steps: int = QP_DEFAULT_STEPS,
+                                  hist_bins: int = QP_DEFAULT_HIST_BINS, out_result: torch.Tensor | None = None,
+                                  out_qp: torch.Tensor | None = None):
+        """Directed search per channel; returns (device DSResult[channels] bytes, device QParams[channels] bytes)."""
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        out_result = self._bytes(C.sizeof(DSResult) * channels) if out_result is None else out_result
+        out_qp = self._bytes(C.sizeof(QParams) * channels) if out_qp is None else out_qp
+        self._check(self._lib.qp_dsaciq_search_channels(self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels,
+                                                        channels, d_stats.data_ptr(), bits, bmode, steps, hist_bins,
+                                                        out_result.data_ptr(), out_qp.data_ptr(), _stream(self.device)))
+        return out_result, out_qp
+
+    def qp_dsaciq_curve_channels(self, channel: int, steps: int):
+        buf = (C.c_double * (steps + 1))()
+        self._check(self._lib.qp_dsaciq_curve_channels(self._h, channel, buf, steps + 1, _stream(self.device)))
+        return list(buf)
 
     def qp_clip_qparams_channels_device(self, d_stats: torch.Tensor, channels: int, bits: int, method: int = QP_CLIP_ACIQ,
                                         dist: int = QP_DIST_LAPLACE, bmode: int = QP_B_MAD,

@@ -128,6 +128,7 @@ extern "C" int32_t qp_destroy(qp_ctx* ctx)
     qp_drop_graphs(ctx);
     if (ctx->d_ch_part) cudaFree(ctx->d_ch_part);
     if (ctx->d_ch_stats) cudaFree(ctx->d_ch_stats);
+    if (ctx->d_ch_search) cudaFree(ctx->d_ch_search);
     const cudaError_t e = cudaFree(ctx->d_base);
     delete ctx;
     return e == cudaSuccess ? QP_OK : QP_ERR_CUDA;

@@ -80,6 +80,11 @@ struct qp_ctx {
     void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
     void* d_ch_part;                     // channel-wise statistics: block partials, allocated on first use
     size_t ch_part_bytes;
+    void* d_ch_search;                   // channel-wise search: histograms, candidates, partials, curves; on first use
+    size_t ch_search_bytes;
+    int ch_last_steps, ch_last_ncp;      // of the last channel-wise search (for qp_dsaciq_curve_channels)
+    uint32_t ch_last_channels;
+    size_t ch_curve_offset;
     void* d_ch_stats;                    // channel-wise sender: statistics when the caller wants none back
     size_t ch_stats_bytes;
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points

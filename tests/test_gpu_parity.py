@@ -982,3 +982,112 @@ def test_channels_sender_in_one_call(ctx):
     with pytest.raises(qp.QuantPipeError):
         ctx.qp_sender_channels_device(d, 384, 4, qp.QP_CLIP_DSACIQ)
     assert ctx.qp_get_status() == 0
+
+
+# ------------------------------------------------- channel-wise directed search
+
+def check_search_channels(ctx, x_np, d_x, channels, bits, bmode=0, steps=100, nb=100):
+    rows = x_np.size // channels
+    d_stats = ctx.qp_stats_channels(d_x, channels)
+    d_res, d_qp = ctx.qp_dsaciq_search_channels(d_x, channels, d_stats, bits, bmode, steps, nb)
+    raw_res = d_res.cpu().numpy().tobytes()
+    raw_qp = d_qp.cpu().numpy().tobytes()
+    rsz, qsz = ctypes.sizeof(qp.DSResult), ctypes.sizeof(qp.QParams)
+    st_o = oracle.stats_channels(x_np, channels)
+    rc_o, res_o, qp_o, curves_o = oracle.ds_search_channels(x_np, channels, st_o, bits, bmode, steps, nb)
+    near_ties = 0
+    for c in range(channels):
+        # A column has few elements.  The two sides' statistics agree to ~1e-9, which can still round a
+        # candidate's clip end to the neighbouring float; that moves every level by one ulp of the end,
+        # i.e. every error by ulp / step of a step, and the column's MSE by about 1.2 * that over sqrt(rows)
+        # as one standard deviation (measured: 1-3 of 101 candidates per channel beyond 2e-6, the worst
+        # of ~10^4 candidate curves at 0.9 * ulp / step with 394 rows); 20 / sqrt(rows) covers the tail.
+        # The per-tensor tests average the same effect over 10^5 and more elements and compare at 2e-6.
+        a_max = max(abs(st_o[c].mean) + res_o[c].alpha_e, abs(st_o[c].mean) + res_o[c].alpha_star, 1e-30)
+        step = 2.0 * min(res_o[c].alpha_e, res_o[c].alpha_star) / (2 ** bits - 1) if res_o[c].alpha_star > 0 else 1.0
+        tol = 2e-6 + 20.0 * float(np.spacing(np.float32(a_max))) / max(step, 1e-30) / np.sqrt(max(rows, 1))
+        res = qp.DSResult.from_buffer_copy(raw_res[c * rsz:(c + 1) * rsz])
+        got = qp.QParams.from_buffer_copy(raw_qp[c * qsz:(c + 1) * qsz])
+        ro = res_o[c]
+        assert (res.steps, res.hist_bins, res.bits) == (steps, nb, bits)
+        assert abs(res.b_e - ro.b_e) <= 1e-5 * abs(ro.b_e) + 1e-300
+        assert abs(res.b_r - ro.b_r) <= 1e-9 * abs(ro.b_r) + 1e-300         # integer-identical histogram
+        if c % max(1, channels // 7) == 0:                                   # curves of a few channels
+            curve = np.array(ctx.qp_dsaciq_curve_channels(c, steps))
+            fin = np.isfinite(curves_o[c])
+            assert np.array_equal(np.isfinite(curve), fin)
+            assert np.all(np.abs(curve[fin] - curves_o[c][fin]) <= tol * curves_o[c][fin] + 1e-300)
+        if res.k_star != ro.k_star:                                          # only a near-tie may differ
+            assert curves_o[c][res.k_star] <= ro.mse_star * (1 + max(1e-6, 2 * tol)), (c, res.k_star, ro.k_star)
+            near_ties += 1
+            continue
+        assert abs(res.alpha_star - ro.alpha_star) <= 1e-4 * abs(ro.alpha_star) + 1e-300
+        assert abs(got.lo - qp_o[c].lo) <= 1e-5 * ro.alpha_star + 1e-30 and abs(got.hi - qp_o[c].hi) <= 1e-5 * ro.alpha_star + 1e-30
+        assert got.bits == bits and got.flags == qp_o[c].flags
+        assert abs(res.mse_star - ro.mse_star) <= tol * ro.mse_star + 1e-300
+    assert near_ties <= max(1, channels // 20)
+    # the quantizers feed the channel-wise packer: bit-exact codes under the library's own quantizers
+    mine = (oracle.QParams * channels)()
+    for c in range(channels):
+        g = qp.QParams.from_buffer_copy(raw_qp[c * qsz:(c + 1) * qsz])
+        mine[c] = oracle.QParams(g.lo, g.hi, g.scale, g.inv_scale, g.bits, g.flags)
+    packed = ctx.qp_quantize_pack_channels(d_x, channels, bits, d_qp)
+    codes_o = oracle.quantize_channels(x_np, channels, mine)
+    assert np.array_equal(packed.cpu().numpy(), oracle.pack(codes_o, bits))
+    return rc_o
+
+
+@pytest.mark.parametrize("bits", [1, 2, 3, 4, 8])
+def test_search_channels_vit(ctx, bits):
+    x = si.vit_activation((2, 197, 96), 131, outlier_frac=0.03).reshape(-1)
+    check_search_channels(ctx, x, dev(x), 96, bits)
+    ctx.qp_get_status()
+
+
+@pytest.mark.parametrize("channels,rows", [(1, 5000), (3, 777), (5, 1), (33, 100), (70, 2049), (1280, 64)])
+def test_search_channels_shapes_and_modes(ctx, channels, rows):
+    x = si.vit_activation((1, rows, channels), 140 + channels % 7, outlier_frac=0.05).reshape(-1)
+    d = dev(x)
+    check_search_channels(ctx, x, d, channels, 2, nb=64)
+    check_search_channels(ctx, x, d, channels, 4, bmode=qp.QP_B_MEAN_ABS | qp.QP_B_MIDRISE, steps=37, nb=256)
+    check_search_channels(ctx, x, d, channels, 3, bmode=qp.QP_B_GAUSS, steps=127, nb=1)
+    ctx.qp_get_status()
+
+
+def test_search_channels_special_values_bf16_and_errors(ctx):
+    channels, rows = 12, 3000
+    x = si.vit_activation((1, rows, channels), 151).reshape(rows, channels).copy()
+    x[:, 4] = np.float32(0.5)                                   # a constant channel: degenerate, b_E kept
+    x[[7, 100, 2999], [0, 3, 11]] = [np.nan, np.inf, -np.inf]
+    flat = x.reshape(-1)
+    assert check_search_channels(ctx, flat, dev(flat), channels, 2) == oracle.WARN_DEGENERATE
+    assert ctx.qp_get_status() & qp.QP_DEV_DEGENERATE
+    h = si.to_bf16_bits(si.vit_activation((1, 500, 40), 152).reshape(-1))
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    check_search_channels(ctx, oracle.widen_bf16(h), d, 40, 4)
+    y = dev(flat)
+    st = ctx.qp_stats_channels(y, channels)
+    for bad in (dict(bits=16), dict(bits=2, steps=128), dict(bits=2, hist_bins=257), dict(bits=2, bmode=qp.QP_B_HIST_IN_STATS),
+                dict(bits=2, steps=0)):
+        with pytest.raises(qp.QuantPipeError):
+            ctx.qp_dsaciq_search_channels(y, channels, st, **bad)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_dsaciq_search_channels(y, y.numel(), st, 2)          # 36000 channels: beyond QP_MAX_CHANNELS
+    ctx.qp_get_status()
+
+
+def test_search_channels_full_size_c3_sampled(ctx):
+    """The outlier-channel config at full size: sampled channels against the oracle's per-tensor search of the column."""
+    x = si.config_tensor("c3").reshape(-1, 1024)
+    d = dev(x.reshape(-1))
+    d_stats = ctx.qp_stats_channels(d, 1024)
+    d_res, d_qp = ctx.qp_dsaciq_search_channels(d, 1024, d_stats, 4)
+    raw = d_res.cpu().numpy().tobytes()
+    rsz = ctypes.sizeof(qp.DSResult)
+    for c in (0, 17, 511, 1023):
+        col = np.ascontiguousarray(x[:, c])
+        _, ro, _, curve_o = oracle.ds_search(col, oracle.stats(col), 4)
+        res = qp.DSResult.from_buffer_copy(raw[c * rsz:(c + 1) * rsz])
+        assert abs(res.b_r - ro.b_r) <= 1e-9 * ro.b_r and abs(res.mse_e - ro.mse_e) <= 2e-6 * ro.mse_e
+        assert res.k_star == ro.k_star or curve_o[res.k_star] <= ro.mse_star * (1 + 1e-6)
+    assert ctx.qp_get_status() & ~qp.QP_DEV_DEGENERATE == 0
