@@ -358,7 +358,8 @@ uint64_t qp_controller_payload_bytes(const qp_controller_t* h_c, int bits);
  *   qp_quantize_pack_channels        code of element i with d_qp[i mod channels].
  *   qp_unpack_dequantize_channels    the inverse, fp32 or bf16 out.
  *   qp_sender_channels_device        the three sender calls in one: statistics -> clip by `method`
- *                                    (Laplace model) -> quantize+pack; writes the packed stream,
+ *                                    (Laplace model; QP_CLIP_DSACIQ runs qp_dsaciq_search_channels with
+ *                                    QP_DEFAULT_STEPS and QP_DEFAULT_HIST_BINS) -> quantize+pack; writes the packed stream,
  *                                    d_qp_out[0..channels) and, if d_stats_out is not NULL, the
  *                                    statistics (otherwise they stay in a buffer of the context,
  *                                    allocated on first use).

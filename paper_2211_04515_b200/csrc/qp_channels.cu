@@ -755,8 +755,10 @@ extern "C" int32_t qp_sender_channels_device(qp_ctx* ctx, const void* d_x, int d
     if (rc) return rc;
     if (!d_qp_out) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null d_qp_out");
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    if (!qp_clip_method_closed_form(method))
-        return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT) or MINMAX, optionally | MIDRISE");
+    const bool use_ds = (method & ~QP_CLIP_MIDRISE) == QP_CLIP_DSACIQ;
+    if (!use_ds && !qp_clip_method_closed_form(method))
+        return qp_fail(ctx, QP_ERR_INVALID_ARG, "method must be ACIQ (| INTERSECT), MINMAX or DSACIQ, optionally | MIDRISE");
+    if (use_ds && bits > 8) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "the search supports 1..8 bits");
     if (packed_capacity < qp_packed_bytes(rows * channels, bits))
         return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(rows * channels, bits)");
     qp_stats_t* st = d_stats_out;
@@ -778,7 +780,12 @@ extern "C" int32_t qp_sender_channels_device(qp_ctx* ctx, const void* d_x, int d
     }
     rc = qp_stats_channels(ctx, d_x, dtype, rows, channels, st, stream);
     if (rc < 0) return rc;
-    rc = qp_clip_qparams_channels_device(ctx, st, channels, bits, method, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
+    if (use_ds)
+        rc = qp_dsaciq_search_channels(ctx, d_x, dtype, rows, channels, st, bits,
+                                       bmode | ((method & QP_CLIP_MIDRISE) ? QP_B_MIDRISE : 0), QP_DEFAULT_STEPS,
+                                       QP_DEFAULT_HIST_BINS, nullptr, d_qp_out, stream);
+    else
+        rc = qp_clip_qparams_channels_device(ctx, st, channels, bits, method, QP_DIST_LAPLACE, bmode, d_qp_out, stream);
     if (rc < 0) return rc;
     return qp_quantize_pack_channels(ctx, d_x, dtype, rows, channels, bits, d_qp_out, d_packed, packed_capacity, stream);
 }

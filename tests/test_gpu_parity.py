@@ -979,9 +979,16 @@ def test_channels_sender_in_one_call(ctx):
         st_out = torch.empty(384 * ctypes.sizeof(qp.Stats), dtype=torch.uint8, device="cuda")
         got2, _ = ctx.qp_sender_channels_device(d, 384, bits, method, out_stats=st_out)
         assert torch.equal(got2, want) and torch.equal(st_out, d_stats)
+    # with the directed search per channel
+    for bits, method, bmode in ((2, qp.QP_CLIP_DSACIQ, 0), (4, qp.QP_CLIP_DSACIQ | qp.QP_CLIP_MIDRISE, qp.QP_B_MIDRISE)):
+        d_stats = ctx.qp_stats_channels(d, 384)
+        _, d_qp = ctx.qp_dsaciq_search_channels(d, 384, d_stats, bits, bmode)
+        want = ctx.qp_quantize_pack_channels(d, 384, bits, d_qp)
+        got, got_qp = ctx.qp_sender_channels_device(d, 384, bits, method)
+        assert torch.equal(got, want) and torch.equal(got_qp, d_qp)
     with pytest.raises(qp.QuantPipeError):
-        ctx.qp_sender_channels_device(d, 384, 4, qp.QP_CLIP_DSACIQ)
-    assert ctx.qp_get_status() == 0
+        ctx.qp_sender_channels_device(d, 384, 16, qp.QP_CLIP_DSACIQ)
+    assert ctx.qp_get_status() & ~qp.QP_DEV_DEGENERATE == 0
 
 
 # ------------------------------------------------- channel-wise directed search
