@@ -571,6 +571,53 @@ def sweep_main(args):
     return 0
 
 
+def quality_main(args):
+    """Quantization error of the clip methods on the ViT-shaped configs (context for the paper's Sec. 3
+    claim that the directed search lowers the MSE of ACIQ): every number is the MSE between the tensor
+    and what the receiver reconstructs, measured on the device from the library's own output."""
+    import torch
+
+    import paper_2211_04515_b200 as qp
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --quality needs a CUDA device")
+    ctx = qp.Context(0)
+    for name in ("c2", "c3"):
+        shape = si.CONFIGS[name]["shape"]
+        channels = shape[-1]
+        x = torch.from_numpy(si.config_tensor(name).reshape(-1)).cuda()
+        n = x.numel()
+        rows = n // channels
+
+        def mse_of(y):
+            return float(((y.double() - x.double()) ** 2).mean())
+
+        for q in (2, 4, 8):
+            row = {"quality": True, "workload": name, "bits": q}
+            d_stats = ctx.qp_stats(x)
+            for label, method in (("naive_minmax", qp.QP_CLIP_MINMAX), ("aciq", qp.QP_CLIP_ACIQ)):
+                d_qp = ctx.qp_clip_qparams_device(d_stats, q, method)
+                y = ctx.qp_unpack_dequantize(ctx.qp_quantize_pack(x, q, d_qp), n, q, d_qp)
+                row[label] = mse_of(y)
+            for nb in (100, 2048):
+                d_sh = ctx.qp_stats(x, hist_bins=nb)
+                d_res, d_qp = ctx.qp_dsaciq_search(x, d_sh, q, hist_bins=nb)
+                res = ctx.read_ds_result(d_res)
+                y = ctx.qp_unpack_dequantize(ctx.qp_quantize_pack(x, q, d_qp), n, q, d_qp)
+                row[f"ds_nb{nb}"] = {"mse_e": res.mse_e, "mse_star": res.mse_star, "k_star": res.k_star,
+                                     "b_r_over_b_e": res.b_r / res.b_e, "measured": mse_of(y)}
+            d_cst = ctx.qp_stats_channels(x, channels)
+            d_cqp = ctx.qp_clip_qparams_channels_device(d_cst, channels, q)
+            y = ctx.qp_unpack_dequantize_channels(ctx.qp_quantize_pack_channels(x, channels, q, d_cqp), rows, channels, q, d_cqp)
+            row["channels_aciq"] = mse_of(y)
+            _, d_cqp = ctx.qp_dsaciq_search_channels(x, channels, d_cst, q)
+            y = ctx.qp_unpack_dequantize_channels(ctx.qp_quantize_pack_channels(x, channels, q, d_cqp), rows, channels, q, d_cqp)
+            row["channels_ds"] = mse_of(y)
+            print(json.dumps(row))
+    ctx.qp_get_status()
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -578,6 +625,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--quality", action="store_true",
+                    help="print the quantization MSE of every clip method on the ViT-shaped configs (one GPU)")
     ap.add_argument("--sweep", action="store_true",
                     help="kernel-by-kernel cold-cache table over the configurations (one JSON line per row)")
     ap.add_argument("--sweep-max-log2", type=int, default=28)
@@ -586,6 +635,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         return reference_main(args)
+    if args.quality:
+        return quality_main(args)
     if args.sweep:
         return sweep_main(args)
     return ours_main(args)
