@@ -115,24 +115,25 @@ __global__ void __launch_bounds__(CS_EVAL_CH * CS_EVAL_LANES, 4) ch_eval_kernel(
         lo[k] = q.x; hi[k] = q.y; sc[k] = q.z; iv[k] = q.w;
         acc[k] = 0.0;
     }
-    if (c < C) {
-        // batches of 8 rows of this lane (fp32 sums per batch), loaded four at a time ahead of their scoring
-        for (uint64_t r = r0 + rl; r < r1; r += 8 * CS_EVAL_LANES) {
+    if (c < C && r0 + rl < r1) {
+        // this lane's rows r0 + rl, r0 + rl + 8, ...: batches of 8 (fp32 sums per batch, then fp64)
+        const T* px = x + (r0 + rl) * C + c;
+        const size_t step = (size_t)CS_EVAL_LANES * C;
+        const uint64_t mine = (r1 - r0 - rl + CS_EVAL_LANES - 1) / CS_EVAL_LANES;
+        auto batch = [&](int count) {                       // count <= 8 rows from px on
             float p[CK];
 #pragma unroll
             for (int k = 0; k < CK; ++k) p[k] = 0.f;
 #pragma unroll
-            for (int half = 0; half < 2; ++half) {
+            for (int half = 0; half < 2; ++half) {          // four loads ahead of their scoring
                 float e[4];
 #pragma unroll
-                for (int it = 0; it < 4; ++it) {
-                    const uint64_t rr = r + (uint64_t)(half * 4 + it) * CS_EVAL_LANES;
-                    e[it] = rr < r1 ? cs_load(x + rr * C + c) : __int_as_float(0x7FC00000);  // NaN: skipped below
-                }
+                for (int it = 0; it < 4; ++it)
+                    e[it] = half * 4 + it < count ? cs_load(px + (half * 4 + it) * step) : __int_as_float(0x7FC00000);
 #pragma unroll
                 for (int it = 0; it < 4; ++it) {
                     const float v = e[it];
-                    const bool fin = qp_is_finite(v);
+                    const bool fin = qp_is_finite(v);       // also skips the rows beyond `count`
 #pragma unroll
                     for (int k = 0; k < CK; ++k) {
                         const float pos = qp_grid_pos(v, lo[k], hi[k], iv[k]);
@@ -144,7 +145,12 @@ __global__ void __launch_bounds__(CS_EVAL_CH * CS_EVAL_LANES, 4) ch_eval_kernel(
             }
 #pragma unroll
             for (int k = 0; k < CK; ++k) acc[k] += (double)p[k];
+        };
+        for (uint64_t b = 0; b < mine / 8; ++b) {
+            batch(8);
+            px += 8 * step;
         }
+        if (mine % 8) batch((int)(mine % 8));
     }
     // the 8 row lanes of a channel, merged in lane order
     __shared__ double sh[CS_EVAL_LANES][CK][CS_EVAL_CH];
