@@ -751,6 +751,39 @@ def test_roofline_sweep_sizes(ctx, log2n, dist):
     assert np.array_equal(ctx.qp_quantize_pack(db, 4, to_qp(qp_o)).cpu().numpy(), oracle.quantize_pack(xw, qp_o))
 
 
+@pytest.mark.parametrize("n", [(1 << 26) + 3, (1 << 27) + 4099])
+def test_search_forms_agree_beyond_one_wave(ctx, n):
+    """Longer tensors make the second form of the moments pass run two or three waves of blocks (its
+    replica sums are 32 bit).  The oracle needs minutes at this size, so the three scoring kernels,
+    each checked against the oracle at smaller sizes, are compared with one another: the two forms
+    of the interval pass share the partition and differ only in who adds what, the
+    candidate-by-candidate kernel is independent of both."""
+    x = si.flat_iid(n, 91, "laplace")
+    x[::1000] *= np.float32(6.0)                          # some elements beyond every clip range
+    d = dev(x)
+    d_stats = ctx.qp_stats(d, hist_bins=100)
+    curves, results = {}, {}
+    for path in (qp.QP_SEARCH_INTERVALS, qp.QP_SEARCH_INTERVALS_PLAIN, qp.QP_SEARCH_CANDIDATES):
+        ctx.qp_set_search_path(path)
+        try:
+            d_res, d_qp = ctx.qp_dsaciq_search(d, d_stats, 3)
+        finally:
+            ctx.qp_set_search_path(qp.QP_SEARCH_AUTO)
+        results[path] = (bytes(ctx.read_ds_result(d_res)), bytes(ctx.read_qparams(d_qp)))
+        curves[path] = np.array(ctx.qp_dsaciq_curve(100))
+    # same integer interval sums; the sums beyond the grid and of the squared offsets are fp32 batches
+    # folded into fp64 in another grouping, so the curves agree to rounding, not bit for bit
+    a, b = curves[qp.QP_SEARCH_INTERVALS], curves[qp.QP_SEARCH_INTERVALS_PLAIN]
+    assert np.all(np.abs(a - b) <= 1e-9 * b)
+    assert results[qp.QP_SEARCH_INTERVALS][1] == results[qp.QP_SEARCH_INTERVALS_PLAIN][1]       # the same winner
+    ref = curves[qp.QP_SEARCH_CANDIDATES]
+    assert np.all(np.abs(curves[qp.QP_SEARCH_INTERVALS] - ref) <= 2e-6 * ref)
+    res_iv = qp.DSResult.from_buffer_copy(results[qp.QP_SEARCH_INTERVALS][0])
+    res_c = qp.DSResult.from_buffer_copy(results[qp.QP_SEARCH_CANDIDATES][0])
+    assert res_iv.k_star == res_c.k_star or ref[res_iv.k_star] <= ref[res_c.k_star] * (1 + 1e-6)
+    assert ctx.qp_get_status() == 0
+
+
 def test_largest_sweep_size_sampled(ctx):
     """1 GiB fp32 (2^28 elements): packed words and reconstructions checked on sampled
     positions the oracle computes one by one, plus whole-buffer invariants."""
