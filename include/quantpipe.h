@@ -110,9 +110,26 @@ typedef struct {
  * qp_destroy frees it.  Errors: QP_ERR_INVALID_ARG, QP_ERR_CUDA. */
 int32_t qp_create(int device, qp_ctx** out);
 int32_t qp_destroy(qp_ctx* ctx);
-/* Waits for `stream`, then returns and clears the device status word (QP_DEV_* bits),
- * or a negative qp_status if a CUDA error is pending. */
+/* Waits for `stream`, then returns and clears the device status word (QP_DEV_* bits), or a
+ * negative qp_status: QP_ERR_CUDA if a CUDA error is pending, QP_ERR_TIMEOUT if the word
+ * carries QP_DEV_STREAM_TIMEOUT (a bounded wait inside a kernel ran out: the results of the
+ * calls since the last qp_get_status are invalid; the call also puts the scratch of the
+ * cooperative kernels back to its initial state, so the context can be used again at once;
+ * qp_last_error gives the whole word). */
 int32_t qp_get_status(qp_ctx* ctx, void* stream);
+/* Test hook for the time-out paths (no counterpart in the paper; not for production use).
+ * Every wait inside the kernels is bounded: a wait for a tile copy by a number of clock
+ * cycles, a wait at a grid-wide barrier by a number of polls.  This call replaces the limits
+ * of later launches on this context: tile_wait_cycles < 0 and barrier_polls = 0 restore the
+ * defaults (about two seconds; a quarter of a second at least); tile_wait_cycles = 0 makes a
+ * wait give up at the first attempt that finds the copy still in flight.  (The second wait that
+ * a block which gave up grants its own copies in flight before it leaves always keeps the
+ * default.)  barrier_extra_arrivals = 1 makes every grid barrier wait for one arrival more
+ * than there are blocks, so that it can only end by running out.  A wait that runs out
+ * raises QP_DEV_STREAM_TIMEOUT, the kernel leaves without output, and nothing faults.
+ * Drops the stored graphs (they carry the old limits).  Errors: QP_ERR_INVALID_ARG. */
+int32_t qp_set_wait_limit_for_testing(qp_ctx* ctx, long long tile_wait_cycles, uint32_t barrier_polls,
+                                      int barrier_extra_arrivals);
 /* Text of the last error recorded on this context (never NULL). */
 const char* qp_last_error(qp_ctx* ctx);
 const char* qp_status_string(int32_t status);
@@ -141,6 +158,9 @@ int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out);
  * One call fills *d_out (device memory, 80 bytes, 8-byte aligned) from the n elements at
  * d_x.  Two passes over x (sums/min/max, then deviations about the mean), fp64 merges in a
  * fixed order: results are bit-reproducible run to run.  n = 0 gives all-zero statistics.
+ * For 16-byte aligned tensors of at least 128 KB both passes run in one cooperative launch
+ * (one block per SM; the second pass starts on the tiles that the first one left in shared
+ * memory), see qp_set_stats_path.
  * hist_bins > 0 asks the second pass to carry the directed search's histogram along
  * (hist_bins equal bins over [min, max]; only its peak count is kept, in hist_peak): a later
  * qp_dsaciq_search with the same hist_bins then skips its own histogram pass.  The fusion is
@@ -155,6 +175,17 @@ int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_b
  * will equal hist_bins), else 0.  Host, pure: it depends only on the pointer's alignment, the
  * size and hist_bins. */
 int qp_stats_carries_histogram(const void* d_x, int dtype, uint64_t n, int hist_bins);
+/* How qp_stats runs its two passes on 16-byte aligned tensors of at least 128 KB (an execution
+ * option without a counterpart in the paper; the statistics agree to the last bits or so, the
+ * histogram's peak count is identical):
+ *   QP_STATS_TWO_KERNELS  one kernel per pass
+ *   QP_STATS_FUSED        one cooperative launch for both (falls back to two kernels on a device
+ *                         that cannot hold it)
+ *   QP_STATS_AUTO         the cooperative launch (default)
+ * A grid barrier or tile wait of the cooperative launch that runs out sets QP_DEV_STREAM_TIMEOUT
+ * and the launch ends without output. */
+enum { QP_STATS_AUTO = 0, QP_STATS_TWO_KERNELS = 1, QP_STATS_FUSED = 2 };
+int32_t qp_set_stats_path(qp_ctx* ctx, int path);
 
 /* Statistics for callers that cannot allocate device memory (no counterpart in the paper;
  * same results as qp_stats).  Some code may not call cudaMalloc or any allocating routine:
@@ -171,6 +202,8 @@ int qp_stats_carries_histogram(const void* d_x, int dtype, uint64_t n, int hist_
  *     (the counters that must start at zero are cleared on `stream` first).  Two calls
  *     that overlap on the GPU (different streams, no ordering between them) race on it and
  *     give wrong statistics: order them.
+ *   - There is no context, hence no status word to read: NaN and +-Inf among the input are
+ *     reported through d_out->nonfinite only.
  * Errors: QP_ERR_INVALID_ARG (NULL), QP_ERR_UNSUPPORTED_DTYPE, QP_ERR_ALIGNMENT,
  * QP_ERR_TOO_LARGE, QP_ERR_CUDA. */
 #define QP_STATS_STATIC_MAX_N (1ull << 31)
@@ -266,6 +299,13 @@ uint64_t qp_graph_replays(qp_ctx* ctx);
 /* Copies the MSE of every candidate of the last search on this context (steps+1 values)
  * to host memory after waiting for `stream`.  Diagnostic. */
 int32_t qp_dsaciq_curve(qp_ctx* ctx, double* h_curve, int capacity, void* stream);
+/* Copies the quantizer of every candidate of the last search on this context (steps+1 entries:
+ * the clip range [mean - F b_k, mean + F b_k] as the kernels rounded it to fp32, its scale and
+ * reciprocal, bits; flags bit 0 marks an empty range, which is also what a step that is not a
+ * candidate looks like) to host memory after waiting for `stream`.  Diagnostic: with it a
+ * candidate's error can be recomputed for exactly the quantizer that the library scored.
+ * Errors: QP_ERR_INVALID_ARG (NULL, no search yet), QP_ERR_BUFFER_TOO_SMALL, QP_ERR_CUDA. */
+int32_t qp_dsaciq_candidates(qp_ctx* ctx, qp_qparams_t* h_out, int capacity, void* stream);
 /* Policy of the paper's evaluation (Sec. 3): the search is switched on at 4 bits and below. */
 int32_t qp_policy_use_ds(int bits);
 
@@ -398,6 +438,9 @@ int32_t qp_dsaciq_search_channels(qp_ctx* ctx, const void* d_x, int dtype, uint6
                                   const qp_stats_t* d_stats, int bits, int bmode, int steps, int hist_bins,
                                   qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, void* stream);
 int32_t qp_dsaciq_curve_channels(qp_ctx* ctx, uint32_t channel, double* h_curve, int capacity, void* stream);
+/* The candidates' quantizers of the last channel-wise search, as qp_dsaciq_candidates:
+ * h_out[c * (steps + 1) + k] for channel c and step k; capacity in entries.  Diagnostic. */
+int32_t qp_dsaciq_candidates_channels(qp_ctx* ctx, qp_qparams_t* h_out, uint64_t capacity, void* stream);
 
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------
@@ -433,7 +476,8 @@ int32_t qp_dsaciq_curve_channels(qp_ctx* ctx, uint32_t channel, double* h_curve,
  *   QP_SENDER_AUTO   fused where it is the faster of the two on a B200: n <= 2^20 with the
  *                    search, n <= 2^21 otherwise (default)
  * A grid barrier that does not complete within about a quarter of a second sets
- * QP_DEV_STREAM_TIMEOUT in the status word and the launch ends without output. */
+ * QP_DEV_STREAM_TIMEOUT in the status word and the launch ends without output
+ * (qp_get_status then returns QP_ERR_TIMEOUT). */
 enum { QP_SENDER_AUTO = 0, QP_SENDER_CHAIN = 1, QP_SENDER_FUSED = 2 };
 int32_t qp_set_sender_path(qp_ctx* ctx, int path);
 int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits, int method, int bmode,

@@ -27,6 +27,7 @@ QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS, QP_SEARCH_INTERVALS_PLAIN = 0, 1, 2, 3
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
+QP_STATS_AUTO, QP_STATS_TWO_KERNELS, QP_STATS_FUSED = 0, 1, 2
 QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT, QP_CLIP_MIDRISE = 0, 1, 2, 0x10, 0x20
 QP_B_MIDRISE = 0x10
 QP_B_GAUSS = 0x20
@@ -40,6 +41,7 @@ EXPORTS = (
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
     "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_dsaciq_search_channels", "qp_dsaciq_curve_channels", "qp_clip_qparams_channels_device",
     "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range", "qp_sender_channels_device",
+    "qp_set_stats_path", "qp_dsaciq_candidates", "qp_dsaciq_candidates_channels", "qp_set_wait_limit_for_testing",
 )
 
 
@@ -130,6 +132,10 @@ def load() -> C.CDLL:
     L.qp_stats_carries_histogram.restype = C.c_int
     L.qp_set_graph_replay.argtypes = [vp, C.c_int]
     L.qp_set_sender_path.argtypes = [vp, C.c_int]
+    L.qp_set_stats_path.argtypes = [vp, C.c_int]
+    L.qp_dsaciq_candidates.argtypes = [vp, C.POINTER(QParams), C.c_int, vp]
+    L.qp_dsaciq_candidates_channels.argtypes = [vp, C.POINTER(QParams), u64, vp]
+    L.qp_set_wait_limit_for_testing.argtypes = [vp, C.c_longlong, C.c_uint32, C.c_int]
     L.qp_graph_replays.argtypes = [vp]
     L.qp_graph_replays.restype = u64
     L.qp_controller_init.argtypes = [C.POINTER(Controller), C.c_int, dbl, dbl, u64, u64, C.POINTER(i32), C.c_int,
@@ -357,6 +363,26 @@ class Context:
 
     def qp_set_sender_path(self, path: int):
         self._check(self._lib.qp_set_sender_path(self._h, path))
+
+    def qp_set_stats_path(self, path: int):
+        self._check(self._lib.qp_set_stats_path(self._h, path))
+
+    def qp_set_wait_limit_for_testing(self, tile_wait_cycles: int = -1, barrier_polls: int = 0,
+                                      barrier_extra_arrivals: int = 0):
+        self._check(self._lib.qp_set_wait_limit_for_testing(self._h, tile_wait_cycles, barrier_polls,
+                                                            barrier_extra_arrivals))
+
+    def qp_dsaciq_candidates(self, steps: int):
+        """Host array of the steps + 1 candidate quantizers of the last search (synchronises)."""
+        buf = (QParams * (steps + 1))()
+        self._check(self._lib.qp_dsaciq_candidates(self._h, buf, steps + 1, _stream(self.device)))
+        return buf
+
+    def qp_dsaciq_candidates_channels(self, channels: int, steps: int):
+        """Host array [channels * (steps + 1)] of the candidate quantizers of the last channel-wise search."""
+        buf = (QParams * (channels * (steps + 1)))()
+        self._check(self._lib.qp_dsaciq_candidates_channels(self._h, buf, channels * (steps + 1), _stream(self.device)))
+        return buf
 
     def qp_set_graph_replay(self, on: bool):
         self._check(self._lib.qp_set_graph_replay(self._h, 1 if on else 0))

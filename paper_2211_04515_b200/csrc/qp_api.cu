@@ -45,6 +45,8 @@ extern "C" const char* qp_last_error(qp_ctx* ctx) { return ctx ? ctx->err : "no 
 
 // ----------------------------------------------------------------- context
 
+static void qp_drop_graphs(qp_ctx* ctx);
+
 static size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 extern "C" int32_t qp_create(int device, qp_ctx** out)
@@ -62,6 +64,8 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     memset(c, 0, sizeof *c);
     c->device = device;
     strcpy(c->err, "ok");
+    c->wait_cycles = QP_WAIT_CYCLES_DEFAULT;
+    c->spin_limit = QP_SPIN_LIMIT_DEFAULT;
     if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
         delete c;
         return QP_ERR_CUDA;
@@ -119,8 +123,6 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     return QP_OK;
 }
 
-static void qp_drop_graphs(qp_ctx* ctx);
-
 extern "C" int32_t qp_destroy(qp_ctx* ctx)
 {
     if (!ctx) return QP_ERR_INVALID_ARG;
@@ -148,13 +150,16 @@ extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
         return QP_ERR_CUDA;
     }
     if (word & QP_DEV_STREAM_TIMEOUT) {
-        // a cooperative sender that gave up left its arrival counter and histogram mid-way
+        // a cooperative launch that gave up may have left its arrival counters and histogram mid-way
         e = cudaMemsetAsync(ctx->d_fused, 0, 256 + sizeof(unsigned long long) * 4096, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) {
             snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_get_status: %s", cudaGetErrorString(e));
             return QP_ERR_CUDA;
         }
+        snprintf(ctx->err, sizeof ctx->err, "%s: a bounded wait on the device ran out (status word 0x%x); "
+                 "the results of the calls since the last qp_get_status are invalid", qp_status_string(QP_ERR_TIMEOUT), word);
+        return QP_ERR_TIMEOUT;
     }
     return (int32_t)word;
 }
@@ -167,6 +172,27 @@ extern "C" int32_t qp_set_search_path(qp_ctx* ctx, int path)
     if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS_PLAIN) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
     ctx->moments_form = path == QP_SEARCH_INTERVALS_PLAIN ? 1 : 0;
     ctx->search_path = path == QP_SEARCH_INTERVALS_PLAIN ? QP_SEARCH_INTERVALS : path;
+    return QP_OK;
+}
+
+extern "C" int32_t qp_set_wait_limit_for_testing(qp_ctx* ctx, long long tile_wait_cycles, uint32_t barrier_polls,
+                                                 int barrier_extra_arrivals)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (barrier_extra_arrivals < 0 || barrier_extra_arrivals > 1) return qp_fail(ctx, QP_ERR_INVALID_ARG, "barrier_extra_arrivals");
+    ctx->wait_cycles = tile_wait_cycles < 0 ? QP_WAIT_CYCLES_DEFAULT : tile_wait_cycles;
+    ctx->spin_limit = barrier_polls == 0 ? QP_SPIN_LIMIT_DEFAULT : barrier_polls;
+    ctx->bar_extra = barrier_extra_arrivals;
+    qp_device_guard guard(ctx->device);
+    qp_drop_graphs(ctx);                      // recorded launches carry the old limits
+    return QP_OK;
+}
+
+extern "C" int32_t qp_set_stats_path(qp_ctx* ctx, int path)
+{
+    if (!ctx) return QP_ERR_INVALID_ARG;
+    if (path < QP_STATS_AUTO || path > QP_STATS_FUSED) return qp_fail(ctx, QP_ERR_INVALID_ARG, "statistics path");
+    ctx->stats_path = path;
     return QP_OK;
 }
 
@@ -425,7 +451,7 @@ static int32_t check_x(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n)
 // launches the stored graph instead.  Calls on the legacy default stream, or on a stream the
 // caller is itself capturing, are enqueued directly as before.
 template <typename F>
-static int32_t qp_graphed(qp_ctx* ctx, cudaStream_t stream, const unsigned long long (&key)[8], F&& enqueue)
+static int32_t qp_graphed(qp_ctx* ctx, cudaStream_t stream, const unsigned long long (&key)[QP_GRAPH_KEY_WORDS], F&& enqueue)
 {
     if (!ctx->graphs_on || stream == nullptr || stream == cudaStreamLegacy || stream == cudaStreamPerThread)
         return enqueue();
@@ -516,8 +542,10 @@ extern "C" int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n,
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const unsigned long long key[8] = {1, (unsigned long long)(uintptr_t)d_x, (unsigned long long)dtype, n,
-                                       (unsigned long long)hist_bins, (unsigned long long)(uintptr_t)d_out, 0, 0};
+    // one word per argument: no two argument sets share a key
+    const unsigned long long key[QP_GRAPH_KEY_WORDS] = {1, (unsigned long long)(uintptr_t)d_x, (unsigned long long)dtype, n,
+                                                        (unsigned long long)hist_bins, (unsigned long long)(uintptr_t)d_out,
+                                                        (unsigned long long)ctx->stats_path};
     ctx->last_x = d_x;                    // the second pass walks backwards (the plain kernels for small tensors do not,
     ctx->last_x_end = 0;                  // but those tensors sit in L2 whole)
     return qp_graphed(ctx, s, key, [&] { return qp_launch_stats(ctx, d_x, dtype, n, hist_bins, d_out, s); });
@@ -571,17 +599,18 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const unsigned long long key[8] = {2, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_stats,
-                                       (unsigned long long)dtype | (unsigned long long)bits << 8 |
-                                           (unsigned long long)bmode << 16 | (unsigned long long)(ctx->search_path | ctx->moments_form << 2) << 24 |
-                                           (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
-                                       (unsigned long long)(uintptr_t)d_out, (unsigned long long)(uintptr_t)d_qp_out, 0};
+    const unsigned long long key[QP_GRAPH_KEY_WORDS] = {
+        2, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_stats,
+        (unsigned long long)(uintptr_t)d_out, (unsigned long long)(uintptr_t)d_qp_out,
+        (unsigned long long)dtype | (unsigned long long)bits << 8 | (unsigned long long)ctx->search_path << 16 |
+            (unsigned long long)ctx->moments_form << 24,                   // each below 256
+        (unsigned long long)(unsigned)bmode, (unsigned long long)steps, (unsigned long long)hist_bins};
     rc = qp_graphed(ctx, s, key, [&] {
         return qp_launch_search(ctx, d_x, dtype, n, d_stats, bits, bmode, steps, hist_bins,
                                 qp_host_aciq_F(bits, (bmode & QP_B_GAUSS) ? QP_DIST_GAUSS : QP_DIST_LAPLACE), d_out,
                                 d_qp_out, s);
     });
-    if (rc == QP_OK) ctx->last_steps = steps;
+    if (rc == QP_OK) { ctx->last_steps = steps; ctx->last_bits = bits; }
     ctx->last_x = d_x;                    // both scoring paths walk x forwards
     ctx->last_x_end = 1;
     return rc;
@@ -601,6 +630,32 @@ extern "C" int32_t qp_dsaciq_curve(qp_ctx* ctx, double* h_curve, int capacity, v
         snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_dsaciq_curve: %s", cudaGetErrorString(e));
         return QP_ERR_CUDA;
     }
+    return QP_OK;
+}
+
+extern "C" int32_t qp_dsaciq_candidates(qp_ctx* ctx, qp_qparams_t* h_out, int capacity, void* stream)
+{
+    if (!ctx || !h_out) return QP_ERR_INVALID_ARG;
+    if (ctx->last_steps < 1) return qp_fail(ctx, QP_ERR_INVALID_ARG, "no search has run on this context");
+    const int ncand = ctx->last_steps + 1;
+    if (capacity < ncand) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "candidate buffer");
+    qp_device_guard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    float4* tmp = new (std::nothrow) float4[ncand];
+    if (!tmp) return qp_fail(ctx, QP_ERR_CUDA, "out of host memory");
+    cudaError_t e = cudaMemcpyAsync(tmp, ctx->d_cand, sizeof(float4) * ncand, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        delete[] tmp;
+        snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_dsaciq_candidates: %s", cudaGetErrorString(e));
+        return QP_ERR_CUDA;
+    }
+    for (int k = 0; k < ncand; ++k) {
+        h_out[k].lo = tmp[k].x; h_out[k].hi = tmp[k].y; h_out[k].scale = tmp[k].z; h_out[k].inv_scale = tmp[k].w;
+        h_out[k].bits = ctx->last_bits;
+        h_out[k].flags = tmp[k].y > tmp[k].x ? 0 : 1;
+    }
+    delete[] tmp;
     return QP_OK;
 }
 
@@ -688,7 +743,7 @@ static int32_t sender_on_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_
         rc = qp_launch_sender_fused(ctx, d_x, dtype, n, bits, method, bmode, steps, hist_bins,
                                     qp_host_aciq_F(bits, QP_DIST_LAPLACE), d_packed, d_qp_out, st,
                                     static_cast<cudaStream_t>(stream));
-        if (rc == QP_OK && use_ds) ctx->last_steps = steps;
+        if (rc == QP_OK && use_ds) { ctx->last_steps = steps; ctx->last_bits = bits; }
         if (rc != QP_WARN_INFEASIBLE) return rc;               // else: this device cannot hold the grid
     }
     rc = qp_stats(ctx, d_x, dtype, n, use_ds ? hist_bins : 0, st, stream);
@@ -715,18 +770,23 @@ extern "C" int32_t qp_sender_device(qp_ctx* ctx, const void* d_x, int dtype, uin
         return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
     qp_stats_t* st = d_stats_out ? d_stats_out : ctx->d_tmp_stats;
     // The inner calls see a capturing stream while this one records, and enqueue directly into it.
-    const unsigned long long key[8] = {3, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_packed,
-                                       (unsigned long long)dtype | (unsigned long long)bits << 8 |
-                                           (unsigned long long)bmode << 16 | (unsigned long long)(ctx->search_path | ctx->moments_form << 2) << 24 |
-                                           (unsigned long long)((method & 0xF) == QP_CLIP_DSACIQ) << 28 | (unsigned long long)method << 56 |
-                                           (unsigned long long)ctx->sender_path << 29 |
-                                           (unsigned long long)steps << 32 | (unsigned long long)hist_bins << 48,
-                                       packed_capacity, (unsigned long long)(uintptr_t)d_qp_out,
-                                       (unsigned long long)(uintptr_t)st};
-    return qp_graphed(ctx, static_cast<cudaStream_t>(stream), key, [&]() -> int32_t {
+    // Every argument and every context option that the recorded kernels depend on has a word (or a
+    // byte of a word whose fields are each below 256) of its own, so that two different calls can
+    // never share a key.
+    const unsigned long long key[QP_GRAPH_KEY_WORDS] = {
+        3, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_packed, packed_capacity,
+        (unsigned long long)(uintptr_t)d_qp_out, (unsigned long long)(uintptr_t)st,
+        (unsigned long long)dtype | (unsigned long long)bits << 8 | (unsigned long long)ctx->search_path << 16 |
+            (unsigned long long)ctx->moments_form << 24 | (unsigned long long)ctx->sender_path << 32 |
+            (unsigned long long)ctx->stats_path << 40,
+        (unsigned long long)(unsigned)method, (unsigned long long)(unsigned)bmode, (unsigned long long)steps,
+        (unsigned long long)hist_bins};
+    const int32_t rc = qp_graphed(ctx, static_cast<cudaStream_t>(stream), key, [&]() -> int32_t {
         return sender_on_device(ctx, d_x, dtype, n, bits, method, bmode, steps, hist_bins, d_packed, packed_capacity,
                                 d_qp_out, st, stream);
     });
+    if (rc >= 0 && (method & 0xF) == QP_CLIP_DSACIQ) { ctx->last_steps = steps; ctx->last_bits = bits; }   // also after a replay
+    return rc;
 }
 
 // ------------------------------------------- host-buffer sender and receiver

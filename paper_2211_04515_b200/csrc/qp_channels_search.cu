@@ -13,6 +13,8 @@
 //                     block partials per (row block, channel, candidate)
 //   ch_pick_kernel    block per channel: partials merged in row-block order, first minimum wins
 // Work is (steps + 1) * 9 fp32 instructions per element, as in the per-tensor candidate path.
+#include <stdlib.h>
+
 #include "qp_internal.cuh"
 
 namespace {
@@ -258,6 +260,8 @@ int32_t search_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C
     ctx->ch_last_ncp = ncp;
     ctx->ch_last_channels = C;
     ctx->ch_curve_offset = o_curve;
+    ctx->ch_cand_offset = o_cand;
+    ctx->ch_last_bits = bits;
     return qp_check_launch(ctx, "qp_dsaciq_search_channels");
 }
 
@@ -311,5 +315,37 @@ extern "C" int32_t qp_dsaciq_curve_channels(qp_ctx* ctx, uint32_t channel, doubl
         cudaGetLastError();
         return qp_fail(ctx, QP_ERR_CUDA, "copying the curve");
     }
+    return QP_OK;
+}
+
+extern "C" int32_t qp_dsaciq_candidates_channels(qp_ctx* ctx, qp_qparams_t* h_out, uint64_t capacity, void* stream)
+{
+    if (!ctx || !h_out) return QP_ERR_INVALID_ARG;
+    if (ctx->ch_last_steps < 1 || !ctx->d_ch_search) return qp_fail(ctx, QP_ERR_INVALID_ARG, "no channel search has run on this context");
+    const int ncand = ctx->ch_last_steps + 1, ncp = ctx->ch_last_ncp;
+    const uint32_t C = ctx->ch_last_channels;
+    if (capacity < (uint64_t)C * ncand) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "candidate buffer");
+    qp_device_guard guard(ctx->device);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t count = (size_t)C * ncp;
+    float4* tmp = static_cast<float4*>(malloc(sizeof(float4) * count));
+    if (!tmp) return qp_fail(ctx, QP_ERR_CUDA, "out of host memory");
+    cudaError_t e = cudaMemcpyAsync(tmp, static_cast<char*>(ctx->d_ch_search) + ctx->ch_cand_offset, sizeof(float4) * count,
+                                    cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) {
+        free(tmp);
+        cudaGetLastError();
+        return qp_fail(ctx, QP_ERR_CUDA, "copying the candidates");
+    }
+    for (uint32_t c = 0; c < C; ++c)
+        for (int k = 0; k < ncand; ++k) {
+            const float4 q = tmp[(size_t)c * ncp + k];
+            qp_qparams_t& o = h_out[(size_t)c * ncand + k];
+            o.lo = q.x; o.hi = q.y; o.scale = q.z; o.inv_scale = q.w;
+            o.bits = ctx->ch_last_bits;
+            o.flags = q.y > q.x ? 0 : 1;
+        }
+    free(tmp);
     return QP_OK;
 }

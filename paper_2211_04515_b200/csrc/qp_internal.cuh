@@ -42,8 +42,9 @@ constexpr int QP_IV_BLOCKS_PER_SM = 3;
 struct qp_iv_total { unsigned long long n, s1; };       // per interval: count, sum of offsets (fixed point)
 
 // One instantiated graph of a multi-kernel call, keyed by every argument that the kernels bake in.
+constexpr int QP_GRAPH_KEY_WORDS = 12;
 struct qp_graph_entry {
-    unsigned long long key[8];
+    unsigned long long key[QP_GRAPH_KEY_WORDS];
     cudaGraphExec_t exec;
     unsigned launches;                   // kernels inside the graph
     int32_t rc;                          // status the recorded call returned (QP_OK or a warning)
@@ -75,7 +76,12 @@ struct qp_ctx {
     int search_path;                     // 0 auto, 1 candidate scoring, 2 interval moments
     int moments_form;                    // interval moments: 0 auto (second form where it applies), 1 always the first form
     int sender_path;                     // 0 auto, 1 kernel chain, 2 single cooperative launch where it applies
+    int stats_path;                      // 0 auto, 1 two kernels, 2 one cooperative launch where it applies
     int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
+    int stats_fused_checked, stats_fused_ok;   // the same for the one-launch statistics
+    long long wait_cycles;               // limit of a wait for a tile copy (clock cycles)
+    unsigned spin_limit;                 // limit of a grid-barrier wait (polls)
+    int bar_extra;                       // test only: arrivals a grid barrier waits for beyond the grid size
     size_t fused_dyn_max;                // largest slice (bytes of dynamic shared memory) per block
     void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
     void* d_ch_part;                     // channel-wise statistics: block partials, allocated on first use
@@ -85,6 +91,8 @@ struct qp_ctx {
     int ch_last_steps, ch_last_ncp;      // of the last channel-wise search (for qp_dsaciq_curve_channels)
     uint32_t ch_last_channels;
     size_t ch_curve_offset;
+    size_t ch_cand_offset;               // candidates of the last channel-wise search inside d_ch_search
+    int ch_last_bits;
     void* d_ch_stats;                    // channel-wise sender: statistics when the caller wants none back
     size_t ch_stats_bytes;
     qp_stats_t* d_tmp_stats;             // statistics / quantizer of the host-buffer entry points
@@ -96,10 +104,14 @@ struct qp_ctx {
     unsigned long long graph_hits;       // calls served by replaying a stored graph
     qp_graph_entry graphs[QP_GRAPH_SLOTS];
     int last_steps;                      // steps of the last search (for qp_dsaciq_curve)
+    int last_bits;                       // its bit-width (for qp_dsaciq_candidates)
     const void* last_x;                  // tensor of the last full pass on this context and where that pass
     int last_x_end;                      // stopped (1 = at the end of the tensor): the next pass starts there (L2)
     char err[256];
 };
+
+constexpr long long QP_WAIT_CYCLES_DEFAULT = 4000000000ll;   // about two seconds
+constexpr unsigned QP_SPIN_LIMIT_DEFAULT = 1u << 22;          // x 64 ns sleeps: a quarter of a second at least
 
 int32_t qp_fail(qp_ctx* ctx, int32_t status, const char* what);
 int32_t qp_check_launch(qp_ctx* ctx, const char* what);

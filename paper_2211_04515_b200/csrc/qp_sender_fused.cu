@@ -22,6 +22,7 @@
 // The grid barrier is an arrival counter in global memory; blocks are co-resident because
 // the launch is cooperative, and the wait is bounded all the same: a block that gives up
 // sets QP_DEV_STREAM_TIMEOUT in the status word and leaves.
+#include "qp_gridbar.cuh"
 #include "qp_internal.cuh"
 
 namespace {
@@ -34,7 +35,6 @@ constexpr uint64_t FS_MAX_N_SEARCH = 1ull << 20;  // above this the per-candidat
 constexpr uint64_t FS_AUTO_N = 1ull << 21;
 constexpr uint64_t FS_MAX_N = 6500000;            // slices of 148 SMs x ~190 KB of shared memory (checked per device)
 constexpr int FS_PART = 8;                        // doubles per block partial
-constexpr unsigned FS_SPIN_LIMIT = 1u << 22;      // x 64 ns sleeps: a quarter of a second at least
 constexpr int K = QP_EVAL_K;
 
 struct FsArgs {
@@ -56,42 +56,9 @@ struct FsArgs {
     qp_ds_setup* setup;
     unsigned* bar;                                // arrival counter, zero at entry
     unsigned* status;
+    unsigned spin_limit;                          // polls a grid-barrier wait may take
+    unsigned bar_extra;                           // 0; a test makes the barriers wait for more arrivals than blocks
 };
-
-__device__ __forceinline__ unsigned fs_ld_acquire(const unsigned* p)
-{
-    unsigned v;
-    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void fs_arrive_release(unsigned* p)
-{
-    asm volatile("red.release.gpu.global.add.u32 [%0], 1;" ::"l"(p) : "memory");
-}
-
-// All blocks arrive, then all leave.  The block's writes are ordered before the arrival by the
-// block barrier and the release; the acquire load orders the other blocks' writes before what
-// follows.  Returns false (for the whole block) when the wait ran out.
-__device__ __forceinline__ bool fs_grid_barrier(unsigned* bar, unsigned target, unsigned* status, int* s_ok)
-{
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        fs_arrive_release(bar);
-        int ok = 1;
-        unsigned spins = 0;
-        while (fs_ld_acquire(bar) < target) {
-            if (++spins > FS_SPIN_LIMIT) {
-                ok = 0;
-                atomicOr(status, QP_DEV_STREAM_TIMEOUT);
-                break;
-            }
-            if (spins > 64) __nanosleep(64);
-        }
-        *s_ok = ok;
-    }
-    __syncthreads();
-    return *s_ok != 0;
-}
 
 // Block reduction of N values at once; every thread gets the results, merged in warp order (the
 // same bits in every block).  OPS: 0 sum, 1 min, 2 max.  sh: FS_WARPS * N doubles.
@@ -214,7 +181,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
             p[0] = v5[0]; p[1] = v5[1]; p[2] = v5[2]; p[3] = v5[3]; p[4] = v5[4];
         }
     }
-    if (!fs_grid_barrier(a.bar, G, a.status, &s_ok)) return;
+    if (!qp_grid::barrier(a.bar, G + a.bar_extra, a.spin_limit, a.status, &s_ok)) return;
 
     // ---- phase 1: tensor-wide first moments (same in every block), then deviations and histogram
     double mean, mean_abs, mn_all, mx_all;
@@ -280,7 +247,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
                 if (c) atomicAdd(&a.hist[b], (unsigned long long)c);
             }
     }
-    if (!fs_grid_barrier(a.bar, 2 * G, a.status, &s_ok)) return;
+    if (!qp_grid::barrier(a.bar, 2 * G + a.bar_extra, a.spin_limit, a.status, &s_ok)) return;
 
     // ---- phase 2: statistics, then the clip range
     {
@@ -385,7 +352,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
             for (int j = 0; j < per_group; ++j) t += s_acc[j * groups + cg][ck];
             a.sums[(size_t)blockIdx.x * (FS_MAX_STEPS + 1) + c] = t;
         }
-        if (!fs_grid_barrier(a.bar, 3 * G, a.status, &s_ok)) return;
+        if (!qp_grid::barrier(a.bar, 3 * G + a.bar_extra, a.spin_limit, a.status, &s_ok)) return;
 
         // ---- phase 3: error curve, first minimum wins.  The G block sums of a candidate are merged
         // by four threads, each over a quarter of the blocks in index order (loads issued in
@@ -568,6 +535,8 @@ int32_t qp_launch_sender_fused(qp_ctx* ctx, const void* d_x, int dtype, uint64_t
     a.setup = ctx->d_setup;
     a.bar = reinterpret_cast<unsigned*>(ctx->d_fused);
     a.status = ctx->d_status;
+    a.spin_limit = ctx->spin_limit;
+    a.bar_extra = (unsigned)ctx->bar_extra;
     void* params[] = {&a};
     if (cudaLaunchCooperativeKernel(kernel, dim3(G), dim3(FS_THREADS), params, dyn, s) != cudaSuccess)
         return qp_check_launch(ctx, "qp_sender_device (cooperative launch)");

@@ -10,6 +10,7 @@
 // block scheduling.
 #include <type_traits>
 
+#include "qp_gridbar.cuh"
 #include "qp_internal.cuh"
 #include "qp_stream.cuh"
 
@@ -257,7 +258,7 @@ template <typename T>
 __global__ void __launch_bounds__(QP_THREADS) stats_stream_a(const T* __restrict__ x, uint64_t n, uint64_t ntiles,
                                                              qp_stats_partial* __restrict__ part,
                                                              unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out,
-                                                             unsigned* __restrict__ status)
+                                                             unsigned* __restrict__ status, long long wait_limit)
 {
     extern __shared__ __align__(128) unsigned char ring[];
     constexpr int EPV = qp_span<T>::EPV;
@@ -267,7 +268,7 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_a(const T* __restrict
     float tmn = inf, tmx = -inf;                             // exact in fp32: kept out of the fp64 path
 
     qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
-        reinterpret_cast<const unsigned char*>(x), ntiles, false, ring, status,
+        reinterpret_cast<const unsigned char*>(x), ntiles, false, ring, status, wait_limit,
         [&](const unsigned char* tile, uint64_t) {
             float e[VPT][EPV];
 #pragma unroll
@@ -359,7 +360,7 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
                                                              qp_stats_partial* __restrict__ part,
                                                              unsigned* __restrict__ ticket, qp_stats_t* __restrict__ out,
                                                              unsigned* __restrict__ status, int nb, int rep_shift,
-                                                             unsigned long long* __restrict__ hist)
+                                                             unsigned long long* __restrict__ hist, long long wait_limit)
 {
     extern __shared__ __align__(128) unsigned char ring[];
     constexpr int EPV = qp_span<T>::EPV;
@@ -395,7 +396,7 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
             }
         };
         qp_stream::for_each_tile<ST_TILE, ST_STAGES>(
-            reinterpret_cast<const unsigned char*>(x), ntiles, true, ring, status,
+            reinterpret_cast<const unsigned char*>(x), ntiles, true, ring, status, wait_limit,
             [&](const unsigned char* tile, uint64_t) {
                 float e[VPT][EPV];
 #pragma unroll
@@ -483,14 +484,383 @@ int32_t launch_streamed(qp_ctx* ctx, const T* x, uint64_t n, uint64_t ntiles, in
         return qp_check_launch(ctx, "qp_stats (histogram reset)");
     const uint64_t cap = (uint64_t)ctx->sm_count * ST_BLOCKS_PER_SM;
     const int blocks = (int)(ntiles > cap ? cap : ntiles);
-    stats_stream_a<T><<<blocks, QP_THREADS, ring, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status);
+    stats_stream_a<T><<<blocks, QP_THREADS, ring, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out, ctx->d_status,
+                                                       ctx->wait_cycles);
     if (fuse)
         stats_stream_b<T, true><<<blocks, QP_THREADS, smem_b, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out,
-                                                                   ctx->d_status, hist_bins, rep_shift, ctx->d_hist);
+                                                                   ctx->d_status, hist_bins, rep_shift, ctx->d_hist,
+                                                                   ctx->wait_cycles);
     else
         stats_stream_b<T, false><<<blocks, QP_THREADS, ring, s>>>(x, n, ntiles, ctx->d_part, ctx->d_ticket, d_out,
-                                                                  ctx->d_status, 0, 0, ctx->d_hist);
+                                                                  ctx->d_status, 0, 0, ctx->d_hist, ctx->wait_cycles);
     ctx->launches += 2;
+    return qp_check_launch(ctx, "qp_stats");
+}
+
+// ---------------------------------------------------------------------------------------
+// Both passes in ONE cooperative launch (one block per SM).  What the two streamed kernels
+// spend twice - a launch, the start of the copy ring, a last-block merge - is spent once, and
+// the second pass reads less: the ring is as large as shared memory allows (6 stages of 32 KB),
+// every block keeps the last tiles of its first pass in it, and the second pass, which walks the
+// block's tiles in the opposite order, starts on those resident tiles and fetches only the rest
+// (all SMs together hold ~28 MB, so a 129 MB tensor costs 129 + 101 MB of reads instead of 258,
+// and one that fits is read once).
+//
+//   pass A    tiles b, b + G, ... of block b through the ring: sum x, sum |x|, min, max, non-finite
+//   barrier   grid-wide (bounded); every block merges the G partials in index order: same mean everywhere
+//   pass B    the same tiles backwards: sum |x - mean|, sum (x - mean)^2, histogram over [min, max]
+//   exit      every block counts itself out; the last one merges pass B's partials, takes the
+//             histogram's peak, writes the statistics and leaves the barrier scratch at zero
+//
+// A block whose wait runs out (tile copy or barrier) raises the abort flag beside the barrier
+// counter and QP_DEV_STREAM_TIMEOUT in the status word, waits for its own copies in flight, and
+// still arrives at the barrier and counts itself out, so nobody waits for it and the scratch is
+// clean afterwards; no statistics are written then.
+constexpr int SF_THREADS = 512;
+constexpr int SF_TILE = 32768;
+constexpr int SF_STAGES = 6;
+
+struct SfArgs {
+    const void* x;
+    uint64_t n, ntiles;
+    qp_stats_partial* part;                       // [2 * grid]: pass A, then pass B
+    qp_stats_t* out;
+    unsigned* status;
+    int nb, rep_shift;                            // histogram bins (0: none) and log2 of the lane replicas per bin
+    unsigned long long* hist;                     // [nb] global counters (zeroed by block 0 before the barrier)
+    unsigned* bar;                                // [0] arrivals, [1] blocks that have left, [2] abort flag; zero at entry
+    long long wait_limit;
+    unsigned spin_limit, bar_extra;
+};
+
+template <typename T, bool HIST>
+__global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs a)
+{
+    extern __shared__ __align__(128) unsigned char smem[];
+    constexpr int EPV = qp_span<T>::EPV;
+    constexpr int VPT = SF_TILE / 16 / SF_THREADS;           // 16-byte vectors per thread and tile (4)
+    using Ring = qp_stream::ring<SF_TILE, SF_STAGES>;
+    __shared__ double sh[SF_THREADS / 32];
+    __shared__ int s_flag, s_ok;
+    __shared__ bool s_last;
+    __shared__ double s_mean, s_mean_abs, s_mn, s_mx;
+    __shared__ unsigned long long s_bad;
+    unsigned* sh_hist = reinterpret_cast<unsigned*>(smem + qp_stream::ring_bytes<SF_TILE, SF_STAGES>());
+    const T* x = static_cast<const T*>(a.x);
+    const unsigned char* base = static_cast<const unsigned char*>(a.x);
+    const uint64_t G = gridDim.x, first = blockIdx.x;
+    const uint64_t m = first < a.ntiles ? (a.ntiles - first + G - 1) / G : 0;     // tiles of this block
+    const float inf = __int_as_float(0x7F800000);
+    auto tile_src = [&](uint64_t i) { return base + (first + i * G) * (uint64_t)SF_TILE; };
+
+    Ring ring;
+    if (threadIdx.x == 0) s_flag = 0;
+    ring.init(smem);
+    unsigned pending = 0u;                                   // thread 0: stages with a copy in flight
+    bool ok = true;
+
+    // ---- pass A
+    if (threadIdx.x == 0)
+        for (uint64_t i = 0; i < (uint64_t)SF_STAGES && i < m; ++i) {
+            ring.issue((int)i, tile_src(i));
+            pending |= 1u << i;
+        }
+    AccA acc = {0.0, 0.0, (double)inf, (double)-inf, 0ull};
+    float tmn = inf, tmx = -inf;                             // exact in fp32: kept out of the fp64 path
+    for (uint64_t i = 0; i < m; ++i) {
+        const int s = (int)(i % SF_STAGES);
+        if (ring.wait(s, a.wait_limit)) { if (threadIdx.x == 0) pending &= ~(1u << s); }
+        else s_flag = 1;                                     // benign race: every writer writes 1
+        __syncthreads();
+        if (s_flag) { ok = false; break; }
+        const unsigned char* tile = ring.stage(s);
+        float e[VPT][EPV];
+#pragma unroll
+        for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * SF_THREADS + threadIdx.x) * 16, e[u]);
+        float ps = 0.f, psa = 0.f, pmn = inf, pmx = -inf;
+#pragma unroll
+        for (int u = 0; u < VPT; ++u)
+#pragma unroll
+            for (int k = 0; k < EPV; ++k) {
+                ps += e[u][k];
+                psa += fabsf(e[u][k]);
+                pmn = fminf(pmn, e[u][k]);
+                pmx = fmaxf(pmx, e[u][k]);
+            }
+        if (psa < inf) {                                     // every element finite (and no fp32 overflow)
+            acc.s += (double)ps;
+            acc.sa += (double)psa;
+            tmn = fminf(tmn, pmn);
+            tmx = fmaxf(tmx, pmx);
+        } else {
+#pragma unroll
+            for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                for (int k = 0; k < EPV; ++k) acc.add_scalar(e[u][k]);
+        }
+        if (i + SF_STAGES < m) {                             // the stage is filled again; the last ones stay resident
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                ring.issue(s, tile_src(i + SF_STAGES));
+                pending |= 1u << s;
+            }
+        }
+    }
+    if (ok) {
+        acc.mn = fmin(acc.mn, (double)tmn);
+        acc.mx = fmax(acc.mx, (double)tmx);
+        if (blockIdx.x == 0) {                               // elements after the last whole tile
+            const uint64_t t0 = a.ntiles * (SF_TILE / sizeof(T));
+            for (uint64_t i = t0 + threadIdx.x; i < a.n; i += SF_THREADS) acc.add_scalar(qp_load_one(x + i));
+            if (HIST)
+                for (int b = threadIdx.x; b < a.nb; b += SF_THREADS) a.hist[b] = 0ull;
+        }
+        const double bs = qp_block_sum(acc.s, sh);
+        const double bsa = qp_block_sum(acc.sa, sh);
+        const double bmn = qp_block_min(acc.mn, sh);
+        const double bmx = qp_block_max(acc.mx, sh);
+        const double bbad = qp_block_sum((double)acc.bad, sh);   // exact: counts are far below 2^53
+        if (threadIdx.x == 0) {
+            qp_stats_partial p;
+            p.s0 = bs; p.s1 = bsa; p.mn = bmn; p.mx = bmx; p.bad = (unsigned long long)bbad; p.pad = 0;
+            a.part[blockIdx.x] = p;
+        }
+    }
+    // a failed block drains its copies, flags the launch, and still arrives so that nobody waits for it
+    auto give_up = [&]() {
+        if (threadIdx.x == 0) {
+            atomicOr(a.status, QP_DEV_STREAM_TIMEOUT);
+            atomicExch(a.bar + 2, 1u);
+            for (int s = 0; s < SF_STAGES; ++s)
+                if (pending & (1u << s)) ring.wait(s, QP_STREAM_TIMEOUT_CYCLES);
+            pending = 0u;
+        }
+        __syncthreads();
+    };
+    if (!ok) give_up();
+    const bool met = qp_grid::barrier(a.bar, (unsigned)G + a.bar_extra, a.spin_limit, a.status, &s_ok);
+    if (!met && threadIdx.x == 0) atomicExch(a.bar + 2, 1u);
+    ok = ok && met && qp_grid::ld_acquire(a.bar + 2) == 0u;  // (the flag is read by all threads after the barrier's block barrier)
+
+    // ---- every block: tensor-wide first moments, merged in index order (the same bits everywhere)
+    if (ok) {
+        double s = 0.0, sa = 0.0, mn = (double)inf, mx = (double)-inf, bad = 0.0;
+        for (unsigned b = threadIdx.x; b < (unsigned)G; b += SF_THREADS) {
+            s += __ldcg(&a.part[b].s0);
+            sa += __ldcg(&a.part[b].s1);
+            mn = fmin(mn, __ldcg(&a.part[b].mn));
+            mx = fmax(mx, __ldcg(&a.part[b].mx));
+            bad += (double)__ldcg(&a.part[b].bad);
+        }
+        s = qp_block_sum(s, sh);
+        sa = qp_block_sum(sa, sh);
+        mn = qp_block_min(mn, sh);
+        mx = qp_block_max(mx, sh);
+        bad = qp_block_sum(bad, sh);
+        if (threadIdx.x == 0) {
+            const unsigned long long nbad = (unsigned long long)bad;
+            const unsigned long long nf = a.n - nbad;
+            s_bad = nbad;
+            s_mean = nf ? s / (double)nf : 0.0;
+            s_mean_abs = nf ? sa / (double)nf : 0.0;
+            s_mn = nf ? mn : 0.0;
+            s_mx = nf ? mx : 0.0;
+        }
+        __syncthreads();
+    }
+
+    // ---- pass B: the same tiles backwards; tile i lives in stage i % SF_STAGES in both passes, so the
+    // last SF_STAGES tiles of pass A are there already and each stage is refilled as it is consumed
+    double sd = 0.0, sv = 0.0;
+    if (ok) {
+        const double mean = s_mean;
+        const bool guard = s_bad != 0;
+        const float m_hi = (float)mean;
+        const float m_lo = (float)(mean - (double)m_hi);
+        const double dmn = s_mn, dmx = s_mx;
+        const bool hist_on = HIST && dmx > dmn;
+        const float fmn = (float)dmn;
+        const float inv_w = hist_on ? (float)((double)a.nb / (dmx - dmn)) : 0.f;
+        unsigned* my_hist = sh_hist + (threadIdx.x & ((1 << a.rep_shift) - 1));   // this lane's replica of the bins
+        const int top_bin = a.nb - 1, rep_shift = a.rep_shift;
+        if (HIST) {
+            for (int i = threadIdx.x; i < (a.nb << rep_shift); i += SF_THREADS) sh_hist[i] = 0u;
+            __syncthreads();
+        }
+        auto run = [&](auto guard_tag) {
+            constexpr bool GD = decltype(guard_tag)::value;
+            auto one = [&](float e, float& d1, float& d2) {
+                const float d = __fsub_rn(__fsub_rn(e, m_hi), m_lo);       // the mean as an unevaluated fp32 pair
+                if (!GD || qp_is_finite(e)) {
+                    d1 += fabsf(d);
+                    d2 = fmaf(d, d, d2);
+                    if (HIST) {      // x >= min, so the position is never negative; an empty range gives bin 0
+                        const int b = min(__float2int_rz(__fmul_rn(__fsub_rn(e, fmn), inv_w)), top_bin);
+                        atomicAdd(&my_hist[b << rep_shift], 1u);
+                    }
+                }
+            };
+            for (uint64_t j = 0; j < m; ++j) {
+                const uint64_t i = m - 1 - j;
+                const int s = (int)(i % SF_STAGES);
+                if (j >= (uint64_t)SF_STAGES) {                             // fetched in this pass
+                    if (ring.wait(s, a.wait_limit)) { if (threadIdx.x == 0) pending &= ~(1u << s); }
+                    else s_flag = 1;
+                    __syncthreads();
+                    if (s_flag) { ok = false; break; }
+                }
+                const unsigned char* tile = ring.stage(s);
+                float e[VPT][EPV];
+#pragma unroll
+                for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * SF_THREADS + threadIdx.x) * 16, e[u]);
+                float d1 = 0.f, d2 = 0.f;
+#pragma unroll
+                for (int u = 0; u < VPT; ++u)
+#pragma unroll
+                    for (int k = 0; k < EPV; ++k) one(e[u][k], d1, d2);
+                sd += (double)d1;
+                sv += (double)d2;
+                if (i >= (uint64_t)SF_STAGES) {
+                    __syncthreads();
+                    if (threadIdx.x == 0) {
+                        ring.issue(s, tile_src(i - SF_STAGES));
+                        pending |= 1u << s;
+                    }
+                }
+            }
+            if (ok && blockIdx.x == 0) {
+                float d1 = 0.f, d2 = 0.f;
+                const uint64_t t0 = a.ntiles * (SF_TILE / sizeof(T));
+                for (uint64_t i = t0 + threadIdx.x; i < a.n; i += SF_THREADS) one(qp_load_one(x + i), d1, d2);
+                sd += (double)d1;
+                sv += (double)d2;
+            }
+        };
+        if (guard) run(std::true_type{}); else run(std::false_type{});
+        if (!ok) give_up();
+        if (ok && HIST) {
+            __syncthreads();
+            const int reps = 1 << rep_shift;
+            for (int b = threadIdx.x; b < a.nb; b += SF_THREADS) {
+                unsigned long long c = 0;
+                for (int r = 0; r < reps; ++r) c += sh_hist[(b << rep_shift) + ((r + threadIdx.x) & (reps - 1))];
+                if (c) atomicAdd(&a.hist[b], c);
+            }
+        }
+    }
+    {
+        const double bsd = qp_block_sum(sd, sh);
+        const double bsv = qp_block_sum(sv, sh);
+        if (threadIdx.x == 0) {
+            a.part[G + blockIdx.x].s0 = bsd;
+            a.part[G + blockIdx.x].s1 = bsv;
+        }
+    }
+    __syncthreads();
+    ring.fini();
+
+    // ---- exit: every block counts itself out (on every path); the last one finishes the call
+    __threadfence();                                         // partials and histogram counts are out first
+    __syncthreads();
+    if (threadIdx.x == 0) s_last = (atomicAdd(a.bar + 1, 1u) == (unsigned)G - 1);
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const bool good = qp_grid::ld_acquire(a.bar + 2) == 0u;  // nobody gave up: this block holds the first moments too
+    if (good) {
+        double sa = 0.0, sb = 0.0;
+        for (unsigned k = threadIdx.x; k < (unsigned)G; k += SF_THREADS) {
+            sa += __ldcg(&a.part[G + k].s0);
+            sb += __ldcg(&a.part[G + k].s1);
+        }
+        sa = qp_block_sum(sa, sh);
+        sb = qp_block_sum(sb, sh);
+        double top = 0.0;
+        if (HIST) {
+            for (int k = threadIdx.x; k < a.nb; k += SF_THREADS) top = fmax(top, (double)__ldcg(&a.hist[k]));   // counts < 2^53
+            top = qp_block_max(top, sh);
+        }
+        if (threadIdx.x == 0) {
+            const unsigned long long nf = a.n - s_bad;
+            qp_stats_t st;
+            st.n = a.n;
+            st.nonfinite = s_bad;
+            st.mean = s_mean;
+            st.mean_abs = s_mean_abs;
+            st.mad = nf ? sa / (double)nf : 0.0;
+            st.var = nf ? sb / (double)nf : 0.0;
+            st.min = s_mn;
+            st.max = s_mx;
+            st.hist_peak = (HIST && s_mx > s_mn) ? (unsigned long long)top : 0ull;   // empty range: no histogram
+            st.hist_bins = HIST ? a.nb : 0;
+            st.reserved = 0;
+            *a.out = st;
+            if (s_bad) atomicOr(a.status, QP_DEV_NONFINITE);
+        }
+    }
+    if (threadIdx.x == 0) {                                  // everybody has left: the scratch goes back to zero
+        a.bar[0] = 0u;
+        a.bar[1] = 0u;
+        a.bar[2] = 0u;
+    }
+}
+
+constexpr size_t SF_RING_BYTES = qp_stream::ring_bytes<SF_TILE, SF_STAGES>();
+constexpr size_t SF_HIST_BYTES = 16 * 1024;
+
+// Whether this device can hold the one-launch statistics (checked once per context).
+bool stats_fused_usable(qp_ctx* ctx)
+{
+    if (!ctx->stats_fused_checked) {
+        ctx->stats_fused_checked = 1;
+        int coop = 0, optin = 0;
+        bool ok = cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
+                  cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, ctx->device) == cudaSuccess &&
+                  2 * ctx->sm_count <= QP_MAX_BLOCKS;
+        void* kernels[4] = {(void*)stats_fused_kernel<float, false>, (void*)stats_fused_kernel<float, true>,
+                            (void*)stats_fused_kernel<unsigned short, false>, (void*)stats_fused_kernel<unsigned short, true>};
+        for (int t = 0; ok && t < 4; ++t) {
+            const size_t dyn = SF_RING_BYTES + ((t & 1) ? SF_HIST_BYTES : 0);
+            cudaFuncAttributes fa;
+            int per_sm = 0;
+            ok = cudaFuncGetAttributes(&fa, kernels[t]) == cudaSuccess && (size_t)optin >= fa.sharedSizeBytes + dyn &&
+                 cudaFuncSetAttribute(kernels[t], cudaFuncAttributeMaxDynamicSharedMemorySize, (int)dyn) == cudaSuccess &&
+                 cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernels[t], SF_THREADS, dyn) == cudaSuccess &&
+                 per_sm >= 1;
+        }
+        if (!ok) cudaGetLastError();
+        ctx->stats_fused_ok = ok ? 1 : 0;
+    }
+    return ctx->stats_fused_ok != 0;
+}
+
+template <typename T>
+int32_t launch_fused(qp_ctx* ctx, const T* x, uint64_t n, int hist_bins, qp_stats_t* d_out, cudaStream_t s)
+{
+    const bool fuse = hist_bins >= 1 && hist_bins <= ST_FUSED_HIST_MAX;
+    int rep_shift = 5;
+    while (fuse && rep_shift > 0 && ((size_t)hist_bins << rep_shift) * sizeof(unsigned) > SF_HIST_BYTES) --rep_shift;
+    SfArgs a;
+    a.x = x;
+    a.n = n;
+    a.ntiles = n * sizeof(T) / SF_TILE;
+    a.part = ctx->d_part;
+    a.out = d_out;
+    a.status = ctx->d_status;
+    a.nb = fuse ? hist_bins : 0;
+    a.rep_shift = fuse ? rep_shift : 0;
+    a.hist = ctx->d_hist;
+    a.bar = reinterpret_cast<unsigned*>(ctx->d_fused) + 8;       // words 8..10 of the barrier scratch (the sender uses 0, 1)
+    a.wait_limit = ctx->wait_cycles;
+    a.spin_limit = ctx->spin_limit;
+    a.bar_extra = (unsigned)ctx->bar_extra;
+    const unsigned G = (unsigned)(a.ntiles < (uint64_t)ctx->sm_count ? a.ntiles : (uint64_t)ctx->sm_count);
+    const size_t dyn = SF_RING_BYTES + (fuse ? SF_HIST_BYTES : 0);
+    void* kernel = fuse ? (void*)stats_fused_kernel<T, true> : (void*)stats_fused_kernel<T, false>;
+    void* params[] = {&a};
+    if (cudaLaunchCooperativeKernel(kernel, dim3(G), dim3(SF_THREADS), params, dyn, s) != cudaSuccess)
+        return qp_check_launch(ctx, "qp_stats (cooperative launch)");
+    ctx->launches += 1;
     return qp_check_launch(ctx, "qp_stats");
 }
 
@@ -526,6 +896,10 @@ int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int
         return QP_OK;
     }
     const uint64_t ntiles = ((uintptr_t)d_x & 15u) ? 0 : n * (dtype == QP_F32 ? 4 : 2) / ST_TILE;
+    if (ntiles >= 8 && ctx->stats_path != QP_STATS_TWO_KERNELS && stats_fused_usable(ctx)) {
+        if (dtype == QP_F32) return launch_fused<float>(ctx, static_cast<const float*>(d_x), n, hist_bins, d_out, s);
+        return launch_fused<unsigned short>(ctx, static_cast<const unsigned short*>(d_x), n, hist_bins, d_out, s);
+    }
     if (ntiles >= 8) {                        // aligned and large enough for the streamed kernels to pay
         if (dtype == QP_F32)
             return launch_streamed<float>(ctx, static_cast<const float*>(d_x), n, ntiles, hist_bins, d_out, s);

@@ -8,9 +8,10 @@
 //   - every thread waits on full[s] (bounded), consumes the tile from shared memory, and a
 //     block barrier hands the stage back to the producer
 //
-// Every wait is bounded: if a tile does not arrive within QP_STREAM_TIMEOUT_CYCLES the block
-// raises QP_DEV_STREAM_TIMEOUT in the status word, stops issuing copies, gives the copies
-// still in flight a second bounded wait and returns, so the context stays usable.
+// Every wait is bounded: if a tile does not arrive within the wait limit (QP_STREAM_TIMEOUT_CYCLES
+// unless the context was given another one) the block raises QP_DEV_STREAM_TIMEOUT in the status
+// word, stops issuing copies, gives the copies still in flight a second bounded wait (always
+// QP_STREAM_TIMEOUT_CYCLES) and returns, so the context stays usable.
 #pragma once
 
 #include <cuda_runtime.h>
@@ -70,13 +71,31 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity)
     return ok != 0;
 }
 
-// Bounded wait; false on timeout.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity)
+// non-blocking form: has the phase with this parity completed?
+__device__ __forceinline__ bool mbar_test_wait(uint64_t* bar, unsigned parity)
 {
+    unsigned ok;
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+        "selp.u32 %0, 1, 0, p;\n"
+        "}\n"
+        : "=r"(ok)
+        : "r"(smem_addr(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Bounded wait; false on timeout.  limit = 0 does not wait at all: one non-blocking look
+// (try_wait may itself suspend the thread for a while, so it is not used then).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, long long limit = QP_STREAM_TIMEOUT_CYCLES)
+{
+    if (limit <= 0) return mbar_test_wait(bar, parity);
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
     while (!mbar_try_wait(bar, parity)) {
-        if (clock64() - t0 > QP_STREAM_TIMEOUT_CYCLES) return false;
+        if (clock64() - t0 > limit) return false;
     }
     return true;
 }
@@ -93,7 +112,7 @@ __host__ __device__ constexpr size_t ring_bytes() { return (size_t)TILE_BYTES * 
 // aligned, ring_bytes() long.  Returns false if a wait timed out (status bit raised).
 template <int TILE_BYTES, int STAGES, typename F>
 __device__ __forceinline__ bool for_each_tile(const unsigned char* __restrict__ base, uint64_t ntiles, bool reverse,
-                                              unsigned char* smem, unsigned* status, F&& consume)
+                                              unsigned char* smem, unsigned* status, long long wait_limit, F&& consume)
 {
     static_assert(TILE_BYTES % 128 == 0, "tile size");
     unsigned char* buf = smem;
@@ -124,7 +143,7 @@ __device__ __forceinline__ bool for_each_tile(const unsigned char* __restrict__ 
     for (uint64_t i = 0; i < mine; ++i) {
         const int s = (int)(i % STAGES);
         const unsigned parity = (unsigned)((i / STAGES) & 1);
-        if (!mbar_wait(&full[s], parity)) timed_out = 1;          // benign race: every writer writes 1
+        if (!mbar_wait(&full[s], parity, wait_limit)) timed_out = 1;   // benign race: every writer writes 1
         __syncthreads();
         if (timed_out) { ok = false; break; }
         consume(buf + (size_t)s * TILE_BYTES, tile_of(i));
@@ -150,5 +169,48 @@ __device__ __forceinline__ bool for_each_tile(const unsigned char* __restrict__ 
         for (int s = 0; s < STAGES; ++s) mbar_inval(&full[s]);
     return ok;
 }
+
+// The same ring as an object, for kernels that make more than one pass with it and want the
+// tiles of the last pass to stay in shared memory: stage s is filled by issue() (one thread),
+// every thread waits for it with wait(), and the caller's block barrier hands a stage back.
+// The parity expected at the next wait of each stage is tracked in a bit mask that every
+// thread keeps alike.
+template <int TILE_BYTES, int STAGES>
+struct ring {
+    static_assert(TILE_BYTES % 128 == 0 && STAGES <= 32, "ring shape");
+    unsigned char* buf;
+    uint64_t* full;
+    unsigned parity;                                    // bit s: parity of the next completion of stage s
+
+    __device__ __forceinline__ void init(unsigned char* smem)      // all threads; ends with a block barrier
+    {
+        buf = smem;
+        full = reinterpret_cast<uint64_t*>(smem + (size_t)TILE_BYTES * STAGES);
+        parity = 0u;
+        if (threadIdx.x == 0) {
+            for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
+            fence_barrier_init();
+        }
+        __syncthreads();
+    }
+    __device__ __forceinline__ unsigned char* stage(int s) const { return buf + (size_t)s * TILE_BYTES; }
+    __device__ __forceinline__ void issue(int s, const unsigned char* src)          // one thread
+    {
+        mbar_arrive_expect_tx(&full[s], TILE_BYTES);
+        bulk_load(stage(s), src, TILE_BYTES, &full[s]);
+    }
+    // all threads; false when the wait ran out (the parity bit is then left as it was)
+    __device__ __forceinline__ bool wait(int s, long long limit)
+    {
+        if (!mbar_wait(&full[s], (parity >> s) & 1u, limit)) return false;
+        parity ^= 1u << s;
+        return true;
+    }
+    __device__ __forceinline__ void fini()                                          // after a block barrier
+    {
+        if (threadIdx.x == 0)
+            for (int s = 0; s < STAGES; ++s) mbar_inval(&full[s]);
+    }
+};
 
 }  // namespace qp_stream

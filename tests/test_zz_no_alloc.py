@@ -38,7 +38,7 @@ def test_static_stats_matches_context_stats_twice():
     ctx = qp.Context(0)
     x1 = torch.from_numpy(si.vit_activation((16, 197, 768), 41).reshape(-1)).cuda()
     x2_h = si.vit_activation((3, 197, 1024), 42, outlier_frac=0.01).reshape(-1)
-    x2_h[[7, 1000]] = [np.nan, np.inf]                      # exercises the non-finite path and the status word
+    x2_h[[7, 1000]] = [np.nan, np.inf]                      # the non-finite path: reported through `nonfinite` only
     x2 = torch.from_numpy(x2_h).cuda()[1:]                  # and a 4-byte-aligned, ragged view
     out = torch.empty(STATS_BYTES, dtype=torch.uint8, device="cuda")  # the caller's buffer; nothing else is needed
     for x in (x1, x2):                                       # two calls in a row on the shared scratch
@@ -47,6 +47,7 @@ def test_static_stats_matches_context_stats_twice():
         assert qp.qp_stats_static(x, out) == qp.QP_OK
         got = ctx.read_stats(out)
         _close(got, want)
+    assert got.nonfinite == 2                                # (this entry point has no status word to read)
     # bf16 input and the empty tensor
     xb = x1[:100003].to(torch.bfloat16)
     want = ctx.read_stats(ctx.qp_stats(xb))
