@@ -34,12 +34,43 @@ import synth_inputs as si  # noqa: E402
 WORKLOAD = "c4"
 METRIC = "quantize+pack and unpack+dequant throughput, fp32 in, whole path per step"
 UNIT = "GB/s"
-# dram__bytes_read.sum + dram__bytes_write.sum per launch of each stage's main kernel on this
-# workload, from the ncu captures summarised in profiles/kernels_c4_ncu_full.md (None once a
-# kernel has changed since its capture)
-NCU_TRAFFIC_BYTES = {"clip": 133.2e6, "stats": 2 * 133.4e6, "quantize_pack": 141.5e6, "unpack_dequantize": 99.3e6}
-SAMPLE_IMAGES = 8              # CPU baseline leg: the first 8 images of the batch (2.0 M elements)
+SAMPLE_IMAGES = 8              # CPU legs: the first 8 images of the batch (2.0 M elements) per step
 ORACLE_US_PER_ELEM = 0.31      # rough cost of one oracle step per element (search on ~half the steps)
+MIN_TIMED_S = 0.5              # the K-step region is repeated until this much device time has been measured
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum per launch) of each stage's main kernel on
+# this workload, from one ncu capture each.  Every entry names the capture's summary and carries a
+# digest of the kernel's source files at capture time: when those files have changed since, the entry
+# is stale and the benchmark reports traffic = null.
+NCU_TRAFFIC = {
+    "stats": {"bytes": None, "kernel": "stats_fused_kernel<float, 0>", "summary": "profiles/stats_fused_kernel_c4.md",
+              "files": ("qp_stats.cu", "qp_stream.cuh", "qp_gridbar.cuh"), "digest": ""},
+    "clip": {"bytes": 133.2e6, "kernel": "iv_moments2_kernel<float>", "summary": "profiles/kernels_c4_ncu_full.md",
+             "files": ("qp_search_fast.cu",), "digest": ""},
+    "quantize_pack": {"bytes": 141.5e6, "kernel": "pack_kernel<8, float>", "summary": "profiles/kernels_c4_ncu_full.md",
+                      "files": ("qp_pack.cu",), "digest": ""},
+    "unpack_dequantize": {"bytes": 99.3e6, "kernel": "unpack_kernel<8, float>", "summary": "profiles/kernels_c4_ncu_full.md",
+                          "files": ("qp_unpack.cu",), "digest": ""},
+}
+
+
+def source_digest(files) -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(ROOT, "paper_2211_04515_b200", "csrc", f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def traffic_of(stage: str):
+    """(bytes or None, source label) of the ncu DRAM traffic recorded for a stage's main kernel."""
+    e = NCU_TRAFFIC.get(stage)
+    if e is None or e["bytes"] is None:
+        return None, "no capture of the current kernel"
+    if source_digest(e["files"]) != e["digest"]:
+        return None, f"stale: {', '.join(e['files'])} changed since the capture in {e['summary']}"
+    return e["bytes"], f"ncu capture of {e['kernel']} summarised in {e['summary']} (source digest {e['digest']})"
 
 
 def peaks():
@@ -63,7 +94,7 @@ def step_bits(n_elems: int, select):
 class ClockSampler(threading.Thread):
     """Samples SM clock and throttle reasons through NVML (read-only) while running."""
 
-    def __init__(self, index: int, period_s: float = 0.02):
+    def __init__(self, index: int, period_s: float = 0.004):
         super().__init__(daemon=True)
         self.index, self.period = index, period_s
         self.samples, self.reasons, self.max_mhz = [], set(), None
@@ -106,7 +137,7 @@ class ClockSampler(threading.Thread):
             self.join(timeout=1.0)
         med = statistics.median(self.samples) if self.samples else None
         return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
-                "samples": len(self.samples)}
+                "samples": len(self.samples), "period_ms": self.period * 1e3}
 
 
 def replica_throughput(local_ms: float, steps: int, bytes_per_step: float, world: int, device=None):
@@ -135,10 +166,11 @@ def oracle_step(oracle, x, bits, use_ds):
     oracle.unpack_dequantize(packed, x.size, qp)
 
 
-def sample_images_for(steps: int, budget_s: float = 90.0) -> int:
-    """Images per step such that `steps` oracle steps take about budget_s seconds."""
+def sample_images_for(steps: int, budget_s: float = 150.0) -> int:
+    """Images per step of the CPU legs: SAMPLE_IMAGES, fewer only where `steps` oracle steps on that
+    many images would take more than about budget_s seconds."""
     per_image = 197 * 1280 * ORACLE_US_PER_ELEM * 1e-6
-    return int(max(1, min(16, budget_s / (steps * per_image))))
+    return int(max(1, min(SAMPLE_IMAGES, budget_s / (max(steps, 1) * per_image))))
 
 
 def run_oracle_steps(first_step: int, count: int, bits_of_step, images: int = SAMPLE_IMAGES):
@@ -151,6 +183,37 @@ def run_oracle_steps(first_step: int, count: int, bits_of_step, images: int = SA
         oracle_step(oracle, x, q, 1 <= q <= 4)
     dt = time.perf_counter() - t0
     return dt, x.size
+
+
+def sample_text(images: int, n_sample: int) -> str:
+    return f"first {images} images of the batch ({n_sample} elements) per step, steps of the same trace"
+
+
+def oracle_all_cores(x, bits_list=(4, 8)):
+    """quantize+pack and unpack+dequantize of the oracle, as it stands, chunk-parallel over the host
+    cores (a chunk that starts at a multiple of 128 elements starts on a byte boundary of the packed
+    stream; ctypes releases the interpreter lock, so threads suffice).  GB/s of fp32 in (out)."""
+    from concurrent.futures import ThreadPoolExecutor
+
+    import oracle
+    cores = os.cpu_count() or 1
+    n = x.size
+    chunk = max(128, (n // (4 * cores)) // 128 * 128)
+    st = oracle.stats(x[:1 << 20])
+    out = {"cores": cores, "sample": f"the whole batch ({n} elements), chunks of {chunk} elements on {cores} threads"}
+    with ThreadPoolExecutor(cores) as ex:
+        for bits in bits_list:
+            _, _, qp_o = oracle.aciq_alpha(st, bits)
+            starts = list(range(0, n, chunk))
+            t0 = time.perf_counter()
+            packed = list(ex.map(lambda s0: oracle.quantize_pack(x[s0:s0 + chunk], qp_o), starts))
+            t1 = time.perf_counter()
+            list(ex.map(lambda a: oracle.unpack_dequantize(a[1], min(chunk, n - a[0]), qp_o), zip(starts, packed)))
+            t2 = time.perf_counter()
+            out[f"quantize_pack@{bits}b"] = round(4.0 * n / (t1 - t0) / 1e9, 3)
+            out[f"unpack_dequantize@{bits}b"] = round(4.0 * n / (t2 - t1) / 1e9, 3)
+    out["unit"] = UNIT
+    return out
 
 
 def reference_main(args):
@@ -166,14 +229,15 @@ def reference_main(args):
     run_oracle_steps(0, args.warmup, bits_of_step, images)
     dt, n_sample = run_oracle_steps(args.warmup, args.steps, bits_of_step, images)
     gbs = args.steps * 4.0 * n_sample / dt / 1e9
-    sample = f"first {images} images of the batch ({n_sample} elements) per step, steps of the same trace"
+    sample = sample_text(images, n_sample)
     line = {
         "impl": "reference", "metric": METRIC, "value": gbs, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
         "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
         "config": {"workload": f"{WORKLOAD}: fp32 {list(shape)} ViT-Huge activations, adaptive bits from a 100-step "
                                f"bandwidth trace; timed on a sample: {sample}"},
-        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": gbs, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(), "kind": "oracle",
+                         "sample": sample},
         "e2e": {"value": gbs, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -182,6 +246,64 @@ def reference_main(args):
 
 
 # ------------------------------------------------------------------------- CUDA arm
+
+def time_groups(torch, fn, nbuf, reps=20, warm=5, groups=5):
+    """Median per-launch time (ms) over `groups` groups of `reps` back-to-back launches of fn(i % nbuf)
+    (events around each group on the current stream, no host synchronisation inside a group)."""
+    for i in range(warm):
+        fn(i % nbuf)
+    torch.cuda.synchronize()
+    ts, k = [], warm
+    for _ in range(groups):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn(k % nbuf)
+            k += 1
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b) / reps)
+    ts.sort()
+    return ts[len(ts) // 2]
+
+
+def cold_kernels(torch, qp, ctx, x_host, hbm_peak, peak_kind):
+    """The metric's two kernels alone and cold: quantize+pack and unpack+dequantize on the workload at
+    2, 4 and 8 bits, and on a 1 GiB tensor at 4 bits.  Consecutive launches use different input and
+    output buffers, rotating through more than 4x the L2 capacity (126 MB) between reuses, so no
+    launch finds its lines in L2."""
+    out = {}
+
+    def row(name, q, n, ms):
+        alg = (4.0 + q / 8.0) * n
+        g = alg / (ms * 1e-3) / 1e9
+        out[f"{name}@{q}b"] = {"us": round(ms * 1e3, 2), "n": n, "gbs_fp32": round(4.0 * n / (ms * 1e-3) / 1e9, 1),
+                               "achieved": round(g, 1), "unit": "GB/s", "frac": round(g / hbm_peak, 4),
+                               "peak": hbm_peak, "peak_kind": peak_kind, "frac_of_8000": round(g / 8000.0, 4)}
+
+    def run(tag, xh, rot, widths):
+        n = xh.numel()
+        xs = [xh.cuda() for _ in range(rot)]
+        ys = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(rot)]
+        st = ctx.read_stats(ctx.qp_stats(xs[0]))
+        for q in widths:
+            _, _, qp_h = qp.qp_aciq_alpha(st, q)
+            pk = [torch.empty(qp.qp_packed_bytes(n, q), dtype=torch.uint8, device="cuda") for _ in range(rot)]
+            ms = time_groups(torch, lambda i: ctx.qp_quantize_pack(xs[i], q, qp_h, out=pk[i]), rot)
+            row(f"{tag}quantize_pack", q, n, ms)
+            ms = time_groups(torch, lambda i: ctx.qp_unpack_dequantize(pk[i], n, q, qp_h, out=ys[i]), rot)
+            row(f"{tag}unpack_dequantize", q, n, ms)
+            del pk
+        del xs, ys
+        torch.cuda.empty_cache()
+
+    run("", x_host, 5, (2, 4, 8))                                   # 5 x 129 MB in, 5 x 129 MB out
+    big = torch.from_numpy(si.flat_iid(1 << 28, si.C5_SEED, "laplace"))
+    run("2^28:", big, 2, (4,))                                       # every launch moves > 1 GiB: nothing survives in L2
+    out["method"] = ("each kernel alone, buffers rotating through > 4x L2 between reuses; median per-launch time of 5 "
+                     "groups of 20 back-to-back launches after 5 warm-ups; achieved = (4 + q/8) n bytes / time")
+    return out
+
 
 def ours_main(args):
     import torch
@@ -220,88 +342,89 @@ def ours_main(args):
 
     assert all(qp.qp_stats_carries_histogram(x, qp.QP_DEFAULT_HIST_BINS) for x in xs)
     stage_names = ("stats", "clip", "quantize_pack", "unpack_dequantize")
-    STAGE_EVERY = 7 if args.steps >= 60 else 1          # coprime with the 100-step trace: every bit-width is sampled
 
-    def step(t, events=None):
+    def step(t):
+        # The step as a user runs it: the sender as the library's single call (statistics -> clip ->
+        # quantize+pack, replayed as one recorded graph), then the receiver.  No events inside.
         q, x = bits_of_step[t % len(bits_of_step)], xs[t % ROT]
-        if events is None:
-            run_one_call(q, x)
-        else:
-            run(q, x, events)
-
-    def run_one_call(q, x):
-        # the sender as the library's single call (statistics -> clip -> quantize+pack, replayed as one
-        # recorded graph), then the receiver: the same kernels as run() below, enqueued back to back
         ctx.qp_sender_device(x, q, qp.qp_policy_use_ds(q), out_packed=packed, out_qp=d_qp, out_stats=d_stats)
         ctx.qp_unpack_dequantize(packed, n, q, d_qp, out=y)
 
-    def run(q, x, events=None):
-        marks = []
-        if events is not None:
-            marks = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
-            marks[0].record()
+    def step_by_stage(t, events):
+        # The same kernels called stage by stage with a CUDA event between the stages (each event makes
+        # the stream drain, about 3.5 us): used only for the per-stage times, after the headline run.
+        q, x = bits_of_step[t % len(bits_of_step)], xs[t % ROT]
+        marks = [torch.cuda.Event(enable_timing=True) for _ in range(5)]
+        marks[0].record()
         use_ds = qp.qp_policy_use_ds(q)
         ctx.qp_stats(x, out=d_stats, hist_bins=qp.QP_DEFAULT_HIST_BINS if use_ds else 0)
-        if events is not None:
-            marks[1].record()
-        if use_ds:      # the statistics just written carry the histogram (checked once below): the search need not look
+        marks[1].record()
+        if use_ds:      # the statistics just written carry the histogram (checked above): the search need not look
             ctx.qp_dsaciq_search(x, d_stats, q, bmode=qp.QP_B_MAD | qp.QP_B_HIST_IN_STATS, out_result=d_res, out_qp=d_qp)
         else:
             ctx.qp_aciq_qparams_device(d_stats, q, out=d_qp)
-        if events is not None:
-            marks[2].record()
+        marks[2].record()
         ctx.qp_quantize_pack(x, q, d_qp, out=packed)
-        if events is not None:
-            marks[3].record()
+        marks[3].record()
         ctx.qp_unpack_dequantize(packed, n, q, d_qp, out=y)
-        if events is not None:
-            marks[4].record()
-            events.append((q, marks))
+        marks[4].record()
+        events.append((q, marks))
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # The step runs on a stream of its own with graph replay on: each multi-kernel call (statistics,
-    # search) is recorded once per (input buffer, bit-width) during warm-up and replayed afterwards.
+    # The step runs on a stream of its own with graph replay on: each multi-kernel call is recorded
+    # once per (input buffer, bit-width) during warm-up and replayed afterwards.
+    sampler = ClockSampler(local)
+    sampler.start()                                      # before warm-up: the clocks of the whole run under load
     main_stream = torch.cuda.Stream()
     ctx.qp_set_graph_replay(True)
     torch.cuda.set_stream(main_stream)
-    for q in sorted(set(bits_of_step)):                  # untimed: every kernel variant loaded, every graph recorded
-        for x in xs:
-            run(q, x)
-            run_one_call(q, x)
+    seen = set()
+    for t in range(len(bits_of_step) * ROT):             # untimed: every (bit-width, input buffer) pair once, so that
+        pair = (bits_of_step[t % len(bits_of_step)], t % ROT)   # every kernel is loaded and every graph recorded
+        if pair not in seen:
+            seen.add(pair)
+            step(t)
+            step_by_stage(t, [])
     for t in range(args.warmup):
         step(t)
     barrier()
     assert ctx.qp_get_status() & ~qp.QP_DEV_NONFINITE == 0
 
-    # ---- timed region: exactly K steps, device-timed
+    # ---- timed region: exactly K steps between two events, bracketed by barrier + synchronize; the region
+    # is repeated until MIN_TIMED_S of device time has been measured, and the median repeat is reported
+    repeats = []
+    launches = graph_hits = 0
+    total_ms = 0.0
+    while total_ms < MIN_TIMED_S * 1e3 and len(repeats) < 200:
+        launches0, hits0 = ctx.qp_launch_count(), ctx.qp_graph_replays()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for t in range(args.warmup, args.warmup + args.steps):
+            step(t)
+        e1.record()
+        barrier()
+        ms_r = e0.elapsed_time(e1)
+        _, ms_r = replica_throughput(ms_r, args.steps, 4.0 * n, world, "cuda")     # MAX over ranks
+        repeats.append(ms_r)
+        total_ms += ms_r
+        launches = ctx.qp_launch_count() - launches0
+        graph_hits = ctx.qp_graph_replays() - hits0
+    ms = statistics.median(repeats)
+    value = world * args.steps * 4.0 * n / (ms * 1e-3) / 1e9
+
+    # ---- per-stage device times: a separate instrumented pass over the trace (events between the stages)
     events = []
-    launches0 = ctx.qp_launch_count()
-    hits0 = ctx.qp_graph_replays()
-    sampler = ClockSampler(local)
-    sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    e0.record()
-    for t in range(args.warmup, args.warmup + args.steps):
-        # A timing event makes the stream drain before the next kernel starts (about 3.5 us each;
-        # five per step cost 17 us of a 160 us step), so only every STAGE_EVERY-th step carries
-        # the per-stage events and makes the four calls one by one: the stage times below are a
-        # sample taken inside the timed region.  The other steps make the sender's one call.
-        step(t, events if (t - args.warmup) % STAGE_EVERY == 0 else None)
-    e1.record()
+    inst_steps = max(args.steps, len(bits_of_step))
+    for t in range(args.warmup, args.warmup + inst_steps):
+        step_by_stage(t, events)
     barrier()
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
-    launches = ctx.qp_launch_count() - launches0
-    graph_hits = ctx.qp_graph_replays() - hits0
     torch.cuda.set_stream(torch.cuda.default_stream())
-    value, ms = replica_throughput(ms, args.steps, 4.0 * n, world, "cuda")
-
-    # ---- per-stage device times from the events recorded inside the timed region
     per = {}
     for q, m in events:
         for i, name in enumerate(stage_names):
@@ -321,13 +444,16 @@ def ours_main(args):
             gbs = bytes_alg / (avg * 1e-3) / 1e9
             kernels[key] = {"ms": round(avg, 4), "bound": "hbm", "achieved": round(gbs, 1), "peak": hbm_peak,
                             "unit": "GB/s", "frac": round(gbs / hbm_peak, 4), "calls": len(v)}
+            if name != "stats":
+                kernels[key]["note"] = ("in the chain, L2-warm: the pass before it left part of x (of the packed stream) "
+                                        "in L2; the cold figures are in kernels_cold")
         elif qp.qp_policy_use_ds(q):
             # the search reads x once (interval moments); it is limited by shared-memory atomics, and
             # is reported against the HBM time of that one pass
             gbs = 4.0 * n / (avg * 1e-3) / 1e9
             kernels[key] = {"ms": round(avg, 4), "bound": "hbm", "achieved": round(gbs, 1), "peak": hbm_peak,
                             "unit": "GB/s", "frac": round(gbs / hbm_peak, 4), "calls": len(v),
-                            "note": "one read of x is the algorithmic traffic; limited by shared-memory atomics"}
+                            "note": "one read of x is the algorithmic traffic; limited by instruction issue and shared-memory atomics"}
         else:
             kernels[key] = {"ms": round(avg, 4), "calls": len(v)}
     # the dominant kernel of the step (largest share of device time)
@@ -336,15 +462,18 @@ def ours_main(args):
     tot_ms = sum(kernels[k]["ms"] * kernels[k]["calls"] for k in dom_keys)
     ach = sum(kernels[k]["achieved"] * kernels[k]["ms"] * kernels[k]["calls"] for k in dom_keys) / tot_ms
     first = kernels[dom_keys[0]]
+    traffic, traffic_source = traffic_of(dom)
     roofline = {"kernel": dom, "bound": first["bound"], "achieved": round(ach, 3), "peak": first["peak"],
                 "unit": first["unit"], "frac": round(ach / first["peak"], 4), "peak_kind": peak_kind,
-                "traffic": NCU_TRAFFIC_BYTES.get(dom), "share_of_step_time": round(stage_ms[dom] / sum(stage_ms.values()), 3)}
-    if dom == "stats":
-        # the call is two streaming kernels that each read x once: `achieved` charges one read of x
-        # to the whole call; per launch each kernel moves the algorithmic bytes in half the time
-        roofline["launches_per_call"] = 2
-        roofline["achieved_per_launch"] = round(2 * ach, 3)
-        roofline["frac_per_launch"] = round(2 * ach / first["peak"], 4)
+                "traffic": traffic, "traffic_source": traffic_source,
+                "share_of_step_time": round(stage_ms[dom] / sum(stage_ms.values()), 3),
+                "measured": f"CUDA events around the stage's call on the launching stream, {inst_steps} instrumented steps "
+                            "after the headline run (algorithmic bytes per call / average call time)"}
+
+    # ---- the metric's kernels alone and cold (rank 0 of a 1-GPU run: it needs ~5 GB of buffers)
+    cold = None
+    if rank == 0 and world == 1 and not args.no_cold:
+        cold = cold_kernels(torch, qp, ctx, x_host, hbm_peak, peak_kind)
 
     # ---- end to end through the host-buffer entry points (pinned host memory, copies timed).
     # Sender and receiver are two parties with their own context, stream and buffers, as on two
@@ -405,16 +534,19 @@ def ours_main(args):
            "overlap": "receiver of step t-1 runs beside the sender of step t (two streams, two contexts)"}
     ctx_r.close()
 
-    # ---- CPU oracle beside it (rank 0, N=1 only): bounded sample, same trace
+    # ---- CPU oracle beside it (rank 0, N=1 only): bounded sample, same trace; 1 thread for the whole
+    # step, and the two element-wise stages also chunk-parallel on every host core
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         cpu_steps = 16
-        dt, n_sample = run_oracle_steps(args.warmup, cpu_steps, bits_of_step)
-        cpu = {"value": cpu_steps * 4.0 * n_sample / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"{cpu_steps} steps of the same trace on the first {SAMPLE_IMAGES} images of the batch "
-                         f"({n_sample} elements), {dt:.1f} s"}
+        images = sample_images_for(cpu_steps)
+        dt, n_sample = run_oracle_steps(args.warmup, cpu_steps, bits_of_step, images)
+        cpu = {"value": cpu_steps * 4.0 * n_sample / dt / 1e9, "unit": UNIT, "cores": 1, "host_cores": os.cpu_count(),
+               "kind": "oracle", "sample": f"{cpu_steps} steps: " + sample_text(images, n_sample) + f", {dt:.1f} s",
+               "all_cores": oracle_all_cores(x_host.numpy())}
 
     if rank == 0:
+        med_mhz = clocks.get("sm_mhz")
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -423,13 +555,19 @@ def ours_main(args):
                                    f"{list(si.C4_ALLOWED_BITS)} from a seeded 100-step bandwidth trace, search at <=4 bits",
                        "replicas": world, "l2": f"inputs larger than L2 (129 MB > 126 MB), {ROT} rotating input buffers",
                        "bits_mix": {str(b): bits_of_step.count(b) for b in sorted(set(bits_of_step))},
-                       "stage_events": f"per-stage CUDA events on 1 timed step in {STAGE_EVERY} ({len(events)} of {args.steps}): every "
-                                       "timing event drains the stream; those steps call qp_stats / clip / "
-                                       "qp_quantize_pack one by one, the others call qp_sender_device",
-                       "graph_replay": f"on: {graph_hits} of the timed multi-kernel calls replayed a graph recorded "
-                                       "in warm-up"},
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches),
-            "clocks": clocks,
+                       "timed_region": f"{args.steps} steps (qp_sender_device + qp_unpack_dequantize per step, no events "
+                                       f"inside) between two events, repeated {len(repeats)} times "
+                                       f"({total_ms:.0f} ms of device time); ms_per_step is the median repeat",
+                       "stage_events": f"per-stage times from {inst_steps} separately instrumented steps after the timed "
+                                       "region (qp_stats / clip / qp_quantize_pack / qp_unpack_dequantize one by one, an "
+                                       "event between them)",
+                       "graph_replay": f"on: {graph_hits} multi-kernel calls of one timed region replayed a graph "
+                                       "recorded in warm-up"},
+            "repeats_ms_per_step": {"min": round(min(repeats) / args.steps, 5), "median": round(ms / args.steps, 5),
+                                    "max": round(max(repeats) / args.steps, 5), "count": len(repeats)},
+            "ms_per_step_x_sm_mhz": round(ms / args.steps * med_mhz, 2) if med_mhz else None,
+            "roofline": roofline, "kernels": kernels, "kernels_cold": cold, "cpu_baseline": cpu, "e2e": e2e,
+            "gpu_launches": int(launches), "clocks": clocks,
         }
         print(json.dumps(line))
     if world > 1:
@@ -644,6 +782,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=("ours", "reference"), default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cold", action="store_true", help="skip the kernels_cold object (it needs ~5 GB of buffers)")
     ap.add_argument("--quality", action="store_true",
                     help="print the quantization MSE of every clip method on the ViT-shaped configs (one GPU)")
     ap.add_argument("--sweep", action="store_true",

@@ -159,8 +159,8 @@ int32_t qp_make_qparams(double lo, double hi, int bits, qp_qparams_t* h_out);
  * d_x.  Two passes over x (sums/min/max, then deviations about the mean), fp64 merges in a
  * fixed order: results are bit-reproducible run to run.  n = 0 gives all-zero statistics.
  * For 16-byte aligned tensors of at least 128 KB both passes run in one cooperative launch
- * (one block per SM; the second pass starts on the tiles that the first one left in shared
- * memory), see qp_set_stats_path.
+ * (the second pass starts on the tiles that the first one left in shared memory), see
+ * qp_set_stats_path.
  * hist_bins > 0 asks the second pass to carry the directed search's histogram along
  * (hist_bins equal bins over [min, max]; only its peak count is kept, in hist_peak): a later
  * qp_dsaciq_search with the same hist_bins then skips its own histogram pass.  The fusion is
@@ -176,11 +176,13 @@ int32_t qp_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int hist_b
  * size and hist_bins. */
 int qp_stats_carries_histogram(const void* d_x, int dtype, uint64_t n, int hist_bins);
 /* How qp_stats runs its two passes on 16-byte aligned tensors of at least 128 KB (an execution
- * option without a counterpart in the paper; the statistics agree to the last bits or so, the
- * histogram's peak count is identical):
+ * option without a counterpart in the paper; min, max, the counts and the histogram's peak are
+ * identical on both paths, the other fields agree to ~1e-8 relative):
  *   QP_STATS_TWO_KERNELS  one kernel per pass
- *   QP_STATS_FUSED        one cooperative launch for both (falls back to two kernels on a device
- *                         that cannot hold it)
+ *   QP_STATS_FUSED        one cooperative launch for both (one block per SM; every block keeps the
+ *                         last tiles of its first pass in shared memory and starts the second pass,
+ *                         which walks backwards, on them).  Falls back to two kernels on a device
+ *                         that cannot hold it.
  *   QP_STATS_AUTO         the cooperative launch (default)
  * A grid barrier or tile wait of the cooperative launch that runs out sets QP_DEV_STREAM_TIMEOUT
  * and the launch ends without output. */

@@ -91,7 +91,7 @@ extern "C" int32_t qp_create(int device, qp_ctx** out)
     const size_t o_ivtot = off;  off = align_up(off + sizeof(qp_iv_total) * (QP_IV_MAXB + 1), 256);
     const size_t o_tstats = off; off = align_up(off + sizeof(qp_stats_t), 256);
     const size_t o_tqp = off;    off = align_up(off + sizeof(qp_qparams_t), 256);
-    const size_t o_fused = off;  off = align_up(off + 256 + sizeof(unsigned long long) * 4096, 256);
+    const size_t o_fused = off;  off = align_up(off + QP_FUSED_BYTES, 256);
 
     if (cudaMalloc(&c->d_base, off) != cudaSuccess || cudaMemset(c->d_base, 0, off) != cudaSuccess) {
         cudaGetLastError();
@@ -151,7 +151,7 @@ extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
     }
     if (word & QP_DEV_STREAM_TIMEOUT) {
         // a cooperative launch that gave up may have left its arrival counters and histogram mid-way
-        e = cudaMemsetAsync(ctx->d_fused, 0, 256 + sizeof(unsigned long long) * 4096, s);
+        e = cudaMemsetAsync(ctx->d_fused, 0, QP_FUSED_BYTES, s);
         if (e == cudaSuccess) e = cudaStreamSynchronize(s);
         if (e != cudaSuccess) {
             snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_get_status: %s", cudaGetErrorString(e));

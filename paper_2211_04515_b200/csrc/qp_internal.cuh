@@ -83,7 +83,7 @@ struct qp_ctx {
     unsigned spin_limit;                 // limit of a grid-barrier wait (polls)
     int bar_extra;                       // test only: arrivals a grid barrier waits for beyond the grid size
     size_t fused_dyn_max;                // largest slice (bytes of dynamic shared memory) per block
-    void* d_fused;                       // cooperative sender: arrival counter (256 B) + histogram [4096]
+    void* d_fused;                       // scratch of the cooperative kernels (QP_FUSED_BYTES, see below)
     void* d_ch_part;                     // channel-wise statistics: block partials, allocated on first use
     size_t ch_part_bytes;
     void* d_ch_search;                   // channel-wise search: histograms, candidates, partials, curves; on first use
@@ -109,6 +109,10 @@ struct qp_ctx {
     int last_x_end;                      // stopped (1 = at the end of the tensor): the next pass starts there (L2)
     char err[256];
 };
+
+// Scratch of the cooperative kernels (d_fused): 256 bytes of barrier counters and the whole-sender
+// kernel's histogram (4096 x 8 bytes).
+constexpr size_t QP_FUSED_BYTES = 256 + sizeof(unsigned long long) * 4096;
 
 constexpr long long QP_WAIT_CYCLES_DEFAULT = 4000000000ll;   // about two seconds
 constexpr unsigned QP_SPIN_LIMIT_DEFAULT = 1u << 22;          // x 64 ns sleeps: a quarter of a second at least

@@ -682,7 +682,8 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
         const float fmn = (float)dmn;
         const float inv_w = hist_on ? (float)((double)a.nb / (dmx - dmn)) : 0.f;
         unsigned* my_hist = sh_hist + (threadIdx.x & ((1 << a.rep_shift) - 1));   // this lane's replica of the bins
-        const int top_bin = a.nb - 1, rep_shift = a.rep_shift;
+        const float top_bin = (float)(a.nb - 1);
+        const int rep_shift = a.rep_shift;
         if (HIST) {
             for (int i = threadIdx.x; i < (a.nb << rep_shift); i += SF_THREADS) sh_hist[i] = 0u;
             __syncthreads();
@@ -694,8 +695,13 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
                 if (!GD || qp_is_finite(e)) {
                     d1 += fabsf(d);
                     d2 = fmaf(d, d, d2);
-                    if (HIST) {      // x >= min, so the position is never negative; an empty range gives bin 0
-                        const int b = min(__float2int_rz(__fmul_rn(__fsub_rn(e, fmn), inv_w)), top_bin);
+                    if (HIST) {
+                        // bin = floor((x - min) * inv_w), the last bin closed; x >= min, so the position is
+                        // never negative (an empty range gives bin 0).  The floor is taken by adding 2^23
+                        // rounding down, which leaves it in the low mantissa bits: no conversion instruction
+                        // (conversions issue at a quarter of the rate of an addition).
+                        const float pos = fminf(__fmul_rn(__fsub_rn(e, fmn), inv_w), top_bin);
+                        const unsigned b = __float_as_uint(__fadd_rd(pos, 8388608.0f)) & 0x7FFFFFu;
                         atomicAdd(&my_hist[b << rep_shift], 1u);
                     }
                 }

@@ -20,6 +20,9 @@ Sec. 4), which need trained weights and a dataset to produce.
 """
 from __future__ import annotations
 
+import os
+from concurrent.futures import ThreadPoolExecutor
+
 import numpy as np
 
 _MASK = np.uint64(0xFFFFFFFFFFFFFFFF)
@@ -36,7 +39,21 @@ STREAM_OUTLIER = 7    # per-channel draw ranking the outlier channels
 STREAM_BANDWIDTH = 8  # per-step bandwidth trace
 STREAM_CODES = 9      # random integer codes for pack/unpack round trips
 
-_CHUNK = 1 << 22
+_CHUNK = 1 << 20
+_WORKERS = max(1, min(16, os.cpu_count() or 1))
+
+
+def _for_chunks(n: int, fill) -> None:
+    """fill(start, count) for every chunk of [0, n); chunks are independent (every value is a pure
+    function of its index), so they are filled by a few threads at once (numpy releases the
+    interpreter lock inside its loops)."""
+    starts = range(0, n, _CHUNK)
+    if _WORKERS == 1 or n <= _CHUNK:
+        for start in starts:
+            fill(start, min(_CHUNK, n - start))
+        return
+    with ThreadPoolExecutor(_WORKERS) as ex:
+        list(ex.map(lambda start: fill(start, min(_CHUNK, n - start)), starts))
 
 
 def _mix(z: np.ndarray) -> np.ndarray:
@@ -103,10 +120,12 @@ def vit_activation(shape, seed: int, outlier_frac: float = 0.0, out: np.ndarray 
     mu, s = channel_params(seed, channels, outlier_frac)
     flat = out.reshape(-1) if out is not None else np.empty(n, dtype=np.float32)
     assert flat.size == n and flat.dtype == np.float32
-    for start in range(0, n, _CHUNK):
-        cnt = min(_CHUNK, n - start)
+
+    def fill(start, cnt):
         c = (np.arange(start, start + cnt, dtype=np.int64) % channels)
         flat[start:start + cnt] = (mu[c] + s[c] * laplace01(seed, STREAM_VALUE, start, cnt)).astype(np.float32)
+
+    _for_chunks(n, fill)
     return flat.reshape(shape)
 
 
@@ -114,15 +133,17 @@ def flat_iid(n: int, seed: int, dist: str = "laplace", out: np.ndarray | None = 
     """Flat fp32 tensor of n i.i.d. Laplace(0,1) or N(0,1) values."""
     flat = out if out is not None else np.empty(n, dtype=np.float32)
     assert flat.size == n and flat.dtype == np.float32
-    for start in range(0, n, _CHUNK):
-        cnt = min(_CHUNK, n - start)
+    if dist not in ("laplace", "normal"):
+        raise ValueError(f"unknown dist {dist!r}")
+
+    def fill(start, cnt):
         if dist == "laplace":
             v = laplace01(seed, STREAM_VALUE, start, cnt)
-        elif dist == "normal":
-            v = normal01(seed, STREAM_VALUE, STREAM_VALUE2, start, cnt)
         else:
-            raise ValueError(f"unknown dist {dist!r}")
+            v = normal01(seed, STREAM_VALUE, STREAM_VALUE2, start, cnt)
         flat[start:start + cnt] = v.astype(np.float32)
+
+    _for_chunks(n, fill)
     return flat
 
 

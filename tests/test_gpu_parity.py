@@ -171,16 +171,45 @@ def test_stats_one_launch_against_oracle_and_two_kernels(ctx, tiles, tail):
             plain = ctx.read_stats(ctx.qp_stats(d))
         finally:
             ctx.qp_set_stats_path(qp.QP_STATS_AUTO)
-        assert launches == (1 if path == qp.QP_STATS_FUSED else 2)
+        assert launches == (2 if path == qp.QP_STATS_TWO_KERNELS else 1)
         check_stats(st, st_o)
         assert st.hist_bins == 100 and st.hist_peak == int(counts.max())
         assert bytes(st) == bytes(again)                              # fixed merge order: bit-reproducible
         assert plain.hist_bins == 0 and (plain.mean, plain.mad, plain.var) == (st.mean, st.mad, st.var)
         got[path] = st
-    a, b = got[STATS_PATHS[0]], got[STATS_PATHS[1]]
+    a, b = got[qp.QP_STATS_FUSED], got[qp.QP_STATS_TWO_KERNELS]
     assert (a.n, a.nonfinite, a.min, a.max, a.hist_peak) == (b.n, b.nonfinite, b.min, b.max, b.hist_peak)
     for f in ("mean_abs", "mad", "var"):         # fp32 sums over 16 elements, grouped differently by the two tile sizes
         assert abs(getattr(a, f) - getattr(b, f)) <= 1e-7 * abs(getattr(b, f))
+    assert ctx.qp_get_status() == 0
+
+
+def test_stats_hard_tensors(sctx):
+    """Tensors that are hard on a streaming reduction: sorted (every block sees another level), a third
+    of the elements exactly at the mean, constant, two levels, a shifted mixture, a mean far from zero,
+    a tiny scale."""
+    ctx = sctx
+    n = 1500 * 8192 + 77
+    base = si.flat_iid(n, 77, "laplace")
+    cases = {
+        "sorted": np.sort(base),
+        "mass_at_mean": np.where(np.arange(n) % 3 == 0, np.float32(0.0),            # 0, +a, -a, 0, +b, -b, ...: mean exactly 0
+                                 np.where(np.arange(n) % 3 == 1, 1.0, -1.0) * np.abs(np.repeat(base[:n // 3 + 1], 3)[:n])
+                                 ).astype(np.float32),
+        "constant": np.full(n, 3.25, dtype=np.float32),
+        "two_levels": np.where(np.arange(n) % 2 == 0, np.float32(-1.0), np.float32(2.0)).astype(np.float32),
+        "mixture": (base + np.where(np.arange(n) % 5 == 0, 40.0, 0.0)).astype(np.float32),
+        "large_offset": (np.float32(4096.0) + base).astype(np.float32),
+        "tiny_scale": (base * np.float32(1e-20)).astype(np.float32),
+    }
+    for name, x in cases.items():
+        st = ctx.read_stats(ctx.qp_stats(dev(x)))
+        st_o = oracle.stats(x)
+        assert (st.min, st.max, st.n) == (st_o.min, st_o.max, st_o.n), name
+        if st_o.mad > 0:
+            check_stats(st, st_o)
+        else:
+            assert st.mad == 0.0 and st.var == 0.0 and st.mean == st_o.mean, name
     assert ctx.qp_get_status() == 0
 
 
