@@ -284,7 +284,8 @@ int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
  * (every element looks its interval up), and one that adds elements of grid cells without a
  * threshold straight into per-cell, per-lane sums and looks up only the others; the second is
  * used up to ~150 M elements, QP_SEARCH_INTERVALS_PLAIN forces the first. */
-enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2, QP_SEARCH_INTERVALS_PLAIN = 3 };
+enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2, QP_SEARCH_INTERVALS_PLAIN = 3,
+       QP_SEARCH_INTERVALS_CHAIN = 4 };
 int32_t qp_set_search_path(qp_ctx* ctx, int path);
 /* Graph replay of the multi-kernel calls (an execution option; the paper has no counterpart,
  * results are unchanged).  With on = 1, qp_stats, qp_dsaciq_search and qp_sender_device

@@ -105,6 +105,12 @@ def lib():
         L.orc_quantize_channels.restype = None
         L.orc_dequantize_channels.argtypes = [u32p, C.c_uint64, C.c_uint64, C.POINTER(QParams), fp]
         L.orc_dequantize_channels.restype = None
+        L.orc_stats_tokens.argtypes = [fp, C.c_uint64, C.c_uint64, C.POINTER(Stats)]
+        L.orc_stats_tokens.restype = C.c_int
+        L.orc_quantize_tokens.argtypes = [fp, C.c_uint64, C.c_uint64, C.POINTER(QParams), u32p]
+        L.orc_quantize_tokens.restype = None
+        L.orc_dequantize_tokens.argtypes = [u32p, C.c_uint64, C.c_uint64, C.POINTER(QParams), fp]
+        L.orc_dequantize_tokens.restype = None
         L.orc_midrise_range.argtypes = [C.c_double, C.c_double, C.c_int, dp, dp]
         L.orc_midrise_range.restype = None
         L.orc_hist_peak.argtypes = [fp, C.c_uint64, C.c_double, C.c_double, C.c_int, u64p]
@@ -255,6 +261,37 @@ def dequantize_channels(codes, channels: int, qp) -> np.ndarray:
     c = np.ascontiguousarray(codes, dtype=np.uint32)
     y = np.empty(c.size, dtype=np.float32)
     lib().orc_dequantize_channels(_ptr(c, C.c_uint32), c.size // channels, channels, qp, _ptr(y, C.c_float))
+    return y
+
+
+def stats_tokens(x, channels: int):
+    """Per-token statistics of a [tokens, channels] tensor: a ctypes array of `tokens` Stats."""
+    a = _f32(x)
+    tokens = a.size // channels
+    assert tokens * channels == a.size
+    out = (Stats * max(tokens, 1))()
+    rc = lib().orc_stats_tokens(_ptr(a, C.c_float), tokens, channels, out)
+    assert rc == 0
+    return out
+
+
+def clip_tokens(st, bits: int, method: int = CLIP_ACIQ, intersect: bool = False, dist: int = 0, bmode: int = 0,
+                midrise: bool = False):
+    """(rc, ctypes array of per-token QParams) from per-token statistics (the same map as clip_channels)."""
+    return clip_channels(st, bits, method, intersect, dist, bmode, midrise)
+
+
+def quantize_tokens(x, channels: int, qp) -> np.ndarray:
+    a = _f32(x)
+    codes = np.empty(a.size, dtype=np.uint32)
+    lib().orc_quantize_tokens(_ptr(a, C.c_float), a.size // channels, channels, qp, _ptr(codes, C.c_uint32))
+    return codes
+
+
+def dequantize_tokens(codes, channels: int, qp) -> np.ndarray:
+    c = np.ascontiguousarray(codes, dtype=np.uint32)
+    y = np.empty(c.size, dtype=np.float32)
+    lib().orc_dequantize_tokens(_ptr(c, C.c_uint32), c.size // channels, channels, qp, _ptr(y, C.c_float))
     return y
 
 

@@ -289,6 +289,31 @@ void orc_dequantize_channels(const uint32_t* codes, uint64_t rows, uint64_t chan
     for (uint64_t i = 0; i < rows * channels; ++i) y[i] = dequantize_one(codes[i], &qp[i % channels]);
 }
 
+/* Token-wise variant: the other axis of the same idea.  The tensor is [tokens, channels], row-major,
+ * and every token (a row of `channels` contiguous elements, one position of a ViT sequence) gets the
+ * statistics, the clip range and the quantizer that the per-tensor functions give for its row alone
+ * (Sec. 3's method with the row in place of the tensor; the paper clips per tensor).  Bit-width and
+ * packed layout are shared.  The clip ranges come from orc_clip_channels, which only maps an array
+ * of statistics to an array of quantizers and does not care what the entries stand for. */
+
+/* Statistics of each row: out[t] = orc_stats of x[t * channels .. (t + 1) * channels). */
+int orc_stats_tokens(const float* x, uint64_t tokens, uint64_t channels, orc_stats_t* out)
+{
+    if (channels < 1) return ORC_ERR_ARG;
+    for (uint64_t t = 0; t < tokens; ++t) orc_stats(x + t * channels, channels, &out[t]);
+    return ORC_OK;
+}
+
+void orc_quantize_tokens(const float* x, uint64_t tokens, uint64_t channels, const orc_qparams_t* qp, uint32_t* codes)
+{
+    for (uint64_t i = 0; i < tokens * channels; ++i) codes[i] = quantize_one(x[i], &qp[i / channels]);
+}
+
+void orc_dequantize_tokens(const uint32_t* codes, uint64_t tokens, uint64_t channels, const orc_qparams_t* qp, float* y)
+{
+    for (uint64_t i = 0; i < tokens * channels; ++i) y[i] = dequantize_one(codes[i], &qp[i / channels]);
+}
+
 /* ----------------------------------------------------------------- packing */
 
 /* Packed length: ceil(n * bits / 8) bytes rounded up to a multiple of 16. */

@@ -25,7 +25,7 @@ QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
 QP_B_MAD, QP_B_MEAN_ABS = 0, 1
 QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT, QP_DEV_HIST_MISSING = 1, 2, 4, 8, 16
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
-QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS, QP_SEARCH_INTERVALS_PLAIN = 0, 1, 2, 3
+QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS, QP_SEARCH_INTERVALS_PLAIN, QP_SEARCH_INTERVALS_CHAIN = 0, 1, 2, 3, 4
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
 QP_STATS_AUTO, QP_STATS_TWO_KERNELS, QP_STATS_FUSED = 0, 1, 2
 QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT, QP_CLIP_MIDRISE = 0, 1, 2, 0x10, 0x20

@@ -79,6 +79,7 @@ struct qp_ctx {
     int stats_path;                      // 0 auto, 1 two kernels, 2 one cooperative launch where it applies
     int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
     int stats_fused_checked, stats_fused_ok;   // the same for the one-launch statistics
+    int ivc_checked, ivc_ok;             // and for the one-launch search (bit 0: fp32, bit 1: bf16)
     long long wait_cycles;               // limit of a wait for a tile copy (clock cycles)
     unsigned spin_limit;                 // limit of a grid-barrier wait (polls)
     int bar_extra;                       // test only: arrivals a grid barrier waits for beyond the grid size

@@ -811,3 +811,80 @@ def test_generator_is_counter_based_and_shaped():
     assert np.max(np.abs(si.bf16_bits_to_f32(h) - a) / np.maximum(np.abs(a), 1e-30)) <= 2.0 ** -8
     bw = si.bandwidth_trace(3, 100)
     assert bw.min() >= 5e6 and bw.max() <= 200e6 and len(np.unique(bw)) == 100
+
+
+# ------------------------------------------------------- per-token quantization
+
+def test_tokens_hand_example_two_scales():
+    """Two tokens whose scales differ by ten: token 0 holds 0, 1, 2, 3 and token 1 holds 0, 10, 20, 30.
+    With the min/max range at 2 bits every token has its own four levels, so every value is a level and
+    is reconstructed exactly; one range for the whole tensor, [0, 30], sends token 0's 1, 2, 3 to 0."""
+    x = np.array([[0, 1, 2, 3], [0, 10, 20, 30]], dtype=np.float32)
+    st = oracle.stats_tokens(x, 4)
+    assert [(s.min, s.max, s.n) for s in st] == [(0.0, 3.0, 4), (0.0, 30.0, 4)]
+    rc, qp = oracle.clip_tokens(st, 2, oracle.CLIP_MINMAX)
+    assert rc == 0 and (qp[0].scale, qp[1].scale) == (1.0, 10.0)
+    codes = oracle.quantize_tokens(x, 4, qp)
+    assert codes.reshape(2, 4).tolist() == [[0, 1, 2, 3], [0, 1, 2, 3]]
+    assert np.array_equal(oracle.dequantize_tokens(codes, 4, qp).reshape(2, 4), x)
+    whole = oracle.clip_range(oracle.stats(x), 2, oracle.CLIP_MINMAX)[3]
+    assert oracle.dequantize(oracle.quantize(x, whole), whole).reshape(2, 4)[0].tolist() == [0.0, 0.0, 0.0, 0.0]
+
+
+def test_tokens_against_numpy_rows_and_against_the_channel_functions_on_the_transpose():
+    x = si.vit_activation((1, 37, 24), 16, outlier_frac=0.1).reshape(37, 24)
+    x[5, 3] = np.nan
+    x[5, 7] = -np.inf
+    st = oracle.stats_tokens(x, 24)
+    x64 = x.astype(np.float64)
+    for t in range(37):
+        row = x64[t][np.isfinite(x64[t])]
+        assert st[t].n == 24 and st[t].nonfinite == (2 if t == 5 else 0)
+        assert st[t].mean == pytest.approx(row.mean(), rel=1e-12, abs=1e-15)
+        assert st[t].mad == pytest.approx(np.abs(row - row.mean()).mean(), rel=1e-12)
+        assert st[t].var == pytest.approx(row.var(), rel=1e-12)
+        assert (st[t].min, st[t].max) == (row.min(), row.max())
+    # the tokens of X are the channels of its transpose: statistics, quantizers, codes and reconstructions
+    # must be those of the (separately pinned) channel-wise functions on the transposed tensor
+    xt = np.ascontiguousarray(x.T)                           # [24, 37]: 37 channels
+    st_c = oracle.stats_channels(xt, 37)
+    assert all(bytes(st[t]) == bytes(st_c[t]) for t in range(37))
+    for bits, method, cut, mid in ((4, oracle.CLIP_ACIQ, False, False), (2, oracle.CLIP_MINMAX, False, True),
+                                   (8, oracle.CLIP_ACIQ, True, False)):
+        rc, qp = oracle.clip_tokens(st, bits, method, cut, midrise=mid)
+        rc_c, qp_c = oracle.clip_channels(st_c, bits, method, cut, midrise=mid)
+        assert rc == rc_c and all(bytes(qp[t]) == bytes(qp_c[t]) for t in range(37))
+        codes = oracle.quantize_tokens(x, 24, qp).reshape(37, 24)
+        codes_c = oracle.quantize_channels(xt, 37, qp_c).reshape(24, 37)
+        assert np.array_equal(codes, codes_c.T)
+        y = oracle.dequantize_tokens(codes.reshape(-1), 24, qp).reshape(37, 24)
+        y_c = oracle.dequantize_channels(codes_c.reshape(-1), 37, qp_c).reshape(24, 37)
+        assert np.array_equal(y, y_c.T)
+
+
+def test_tokens_one_token_is_the_per_tensor_path_and_tokens_do_not_interact():
+    y = si.flat_iid(5000, 17, "laplace")
+    st1 = oracle.stats_tokens(y, y.size)                     # a single token: exactly the per-tensor functions
+    assert bytes(st1[0]) == bytes(oracle.stats(y))
+    for bits in (2, 4, 8, 16):
+        rc, qp1 = oracle.clip_tokens(st1, bits)
+        q = oracle.aciq_alpha(oracle.stats(y), bits)[2]
+        assert bytes(qp1[0]) == bytes(q)
+        assert np.array_equal(oracle.quantize_tokens(y, y.size, qp1), oracle.quantize(y, q))
+        assert np.array_equal(oracle.pack(oracle.quantize_tokens(y, y.size, qp1), bits), oracle.quantize_pack(y, q))
+    x = si.vit_activation((1, 30, 16), 18, outlier_frac=0.2).reshape(30, 16)
+    st = oracle.stats_tokens(x, 16)
+    rc, qp = oracle.clip_tokens(st, 4)
+    codes = oracle.quantize_tokens(x, 16, qp).reshape(30, 16)
+    x2 = x.copy()
+    x2[11] *= np.float32(4.0)                                # a power of two: token 11's range scales, nothing else moves
+    st2 = oracle.stats_tokens(x2, 16)
+    rc, qp2 = oracle.clip_tokens(st2, 4)
+    assert (qp2[11].lo, qp2[11].hi, qp2[11].scale) == (4 * qp[11].lo, 4 * qp[11].hi, 4 * qp[11].scale)
+    assert all(bytes(qp2[t]) == bytes(qp[t]) for t in range(30) if t != 11)
+    assert np.array_equal(oracle.quantize_tokens(x2, 16, qp2).reshape(30, 16), codes)
+    x[7] = np.float32(-2.5)                                  # a constant token is degenerate: code 0, exact
+    rc, qz = oracle.clip_tokens(oracle.stats_tokens(x, 16), 4)
+    assert rc == oracle.WARN_DEGENERATE and qz[7].flags == 1
+    back = oracle.dequantize_tokens(oracle.quantize_tokens(x, 16, qz), 16, qz).reshape(30, 16)
+    assert np.all(back[7] == np.float32(-2.5))
