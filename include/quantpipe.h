@@ -284,8 +284,7 @@ int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
  * (every element looks its interval up), and one that adds elements of grid cells without a
  * threshold straight into per-cell, per-lane sums and looks up only the others; the second is
  * used up to ~150 M elements, QP_SEARCH_INTERVALS_PLAIN forces the first. */
-enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2, QP_SEARCH_INTERVALS_PLAIN = 3,
-       QP_SEARCH_INTERVALS_CHAIN = 4 };
+enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2, QP_SEARCH_INTERVALS_PLAIN = 3 };
 int32_t qp_set_search_path(qp_ctx* ctx, int path);
 /* Graph replay of the multi-kernel calls (an execution option; the paper has no counterpart,
  * results are unchanged).  With on = 1, qp_stats, qp_dsaciq_search and qp_sender_device
@@ -444,6 +443,37 @@ int32_t qp_dsaciq_curve_channels(qp_ctx* ctx, uint32_t channel, double* h_curve,
 /* The candidates' quantizers of the last channel-wise search, as qp_dsaciq_candidates:
  * h_out[c * (steps + 1) + k] for channel c and step k; capacity in entries.  Diagnostic. */
 int32_t qp_dsaciq_candidates_channels(qp_ctx* ctx, qp_qparams_t* h_out, uint64_t capacity, void* stream);
+
+/* ---- token-wise variant (the other axis of the channel-wise variant above; the paper clips per
+ * tensor) -------------------------------------------------------------------------------------
+ * The tensor is [tokens, channels], row-major: token t is the row of `channels` contiguous elements
+ * t * channels .. (t + 1) * channels - 1 (one position of a ViT sequence).  Every token gets the
+ * statistics, clip range and quantizer that the per-tensor calls give for its row alone; bit-width
+ * and packed layout (qp_packed_bytes(tokens * channels, bits)) are shared, so the receiver needs the
+ * `tokens` quantizers (24 bytes each) with the stream.
+ *   qp_stats_tokens                fills d_out[0..tokens) (hist fields 0); a warp per token, the
+ *                                  tensor is read from HBM once
+ *   qp_clip_qparams_tokens_device  d_qp_out[t] from d_stats[t]; method, dist, bmode as
+ *                                  qp_clip_qparams_device (closed-form clips only: no search per token)
+ *   qp_quantize_pack_tokens        code of element i with d_qp[i / channels]
+ *   qp_unpack_dequantize_tokens    the inverse, fp32 or bf16 out
+ *   qp_sender_tokens_device        the three sender calls in one; d_stats_work is the caller's device
+ *                                  memory for `tokens` statistics
+ * The fast kernels need a 16-byte aligned tensor, `channels` a multiple of 4 (fp32) or 8 (bf16) and
+ * bits <= 8; other shapes, and 16 bits, take a scalar kernel (one thread per 32 elements).
+ * d_stats, d_qp: device arrays of `tokens` entries; channels >= 1.
+ * Errors: as the per-tensor calls. */
+int32_t qp_stats_tokens(qp_ctx* ctx, const void* d_x, int dtype, uint64_t tokens, uint32_t channels, qp_stats_t* d_out,
+                        void* stream);
+int32_t qp_clip_qparams_tokens_device(qp_ctx* ctx, const qp_stats_t* d_stats, uint64_t tokens, int bits, int method,
+                                      int dist, int bmode, qp_qparams_t* d_qp_out, void* stream);
+int32_t qp_quantize_pack_tokens(qp_ctx* ctx, const void* d_x, int dtype, uint64_t tokens, uint32_t channels, int bits,
+                                const qp_qparams_t* d_qp, void* d_packed, uint64_t packed_capacity, void* stream);
+int32_t qp_unpack_dequantize_tokens(qp_ctx* ctx, const void* d_packed, uint64_t tokens, uint32_t channels, int bits,
+                                    const qp_qparams_t* d_qp, void* d_y, int out_dtype, void* stream);
+int32_t qp_sender_tokens_device(qp_ctx* ctx, const void* d_x, int dtype, uint64_t tokens, uint32_t channels, int bits,
+                                int method, int bmode, void* d_packed, uint64_t packed_capacity, qp_qparams_t* d_qp_out,
+                                qp_stats_t* d_stats_work, void* stream);
 
 /* ---- whole sender / receiver on HOST buffers (Sec. 3: the module sits between a stage's
  * output and the link, and between the link and the next stage's input) -------------------

@@ -25,7 +25,7 @@ QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
 QP_B_MAD, QP_B_MEAN_ABS = 0, 1
 QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT, QP_DEV_HIST_MISSING = 1, 2, 4, 8, 16
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
-QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS, QP_SEARCH_INTERVALS_PLAIN, QP_SEARCH_INTERVALS_CHAIN = 0, 1, 2, 3, 4
+QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS, QP_SEARCH_INTERVALS_PLAIN = 0, 1, 2, 3
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
 QP_STATS_AUTO, QP_STATS_TWO_KERNELS, QP_STATS_FUSED = 0, 1, 2
 QP_CLIP_ACIQ, QP_CLIP_DSACIQ, QP_CLIP_MINMAX, QP_CLIP_INTERSECT, QP_CLIP_MIDRISE = 0, 1, 2, 0x10, 0x20
@@ -41,6 +41,8 @@ EXPORTS = (
     "qp_controller_payload_bytes", "qp_sender_device", "qp_set_graph_replay", "qp_graph_replays", "qp_set_sender_path",
     "qp_clip_range", "qp_clip_qparams_device", "qp_stats_channels", "qp_dsaciq_search_channels", "qp_dsaciq_curve_channels", "qp_clip_qparams_channels_device",
     "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range", "qp_sender_channels_device",
+    "qp_stats_tokens", "qp_clip_qparams_tokens_device", "qp_quantize_pack_tokens", "qp_unpack_dequantize_tokens",
+    "qp_sender_tokens_device",
     "qp_set_stats_path", "qp_dsaciq_candidates", "qp_dsaciq_candidates_channels", "qp_set_wait_limit_for_testing",
 )
 
@@ -119,6 +121,11 @@ def load() -> C.CDLL:
     L.qp_quantize_pack_channels.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, vp, vp, u64, vp]
     L.qp_unpack_dequantize_channels.argtypes = [vp, vp, u64, C.c_uint32, C.c_int, vp, vp, C.c_int, vp]
     L.qp_sender_channels_device.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, C.c_int, C.c_int, vp, u64, vp, vp, vp]
+    L.qp_stats_tokens.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, vp, vp]
+    L.qp_clip_qparams_tokens_device.argtypes = [vp, vp, u64, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp]
+    L.qp_quantize_pack_tokens.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, vp, vp, u64, vp]
+    L.qp_unpack_dequantize_tokens.argtypes = [vp, vp, u64, C.c_uint32, C.c_int, vp, vp, C.c_int, vp]
+    L.qp_sender_tokens_device.argtypes = [vp, vp, C.c_int, u64, C.c_uint32, C.c_int, C.c_int, C.c_int, vp, u64, vp, vp, vp]
     L.qp_dsaciq_search.argtypes = [vp, vp, C.c_int, u64, vp, C.c_int, C.c_int, C.c_int, C.c_int, vp, vp, vp]
     L.qp_dsaciq_curve.argtypes = [vp, C.POINTER(dbl), C.c_int, vp]
     L.qp_policy_use_ds.argtypes = [C.c_int]
@@ -500,6 +507,54 @@ class Context:
             self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels, channels, bits, method, bmode,
             out_packed.data_ptr(), out_packed.numel() * out_packed.element_size(), out_qp.data_ptr(),
             out_stats.data_ptr() if out_stats is not None else None, _stream(self.device)))
+        return out_packed, out_qp
+
+    # -- token-wise variant: x is [tokens, channels], a token = a row of `channels` contiguous elements
+    def qp_stats_tokens(self, x: torch.Tensor, channels: int, out: torch.Tensor | None = None) -> torch.Tensor:
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        tokens = x.numel() // channels
+        out = self._bytes(C.sizeof(Stats) * tokens) if out is None else out
+        self._check(self._lib.qp_stats_tokens(self._h, x.data_ptr(), _dtype_code(x), tokens, channels, out.data_ptr(),
+                                              _stream(self.device)))
+        return out
+
+    def qp_clip_qparams_tokens_device(self, d_stats: torch.Tensor, tokens: int, bits: int, method: int = QP_CLIP_ACIQ,
+                                      dist: int = QP_DIST_LAPLACE, bmode: int = QP_B_MAD,
+                                      out: torch.Tensor | None = None) -> torch.Tensor:
+        out = self._bytes(C.sizeof(QParams) * tokens) if out is None else out
+        self._check(self._lib.qp_clip_qparams_tokens_device(self._h, d_stats.data_ptr(), tokens, bits, method, dist, bmode,
+                                                            out.data_ptr(), _stream(self.device)))
+        return out
+
+    def qp_quantize_pack_tokens(self, x: torch.Tensor, channels: int, bits: int, d_qp: torch.Tensor,
+                                out: torch.Tensor | None = None) -> torch.Tensor:
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        out = self._bytes(qp_packed_bytes(x.numel(), bits)) if out is None else out
+        self._check(self._lib.qp_quantize_pack_tokens(self._h, x.data_ptr(), _dtype_code(x), x.numel() // channels, channels,
+                                                      bits, d_qp.data_ptr(), out.data_ptr(),
+                                                      out.numel() * out.element_size(), _stream(self.device)))
+        return out
+
+    def qp_unpack_dequantize_tokens(self, packed: torch.Tensor, tokens: int, channels: int, bits: int, d_qp: torch.Tensor,
+                                    out: torch.Tensor | None = None, out_dtype=torch.float32) -> torch.Tensor:
+        out = torch.empty(tokens * channels, dtype=out_dtype, device=packed.device) if out is None else out
+        self._check(self._lib.qp_unpack_dequantize_tokens(self._h, packed.data_ptr(), tokens, channels, bits,
+                                                          d_qp.data_ptr(), out.data_ptr(), _dtype_code(out),
+                                                          _stream(self.device)))
+        return out
+
+    def qp_sender_tokens_device(self, x: torch.Tensor, channels: int, bits: int, method: int = QP_CLIP_ACIQ,
+                                bmode: int = QP_B_MAD, out_packed: torch.Tensor | None = None,
+                                out_qp: torch.Tensor | None = None, stats_work: torch.Tensor | None = None):
+        """Token-wise statistics -> clip -> quantize+pack in one call; returns (packed, device QParams[tokens])."""
+        assert x.is_cuda and x.is_contiguous() and x.numel() % channels == 0
+        tokens = x.numel() // channels
+        out_packed = self._bytes(qp_packed_bytes(x.numel(), bits)) if out_packed is None else out_packed
+        out_qp = self._bytes(C.sizeof(QParams) * tokens) if out_qp is None else out_qp
+        stats_work = self._bytes(C.sizeof(Stats) * tokens) if stats_work is None else stats_work
+        self._check(self._lib.qp_sender_tokens_device(
+            self._h, x.data_ptr(), _dtype_code(x), tokens, channels, bits, method, bmode, out_packed.data_ptr(),
+            out_packed.numel() * out_packed.element_size(), out_qp.data_ptr(), stats_work.data_ptr(), _stream(self.device)))
         return out_packed, out_qp
 
     # -- host-buffer sender / receiver

@@ -169,9 +169,9 @@ extern "C" uint64_t qp_launch_count(qp_ctx* ctx) { return ctx ? ctx->launches : 
 extern "C" int32_t qp_set_search_path(qp_ctx* ctx, int path)
 {
     if (!ctx) return QP_ERR_INVALID_ARG;
-    if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS_CHAIN) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
-    ctx->moments_form = path == QP_SEARCH_INTERVALS_PLAIN ? 1 : (path == QP_SEARCH_INTERVALS_CHAIN ? 2 : 0);
-    ctx->search_path = path >= QP_SEARCH_INTERVALS_PLAIN ? QP_SEARCH_INTERVALS : path;
+    if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS_PLAIN) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
+    ctx->moments_form = path == QP_SEARCH_INTERVALS_PLAIN ? 1 : 0;
+    ctx->search_path = path == QP_SEARCH_INTERVALS_PLAIN ? QP_SEARCH_INTERVALS : path;
     return QP_OK;
 }
 

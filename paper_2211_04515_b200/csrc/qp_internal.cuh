@@ -79,7 +79,6 @@ struct qp_ctx {
     int stats_path;                      // 0 auto, 1 two kernels, 2 one cooperative launch where it applies
     int fused_checked, fused_ok;         // whether this device can hold the cooperative sender's grid
     int stats_fused_checked, stats_fused_ok;   // the same for the one-launch statistics
-    int ivc_checked, ivc_ok;             // and for the one-launch search (bit 0: fp32, bit 1: bf16)
     long long wait_cycles;               // limit of a wait for a tile copy (clock cycles)
     unsigned spin_limit;                 // limit of a grid-barrier wait (polls)
     int bar_extra;                       // test only: arrivals a grid barrier waits for beyond the grid size
@@ -139,6 +138,40 @@ bool qp_clip_method_closed_form(int method);     // ACIQ (| INTERSECT) or MINMAX
 
 // ------------------------------------------------------------- device helpers
 #ifdef __CUDACC__
+
+// Index checks of the debug build (-DQP_CHECK_BOUNDS; python -m paper_2211_04515_b200.build --check).
+// QP_CK(i, n) is `i` in the ordinary build.  In the debug build an index outside [0, n) is replaced by
+// 0, so the access stays inside its table, and a flag of the translation unit is raised, which
+// qp_get_status reports as QP_DEV_INDEX_RANGE: nothing traps and nothing faults.  Every translation
+// unit that uses QP_CK says QP_CK_UNIT once at file scope (it registers the unit's flag with the host).
+#ifdef QP_CHECK_BOUNDS
+static __device__ unsigned qp_ck_flag;
+template <typename I, typename N>
+__device__ __forceinline__ I qp_ck(I i, N n)
+{
+    if ((unsigned long long)(long long)i >= (unsigned long long)(long long)n) {
+        atomicOr(&qp_ck_flag, 1u);
+        return (I)0;
+    }
+    return i;
+}
+#define QP_CK(i, n) qp_ck((i), (n))
+struct qp_ck_unit { qp_ck_unit* next; unsigned (*read_and_clear)(); };
+void qp_ck_register(qp_ck_unit* u);
+#define QP_CK_UNIT                                                                                          \
+    static unsigned qp_ck_read_and_clear()                                                                  \
+    {                                                                                                       \
+        unsigned v = 0, z = 0;                                                                              \
+        if (cudaMemcpyFromSymbol(&v, qp_ck_flag, sizeof v) != cudaSuccess) { cudaGetLastError(); return 0; } \
+        if (v) cudaMemcpyToSymbol(qp_ck_flag, &z, sizeof z);                                                \
+        return v;                                                                                           \
+    }                                                                                                       \
+    static qp_ck_unit qp_ck_this_unit = {nullptr, qp_ck_read_and_clear};                                    \
+    static const int qp_ck_registered = (qp_ck_register(&qp_ck_this_unit), 0);
+#else
+#define QP_CK(i, n) (i)
+#define QP_CK_UNIT
+#endif
 
 // Quantizer set-up from a clip range, same on host and device: ends rounded to fp32, scale
 // and reciprocal from the rounded ends in fp64, rounded once.

@@ -23,7 +23,6 @@
 // relative in the worst case (all roundings aligned) and by ~1e-11 in practice.
 #include <type_traits>
 
-#include "qp_gridbar.cuh"
 #include "qp_internal.cuh"
 
 namespace {
@@ -785,529 +784,6 @@ __global__ void __launch_bounds__(IV_CURVE_THREADS) iv_curve_kernel(const qp_iv_
     qp_ds_pick(curve, steps, nb, bits, cand, setup, out, qp_out, status, s_curve);
 }
 
-// ---------------------------------------------------------------- the whole search in one launch
-//
-// The five kernels above (boundaries, rank sort, moments, reduce, curve) as ONE cooperative launch
-// of one block of 1024 threads per SM; what were kernel boundaries become two grid barriers, and the
-// tables that the first two kernels pass through global memory are built by every block for itself
-// in shared memory (2-3 us of redundant work instead of two launches and a sort over the grid):
-//
-//   tables    candidates and grid as in iv_bounds_kernel.  Thresholds and cell edges by bisection
-//             over float bit patterns as before, but started from a bracket of +-64 ulps about the
-//             value that real arithmetic gives (lo + (j - 1/2) scale; g_lo + (c - 1/2) gw): six
-//             evaluations of the code function instead of thirty (the full range is the fall-back,
-//             the result is the same smallest float either way).  No sort: a boundary's grid cell
-//             is monotone in its value, so its rank is the number of boundaries in lower cells
-//             (a prefix sum over the cells' counts) plus its rank among the few boundaries of its
-//             own cell (a cell's edge is its smallest element)
-//   moments   the second form of the pass (iv2_one): whole cells into per-cell, per-lane sums,
-//             elements of split cells through the warp's buffer into interval sums.  The 32-bit
-//             replica sums are folded into the interval sums every 327 680 elements per block, so
-//             one block per SM serves any tensor length
-//   barrier   rows of all blocks are out; block b adds up its slice of the intervals
-//   barrier   totals are out; block k scores candidate k; the last block to finish picks the winner
-//
-// Both barriers are bounded (qp_gridbar.cuh); a block whose wait runs out raises the abort flag, and
-// every block counts itself out on every path, so the counters are left at zero.
-constexpr int IVC_THREADS = IV2_THREADS;                 // 1024
-constexpr int IVC_WARPS = IVC_THREADS / 32;
-constexpr int IVC_WAVE_ITERS = 40;                       // double iterations (2 vectors per thread) between two folds
-
-struct IvcArgs {
-    const void* x;
-    uint64_t n;
-    const qp_stats_t* st;
-    const unsigned long long* hist;
-    int nb, bits, bmode, steps;
-    double F;
-    float4* cand;
-    int* valid;
-    qp_ds_setup* setup;
-    unsigned long long* part;                     // [grid][MAXB + 1]
-    double* outer;                                // [grid + 1][8]
-    qp_iv_total* tot;                             // [MAXB + 1]
-    double* curve;
-    qp_ds_result_t* out;
-    qp_qparams_t* qp_out;
-    unsigned* status;
-    unsigned* bar;                                // [0] arrivals, [1] blocks that have left, [2] abort flag; zero at entry
-    unsigned spin_limit, bar_extra;
-};
-
-// smallest float in [g_lo, g_hi] for which pred holds (pred monotone), +inf if there is none or if it
-// already holds at g_lo; `est` is where real arithmetic puts it
-template <typename P>
-__device__ __forceinline__ float ivc_first_true(float g_lo, float g_hi, float est, P pred)
-{
-    const float inf = __int_as_float(0x7F800000);
-    if (!(g_hi > g_lo) || pred(g_lo) || !pred(g_hi)) return inf;
-    const unsigned k_lo = key_of(g_lo), k_hi = key_of(g_hi);
-    unsigned lo = k_lo, hi = k_hi;
-    if (est == est && fabsf(est) < inf) {                    // narrow the bracket where that keeps the invariant
-        const unsigned ke = key_of(est);
-        if (ke >= k_lo && ke <= k_hi) {
-            const unsigned a = ke - k_lo > 64u ? ke - 64u : k_lo;
-            const unsigned b = k_hi - ke > 64u ? ke + 64u : k_hi;
-            if (a > k_lo && !pred(float_of(a))) lo = a;
-            if (b < k_hi && pred(float_of(b))) hi = b;
-        }
-    }
-    while (hi - lo > 1u) {
-        const unsigned mid = lo + ((hi - lo) >> 1);
-        if (pred(float_of(mid))) hi = mid; else lo = mid;
-    }
-    return float_of(hi);
-}
-
-// exclusive prefix sum of v[0 .. count) in place (count <= 3 * IVC_THREADS), all threads; returns the total
-__device__ __forceinline__ unsigned ivc_scan(unsigned* v, int count, unsigned* s_warp)
-{
-    const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
-    unsigned a[3], mine = 0;
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-        const int i = t * 3 + j;
-        a[j] = i < count ? v[i] : 0u;
-        mine += a[j];
-    }
-    unsigned incl = mine;
-    for (int o = 1; o < 32; o <<= 1) {
-        const unsigned up = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    if (lane == 31) s_warp[warp] = incl;
-    __syncthreads();
-    if (warp == 0) {
-        unsigned w = s_warp[lane];
-        unsigned wi = w;
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned up = __shfl_up_sync(0xFFFFFFFFu, wi, o);
-            if (lane >= o) wi += up;
-        }
-        s_warp[lane] = wi - w;                               // exclusive over the warps
-        if (lane == 31) s_warp[32] = wi;                     // the total
-    }
-    __syncthreads();
-    unsigned run = s_warp[warp] + incl - mine;
-#pragma unroll
-    for (int j = 0; j < 3; ++j) {
-        const int i = t * 3 + j;
-        if (i < count) v[i] = run;
-        run += a[j];
-    }
-    const unsigned total = s_warp[32];
-    __syncthreads();
-    return total;
-}
-
-template <typename T>
-__global__ void __launch_bounds__(IVC_THREADS, 1) iv_search_kernel(const IvcArgs a)
-{
-    extern __shared__ __align__(16) unsigned char raw[];
-    IvShared sh;
-    Iv2Shared s2;
-    s2.rcnt = reinterpret_cast<unsigned*>(raw);
-    s2.rs1 = s2.rcnt + (G + 1) * IV2_R;
-    sh.cnt = s2.rs1 + (G + 1) * IV2_R;
-    sh.s1 = sh.cnt + (MAXB + 1);
-    sh.bb = reinterpret_cast<float*>(sh.s1 + (MAXB + 1));
-    sh.cell = reinterpret_cast<unsigned*>(sh.bb + (MAXB + 1));
-    s2.stage = reinterpret_cast<float*>(sh.cell + (G + 1));
-    // while the tables are built, the replica tables' memory holds the temporaries
-    float4* t_cand = reinterpret_cast<float4*>(raw);                         // [IV_MAX_CAND]
-    float* t_thr = reinterpret_cast<float*>(t_cand + IV_MAX_CAND);           // [MAXB] thresholds, any order
-    unsigned* t_pos = reinterpret_cast<unsigned*>(t_thr + MAXB);             // [MAXB] where a threshold went in t_val
-    float* t_val = reinterpret_cast<float*>(t_pos + MAXB);                   // [MAXB] boundaries grouped by cell
-    unsigned* t_idx = reinterpret_cast<unsigned*>(t_val + MAXB);             // [MAXB] their original index
-    float* t_edge = reinterpret_cast<float*>(t_idx + MAXB);                  // [G + 1] left edge of every cell (cell 0: none)
-    unsigned* t_cnt = reinterpret_cast<unsigned*>(t_edge + (G + 1));         // [G + 2] boundaries per cell, then their prefix sums
-    unsigned* t_fill = t_cnt + (G + 2);                                      // [G + 2]
-    unsigned char* t_valid = reinterpret_cast<unsigned char*>(t_fill + (G + 2));   // [IV_MAX_CAND]
-    static_assert(sizeof(float4) * IV_MAX_CAND + 4 * 4 * MAXB + 4 * (G + 1) + 8 * (G + 2) + IV_MAX_CAND <= 8 * (G + 1) * IV2_R,
-                  "temporaries fit the replica tables");
-
-    __shared__ qp_ds_setup s;
-    __shared__ double red[IVC_WARPS];
-    __shared__ unsigned s_warp[33];
-    __shared__ unsigned s_m;
-    __shared__ int s_okflag;
-    __shared__ bool s_last;
-    __shared__ float s_lo[IVC_WARPS], s_hi[IVC_WARPS];
-    __shared__ unsigned long long s_top[IVC_WARPS];
-    __shared__ double s_curve[IV_MAX_CAND];
-    __shared__ unsigned long long s_n[IVC_WARPS][32], s_s[IVC_WARPS][32];
-
-    const T* x = static_cast<const T*>(a.x);
-    const float inf = __int_as_float(0x7F800000);
-    const unsigned NB = gridDim.x;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int ncand = a.steps + 1, L1 = (1 << a.bits) - 1, nthr = ncand * L1;
-    const unsigned cmask = (unsigned)L1;
-
-    // ---- tables: set-up, candidates, grid
-    {
-        unsigned long long top = 0;
-        const bool from_stats = a.st->hist_bins == a.nb;
-        const bool promised = (a.bmode & QP_B_HIST_IN_STATS) != 0;   // then nobody has counted into hist
-        if (promised && !from_stats && blockIdx.x == 0 && tid == 0) atomicOr(a.status, QP_DEV_HIST_MISSING);
-        for (int b = tid; !from_stats && !promised && b < a.nb; b += IVC_THREADS) {
-            const unsigned long long c = a.hist[b];
-            top = c > top ? c : top;
-        }
-        for (int o = 16; o > 0; o >>= 1) {
-            const unsigned long long other = __shfl_down_sync(0xFFFFFFFFu, top, o);
-            top = other > top ? other : top;
-        }
-        if (lane == 0) s_top[warp] = top;
-        __syncthreads();
-        if (tid == 0) {
-            for (int w = 1; w < IVC_WARPS; ++w) top = s_top[w] > top ? s_top[w] : top;
-            if (from_stats) top = a.st->hist_peak;
-            qp_ds_make_setup(a.st, top, a.nb, a.bmode, a.F, s);
-        }
-        __syncthreads();
-        float lo = inf, hi = -inf;
-        for (int k = tid; k < ncand; k += IVC_THREADS) {
-            float4 c;
-            int ok;
-            qp_ds_candidate(s, k, a.steps, a.bits, a.bmode & QP_B_MIDRISE, c, ok);
-            t_cand[k] = c;
-            t_valid[k] = (unsigned char)ok;
-            if (blockIdx.x == 0) { a.cand[k] = c; a.valid[k] = ok; }
-            if (ok) { lo = fminf(lo, c.x); hi = fmaxf(hi, c.y); }
-        }
-        for (int o = 16; o > 0; o >>= 1) {
-            lo = fminf(lo, __shfl_down_sync(0xFFFFFFFFu, lo, o));
-            hi = fmaxf(hi, __shfl_down_sync(0xFFFFFFFFu, hi, o));
-        }
-        if (lane == 0) { s_lo[warp] = lo; s_hi[warp] = hi; }
-        __syncthreads();
-        if (tid == 0) {
-            for (int w = 1; w < IVC_WARPS; ++w) { lo = fminf(lo, s_lo[w]); hi = fmaxf(hi, s_hi[w]); }
-            const double width = (double)hi - (double)lo;
-            float inv_gw = 0.f;
-            double u = 1.0;
-            if (width > 0.0) {
-                inv_gw = (float)((double)G / width);
-                int e;
-                frexp(width / (double)G, &e);               // cell width in [2^(e-1), 2^e)
-                u = ldexp(1.0, e - 16);                     // offsets (up to ~1.5 cells) stay below 2^17.6 units
-            }
-            s.g_lo = lo;
-            s.g_hi = hi;
-            s.inv_gw = inv_gw;
-            s.u = u;
-            s.inv_u = (float)(1.0 / u);
-            s.gw = (float)(width / (double)G);
-            s.pad2 = 0.f;
-            if (blockIdx.x == 0) *a.setup = s;
-        }
-        for (int c = tid; c < G + 2; c += IVC_THREADS) { t_cnt[c] = 0u; t_fill[c] = 0u; }
-        __syncthreads();
-    }
-    const float g_lo = s.g_lo, g_hi = s.g_hi, inv_gw = s.inv_gw, gw = s.gw;
-
-    // ---- tables: thresholds, cell edges, how many boundaries every cell holds
-    for (int t = tid; t < MAXB; t += IVC_THREADS) {
-        float v = inf;
-        if (t < nthr) {
-            const int k = t / L1, j = 1 + t % L1;
-            if (t_valid[k]) {
-                const float4 q = t_cand[k];
-                auto pred = [&](float xx) { return (int)qp_code(xx, q.x, q.y, q.w, cmask) >= j; };
-                v = ivc_first_true(g_lo, g_hi, fmaf((float)j - 0.5f, q.z, q.x), pred);
-            }
-            if (v < inf) atomicAdd(&t_cnt[cell_of(v, g_lo, inv_gw)], 1u);
-        }
-        t_thr[t] = v;
-    }
-    for (int c = tid; c <= G; c += IVC_THREADS) {
-        float v = inf;
-        if (c >= 1) {
-            auto pred = [&](float xx) { return cell_of(xx, g_lo, inv_gw) >= c; };
-            v = ivc_first_true(g_lo, g_hi, fmaf((float)c - 0.5f, gw, g_lo), pred);
-            if (v < inf) atomicAdd(&t_cnt[c], 1u);
-        }
-        t_edge[c] = v;
-    }
-    __syncthreads();
-    const unsigned m = ivc_scan(t_cnt, G + 1, s_warp);      // t_cnt[c] = boundaries in cells below c; m = all finite ones
-    if (tid == 0) { t_cnt[G + 1] = m; s_m = m; }
-    __syncthreads();
-
-    // ---- tables: boundaries grouped by cell (a cell's edge first), then ranked inside their cell
-    for (int t = tid; t < nthr; t += IVC_THREADS) {
-        const float v = t_thr[t];
-        unsigned pos = 0xFFFFFFFFu;
-        if (v < inf) {
-            const int c = cell_of(v, g_lo, inv_gw);
-            const unsigned e = (c >= 1 && t_edge[c] < inf) ? 1u : 0u;
-            pos = t_cnt[c] + e + atomicAdd(&t_fill[c], 1u);
-            t_val[pos] = v;
-            t_idx[pos] = (unsigned)t;
-        }
-        t_pos[t] = pos;
-    }
-    for (int c = 1 + tid; c <= G; c += IVC_THREADS)
-        if (t_edge[c] < inf) sh.bb[1 + t_cnt[c]] = t_edge[c];
-    for (int i = (int)m + 1 + tid; i <= MAXB; i += IVC_THREADS) sh.bb[i] = inf;
-    if (tid == 0) sh.bb[0] = g_lo;
-    __syncthreads();
-    for (int t = tid; t < nthr; t += IVC_THREADS) {
-        const unsigned pos = t_pos[t];
-        if (pos == 0xFFFFFFFFu) continue;
-        const float v = t_thr[t];
-        const int c = cell_of(v, g_lo, inv_gw);
-        const unsigned e = (c >= 1 && t_edge[c] < inf) ? 1u : 0u;
-        const unsigned a0 = t_cnt[c] + e, a1 = t_cnt[c + 1];     // the thresholds of this cell
-        unsigned r = 0;
-        for (unsigned q = a0; q < a1; ++q) {
-            const float w = t_val[q];
-            r += (w < v || (w == v && t_idx[q] < (unsigned)t)) ? 1u : 0u;
-        }
-        sh.bb[1 + a0 + r] = v;
-    }
-    // cell c meets the intervals i0 .. i1: the one that starts at its edge (interval 0 for cell 0) up to
-    // the one that starts at its last threshold; a cell that does not exist gets m + 1 (and no elements)
-    for (int c = tid; c <= G; c += IVC_THREADS) {
-        unsigned i0 = c == 0 ? 0u : t_cnt[c] + 1u, i1 = t_cnt[c + 1];
-        if (c >= 1 && !(t_edge[c] < inf)) i0 = i1 = m + 1u;
-        sh.cell[c] = (i0 & 0xFFFFu) | (i1 << 16);
-    }
-    for (unsigned i = tid; i <= (unsigned)MAXB; i += IVC_THREADS) { sh.cnt[i] = 0u; sh.s1[i] = 0u; }
-    __syncthreads();                                         // the temporaries are dead from here on
-    for (unsigned i = tid; i < (unsigned)(G + 1) * IV2_R; i += IVC_THREADS) {
-        const unsigned ci = sh.cell[i >> IV2_RS];
-        s2.rcnt[i] = ((ci >> 16) != (ci & 0xFFFFu)) ? IV2_SPLIT : 0u;
-        s2.rs1[i] = 0u;
-    }
-    __syncthreads();
-
-    // ---- moments: one pass over x, the replica sums folded into the interval sums between waves
-    const IvConst k = {g_lo, g_hi, inv_gw, gw, s.inv_u};
-    const bool guard = a.st->nonfinite != 0;
-    IvOuter o = {0.0, 0.0, 0.0, 0.0};
-    float* my_stage = s2.stage + warp * IV2_STAGE;
-    unsigned staged = 0;                                     // warp-uniform
-    // whole cells: replicas added up into the cell's one interval (count in 24 bits, 40-bit sum with its
-    // top byte beside the count), replicas back to zero; called by all threads between block barriers
-    auto fold = [&]() {
-        for (unsigned c = tid; c <= (unsigned)G; c += IVC_THREADS) {
-            const unsigned ci = sh.cell[c];
-            const unsigned i0 = ci & 0xFFFFu, i1 = ci >> 16;
-            if (i0 != i1 || i0 > m) continue;
-            unsigned long long cn = 0, cs = 0;
-            for (unsigned r = 0; r < IV2_R; ++r) {
-                const unsigned rr = (r + (unsigned)lane) & (IV2_R - 1u);   // lanes start at different replicas
-                cn += s2.rcnt[(c << IV2_RS) + rr];
-                cs += s2.rs1[(c << IV2_RS) + rr];
-                s2.rcnt[(c << IV2_RS) + rr] = 0u;
-                s2.rs1[(c << IV2_RS) + rr] = 0u;
-            }
-            const unsigned cw = sh.cnt[i0];
-            const unsigned long long sum = (((unsigned long long)(cw >> 24) << 32) | sh.s1[i0]) + cs;
-            sh.cnt[i0] = (unsigned)(((cw & 0xFFFFFFu) + cn) & 0xFFFFFFu) | ((unsigned)(sum >> 32) << 24);
-            sh.s1[i0] = (unsigned)sum;
-        }
-    };
-    {
-        constexpr int EPV = qp_span<T>::EPV;
-        const qp_span<T> sp(x, a.n);
-        const T* xv = x + sp.head;
-        const uint64_t stride = (uint64_t)NB * IVC_THREADS;
-        auto body = [&](auto guard_tag) {
-            constexpr bool GD = decltype(guard_tag)::value;
-            const float skip = __int_as_float(0x7FC00000);   // NaN: ignored by the guarded form
-            uint64_t v = (uint64_t)blockIdx.x * IVC_THREADS + tid;
-            // Two vectors per lane for as many iterations as the block's LAST warp has both (a count that is
-            // the same for every thread of the block, so the block barriers of the folds line up); every
-            // `wave` iterations, i.e. 327 680 elements per block, the replica sums are folded.
-            const uint64_t last = (uint64_t)blockIdx.x * IVC_THREADS + (IVC_THREADS - 1) + stride;
-            const uint64_t iters = last < sp.nvec ? (sp.nvec - 1 - last) / (2 * stride) + 1 : 0;
-            constexpr int wave = IVC_WAVE_ITERS * 4 / EPV;
-            int since_fold = 0;
-            for (uint64_t it = 0; it < iters; ++it, v += 2 * stride) {
-                float e0[EPV], e1[EPV];
-                qp_load_vec(xv + v * EPV, e0);
-                qp_load_vec(xv + (v + stride) * EPV, e1);
-                IvBatch bt = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int i = 0; i < EPV; ++i) iv2_one<GD>(e0[i], sh, s2, k, bt, my_stage, staged, lane);
-#pragma unroll
-                for (int i = 0; i < EPV; ++i) iv2_one<GD>(e1[i], sh, s2, k, bt, my_stage, staged, lane);
-                iv_flush(o, bt);
-                if (++since_fold == wave) {
-                    since_fold = 0;
-                    __syncthreads();
-                    fold();
-                    __syncthreads();
-                }
-            }
-            // the rest (at most three vectors per lane): warps may be partly filled, so every lane of a warp
-            // that still has work goes on
-            const uint64_t warp_v0 = v - lane;               // vector of lane 0 (v advanced alike in all lanes)
-            for (uint64_t w0 = warp_v0; w0 < sp.nvec; w0 += stride) {
-                const uint64_t mine = w0 + lane;
-                const bool have = mine < sp.nvec;
-                float e0[EPV];
-                if (have) qp_load_vec(xv + mine * EPV, e0);
-                IvBatch bt = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-                for (int i = 0; i < EPV; ++i) iv2_one<true>(have ? e0[i] : skip, sh, s2, k, bt, my_stage, staged, lane);
-                iv_flush(o, bt);
-            }
-            if (blockIdx.x == 0) {
-                const uint64_t t0 = sp.head + sp.nvec * EPV;
-                const uint64_t extra = sp.head + sp.tail;
-                for (uint64_t i0 = (tid & ~31u); i0 < extra; i0 += IVC_THREADS) {
-                    const uint64_t i = i0 + lane;
-                    const bool have = i < extra;
-                    IvBatch bt = {0.f, 0.f, 0.f, 0.f};
-                    const float x1 = have ? qp_load_one(x + (i < sp.head ? i : t0 + (i - sp.head))) : skip;
-                    iv2_one<true>(x1, sh, s2, k, bt, my_stage, staged, lane);
-                    iv_flush(o, bt);
-                }
-            }
-        };
-        if (guard) body(std::true_type{}); else body(std::false_type{});
-    }
-    __syncwarp();
-    if ((unsigned)lane < staged) iv2_exact(my_stage[lane], sh, k);     // what is left in the warp's buffer (< 32)
-    __syncthreads();
-    fold();
-    __syncthreads();
-
-    // ---- this block's row (count << 40 | 40-bit sum of offsets per interval) and outer sums
-    unsigned long long* mine = a.part + (size_t)blockIdx.x * (MAXB + 1);
-    for (unsigned i = tid; i <= m; i += IVC_THREADS) {
-        const unsigned cw = sh.cnt[i];
-        mine[i] = ((unsigned long long)(cw & 0xFFFFFFu) << 40) | ((unsigned long long)(cw >> 24) << 32) | sh.s1[i];
-    }
-    {
-        const double r0 = qp_block_sum(o.s1, red), r1 = qp_block_sum(o.s1a, red);
-        const double r2 = qp_block_sum(o.s2, red);
-        const double r6 = qp_block_sum(o.s2_in, red);
-        if (tid == 0) {
-            double* dst = a.outer + (size_t)blockIdx.x * 8;
-            dst[0] = r0; dst[1] = r1; dst[2] = r2; dst[3] = 0.0; dst[4] = 0.0; dst[5] = 0.0; dst[6] = r6;
-        }
-    }
-    bool ok = qp_grid::barrier(a.bar, NB + a.bar_extra, a.spin_limit, a.status, &s_okflag);
-    if (!ok && tid == 0) atomicExch(a.bar + 2, 1u);
-
-    // ---- totals: block b adds up intervals [b * per, (b + 1) * per) over all rows; warp = row group, lane = interval
-    if (ok) {
-        const unsigned per = (m + 1u + NB - 1u) / NB;        // <= 32 from 129 blocks on; otherwise a loop over lane groups
-        for (unsigned base = 0; base < per; base += 32u) {
-            const unsigned i = blockIdx.x * per + base + lane;
-            const bool have = base + lane < per && i <= m;
-            unsigned long long cn = 0, cs = 0;
-            if (have)
-                for (unsigned r = warp; r < NB; r += IVC_WARPS) {
-                    const unsigned long long p = __ldcg(&a.part[(size_t)r * (MAXB + 1) + i]);
-                    cn += p >> 40;
-                    cs += p & S1_MASK;
-                }
-            __syncthreads();
-            s_n[warp][lane] = cn;
-            s_s[warp][lane] = cs;
-            __syncthreads();
-            if (warp == 0 && have) {
-                for (int w = 1; w < IVC_WARPS; ++w) { cn += s_n[w][lane]; cs += s_s[w][lane]; }
-                a.tot[i].n = cn;
-                a.tot[i].s1 = cs;
-            }
-        }
-        if (blockIdx.x == 0 && tid < 7 * 32) {               // outer sums in block order: warp w adds up quantity w
-            double t = 0.0;
-            for (unsigned b = lane; b < NB; b += 32) t += __ldcg(&a.outer[(size_t)b * 8 + warp]);
-            for (int of = 16; of > 0; of >>= 1) t += __shfl_down_sync(0xFFFFFFFFu, t, of);
-            if (lane == 0) a.outer[(size_t)NB * 8 + warp] = t;
-        }
-    }
-    {
-        const bool met = qp_grid::barrier(a.bar, 2u * NB + a.bar_extra, a.spin_limit, a.status, &s_okflag);
-        if (!met && tid == 0) atomicExch(a.bar + 2, 1u);
-        ok = ok && met && qp_grid::ld_acquire(a.bar + 2) == 0u;
-    }
-
-    // ---- curve: block k scores candidates k, k + grid, ...: sum_i N_i a^2 - 2 a S1_i with a = level - reference
-    if (ok) {
-        const double u = s.u;
-        const double* outer_tot = a.outer + (size_t)NB * 8;
-        for (int kc = blockIdx.x; kc < ncand; kc += (int)NB) {
-            const bool valid = __ldcg(&a.valid[kc]) != 0;
-            const float4 q = __ldcg(&a.cand[kc]);
-            auto level = [&](float r) {      // reconstruction level that the candidate assigns to r
-                const unsigned c = qp_code(r, q.x, q.y, q.w, cmask);
-                return (double)fmaf(__fsub_rn(__uint_as_float(0x4B000000u | c), 8388608.0f), q.z, q.x);
-            };
-            double acc = 0.0;
-            if (valid) {
-                constexpr int PER = (MAXB + 1 + IVC_THREADS - 1) / IVC_THREADS;
-                ulonglong2 t[PER];
-#pragma unroll
-                for (int j = 0; j < PER; ++j) {              // all loads first (independent), then the arithmetic
-                    const unsigned i = tid + j * IVC_THREADS;
-                    t[j] = i <= m ? __ldcg(reinterpret_cast<const ulonglong2*>(&a.tot[i])) : make_ulonglong2(0ull, 0ull);
-                }
-#pragma unroll
-                for (int j = 0; j < PER; ++j) {
-                    if (t[j].x == 0) continue;
-                    const float left = sh.bb[tid + j * IVC_THREADS];       // an element of the interval: fixes its codes
-                    const float r = cell_ref(cell_pm(left, g_lo, inv_gw), g_lo, gw);
-                    const double av = level(left) - (double)r;
-                    acc += (double)t[j].x * av * av - 2.0 * av * ((double)t[j].y * u);
-                }
-            }
-            const double total = qp_block_sum(acc, red);
-            if (tid == 0) {
-                double mse = __longlong_as_double(0x7FF0000000000000ll);
-                if (valid) {
-                    const double s1 = __ldcg(&outer_tot[0]), s1a = __ldcg(&outer_tot[1]), s2o = __ldcg(&outer_tot[2]);
-                    const double s1_lo = 0.5 * (s1a - s1), s1_hi = 0.5 * (s1a + s1);   // sums of the distances beyond each end
-                    const double s2_in = __ldcg(&outer_tot[6]);
-                    const double a_lo = level(g_lo) - (double)g_lo;                    // >= 0: below every clip range
-                    const double a_hi = level(g_hi) - (double)g_hi;                    // <= 0: above every clip range
-                    double tt = total + s2_in * (u * u);               // sum of squared offsets: the same for every candidate
-                    tt += 2.0 * a_lo * s1_lo - 2.0 * a_hi * s1_hi + s2o;                // what lies beyond the ends (see IvOuter)
-                    const unsigned long long nf = s.n_finite;
-                    mse = nf ? tt / (double)nf : 0.0;
-                }
-                a.curve[kc] = mse;
-            }
-            __syncthreads();
-        }
-    }
-
-    // ---- exit: every block counts itself out (on every path); the last one picks the winner
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(a.bar + 1, 1u) == NB - 1u);
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const bool good = ok && qp_grid::ld_acquire(a.bar + 2) == 0u;
-    if (good) qp_ds_pick(a.curve, a.steps, a.nb, a.bits, a.cand, a.setup, a.out, a.qp_out, a.status, s_curve);
-    __syncthreads();
-    if (tid == 0) {                                          // everybody has left: the counters go back to zero
-        a.bar[0] = 0u;
-        a.bar[1] = 0u;
-        a.bar[2] = 0u;
-    }
-}
-
-// Whether this device can hold the one-launch search (checked once per context).
-template <typename T>
-bool ivc_usable(qp_ctx* ctx, size_t smem)
-{
-    int coop = 0, per_sm = 0;
-    return cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, ctx->device) == cudaSuccess && coop &&
-           cudaFuncSetAttribute(iv_search_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
-           cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, iv_search_kernel<T>, IVC_THREADS, smem) == cudaSuccess &&
-           per_sm >= 1;
-}
-
 template <typename T>
 int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_stats, int bits, int bmode, int steps,
                        int nb, double F, qp_ds_result_t* d_out, qp_qparams_t* d_qp_out, cudaStream_t s)
@@ -1320,35 +796,6 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)(G + 1) * 4 + 16;
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
-    constexpr size_t smem_c = (size_t)(G + 1) * IV2_R * 8 + (size_t)(MAXB + 1) * 12 + (size_t)(G + 1) * 4 +
-                              (size_t)IV2_WARPS * IV2_STAGE * 4 + 16;
-    const int tsel = sizeof(T) == 4 ? 0 : 1;
-    if (ctx->moments_form == 0 && n < (1ull << 30)) {        // the second form: the whole search as one cooperative launch
-        if (!(ctx->ivc_checked & (1 << tsel))) {
-            ctx->ivc_checked |= 1 << tsel;
-            if (ivc_usable<T>(ctx, smem_c)) ctx->ivc_ok |= 1 << tsel; else cudaGetLastError();
-        }
-        if (ctx->ivc_ok & (1 << tsel)) {
-            IvcArgs a;
-            a.x = x; a.n = n; a.st = d_stats; a.hist = ctx->d_hist; a.nb = nb; a.bits = bits; a.bmode = bmode; a.steps = steps;
-            a.F = F; a.cand = ctx->d_cand; a.valid = ctx->d_valid; a.setup = ctx->d_setup; a.part = ctx->d_iv_part;
-            a.outer = ctx->d_iv_outer; a.tot = ctx->d_iv_tot; a.curve = ctx->d_curve; a.out = d_out; a.qp_out = d_qp_out;
-            a.status = ctx->d_status;
-            a.bar = reinterpret_cast<unsigned*>(ctx->d_fused) + 16;      // words 16..18 of the barrier scratch
-            a.spin_limit = ctx->spin_limit;
-            a.bar_extra = (unsigned)ctx->bar_extra;
-            const uint64_t nvec = n / (16 / sizeof(T));
-            uint64_t want = (nvec + IVC_THREADS - 1) / IVC_THREADS;
-            if (want < 1) want = 1;
-            const unsigned grid = (unsigned)(want < (uint64_t)ctx->sm_count ? want : (uint64_t)ctx->sm_count);
-            void* params[] = {&a};
-            if (cudaLaunchCooperativeKernel((void*)iv_search_kernel<T>, dim3(grid), dim3(IVC_THREADS), params, smem_c, s) !=
-                cudaSuccess)
-                return qp_check_launch(ctx, "qp_dsaciq_search (cooperative launch)");
-            ctx->launches += 1;
-            return qp_check_launch(ctx, "qp_dsaciq_search (interval path)");
-        }
-    }
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
                                                 ctx->d_setup, ctx->d_iv_bnd, ctx->d_status);
     unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]

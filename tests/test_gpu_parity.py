@@ -1257,3 +1257,120 @@ def test_search_channels_full_size_c3_sampled(ctx):
         assert abs(res.b_r - ro.b_r) <= 1e-9 * ro.b_r and abs(res.mse_e - ro.mse_e) <= 2e-6 * ro.mse_e
         assert res.k_star == ro.k_star or curve_o[res.k_star] <= ro.mse_star * (1 + 1e-6)
     assert ctx.qp_get_status() & ~qp.QP_DEV_DEGENERATE == 0
+
+
+# ------------------------------------------------------------------ token-wise variant
+
+def check_tokens(ctx, x_np, d_x, channels, bits, method=qp.QP_CLIP_ACIQ, out_bf16=False):
+    """Statistics, quantizers, packed stream and reconstruction of the token-wise calls against the oracle:
+    statistics at 1e-5; the packed stream bit for bit under the quantizers the kernels produced, and those
+    quantizers against the oracle's per token; reconstruction at 1e-6 (bf16: the rounded oracle value)."""
+    tokens = x_np.size // channels
+    d_stats = ctx.qp_stats_tokens(d_x, channels)
+    st = _read_array(d_stats, qp.Stats, tokens)
+    st_o = oracle.stats_tokens(x_np, channels)
+    for t in range(tokens):
+        check_stats(st[t], st_o[t])
+    o_method, cut = (oracle.CLIP_MINMAX, False) if method & 0xF == qp.QP_CLIP_MINMAX else (oracle.CLIP_ACIQ, bool(method & qp.QP_CLIP_INTERSECT))
+    d_qp = ctx.qp_clip_qparams_tokens_device(d_stats, tokens, bits, method)
+    got = _read_array(d_qp, qp.QParams, tokens)
+    rc_o, qp_o = oracle.clip_tokens(st_o, bits, o_method, cut, midrise=bool(method & qp.QP_CLIP_MIDRISE))
+    for t in range(tokens):
+        width = max(qp_o[t].hi - qp_o[t].lo, 1e-30)
+        assert abs(got[t].lo - qp_o[t].lo) <= 1e-5 * width and abs(got[t].hi - qp_o[t].hi) <= 1e-5 * width, t
+        assert got[t].bits == bits and got[t].flags == qp_o[t].flags
+        rc2, again = oracle.make_qparams(got[t].lo, got[t].hi, bits)
+        assert (again.scale, again.inv_scale) == (got[t].scale, got[t].inv_scale)
+    mine = (oracle.QParams * tokens)(*[oracle.QParams(g.lo, g.hi, g.scale, g.inv_scale, g.bits, g.flags) for g in got])
+    nbytes = qp.qp_packed_bytes(x_np.size, bits)
+    whole, packed = guarded(nbytes)
+    ctx.qp_quantize_pack_tokens(d_x, channels, bits, d_qp, out=packed)
+    codes_o = oracle.quantize_tokens(x_np, channels, mine)
+    assert np.array_equal(packed.cpu().numpy(), oracle.pack(codes_o, bits))
+    assert canaries_intact(whole, nbytes)
+    esz = 2 if out_bf16 else 4
+    whole_y, y_bytes = guarded(x_np.size * esz)
+    y = y_bytes.view(torch.bfloat16 if out_bf16 else torch.float32)
+    ctx.qp_unpack_dequantize_tokens(packed, tokens, channels, bits, d_qp, out=y)
+    y_o = oracle.dequantize_tokens(codes_o, channels, mine)
+    if out_bf16:
+        assert np.array_equal(y.float().cpu().numpy(), si.bf16_bits_to_f32(si.to_bf16_bits(y_o)))
+    else:
+        assert np.max(np.abs(y.cpu().numpy().astype(np.float64) - y_o.astype(np.float64)), initial=0.0) <= 1e-6
+    assert canaries_intact(whole_y, x_np.size * esz)
+    # the one-call sender gives the same stream and quantizers
+    got_packed, got_qp = ctx.qp_sender_tokens_device(d_x, channels, bits, method)
+    assert torch.equal(got_packed, packed) and torch.equal(got_qp, d_qp)
+    return got
+
+
+@pytest.mark.parametrize("bits", ALL_BITS)
+def test_tokens_vit_shapes(ctx, bits):
+    x = si.vit_activation((2, 197, 768), 161, outlier_frac=0.01).reshape(-1)
+    check_tokens(ctx, x, dev(x), 768, bits)
+    assert ctx.qp_get_status() == 0
+
+
+@pytest.mark.parametrize("channels,tokens", [(1, 700), (3, 777), (4, 1), (20, 411), (64, 2049), (100, 333), (1000, 37),
+                                              (1280, 300), (5000, 9)])
+def test_tokens_shapes_ragged_and_methods(ctx, channels, tokens):
+    x = si.vit_activation((1, tokens, channels), 162 + channels % 5, outlier_frac=0.05).reshape(-1)
+    d = dev(x)
+    for bits, method in ((2, qp.QP_CLIP_ACIQ), (5, qp.QP_CLIP_MINMAX), (8, qp.QP_CLIP_ACIQ | qp.QP_CLIP_INTERSECT),
+                         (16, qp.QP_CLIP_ACIQ), (4, qp.QP_CLIP_ACIQ | qp.QP_CLIP_MIDRISE),
+                         (3, qp.QP_CLIP_MINMAX | qp.QP_CLIP_MIDRISE)):
+        check_tokens(ctx, x, d, channels, bits, method)
+    ctx.qp_get_status()                                         # one-channel tokens have no spread: degenerate
+
+
+def test_tokens_misaligned_nonfinite_bf16_and_errors(ctx):
+    x = si.vit_activation((1, 301, 96), 167, outlier_frac=0.03).reshape(-1).astype(np.float32)
+    big = dev(np.concatenate([np.zeros(1, np.float32), x]))
+    check_tokens(ctx, x, big[1:], 96, 4)                        # 4-byte aligned only: scalar paths
+    x[[5, 96 * 7 + 5, 96 * 100 + 17]] = [np.nan, np.inf, -np.inf]
+    check_tokens(ctx, x, dev(x), 96, 3)
+    assert ctx.qp_get_status() & qp.QP_DEV_NONFINITE
+    h = si.to_bf16_bits(si.vit_activation((1, 150, 256), 168).reshape(-1))
+    d = torch.from_numpy(h.view(np.int16)).cuda().view(torch.bfloat16)
+    check_tokens(ctx, oracle.widen_bf16(h), d, 256, 4)
+    check_tokens(ctx, oracle.widen_bf16(h), d, 256, 8, out_bf16=True)
+    check_tokens(ctx, oracle.widen_bf16(h[:150 * 100]), d[:150 * 100], 100, 6, out_bf16=True)   # 100 % 8 != 0
+    const = np.repeat(np.array([1.5, -2.0, 0.0, 7.25], dtype=np.float32), 500)                  # every token constant
+    got = check_tokens(ctx, const, dev(const), 500, 4)
+    assert all(g.flags == 1 for g in got) and ctx.qp_get_status() & qp.QP_DEV_DEGENERATE
+    y = dev(si.flat_iid(4096, 6, "laplace"))
+    d_stats = ctx.qp_stats_tokens(y, 64)
+    for bad in (qp.QP_CLIP_DSACIQ, 3):
+        with pytest.raises(qp.QuantPipeError):
+            ctx.qp_clip_qparams_tokens_device(d_stats, 64, 4, bad)
+    d_qp = ctx.qp_clip_qparams_tokens_device(d_stats, 64, 4)
+    with pytest.raises(qp.QuantPipeError):
+        ctx.qp_quantize_pack_tokens(y, 64, 4, d_qp, out=torch.empty(16, dtype=torch.uint8, device="cuda"))
+    ctx.qp_quantize_pack_tokens(y, 64, 8, d_qp)                 # quantizers made for 4 bits: flagged on the device
+    assert ctx.qp_get_status() & qp.QP_DEV_BITS_MISMATCH
+
+
+def test_tokens_full_size_c2_sampled(ctx):
+    """ViT-Base micro-batch of 64 images (12 608 tokens of 768 channels): every token's statistics, and the
+    packed words and reconstructions of sampled tokens, against the oracle."""
+    x = si.config_tensor("c2").reshape(-1, 768)
+    tokens = x.shape[0]
+    d = dev(x.reshape(-1))
+    d_stats = ctx.qp_stats_tokens(d, 768)
+    st = _read_array(d_stats, qp.Stats, tokens)
+    st_o = oracle.stats_tokens(x.reshape(-1), 768)
+    for t in range(0, tokens, 97):
+        check_stats(st[t], st_o[t])
+    d_qp = ctx.qp_clip_qparams_tokens_device(d_stats, tokens, 4)
+    got = _read_array(d_qp, qp.QParams, tokens)
+    packed = ctx.qp_quantize_pack_tokens(d, 768, 4, d_qp)
+    y = ctx.qp_unpack_dequantize_tokens(packed, tokens, 768, 4, d_qp).cpu().numpy().reshape(-1, 768)
+    packed = packed.cpu().numpy()
+    for t0 in (0, 4097, tokens - 3):
+        rows = np.ascontiguousarray(x[t0:t0 + 3])
+        mine = (oracle.QParams * 3)(*[oracle.QParams(g.lo, g.hi, g.scale, g.inv_scale, g.bits, g.flags) for g in got[t0:t0 + 3]])
+        codes = oracle.quantize_tokens(rows, 768, mine)
+        nb = 3 * 768 * 4 // 8
+        assert np.array_equal(packed[t0 * 768 // 2: t0 * 768 // 2 + nb], oracle.pack(codes, 4)[:nb])
+        assert np.max(np.abs(y[t0:t0 + 3].reshape(-1) - oracle.dequantize_tokens(codes, 768, mine))) <= 1e-6
+    assert ctx.qp_get_status() == 0
