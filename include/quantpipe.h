@@ -67,6 +67,7 @@ enum { QP_B_MAD = 0 /* sum|x-mean|/N */, QP_B_MEAN_ABS = 1 /* sum|x|/N, the form
 #define QP_DEV_NONFINITE 4u
 #define QP_DEV_STREAM_TIMEOUT 8u  /* a bounded wait for a tile copy ran out; results of that call are invalid */
 #define QP_DEV_HIST_MISSING 16u   /* a search was promised a histogram in the statistics (QP_B_HIST_IN_STATS) that is not there */
+#define QP_DEV_INDEX_RANGE 32u    /* debug build only: an index into a shared-memory or scratch table was out of range (redirected to entry 0) */
 
 /* Per-tensor statistics (Sec. 3: min/max of naive PTQ; mean and Laplace scale b of ACIQ;
  * b_E of the directed search).  All fields but n are over the finite elements. */
@@ -133,6 +134,12 @@ int32_t qp_set_wait_limit_for_testing(qp_ctx* ctx, long long tile_wait_cycles, u
 /* Text of the last error recorded on this context (never NULL). */
 const char* qp_last_error(qp_ctx* ctx);
 const char* qp_status_string(int32_t status);
+/* 1 if the library was built with index checks (-DQP_CHECK_BOUNDS; `python -m paper_2211_04515_b200.build
+ * --check` writes libquantpipe_check.so): every index into the kernels' shared-memory tables and scratch
+ * rows is then range-checked, an index out of range is redirected to entry 0 (nothing traps or faults) and
+ * qp_get_status reports QP_DEV_INDEX_RANGE.  The stand-in, on this library's own tables, for a memory
+ * checker where none can be run.  0 for the ordinary build. */
+int32_t qp_built_with_index_checks(void);
 /* Number of kernels this context has launched since qp_create (host-side count). */
 uint64_t qp_launch_count(qp_ctx* ctx);
 
@@ -283,7 +290,9 @@ int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, co
  * The pass over x that gathers the moments has two forms with identical results: the plain one
  * (every element looks its interval up), and one that adds elements of grid cells without a
  * threshold straight into per-cell, per-lane sums and looks up only the others; the second is
- * used up to ~150 M elements, QP_SEARCH_INTERVALS_PLAIN forces the first. */
+ * used up to ~150 M elements, QP_SEARCH_INTERVALS_PLAIN forces the first.  Around the pass, two small
+ * kernels build the tables (candidates and thresholds; their sorted order and the cell table) and two
+ * finish (the blocks' partials added up; every candidate scored and the winner picked). */
 enum { QP_SEARCH_AUTO = 0, QP_SEARCH_CANDIDATES = 1, QP_SEARCH_INTERVALS = 2, QP_SEARCH_INTERVALS_PLAIN = 3 };
 int32_t qp_set_search_path(qp_ctx* ctx, int path);
 /* Graph replay of the multi-kernel calls (an execution option; the paper has no counterpart,

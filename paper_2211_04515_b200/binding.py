@@ -12,7 +12,8 @@ import os
 import torch
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_PKG, "libquantpipe.so")
+# QUANTPIPE_LIB selects another build of the library (the one with index checks, libquantpipe_check.so)
+LIB_PATH = os.environ.get("QUANTPIPE_LIB") or os.path.join(_PKG, "libquantpipe.so")
 
 QP_OK = 0
 QP_ERR_INVALID_ARG, QP_ERR_UNSUPPORTED_BITS, QP_ERR_UNSUPPORTED_DTYPE = -1, -2, -3
@@ -24,6 +25,7 @@ QP_F32, QP_BF16 = 0, 1
 QP_DIST_LAPLACE, QP_DIST_GAUSS = 0, 1
 QP_B_MAD, QP_B_MEAN_ABS = 0, 1
 QP_DEV_BITS_MISMATCH, QP_DEV_DEGENERATE, QP_DEV_NONFINITE, QP_DEV_STREAM_TIMEOUT, QP_DEV_HIST_MISSING = 1, 2, 4, 8, 16
+QP_DEV_INDEX_RANGE = 32
 QP_DEFAULT_STEPS, QP_DEFAULT_HIST_BINS = 100, 100
 QP_SEARCH_AUTO, QP_SEARCH_CANDIDATES, QP_SEARCH_INTERVALS, QP_SEARCH_INTERVALS_PLAIN = 0, 1, 2, 3
 QP_SENDER_AUTO, QP_SENDER_CHAIN, QP_SENDER_FUSED = 0, 1, 2
@@ -43,7 +45,7 @@ EXPORTS = (
     "qp_quantize_pack_channels", "qp_unpack_dequantize_channels", "qp_midrise_range", "qp_sender_channels_device",
     "qp_stats_tokens", "qp_clip_qparams_tokens_device", "qp_quantize_pack_tokens", "qp_unpack_dequantize_tokens",
     "qp_sender_tokens_device",
-    "qp_set_stats_path", "qp_dsaciq_candidates", "qp_dsaciq_candidates_channels", "qp_set_wait_limit_for_testing",
+    "qp_built_with_index_checks", "qp_set_stats_path", "qp_dsaciq_candidates", "qp_dsaciq_candidates_channels", "qp_set_wait_limit_for_testing",
 )
 
 
@@ -140,6 +142,7 @@ def load() -> C.CDLL:
     L.qp_set_graph_replay.argtypes = [vp, C.c_int]
     L.qp_set_sender_path.argtypes = [vp, C.c_int]
     L.qp_set_stats_path.argtypes = [vp, C.c_int]
+    L.qp_built_with_index_checks.argtypes = []
     L.qp_dsaciq_candidates.argtypes = [vp, C.POINTER(QParams), C.c_int, vp]
     L.qp_dsaciq_candidates_channels.argtypes = [vp, C.POINTER(QParams), u64, vp]
     L.qp_set_wait_limit_for_testing.argtypes = [vp, C.c_longlong, C.c_uint32, C.c_int]
@@ -166,6 +169,10 @@ def load() -> C.CDLL:
 
 
 # ------------------------------------------------------------- host, pure
+
+def qp_built_with_index_checks() -> bool:
+    return bool(load().qp_built_with_index_checks())
+
 
 def qp_packed_bytes(n: int, bits: int) -> int:
     return int(load().qp_packed_bytes(n, bits))

@@ -43,6 +43,32 @@ extern "C" const char* qp_status_string(int32_t s)
 
 extern "C" const char* qp_last_error(qp_ctx* ctx) { return ctx ? ctx->err : "no context"; }
 
+// ----------------------------------------------------------------- index checks of the debug build
+
+#ifdef QP_CHECK_BOUNDS
+static qp_ck_unit* g_ck_units = nullptr;
+void qp_ck_register(qp_ck_unit* u)
+{
+    u->next = g_ck_units;
+    g_ck_units = u;
+}
+static unsigned qp_ck_collect()
+{
+    unsigned any = 0;
+    for (qp_ck_unit* u = g_ck_units; u; u = u->next) any |= u->read_and_clear();
+    return any;
+}
+#endif
+
+extern "C" int32_t qp_built_with_index_checks(void)
+{
+#ifdef QP_CHECK_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
+
 // ----------------------------------------------------------------- context
 
 static void qp_drop_graphs(qp_ctx* ctx);
@@ -149,6 +175,9 @@ extern "C" int32_t qp_get_status(qp_ctx* ctx, void* stream)
         snprintf(ctx->err, sizeof ctx->err, "CUDA error in qp_get_status: %s", cudaGetErrorString(e));
         return QP_ERR_CUDA;
     }
+#ifdef QP_CHECK_BOUNDS
+    if (qp_ck_collect()) word |= QP_DEV_INDEX_RANGE;         // (the flags are per translation unit, not per context)
+#endif
     if (word & QP_DEV_STREAM_TIMEOUT) {
         // a cooperative launch that gave up may have left its arrival counters and histogram mid-way
         e = cudaMemsetAsync(ctx->d_fused, 0, QP_FUSED_BYTES, s);
@@ -171,7 +200,7 @@ extern "C" int32_t qp_set_search_path(qp_ctx* ctx, int path)
     if (!ctx) return QP_ERR_INVALID_ARG;
     if (path < QP_SEARCH_AUTO || path > QP_SEARCH_INTERVALS_PLAIN) return qp_fail(ctx, QP_ERR_INVALID_ARG, "search path");
     ctx->moments_form = path == QP_SEARCH_INTERVALS_PLAIN ? 1 : 0;
-    ctx->search_path = path == QP_SEARCH_INTERVALS_PLAIN ? QP_SEARCH_INTERVALS : path;
+    ctx->search_path = path >= QP_SEARCH_INTERVALS_PLAIN ? QP_SEARCH_INTERVALS : path;
     return QP_OK;
 }
 
@@ -603,7 +632,7 @@ extern "C" int32_t qp_dsaciq_search(qp_ctx* ctx, const void* d_x, int dtype, uin
         2, (unsigned long long)(uintptr_t)d_x, n, (unsigned long long)(uintptr_t)d_stats,
         (unsigned long long)(uintptr_t)d_out, (unsigned long long)(uintptr_t)d_qp_out,
         (unsigned long long)dtype | (unsigned long long)bits << 8 | (unsigned long long)ctx->search_path << 16 |
-            (unsigned long long)ctx->moments_form << 24,                   // each below 256
+            (unsigned long long)ctx->moments_form << 24,
         (unsigned long long)(unsigned)bmode, (unsigned long long)steps, (unsigned long long)hist_bins};
     rc = qp_graphed(ctx, s, key, [&] {
         return qp_launch_search(ctx, d_x, dtype, n, d_stats, bits, bmode, steps, hist_bins,

@@ -17,6 +17,8 @@
 //   ch_unpack_kernel          mirror image: words -> codes in the staging rows -> coalesced stores
 #include "qp_internal.cuh"
 
+QP_CK_UNIT
+
 namespace {
 
 constexpr int CH_THREADS = 256;
@@ -344,9 +346,9 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
 #pragma unroll
                 for (int h = 0; h < EPV; h += 4) {               // EPV divides C: the vector stays in one row
                     float lo[4], hi[4], inv[4];
-                    ch_lds4(tab.lo + c + h, lo);
-                    ch_lds4(tab.hi + c + h, hi);
-                    ch_lds4(tab.inv + c + h, inv);
+                    ch_lds4(tab.lo + QP_CK(c + h, C - 3), lo);
+                    ch_lds4(tab.hi + QP_CK(c + h, C - 3), hi);
+                    ch_lds4(tab.inv + QP_CK(c + h, C - 3), inv);
 #pragma unroll
                     for (int i = 0; i < 4; ++i) cd[h + i] = qp_code(e[j][h + i], lo[i], hi[i], inv[i], mask);
                 }
@@ -355,7 +357,7 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
                     for (int i = 0; i < EPV; ++i) cd[i] = el + i < n ? cd[i] : 0u;
                 }
 #pragma unroll
-                for (int i = 0; i < EPV; i += 2) codes[ch_code_word(le + i)] = cd[i] | (cd[i + 1] << 16);
+                for (int i = 0; i < EPV; i += 2) codes[QP_CK(ch_code_word(le + i), CH_STAGE_WORDS)] = cd[i] | (cd[i + 1] << 16);
                 c += cstep;
                 if (c >= C) c -= C;
             }
@@ -486,8 +488,8 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
                 const uint32_t a = codes[ch_code_word(le)], b = codes[ch_code_word(le + 2)];
                 const unsigned cd[4] = {a & 0xFFFFu, a >> 16, b & 0xFFFFu, b >> 16};
                 float v[4], lo[4], sc[4];
-                ch_lds4(tab.lo + c, lo);
-                ch_lds4(tab.scale + c, sc);
+                ch_lds4(tab.lo + QP_CK(c, C - 3), lo);
+                ch_lds4(tab.scale + QP_CK(c, C - 3), sc);
 #pragma unroll
                 for (int i = 0; i < 4; ++i) v[i] = fmaf(ch_code_to_float(cd[i]), sc[i], lo[i]);
                 if (el + 4 <= n) {

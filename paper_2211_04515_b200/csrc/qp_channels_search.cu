@@ -17,6 +17,8 @@
 
 #include "qp_internal.cuh"
 
+QP_CK_UNIT
+
 namespace {
 
 constexpr int CK = QP_EVAL_K;                       // candidates per thread
@@ -56,7 +58,7 @@ __global__ void __launch_bounds__(256) ch_hist_kernel(const T* __restrict__ x, u
                 if (!qp_is_finite(e)) continue;
                 int b = __float2int_rz(__fmul_rn(__fsub_rn(e, fmn), inv_w));
                 b = min(max(b, 0), nb - 1);
-                atomicAdd(&mine[b], 1u);
+                atomicAdd(&mine[QP_CK(b, nb)], 1u);
             }
         }
     }

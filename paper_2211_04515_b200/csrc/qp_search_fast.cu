@@ -25,6 +25,8 @@
 
 #include "qp_internal.cuh"
 
+QP_CK_UNIT
+
 namespace {
 
 constexpr int G = QP_IV_CELLS;
@@ -296,12 +298,13 @@ __device__ __forceinline__ void iv_one(float x, const IvShared& sh, const IvCons
         b.s1 += e; b.s1a += fabsf(e); b.s2 = fmaf(e, e, b.s2);
         x = xc;
         const float pm = cell_pm(x, k.g_lo, k.inv_gw);
-        const unsigned ci = sh.cell[__float_as_uint(pm) & 0x7FFFFFu];
+        const unsigned ci = sh.cell[QP_CK(__float_as_uint(pm) & 0x7FFFFFu, G + 1)];
         unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
         while (lo < hi) {                                   // largest i in [lo, hi] with bb[i] <= x
             const unsigned mid = (lo + hi + 1u) >> 1;
-            if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
+            if (sh.bb[QP_CK(mid, MAXB + 1)] <= x) lo = mid; else hi = mid - 1u;
         }
+        lo = QP_CK(lo, MAXB + 1);
         // offset in units of u, rounded to an integer by the same 2^23 trick (u is a power of two,
         // so the product is exact and the only rounding is the one to the integer)
         const float dm = fmaf(__fsub_rn(x, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
@@ -453,12 +456,13 @@ struct Iv2Shared {
 __device__ __forceinline__ void iv2_exact(float x, const IvShared& sh, const IvConst& k)
 {
     const float pm = cell_pm(x, k.g_lo, k.inv_gw);
-    const unsigned ci = sh.cell[__float_as_uint(pm) & 0x7FFFFFu];
+    const unsigned ci = sh.cell[QP_CK(__float_as_uint(pm) & 0x7FFFFFu, G + 1)];
     unsigned lo = ci & 0xFFFFu, hi = ci >> 16;
     while (lo < hi) {                                   // largest i in [lo, hi] with bb[i] <= x
         const unsigned mid = (lo + hi + 1u) >> 1;
-        if (sh.bb[mid] <= x) lo = mid; else hi = mid - 1u;
+        if (sh.bb[QP_CK(mid, MAXB + 1)] <= x) lo = mid; else hi = mid - 1u;
     }
+    lo = QP_CK(lo, MAXB + 1);
     const float dm = fmaf(__fsub_rn(x, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
     const unsigned d1 = __float_as_uint(dm) & 0x7FFFFFu;
     atomicAdd(&sh.cnt[lo], 1u);
@@ -485,14 +489,14 @@ __device__ __forceinline__ void iv2_one(float x, const IvShared& sh, const Iv2Sh
         const float dm = fmaf(__fsub_rn(xc, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
         const float d1f = __fsub_rn(dm, IV_MAGIC);
         b.s2_in = fmaf(d1f, d1f, b.s2_in);
-        const unsigned idx = ((__float_as_uint(pm) & 0x7FFFFFu) << IV2_RS) + (lane & (IV2_R - 1u));
+        const unsigned idx = QP_CK(((__float_as_uint(pm) & 0x7FFFFFu) << IV2_RS) + (lane & (IV2_R - 1u)), (G + 1) * IV2_R);
         const unsigned old = atomicAdd(&s2.rcnt[idx], 1u);
         atomicAdd(&s2.rs1[idx], __float_as_uint(dm) & 0x7FFFFFu);     // ignored later if the cell is split
         split = (old & IV2_SPLIT) != 0u;
     }
     const unsigned m = __ballot_sync(full, split);
     if (m) {                                             // warp-uniform
-        if (split) my_stage[staged + __popc(m & ((1u << lane) - 1u))] = xc;
+        if (split) my_stage[QP_CK(staged + __popc(m & ((1u << lane) - 1u)), IV2_STAGE)] = xc;
         staged += __popc(m);
         if (staged >= 32u) {
             __syncwarp();
@@ -796,9 +800,9 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
     constexpr size_t smem = (size_t)(MAXB + 1) * (8 + 4) + (size_t)(G + 1) * 4 + 16;
     if (cudaFuncSetAttribute(iv_moments_kernel<T>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return qp_check_launch(ctx, "qp_dsaciq_search (interval shared memory)");
+    unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]
     iv_bounds_kernel<<<MAXB / 256, 256, 0, s>>>(d_stats, ctx->d_hist, nb, bits, bmode, steps, F, ctx->d_cand, ctx->d_valid,
                                                 ctx->d_setup, ctx->d_iv_bnd, ctx->d_status);
-    unsigned* g_m = ctx->d_iv_first + G + 2;                 // behind first[0..G+1]
     iv_rank_kernel<<<MAXB / IV_RANK_PER_BLOCK, 512, 0, s>>>(ctx->d_iv_bnd, ctx->d_setup, ncand * L1, ctx->d_iv_bb,
                                                             ctx->d_iv_first);
     // second form where its 32-bit replica sums cannot wrap: one block per SM, more for longer tensors
@@ -818,13 +822,11 @@ int32_t interval_typed(qp_ctx* ctx, const T* x, uint64_t n, const qp_stats_t* d_
         iv_moments_kernel<T><<<blocks, QP_IV_THREADS, smem, s>>>(x, n, d_stats, ctx->d_setup, ctx->d_iv_bb, ctx->d_iv_first,
                                                                  g_m, ctx->d_iv_part, ctx->d_iv_outer);
     }
-    iv_reduce_kernel<<<(MAXB + 1 + 31) / 32, IV_RED_THREADS, 0, s>>>(ctx->d_iv_part, blocks, g_m, ctx->d_iv_tot,
-                                                                    ctx->d_iv_outer,
+    iv_reduce_kernel<<<(MAXB + 1 + 31) / 32, IV_RED_THREADS, 0, s>>>(ctx->d_iv_part, blocks, g_m, ctx->d_iv_tot, ctx->d_iv_outer,
                                                                     ctx->d_iv_outer + (size_t)blocks * 8);
-    iv_curve_kernel<<<ncand, IV_CURVE_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, g_m,
-                                                       ctx->d_iv_outer + (size_t)blocks * 8, ctx->d_cand, ctx->d_valid,
-                                                       bits, steps, nb, ctx->d_setup, ctx->d_curve, ctx->d_ticket + 2,
-                                                       d_out, d_qp_out, ctx->d_status);
+    iv_curve_kernel<<<ncand, IV_CURVE_THREADS, 0, s>>>(ctx->d_iv_tot, ctx->d_iv_bb, g_m, ctx->d_iv_outer + (size_t)blocks * 8,
+                                                       ctx->d_cand, ctx->d_valid, bits, steps, nb, ctx->d_setup, ctx->d_curve,
+                                                       ctx->d_ticket + 2, d_out, d_qp_out, ctx->d_status);
     ctx->launches += 5;
     return qp_check_launch(ctx, "qp_dsaciq_search (interval path)");
 }

@@ -25,6 +25,8 @@
 #include "qp_gridbar.cuh"
 #include "qp_internal.cuh"
 
+QP_CK_UNIT
+
 namespace {
 
 constexpr int FS_THREADS = 512;
@@ -148,7 +150,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
                 const int v = v0 + u * FS_THREADS;
                 if (v >= nvec) break;
                 const int i0 = v * EPV;                       // EPV consecutive elements stay inside one 32-element row
-                float* dst = xs + i0 + (i0 >> 5);
+                float* dst = xs + QP_CK(i0 + (i0 >> 5), (int)a.groups_per_block * 33 - (EPV - 1));
                 float ps = 0.f, psa = 0.f, pmn = finf, pmx = -finf;
 #pragma unroll
                 for (int i = 0; i < EPV; ++i) {
@@ -172,7 +174,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
         }
         for (int i = nvec * EPV + tid; i < cnt; i += FS_THREADS) {   // unaligned slice, ragged end
             const float v = qp_load_one(xb + i);
-            xs[i + (i >> 5)] = v;
+            xs[QP_CK(i + (i >> 5), (int)a.groups_per_block * 33)] = v;
             one(v);
         }
         fs_reduce<0, 0, 1, 2, 0>(v5, s_red);
@@ -230,7 +232,7 @@ __global__ void __launch_bounds__(FS_THREADS, 1) sender_fused_kernel(const FsArg
                     // bin = floor((x - min) * inv_w), the last bin closed; fp32, each op rounded once
                     int b = __float2int_rz(__fmul_rn(__fsub_rn(v, h_mn), inv_w));
                     b = min(max(b, 0), a.nb - 1);
-                    atomicAdd(&s_hist[b], 1u);
+                    atomicAdd(&s_hist[QP_CK(b, FS_MAX_BINS)], 1u);
                 }
             }
             v2[0] += (double)d1;

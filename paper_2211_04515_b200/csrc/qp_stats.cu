@@ -14,6 +14,8 @@
 #include "qp_internal.cuh"
 #include "qp_stream.cuh"
 
+QP_CK_UNIT
+
 namespace {
 
 constexpr int UNROLL = 4;   // 16-byte loads in flight per thread
@@ -391,7 +393,7 @@ __global__ void __launch_bounds__(QP_THREADS) stats_stream_b(const T* __restrict
                 d2 = fmaf(d, d, d2);
                 if (HIST) {      // x >= min, so the position is never negative; an empty range gives bin 0
                     const int b = min(__float2int_rz(__fmul_rn(__fsub_rn(e, mn), inv_w)), top_bin);
-                    atomicAdd(&my_hist[b << rep_shift], 1u);
+                    atomicAdd(&my_hist[QP_CK(b << rep_shift, nb << rep_shift)], 1u);
                 }
             }
         };
@@ -702,7 +704,7 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
                         // (conversions issue at a quarter of the rate of an addition).
                         const float pos = fminf(__fmul_rn(__fsub_rn(e, fmn), inv_w), top_bin);
                         const unsigned b = __float_as_uint(__fadd_rd(pos, 8388608.0f)) & 0x7FFFFFu;
-                        atomicAdd(&my_hist[b << rep_shift], 1u);
+                        atomicAdd(&my_hist[QP_CK(b << rep_shift, (unsigned)a.nb << rep_shift)], 1u);
                     }
                 }
             };

@@ -36,3 +36,29 @@ def load_hand_examples():
 @pytest.fixture(scope="session")
 def hand_examples():
     return load_hand_examples()
+
+
+_INDEX_CHECK_REPORT = []
+
+
+def pytest_terminal_summary(terminalreporter):
+    for line in _INDEX_CHECK_REPORT:
+        terminalreporter.write_line(line)
+
+
+@pytest.fixture(scope="session", autouse=True)
+def index_checked_build_reports_clean(request):
+    """When the tests run against the library built with index checks (QUANTPIPE_LIB points at it), the
+    session ends by reading the status once more: no index may have been out of range."""
+    yield
+    if not os.environ.get("QUANTPIPE_LIB"):
+        return
+    import torch
+    if not torch.cuda.is_available():
+        return
+    import paper_2211_04515_b200 as qp
+    assert qp.qp_built_with_index_checks()
+    c = qp.Context(0)
+    assert c.qp_get_status() & qp.QP_DEV_INDEX_RANGE == 0
+    c.close()
+    _INDEX_CHECK_REPORT.append("index checks: on, no index out of range")
