@@ -502,29 +502,39 @@ int32_t launch_streamed(qp_ctx* ctx, const T* x, uint64_t n, uint64_t ntiles, in
 // ---------------------------------------------------------------------------------------
 // Both passes in ONE cooperative launch (one block per SM).  What the two streamed kernels
 // spend twice - a launch, the start of the copy ring, a last-block merge - is spent once, and
-// the second pass reads less: the ring is as large as shared memory allows (6 stages of 32 KB),
-// every block keeps the last tiles of its first pass in it, and the second pass, which walks the
-// block's tiles in the opposite order, starts on those resident tiles and fetches only the rest
-// (all SMs together hold ~28 MB, so a 129 MB tensor costs 129 + 101 MB of reads instead of 258,
-// and one that fits is read once).
+// the second pass reads less: every warp keeps the last tile of its first pass in shared memory,
+// and the second pass, which walks the warp's tiles in the opposite order, starts on that
+// resident tile and fetches only the rest (all SMs together hold ~19 MB; with what L2 still holds
+// of the tensor's end, a 129 MB tensor costs ~173 MB of DRAM reads instead of 258, and one that
+// fits in L2 is read once).
 //
-//   pass A    tiles b, b + G, ... of block b through the ring: sum x, sum |x|, min, max, non-finite
+// Every warp has a ring of its own (qp_stream::warp_ring): the tile loops hold no block barrier,
+// a warp refills its stage as soon as its lanes have the tile in registers, and a lane works on
+// 64 elements per tile in four independent chains per sum.  Measured on a 129 MB tensor: fewer
+// and larger tiles beat more stages (16 warps x 1 stage of 8 KB: 43.6 us; 3 stages of 4 KB: 45.3;
+// 6 stages of 2 KB: 51.7; 32 warps x 3 x 2 KB: 57.0), because the work per tile outside the sums
+// (wait, address, refill, the fp64 adds) is what the issue slots go to; the block-wide ring of 6 x 32 KB
+// with two block barriers per tile that came before took 53 us.
+//
+//   pass A    warp w of block b takes 8 KB tiles 16 b + w, + 16 G, ...: sum x, sum |x|, min, max, non-finite
 //   barrier   grid-wide (bounded); every block merges the G partials in index order: same mean everywhere
 //   pass B    the same tiles backwards: sum |x - mean|, sum (x - mean)^2, histogram over [min, max]
 //   exit      every block counts itself out; the last one merges pass B's partials, takes the
 //             histogram's peak, writes the statistics and leaves the barrier scratch at zero
 //
-// A block whose wait runs out (tile copy or barrier) raises the abort flag beside the barrier
-// counter and QP_DEV_STREAM_TIMEOUT in the status word, waits for its own copies in flight, and
-// still arrives at the barrier and counts itself out, so nobody waits for it and the scratch is
-// clean afterwards; no statistics are written then.
+// A warp whose wait runs out flags its block; the block then (after its loops) raises the abort
+// flag beside the barrier counter and QP_DEV_STREAM_TIMEOUT in the status word, every warp waits
+// for its own copies in flight, and the block still arrives at the barrier and counts itself out,
+// so nobody waits for it and the scratch is clean afterwards; no statistics are written then.
 constexpr int SF_THREADS = 512;
-constexpr int SF_TILE = 32768;
-constexpr int SF_STAGES = 6;
+constexpr int SF_WARPS = SF_THREADS / 32;
+constexpr int SF_TILE = 8192;                     // bytes of one warp's tile
+constexpr int SF_STAGES = 1;
+constexpr int SF_VPT = SF_TILE / 16 / 32;         // 16-byte vectors per lane and tile (16)
 
 struct SfArgs {
     const void* x;
-    uint64_t n, ntiles;
+    uint64_t n, ntiles;                           // ntiles: whole SF_TILE-byte tiles
     qp_stats_partial* part;                       // [2 * grid]: pass A, then pass B
     qp_stats_t* out;
     unsigned* status;
@@ -535,79 +545,86 @@ struct SfArgs {
     unsigned spin_limit, bar_extra;
 };
 
+// element k of a 16-byte vector held as four words
+template <typename T>
+__device__ __forceinline__ float sf_elem(const uint4& v, int k)
+{
+    if constexpr (sizeof(T) == 4) {
+        return __uint_as_float(k == 0 ? v.x : k == 1 ? v.y : k == 2 ? v.z : v.w);
+    } else {
+        const unsigned w = (k >> 1) == 0 ? v.x : (k >> 1) == 1 ? v.y : (k >> 1) == 2 ? v.z : v.w;
+        return __uint_as_float((k & 1) ? (w & 0xFFFF0000u) : (w << 16));
+    }
+}
+
 template <typename T, bool HIST>
 __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs a)
 {
     extern __shared__ __align__(128) unsigned char smem[];
     constexpr int EPV = qp_span<T>::EPV;
-    constexpr int VPT = SF_TILE / 16 / SF_THREADS;           // 16-byte vectors per thread and tile (4)
-    using Ring = qp_stream::ring<SF_TILE, SF_STAGES>;
+    using Ring = qp_stream::warp_ring<SF_TILE, SF_STAGES>;
     __shared__ double sh[SF_THREADS / 32];
     __shared__ int s_flag, s_ok;
     __shared__ bool s_last;
     __shared__ double s_mean, s_mean_abs, s_mn, s_mx;
     __shared__ unsigned long long s_bad;
-    unsigned* sh_hist = reinterpret_cast<unsigned*>(smem + qp_stream::ring_bytes<SF_TILE, SF_STAGES>());
+    unsigned* sh_hist = reinterpret_cast<unsigned*>(smem + Ring::bytes(SF_WARPS));
     const T* x = static_cast<const T*>(a.x);
     const unsigned char* base = static_cast<const unsigned char*>(a.x);
-    const uint64_t G = gridDim.x, first = blockIdx.x;
-    const uint64_t m = first < a.ntiles ? (a.ntiles - first + G - 1) / G : 0;     // tiles of this block
+    const int lane = threadIdx.x & 31;
+    const uint64_t G = gridDim.x;
+    const uint64_t GW = G * SF_WARPS, first = (uint64_t)blockIdx.x * SF_WARPS + (threadIdx.x >> 5);
+    const uint64_t m = first < a.ntiles ? (a.ntiles - first + GW - 1) / GW : 0;   // tiles of this warp
     const float inf = __int_as_float(0x7F800000);
-    auto tile_src = [&](uint64_t i) { return base + (first + i * G) * (uint64_t)SF_TILE; };
-
+    auto tile_src = [&](uint64_t i) { return base + (first + i * GW) * (uint64_t)SF_TILE; };
     Ring ring;
     if (threadIdx.x == 0) s_flag = 0;
-    ring.init(smem);
-    unsigned pending = 0u;                                   // thread 0: stages with a copy in flight
+    ring.init(smem, SF_WARPS);
     bool ok = true;
 
     // ---- pass A
-    if (threadIdx.x == 0)
-        for (uint64_t i = 0; i < (uint64_t)SF_STAGES && i < m; ++i) {
-            ring.issue((int)i, tile_src(i));
-            pending |= 1u << i;
-        }
+    for (uint64_t i = 0; i < (uint64_t)SF_STAGES && i < m; ++i) ring.issue((int)i, tile_src(i));
     AccA acc = {0.0, 0.0, (double)inf, (double)-inf, 0ull};
     float tmn = inf, tmx = -inf;                             // exact in fp32: kept out of the fp64 path
-    for (uint64_t i = 0; i < m; ++i) {
-        const int s = (int)(i % SF_STAGES);
-        if (ring.wait(s, a.wait_limit)) { if (threadIdx.x == 0) pending &= ~(1u << s); }
-        else s_flag = 1;                                     // benign race: every writer writes 1
-        __syncthreads();
-        if (s_flag) { ok = false; break; }
-        const unsigned char* tile = ring.stage(s);
-        float e[VPT][EPV];
+    {
+        int s = 0;
+        for (uint64_t i = 0; i < m; ++i) {
+            if (!ring.wait(s, a.wait_limit)) { s_flag = 1; break; }      // benign race: every writer writes 1
+            const unsigned char* tile = ring.stage(s);
+            uint4 v[SF_VPT];
 #pragma unroll
-        for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * SF_THREADS + threadIdx.x) * 16, e[u]);
-        float ps = 0.f, psa = 0.f, pmn = inf, pmx = -inf;
+            for (int u = 0; u < SF_VPT; ++u) v[u] = *reinterpret_cast<const uint4*>(tile + (size_t)(u * 32 + lane) * 16);
+            __syncwarp();
+            if (i + SF_STAGES < m) ring.issue(s, tile_src(i + SF_STAGES));   // the last ones stay resident
+            float cs[4] = {0.f, 0.f, 0.f, 0.f}, ca[4] = {0.f, 0.f, 0.f, 0.f};
+            float cmn[4] = {inf, inf, inf, inf}, cmx[4] = {-inf, -inf, -inf, -inf};
 #pragma unroll
-        for (int u = 0; u < VPT; ++u)
+            for (int u = 0; u < SF_VPT; ++u)
 #pragma unroll
-            for (int k = 0; k < EPV; ++k) {
-                ps += e[u][k];
-                psa += fabsf(e[u][k]);
-                pmn = fminf(pmn, e[u][k]);
-                pmx = fmaxf(pmx, e[u][k]);
+                for (int k = 0; k < EPV; ++k) {
+                    const float e = sf_elem<T>(v[u], k);
+                    cs[k & 3] += e;
+                    ca[k & 3] += fabsf(e);
+                    cmn[k & 3] = fminf(cmn[k & 3], e);
+                    cmx[k & 3] = fmaxf(cmx[k & 3], e);
+                }
+            const float psa = (ca[0] + ca[1]) + (ca[2] + ca[3]);
+            if (psa < inf) {                                 // every element finite (and no fp32 overflow)
+                acc.s += (double)((cs[0] + cs[1]) + (cs[2] + cs[3]));
+                acc.sa += (double)psa;
+                tmn = fminf(tmn, fminf(fminf(cmn[0], cmn[1]), fminf(cmn[2], cmn[3])));
+                tmx = fmaxf(tmx, fmaxf(fmaxf(cmx[0], cmx[1]), fmaxf(cmx[2], cmx[3])));
+            } else {
+#pragma unroll
+                for (int u = 0; u < SF_VPT; ++u)
+#pragma unroll
+                    for (int k = 0; k < EPV; ++k) acc.add_scalar(sf_elem<T>(v[u], k));
             }
-        if (psa < inf) {                                     // every element finite (and no fp32 overflow)
-            acc.s += (double)ps;
-            acc.sa += (double)psa;
-            tmn = fminf(tmn, pmn);
-            tmx = fmaxf(tmx, pmx);
-        } else {
-#pragma unroll
-            for (int u = 0; u < VPT; ++u)
-#pragma unroll
-                for (int k = 0; k < EPV; ++k) acc.add_scalar(e[u][k]);
-        }
-        if (i + SF_STAGES < m) {                             // the stage is filled again; the last ones stay resident
-            __syncthreads();
-            if (threadIdx.x == 0) {
-                ring.issue(s, tile_src(i + SF_STAGES));
-                pending |= 1u << s;
-            }
+            s = s + 1 == SF_STAGES ? 0 : s + 1;
         }
     }
+    __syncthreads();
+    ok = s_flag == 0;
     if (ok) {
         acc.mn = fmin(acc.mn, (double)tmn);
         acc.mx = fmax(acc.mx, (double)tmx);
@@ -633,10 +650,8 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
         if (threadIdx.x == 0) {
             atomicOr(a.status, QP_DEV_STREAM_TIMEOUT);
             atomicExch(a.bar + 2, 1u);
-            for (int s = 0; s < SF_STAGES; ++s)
-                if (pending & (1u << s)) ring.wait(s, QP_STREAM_TIMEOUT_CYCLES);
-            pending = 0u;
         }
+        ring.drain();
         __syncthreads();
     };
     if (!ok) give_up();
@@ -671,7 +686,7 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
         __syncthreads();
     }
 
-    // ---- pass B: the same tiles backwards; tile i lives in stage i % SF_STAGES in both passes, so the
+    // ---- pass B: the warp's tiles backwards; tile i lives in stage i % SF_STAGES in both passes, so the
     // last SF_STAGES tiles of pass A are there already and each stage is refilled as it is consumed
     double sd = 0.0, sv = 0.0;
     if (ok) {
@@ -708,35 +723,27 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
                     }
                 }
             };
+            int s = m ? (int)((m - 1) % SF_STAGES) : 0;
             for (uint64_t j = 0; j < m; ++j) {
                 const uint64_t i = m - 1 - j;
-                const int s = (int)(i % SF_STAGES);
-                if (j >= (uint64_t)SF_STAGES) {                             // fetched in this pass
-                    if (ring.wait(s, a.wait_limit)) { if (threadIdx.x == 0) pending &= ~(1u << s); }
-                    else s_flag = 1;
-                    __syncthreads();
-                    if (s_flag) { ok = false; break; }
-                }
+                if (j >= (uint64_t)SF_STAGES && !ring.wait(s, a.wait_limit)) { s_flag = 1; break; }   // fetched in this pass
                 const unsigned char* tile = ring.stage(s);
-                float e[VPT][EPV];
+                uint4 v[SF_VPT];
 #pragma unroll
-                for (int u = 0; u < VPT; ++u) lds_vec<T>(tile + (size_t)(u * SF_THREADS + threadIdx.x) * 16, e[u]);
-                float d1 = 0.f, d2 = 0.f;
+                for (int u = 0; u < SF_VPT; ++u)
+                    v[u] = *reinterpret_cast<const uint4*>(tile + (size_t)(u * 32 + lane) * 16);
+                __syncwarp();
+                if (i >= (uint64_t)SF_STAGES) ring.issue(s, tile_src(i - SF_STAGES));
+                float c1[4] = {0.f, 0.f, 0.f, 0.f}, c2[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-                for (int u = 0; u < VPT; ++u)
+                for (int u = 0; u < SF_VPT; ++u)
 #pragma unroll
-                    for (int k = 0; k < EPV; ++k) one(e[u][k], d1, d2);
-                sd += (double)d1;
-                sv += (double)d2;
-                if (i >= (uint64_t)SF_STAGES) {
-                    __syncthreads();
-                    if (threadIdx.x == 0) {
-                        ring.issue(s, tile_src(i - SF_STAGES));
-                        pending |= 1u << s;
-                    }
-                }
+                    for (int k = 0; k < EPV; ++k) one(sf_elem<T>(v[u], k), c1[k & 3], c2[k & 3]);
+                sd += (double)((c1[0] + c1[1]) + (c1[2] + c1[3]));
+                sv += (double)((c2[0] + c2[1]) + (c2[2] + c2[3]));
+                s = s == 0 ? SF_STAGES - 1 : s - 1;
             }
-            if (ok && blockIdx.x == 0) {
+            if (blockIdx.x == 0) {
                 float d1 = 0.f, d2 = 0.f;
                 const uint64_t t0 = a.ntiles * (SF_TILE / sizeof(T));
                 for (uint64_t i = t0 + threadIdx.x; i < a.n; i += SF_THREADS) one(qp_load_one(x + i), d1, d2);
@@ -745,9 +752,10 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
             }
         };
         if (guard) run(std::true_type{}); else run(std::false_type{});
+        __syncthreads();
+        ok = s_flag == 0;
         if (!ok) give_up();
         if (ok && HIST) {
-            __syncthreads();
             const int reps = 1 << rep_shift;
             for (int b = threadIdx.x; b < a.nb; b += SF_THREADS) {
                 unsigned long long c = 0;
@@ -813,7 +821,7 @@ __global__ void __launch_bounds__(SF_THREADS, 1) stats_fused_kernel(const SfArgs
     }
 }
 
-constexpr size_t SF_RING_BYTES = qp_stream::ring_bytes<SF_TILE, SF_STAGES>();
+constexpr size_t SF_RING_BYTES = qp_stream::warp_ring<SF_TILE, SF_STAGES>::bytes(SF_WARPS);
 constexpr size_t SF_HIST_BYTES = 16 * 1024;
 
 // Whether this device can hold the one-launch statistics (checked once per context).
@@ -862,7 +870,8 @@ int32_t launch_fused(qp_ctx* ctx, const T* x, uint64_t n, int hist_bins, qp_stat
     a.wait_limit = ctx->wait_cycles;
     a.spin_limit = ctx->spin_limit;
     a.bar_extra = (unsigned)ctx->bar_extra;
-    const unsigned G = (unsigned)(a.ntiles < (uint64_t)ctx->sm_count ? a.ntiles : (uint64_t)ctx->sm_count);
+    const uint64_t want = (a.ntiles + SF_WARPS - 1) / SF_WARPS;                 // a tile per warp at least
+    const unsigned G = (unsigned)(want < (uint64_t)ctx->sm_count ? want : (uint64_t)ctx->sm_count);
     const size_t dyn = SF_RING_BYTES + (fuse ? SF_HIST_BYTES : 0);
     void* kernel = fuse ? (void*)stats_fused_kernel<T, true> : (void*)stats_fused_kernel<T, false>;
     void* params[] = {&a};

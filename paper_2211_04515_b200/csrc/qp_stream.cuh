@@ -213,4 +213,69 @@ struct ring {
     }
 };
 
+// A ring per WARP: every warp of the block streams its own sequence of tiles through its own
+// stages and barriers, so the tile loop holds no block barrier at all (a block-wide ring hands a
+// stage back through __syncthreads twice per tile, and with a few dozen instructions of work per
+// thread and tile the warps spend more time at that barrier than on the data).  Lane 0 issues the
+// warp's copies; all lanes wait (the outcome is made uniform with a vote) and __syncwarp hands a
+// stage back.  All lanes keep `parity` and `pending` alike.
+template <int TILE_BYTES, int STAGES>
+struct warp_ring {
+    static_assert(TILE_BYTES % 128 == 0 && STAGES <= 32, "ring shape");
+    unsigned char* buf;
+    uint64_t* full;
+    unsigned parity;                                    // bit s: parity of the next completion of stage s
+    unsigned pending;                                   // bit s: a copy into stage s is in flight
+
+    static __host__ __device__ constexpr size_t bytes(int warps) { return (size_t)warps * STAGES * (TILE_BYTES + 8); }
+
+    // all threads of the block; smem: 128-byte aligned, bytes(warps) long; ends with a block barrier
+    __device__ __forceinline__ void init(unsigned char* smem, int warps)
+    {
+        const int warp = threadIdx.x >> 5;
+        buf = smem + (size_t)warp * STAGES * TILE_BYTES;
+        full = reinterpret_cast<uint64_t*>(smem + (size_t)warps * STAGES * TILE_BYTES) + warp * STAGES;
+        parity = 0u;
+        pending = 0u;
+        if ((threadIdx.x & 31) == 0) {
+            for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
+            fence_barrier_init();
+        }
+        __syncthreads();
+    }
+    __device__ __forceinline__ const unsigned char* stage(int s) const { return buf + (size_t)s * TILE_BYTES; }
+    // all lanes (lane 0 copies); the stage's earlier contents must have been read (__syncwarp before)
+    __device__ __forceinline__ void issue(int s, const unsigned char* src)
+    {
+        if ((threadIdx.x & 31) == 0) {
+            mbar_arrive_expect_tx(&full[s], TILE_BYTES);
+            bulk_load(buf + (size_t)s * TILE_BYTES, src, TILE_BYTES, &full[s]);
+        }
+        pending |= 1u << s;
+    }
+    // all lanes; false for the whole warp when any lane's wait ran out (the state is then left as it was)
+    __device__ __forceinline__ bool wait(int s, long long limit)
+    {
+        const bool ok = mbar_wait(&full[s], (parity >> s) & 1u, limit);
+        if (!__all_sync(0xFFFFFFFFu, ok)) return false;
+        parity ^= 1u << s;
+        pending &= ~(1u << s);
+        return true;
+    }
+    // all lanes: a second, bounded wait for every copy still in flight (after a failed wait)
+    __device__ __forceinline__ void drain()
+    {
+        if ((threadIdx.x & 31) == 0)
+            for (int s = 0; s < STAGES; ++s)
+                if (pending & (1u << s)) mbar_wait(&full[s], (parity >> s) & 1u, QP_STREAM_TIMEOUT_CYCLES);
+        pending = 0u;
+        __syncwarp();
+    }
+    __device__ __forceinline__ void fini()                                          // after a block barrier
+    {
+        if ((threadIdx.x & 31) == 0)
+            for (int s = 0; s < STAGES; ++s) mbar_inval(&full[s]);
+    }
+};
+
 }  // namespace qp_stream
