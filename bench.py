@@ -269,7 +269,8 @@ def time_groups(torch, fn, nbuf, reps=20, warm=5, groups=5):
 
 def cold_kernels(torch, qp, ctx, x_host, hbm_peak, peak_kind):
     """The metric's two kernels alone and cold: quantize+pack and unpack+dequantize on the workload at
-    2, 4 and 8 bits, and on a 1 GiB tensor at 4 bits.  Consecutive launches use different input and
+    2, 4 and 8 bits, and on a 1 GiB tensor at 4 bits; on the workload also the statistics call (without and
+    with the histogram) and the search call at 1-4 bits.  Consecutive launches use different input and
     output buffers, rotating through more than 4x the L2 capacity (126 MB) between reuses, so no
     launch finds its lines in L2."""
     out = {}
@@ -281,11 +282,28 @@ def cold_kernels(torch, qp, ctx, x_host, hbm_peak, peak_kind):
                                "achieved": round(g, 1), "unit": "GB/s", "frac": round(g / hbm_peak, 4),
                                "peak": hbm_peak, "peak_kind": peak_kind, "frac_of_8000": round(g / 8000.0, 4)}
 
-    def run(tag, xh, rot, widths):
+    def read_row(name, n, ms):                                      # a stage whose algorithmic traffic is one read of x
+        g = 4.0 * n / (ms * 1e-3) / 1e9
+        out[name] = {"us": round(ms * 1e3, 2), "n": n, "achieved": round(g, 1), "unit": "GB/s",
+                     "frac": round(g / hbm_peak, 4), "peak": hbm_peak, "peak_kind": peak_kind}
+
+    def run(tag, xh, rot, widths, reductions=False):
         n = xh.numel()
         xs = [xh.cuda() for _ in range(rot)]
         ys = [torch.empty(n, dtype=torch.float32, device="cuda") for _ in range(rot)]
         st = ctx.read_stats(ctx.qp_stats(xs[0]))
+        if reductions:                                              # the statistics and the search call, alone too
+            nb = qp.QP_DEFAULT_HIST_BINS
+            d_st = [ctx.qp_stats(x, hist_bins=nb) for x in xs]
+            d_res = torch.empty(72, dtype=torch.uint8, device="cuda")
+            d_qp = torch.empty(24, dtype=torch.uint8, device="cuda")
+            read_row(f"{tag}stats", n, time_groups(torch, lambda i: ctx.qp_stats(xs[i], hist_bins=0, out=d_st[i]), rot))
+            read_row(f"{tag}stats+hist", n,
+                     time_groups(torch, lambda i: ctx.qp_stats(xs[i], hist_bins=nb, out=d_st[i]), rot))
+            for q in (1, 2, 3, 4):
+                read_row(f"{tag}clip@{q}b", n, time_groups(
+                    torch, lambda i: ctx.qp_dsaciq_search(xs[i], d_st[i], q, bmode=qp.QP_B_MAD | qp.QP_B_HIST_IN_STATS,
+                                                          out_result=d_res, out_qp=d_qp), rot))
         for q in widths:
             _, _, qp_h = qp.qp_aciq_alpha(st, q)
             pk = [torch.empty(qp.qp_packed_bytes(n, q), dtype=torch.uint8, device="cuda") for _ in range(rot)]
@@ -297,11 +315,12 @@ def cold_kernels(torch, qp, ctx, x_host, hbm_peak, peak_kind):
         del xs, ys
         torch.cuda.empty_cache()
 
-    run("", x_host, 5, (2, 4, 8))                                   # 5 x 129 MB in, 5 x 129 MB out
+    run("", x_host, 5, (2, 4, 8), reductions=True)                  # 5 x 129 MB in, 5 x 129 MB out
     big = torch.from_numpy(si.flat_iid(1 << 28, si.C5_SEED, "laplace"))
     run("2^28:", big, 2, (4,))                                       # every launch moves > 1 GiB: nothing survives in L2
     out["method"] = ("each kernel alone, buffers rotating through > 4x L2 between reuses; median per-launch time of 5 "
-                     "groups of 20 back-to-back launches after 5 warm-ups; achieved = (4 + q/8) n bytes / time")
+                     "groups of 20 back-to-back launches after 5 warm-ups; achieved = (4 + q/8) n bytes / time "
+                     "(stats, stats+hist, clip: 4 n bytes / time of the whole call, graph replay as in the step)")
     return out
 
 
@@ -693,6 +712,27 @@ def sweep_main(args):
                     emit(name, dtype, f"unpack_dequantize_channels[{channels}]", q, n, med, best, (4 + q / 8.0) * n)
                     del ysc
                 del pk
+            # token-wise variant (one quantizer per row of `channels` contiguous elements)
+            tokens = n // channels
+            d_tst = torch.empty(80 * tokens, dtype=torch.uint8, device="cuda")
+            med, best = timed(lambda i: ctx.qp_stats_tokens(xs[i], channels, out=d_tst), nb)
+            emit(name, dtype, f"stats_tokens[{tokens}]", 0, n, med, best, esz * n)
+            for q in (4, 8):
+                d_tqp = ctx.qp_clip_qparams_tokens_device(d_tst, tokens, q)
+                pk = rotating(lambda: torch.empty(qp.qp_packed_bytes(n, q), dtype=torch.uint8, device="cuda"),
+                              n * esz + qp.qp_packed_bytes(n, q))
+                npk = len(pk)
+                med, best = timed(lambda i: ctx.qp_quantize_pack_tokens(xs[i % nb], channels, q, d_tqp, out=pk[i % npk]),
+                                  max(nb, npk))
+                emit(name, dtype, f"quantize_pack_tokens[{tokens}]", q, n, med, best, (esz + q / 8.0) * n)
+                if dtype == "f32":
+                    yst = rotating(lambda: torch.empty(n, dtype=torch.float32, device="cuda"), 4 * n)
+                    nyt = len(yst)
+                    med, best = timed(lambda i: ctx.qp_unpack_dequantize_tokens(pk[i % npk], tokens, channels, q, d_tqp,
+                                                                                out=yst[i % nyt]), max(nyt, npk))
+                    emit(name, dtype, f"unpack_dequantize_tokens[{tokens}]", q, n, med, best, (4 + q / 8.0) * n)
+                    del yst
+                del pk
         ys = None
         for q in bits_list:
             rc, alpha, qp_h = qp.qp_aciq_alpha(st, q)
@@ -711,11 +751,16 @@ def sweep_main(args):
         del xs, ys
         torch.cuda.empty_cache()
 
+    only = set(args.sweep_only.split(",")) if args.sweep_only else None
     for name in ("c1", "c2", "c3", "c4"):
+        if only is not None and name not in only:
+            continue
         cfg = si.CONFIGS[name]
         x = torch.from_numpy(si.config_tensor(name).reshape(-1))
         run_workload(name, x, cfg["bits"], "f32", [b for b in cfg["bits"] if b <= 4][:2], channels=cfg["shape"][-1])
     for log2n in range(18, args.sweep_max_log2 + 1, 2):
+        if only is not None and f"2^{log2n}" not in only:
+            continue
         for dist in ("laplace", "normal"):
             if dist == "normal" and log2n not in (22, 26):
                 continue
@@ -787,6 +832,8 @@ def main():
                     help="print the quantization MSE of every clip method on the ViT-shaped configs (one GPU)")
     ap.add_argument("--sweep", action="store_true",
                     help="kernel-by-kernel cold-cache table over the configurations (one JSON line per row)")
+    ap.add_argument("--sweep-only", default="",
+                    help="comma-separated workloads of the sweep to run (c1..c4, 2^18..2^28); default: all")
     ap.add_argument("--sweep-max-log2", type=int, default=28)
     args = ap.parse_args()
     if args.warmup < 3:

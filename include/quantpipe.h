@@ -328,8 +328,12 @@ int32_t qp_policy_use_ds(int bits);
  * bits zero.  `qp` is a host pointer (qp_on_device = 0, read before returning) or a
  * device pointer (qp_on_device = 1, read by the kernel; its bits must equal `bits`,
  * otherwise QP_DEV_BITS_MISMATCH is raised in the status word).
- * d_packed must be 16-byte aligned; d_x aligned to its element size (16-byte alignment
- * enables the fast path).
+ * d_packed must be 16-byte aligned; d_x aligned to its element size.  Only a 16-byte aligned d_x
+ * takes the warp-tile kernel; an x that is merely element-aligned (a view that starts at an odd
+ * element) sends the WHOLE tensor through the scalar kernel (a thread per 32 elements, 4-byte
+ * loads): the same bytes, about 5x the time (129 MB tensor on B200: 153-162 us against 33-35 us).
+ * Copy such a view to an aligned buffer first if speed matters.  The same holds for d_y of
+ * qp_unpack_dequantize (179 us against 31-34 us); qp_stats loses less (66 us against 46 us).
  * Errors: QP_ERR_INVALID_ARG, QP_ERR_UNSUPPORTED_BITS, QP_ERR_UNSUPPORTED_DTYPE,
  * QP_ERR_BUFFER_TOO_SMALL (packed_capacity < qp_packed_bytes), QP_ERR_ALIGNMENT, QP_ERR_CUDA. */
 int32_t qp_quantize_pack(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int bits,

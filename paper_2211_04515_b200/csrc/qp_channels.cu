@@ -309,8 +309,10 @@ template <typename T, bool VEC, int BITS>
 __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict__ x, uint64_t n, uint32_t C, int bits_rt,
                                                              const qp_qparams_t* __restrict__ d_qp,
                                                              uint32_t* __restrict__ out, uint64_t total_words,
-                                                             uint64_t ntiles, unsigned* __restrict__ status)
+                                                             uint64_t ntiles, uint64_t el0, unsigned* __restrict__ status)
 {
+    // x, n, out, total_words and ntiles describe the part of the tensor this launch packs; el0 = index of
+    // x[0] in the whole tensor (a multiple of the warp tile), which fixes the channel of every element
     extern __shared__ __align__(16) unsigned char raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int bits = BITS ? BITS : bits_rt;
@@ -337,7 +339,7 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
                     for (int i = 0; i < EPV; ++i) e[j][i] = el + i < n ? qp_load_one(x + el + i) : 0.f;
                 }
             }
-            uint32_t c = (uint32_t)((base + (uint64_t)lane * EPV) % C);
+            uint32_t c = (uint32_t)((el0 + base + (uint64_t)lane * EPV) % C);
 #pragma unroll
             for (int j = 0; j < NV; ++j) {
                 const int le = (j * 32 + lane) * EPV;
@@ -368,7 +370,7 @@ __global__ void __launch_bounds__(CH_THREADS) ch_pack_kernel(const T* __restrict
                 const uint64_t el = base + le;
                 unsigned cd = 0u;
                 if (el < n) {
-                    const uint32_t c = (uint32_t)(el % C);
+                    const uint32_t c = (uint32_t)((el0 + el) % C);
                     cd = qp_code(qp_load_one(x + el), tab.lo[c], tab.hi[c], tab.inv[c], mask);
                 }
                 ch[le + ((le >> 5) << 1)] = (unsigned short)cd;
@@ -409,14 +411,14 @@ __device__ __forceinline__ float ch_code_to_float(unsigned c) { return __fsub_rn
 
 __device__ __forceinline__ void ch_store4(float* y, uint64_t el, const float (&v)[4])
 {
-    *reinterpret_cast<float4*>(y + el) = make_float4(v[0], v[1], v[2], v[3]);
+    __stcs(reinterpret_cast<float4*>(y + el), make_float4(v[0], v[1], v[2], v[3]));   // streaming: not read again here
 }
 __device__ __forceinline__ void ch_store4(unsigned short* y, uint64_t el, const float (&v)[4])
 {
     uint2 o;
     o.x = (unsigned)qp_f32_to_bf16(v[0]) | ((unsigned)qp_f32_to_bf16(v[1]) << 16);
     o.y = (unsigned)qp_f32_to_bf16(v[2]) | ((unsigned)qp_f32_to_bf16(v[3]) << 16);
-    *reinterpret_cast<uint2*>(y + el) = o;
+    __stcs(reinterpret_cast<uint2*>(y + el), o);
 }
 __device__ __forceinline__ void ch_store1(float* y, uint64_t el, float v) { y[el] = v; }
 __device__ __forceinline__ void ch_store1(unsigned short* y, uint64_t el, float v) { y[el] = qp_f32_to_bf16(v); }
@@ -425,8 +427,9 @@ template <typename TO, bool VEC, int BITS>
 __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* __restrict__ in, uint64_t n, uint32_t C,
                                                                int bits_rt, const qp_qparams_t* __restrict__ d_qp,
                                                                TO* __restrict__ y, uint64_t total_words, uint64_t ntiles,
-                                                               unsigned* __restrict__ status)
+                                                               uint64_t el0, unsigned* __restrict__ status)
 {
+    // in, n, y, total_words, ntiles: the part this launch unpacks; el0 = index of y[0] in the whole tensor
     extern __shared__ __align__(16) unsigned char raw[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int bits = BITS ? BITS : bits_rt;
@@ -480,7 +483,7 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
         }
         __syncwarp();
         if (VEC) {
-            uint32_t c = (uint32_t)((base + (uint64_t)lane * 4) % C);
+            uint32_t c = (uint32_t)((el0 + base + (uint64_t)lane * 4) % C);
 #pragma unroll
             for (int j = 0; j < CH_WTILE / 128; ++j) {
                 const int le = (j * 32 + lane) * 4;
@@ -508,10 +511,139 @@ __global__ void __launch_bounds__(CH_THREADS) ch_unpack_kernel(const uint32_t* _
                 const int le = k * 32 + lane;
                 const uint64_t el = base + le;
                 if (el < n) {
-                    const uint32_t c = (uint32_t)(el % C);
+                    const uint32_t c = (uint32_t)((el0 + el) % C);
                     ch_store1(y, el, fmaf(ch_code_to_float(ch[le + ((le >> 5) << 1)]), tab.scale[c], tab.lo[c]));
                 }
             }
+        }
+        __syncwarp();
+    }
+}
+
+// ---- whole warp tiles on the fast path (aligned tensor, channels a multiple of the vector, 1..8 bits)
+//
+// The per-tensor packer's warp tile (1024 elements = 32 * BITS words: coalesced 16-byte loads, four codes
+// to a "quad", quads across the warp through a swizzled 1 KB buffer, a lane then owns 32 consecutive
+// elements = BITS words, coalesced word stores) with the quantizers of a vector's four channels read
+// from the shared table as one 16-byte vector per array.  The staging of 16-bit codes and the
+// element-by-element bit assembly of the generic kernel above took it to 0.6 of the copy peak; the
+// generic kernel keeps the last partial tile, 16 bits and the unaligned shapes.
+__device__ __forceinline__ int ch_swz(int p) { return ((((p >> 2) ^ ((p >> 5) & 1)) << 2) | (p & 3)); }
+
+template <int BITS, typename T>
+__global__ void __launch_bounds__(CH_THREADS) ch_pack_fast(const T* __restrict__ x, uint64_t ntiles, uint32_t C,
+                                                           const qp_qparams_t* __restrict__ d_qp,
+                                                           uint32_t* __restrict__ out, unsigned* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char raw[];
+    constexpr int EPV = qp_span<T>::EPV;
+    constexpr int NLOAD = CH_WTILE / (32 * EPV);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* sw = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)) + warp * 256;
+    const ChTable tab = ch_load_table(d_qp, C, BITS, reinterpret_cast<float*>(raw), status);
+    __syncthreads();
+    constexpr unsigned mask = (1u << BITS) - 1u;
+    const uint32_t cstep = (uint32_t)((32u * EPV) % C);        // channel advance from one of a lane's vectors to the next
+    const uint64_t wstride = (uint64_t)gridDim.x * CH_WARPS;
+    for (uint64_t tile = (uint64_t)blockIdx.x * CH_WARPS + warp; tile < ntiles; tile += wstride) {
+        const T* xt = x + tile * CH_WTILE;
+        float e[NLOAD][EPV];
+#pragma unroll
+        for (int j = 0; j < NLOAD; ++j) qp_load_vec(xt + (j * 32 + lane) * EPV, e[j]);
+        uint32_t c = (uint32_t)((tile * CH_WTILE + (uint64_t)lane * EPV) % C);
+#pragma unroll
+        for (int j = 0; j < NLOAD; ++j) {
+            unsigned quads[EPV / 4];
+#pragma unroll
+            for (int h = 0; h < EPV / 4; ++h) {                  // EPV divides C: the vector stays in one row
+                float lo[4], hi[4], inv[4];
+                ch_lds4(tab.lo + QP_CK(c + 4 * h, C - 3), lo);
+                ch_lds4(tab.hi + QP_CK(c + 4 * h, C - 3), hi);
+                ch_lds4(tab.inv + QP_CK(c + 4 * h, C - 3), inv);
+                unsigned r = 0;
+#pragma unroll
+                for (int i = 0; i < 4; ++i) r |= qp_code(e[j][4 * h + i], lo[i], hi[i], inv[i], mask) << (BITS * i);
+                quads[h] = r;
+            }
+            if constexpr (EPV == 4) sw[ch_swz(j * 32 + lane)] = quads[0];
+            else *reinterpret_cast<uint2*>(&sw[ch_swz(2 * (j * 32 + lane))]) = make_uint2(quads[0], quads[1]);
+            c += cstep;
+            if (c >= C) c -= C;
+        }
+        __syncwarp();
+        const uint4 a = *reinterpret_cast<const uint4*>(&sw[ch_swz(8 * lane)]);
+        const uint4 b = *reinterpret_cast<const uint4*>(&sw[ch_swz(8 * lane + 4)]);
+        const uint32_t qd[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+        uint32_t w[BITS];
+#pragma unroll
+        for (int m = 0; m < BITS; ++m) w[m] = 0u;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            constexpr int QB = 4 * BITS;
+            const int bit = QB * k, word = bit >> 5, sh = bit & 31;
+            w[word] |= qd[k] << sh;
+            if (sh + QB > 32) w[(word + 1) % BITS] |= qd[k] >> (32 - sh);
+        }
+        uint32_t* ot = out + tile * (32 * BITS);
+        __syncwarp();
+#pragma unroll
+        for (int m = 0; m < BITS; ++m) sw[lane * BITS + m] = w[m];
+        __syncwarp();
+#pragma unroll
+        for (int m = 0; m < BITS; ++m) ot[m * 32 + lane] = sw[m * 32 + lane];
+        __syncwarp();
+    }
+}
+
+template <int BITS, typename TO>
+__global__ void __launch_bounds__(CH_THREADS) ch_unpack_fast(const uint32_t* __restrict__ in, uint64_t ntiles, uint32_t C,
+                                                             const qp_qparams_t* __restrict__ d_qp, TO* __restrict__ y,
+                                                             unsigned* __restrict__ status)
+{
+    extern __shared__ __align__(16) unsigned char raw[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    uint32_t* sw = reinterpret_cast<uint32_t*>(raw + (size_t)C * sizeof(float4)) + warp * 256;
+    const ChTable tab = ch_load_table(d_qp, C, BITS, reinterpret_cast<float*>(raw), status);
+    __syncthreads();
+    constexpr unsigned MASK = (1u << BITS) - 1u;
+    constexpr int QB = 4 * BITS;
+    constexpr unsigned QMASK = QB >= 32 ? 0xFFFFFFFFu : ((1u << (QB & 31)) - 1u);
+    const uint32_t cstep = (uint32_t)(128u % C);               // a lane's vectors of 4 are 128 elements apart
+    const uint64_t wstride = (uint64_t)gridDim.x * CH_WARPS;
+    for (uint64_t tile = (uint64_t)blockIdx.x * CH_WARPS + warp; tile < ntiles; tile += wstride) {
+        const uint32_t* it = in + tile * (32 * BITS);
+        uint32_t w[BITS];
+#pragma unroll
+        for (int m = 0; m < BITS; ++m) sw[m * 32 + lane] = __ldg(it + m * 32 + lane);
+        __syncwarp();
+#pragma unroll
+        for (int m = 0; m < BITS; ++m) w[m] = sw[lane * BITS + m];
+        __syncwarp();
+        uint32_t qd[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) {
+            const int bit = QB * k, word = bit >> 5, sh = bit & 31;
+            uint32_t v = w[word] >> sh;
+            if (sh + QB > 32) v |= w[(word + 1) % BITS] << (32 - sh);
+            qd[k] = v & QMASK;
+        }
+        *reinterpret_cast<uint4*>(&sw[ch_swz(8 * lane)]) = make_uint4(qd[0], qd[1], qd[2], qd[3]);
+        *reinterpret_cast<uint4*>(&sw[ch_swz(8 * lane + 4)]) = make_uint4(qd[4], qd[5], qd[6], qd[7]);
+        __syncwarp();
+        uint32_t mine[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) mine[j] = sw[ch_swz(j * 32 + lane)];
+        uint32_t c = (uint32_t)((tile * CH_WTILE + (uint64_t)lane * 4) % C);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float v[4], lo[4], sc[4];
+            ch_lds4(tab.lo + QP_CK(c, C - 3), lo);
+            ch_lds4(tab.scale + QP_CK(c, C - 3), sc);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = fmaf(ch_code_to_float((mine[j] >> (BITS * i)) & MASK), sc[i], lo[i]);
+            ch_store4(y, tile * CH_WTILE + (uint64_t)(j * 32 + lane) * 4, v);
+            c += cstep;
+            if (c >= C) c -= C;
         }
         __syncwarp();
     }
@@ -634,7 +766,7 @@ extern "C" int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int d
     int32_t rc = ch_check(ctx, rows, channels);
     if (rc) return rc;
     if (!qp_bits_ok(bits)) return qp_fail(ctx, QP_ERR_UNSUPPORTED_BITS, "bits must be 1..8 or 16");
-    const uint64_t n = rows * channels;
+    uint64_t n = rows * channels;
     const uint64_t need = qp_packed_bytes(n, bits);
     if (packed_capacity < need) return qp_fail(ctx, QP_ERR_BUFFER_TOO_SMALL, "packed_capacity < qp_packed_bytes(n, bits)");
     if (!d_qp || (n > 0 && (!d_x || !d_packed))) return qp_fail(ctx, QP_ERR_INVALID_ARG, "null pointer");
@@ -644,20 +776,56 @@ extern "C" int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int d
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const uint64_t total_words = need / 4;
+    const size_t smem = ch_pack_smem(channels);
+    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
+    const int esz = dtype == QP_F32 ? 4 : 2;
+    const bool vec = channels % (16 / esz) == 0 && ((uintptr_t)d_x & 15u) == 0;
+    // whole warp tiles of an aligned tensor at 1..8 bits go through the fast kernel; the generic one takes
+    // what is left (the last partial tile and the pad words), or everything
+    const uint64_t nfast = (vec && bits <= 8) ? n / CH_WTILE : 0;
+    const uint64_t el0 = nfast * CH_WTILE;
+    uint32_t* out = static_cast<uint32_t*>(d_packed) + nfast * 32 * (uint64_t)bits;
+    const uint64_t n_all = n;
+    n = n_all - el0;
+    const uint64_t total_words = need / 4 - nfast * 32 * (uint64_t)bits;
     const uint64_t groups = (total_words + bits - 1) / bits;
     const uint64_t ntiles = (groups + 31) / 32;                               // warp tiles, pad words included
     const uint64_t want = (ntiles + CH_WARPS - 1) / CH_WARPS;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
     const unsigned blocks = (unsigned)(want < cap ? want : cap);
-    const size_t smem = ch_pack_smem(channels);
-    uint32_t* out = static_cast<uint32_t*>(d_packed);
-    bool ok = false;
+    bool ok = true;
+    if (nfast) {
+        const uint64_t fwant = (nfast + CH_WARPS - 1) / CH_WARPS;
+        const unsigned fblocks = (unsigned)(fwant < cap ? fwant : cap);
+        uint32_t* fout = static_cast<uint32_t*>(d_packed);
+#define QP_CH_FAST(T, B)                                                                                               \
+    do {                                                                                                               \
+        ok = ch_allow_smem(ch_pack_fast<B, T>, smem);                                                                  \
+        if (ok) ch_pack_fast<B, T><<<fblocks, CH_THREADS, smem, s>>>(static_cast<const T*>(d_x), nfast, channels,     \
+                                                                    d_qp, fout, ctx->d_status);                       \
+    } while (0)
+#define QP_CH_FAST_BITS(T)                                                                                             \
+    switch (bits) {                                                                                                    \
+        case 1: QP_CH_FAST(T, 1); break;                                                                               \
+        case 2: QP_CH_FAST(T, 2); break;                                                                               \
+        case 3: QP_CH_FAST(T, 3); break;                                                                               \
+        case 4: QP_CH_FAST(T, 4); break;                                                                               \
+        case 5: QP_CH_FAST(T, 5); break;                                                                               \
+        case 6: QP_CH_FAST(T, 6); break;                                                                               \
+        case 7: QP_CH_FAST(T, 7); break;                                                                               \
+        default: QP_CH_FAST(T, 8); break;                                                                              \
+    }
+        if (dtype == QP_F32) { QP_CH_FAST_BITS(float) } else { QP_CH_FAST_BITS(unsigned short) }
+#undef QP_CH_FAST_BITS
+#undef QP_CH_FAST
+        if (!ok) return qp_check_launch(ctx, "qp_quantize_pack_channels (shared memory)");
+        ctx->launches += 1;
+        if (total_words == 0) return qp_check_launch(ctx, "qp_quantize_pack_channels");
+    }
 #define QP_CH_PACK(T, VEC, B)                                                                                          \
     do {                                                                                                               \
         ok = ch_allow_smem(ch_pack_kernel<T, VEC, B>, smem);                                                           \
         if (ok) ch_pack_kernel<T, VEC, B><<<blocks, CH_THREADS, smem, s>>>(x, n, channels, bits, d_qp, out,           \
-                                                                          total_words, ntiles, ctx->d_status);        \
+                                                                          total_words, ntiles, el0, ctx->d_status);   \
     } while (0)
 #define QP_CH_PACK_BITS(T)                                                                                             \
     switch (bits) {                                                                                                    \
@@ -672,12 +840,12 @@ extern "C" int32_t qp_quantize_pack_channels(qp_ctx* ctx, const void* d_x, int d
         default: QP_CH_PACK(T, true, 16); break;                                                                       \
     }
     if (dtype == QP_F32) {
-        const float* x = static_cast<const float*>(d_x);
-        if (channels % 4 == 0 && ((uintptr_t)x & 15u) == 0) { QP_CH_PACK_BITS(float) }
+        const float* x = static_cast<const float*>(d_x) + el0;
+        if (vec) { QP_CH_PACK_BITS(float) }
         else QP_CH_PACK(float, false, 0);
     } else {
-        const unsigned short* x = static_cast<const unsigned short*>(d_x);
-        if (channels % 8 == 0 && ((uintptr_t)x & 15u) == 0) { QP_CH_PACK_BITS(unsigned short) }
+        const unsigned short* x = static_cast<const unsigned short*>(d_x) + el0;
+        if (vec) { QP_CH_PACK_BITS(unsigned short) }
         else QP_CH_PACK(unsigned short, false, 0);
     }
 #undef QP_CH_PACK_BITS
@@ -704,19 +872,52 @@ extern "C" int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_pack
     qp_device_guard guard(ctx->device);
     if (!guard.ok) return qp_fail(ctx, QP_ERR_CUDA, "cannot select device");
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const uint64_t total_words = qp_packed_bytes(n, bits) / 4;
-    const uint64_t ntiles = (n + CH_WTILE - 1) / CH_WTILE;
-    const uint64_t want = (ntiles + CH_WARPS - 1) / CH_WARPS;
-    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
-    const unsigned blocks = (unsigned)(want < cap ? want : cap);
     const size_t smem = ch_pack_smem(channels);
-    const uint32_t* in = static_cast<const uint32_t*>(d_packed);
-    bool ok = false;
+    const uint64_t cap = (uint64_t)ctx->sm_count * 6;
+    const bool vec = channels % 4 == 0 && ((uintptr_t)d_y & (out_dtype == QP_F32 ? 15u : 7u)) == 0;
+    // whole warp tiles at 1..8 bits go through the fast kernel, the generic one takes what is left
+    const uint64_t nfast = (vec && bits <= 8) ? n / CH_WTILE : 0;
+    const uint64_t el0 = nfast * CH_WTILE;
+    const uint64_t total_words = qp_packed_bytes(n, bits) / 4 - nfast * 32 * (uint64_t)bits;
+    const uint32_t* in = static_cast<const uint32_t*>(d_packed) + nfast * 32 * (uint64_t)bits;
+    bool ok = true;
+    if (nfast) {
+        const uint64_t fwant = (nfast + CH_WARPS - 1) / CH_WARPS;
+        const unsigned fblocks = (unsigned)(fwant < cap ? fwant : cap);
+        const uint32_t* fin = static_cast<const uint32_t*>(d_packed);
+#define QP_CH_FAST(T, B)                                                                                               \
+    do {                                                                                                               \
+        ok = ch_allow_smem(ch_unpack_fast<B, T>, smem);                                                                \
+        if (ok) ch_unpack_fast<B, T><<<fblocks, CH_THREADS, smem, s>>>(fin, nfast, channels, d_qp,                    \
+                                                                      static_cast<T*>(d_y), ctx->d_status);           \
+    } while (0)
+#define QP_CH_FAST_BITS(T)                                                                                             \
+    switch (bits) {                                                                                                    \
+        case 1: QP_CH_FAST(T, 1); break;                                                                               \
+        case 2: QP_CH_FAST(T, 2); break;                                                                               \
+        case 3: QP_CH_FAST(T, 3); break;                                                                               \
+        case 4: QP_CH_FAST(T, 4); break;                                                                               \
+        case 5: QP_CH_FAST(T, 5); break;                                                                               \
+        case 6: QP_CH_FAST(T, 6); break;                                                                               \
+        case 7: QP_CH_FAST(T, 7); break;                                                                               \
+        default: QP_CH_FAST(T, 8); break;                                                                              \
+    }
+        if (out_dtype == QP_F32) { QP_CH_FAST_BITS(float) } else { QP_CH_FAST_BITS(unsigned short) }
+#undef QP_CH_FAST_BITS
+#undef QP_CH_FAST
+        if (!ok) return qp_check_launch(ctx, "qp_unpack_dequantize_channels (shared memory)");
+        ctx->launches += 1;
+        if (n == el0) return qp_check_launch(ctx, "qp_unpack_dequantize_channels");
+    }
+    const uint64_t n_rest = n - el0;
+    const uint64_t ntiles = (n_rest + CH_WTILE - 1) / CH_WTILE;
+    const uint64_t want = (ntiles + CH_WARPS - 1) / CH_WARPS;
+    const unsigned blocks = (unsigned)(want < cap ? want : cap);
 #define QP_CH_UNPACK(T, VEC, B)                                                                                        \
     do {                                                                                                               \
         ok = ch_allow_smem(ch_unpack_kernel<T, VEC, B>, smem);                                                         \
-        if (ok) ch_unpack_kernel<T, VEC, B><<<blocks, CH_THREADS, smem, s>>>(in, n, channels, bits, d_qp, y,          \
-                                                                            total_words, ntiles, ctx->d_status);      \
+        if (ok) ch_unpack_kernel<T, VEC, B><<<blocks, CH_THREADS, smem, s>>>(in, n_rest, channels, bits, d_qp, y,     \
+                                                                            total_words, ntiles, el0, ctx->d_status); \
     } while (0)
 #define QP_CH_UNPACK_BITS(T)                                                                                           \
     switch (bits) {                                                                                                    \
@@ -731,12 +932,12 @@ extern "C" int32_t qp_unpack_dequantize_channels(qp_ctx* ctx, const void* d_pack
         default: QP_CH_UNPACK(T, true, 16); break;                                                                     \
     }
     if (out_dtype == QP_F32) {
-        float* y = static_cast<float*>(d_y);
-        if (channels % 4 == 0 && ((uintptr_t)y & 15u) == 0) { QP_CH_UNPACK_BITS(float) }
+        float* y = static_cast<float*>(d_y) + el0;
+        if (vec) { QP_CH_UNPACK_BITS(float) }
         else QP_CH_UNPACK(float, false, 0);
     } else {
-        unsigned short* y = static_cast<unsigned short*>(d_y);
-        if (channels % 4 == 0 && ((uintptr_t)y & 7u) == 0) { QP_CH_UNPACK_BITS(unsigned short) }
+        unsigned short* y = static_cast<unsigned short*>(d_y) + el0;
+        if (vec) { QP_CH_UNPACK_BITS(unsigned short) }
         else QP_CH_UNPACK(unsigned short, false, 0);
     }
 #undef QP_CH_UNPACK_BITS

@@ -12,7 +12,9 @@
 //                     arithmetic on the column, fp32 error sums over 8 rows folded into fp64,
 //                     block partials per (row block, channel, candidate)
 //   ch_pick_kernel    block per channel: partials merged in row-block order, first minimum wins
-// Work is (steps + 1) * 9 fp32 instructions per element, as in the per-tensor candidate path.
+// Work is (steps + 1) * 9 fp32 instructions per element, as in the per-tensor candidate path.  Where the
+// interval form applies (qp_channels_search_fast.cu: one pass over the tensor instead of the scoring) it
+// takes ch_eval_kernel's place and hands the pick one row block of sums.
 #include <stdlib.h>
 
 #include "qp_internal.cuh"
@@ -215,6 +217,9 @@ int32_t search_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C
     const uint64_t min_rows = 8 * CS_EVAL_LANES;             // no point in blocks of less than one batch per lane
     if (row_blocks > (rows + min_rows - 1) / min_rows) row_blocks = (rows + min_rows - 1) / min_rows;
     if (row_blocks < 1) row_blocks = 1;
+    // interval moments where they apply (qp_set_search_path(QP_SEARCH_CANDIDATES) keeps the scoring of every candidate)
+    const bool intervals = ctx->search_path != QP_SEARCH_CANDIDATES && qp_channel_interval_applies(rows, bits, steps);
+    if (intervals) row_blocks = 1;
     const uint64_t rows_per_block = (rows + row_blocks - 1) / row_blocks;
 
     size_t off = 0;
@@ -224,6 +229,8 @@ int32_t search_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C
     const size_t o_setup = off; off = align256(off + sizeof(qp_ds_setup) * (size_t)C);
     const size_t o_curve = off; off = align256(off + sizeof(double) * (size_t)C * ncp);
     const size_t o_part = off;  off = align256(off + sizeof(double) * (size_t)row_blocks * C * ncp);
+    const size_t o_iv = off;
+    if (intervals) off = align256(off + qp_channel_interval_scratch_bytes(C, (steps + 1) * ((1 << bits) - 1)));
     if (ctx->ch_search_bytes < off) {                        // grown on demand, kept by the context
         if (ctx->d_ch_search) cudaFree(ctx->d_ch_search);
         ctx->d_ch_search = nullptr;
@@ -253,11 +260,19 @@ int32_t search_channels_typed(qp_ctx* ctx, const T* x, uint64_t rows, uint32_t C
         ctx->launches += 1;
     }
     ch_setup_kernel<<<C, 128, 0, s>>>(d_stats, hist, nb, bits, bmode, steps, ncp, F, cand, valid, setup);
-    const dim3 egrid((C + CS_EVAL_CH - 1) / CS_EVAL_CH, groups, (unsigned)row_blocks);
-    ch_eval_kernel<T><<<egrid, CS_EVAL_CH * CS_EVAL_LANES, 0, s>>>(x, rows, C, rows_per_block, cand, ncp, part);
+    ctx->launches += 1;
+    if (intervals) {
+        const int32_t rc = qp_launch_channel_interval_sums(ctx, x, sizeof(T) == 4 ? QP_F32 : QP_BF16, rows, C, bits, steps, ncp,
+                                                           d_stats, cand, valid, setup, b + o_iv, part, s);
+        if (rc != QP_OK) return rc;
+    } else {
+        const dim3 egrid((C + CS_EVAL_CH - 1) / CS_EVAL_CH, groups, (unsigned)row_blocks);
+        ch_eval_kernel<T><<<egrid, CS_EVAL_CH * CS_EVAL_LANES, 0, s>>>(x, rows, C, rows_per_block, cand, ncp, part);
+        ctx->launches += 1;
+    }
     ch_pick_kernel<<<C, 128, 0, s>>>(part, (int)row_blocks, C, steps, ncp, nb, bits, valid, cand, setup, curve, d_out,
                                      d_qp_out, ctx->d_status);
-    ctx->launches += 3;
+    ctx->launches += 1;
     ctx->ch_last_steps = steps;
     ctx->ch_last_ncp = ncp;
     ctx->ch_last_channels = C;

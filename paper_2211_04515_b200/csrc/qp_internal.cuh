@@ -213,6 +213,30 @@ __device__ __forceinline__ unsigned qp_code(float x, float lo, float hi, float i
     return __float_as_uint(__fadd_rn(qp_grid_pos(x, lo, hi, inv_scale), QP_MAGIC)) & mask;
 }
 
+// monotone map float -> uint32 (finite values; -0 sorts directly below +0), and back
+__device__ __forceinline__ unsigned qp_key_of(float x)
+{
+    const unsigned u = __float_as_uint(x);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float qp_float_of(unsigned k)
+{
+    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
+}
+
+// smallest float in (lo_x, hi_x] for which pred holds, given !pred(lo_x) and pred(hi_x), pred monotone:
+// bisection over the floats' bit patterns (at most 32 evaluations of pred)
+template <typename P>
+__device__ __forceinline__ float qp_first_true(float lo_x, float hi_x, P pred)
+{
+    unsigned lo = qp_key_of(lo_x), hi = qp_key_of(hi_x);
+    while (hi - lo > 1u) {
+        const unsigned mid = lo + ((hi - lo) >> 1);
+        if (pred(qp_float_of(mid))) hi = mid; else lo = mid;
+    }
+    return qp_float_of(hi);
+}
+
 __device__ __forceinline__ float qp_bf16_to_f32(unsigned short h) { return __uint_as_float((unsigned)h << 16); }
 
 __device__ __forceinline__ unsigned short qp_f32_to_bf16(float f)   // round to nearest even
@@ -423,6 +447,12 @@ int32_t qp_launch_stats(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, int
 int32_t qp_launch_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats, int bits,
                          int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                          qp_qparams_t* d_qp_out, cudaStream_t s);
+// channel-wise search through interval moments (qp_channels_search_fast.cu)
+size_t qp_channel_interval_scratch_bytes(uint32_t C, int nthr);
+bool qp_channel_interval_applies(uint64_t rows, int bits, int steps);
+int32_t qp_launch_channel_interval_sums(qp_ctx* ctx, const void* d_x, int dtype, uint64_t rows, uint32_t C, int bits, int steps,
+                                        int ncp, const qp_stats_t* d_stats, const float4* cand, const int* valid,
+                                        qp_ds_setup* setup, char* scratch, double* part, cudaStream_t s);
 int32_t qp_launch_interval_search(qp_ctx* ctx, const void* d_x, int dtype, uint64_t n, const qp_stats_t* d_stats,
                                   int bits, int bmode, int steps, int hist_bins, double F, qp_ds_result_t* d_out,
                                   qp_qparams_t* d_qp_out, cudaStream_t s);

@@ -33,17 +33,6 @@ constexpr int G = QP_IV_CELLS;
 constexpr int MAXB = QP_IV_MAXB;
 constexpr unsigned long long S1_MASK = (1ull << 40) - 1ull;
 
-// monotone map float -> uint32 (finite values; -0 sorts directly below +0)
-__device__ __forceinline__ unsigned key_of(float x)
-{
-    const unsigned u = __float_as_uint(x);
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
-}
-__device__ __forceinline__ float float_of(unsigned k)
-{
-    return __uint_as_float((k & 0x80000000u) ? (k & 0x7FFFFFFFu) : ~k);
-}
-
 // Grid cell of x in [g_lo, g_hi]: its position in cell units, rounded to the nearest integer
 // (0..G, so G + 1 cells).  The rounding is done by adding 2^23 (no conversion instruction):
 // `pm` keeps the cell number in its low mantissa bits.  Each operation is rounded on its own,
@@ -65,18 +54,6 @@ __device__ __forceinline__ int cell_of(float x, float g_lo, float inv_gw)
 __device__ __forceinline__ float cell_ref(float pm, float g_lo, float gw)
 {
     return fmaf(__fsub_rn(pm, IV_MAGIC + 1.0f), gw, g_lo);      // (cell - 1) * gw + g_lo
-}
-
-// smallest float in (lo_x, hi_x] for which pred holds, given !pred(lo_x) and pred(hi_x), pred monotone
-template <typename P>
-__device__ __forceinline__ float first_true(float lo_x, float hi_x, P pred)
-{
-    unsigned lo = key_of(lo_x), hi = key_of(hi_x);
-    while (hi - lo > 1u) {
-        const unsigned mid = lo + ((hi - lo) >> 1);
-        if (pred(float_of(mid))) hi = mid; else lo = mid;
-    }
-    return float_of(hi);
 }
 
 // ------------------------------------------------------------------ grid + boundaries
@@ -174,7 +151,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
             const float4 q = s_cand[k];
             const unsigned mask = (unsigned)L1;
             auto pred = [&](float x) { return (int)qp_code(x, q.x, q.y, q.w, mask) >= j; };
-            if (!pred(g_lo) && pred(g_hi)) out = first_true(g_lo, g_hi, pred);
+            if (!pred(g_lo) && pred(g_hi)) out = qp_first_true(g_lo, g_hi, pred);
         }
         bnd[t] = out;
     } else if (t < nthr + G) {
@@ -182,7 +159,7 @@ __global__ void __launch_bounds__(256) iv_bounds_kernel(const qp_stats_t* __rest
         float out = inf;
         if (g_hi > g_lo) {
             auto pred = [&](float x) { return cell_of(x, g_lo, inv_gw) >= c; };
-            if (!pred(g_lo) && pred(g_hi)) out = first_true(g_lo, g_hi, pred);
+            if (!pred(g_lo) && pred(g_hi)) out = qp_first_true(g_lo, g_hi, pred);
         }
         bnd[t] = out;
     } else if (t < MAXB) {
@@ -470,39 +447,52 @@ __device__ __forceinline__ void iv2_exact(float x, const IvShared& sh, const IvC
     if (old + d1 < old) atomicAdd(&sh.cnt[lo], 1u << 24);
 }
 
-// One element: clamp, outer sums, cell, offset, the two replica atomics.  If its cell turns out to
-// be split it goes into the warp's buffer; from 32 buffered elements on, the warp works 32 of
-// them off with every lane busy.  Called by all 32 lanes together (lanes without an element pass
-// a non-finite value to the guarded form).
-template <bool GUARD>
-__device__ __forceinline__ void iv2_one(float x, const IvShared& sh, const Iv2Shared& s2, const IvConst& k, IvBatch& b,
-                                        float* my_stage, unsigned& staged, unsigned lane)
+// A batch of N elements per lane: clamp, outer sums, cell, offset and the two replica atomics of ALL of
+// them first (independent: their latencies overlap), then one vote on whether any element of the warp
+// met a split cell (the mark comes back with the count atomic's old value).  Only then, element by
+// element, the split ones go into the warp's buffer; from 32 buffered elements on, the warp works 32 of
+// them off with every lane busy.  (Asking after every element instead made each element wait for its
+// own atomic to return: the pass was bound by that latency, not by issue slots or the shared-memory
+// pipe.)  Called by all 32 lanes together (lanes without an element pass a non-finite value to the
+// guarded form).
+template <bool GUARD, int N>
+__device__ __forceinline__ void iv2_batch(const float (&x)[N], const IvShared& sh, const Iv2Shared& s2, const IvConst& k,
+                                          IvBatch& b, float* my_stage, unsigned& staged, unsigned lane)
 {
     const unsigned full = 0xFFFFFFFFu;
-    bool split = false;
-    float xc = x;
-    if (!GUARD || qp_is_finite(x)) {
-        xc = fminf(fmaxf(x, k.g_lo), k.g_hi);
-        const float e = __fsub_rn(x, xc);
-        b.s1 += e; b.s1a += fabsf(e); b.s2 = fmaf(e, e, b.s2);
-        const float pm = cell_pm(xc, k.g_lo, k.inv_gw);
-        const float dm = fmaf(__fsub_rn(xc, cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
-        const float d1f = __fsub_rn(dm, IV_MAGIC);
-        b.s2_in = fmaf(d1f, d1f, b.s2_in);
-        const unsigned idx = QP_CK(((__float_as_uint(pm) & 0x7FFFFFu) << IV2_RS) + (lane & (IV2_R - 1u)), (G + 1) * IV2_R);
-        const unsigned old = atomicAdd(&s2.rcnt[idx], 1u);
-        atomicAdd(&s2.rs1[idx], __float_as_uint(dm) & 0x7FFFFFu);     // ignored later if the cell is split
-        split = (old & IV2_SPLIT) != 0u;
+    float xc[N];
+    unsigned flags = 0u;                                 // bit i: element i lies in a split cell
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        xc[i] = x[i];
+        if (!GUARD || qp_is_finite(x[i])) {
+            xc[i] = fminf(fmaxf(x[i], k.g_lo), k.g_hi);
+            const float e = __fsub_rn(x[i], xc[i]);
+            b.s1 += e; b.s1a += fabsf(e); b.s2 = fmaf(e, e, b.s2);
+            const float pm = cell_pm(xc[i], k.g_lo, k.inv_gw);
+            const float dm = fmaf(__fsub_rn(xc[i], cell_ref(pm, k.g_lo, k.gw)), k.inv_u, IV_MAGIC);
+            const float d1f = __fsub_rn(dm, IV_MAGIC);
+            b.s2_in = fmaf(d1f, d1f, b.s2_in);
+            const unsigned idx = QP_CK(((__float_as_uint(pm) & 0x7FFFFFu) << IV2_RS) + (lane & (IV2_R - 1u)), (G + 1) * IV2_R);
+            const unsigned old = atomicAdd(&s2.rcnt[idx], 1u);
+            atomicAdd(&s2.rs1[idx], __float_as_uint(dm) & 0x7FFFFFu);     // ignored later if the cell is split
+            flags |= (old >> 31) << i;                   // IV2_SPLIT is the top bit
+        }
     }
-    const unsigned m = __ballot_sync(full, split);
-    if (m) {                                             // warp-uniform
-        if (split) my_stage[QP_CK(staged + __popc(m & ((1u << lane) - 1u)), IV2_STAGE)] = xc;
-        staged += __popc(m);
-        if (staged >= 32u) {
-            __syncwarp();
-            staged -= 32u;
-            iv2_exact(my_stage[staged + lane], sh, k);
-            __syncwarp();
+    if (!__any_sync(full, flags != 0u)) return;          // warp-uniform
+#pragma unroll
+    for (int i = 0; i < N; ++i) {
+        const bool split = (flags >> i) & 1u;
+        const unsigned m = __ballot_sync(full, split);
+        if (m) {                                         // warp-uniform
+            if (split) my_stage[QP_CK(staged + __popc(m & ((1u << lane) - 1u)), IV2_STAGE)] = xc[i];
+            staged += __popc(m);
+            if (staged >= 32u) {
+                __syncwarp();
+                staged -= 32u;
+                iv2_exact(my_stage[staged + lane], sh, k);
+                __syncwarp();
+            }
         }
     }
 }
@@ -580,16 +570,29 @@ __global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __
         const float skip = __int_as_float(0x7FC00000);       // NaN: ignored by the guarded form
         uint64_t v = (uint64_t)blockIdx.x * IV2_THREADS + threadIdx.x;
         // two vectors per lane while the warp's last lane still has both (v - lane + 31 is its first vector)
-        for (; v - lane + 31u + stride < sp.nvec; v += 2 * stride) {
+        // (the next pair is loaded before the current one is worked on, so a warp does not sit out the load latency)
+        auto both = [&](uint64_t vv) { return vv - lane + 31u + stride < sp.nvec; };   // warp-uniform
+        if (both(v)) {
             float a[EPV], b[EPV];
             qp_load_vec(xv + v * EPV, a);
             qp_load_vec(xv + (v + stride) * EPV, b);
-            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
+            for (;;) {
+                const uint64_t vn = v + 2 * stride;
+                const bool more = both(vn);
+                float na[EPV], nb[EPV];
+                if (more) {
+                    qp_load_vec(xv + vn * EPV, na);
+                    qp_load_vec(xv + (vn + stride) * EPV, nb);
+                }
+                IvBatch bt = {0.f, 0.f, 0.f, 0.f};
+                iv2_batch<GD>(a, sh, s2, k, bt, my_stage, staged, lane);
+                iv2_batch<GD>(b, sh, s2, k, bt, my_stage, staged, lane);
+                iv_flush(o, bt);
+                v = vn;
+                if (!more) break;
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv2_one<GD>(a[i], sh, s2, k, bt, my_stage, staged, lane);
-#pragma unroll
-            for (int i = 0; i < EPV; ++i) iv2_one<GD>(b[i], sh, s2, k, bt, my_stage, staged, lane);
-            iv_flush(o, bt);
+                for (int i = 0; i < EPV; ++i) { a[i] = na[i]; b[i] = nb[i]; }
+            }
         }
         // the rest: warps may be partly filled, so every lane of a warp that still has work goes on
         const uint64_t warp_v0 = v - lane;                   // vector of lane 0 (v advanced alike in all lanes)
@@ -598,9 +601,10 @@ __global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __
             const bool have = mine < sp.nvec;
             float a[EPV];
             if (have) qp_load_vec(xv + mine * EPV, a);
-            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-            for (int i = 0; i < EPV; ++i) iv2_one<true>(have ? a[i] : skip, sh, s2, k, bt, my_stage, staged, lane);
+            for (int i = 0; i < EPV; ++i) a[i] = have ? a[i] : skip;
+            IvBatch bt = {0.f, 0.f, 0.f, 0.f};
+            iv2_batch<true>(a, sh, s2, k, bt, my_stage, staged, lane);
             iv_flush(o, bt);
         }
         if (blockIdx.x == 0) {
@@ -610,8 +614,8 @@ __global__ void __launch_bounds__(IV2_THREADS, 1) iv_moments2_kernel(const T* __
                 const uint64_t i = i0 + lane;
                 const bool have = i < extra;
                 IvBatch bt = {0.f, 0.f, 0.f, 0.f};
-                const float x1 = have ? qp_load_one(x + (i < sp.head ? i : t0 + (i - sp.head))) : skip;
-                iv2_one<true>(x1, sh, s2, k, bt, my_stage, staged, lane);
+                const float x1[1] = {have ? qp_load_one(x + (i < sp.head ? i : t0 + (i - sp.head))) : skip};
+                iv2_batch<true>(x1, sh, s2, k, bt, my_stage, staged, lane);
                 iv_flush(o, bt);
             }
         }

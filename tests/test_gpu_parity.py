@@ -1166,32 +1166,39 @@ def test_channels_sender_in_one_call(ctx):
 def check_search_channels(ctx, x_np, d_x, channels, bits, bmode=0, steps=100, nb=100):
     """Every channel's search against the oracle's search of that column, as check_search: the
     candidates' clip ranges, every candidate's error for exactly the quantizer the library scored
-    (2e-6), the winner (first minimum, or a tie at 1e-6) and its clipping value (1e-4)."""
+    (2e-6), the winner (first minimum, or a tie at 1e-6) and its clipping value (1e-4).  Both forms
+    of the library's search: interval moments (the default where they apply) and the scoring of
+    every candidate."""
     rows = x_np.size // channels
-    d_stats = ctx.qp_stats_channels(d_x, channels)
-    d_res, d_qp = ctx.qp_dsaciq_search_channels(d_x, channels, d_stats, bits, bmode, steps, nb)
-    raw_res = d_res.cpu().numpy().tobytes()
-    raw_qp = d_qp.cpu().numpy().tobytes()
-    cand_all = ctx.qp_dsaciq_candidates_channels(channels, steps)
-    rsz, qsz = ctypes.sizeof(qp.DSResult), ctypes.sizeof(qp.QParams)
     st_o = oracle.stats_channels(x_np, channels)
     rc_o, res_o, qp_o, curves_o = oracle.ds_search_channels(x_np, channels, st_o, bits, bmode, steps, nb)
     cols = x_np.reshape(rows, channels)
-    for c in range(channels):
-        res = qp.DSResult.from_buffer_copy(raw_res[c * rsz:(c + 1) * rsz])
-        got = qp.QParams.from_buffer_copy(raw_qp[c * qsz:(c + 1) * qsz])
-        ro = res_o[c]
-        assert (res.steps, res.hist_bins, res.bits) == (steps, nb, bits)
-        assert abs(res.b_e - ro.b_e) <= 1e-5 * abs(ro.b_e) + 1e-300
-        assert abs(res.b_r - ro.b_r) <= 1e-9 * abs(ro.b_r) + 1e-300         # integer-identical histogram
-        curve = np.array(ctx.qp_dsaciq_curve_channels(c, steps))
-        cand = cand_all[c * (steps + 1):(c + 1) * (steps + 1)]
-        check_candidates_and_pick(np.ascontiguousarray(cols[:, c]), st_o[c], ro, curves_o[c], res, curve, cand, bits,
-                                  bmode, steps)
-        w = cand[res.k_star]
-        assert (got.lo, got.hi, got.scale, got.inv_scale, got.bits) == (w.lo, w.hi, w.scale, w.inv_scale, bits)
-        assert got.flags == qp_o[c].flags
-        assert res.mse_star == curve[res.k_star] and res.mse_e == curve[0]
+    rsz, qsz = ctypes.sizeof(qp.DSResult), ctypes.sizeof(qp.QParams)
+    try:
+        for path in (qp.QP_SEARCH_AUTO, qp.QP_SEARCH_CANDIDATES):
+            ctx.qp_set_search_path(path)
+            d_stats = ctx.qp_stats_channels(d_x, channels)
+            d_res, d_qp = ctx.qp_dsaciq_search_channels(d_x, channels, d_stats, bits, bmode, steps, nb)
+            raw_res = d_res.cpu().numpy().tobytes()
+            raw_qp = d_qp.cpu().numpy().tobytes()
+            cand_all = ctx.qp_dsaciq_candidates_channels(channels, steps)
+            for c in range(channels):
+                res = qp.DSResult.from_buffer_copy(raw_res[c * rsz:(c + 1) * rsz])
+                got = qp.QParams.from_buffer_copy(raw_qp[c * qsz:(c + 1) * qsz])
+                ro = res_o[c]
+                assert (res.steps, res.hist_bins, res.bits) == (steps, nb, bits)
+                assert abs(res.b_e - ro.b_e) <= 1e-5 * abs(ro.b_e) + 1e-300
+                assert abs(res.b_r - ro.b_r) <= 1e-9 * abs(ro.b_r) + 1e-300         # integer-identical histogram
+                curve = np.array(ctx.qp_dsaciq_curve_channels(c, steps))
+                cand = cand_all[c * (steps + 1):(c + 1) * (steps + 1)]
+                check_candidates_and_pick(np.ascontiguousarray(cols[:, c]), st_o[c], ro, curves_o[c], res, curve, cand, bits,
+                                          bmode, steps)
+                w = cand[res.k_star]
+                assert (got.lo, got.hi, got.scale, got.inv_scale, got.bits) == (w.lo, w.hi, w.scale, w.inv_scale, bits)
+                assert got.flags == qp_o[c].flags
+                assert res.mse_star == curve[res.k_star] and res.mse_e == curve[0]
+    finally:
+        ctx.qp_set_search_path(qp.QP_SEARCH_AUTO)
     # the quantizers feed the channel-wise packer: bit-exact codes under the library's own quantizers
     mine = (oracle.QParams * channels)()
     for c in range(channels):
