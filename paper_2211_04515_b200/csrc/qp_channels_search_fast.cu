@@ -53,15 +53,15 @@ __device__ __forceinline__ int ci_cell(float x, float g0, float inv_cw)
 
 // ---------------------------------------------------------------- thresholds, sorted
 
-// block c: thresholds of channel c.  thr[c][k * L1 + j - 1] = T(k, j) (+inf: candidate not valid),
-// bb[c][0 .. nthr) = the same values in ascending order, pos[c][.] = for every threshold the number of
-// thresholds <= it, m[c] = how many are finite; the offsets' unit, the reference point and the look-up
+// block c: thresholds T(k, j) of channel c (+inf: candidate not valid).  bb[c][0 .. nthr) = their values in
+// ascending order, pos[c][(j - 1) * ncand + k] = the number of thresholds <= T(k, j) (0xFFFF for +inf),
+// m[c] = how many are finite; the offsets' unit, the reference point and the look-up
 // grid go into setup[c] (u, inv_u, g_lo = the channel's minimum, gw / inv_gw = the grid).
 __global__ void __launch_bounds__(CI_TAB_THREADS) ci_tables_kernel(const qp_stats_t* __restrict__ st,
                                                                    const float4* __restrict__ cand,
                                                                    const int* __restrict__ valid, int ncp, int ncand,
                                                                    int bits, int nthr, int p2,
-                                                                   qp_ds_setup* __restrict__ setup, float* __restrict__ thr,
+                                                                   qp_ds_setup* __restrict__ setup,
                                                                    float* __restrict__ bb, unsigned* __restrict__ m_out,
                                                                    unsigned* __restrict__ cells,
                                                                    unsigned short* __restrict__ pos)
@@ -132,7 +132,6 @@ __global__ void __launch_bounds__(CI_TAB_THREADS) ci_tables_kernel(const qp_stat
                 if (xa < xb && !pred(xa) && pred(xb)) out = qp_first_true(xa, xb, pred);
                 else if (!pred(g_lo) && pred(g_hi)) out = qp_first_true(g_lo, g_hi, pred);
             }
-            thr[(size_t)c * nthr + t] = out;
         }
         s_thr[t] = out;
     }
@@ -195,11 +194,12 @@ __global__ void __launch_bounds__(CI_TAB_THREADS) ci_tables_kernel(const qp_stat
         for (int t = threadIdx.x; t < nthr; t += CI_TAB_THREADS) s_key[t] = src[t];
         __syncthreads();
     }
-    for (int t = threadIdx.x; t < nthr; t += CI_TAB_THREADS) {         // pos(T) = sorted thresholds <= T
-        const float T = s_thr[t];
+    for (int r = threadIdx.x; r < nthr; r += CI_TAB_THREADS) {         // pos(T) = sorted thresholds <= T, run by run
+        const int jj = r / ncand, k = r - jj * ncand;
+        const float T = s_thr[k * L1 + jj];
         int lo = 0, hi = nthr;
         while (lo < hi) { const int mid = (lo + hi) >> 1; if (s_key[mid] <= T) lo = mid + 1; else hi = mid; }
-        pos[(size_t)c * nthr + t] = (unsigned short)lo;
+        pos[(size_t)c * nthr + r] = T < inf ? (unsigned short)lo : (unsigned short)0xFFFFu;
     }
     for (int t = threadIdx.x; t < nthr; t += CI_TAB_THREADS) bb[(size_t)c * nthr + t] = s_key[t];
     __shared__ int s_m;
@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(CI_MOM_THREADS, 1) ci_moments_kernel(const T* 
 // pos(T) = number of thresholds <= T (all intervals from there on hold elements >= T, the ones before
 // it elements < T), and the total of its squared error goes to part[c][k] for the pick.
 __global__ void __launch_bounds__(CI_CURVE_THREADS) ci_curve_kernel(const unsigned long long* __restrict__ tot,
-                                                                    const float* __restrict__ bb, const float* __restrict__ thr,
+                                                                    const float* __restrict__ bb,
                                                                     const unsigned short* __restrict__ pos,
                                                                     const unsigned* __restrict__ m_in,
                                                                     const qp_ds_setup* __restrict__ setup,
@@ -347,27 +347,31 @@ __global__ void __launch_bounds__(CI_CURVE_THREADS) ci_curve_kernel(const unsign
     const unsigned m = m_in[c];
     const qp_ds_setup s = setup[c];
     const double u = s.u, ref0 = (double)s.g_lo;
-    const float inf = __int_as_float(0x7F800000);
 
-    // exclusive prefix sums over intervals 0..m: thread t takes the chunk [t * per, t * per + per)
-    const int count = (int)m + 1, per = (count + CI_CURVE_THREADS - 1) / CI_CURVE_THREADS;
-    const int i0 = threadIdx.x * per, i1 = min(i0 + per, count);
-    auto interval = [&](int i, double& n, double& sx, double& sxx) {
-        const unsigned long long w = tot[(size_t)c * stride + i];
-        n = (double)(w >> 48);
-        const double s1 = u * (double)(w & CI_SUM_MASK);
-        const double r = i ? fmax((double)bb[(size_t)c * nthr + QP_CK(i - 1, nthr)], ref0) - ref0 : 0.0;
-        sx = n * r + s1;
-        sxx = n * r * r + 2.0 * r * s1;
-    };
+    // per interval: count and sum of (x - ref0), into PN / PSX (loads independent of one another), and every
+    // thread's share of SXX
+    const int count = (int)m + 1;
     {
-        double a = 0.0, b = 0.0, d = 0.0;
-        for (int i = i0; i < i1; ++i) {
-            double n, sx, sxx;
-            interval(i, n, sx, sxx);
-            a += n; b += sx; d += sxx;
+        double d = 0.0;
+        for (int i = threadIdx.x; i < count; i += CI_CURVE_THREADS) {
+            const unsigned long long w = tot[(size_t)c * stride + i];
+            const double n = (double)(w >> 48);
+            const double s1 = u * (double)(w & CI_SUM_MASK);
+            const double r = i ? fmax((double)bb[(size_t)c * nthr + QP_CK(i - 1, nthr)], ref0) - ref0 : 0.0;
+            PN[QP_CK(i, nthr + 2)] = n;
+            PSX[QP_CK(i, nthr + 2)] = n * r + s1;
+            d += n * r * r + 2.0 * r * s1;
         }
-        c_n[threadIdx.x] = a; c_sx[threadIdx.x] = b; c_sxx[threadIdx.x] = d;
+        c_sxx[threadIdx.x] = d;
+    }
+    __syncthreads();
+    // exclusive prefix sums in place: thread t takes the chunk [t * per, t * per + per)
+    const int per = (count + CI_CURVE_THREADS - 1) / CI_CURVE_THREADS;
+    const int i0 = min((int)threadIdx.x * per, count), i1 = min(i0 + per, count);
+    {
+        double a = 0.0, b = 0.0;
+        for (int i = i0; i < i1; ++i) { a += PN[i]; b += PSX[i]; }
+        c_n[threadIdx.x] = a; c_sx[threadIdx.x] = b;
     }
     __syncthreads();
     if (threadIdx.x == 0) {                              // chunk sums -> chunk offsets, in chunk order
@@ -378,19 +382,17 @@ __global__ void __launch_bounds__(CI_CURVE_THREADS) ci_curve_kernel(const unsign
             a += n; b += sx; d += c_sxx[t];
         }
         s_sxx = d + u * u * sumd2[c];
+        PN[count] = a; PSX[count] = b;                   // the totals: the end of the last code's range
     }
     __syncthreads();
     {
         double a = c_n[threadIdx.x], b = c_sx[threadIdx.x];
         for (int i = i0; i < i1; ++i) {
-            double n, sx, sxx;
-            interval(i, n, sx, sxx);
-            PN[QP_CK(i, nthr + 2)] = a; PSX[QP_CK(i, nthr + 2)] = b;
+            const double n = PN[i], sx = PSX[i];
+            PN[i] = a; PSX[i] = b;
             a += n; b += sx;
         }
-        if (i1 == count && i0 < i1) { PN[count] = a; PSX[count] = b; }
     }
-    if (count <= 0 && threadIdx.x == 0) { PN[0] = 0.0; PSX[0] = 0.0; }
     __syncthreads();
 
     const int L1 = (1 << bits) - 1;
@@ -398,21 +400,26 @@ __global__ void __launch_bounds__(CI_CURVE_THREADS) ci_curve_kernel(const unsign
         double total = 0.0;
         if (k < ncand && valid[(size_t)c * ncp + k]) {
             const float4 q = cand[(size_t)c * ncp + k];
+            const unsigned short* pk = pos + (size_t)c * nthr + k;    // T(k, j + 1) at pk[j * ncand]
             total = s_sxx;
             unsigned prev = 0u;
-            for (int j = 0; j <= L1; ++j) {
-                unsigned next = m + 1u;                  // the last code runs to the end
-                if (j < L1) {
-                    const float T = thr[(size_t)c * nthr + (size_t)k * L1 + j];      // T(k, j + 1)
-                    if (T < inf) next = pos[(size_t)c * nthr + (size_t)k * L1 + j];      // thresholds <= T
+            for (int j0 = 0; j0 <= L1; j0 += 8) {        // eight positions loaded ahead of their use
+                unsigned p8[8];
+#pragma unroll
+                for (int h = 0; h < 8; ++h) p8[h] = j0 + h < L1 ? (unsigned)pk[(size_t)(j0 + h) * ncand] : 0xFFFFu;
+#pragma unroll
+                for (int h = 0; h < 8; ++h) {
+                    const int j = j0 + h;
+                    if (j > L1) break;
+                    unsigned next = p8[h] == 0xFFFFu ? m + 1u : p8[h];   // the last code (and a code never reached) runs to the end
+                    if (next < prev) next = prev;
+                    const double n = PN[QP_CK(next, nthr + 2)] - PN[QP_CK(prev, nthr + 2)];
+                    const double sx = PSX[next] - PSX[prev];
+                    const float level = fmaf(__fsub_rn(__uint_as_float(0x4B000000u | (unsigned)j), CI_MAGIC), q.z, q.x);
+                    const double a = (double)level - ref0;
+                    total += n * a * a - 2.0 * a * sx;
+                    prev = next;
                 }
-                if (next < prev) next = prev;
-                const double n = PN[QP_CK(next, nthr + 2)] - PN[QP_CK(prev, nthr + 2)];
-                const double sx = PSX[next] - PSX[prev];
-                const float level = fmaf(__fsub_rn(__uint_as_float(0x4B000000u | (unsigned)j), CI_MAGIC), q.z, q.x);
-                const double a = (double)level - ref0;
-                total += n * a * a - 2.0 * a * sx;
-                prev = next;
             }
         }
         part[(size_t)c * ncp + k] = total;
@@ -425,7 +432,7 @@ __global__ void __launch_bounds__(CI_CURVE_THREADS) ci_curve_kernel(const unsign
 size_t qp_channel_interval_scratch_bytes(uint32_t C, int nthr)
 {
     auto al = [](size_t v) { return (v + 255) / 256 * 256; };
-    return al(sizeof(float) * (size_t)C * nthr) * 2 + al(sizeof(unsigned) * (size_t)C) + al(sizeof(double) * (size_t)C) +
+    return al(sizeof(float) * (size_t)C * nthr) + al(sizeof(unsigned) * (size_t)C) + al(sizeof(double) * (size_t)C) +
            al(sizeof(unsigned long long) * (size_t)C * (nthr + 1)) + al(sizeof(unsigned) * (size_t)C * 128) +
            al(sizeof(unsigned short) * (size_t)C * nthr);
 }
@@ -448,7 +455,6 @@ int32_t qp_launch_channel_interval_sums(qp_ctx* ctx, const void* d_x, int dtype,
     const int ncand = steps + 1, L1 = (1 << bits) - 1, nthr = ncand * L1;
     const int p2 = (nthr + 3) & ~3;                      // the three arrays of the tables kernel, a multiple of 16 bytes each
     size_t off = 0;
-    float* thr = reinterpret_cast<float*>(scratch + off);            off += al(sizeof(float) * (size_t)C * nthr);
     float* bb = reinterpret_cast<float*>(scratch + off);             off += al(sizeof(float) * (size_t)C * nthr);
     unsigned* m = reinterpret_cast<unsigned*>(scratch + off);        off += al(sizeof(unsigned) * (size_t)C);
     double* sumd2 = reinterpret_cast<double*>(scratch + off);        off += al(sizeof(double) * (size_t)C);
@@ -457,7 +463,7 @@ int32_t qp_launch_channel_interval_sums(qp_ctx* ctx, const void* d_x, int dtype,
     unsigned short* pos = reinterpret_cast<unsigned short*>(scratch + off);
 
     ci_tables_kernel<<<C, CI_TAB_THREADS, 3 * sizeof(float) * (size_t)p2, s>>>(d_stats, cand, valid, ncp, ncand, bits, nthr,
-                                                                             p2, setup, thr, bb, m, cells, pos);
+                                                                             p2, setup, bb, m, cells, pos);
     // channels per block: one block per SM where the tables of that many channels fit in shared memory
     const size_t per_channel = 16 * (size_t)(nthr + 1) + 4 * (size_t)CI_CELLS;
     const size_t fixed = sizeof(double) * CI_MOM_THREADS + 8;
@@ -480,7 +486,7 @@ int32_t qp_launch_channel_interval_sums(qp_ctx* ctx, const void* d_x, int dtype,
                                                                               cpb, nthr, bb, cells, setup, tot, sumd2);
     }
     const size_t csmem = sizeof(double) * 2 * (size_t)(nthr + 2);
-    ci_curve_kernel<<<C, CI_CURVE_THREADS, csmem, s>>>(tot, bb, thr, pos, m, setup, sumd2, cand, valid, ncp, ncand, bits, nthr, part);
+    ci_curve_kernel<<<C, CI_CURVE_THREADS, csmem, s>>>(tot, bb, pos, m, setup, sumd2, cand, valid, ncp, ncand, bits, nthr, part);
     ctx->launches += 3;
     return qp_check_launch(ctx, "qp_dsaciq_search_channels (interval path)");
 }
