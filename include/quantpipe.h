@@ -438,12 +438,16 @@ int32_t qp_sender_channels_device(qp_ctx* ctx, const void* d_x, int dtype, uint6
  * [rows, channels] tensor; the paper searches per tensor): channel c gets the histogram,
  * b_R, candidates, MSE curve and winner that qp_dsaciq_search gives for its column alone with
  * d_stats[c] (from qp_stats_channels).  Writes d_qp_out[0..channels) and, if not NULL,
- * d_out[0..channels).  Every candidate is scored on every element (the per-tensor candidate
- * path's arithmetic), so the cost is (steps + 1) * 9 fp32 instructions per element.
+ * d_out[0..channels).  Two ways, same winner: where (steps + 1) * (2^bits - 1) <= 2048 and
+ * rows <= 65535, one pass over the tensor gathers count and sum per interval between the
+ * candidates' decision thresholds of every channel and every candidate is evaluated from prefix
+ * sums (the default); otherwise, and under qp_set_search_path(QP_SEARCH_CANDIDATES), every
+ * candidate is scored on every element ((steps + 1) * 9 fp32 instructions per element).
  * bits 1..8; 1 <= steps <= QP_CH_MAX_STEPS; 1 <= hist_bins <= QP_CH_MAX_HIST_BINS; bmode as for
  * qp_dsaciq_search (QP_B_HIST_IN_STATS has no meaning here and is rejected).  Scratch
- * (histograms, candidates, block partials: about (4 hist_bins + 28 (steps + 1) + 8 (steps + 1)
- * * row blocks) bytes per channel) is allocated by the context on first use and kept.
+ * (histograms, candidates, sums; for the first way also thresholds, positions and interval sums:
+ * about 18 (steps + 1) (2^bits - 1) bytes per channel) is allocated by the context on first use
+ * (cudaMalloc: not during capture) and kept.
  * qp_dsaciq_curve_channels copies the MSE curve of one channel of the last such search to
  * host memory (steps + 1 doubles) and synchronizes the stream.
  * Errors: as qp_dsaciq_search, plus QP_ERR_INVALID_ARG for channels out of range. */
