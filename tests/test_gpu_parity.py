@@ -1249,21 +1249,49 @@ def test_search_channels_special_values_bf16_and_errors(ctx):
     ctx.qp_get_status()
 
 
-def test_search_channels_full_size_c3_sampled(ctx):
-    """The outlier-channel config at full size: sampled channels against the oracle's per-tensor search of the column."""
-    x = si.config_tensor("c3").reshape(-1, 1024)
+@pytest.mark.parametrize("name,bits", [("c3", 4), ("c4", 2)])
+def test_search_channels_full_size_sampled(ctx, name, bits):
+    """Full-size configs (c3: outlier channels; c4: the largest, 9 channels per block of the interval pass):
+    sampled channels against the oracle's search of the column, the whole curve on the library's own
+    quantizers, both forms of the search."""
+    C = si.CONFIGS[name]["shape"][-1]
+    x = si.config_tensor(name).reshape(-1, C)
     d = dev(x.reshape(-1))
-    d_stats = ctx.qp_stats_channels(d, 1024)
-    d_res, d_qp = ctx.qp_dsaciq_search_channels(d, 1024, d_stats, 4)
-    raw = d_res.cpu().numpy().tobytes()
+    d_stats = ctx.qp_stats_channels(d, C)
     rsz = ctypes.sizeof(qp.DSResult)
-    for c in (0, 17, 511, 1023):
+    sample = (0, 17, C // 2 - 1, C - 1)
+    ref = {}
+    for c in sample:
         col = np.ascontiguousarray(x[:, c])
-        _, ro, _, curve_o = oracle.ds_search(col, oracle.stats(col), 4)
-        res = qp.DSResult.from_buffer_copy(raw[c * rsz:(c + 1) * rsz])
-        assert abs(res.b_r - ro.b_r) <= 1e-9 * ro.b_r and abs(res.mse_e - ro.mse_e) <= 2e-6 * ro.mse_e
-        assert res.k_star == ro.k_star or curve_o[res.k_star] <= ro.mse_star * (1 + 1e-6)
+        st_c = oracle.stats(col)
+        ref[c] = (col, st_c) + tuple(oracle.ds_search(col, st_c, bits)[i] for i in (1, 3))
+    try:
+        for path in (qp.QP_SEARCH_AUTO, qp.QP_SEARCH_CANDIDATES):
+            ctx.qp_set_search_path(path)
+            d_res, d_qp = ctx.qp_dsaciq_search_channels(d, C, d_stats, bits)
+            raw = d_res.cpu().numpy().tobytes()
+            cand_all = ctx.qp_dsaciq_candidates_channels(C, 100)
+            for c in sample:
+                col, st_c, ro, curve_o = ref[c]
+                res = qp.DSResult.from_buffer_copy(raw[c * rsz:(c + 1) * rsz])
+                assert abs(res.b_r - ro.b_r) <= 1e-9 * ro.b_r
+                curve = np.array(ctx.qp_dsaciq_curve_channels(c, 100))
+                check_candidates_and_pick(col, st_c, ro, curve_o, res, curve, cand_all[c * 101:(c + 1) * 101], bits, 0, 100)
+    finally:
+        ctx.qp_set_search_path(qp.QP_SEARCH_AUTO)
     assert ctx.qp_get_status() & ~qp.QP_DEV_DEGENERATE == 0
+
+
+@pytest.mark.parametrize("rows", [65535, 65536])
+def test_search_channels_at_the_row_limit_of_the_interval_form(ctx, rows):
+    """65535 rows is the most the interval form's 16-bit counts hold; one more row and the call scores every
+    candidate on every element instead.  A constant-heavy channel puts nearly all rows into one interval."""
+    channels = 3
+    x = si.vit_activation((1, rows, channels), 161).reshape(rows, channels).copy()
+    x[: rows - 40, 1] = np.float32(-0.25)                       # one interval holds rows - 40 elements
+    flat = x.reshape(-1)
+    check_search_channels(ctx, flat, dev(flat), channels, 2)
+    ctx.qp_get_status()
 
 
 # ------------------------------------------------------------------ token-wise variant
