@@ -190,7 +190,9 @@ int qp_stats_carries_histogram(const void* d_x, int dtype, uint64_t n, int hist_
  *                         last tiles of its first pass in shared memory and starts the second pass,
  *                         which walks backwards, on them).  Falls back to two kernels on a device
  *                         that cannot hold it.
- *   QP_STATS_AUTO         the cooperative launch (default)
+ *   QP_STATS_AUTO         the cooperative launch for hist_bins = 0, the two kernels when the histogram
+ *                         rides along (default: the faster of the two inside the sender chain; called
+ *                         alone the cooperative launch is the faster with the histogram too)
  * A grid barrier or tile wait of the cooperative launch that runs out sets QP_DEV_STREAM_TIMEOUT
  * and the launch ends without output. */
 enum { QP_STATS_AUTO = 0, QP_STATS_TWO_KERNELS = 1, QP_STATS_FUSED = 2 };
