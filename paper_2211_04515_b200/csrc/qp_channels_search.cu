@@ -55,13 +55,22 @@ __global__ void __launch_bounds__(256) ch_hist_kernel(const T* __restrict__ x, u
             const uint64_t r0 = (uint64_t)blockIdx.x * CS_HIST_ROWS;
             const uint64_t r1 = r0 + CS_HIST_ROWS < rows ? r0 + CS_HIST_ROWS : rows;
             unsigned* mine = sh + cl * nb;
-            for (uint64_t r = r0 + rl; r < r1; r += 256 / CS_HIST_CH) {
-                const float e = cs_load(x + r * C + c);
-                if (!qp_is_finite(e)) continue;
+            constexpr uint64_t RL = 256 / CS_HIST_CH;           // row lanes of a block
+            auto count = [&](float e) {
+                if (!qp_is_finite(e)) return;
                 int b = __float2int_rz(__fmul_rn(__fsub_rn(e, fmn), inv_w));
                 b = min(max(b, 0), nb - 1);
                 atomicAdd(&mine[QP_CK(b, nb)], 1u);
+            };
+            uint64_t r = r0 + rl;
+            for (; r + 7 * RL < r1; r += 8 * RL) {              // eight loads ahead of their counting
+                float e[8];
+#pragma unroll
+                for (int q = 0; q < 8; ++q) e[q] = cs_load(x + (r + q * RL) * C + c);
+#pragma unroll
+                for (int q = 0; q < 8; ++q) count(e[q]);
             }
+            for (; r < r1; r += RL) count(cs_load(x + r * C + c));
         }
     }
     __syncthreads();
